@@ -1,0 +1,137 @@
+"""Oracle of the swap protocol (Section 3.3) and of the adaptive-expansion controller (Section 3.4.2).
+
+TEST INFRASTRUCTURE ONLY; shares no code with the CUDA library.  Both are heuristics, so the oracle
+takes the paper's steps in the paper's order, on a simulated clock.
+
+Protocol, at the instant layer k starts computing (Section 3.3):
+  1. completions are applied: a finished swap-out frees its GPU region, a finished swap-in makes its
+     layer usable and frees its CPU region;
+  2. if no swap-out is in flight, the coldest GPU layer (the one whose next use is farthest away,
+     i.e. the layer that just finished) is swapped out, unless every CPU layer is colder than it or
+     no CPU region is free;
+  3. if no swap-in is in flight, the hottest CPU layer (next use nearest) is swapped in, unless no
+     GPU region is free.
+A layer in transit holds a region on both sides (Section 3.2).  If layer k is not on the GPU when its
+turn comes the computation waits (Section 3.2) and the wait is counted as a stall.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+GPU, CPU, OUT, IN = "GPU", "CPU", "OUT", "IN"
+
+
+@dataclasses.dataclass
+class ProtocolResult:
+    events: list          # (time, "out"|"in", layer) in start order; layers are 1-based as in the paper
+    stall: float          # total time computation waited
+    trips: list           # (layer, out_start, in_finish)
+    max_off_gpu: int      # most layers simultaneously on the CPU or in transit
+    swaps_per_token: float
+    finish_time: float
+
+
+def simulate_protocol(n_layers, t_swap, gpu_regions, cpu_regions, cpu_layers, n_tokens, t_compute=1.0):
+    loc = {l: (CPU if l in cpu_layers else GPU) for l in range(1, n_layers + 1)}
+    assert sum(v == GPU for v in loc.values()) <= gpu_regions
+    assert sum(v == CPU for v in loc.values()) <= cpu_regions
+    out_busy = None  # (finish, layer)
+    in_busy = None
+    events, trips, open_trip = [], [], {}
+    stall, now, max_off, n_swaps = 0.0, 0.0, 0, 0
+
+    def dist(l, k):  # compute-steps until layer l is needed again, seen from the start of layer k
+        return (l - k) % n_layers
+
+    def complete(t):
+        nonlocal out_busy, in_busy
+        if out_busy and out_busy[0] <= t:
+            loc[out_busy[1]] = CPU
+            out_busy = None
+        if in_busy and in_busy[0] <= t:
+            loc[in_busy[1]] = GPU
+            trips.append((in_busy[1], open_trip.pop(in_busy[1], None), in_busy[0]))
+            in_busy = None
+
+    def start_swaps(t, k):
+        nonlocal out_busy, in_busy, n_swaps
+        gpu_used = sum(v in (GPU, OUT, IN) for v in loc.values())
+        cpu_used = sum(v in (CPU, OUT, IN) for v in loc.values())
+        if out_busy is None:
+            cand = [l for l in loc if loc[l] == GPU and l != k]
+            on_cpu = [l for l in loc if loc[l] == CPU]
+            if cand and on_cpu and cpu_used < cpu_regions:
+                victim = max(cand, key=lambda l: dist(l, k))
+                if any(dist(c, k) < dist(victim, k) for c in on_cpu):
+                    loc[victim] = OUT
+                    out_busy = (t + t_swap, victim)
+                    open_trip[victim] = t
+                    events.append((t, "out", victim))
+                    cpu_used += 1
+                    n_swaps += 1
+        if in_busy is None:
+            on_cpu = [l for l in loc if loc[l] == CPU]
+            if on_cpu and gpu_used < gpu_regions:
+                hot = min(on_cpu, key=lambda l: dist(l, k))
+                loc[hot] = IN
+                in_busy = (t + t_swap, hot)
+                events.append((t, "in", hot))
+
+    for _tok in range(n_tokens):
+        for k in range(1, n_layers + 1):
+            complete(now)
+            start_swaps(now, k)
+            while loc[k] != GPU:  # presence check failed: wait for the next completion
+                nxt = min(b[0] for b in (out_busy, in_busy) if b is not None)
+                stall += nxt - now
+                now = nxt
+                complete(now)
+                start_swaps(now, k)
+            max_off = max(max_off, sum(v != GPU for v in loc.values()))
+            now += t_compute
+    return ProtocolResult(events, stall, trips, max_off, n_swaps / n_tokens, now)
+
+
+# ---------------------------------------------------------------------------------------------
+# Adaptive expansion (Section 3.4.2), block-granular: r = fraction of units kept host resident.
+#   - start with everything on the GPU (r = 0);
+#   - decrease when the computation had to wait for a swap (stall above eps of compute time) in at
+#     least k_dec of the last `window` steps - a single disturbed step is tolerated;
+#   - increase by one step when there was no stall and the link was busy for less than u_hi of the
+#     compute time (the link has slack and nothing on the host was needed late);
+#   - hold otherwise.
+# The paper gives no constants; these are the build's: step = 1/n_layers ("one layer"), eps = 0.02,
+# k_dec = 2 of window = 4, u_hi = 0.9.
+# ---------------------------------------------------------------------------------------------
+
+@dataclasses.dataclass
+class Controller:
+    step: float
+    eps: float = 0.02
+    k_dec: int = 2
+    window: int = 4
+    u_hi: float = 0.9
+    r_max: float = 1.0
+    r: float = 0.0
+    history: list = dataclasses.field(default_factory=list)
+
+    def tick(self, stall, compute, swap_busy):
+        """One decode step's measurements (same time unit) -> new ratio."""
+        stalled = stall > self.eps * compute
+        self.history.append(stalled)
+        self.history = self.history[-self.window:]
+        if stalled:
+            if sum(self.history) >= self.k_dec:
+                self.r = max(0.0, self.r - self.step)
+                self.history = []
+        elif swap_busy < self.u_hi * compute and self.r < self.r_max:
+            self.r = min(self.r_max, self.r + self.step)
+        return self.r
+
+
+def fake_clock_step(r, bytes_layer, bw, t_compute_layer, n_layers):
+    """Timings of one decode step on an ideal machine: layer l+1's host-resident share streams in
+    while layer l computes; computation waits for whatever has not arrived."""
+    t_in = r * bytes_layer / bw
+    stall_per_layer = max(0.0, t_in - t_compute_layer)
+    return stall_per_layer * n_layers, t_compute_layer * n_layers, t_in * n_layers

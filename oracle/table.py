@@ -1,0 +1,264 @@
+"""Oracle of the mapping table (Section 3.2) in block-granular, stream-ordered form.
+
+TEST INFRASTRUCTURE ONLY; shares no code with the CUDA library.
+
+The paper's table maps a logical unit to its CPU pointer, its GPU pointer and a timestamp, and is
+updated in two phases: (1) the destination is allocated and recorded and the copy starts in the
+background; (2) only once the copy is confirmed complete is the unit marked present at the
+destination (Section 3.2).  Units have no fixed home: the source region is given up after the move.
+
+Here the unit is one (layer, 16-token logical block).  Its state is one of
+    FREE, GPU, TO_HOST, HOST, TO_GPU
+and copies are *stream ordered*: every swap call gets a ticket on its direction's queue ("in" or
+"out"); tickets of one queue complete in order; a call may depend on a ticket of the other queue
+(the copy that last touched one of its units, or the copy that must finish before a recycled slot
+may be overwritten) or on a compute ticket (an attention call that may still read a recycled slot).
+A source slot is released when its copy is *issued*, tagged with that copy's ticket: it may be
+handed out again at once, but whoever receives it must wait for that ticket.  So a slot is never
+overwritten before the copy reading it has finished, and a unit's bytes are never read at the
+destination before the copy writing them has finished.
+
+Slot hand-out order (shared rule, so that two implementations can be compared slot by slot):
+``ready`` is a stack that starts as n-1 .. 0 (slot 0 on top); ``pending`` is a queue of released
+slots still waiting for their ticket.  At the start of every call pending slots whose ticket is
+confirmed move to ``ready`` in queue order.  Allocation pops ``ready`` first, then takes
+``pending`` from the front and reports the tickets to wait for.
+"""
+from __future__ import annotations
+
+FREE, GPU, TO_HOST, HOST, TO_GPU = 0, 1, 2, 3, 4
+STATE_NAMES = {FREE: "FREE", GPU: "GPU", TO_HOST: "TO_HOST", HOST: "HOST", TO_GPU: "TO_GPU"}
+
+OK = 0
+ERR_INVALID = -1
+ERR_RANGE = -2
+ERR_NOMEM = -3
+ERR_BUSY = -4
+ERR_NOT_RESIDENT = -5
+
+Q_NONE, Q_IN, Q_OUT, Q_COMPUTE = 0, 1, 2, 3
+
+
+class _SlotPool:
+    def __init__(self, n):
+        self.ready = list(range(n - 1, -1, -1))
+        self.pending = []  # (slot, queue, ticket)
+
+    def settle(self, done):
+        keep = []
+        for slot, qu, tk in self.pending:
+            if tk <= done[qu]:
+                self.ready.append(slot)
+            else:
+                keep.append((slot, qu, tk))
+        self.pending = keep
+
+    def available(self):
+        return len(self.ready) + len(self.pending)
+
+    def take(self, n):
+        """-> (slots, {queue: max ticket to wait for}, per-slot (queue, ticket) tags)"""
+        slots, waits, tags = [], {}, []
+        for _ in range(n):
+            if self.ready:
+                slots.append(self.ready.pop())
+                tags.append((Q_NONE, 0))
+            else:
+                slot, qu, tk = self.pending.pop(0)
+                slots.append(slot)
+                tags.append((qu, tk))
+                waits[qu] = max(waits.get(qu, 0), tk)
+        return slots, waits, tags
+
+    def release(self, slot, queue, ticket):
+        if queue == Q_NONE:
+            self.ready.append(slot)
+        else:
+            self.pending.append((slot, queue, ticket))
+
+
+class MappingTable:
+    def __init__(self, n_layers, n_logical, n_gpu_slots, n_host_slots):
+        self.L, self.NB = n_layers, n_logical
+        self.gpu = _SlotPool(n_gpu_slots)
+        self.host = _SlotPool(n_host_slots)
+        n = n_layers * n_logical
+        self.side = [FREE] * n          # FREE / GPU / HOST : where the unit is or is heading
+        self.gpu_slot = [-1] * n
+        self.host_slot = [-1] * n
+        self.last_q = [Q_NONE] * n      # queue and ticket of the last copy issued on the unit
+        self.last_t = [0] * n
+        self.allocated = [False] * n_logical
+        self.issued = {Q_IN: 0, Q_OUT: 0, Q_COMPUTE: 0}
+        self.done = {Q_NONE: 0, Q_IN: 0, Q_OUT: 0, Q_COMPUTE: 0}
+        self.clock = 0
+        self.t_last = [0] * n           # the table's timestamp column
+        self.last_compute = [0] * n_layers  # ticket of the newest attention call on each layer
+
+    # ---- helpers -------------------------------------------------------------------
+    def _u(self, layer, block):
+        return layer * self.NB + block
+
+    def _settle(self):
+        self.gpu.settle(self.done)
+        self.host.settle(self.done)
+
+    def _in_flight(self, u):
+        return self.last_q[u] != Q_NONE and self.last_t[u] > self.done[self.last_q[u]]
+
+    def state(self, layer, block):
+        u = self._u(layer, block)
+        if self.side[u] == FREE:
+            return FREE
+        if self._in_flight(u):
+            return TO_GPU if self.side[u] == GPU else TO_HOST
+        return self.side[u]
+
+    def confirm(self, queue, ticket):
+        """Phase 2: the copies (or attention calls) of `queue` up to `ticket` are known complete."""
+        if ticket > self.issued[queue]:
+            return ERR_RANGE
+        self.done[queue] = max(self.done[queue], ticket)
+        self._settle()
+        return OK
+
+    # ---- logical block allocation ----------------------------------------------------
+    def alloc(self, block):
+        """One unit per layer: a GPU slot while any is available, else a host slot.  A recycled slot
+        whose ticket is still open makes the new unit "in flight" on that ticket, so that whatever
+        touches the unit next waits for it."""
+        if not 0 <= block < self.NB:
+            return ERR_RANGE
+        if self.allocated[block]:
+            return ERR_INVALID
+        self._settle()
+        n_gpu = min(self.L, self.gpu.available())
+        if self.L - n_gpu > self.host.available():
+            return ERR_NOMEM
+        for layer in range(self.L):
+            u = self._u(layer, block)
+            pool, side = (self.gpu, GPU) if layer < n_gpu else (self.host, HOST)
+            (slot,), _, (tag,) = pool.take(1)
+            self.side[u] = side
+            self.gpu_slot[u] = slot if side == GPU else -1
+            self.host_slot[u] = slot if side == HOST else -1
+            self.last_q[u], self.last_t[u] = tag
+        self.allocated[block] = True
+        return OK
+
+    def free(self, block):
+        """Units must be settled (no copy in flight).  GPU slots carry the last compute ticket:
+        an attention call issued earlier may still be reading them."""
+        if not 0 <= block < self.NB:
+            return ERR_RANGE
+        if not self.allocated[block]:
+            return ERR_INVALID
+        self._settle()
+        for layer in range(self.L):
+            if self._in_flight(self._u(layer, block)):
+                return ERR_BUSY
+        for layer in range(self.L):
+            u = self._u(layer, block)
+            if self.side[u] == GPU:
+                ct = self.issued[Q_COMPUTE]
+                self.gpu.release(self.gpu_slot[u], Q_COMPUTE if ct > self.done[Q_COMPUTE] else Q_NONE, ct)
+            else:
+                self.host.release(self.host_slot[u], Q_NONE, 0)
+            self.side[u], self.gpu_slot[u], self.host_slot[u] = FREE, -1, -1
+            self.last_q[u], self.last_t[u] = Q_NONE, 0
+        self.allocated[block] = False
+        return OK
+
+    # ---- swaps -----------------------------------------------------------------------
+    def _check_ids(self, layer, ids):
+        if not 0 <= layer < self.L:
+            return ERR_RANGE
+        seen = set()
+        for b in ids:
+            if not 0 <= b < self.NB:
+                return ERR_RANGE
+            if b in seen or not self.allocated[b]:
+                return ERR_INVALID
+            seen.add(b)
+        return OK
+
+    def swap(self, direction, layer, ids):
+        """direction Q_OUT: make the units host resident; Q_IN: GPU resident.
+
+        Returns (status, ticket, pairs, waits): pairs = [(block, src_slot, dst_slot)] of the units
+        that actually move (units already on, or heading to, the requested side are skipped);
+        waits = {queue: ticket} the copy must wait for besides its own queue's order.
+        A failed call changes nothing.  ticket is 0 when nothing moves.
+        """
+        st = self._check_ids(layer, ids)
+        if st != OK:
+            return st, 0, [], {}
+        self._settle()
+        want = HOST if direction == Q_OUT else GPU
+        movers = [b for b in ids if self.side[self._u(layer, b)] != want]
+        dst_pool = self.host if direction == Q_OUT else self.gpu
+        src_pool = self.gpu if direction == Q_OUT else self.host
+        if len(movers) > dst_pool.available():
+            return ERR_NOMEM, 0, [], {}
+        if not movers:
+            return OK, 0, [], {}
+        slots, waits, _ = dst_pool.take(len(movers))
+        self.issued[direction] += 1
+        ticket = self.issued[direction]
+        self.clock += 1
+        pairs = []
+        for b, dst in zip(movers, slots):
+            u = self._u(layer, b)
+            if self._in_flight(u):  # the copy that is still bringing the unit to where it is now
+                waits[self.last_q[u]] = max(waits.get(self.last_q[u], 0), self.last_t[u])
+            if direction == Q_OUT:
+                src = self.gpu_slot[u]
+                self.host_slot[u], self.gpu_slot[u] = dst, -1
+            else:
+                src = self.host_slot[u]
+                self.gpu_slot[u], self.host_slot[u] = dst, -1
+            src_pool.release(src, direction, ticket)
+            self.side[u] = want
+            self.last_q[u], self.last_t[u] = direction, ticket
+            self.t_last[u] = self.clock
+            pairs.append((b, src, dst))
+        if direction == Q_OUT and self.last_compute[layer] > self.done[Q_COMPUTE]:
+            # the layer's attention call also appends the new token: copy out only after it
+            waits[Q_COMPUTE] = max(waits.get(Q_COMPUTE, 0), self.last_compute[layer])
+        waits.pop(direction, None)  # same queue: ordered anyway
+        return OK, ticket, pairs, waits
+
+    # ---- presence check (Section 3.2: computation may start only on units present on the GPU) ----
+    def attention(self, layer, ids):
+        """-> (status, compute ticket, waits).  Every unit must be on the GPU or arriving; the call
+        then waits for the newest arriving copy among them."""
+        st = self._check_ids(layer, ids)
+        if st != OK:
+            return st, 0, {}
+        self._settle()
+        waits = {}
+        for b in ids:
+            u = self._u(layer, b)
+            if self.side[u] != GPU:
+                return ERR_NOT_RESIDENT, 0, {}
+            if self._in_flight(u):
+                waits[self.last_q[u]] = max(waits.get(self.last_q[u], 0), self.last_t[u])
+        self.issued[Q_COMPUTE] += 1
+        self.last_compute[layer] = self.issued[Q_COMPUTE]
+        return OK, self.issued[Q_COMPUTE], waits
+
+    # ---- invariants ------------------------------------------------------------------
+    def check_invariants(self):
+        for pool, slots, n in ((self.gpu, self.gpu_slot, "gpu"), (self.host, self.host_slot, "host")):
+            held = [s for s in slots if s >= 0]
+            free = list(pool.ready) + [p[0] for p in pool.pending]
+            assert len(set(held)) == len(held), f"{n}: a slot is mapped twice"
+            assert not (set(held) & set(free)), f"{n}: a mapped slot is on the free list"
+            assert len(set(free)) == len(free), f"{n}: a slot is free twice"
+        for u, side in enumerate(self.side):
+            if side == GPU:
+                assert self.gpu_slot[u] >= 0 and self.host_slot[u] < 0
+            elif side == HOST:
+                assert self.host_slot[u] >= 0 and self.gpu_slot[u] < 0
+            else:
+                assert self.gpu_slot[u] < 0 and self.host_slot[u] < 0

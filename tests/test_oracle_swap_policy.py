@@ -1,0 +1,307 @@
+"""Pins of the oracle's swap semantics, mapping-table state machine, swap protocol and controller."""
+import itertools
+import os
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import policy, table
+from paper_2411_09317_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------------------- swap = block memcpy
+def test_swap_raw_definition_and_untouched_bytes():
+    BB = 256
+    G = synth.random_bytes(1, 8 * BB).copy()
+    H = synth.random_bytes(2, 6 * BB).copy()
+    G0, H0 = G.copy(), H.copy()
+    assert oracle.swap_raw(H, G, BB, [7, 0, 3], [5, 1, 2]) == 0
+    assert np.array_equal(G, G0)                                  # the source is left as it was
+    for s, d in [(7, 5), (0, 1), (3, 2)]:
+        assert np.array_equal(H[d * BB:(d + 1) * BB], G0[s * BB:(s + 1) * BB])
+    for d in (0, 3, 4):
+        assert np.array_equal(H[d * BB:(d + 1) * BB], H0[d * BB:(d + 1) * BB])
+    # round trip into other slots returns the bytes
+    assert oracle.swap_raw(G, H, BB, [5, 1, 2], [4, 6, 2]) == 0
+    for s, d in [(7, 4), (0, 6), (3, 2)]:
+        assert np.array_equal(G[d * BB:(d + 1) * BB], G0[s * BB:(s + 1) * BB])
+
+
+def test_swap_raw_rejects_bad_lists_without_copying():
+    BB = 64
+    G = synth.random_bytes(3, 4 * BB).copy()
+    H = synth.random_bytes(4, 4 * BB).copy()
+    H0 = H.copy()
+    assert oracle.swap_raw(H, G, BB, [0, 1], [2, 2]) == -1       # duplicate destination
+    assert oracle.swap_raw(H, G, BB, [0, 4], [1, 2]) == -1       # source out of range
+    assert oracle.swap_raw(H, G, BB, [0, 1], [-1, 2]) == -1
+    assert np.array_equal(H, H0)
+    assert oracle.swap_raw(H, G, BB, [], []) == 0
+
+
+# --------------------------------------------------------- mapping table: device-order executor
+class Executor:
+    """Runs the copies a MappingTable issued in a random order that respects tickets and waits, with a
+    content tag per slot, and checks that every read finds the unit it expects."""
+
+    def __init__(self, tbl, rng):
+        self.t, self.rng = tbl, rng
+        self.g = {}   # gpu slot -> tag
+        self.h = {}
+        self.ops = {table.Q_IN: [], table.Q_OUT: [], table.Q_COMPUTE: []}
+        self.ran = {table.Q_IN: 0, table.Q_OUT: 0, table.Q_COMPUTE: 0}
+
+    def write_unit(self, layer, block):  # host-side initial fill at alloc time (synchronous)
+        u = self.t._u(layer, block)
+        if self.t.side[u] == table.GPU:
+            self.g[self.t.gpu_slot[u]] = (layer, block)
+        else:
+            self.h[self.t.host_slot[u]] = (layer, block)
+
+    def issue(self, queue, ticket, waits, body):
+        assert ticket == len(self.ops[queue]) + 1
+        self.ops[queue].append((dict(waits), body))
+
+    def runnable(self, queue):
+        i = self.ran[queue]
+        if i >= len(self.ops[queue]):
+            return False
+        return all(self.ran[q] >= t for q, t in self.ops[queue][i][0].items())
+
+    def step(self):
+        qs = [q for q in self.ops if self.runnable(q)]
+        if not qs:
+            return False
+        q = self.rng.choice(qs)
+        self.ops[q][self.ran[q]][1]()
+        self.ran[q] += 1
+        return True
+
+    def drain(self):
+        while self.step():
+            pass
+        assert all(self.ran[q] == len(self.ops[q]) for q in self.ops), "dependency cycle"
+
+
+def apply_op(tbl, ex, op):
+    kind = op[0]
+    if kind == "alloc":
+        st = tbl.alloc(op[1])
+        if st == table.OK:
+            # the harness writes a fresh unit only after the slot's open ticket: model by draining
+            ex.drain()
+            for l in range(tbl.L):
+                ex.write_unit(l, op[1])
+        return st
+    if kind == "free":
+        return tbl.free(op[1])
+    if kind in ("out", "in"):
+        q = table.Q_OUT if kind == "out" else table.Q_IN
+        st, ticket, pairs, waits = tbl.swap(q, op[1], list(op[2]))
+        if st == table.OK and ticket:
+            layer = op[1]
+
+            def body(pairs=pairs, layer=layer, q=q):
+                src, dst = (ex.g, ex.h) if q == table.Q_OUT else (ex.h, ex.g)
+                for b, s, d in pairs:
+                    assert src.get(s) == (layer, b), f"copy read slot {s}: {src.get(s)} != {(layer, b)}"
+                    dst[d] = src[s]
+            ex.issue(q, ticket, waits, body)
+        return st
+    if kind == "attn":
+        st, ticket, waits = tbl.attention(op[1], list(op[2]))
+        if st == table.OK:
+            layer, ids = op[1], list(op[2])
+            slots = [tbl.gpu_slot[tbl._u(layer, b)] for b in ids]
+
+            def body():
+                for b, s in zip(ids, slots):
+                    assert ex.g.get(s) == (layer, b), f"attention read slot {s}: {ex.g.get(s)}"
+            ex.issue(table.Q_COMPUTE, ticket, waits, body)
+        return st
+    if kind == "confirm":  # the host learns how far the device got
+        ex.drain() if op[1] else None
+        for q in ex.ran:
+            tbl.confirm(q, ex.ran[q])
+        return table.OK
+    if kind == "run":       # let the device make some progress
+        for _ in range(op[1]):
+            ex.step()
+        return table.OK
+    raise ValueError(kind)
+
+
+def final_check(tbl, ex):
+    ex.drain()
+    for l in range(tbl.L):
+        for b in range(tbl.NB):
+            u = tbl._u(l, b)
+            if tbl.side[u] == table.GPU:
+                assert ex.g.get(tbl.gpu_slot[u]) == (l, b)
+            elif tbl.side[u] == table.HOST:
+                assert ex.h.get(tbl.host_slot[u]) == (l, b)
+    tbl.check_invariants()
+
+
+def test_table_exhaustive_tiny():
+    """Every call sequence of length <= 5 over a small alphabet on a 2-layer, 2-block table with 3 + 3
+    slots: invariants hold, failed calls change nothing, and data survives in device order."""
+    alphabet = [("alloc", 0), ("alloc", 1), ("free", 0), ("out", 0, (0,)), ("out", 1, (0, 1)), ("in", 0, (0,)),
+                ("in", 1, (1, 0)), ("attn", 0, (0,)), ("attn", 1, (0, 1)), ("confirm", True), ("run", 1)]
+    n_seq = 0
+    for length in range(1, 6):
+        for seq in itertools.product(alphabet, repeat=length):
+            if seq[0][0] not in ("alloc",):
+                continue  # everything else fails on an empty table; covered by the length-1 cases below
+            tbl = table.MappingTable(2, 2, 3, 3)
+            ex = Executor(tbl, random.Random(n_seq))
+            for op in seq:
+                snap = (list(tbl.side), list(tbl.gpu_slot), list(tbl.host_slot), list(tbl.gpu.ready), list(tbl.host.ready))
+                st = apply_op(tbl, ex, op)
+                if st != table.OK:
+                    assert snap == (list(tbl.side), list(tbl.gpu_slot), list(tbl.host_slot), list(tbl.gpu.ready),
+                                    list(tbl.host.ready)), f"failed call {op} changed the table"
+                tbl.check_invariants()
+            final_check(tbl, ex)
+            n_seq += 1
+    assert n_seq > 10000
+
+
+def test_table_error_codes_and_two_phase_states():
+    t = table.MappingTable(2, 3, 4, 4)
+    assert t.swap(table.Q_OUT, 0, [0])[0] == table.ERR_INVALID      # not allocated
+    assert t.alloc(0) == table.OK and t.alloc(0) == table.ERR_INVALID
+    assert t.alloc(7) == table.ERR_RANGE
+    assert t.swap(table.Q_OUT, 5, [0])[0] == table.ERR_RANGE
+    assert t.swap(table.Q_OUT, 0, [0, 0])[0] == table.ERR_INVALID   # duplicate id
+    assert t.state(0, 0) == table.GPU
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [0])
+    assert (st, tk) == (table.OK, 1) and pairs == [(0, 0, 0)]
+    assert t.state(0, 0) == table.TO_HOST                            # phase 1: in transit
+    assert t.attention(0, [0])[0] == table.ERR_NOT_RESIDENT          # presence check fails
+    assert t.free(0) == table.ERR_BUSY
+    assert t.swap(table.Q_OUT, 0, [0]) == (table.OK, 0, [], {})      # already heading there: no-op
+    t.confirm(table.Q_OUT, 1)
+    assert t.state(0, 0) == table.HOST                               # phase 2
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [0])
+    assert st == table.OK and t.state(0, 0) == table.TO_GPU
+    st, ctk, waits = t.attention(0, [0])                             # arriving: allowed, waits for it
+    assert st == table.OK and waits == {table.Q_IN: 1}
+    # an out-copy issued before the in-copy is confirmed must wait for it and for the attention call
+    st, tk2, pairs, waits = t.swap(table.Q_OUT, 0, [0])
+    assert st == table.OK and waits == {table.Q_IN: 1, table.Q_COMPUTE: 1}
+
+
+def test_table_nomem_and_slot_recycling_waits():
+    t = table.MappingTable(1, 4, 2, 2)
+    assert [t.alloc(b) for b in range(4)] == [table.OK] * 4           # 2 on the GPU, 2 on the host
+    assert [t.state(0, b) for b in range(4)] == [table.GPU, table.GPU, table.HOST, table.HOST]
+    assert t.swap(table.Q_IN, 0, [2])[0] == table.ERR_NOMEM           # no GPU slot
+    assert t.swap(table.Q_OUT, 0, [0])[0] == table.ERR_NOMEM          # no host slot
+    t.free(3)
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [0])                 # into the freed host slot
+    assert st == table.OK and waits == {}
+    # block 2 may now come in, into block 0's old GPU slot - but only after the out-copy has read it
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [2])
+    assert st == table.OK and pairs[0][2] == 0 and waits == {table.Q_OUT: 1}
+
+
+def test_table_random_long_runs():
+    rng = random.Random(5)
+    for trial in range(60):
+        L, NB = rng.choice([(1, 6), (3, 4), (2, 8)])
+        tbl = table.MappingTable(L, NB, rng.randint(NB, L * NB), rng.randint(NB, L * NB))
+        ex = Executor(tbl, rng)
+        for _ in range(120):
+            k = rng.random()
+            ids = tuple(rng.sample(range(NB), rng.randint(1, NB)))
+            layer = rng.randrange(L)
+            op = (("alloc", rng.randrange(NB)) if k < 0.15 else ("free", rng.randrange(NB)) if k < 0.2 else
+                  ("out", layer, ids) if k < 0.45 else ("in", layer, ids) if k < 0.7 else
+                  ("attn", layer, ids) if k < 0.85 else ("confirm", rng.random() < 0.3) if k < 0.93 else ("run", 2))
+            apply_op(tbl, ex, op)
+            tbl.check_invariants()
+        final_check(tbl, ex)
+
+
+# ------------------------------------------------------------------------- protocol golden trace
+def read_golden():
+    rows, totals = [], {}
+    for line in open(os.path.join(GOLD, "fifo_9layer.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        f = line.split()
+        if f[0] in ("P", "D"):
+            rows.append((f[0], int(f[1]), int(f[2]), int(f[3]), int(f[4])))
+        else:
+            totals[f[0]] = int(f[1])
+    return rows, totals
+
+
+def test_protocol_reproduces_the_nine_layer_example():
+    rows, totals = read_golden()
+    res = policy.simulate_protocol(9, 2.0, 7, 4, {8, 9}, n_tokens=6)
+    started = {}
+    for t, kind, layer in res.events:
+        started.setdefault(int(t), {})[kind] = layer
+    for tag, t, layer_starting, out, inn in rows:
+        assert (t % 9) + 1 == layer_starting
+        assert started.get(t, {}).get("out", 0) == out, (tag, t)
+        assert started.get(t, {}).get("in", 0) == inn, (tag, t)
+    assert res.stall == totals["stall"]
+    assert res.max_off_gpu == totals["fifo_length"]
+    steady = [tr for tr in res.trips if tr[1] is not None and tr[1] >= 3]
+    assert steady and all(fin - start == totals["trip_time"] for _, start, fin in steady)
+    # Section 3.1: t_swap * m <= t_compute * n with t_swap = 2, n = 9 allows m <= 4.5 swaps per token
+    late = [e for e in res.events if e[1] == "out" and 18 <= e[0] < 54]
+    assert len(late) / 4 == pytest.approx(4.5)
+
+
+def test_protocol_sensitivity():
+    # one GPU region fewer, or slower swaps: the computation has to wait (Section 3.4.1)
+    assert policy.simulate_protocol(9, 2.0, 6, 4, {7, 8, 9}, 6).stall > 0
+    assert policy.simulate_protocol(9, 3.0, 7, 4, {8, 9}, 6).stall > 0
+    # a smaller expansion under "swap whenever the link is free" moves as much data for shorter stays
+    small = policy.simulate_protocol(9, 2.0, 8, 3, {9}, 8)
+    best = policy.simulate_protocol(9, 2.0, 7, 4, {8, 9}, 8)
+    assert small.stall == 0
+    trip = lambda r: max(fin - st for _, st, fin in r.trips if st is not None and st > 9)
+    assert trip(small) < trip(best)
+    assert small.swaps_per_token == pytest.approx(best.swaps_per_token, abs=0.6)
+    # everything on the GPU: nothing ever moves
+    none = policy.simulate_protocol(9, 2.0, 9, 2, set(), 3)
+    assert none.events == [] and none.stall == 0
+
+
+# ------------------------------------------------------------------------------------ controller
+@pytest.mark.parametrize("bw,tc,bytes_layer,L", [(50e9, 200e-6, 400e6, 32), (400e9, 300e-6, 400e6, 32),
+                                                  (50e9, 2e-3, 100e6, 10), (1e12, 1e-3, 100e6, 8)])
+def test_controller_settles_at_the_transparent_ratio(bw, tc, bytes_layer, L):
+    r_star = min(1.0, bw * tc / bytes_layer)      # t_swap * m = t_compute * n, per layer (Section 3.1)
+    c = policy.Controller(step=1.0 / L)
+    trace = []
+    for _ in range(200):
+        trace.append(c.tick(*policy.fake_clock_step(c.r, bytes_layer, bw, tc, L)))
+    tail = trace[-40:]
+    tol = c.step + 0.1 * r_star + 1e-9
+    assert all(abs(r - r_star) <= tol for r in tail), (r_star, tail[-5:])
+    # bandwidth halves (prolonged interference, Section 3.4.2): it follows
+    for _ in range(200):
+        trace.append(c.tick(*policy.fake_clock_step(c.r, bytes_layer, bw / 2, tc, L)))
+    r2 = min(1.0, bw / 2 * tc / bytes_layer)
+    assert all(abs(r - r2) <= c.step + 0.1 * r2 + 1e-9 for r in trace[-40:])
+
+
+def test_controller_tolerates_one_disturbed_step():
+    c = policy.Controller(step=0.1)
+    for _ in range(3):
+        c.tick(0.0, 1.0, 0.5)
+    r = c.r
+    assert c.tick(0.5, 1.0, 0.5) == r           # a single stall: no change
+    assert c.tick(0.0, 1.0, 0.95) == r          # quiet again, link nearly full: hold
+    assert c.tick(0.5, 1.0, 0.5) == pytest.approx(r - 0.1)  # second stall within the window: back off
