@@ -1,0 +1,245 @@
+/*
+ * pie.h - C ABI of the B200-native KV-block swapping + paged decode-attention library.
+ *
+ * The library implements the hot path of performance-transparent swapping (Pie, arXiv 2411.09317,
+ * Section 3): paged KV-cache blocks live in an HBM block pool or in a pinned host pool; a mapping table
+ * (Section 3.2) says where each (layer, logical block) unit is; background copies move units between
+ * the pools while the paged decode attention of the current layer runs, and an adaptive controller
+ * (Section 3.4.2) sizes the host-resident share so that copies stay hidden behind compute.
+ *
+ * Conventions
+ *   - every call returns a pie_status (0 = PIE_OK, negative = error); nothing aborts, traps or throws.
+ *   - argument errors are found before anything is enqueued: a failed call enqueues nothing and leaves
+ *     the mapping table as it was.  Asynchronous CUDA errors surface at a later call as PIE_ERR_CUDA.
+ *   - "host" pointers are read during the call and may be freed at return.  "device" pointers must stay
+ *     valid until the pool's compute stream has passed the call.
+ *   - one host thread per pool.  The library never calls the batched-memcpy runtime entry points.
+ *   - slot layout: one slot holds one layer's K and V of one 16-token block as 16-bit elements
+ *     [n_kv_heads][2 (K, V)][16 tokens][head_dim]; slot s starts at byte s * block_bytes of its pool.
+ *     The paper states no layout; this one makes a head's K+V tile of a block one contiguous piece.
+ */
+#ifndef PIE_H
+#define PIE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pie_status {
+    PIE_OK = 0,
+    PIE_ERR_INVALID = -1,      /* null pointer, bad shape or dtype, duplicate id, unallocated block */
+    PIE_ERR_RANGE = -2,        /* layer, block or slot id out of range */
+    PIE_ERR_NOMEM = -3,        /* no free slot on the destination side / allocation failed */
+    PIE_ERR_BUSY = -4,         /* a copy on the unit is still in flight (block free / read / write) */
+    PIE_ERR_NOT_RESIDENT = -5, /* attention needs a unit that is neither on the GPU nor arriving */
+    PIE_ERR_TIMEOUT = -6,      /* a bounded wait ran out */
+    PIE_ERR_CUDA = -7,         /* a CUDA call failed: see pie_last_cuda_error */
+    PIE_ERR_UNSUPPORTED = -8   /* head_dim / group size / block size outside the built set */
+} pie_status;
+
+enum { PIE_F16 = 0, PIE_BF16 = 1 };
+enum { PIE_MODE_AUTO = 0, PIE_MODE_KERNEL = 1, PIE_MODE_COPY_ENGINE = 2 };
+enum { PIE_H2D = 0, PIE_D2H = 1 };
+/* unit states of the two-phase mapping table (Section 3.2) */
+enum { PIE_FREE = 0, PIE_GPU = 1, PIE_TO_HOST = 2, PIE_HOST = 3, PIE_TO_GPU = 4 };
+/* copy queues: tickets of one queue complete in order */
+enum { PIE_Q_NONE = 0, PIE_Q_IN = 1, PIE_Q_OUT = 2, PIE_Q_COMPUTE = 3 };
+
+typedef struct pie_pool pie_pool;
+typedef struct pie_table pie_table;
+typedef struct pie_fifo pie_fifo;
+
+typedef struct pie_pool_config {
+    int32_t n_layers;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;        /* divides n_q_heads; n_q_heads / n_kv_heads <= 8 */
+    int32_t head_dim;          /* 64 or 128 */
+    int32_t block_tokens;      /* 16 */
+    int32_t dtype;             /* PIE_F16 or PIE_BF16 */
+    int32_t n_logical_blocks;  /* logical block ids 0 .. n-1, shared by all layers */
+    int32_t max_seqs;          /* largest batch pie_decode_attention will see (scratch sizing) */
+    int64_t n_gpu_slots;
+    int64_t n_host_slots;
+    void *gpu_base;            /* device memory of n_gpu_slots * block_bytes, 128-byte aligned, or NULL:
+                                  the library allocates and owns it */
+    void *host_base;           /* pinned host memory of n_host_slots * block_bytes, or NULL: the library
+                                  allocates (cudaHostAlloc) and owns it */
+    void *compute_stream;      /* cudaStream_t values; used only when own_streams == 0 */
+    void *copy_in_stream;
+    void *copy_out_stream;
+    int32_t own_streams;       /* 1: the library creates three non-blocking streams */
+    int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (256) */
+    int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
+    int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
+    int32_t timing;            /* 1: record per-layer events for pie_controller_tick / pie_get_stats */
+    int32_t reserved[7];
+} pie_pool_config;
+
+typedef struct pie_stats {
+    double bytes_in, bytes_out;            /* swapped so far, per direction */
+    double calls_kernel, calls_copy_engine;
+    double last_step_compute_ms;           /* sum over layers: attention (+append, combine) time */
+    double last_step_stall_ms;             /* sum over layers: compute stream waiting for swap-in */
+    double last_step_swap_in_ms, last_step_swap_out_ms;
+    double last_step_ms;                   /* first layer's start to last layer's end */
+    double ratio;                          /* current extension ratio */
+    int64_t n_units_gpu, n_units_host, n_units_in_flight;
+    int64_t steps_measured;
+    double reserved[8];
+} pie_stats;
+
+/* ---- pool (Section 3.1: the physical pools; Section 3.2: the mapping table) --------------------- */
+
+/* Create a pool.  Validates the configuration (PIE_ERR_INVALID / PIE_ERR_UNSUPPORTED), allocates what
+ * the caller did not supply (PIE_ERR_NOMEM), builds the free lists, the per-layer device slot tables
+ * and the TMA descriptor of the HBM pool.  Needs a CUDA device: without one it fails with
+ * PIE_ERR_CUDA - there is no CPU path.  *out is written only on success. */
+int pie_pool_create(const pie_pool_config *cfg, pie_pool **out);
+/* Drain the streams (bounded: 10 s, then PIE_ERR_TIMEOUT is returned but the pool is still freed) and
+ * free what the library owns.  NULL is accepted. */
+int pie_pool_destroy(pie_pool *pool);
+size_t pie_block_bytes(const pie_pool *pool);
+
+/* Allocate n logical blocks (one unit per layer each).  on_host (host, n bytes, may be NULL): non-zero
+ * puts every unit of that block in the host pool; zero / NULL puts units on the GPU while slots are
+ * available, else on the host (Section 4.1: the block manager hands out blocks).  ids_out (host, n)
+ * receives the ids.  All or nothing: PIE_ERR_NOMEM allocates none. */
+int pie_block_alloc(pie_pool *pool, int64_t n, const uint8_t *on_host, int32_t *ids_out);
+/* Give n blocks back.  PIE_ERR_BUSY if a copy on any unit is still in flight (call pie_sync first). */
+int pie_block_free(pie_pool *pool, const int32_t *ids, int64_t n);
+/* Synchronous access to one unit wherever it lives (test set-up, read-back).  host_buf holds
+ * block_bytes.  These wait for the unit's copies and use plain cudaMemcpy, not the swap path. */
+int pie_block_write(pie_pool *pool, int32_t layer, int32_t block, const void *host_buf);
+int pie_block_read(pie_pool *pool, int32_t layer, int32_t block, void *host_buf);
+/* Table look-up: state (PIE_GPU ...), slots (-1 if none).  Any out pointer may be NULL. */
+int pie_block_state(pie_pool *pool, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot,
+                    int32_t *host_slot);
+/* Bulk look-up: side[L*NB] (PIE_FREE / PIE_GPU / PIE_HOST: where the unit is or is heading) and
+ * slot[L*NB]; host arrays. */
+int pie_get_placement(pie_pool *pool, int32_t *side, int32_t *slot);
+
+/* ---- swapping (Section 3.2 two-phase update; Section 3.3 protocol; Section 4 swap kernel) -------- */
+
+/* Make these logical blocks of `layer` host resident.  Phase 1 (during the call): host slots are
+ * chosen and recorded, the copy is enqueued on the copy-out stream behind the layer's last attention
+ * call, and the GPU slots are released tagged with this copy's ticket.  Phase 2: once the copy is
+ * known complete (observed with cudaEventQuery at any later call) the units read PIE_HOST.
+ * Blocks already on, or heading to, the host are skipped.  block_ids: host, n entries, distinct.
+ * mode: PIE_MODE_KERNEL = gather/scatter kernel, PIE_MODE_COPY_ENGINE = one cudaMemcpyAsync per run of
+ * consecutive slots, PIE_MODE_AUTO = chosen from the run lengths. */
+int pie_swap_out(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode);
+/* The mirror image on the copy-in stream.  The layer's next pie_decode_attention waits for it
+ * (Section 3.2: presence check). */
+int pie_swap_in(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode);
+/* The mechanism under both: copy n whole slots between the pools by PHYSICAL slot id, no table change.
+ * dir PIE_H2D: src = host slots, dst = GPU slots; PIE_D2H the reverse.  dst ids must be distinct.
+ * stream: a cudaStream_t, or NULL for the direction's copy stream.  For the swap microbenchmark and for
+ * byte-exact checks. */
+int pie_swap_raw(pie_pool *pool, int32_t dir, const int32_t *src_slots, const int32_t *dst_slots, int64_t n,
+                 int32_t mode, void *stream);
+
+/* ---- paged decode attention (Section 2.1 decode stage; Section 2.3 paged KV; Section 3.2) --------- */
+
+/* One layer's decode attention for n_seqs sequences, enqueued on the compute stream:
+ *   wait for the layer's arriving units -> [append k_new/v_new at position ctx_len-1] -> split-K paged
+ *   attention -> combine -> out.
+ * q, out: device [n_seqs][n_q_heads][head_dim] in the pool dtype.  k_new, v_new: device
+ * [n_seqs][n_kv_heads][head_dim] or NULL (no append).  block_table_dev: device int32
+ * [n_seqs][max_blocks_per_seq] of LOGICAL block ids - the kernel resolves them through the layer's slot
+ * table, so callers pass the same table whether or not blocks were swapped (Section 4.1: base pointer
+ * from the mapping table, offsets unchanged).  ctx_lens_dev: device int32 [n_seqs], context length
+ * INCLUDING the appended token; 0 gives a zero output row.
+ * block_table_host / ctx_lens_host (host, optional): when given, residency of every referenced unit is
+ * checked before anything is enqueued (PIE_ERR_NOT_RESIDENT) and lengths beyond the table are rejected
+ * (PIE_ERR_INVALID).  Without them a missing unit makes the kernel skip the tile, set a device status
+ * word, and the NEXT call returns PIE_ERR_NOT_RESIDENT.
+ * scale multiplies q.k (pass 1/sqrt(head_dim)). */
+int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
+                         int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, const int32_t *block_table_host,
+                         const int32_t *ctx_lens_host, int32_t n_seqs, float scale, const void *k_new,
+                         const void *v_new);
+
+/* One decode step: for every layer l, prefetch layer l+1's host-resident units (wrapping to layer 0 of
+ * the next token, Section 3.4.2), run layer l's attention, push layer l's share back out (Section 3.3:
+ * the layer that just finished is the coldest).  q_all/out_all: device [n_layers][n_seqs][Hq][D];
+ * k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D] or NULL.  Runs pie_controller_tick at the end
+ * when the ratio is adaptive.  Never blocks the host on the GPU. */
+int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev,
+                    int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale,
+                    const void *k_new_all, const void *v_new_all, int32_t mode);
+/* The same with q / k_new / v_new / out in HOST memory (pinned for full speed): copies the inputs in,
+ * runs the step, copies out_all back and waits for it.  ctx_lens_host/block_table_host are uploaded too. */
+int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_host, const int32_t *block_table_host,
+                         int32_t max_blocks_per_seq, const int32_t *ctx_lens_host, int32_t n_seqs, float scale,
+                         const void *k_new_all_host, const void *v_new_all_host, int32_t mode);
+/* Marks a step boundary for the per-step timing sets (pie_decode_step calls it itself). */
+int pie_step_begin(pie_pool *pool);
+
+/* ---- policy and controller (Section 3.3, Section 3.4.2) ------------------------------------------ */
+
+/* r in [0,1]: target fraction of each layer's allocated units kept host resident between uses
+ * (expansion X = 1/(1-r), Section 3.1).  r < 0: adaptive - the controller owns the ratio, starting from
+ * the current one.  Until the first call the host-resident sets are whatever the caller established. */
+int pie_set_extension_ratio(pie_pool *pool, float r);
+int pie_get_extension_ratio(pie_pool *pool, float *r);
+/* The per-layer plan at the start of layer `layer`: in_ids = units of layer (layer+1) mod L to bring in
+ * (ascending id, as many as the GPU pool can take), out_ids = units of `layer` to push out once it has
+ * computed.  Arrays are host, capacity n_logical_blocks each. */
+int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in, int32_t *out_ids, int64_t *n_out);
+/* Read the previous step's events (no blocking: returns PIE_OK with *changed = 0 if they have not all
+ * completed), update the stats, and in adaptive mode adjust the ratio. */
+int pie_controller_tick(pie_pool *pool, int32_t *changed);
+int pie_get_stats(pie_pool *pool, pie_stats *out);
+/* Wait until everything enqueued so far has completed, at most timeout_us (PIE_ERR_TIMEOUT); applies
+ * phase-2 updates and reports a pending device status word (PIE_ERR_NOT_RESIDENT ...). */
+int pie_sync(pie_pool *pool, int64_t timeout_us);
+const char *pie_status_str(int status);
+int pie_last_cuda_error(void);
+/* Host-link probe: time a pinned cudaMemcpyAsync of `bytes` in direction dir (or both at once when
+ * dir == 2) `reps` times; *gbps = best bytes/time per direction. */
+int pie_probe_link(int64_t bytes, int32_t dir, int32_t reps, double *gbps);
+/* HBM probe: device-to-device copy kernel-free cudaMemcpyAsync of `bytes`; *gbps counts read+write. */
+int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps);
+
+/* ---- host-only pieces, usable without a GPU ------------------------------------------------------ */
+
+/* The mapping table by itself (what pie_pool uses inside).  Stream-ordered two-phase semantics:
+ * pie_table_swap picks destination slots, releases the source slots tagged with the new ticket, and
+ * reports the tickets of other queues the copy must wait for; pie_table_confirm is phase 2. */
+pie_table *pie_table_create(int32_t n_layers, int32_t n_logical, int64_t n_gpu_slots, int64_t n_host_slots);
+void pie_table_destroy(pie_table *t);
+int pie_table_alloc(pie_table *t, int32_t block, int32_t on_host);
+int pie_table_free(pie_table *t, int32_t block);
+/* queue = PIE_Q_IN / PIE_Q_OUT.  Outputs (host): ticket; moved_ids/src_slots/dst_slots with capacity n;
+ * n_moved; waits[4] indexed by queue (0 = none). */
+int pie_table_swap(pie_table *t, int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket,
+                   int32_t *moved_ids, int32_t *src_slots, int32_t *dst_slots, int64_t *n_moved, int64_t *waits);
+/* Presence check + compute ticket.  ids may be NULL (n = 0): then no residency check is made and the
+ * waits cover every arriving unit of the layer. */
+int pie_table_attention(pie_table *t, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits);
+int pie_table_confirm(pie_table *t, int32_t queue, int64_t ticket);
+int pie_table_state(pie_table *t, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot);
+
+/* The whole-layer swap protocol of Section 3.3 as a scheduler object.  on_cpu: n_layers flags. */
+pie_fifo *pie_fifo_create(int32_t n_layers, int32_t gpu_regions, int32_t cpu_regions, const uint8_t *on_cpu);
+void pie_fifo_destroy(pie_fifo *f);
+/* A swap in direction dir (PIE_Q_IN / PIE_Q_OUT) has been confirmed complete. */
+int pie_fifo_complete(pie_fifo *f, int32_t dir);
+/* Layer k (0-based) starts computing: *start_out / *start_in receive the layer to swap out / in now, or
+ * -1.  The caller starts those copies and later reports them with pie_fifo_complete. */
+int pie_fifo_layer_start(pie_fifo *f, int32_t k, int32_t *start_out, int32_t *start_in);
+/* 0 GPU, 1 CPU, 2 in transit to the CPU, 3 in transit to the GPU */
+int pie_fifo_location(pie_fifo *f, int32_t layer);
+
+/* The controller's decision rule by itself.  state: 8 doubles owned by the caller, zero-initialised
+ * (history).  Returns the new ratio for one decode step's measurements (same unit for all three). */
+double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
+                             double swap_busy);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIE_H */

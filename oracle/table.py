@@ -123,8 +123,8 @@ class MappingTable:
         return OK
 
     # ---- logical block allocation ----------------------------------------------------
-    def alloc(self, block):
-        """One unit per layer: a GPU slot while any is available, else a host slot.  A recycled slot
+    def alloc(self, block, on_host=False):
+        """One unit per layer: a GPU slot while any is available (never, if on_host), else a host slot.  A recycled slot
         whose ticket is still open makes the new unit "in flight" on that ticket, so that whatever
         touches the unit next waits for it."""
         if not 0 <= block < self.NB:
@@ -132,7 +132,7 @@ class MappingTable:
         if self.allocated[block]:
             return ERR_INVALID
         self._settle()
-        n_gpu = min(self.L, self.gpu.available())
+        n_gpu = 0 if on_host else min(self.L, self.gpu.available())
         if self.L - n_gpu > self.host.available():
             return ERR_NOMEM
         for layer in range(self.L):

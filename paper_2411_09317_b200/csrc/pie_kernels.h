@@ -1,0 +1,71 @@
+// Launch interface between the pool (host control) and the sm_100a kernels.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace pie {
+
+// device status word bits (written by kernels into mapped pinned memory, read by the host later)
+enum : int32_t {
+    STATUS_MISSING_UNIT = 1,   // a block id or slot was out of range / not on the GPU
+    STATUS_CTX_TOO_LONG = 2,   // ctx_len exceeded 16 * max_blocks_per_seq (clamped)
+    STATUS_WAIT_TIMEOUT = 4    // a bounded mbarrier wait ran out
+};
+
+// ---- swap ----------------------------------------------------------------------------------------
+// list: device int32 triples {src_slot, dst_slot, logical_block} x n.  slot_table may be NULL;
+// table_mode 1: slot_table[block] = dst_slot (swap-in), 2: slot_table[block] = -1 (swap-out).
+cudaError_t launch_swap(const void *src_pool, void *dst_pool, const int32_t *list, int64_t n, int64_t block_bytes,
+                        int32_t *slot_table, int table_mode, int n_ctas, cudaStream_t stream);
+// table update only (copy-engine path, alloc/free): entries = device int32 pairs {index, value} x n.
+cudaError_t launch_patch(int32_t *table, const int32_t *entries, int64_t n, cudaStream_t stream);
+// same, from triples {src, dst, block} as launch_swap
+cudaError_t launch_patch_from_list(int32_t *slot_table, const int32_t *list, int64_t n, int table_mode,
+                                   cudaStream_t stream);
+
+// ---- attention -----------------------------------------------------------------------------------
+struct AttnShape {
+    int head_dim;      // 64 or 128
+    int dtype;         // PIE_F16 / PIE_BF16
+    int n_q_heads, n_kv_heads;
+    int n_logical;
+    int64_t n_gpu_slots;
+};
+
+struct AttnScratch {
+    int32_t *chunk_off;  // [max_seqs + 1]
+    float *part_o;       // [max_items][G][D]
+    float *part_ml;      // [max_items][G][2]
+    int64_t max_items;   // capacity in items (chunk, kv head)
+    int32_t max_seqs;
+};
+
+struct AttnLaunch {
+    const void *q;
+    void *out;
+    const int32_t *block_table;
+    int32_t max_blocks;
+    const int32_t *ctx_lens;
+    const int32_t *slot_table;  // this layer's row of the device slot table
+    int32_t n_seqs;
+    float scale;
+    const void *k_new, *v_new;  // optional
+    void *gpu_pool;
+    int32_t split_tokens;
+    int32_t grid;               // persistent CTAs
+    int32_t *status;            // device-visible status word
+};
+
+// Build the TMA descriptors of the HBM pool: map3d covers a whole K+V tile in one copy
+// (dims {64, rows, D/64}); map2d is the fallback with one copy per 128-byte half.  Returns which
+// is usable in *use3d.
+cudaError_t make_pool_tensor_maps(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, int head_dim, CUtensorMap *map3d,
+                                  CUtensorMap *map2d, int *use3d);
+int attn_smem_bytes(int head_dim);
+cudaError_t attn_configure(int head_dim, int dtype, int *ctas_per_sm);
+cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
+                             int use3d, cudaStream_t stream);
+
+}  // namespace pie

@@ -1,0 +1,1106 @@
+// pie_pool: the HBM + pinned-host block pools, streams and events around the mapping table, the swap
+// and attention entry points, the per-layer decode loop, the controller tick and the C ABI.
+#include <algorithm>
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <vector>
+
+#include "pie_kernels.h"
+#include "pie_table.h"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+constexpr int EV_RING = 512;       // events per queue: ticket t uses slot t % EV_RING
+constexpr int LIST_EVENTS = 512;   // events guarding regions of the id-list ring
+constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB
+
+#define PIE_CUDA(call)                                  \
+    do {                                                \
+        cudaError_t e__ = (call);                       \
+        if (e__ != cudaSuccess) {                       \
+            g_last_cuda_error = (int)e__;               \
+            return PIE_ERR_CUDA;                        \
+        }                                               \
+    } while (0)
+
+struct LayerEvents {
+    cudaEvent_t pre = nullptr, go = nullptr, done = nullptr;  // compute stream: before wait, after wait, after layer
+    cudaEvent_t in0 = nullptr, in1 = nullptr, out0 = nullptr, out1 = nullptr;
+    bool has_in = false, has_out = false, has_compute = false;
+};
+
+struct ListRecord {
+    int64_t start, end;
+    int ev;  // index into list_events
+};
+
+}  // namespace
+
+struct pie_pool {
+    pie_pool_config cfg{};
+    int64_t block_bytes = 0;
+    pie::Table *table = nullptr;
+    uint8_t *gpu_base = nullptr, *host_base = nullptr;
+    bool own_gpu = false, own_host = false, own_streams = false;
+    cudaStream_t stream[4] = {nullptr, nullptr, nullptr, nullptr};  // indexed by queue id
+    cudaEvent_t ticket_ev[4][EV_RING] = {};
+    int64_t recorded[4] = {0, 0, 0, 0};  // newest ticket of each queue whose event has been recorded
+    int32_t *slot_table_dev = nullptr;  // [L][NB]
+    // id lists: pinned ring + device mirror at the same offsets
+    int32_t *list_host = nullptr, *list_dev = nullptr;
+    int64_t list_words = 0, list_head = 0;
+    std::deque<ListRecord> list_live;
+    cudaEvent_t list_events[LIST_EVENTS] = {};
+    int list_ev_next = 0;
+    // device status word (mapped pinned memory)
+    int32_t *status_host = nullptr, *status_dev = nullptr;
+    // attention
+    pie::AttnScratch scratch{};
+    CUtensorMap map3d{}, map2d{};
+    int use3d = 0, attn_grid = 0, n_sms = 0;
+    // decode-step staging (device copies of host inputs)
+    void *stage_q = nullptr, *stage_out = nullptr, *stage_k = nullptr, *stage_v = nullptr;
+    int32_t *stage_bt = nullptr, *stage_ctx = nullptr;
+    int64_t stage_q_bytes = 0, stage_kv_bytes = 0, stage_bt_words = 0;
+    // policy / controller
+    int ratio_mode = 0;  // 0 unset (keep the caller's sets), 1 fixed, 2 adaptive
+    double ratio = 0.0;
+    double ctrl_state[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    std::vector<int64_t> home_count;  // per layer: units whose home is the host
+    // timing
+    std::vector<LayerEvents> lev[2];
+    int64_t step = 0;
+    bool prev_step_valid = false, prev_step_ticked = true;
+    pie_stats stats{};
+    // scratch vectors
+    std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
+    int sticky = PIE_OK;
+};
+
+namespace {
+
+int poll(pie_pool *p) {
+    for (int q = 1; q <= 3; ++q) {
+        int64_t d = p->table->done(q);
+        const int64_t issued = p->recorded[q];  // a ticket whose event is not recorded yet cannot be queried
+        while (d < issued) {
+            cudaError_t e = cudaEventQuery(p->ticket_ev[q][(d + 1) % EV_RING]);
+            if (e == cudaSuccess) ++d;
+            else if (e == cudaErrorNotReady) break;
+            else {
+                g_last_cuda_error = (int)e;
+                p->sticky = PIE_ERR_CUDA;
+                return PIE_ERR_CUDA;
+            }
+        }
+        if (d > p->table->done(q)) p->table->confirm(q, d);
+    }
+    return PIE_OK;
+}
+
+// make `stream` wait for ticket t of queue q (no-op if already known complete)
+int wait_ticket(pie_pool *p, cudaStream_t stream, int q, int64_t t) {
+    if (t <= 0 || t <= p->table->done(q)) return PIE_OK;
+    PIE_CUDA(cudaStreamWaitEvent(stream, p->ticket_ev[q][t % EV_RING], 0));
+    return PIE_OK;
+}
+
+// before ticket t of queue q records its event: the slot's previous user (t - EV_RING) must be done
+int reserve_ticket_event(pie_pool *p, int q, int64_t t) {
+    const int64_t prev = t - EV_RING;
+    if (prev > 0 && prev > p->table->done(q)) {
+        PIE_CUDA(cudaEventSynchronize(p->ticket_ev[q][prev % EV_RING]));
+        poll(p);
+    }
+    return PIE_OK;
+}
+
+int record_ticket(pie_pool *p, int q, int64_t t) {
+    PIE_CUDA(cudaEventRecord(p->ticket_ev[q][t % EV_RING], p->stream[q]));
+    p->recorded[q] = t;
+    return PIE_OK;
+}
+
+// reserve `words` int32 in the list ring; waits (bounded by the GPU finishing earlier work) if the ring is full
+int list_alloc(pie_pool *p, int64_t words, int64_t *offset) {
+    words = (words + 3) & ~int64_t(3);  // 16-byte granules
+    if (words > p->list_words) return PIE_ERR_INVALID;
+    if (p->list_head + words > p->list_words) p->list_head = 0;
+    const int64_t a = p->list_head, b = a + words;
+    while (!p->list_live.empty() && cudaEventQuery(p->list_events[p->list_live.front().ev]) == cudaSuccess)
+        p->list_live.pop_front();
+    for (;;) {
+        bool clash = false;
+        for (size_t i = 0; i < p->list_live.size(); ++i) {
+            const ListRecord &r = p->list_live[i];
+            if (r.start < b && a < r.end) {
+                PIE_CUDA(cudaEventSynchronize(p->list_events[r.ev]));
+                p->list_live.erase(p->list_live.begin() + (long)i);
+                clash = true;
+                break;
+            }
+        }
+        if (!clash) break;
+    }
+    if ((int)p->list_live.size() >= LIST_EVENTS - 1) {
+        PIE_CUDA(cudaEventSynchronize(p->list_events[p->list_live.front().ev]));
+        p->list_live.pop_front();
+    }
+    *offset = a;
+    p->list_head = b;
+    return PIE_OK;
+}
+
+// the list at `offset` is consumed by work already enqueued on `stream`: guard it with an event
+int list_commit(pie_pool *p, int64_t offset, int64_t words, cudaStream_t stream) {
+    words = (words + 3) & ~int64_t(3);
+    const int ev = p->list_ev_next;
+    p->list_ev_next = (p->list_ev_next + 1) % LIST_EVENTS;
+    PIE_CUDA(cudaEventRecord(p->list_events[ev], stream));
+    p->list_live.push_back({offset, offset + words, ev});
+    return PIE_OK;
+}
+
+int check_status_word(pie_pool *p) {
+    volatile int32_t *w = p->status_host;  // [0] missing unit, [1] context too long, [2] wait timed out
+    if (w[0] == 0 && w[1] == 0 && w[2] == 0) return PIE_OK;
+    const int st = w[2] ? PIE_ERR_TIMEOUT : w[0] ? PIE_ERR_NOT_RESIDENT : PIE_ERR_INVALID;
+    w[0] = w[1] = w[2] = 0;
+    return st;
+}
+
+LayerEvents *timing_slot(pie_pool *p, int32_t layer) {
+    if (!p->cfg.timing) return nullptr;
+    return &p->lev[p->step & 1][(size_t)layer];
+}
+
+// ---- one swap call ------------------------------------------------------------------------------------
+int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst, int64_t n, const int32_t *blocks,
+              int32_t *slot_table_row, int mode, cudaStream_t stream) {
+    // dir_queue PIE_Q_IN: host -> GPU; PIE_Q_OUT: GPU -> host
+    const uint8_t *src_pool = dir_queue == PIE_Q_IN ? p->host_base : p->gpu_base;
+    uint8_t *dst_pool = dir_queue == PIE_Q_IN ? p->gpu_base : p->host_base;
+    const int64_t BB = p->block_bytes;
+    if (mode == PIE_MODE_AUTO) {
+        int64_t runs = 1;
+        for (int64_t i = 1; i < n; ++i)
+            if (src[i] != src[i - 1] + 1 || dst[i] != dst[i - 1] + 1) ++runs;
+        mode = (n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES ? PIE_MODE_COPY_ENGINE : PIE_MODE_KERNEL;
+    }
+    const bool need_list = mode == PIE_MODE_KERNEL || slot_table_row != nullptr;
+    int64_t off = 0;
+    if (need_list) {
+        int st = list_alloc(p, 3 * n, &off);
+        if (st != PIE_OK) return st;
+        int32_t *h = p->list_host + off;
+        for (int64_t i = 0; i < n; ++i) {
+            h[3 * i + 0] = src[i];
+            h[3 * i + 1] = dst[i];
+            h[3 * i + 2] = blocks ? blocks[i] : 0;
+        }
+        PIE_CUDA(cudaMemcpyAsync(p->list_dev + off, h, (size_t)(3 * n) * 4, cudaMemcpyHostToDevice, stream));
+    }
+    const int table_mode = slot_table_row ? (dir_queue == PIE_Q_IN ? 1 : 2) : 0;
+    if (mode == PIE_MODE_KERNEL) {
+        const int ctas = p->cfg.swap_ctas > 0 ? p->cfg.swap_ctas : 16;
+        PIE_CUDA(pie::launch_swap(src_pool, dst_pool, p->list_dev + off, n, BB, slot_table_row, table_mode, ctas, stream));
+        p->stats.calls_kernel += 1;
+    } else {
+        // copy engine: one cudaMemcpyAsync per run of consecutive (src, dst) slots
+        const cudaMemcpyKind kind = dir_queue == PIE_Q_IN ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+        int64_t i = 0;
+        while (i < n) {
+            int64_t j = i + 1;
+            while (j < n && src[j] == src[j - 1] + 1 && dst[j] == dst[j - 1] + 1) ++j;
+            PIE_CUDA(cudaMemcpyAsync(dst_pool + (int64_t)dst[i] * BB, src_pool + (int64_t)src[i] * BB, (size_t)((j - i) * BB),
+                                     kind, stream));
+            i = j;
+        }
+        if (slot_table_row) PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_dev + off, n, table_mode, stream));
+        p->stats.calls_copy_engine += 1;
+    }
+    if (need_list) {
+        int st = list_commit(p, off, 3 * n, stream);
+        if (st != PIE_OK) return st;
+    }
+    return PIE_OK;
+}
+
+int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t n, int32_t mode) {
+    if (!p) return PIE_ERR_INVALID;
+    if (p->sticky != PIE_OK) return p->sticky;
+    if (mode < PIE_MODE_AUTO || mode > PIE_MODE_COPY_ENGINE) return PIE_ERR_INVALID;
+    if (n < 0 || (n > 0 && !ids)) return PIE_ERR_INVALID;
+    int st = poll(p);
+    if (st != PIE_OK) return st;
+    if (n == 0) return (layer < 0 || layer >= p->cfg.n_layers) ? PIE_ERR_RANGE : PIE_OK;
+    if ((int64_t)p->v_moved.size() < n) {
+        p->v_moved.resize((size_t)n);
+        p->v_src.resize((size_t)n);
+        p->v_dst.resize((size_t)n);
+    }
+    int64_t ticket = 0, n_moved = 0, waits[4];
+    st = p->table->swap(queue, layer, ids, n, &ticket, p->v_moved.data(), p->v_src.data(), p->v_dst.data(), &n_moved, waits);
+    if (st != PIE_OK || n_moved == 0) return st;
+    // a unit that is pushed out belongs to the host-resident set from now on; bringing it in for a layer's
+    // turn does not take it out of the set (only a lower ratio does)
+    if (queue == PIE_Q_OUT)
+        for (int64_t i = 0; i < n_moved; ++i) {
+            pie::Unit &u = p->table->unit(layer, p->v_moved[(size_t)i]);
+            if (!u.home_host) {
+                u.home_host = 1;
+                p->home_count[(size_t)layer] += 1;
+            }
+        }
+    cudaStream_t stream = p->stream[queue];
+    st = reserve_ticket_event(p, queue, ticket);
+    if (st != PIE_OK) return st;
+    for (int q = 1; q <= 3; ++q) {
+        st = wait_ticket(p, stream, q, waits[q]);
+        if (st != PIE_OK) { p->sticky = st; return st; }
+    }
+    LayerEvents *le = timing_slot(p, layer);
+    if (le) PIE_CUDA(cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream));
+    st = do_copies(p, queue, p->v_src.data(), p->v_dst.data(), n_moved, p->v_moved.data(),
+                   p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream);
+    if (st != PIE_OK) { p->sticky = st; return st; }
+    if (le) {
+        PIE_CUDA(cudaEventRecord(queue == PIE_Q_IN ? le->in1 : le->out1, stream));
+        (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
+    }
+    st = record_ticket(p, queue, ticket);
+    if (st != PIE_OK) { p->sticky = st; return st; }
+    (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)n_moved * (double)p->block_bytes;
+    return PIE_OK;
+}
+
+int sync_all(pie_pool *p, int64_t timeout_us) {
+    const auto t0 = std::chrono::steady_clock::now();
+    for (int q = 1; q <= 3; ++q) {
+        for (;;) {
+            cudaError_t e = cudaStreamQuery(p->stream[q]);
+            if (e == cudaSuccess) break;
+            if (e != cudaErrorNotReady) {
+                g_last_cuda_error = (int)e;
+                p->sticky = PIE_ERR_CUDA;
+                return PIE_ERR_CUDA;
+            }
+            const auto us = std::chrono::duration_cast<std::chrono::microseconds>(std::chrono::steady_clock::now() - t0).count();
+            if (timeout_us >= 0 && us > timeout_us) return PIE_ERR_TIMEOUT;
+        }
+    }
+    return poll(p);
+}
+
+int patch_units(pie_pool *p, const std::vector<int32_t> &entries) {
+    const int64_t n = (int64_t)entries.size() / 2;
+    if (n == 0) return PIE_OK;
+    // large updates go in pieces that fit the ring
+    const int64_t piece = std::max<int64_t>(1, p->list_words / 8);
+    for (int64_t done = 0; done < n; done += piece) {
+        const int64_t m = std::min(piece, n - done);
+        int64_t off;
+        int st = list_alloc(p, 2 * m, &off);
+        if (st != PIE_OK) return st;
+        std::memcpy(p->list_host + off, entries.data() + 2 * done, (size_t)(2 * m) * 4);
+        cudaStream_t s = p->stream[PIE_Q_COMPUTE];
+        PIE_CUDA(cudaMemcpyAsync(p->list_dev + off, p->list_host + off, (size_t)(2 * m) * 4, cudaMemcpyHostToDevice, s));
+        PIE_CUDA(pie::launch_patch(p->slot_table_dev, p->list_dev + off, m, s));
+        st = list_commit(p, off, 2 * m, s);
+        if (st != PIE_OK) return st;
+    }
+    return PIE_OK;
+}
+
+void destroy_pool(pie_pool *p) {
+    if (!p) return;
+    for (int q = 1; q <= 3; ++q)
+        for (int i = 0; i < EV_RING; ++i)
+            if (p->ticket_ev[q][i]) cudaEventDestroy(p->ticket_ev[q][i]);
+    for (int i = 0; i < LIST_EVENTS; ++i)
+        if (p->list_events[i]) cudaEventDestroy(p->list_events[i]);
+    for (int k = 0; k < 2; ++k)
+        for (LayerEvents &e : p->lev[k])
+            for (cudaEvent_t ev : {e.pre, e.go, e.done, e.in0, e.in1, e.out0, e.out1})
+                if (ev) cudaEventDestroy(ev);
+    if (p->own_streams)
+        for (int q = 1; q <= 3; ++q)
+            if (p->stream[q]) cudaStreamDestroy(p->stream[q]);
+    if (p->own_gpu && p->gpu_base) cudaFree(p->gpu_base);
+    if (p->own_host && p->host_base) cudaFreeHost(p->host_base);
+    cudaFree(p->slot_table_dev);
+    cudaFree(p->list_dev);
+    if (p->list_host) cudaFreeHost(p->list_host);
+    if (p->status_host) cudaFreeHost(p->status_host);
+    cudaFree(p->scratch.chunk_off);
+    cudaFree(p->scratch.part_o);
+    cudaFree(p->scratch.part_ml);
+    cudaFree(p->stage_q);
+    cudaFree(p->stage_out);
+    cudaFree(p->stage_k);
+    cudaFree(p->stage_v);
+    cudaFree(p->stage_bt);
+    cudaFree(p->stage_ctx);
+    delete p->table;
+    delete p;
+}
+
+int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const int32_t *bt_dev, int32_t max_blocks,
+                   const int32_t *ctx_dev, const int32_t *bt_host, const int32_t *ctx_host, int32_t n_seqs, float scale,
+                   const void *k_new, const void *v_new) {
+    if (!p) return PIE_ERR_INVALID;
+    if (p->sticky != PIE_OK) return p->sticky;
+    if (layer < 0 || layer >= p->cfg.n_layers) return PIE_ERR_RANGE;
+    if (!q || !out || !bt_dev || !ctx_dev || n_seqs < 0 || max_blocks <= 0) return PIE_ERR_INVALID;
+    if (n_seqs > p->scratch.max_seqs) return PIE_ERR_INVALID;
+    if ((k_new == nullptr) != (v_new == nullptr)) return PIE_ERR_INVALID;
+    if ((bt_host == nullptr) != (ctx_host == nullptr)) return PIE_ERR_INVALID;
+    int st = poll(p);
+    if (st != PIE_OK) return st;
+    st = check_status_word(p);  // a flag raised by an earlier call's kernels
+    if (st != PIE_OK) return st;
+    if (n_seqs == 0) return PIE_OK;
+    const int64_t split = p->cfg.split_tokens;
+    // host-side checks when the caller supplied host copies of the tables
+    int64_t ticket = 0, waits[4];
+    if (bt_host) {
+        p->v_in.clear();
+        int64_t chunks = 0;
+        for (int32_t s = 0; s < n_seqs; ++s) {
+            const int32_t ctx = ctx_host[s];
+            if (ctx < 0 || ctx > max_blocks * 16) return PIE_ERR_INVALID;
+            chunks += (ctx + split - 1) / split;
+            for (int32_t b = 0; b < (ctx + 15) / 16; ++b) p->v_in.push_back(bt_host[(int64_t)s * max_blocks + b]);
+        }
+        if (chunks * p->cfg.n_kv_heads > p->scratch.max_items) return PIE_ERR_INVALID;
+        st = p->table->attention(layer, p->v_in.data(), (int64_t)p->v_in.size(), &ticket, waits);
+    } else {
+        st = p->table->attention(layer, nullptr, 0, &ticket, waits);
+    }
+    if (st != PIE_OK) return st;
+    cudaStream_t stream = p->stream[PIE_Q_COMPUTE];
+    st = reserve_ticket_event(p, PIE_Q_COMPUTE, ticket);
+    if (st != PIE_OK) return st;
+    LayerEvents *le = timing_slot(p, layer);
+    if (le) PIE_CUDA(cudaEventRecord(le->pre, stream));
+    for (int qd = 1; qd <= 2; ++qd) {
+        st = wait_ticket(p, stream, qd, waits[qd]);
+        if (st != PIE_OK) { p->sticky = st; return st; }
+    }
+    if (le) PIE_CUDA(cudaEventRecord(le->go, stream));
+    pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
+                      p->cfg.n_gpu_slots};
+    pie::AttnLaunch a{};
+    a.q = q;
+    a.out = out;
+    a.block_table = bt_dev;
+    a.max_blocks = max_blocks;
+    a.ctx_lens = ctx_dev;
+    a.slot_table = p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks;
+    a.n_seqs = n_seqs;
+    a.scale = scale;
+    a.k_new = k_new;
+    a.v_new = v_new;
+    a.gpu_pool = p->gpu_base;
+    a.split_tokens = (int32_t)split;
+    a.grid = p->attn_grid;
+    a.status = p->status_dev;
+    cudaError_t e = pie::launch_attention(sh, p->scratch, a, p->use3d ? p->map3d : p->map2d, p->use3d, stream);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        p->sticky = PIE_ERR_CUDA;
+        return PIE_ERR_CUDA;
+    }
+    if (le) {
+        PIE_CUDA(cudaEventRecord(le->done, stream));
+        le->has_compute = true;
+    }
+    st = record_ticket(p, PIE_Q_COMPUTE, ticket);
+    if (st != PIE_OK) p->sticky = st;
+    return st;
+}
+
+// the host-resident set of `layer` follows the ratio: mark / unmark units in id order
+void apply_ratio_to_layer(pie_pool *p, int32_t layer) {
+    if (p->ratio_mode == 0) return;
+    const int32_t NB = p->cfg.n_logical_blocks;
+    const int64_t target = (int64_t)std::llround(p->ratio * (double)p->table->n_allocated());
+    int64_t &count = p->home_count[(size_t)layer];
+    if (count < target) {
+        for (int32_t b = 0; b < NB && count < target; ++b) {
+            if (!p->table->allocated(b)) continue;
+            pie::Unit &u = p->table->unit(layer, b);
+            if (!u.home_host) { u.home_host = 1; ++count; }
+        }
+    } else if (count > target) {
+        for (int32_t b = NB - 1; b >= 0 && count > target; --b) {
+            if (!p->table->allocated(b)) continue;
+            pie::Unit &u = p->table->unit(layer, b);
+            if (u.home_host) { u.home_host = 0; --count; }
+        }
+    }
+}
+
+int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::vector<int32_t> &out_ids) {
+    const int32_t L = p->cfg.n_layers, NB = p->cfg.n_logical_blocks;
+    const int32_t next = (layer + 1) % L;
+    in_ids.clear();
+    out_ids.clear();
+    apply_ratio_to_layer(p, layer);
+    apply_ratio_to_layer(p, next);
+    // hottest first: the next layer's host-resident units, as many as the GPU pool can take
+    int64_t room = p->table->gpu_available();
+    for (int32_t b = 0; b < NB && room > 0; ++b) {
+        if (!p->table->allocated(b)) continue;
+        if (p->table->unit(next, b).side == PIE_HOST) {
+            in_ids.push_back(b);
+            --room;
+        }
+    }
+    // coldest: this layer's host-home units go back once it has computed
+    for (int32_t b = 0; b < NB; ++b) {
+        if (!p->table->allocated(b)) continue;
+        const pie::Unit &u = p->table->unit(layer, b);
+        if (u.home_host && u.side == PIE_GPU) out_ids.push_back(b);
+    }
+    return PIE_OK;
+}
+
+int ensure_stage(pie_pool *p, int32_t n_seqs, int32_t max_blocks) {
+    const int64_t E = 2;
+    const int64_t qb = (int64_t)p->cfg.n_layers * n_seqs * p->cfg.n_q_heads * p->cfg.head_dim * E;
+    const int64_t kb = (int64_t)p->cfg.n_layers * n_seqs * p->cfg.n_kv_heads * p->cfg.head_dim * E;
+    if (qb > p->stage_q_bytes) {
+        cudaFree(p->stage_q);
+        cudaFree(p->stage_out);
+        p->stage_q = p->stage_out = nullptr;
+        p->stage_q_bytes = 0;
+        PIE_CUDA(cudaMalloc(&p->stage_q, (size_t)qb));
+        PIE_CUDA(cudaMalloc(&p->stage_out, (size_t)qb));
+        p->stage_q_bytes = qb;
+    }
+    if (kb > p->stage_kv_bytes) {
+        cudaFree(p->stage_k);
+        cudaFree(p->stage_v);
+        p->stage_k = p->stage_v = nullptr;
+        p->stage_kv_bytes = 0;
+        PIE_CUDA(cudaMalloc(&p->stage_k, (size_t)kb));
+        PIE_CUDA(cudaMalloc(&p->stage_v, (size_t)kb));
+        p->stage_kv_bytes = kb;
+    }
+    const int64_t bw = (int64_t)n_seqs * max_blocks;
+    if (bw > p->stage_bt_words) {
+        cudaFree(p->stage_bt);
+        p->stage_bt = nullptr;
+        p->stage_bt_words = 0;
+        PIE_CUDA(cudaMalloc(&p->stage_bt, (size_t)bw * 4));
+        p->stage_bt_words = bw;
+    }
+    if (!p->stage_ctx) PIE_CUDA(cudaMalloc(&p->stage_ctx, (size_t)p->scratch.max_seqs * 4));
+    return PIE_OK;
+}
+
+}  // namespace
+
+// =========================================================================================================
+// C ABI
+// =========================================================================================================
+extern "C" {
+
+const char *pie_status_str(int status) {
+    switch (status) {
+        case PIE_OK: return "ok";
+        case PIE_ERR_INVALID: return "invalid argument";
+        case PIE_ERR_RANGE: return "id out of range";
+        case PIE_ERR_NOMEM: return "no free slot / out of memory";
+        case PIE_ERR_BUSY: return "unit busy (copy in flight)";
+        case PIE_ERR_NOT_RESIDENT: return "unit not resident on the GPU";
+        case PIE_ERR_TIMEOUT: return "timeout";
+        case PIE_ERR_CUDA: return "CUDA error";
+        case PIE_ERR_UNSUPPORTED: return "unsupported configuration";
+        default: return "unknown status";
+    }
+}
+
+int pie_last_cuda_error(void) { return g_last_cuda_error; }
+
+size_t pie_block_bytes(const pie_pool *pool) { return pool ? (size_t)pool->block_bytes : 0; }
+
+int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
+    if (!cfg || !out) return PIE_ERR_INVALID;
+    if (cfg->n_layers <= 0 || cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->n_logical_blocks <= 0 ||
+        cfg->n_gpu_slots <= 0 || cfg->n_host_slots < 0 || cfg->max_seqs <= 0)
+        return PIE_ERR_INVALID;
+    if (cfg->n_q_heads % cfg->n_kv_heads != 0) return PIE_ERR_INVALID;
+    if (cfg->dtype != PIE_F16 && cfg->dtype != PIE_BF16) return PIE_ERR_INVALID;
+    if (cfg->block_tokens != 16 || (cfg->head_dim != 64 && cfg->head_dim != 128)) return PIE_ERR_UNSUPPORTED;
+    if (cfg->n_q_heads / cfg->n_kv_heads > 8) return PIE_ERR_UNSUPPORTED;
+    if (cfg->split_tokens < 0 || cfg->split_tokens % 16 != 0) return PIE_ERR_INVALID;
+    if (cfg->gpu_base && ((uintptr_t)cfg->gpu_base & 127)) return PIE_ERR_INVALID;
+    if ((uint64_t)cfg->n_gpu_slots * (uint64_t)cfg->n_kv_heads * 32u > 0x7fffffffull) return PIE_ERR_UNSUPPORTED;
+
+    int n_dev = 0;
+    PIE_CUDA(cudaGetDeviceCount(&n_dev));
+    if (n_dev <= 0) {
+        g_last_cuda_error = (int)cudaErrorNoDevice;
+        return PIE_ERR_CUDA;
+    }
+    int dev = 0;
+    PIE_CUDA(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    PIE_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major < 10) return PIE_ERR_UNSUPPORTED;  // built for sm_100a only
+
+    pie_pool *p = new (std::nothrow) pie_pool();
+    if (!p) return PIE_ERR_NOMEM;
+    p->cfg = *cfg;
+    if (p->cfg.split_tokens == 0) p->cfg.split_tokens = 256;
+    p->block_bytes = (int64_t)2 * 16 * cfg->n_kv_heads * cfg->head_dim * 2;
+    p->n_sms = prop.multiProcessorCount;
+    p->table = new (std::nothrow) pie::Table(cfg->n_layers, cfg->n_logical_blocks, cfg->n_gpu_slots, cfg->n_host_slots);
+    if (!p->table) { destroy_pool(p); return PIE_ERR_NOMEM; }
+    p->home_count.assign((size_t)cfg->n_layers, 0);
+
+#define PIE_TRY(call, code)                            \
+    do {                                               \
+        cudaError_t e__ = (call);                      \
+        if (e__ != cudaSuccess) {                      \
+            g_last_cuda_error = (int)e__;              \
+            destroy_pool(p);                           \
+            return (code);                             \
+        }                                              \
+    } while (0)
+
+    if (cfg->gpu_base) p->gpu_base = (uint8_t *)cfg->gpu_base;
+    else {
+        PIE_TRY(cudaMalloc((void **)&p->gpu_base, (size_t)(cfg->n_gpu_slots * p->block_bytes)), PIE_ERR_NOMEM);
+        p->own_gpu = true;
+    }
+    if (cfg->host_base) p->host_base = (uint8_t *)cfg->host_base;
+    else if (cfg->n_host_slots > 0) {
+        PIE_TRY(cudaHostAlloc((void **)&p->host_base, (size_t)(cfg->n_host_slots * p->block_bytes), cudaHostAllocDefault),
+                PIE_ERR_NOMEM);
+        p->own_host = true;
+    }
+    if (cfg->own_streams) {
+        int lo = 0, hi = 0;
+        PIE_TRY(cudaDeviceGetStreamPriorityRange(&lo, &hi), PIE_ERR_CUDA);
+        PIE_TRY(cudaStreamCreateWithPriority(&p->stream[PIE_Q_COMPUTE], cudaStreamNonBlocking, lo), PIE_ERR_CUDA);
+        PIE_TRY(cudaStreamCreateWithPriority(&p->stream[PIE_Q_IN], cudaStreamNonBlocking, hi), PIE_ERR_CUDA);
+        PIE_TRY(cudaStreamCreateWithPriority(&p->stream[PIE_Q_OUT], cudaStreamNonBlocking, hi), PIE_ERR_CUDA);
+        p->own_streams = true;
+    } else {
+        p->stream[PIE_Q_COMPUTE] = (cudaStream_t)cfg->compute_stream;
+        p->stream[PIE_Q_IN] = (cudaStream_t)cfg->copy_in_stream;
+        p->stream[PIE_Q_OUT] = (cudaStream_t)cfg->copy_out_stream;
+    }
+    for (int q = 1; q <= 3; ++q)
+        for (int i = 0; i < EV_RING; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->ticket_ev[q][i], cudaEventDisableTiming), PIE_ERR_CUDA);
+    for (int i = 0; i < LIST_EVENTS; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->list_events[i], cudaEventDisableTiming), PIE_ERR_CUDA);
+    if (cfg->timing) {
+        for (int k = 0; k < 2; ++k) {
+            p->lev[k].resize((size_t)cfg->n_layers);
+            for (LayerEvents &e : p->lev[k])
+                for (cudaEvent_t *ev : {&e.pre, &e.go, &e.done, &e.in0, &e.in1, &e.out0, &e.out1})
+                    PIE_TRY(cudaEventCreate(ev), PIE_ERR_CUDA);
+        }
+    }
+    const size_t table_bytes = (size_t)cfg->n_layers * (size_t)cfg->n_logical_blocks * 4;
+    PIE_TRY(cudaMalloc((void **)&p->slot_table_dev, table_bytes), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMemset(p->slot_table_dev, 0xff, table_bytes), PIE_ERR_CUDA);
+    p->list_words = std::max<int64_t>(1 << 20, (int64_t)cfg->n_logical_blocks * 3 * 8);
+    PIE_TRY(cudaHostAlloc((void **)&p->list_host, (size_t)p->list_words * 4, cudaHostAllocDefault), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMalloc((void **)&p->list_dev, (size_t)p->list_words * 4), PIE_ERR_NOMEM);
+    PIE_TRY(cudaHostAlloc((void **)&p->status_host, 64, cudaHostAllocMapped), PIE_ERR_NOMEM);
+    std::memset(p->status_host, 0, 64);
+    PIE_TRY(cudaHostGetDevicePointer((void **)&p->status_dev, p->status_host, 0), PIE_ERR_CUDA);
+
+    // attention scratch: every chunk of every sequence, all KV heads
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    const int64_t max_chunks = ((int64_t)cfg->n_logical_blocks * 16 + p->cfg.split_tokens - 1) / p->cfg.split_tokens + cfg->max_seqs;
+    p->scratch.max_items = max_chunks * cfg->n_kv_heads;
+    p->scratch.max_seqs = cfg->max_seqs;
+    PIE_TRY(cudaMalloc((void **)&p->scratch.chunk_off, (size_t)(cfg->max_seqs + 1) * 4), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMalloc((void **)&p->scratch.part_o, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
+    PIE_TRY(pie::make_pool_tensor_maps(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, cfg->head_dim, &p->map3d, &p->map2d,
+                                       &p->use3d),
+            PIE_ERR_CUDA);
+    if (const char *env = std::getenv("PIE_TMA_2D"))
+        if (env[0] == '1') p->use3d = 0;
+    int per_sm = 0;
+    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, &per_sm), PIE_ERR_CUDA);
+    if (per_sm <= 0) { destroy_pool(p); return PIE_ERR_UNSUPPORTED; }
+    if (cfg->attn_ctas_per_sm > 0) per_sm = std::min(per_sm, cfg->attn_ctas_per_sm);
+    p->attn_grid = per_sm * p->n_sms;
+#undef PIE_TRY
+    *out = p;
+    return PIE_OK;
+}
+
+int pie_pool_destroy(pie_pool *pool) {
+    if (!pool) return PIE_OK;
+    int st = sync_all(pool, 10 * 1000 * 1000);
+    destroy_pool(pool);
+    return st == PIE_ERR_TIMEOUT ? st : PIE_OK;
+}
+
+int pie_block_alloc(pie_pool *pool, int64_t n, const uint8_t *on_host, int32_t *ids_out) {
+    if (!pool || n < 0 || (n > 0 && !ids_out)) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    pie::Table *t = pool->table;
+    const int32_t NB = pool->cfg.n_logical_blocks, L = pool->cfg.n_layers;
+    if (n > NB - t->n_allocated()) return PIE_ERR_NOMEM;
+    // all-or-nothing: check the slot budget first
+    int64_t need_host = 0, need_gpu = 0;
+    {
+        int64_t gpu_left = t->gpu_available();
+        for (int64_t i = 0; i < n; ++i) {
+            if (on_host && on_host[i]) need_host += L;
+            else {
+                const int64_t g = std::min<int64_t>(L, gpu_left - need_gpu);
+                need_gpu += g;
+                need_host += L - g;
+            }
+        }
+        if (need_host > t->host_available()) return PIE_ERR_NOMEM;
+    }
+    std::vector<int32_t> entries;
+    entries.reserve((size_t)(n * L * 2));
+    int32_t next = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        while (next < NB && t->allocated(next)) ++next;
+        st = t->alloc(next, on_host && on_host[i]);
+        if (st != PIE_OK) return st;  // cannot happen after the budget check
+        ids_out[i] = next;
+        for (int32_t l = 0; l < L; ++l) {
+            const pie::Unit &u = t->unit(l, next);
+            if (u.home_host) pool->home_count[(size_t)l] += 1;
+            if (u.side == PIE_GPU) {
+                entries.push_back(l * NB + next);
+                entries.push_back(u.gpu_slot);
+            }
+        }
+    }
+    st = patch_units(pool, entries);
+    if (st != PIE_OK) pool->sticky = st;
+    return st;
+}
+
+int pie_block_free(pie_pool *pool, const int32_t *ids, int64_t n) {
+    if (!pool || n < 0 || (n > 0 && !ids)) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    pie::Table *t = pool->table;
+    const int32_t NB = pool->cfg.n_logical_blocks, L = pool->cfg.n_layers;
+    for (int64_t i = 0; i < n; ++i) {
+        if (ids[i] < 0 || ids[i] >= NB) return PIE_ERR_RANGE;
+        if (!t->allocated(ids[i])) return PIE_ERR_INVALID;
+        for (int64_t j = 0; j < i; ++j)
+            if (ids[j] == ids[i]) return PIE_ERR_INVALID;
+        for (int32_t l = 0; l < L; ++l)
+            if (t->in_flight(t->unit(l, ids[i]))) return PIE_ERR_BUSY;
+    }
+    std::vector<int32_t> entries;
+    for (int64_t i = 0; i < n; ++i) {
+        for (int32_t l = 0; l < L; ++l) {
+            const pie::Unit &u = t->unit(l, ids[i]);
+            if (u.home_host) pool->home_count[(size_t)l] -= 1;
+            if (u.side == PIE_GPU) {
+                entries.push_back(l * NB + ids[i]);
+                entries.push_back(-1);
+            }
+        }
+        t->free_block(ids[i]);
+    }
+    st = patch_units(pool, entries);
+    if (st != PIE_OK) pool->sticky = st;
+    return st;
+}
+
+static int unit_access(pie_pool *pool, int32_t layer, int32_t block, void *host_buf, bool write) {
+    if (!pool || !host_buf) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    if (layer < 0 || layer >= pool->cfg.n_layers || block < 0 || block >= pool->cfg.n_logical_blocks) return PIE_ERR_RANGE;
+    if (!pool->table->allocated(block)) return PIE_ERR_INVALID;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    pie::Unit &u = pool->table->unit(layer, block);
+    if (pool->table->in_flight(u) || write) {
+        // wait for the copies on the unit; a write must also not race an attention call still reading it
+        st = sync_all(pool, 30 * 1000 * 1000);
+        if (st != PIE_OK) return st;
+    }
+    uint8_t *p = u.side == PIE_GPU ? pool->gpu_base + (int64_t)u.gpu_slot * pool->block_bytes
+                                   : pool->host_base + (int64_t)u.host_slot * pool->block_bytes;
+    if (u.side == PIE_GPU) {
+        if (write) PIE_CUDA(cudaMemcpy(p, host_buf, (size_t)pool->block_bytes, cudaMemcpyHostToDevice));
+        else PIE_CUDA(cudaMemcpy(host_buf, p, (size_t)pool->block_bytes, cudaMemcpyDeviceToHost));
+    } else {
+        if (write) std::memcpy(p, host_buf, (size_t)pool->block_bytes);
+        else std::memcpy(host_buf, p, (size_t)pool->block_bytes);
+    }
+    return PIE_OK;
+}
+
+int pie_block_write(pie_pool *pool, int32_t layer, int32_t block, const void *host_buf) {
+    return unit_access(pool, layer, block, const_cast<void *>(host_buf), true);
+}
+int pie_block_read(pie_pool *pool, int32_t layer, int32_t block, void *host_buf) {
+    return unit_access(pool, layer, block, host_buf, false);
+}
+
+int pie_block_state(pie_pool *pool, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot) {
+    if (!pool) return PIE_ERR_INVALID;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    return pool->table->state(layer, block, state, gpu_slot, host_slot);
+}
+
+int pie_get_placement(pie_pool *pool, int32_t *side, int32_t *slot) {
+    if (!pool || !side || !slot) return PIE_ERR_INVALID;
+    const int64_t n = (int64_t)pool->cfg.n_layers * pool->cfg.n_logical_blocks;
+    for (int64_t i = 0; i < n; ++i) {
+        const pie::Unit &u = pool->table->unit((int32_t)(i / pool->cfg.n_logical_blocks), (int32_t)(i % pool->cfg.n_logical_blocks));
+        side[i] = u.side;
+        slot[i] = u.side == PIE_GPU ? u.gpu_slot : u.side == PIE_HOST ? u.host_slot : -1;
+    }
+    return PIE_OK;
+}
+
+int pie_swap_out(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode) {
+    return pool_swap(pool, PIE_Q_OUT, layer, block_ids, n, mode);
+}
+int pie_swap_in(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode) {
+    return pool_swap(pool, PIE_Q_IN, layer, block_ids, n, mode);
+}
+
+int pie_swap_raw(pie_pool *pool, int32_t dir, const int32_t *src_slots, const int32_t *dst_slots, int64_t n, int32_t mode,
+                 void *stream) {
+    if (!pool || n < 0 || (n > 0 && (!src_slots || !dst_slots))) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    if (dir != PIE_H2D && dir != PIE_D2H) return PIE_ERR_INVALID;
+    if (mode < PIE_MODE_AUTO || mode > PIE_MODE_COPY_ENGINE) return PIE_ERR_INVALID;
+    const int64_t n_src = dir == PIE_H2D ? pool->cfg.n_host_slots : pool->cfg.n_gpu_slots;
+    const int64_t n_dst = dir == PIE_H2D ? pool->cfg.n_gpu_slots : pool->cfg.n_host_slots;
+    for (int64_t i = 0; i < n; ++i)
+        if (src_slots[i] < 0 || src_slots[i] >= n_src || dst_slots[i] < 0 || dst_slots[i] >= n_dst) return PIE_ERR_RANGE;
+    {
+        std::vector<int32_t> sorted(dst_slots, dst_slots + n);
+        std::sort(sorted.begin(), sorted.end());
+        if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return PIE_ERR_INVALID;
+    }
+    if (n == 0) return PIE_OK;
+    const int queue = dir == PIE_H2D ? PIE_Q_IN : PIE_Q_OUT;
+    cudaStream_t s = stream ? (cudaStream_t)stream : pool->stream[queue];
+    int st = do_copies(pool, queue, src_slots, dst_slots, n, nullptr, nullptr, mode, s);
+    if (st == PIE_OK) (queue == PIE_Q_IN ? pool->stats.bytes_in : pool->stats.bytes_out) += (double)n * (double)pool->block_bytes;
+    return st;
+}
+
+int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
+                         int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, const int32_t *block_table_host,
+                         const int32_t *ctx_lens_host, int32_t n_seqs, float scale, const void *k_new, const void *v_new) {
+    return attention_call(pool, layer, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, block_table_host,
+                          ctx_lens_host, n_seqs, scale, k_new, v_new);
+}
+
+int pie_step_begin(pie_pool *pool) {
+    if (!pool) return PIE_ERR_INVALID;
+    if (pool->cfg.timing) {
+        // the set about to be reused belongs to step-1's predecessor: it must have been read (or is dropped)
+        pool->prev_step_valid = pool->step > 0;
+        pool->prev_step_ticked = false;
+        ++pool->step;
+        for (LayerEvents &e : pool->lev[pool->step & 1]) e.has_in = e.has_out = e.has_compute = false;
+    } else {
+        ++pool->step;
+    }
+    return PIE_OK;
+}
+
+int pie_set_extension_ratio(pie_pool *pool, float r) {
+    if (!pool || r > 1.0f || r != r) return PIE_ERR_INVALID;
+    if (r < 0.f) {
+        if (pool->ratio_mode == 0) pool->ratio = 0.0;  // Section 3.4.2: start with everything on the GPU
+        pool->ratio_mode = 2;
+        if (!pool->cfg.timing) return PIE_ERR_INVALID;  // the controller needs the per-layer events
+    } else {
+        pool->ratio_mode = 1;
+        pool->ratio = r;
+    }
+    return PIE_OK;
+}
+
+int pie_get_extension_ratio(pie_pool *pool, float *r) {
+    if (!pool || !r) return PIE_ERR_INVALID;
+    if (pool->ratio_mode == 0) {
+        int64_t home = 0;
+        for (int64_t c : pool->home_count) home += c;
+        const int64_t units = (int64_t)pool->table->n_allocated() * pool->cfg.n_layers;
+        *r = units > 0 ? (float)((double)home / (double)units) : 0.f;
+    } else {
+        *r = (float)pool->ratio;
+    }
+    return PIE_OK;
+}
+
+int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in, int32_t *out_ids, int64_t *n_out) {
+    if (!pool || !in_ids || !n_in || !out_ids || !n_out) return PIE_ERR_INVALID;
+    if (layer < 0 || layer >= pool->cfg.n_layers) return PIE_ERR_RANGE;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    plan_layer(pool, layer, pool->v_in, pool->v_out);
+    std::copy(pool->v_in.begin(), pool->v_in.end(), in_ids);
+    std::copy(pool->v_out.begin(), pool->v_out.end(), out_ids);
+    *n_in = (int64_t)pool->v_in.size();
+    *n_out = (int64_t)pool->v_out.size();
+    return PIE_OK;
+}
+
+int pie_controller_tick(pie_pool *pool, int32_t *changed) {
+    if (!pool) return PIE_ERR_INVALID;
+    if (changed) *changed = 0;
+    if (!pool->cfg.timing || !pool->prev_step_valid || pool->prev_step_ticked) return PIE_OK;
+    std::vector<LayerEvents> &ev = pool->lev[(pool->step - 1) & 1];
+    // everything of the previous step must have completed; never block
+    for (LayerEvents &e : ev) {
+        if (e.has_compute && cudaEventQuery(e.done) != cudaSuccess) return PIE_OK;
+        if (e.has_in && cudaEventQuery(e.in1) != cudaSuccess) return PIE_OK;
+        if (e.has_out && cudaEventQuery(e.out1) != cudaSuccess) return PIE_OK;
+    }
+    double compute = 0, stall = 0, t_in = 0, t_out = 0;
+    cudaEvent_t first = nullptr, last = nullptr;
+    for (LayerEvents &e : ev) {
+        float ms = 0;
+        if (e.has_compute) {
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.go, e.done));
+            compute += ms;
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
+            stall += ms;
+            if (!first) first = e.pre;
+            last = e.done;
+        }
+        if (e.has_in) {
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.in0, e.in1));
+            t_in += ms;
+        }
+        if (e.has_out) {
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.out0, e.out1));
+            t_out += ms;
+        }
+    }
+    pool->prev_step_ticked = true;
+    pool->stats.last_step_compute_ms = compute;
+    pool->stats.last_step_stall_ms = stall;
+    pool->stats.last_step_swap_in_ms = t_in;
+    pool->stats.last_step_swap_out_ms = t_out;
+    if (first && last) {
+        float ms = 0;
+        PIE_CUDA(cudaEventElapsedTime(&ms, first, last));
+        pool->stats.last_step_ms = ms;
+    }
+    pool->stats.steps_measured += 1;
+    if (pool->ratio_mode == 2 && compute > 0) {
+        const double step = 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
+        const double r = pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall, compute, std::max(t_in, t_out));
+        if (r != pool->ratio) {
+            pool->ratio = r;
+            if (changed) *changed = 1;
+        }
+    }
+    return PIE_OK;
+}
+
+int pie_get_stats(pie_pool *pool, pie_stats *out) {
+    if (!pool || !out) return PIE_ERR_INVALID;
+    poll(pool);
+    *out = pool->stats;
+    float r = 0;
+    pie_get_extension_ratio(pool, &r);
+    out->ratio = r;
+    int64_t g = 0, h = 0, f = 0;
+    const int64_t n = (int64_t)pool->cfg.n_layers * pool->cfg.n_logical_blocks;
+    for (int64_t i = 0; i < n; ++i) {
+        const pie::Unit &u = pool->table->unit((int32_t)(i / pool->cfg.n_logical_blocks), (int32_t)(i % pool->cfg.n_logical_blocks));
+        if (u.side == PIE_FREE) continue;
+        if (pool->table->in_flight(u)) ++f;
+        else if (u.side == PIE_GPU) ++g;
+        else ++h;
+    }
+    out->n_units_gpu = g;
+    out->n_units_host = h;
+    out->n_units_in_flight = f;
+    return PIE_OK;
+}
+
+int pie_sync(pie_pool *pool, int64_t timeout_us) {
+    if (!pool) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    int st = sync_all(pool, timeout_us);
+    if (st != PIE_OK) return st;
+    return check_status_word(pool);
+}
+
+int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev, int32_t max_blocks_per_seq,
+                    const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new_all, const void *v_new_all,
+                    int32_t mode) {
+    if (!pool || !q_all || !out_all) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    const int32_t L = pool->cfg.n_layers;
+    const int64_t q_stride = (int64_t)n_seqs * pool->cfg.n_q_heads * pool->cfg.head_dim * 2;
+    const int64_t kv_stride = (int64_t)n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;
+    int st = pie_step_begin(pool);
+    if (st != PIE_OK) return st;
+    // layer 0 has no predecessor in the first step: fetch what it needs now (later steps prefetch it from layer L-1)
+    {
+        pool->v_in.clear();
+        for (int32_t b = 0; b < pool->cfg.n_logical_blocks; ++b)
+            if (pool->table->allocated(b) && pool->table->unit(0, b).side == PIE_HOST) pool->v_in.push_back(b);
+        if (!pool->v_in.empty()) {
+            std::vector<int32_t> ids(pool->v_in);
+            st = pool_swap(pool, PIE_Q_IN, 0, ids.data(), (int64_t)ids.size(), mode);
+            if (st != PIE_OK) return st;
+        }
+    }
+    std::vector<int32_t> in_ids, out_ids;
+    for (int32_t l = 0; l < L; ++l) {
+        st = poll(pool);
+        if (st != PIE_OK) return st;
+        plan_layer(pool, l, in_ids, out_ids);
+        if (L > 1 && !in_ids.empty()) {
+            st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode);
+            if (st != PIE_OK) return st;
+        }
+        st = attention_call(pool, l, (const uint8_t *)q_all + l * q_stride, (uint8_t *)out_all + l * q_stride, block_table_dev,
+                            max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
+                            k_new_all ? (const uint8_t *)k_new_all + l * kv_stride : nullptr,
+                            v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr);
+        if (st != PIE_OK) return st;
+        if (L > 1 && !out_ids.empty()) {
+            st = pool_swap(pool, PIE_Q_OUT, l, out_ids.data(), (int64_t)out_ids.size(), mode);
+            if (st != PIE_OK) return st;
+        }
+    }
+    return pie_controller_tick(pool, nullptr);
+}
+
+int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_host, const int32_t *block_table_host,
+                         int32_t max_blocks_per_seq, const int32_t *ctx_lens_host, int32_t n_seqs, float scale,
+                         const void *k_new_all_host, const void *v_new_all_host, int32_t mode) {
+    if (!pool || !q_all_host || !out_all_host || !block_table_host || !ctx_lens_host) return PIE_ERR_INVALID;
+    if (n_seqs <= 0 || n_seqs > pool->scratch.max_seqs || max_blocks_per_seq <= 0) return PIE_ERR_INVALID;
+    if ((k_new_all_host == nullptr) != (v_new_all_host == nullptr)) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    int st = ensure_stage(pool, n_seqs, max_blocks_per_seq);
+    if (st != PIE_OK) return st;
+    cudaStream_t s = pool->stream[PIE_Q_COMPUTE];
+    const int64_t qb = (int64_t)pool->cfg.n_layers * n_seqs * pool->cfg.n_q_heads * pool->cfg.head_dim * 2;
+    const int64_t kb = (int64_t)pool->cfg.n_layers * n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;
+    PIE_CUDA(cudaMemcpyAsync(pool->stage_q, q_all_host, (size_t)qb, cudaMemcpyHostToDevice, s));
+    if (k_new_all_host) {
+        PIE_CUDA(cudaMemcpyAsync(pool->stage_k, k_new_all_host, (size_t)kb, cudaMemcpyHostToDevice, s));
+        PIE_CUDA(cudaMemcpyAsync(pool->stage_v, v_new_all_host, (size_t)kb, cudaMemcpyHostToDevice, s));
+    }
+    PIE_CUDA(cudaMemcpyAsync(pool->stage_bt, block_table_host, (size_t)n_seqs * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, s));
+    PIE_CUDA(cudaMemcpyAsync(pool->stage_ctx, ctx_lens_host, (size_t)n_seqs * 4, cudaMemcpyHostToDevice, s));
+    st = pie_decode_step(pool, pool->stage_q, pool->stage_out, pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
+                         k_new_all_host ? pool->stage_k : nullptr, k_new_all_host ? pool->stage_v : nullptr, mode);
+    if (st != PIE_OK) return st;
+    PIE_CUDA(cudaMemcpyAsync(out_all_host, pool->stage_out, (size_t)qb, cudaMemcpyDeviceToHost, s));
+    PIE_CUDA(cudaStreamSynchronize(s));
+    return check_status_word(pool);
+}
+
+int pie_probe_link(int64_t bytes, int32_t dir, int32_t reps, double *gbps) {
+    if (bytes <= 0 || dir < 0 || dir > 2 || reps <= 0 || !gbps) return PIE_ERR_INVALID;
+    void *h[2] = {nullptr, nullptr}, *d[2] = {nullptr, nullptr};
+    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaEvent_t e0 = nullptr, e1[2] = {nullptr, nullptr};
+    int rc = PIE_OK;
+    double best = 0;
+    auto cleanup = [&]() {
+        for (int i = 0; i < 2; ++i) {
+            if (h[i]) cudaFreeHost(h[i]);
+            if (d[i]) cudaFree(d[i]);
+            if (s[i]) cudaStreamDestroy(s[i]);
+            if (e1[i]) cudaEventDestroy(e1[i]);
+        }
+        if (e0) cudaEventDestroy(e0);
+    };
+#define PROBE(call) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) { g_last_cuda_error = (int)e__; cleanup(); return PIE_ERR_CUDA; } } while (0)
+    const int n = dir == 2 ? 2 : 1;
+    for (int i = 0; i < n; ++i) {
+        PROBE(cudaHostAlloc(&h[i], (size_t)bytes, cudaHostAllocDefault));
+        std::memset(h[i], 1, (size_t)bytes);
+        PROBE(cudaMalloc(&d[i], (size_t)bytes));
+        PROBE(cudaStreamCreateWithFlags(&s[i], cudaStreamNonBlocking));
+        PROBE(cudaEventCreate(&e1[i]));
+    }
+    PROBE(cudaEventCreate(&e0));
+    for (int r = 0; r < reps + 1; ++r) {  // first repetition is a warm-up
+        PROBE(cudaEventRecord(e0, s[0]));
+        if (n == 2) PROBE(cudaStreamWaitEvent(s[1], e0, 0));
+        for (int i = 0; i < n; ++i) {
+            const bool h2d = dir == PIE_H2D || (dir == 2 && i == 0);
+            if (h2d) PROBE(cudaMemcpyAsync(d[i], h[i], (size_t)bytes, cudaMemcpyHostToDevice, s[i]));
+            else PROBE(cudaMemcpyAsync(h[i], d[i], (size_t)bytes, cudaMemcpyDeviceToHost, s[i]));
+            PROBE(cudaEventRecord(e1[i], s[i]));
+        }
+        float worst = 0;
+        for (int i = 0; i < n; ++i) {
+            PROBE(cudaEventSynchronize(e1[i]));
+            float ms = 0;
+            PROBE(cudaEventElapsedTime(&ms, e0, e1[i]));
+            worst = std::max(worst, ms);
+        }
+        if (r > 0 && worst > 0) best = std::max(best, (double)bytes / (worst * 1e-3) / 1e9);
+    }
+#undef PROBE
+    cleanup();
+    *gbps = best;
+    return rc;
+}
+
+int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps) {
+    if (bytes <= 0 || reps <= 0 || !gbps) return PIE_ERR_INVALID;
+    void *a = nullptr, *b = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    auto cleanup = [&]() {
+        cudaFree(a);
+        cudaFree(b);
+        if (e0) cudaEventDestroy(e0);
+        if (e1) cudaEventDestroy(e1);
+    };
+#define PROBE(call) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) { g_last_cuda_error = (int)e__; cleanup(); return PIE_ERR_CUDA; } } while (0)
+    PROBE(cudaMalloc(&a, (size_t)bytes));
+    PROBE(cudaMalloc(&b, (size_t)bytes));
+    PROBE(cudaMemset(a, 1, (size_t)bytes));
+    PROBE(cudaEventCreate(&e0));
+    PROBE(cudaEventCreate(&e1));
+    double best = 0;
+    for (int r = 0; r < reps + 1; ++r) {
+        PROBE(cudaEventRecord(e0, 0));
+        PROBE(cudaMemcpyAsync(b, a, (size_t)bytes, cudaMemcpyDeviceToDevice, 0));
+        PROBE(cudaEventRecord(e1, 0));
+        PROBE(cudaEventSynchronize(e1));
+        float ms = 0;
+        PROBE(cudaEventElapsedTime(&ms, e0, e1));
+        if (r > 0 && ms > 0) best = std::max(best, 2.0 * (double)bytes / (ms * 1e-3) / 1e9);
+    }
+#undef PROBE
+    cleanup();
+    *gbps = best;
+    return PIE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,370 @@
+// Mapping table with stream-ordered two-phase updates (Section 3.2), the whole-layer swap protocol
+// (Section 3.3) and the controller's decision rule (Section 3.4.2).  Host only.
+#include "pie_table.h"
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+namespace pie {
+
+// ------------------------------------------------------------------------------------ SlotPool
+SlotPool::SlotPool(int64_t n) {
+    ready_.reserve((size_t)n);
+    for (int64_t s = n - 1; s >= 0; --s) ready_.push_back((int32_t)s);
+}
+
+void SlotPool::settle(const int64_t *done) {
+    if (pending_.empty()) return;
+    size_t keep = 0;
+    for (size_t i = 0; i < pending_.size(); ++i) {
+        const Pending p = pending_[i];
+        if (p.ticket <= done[p.queue]) ready_.push_back(p.slot);
+        else pending_[keep++] = p;
+    }
+    pending_.resize(keep);
+}
+
+int32_t SlotPool::take(SlotTag *tag) {
+    if (!ready_.empty()) {
+        int32_t s = ready_.back();
+        ready_.pop_back();
+        tag->queue = PIE_Q_NONE;
+        tag->ticket = 0;
+        return s;
+    }
+    Pending p = pending_.front();
+    pending_.pop_front();
+    tag->queue = p.queue;
+    tag->ticket = p.ticket;
+    return p.slot;
+}
+
+void SlotPool::release(int32_t slot, int32_t queue, int64_t ticket) {
+    if (queue == PIE_Q_NONE) ready_.push_back(slot);
+    else pending_.push_back({slot, queue, ticket});
+}
+
+// --------------------------------------------------------------------------------------- Table
+Table::Table(int32_t n_layers, int32_t n_logical, int64_t n_gpu_slots, int64_t n_host_slots)
+    : L(n_layers), NB(n_logical), gpu_(n_gpu_slots), host_(n_host_slots),
+      units_((size_t)n_layers * (size_t)n_logical), allocated_((size_t)n_logical, 0), seen_((size_t)n_logical, 0),
+      last_compute_((size_t)n_layers, 0), layer_wait_((size_t)n_layers * 4, 0) {}
+
+int Table::alloc(int32_t block, bool on_host) {
+    if (block < 0 || block >= NB) return PIE_ERR_RANGE;
+    if (allocated_[block]) return PIE_ERR_INVALID;
+    settle();
+    int64_t n_gpu = on_host ? 0 : std::min<int64_t>(L, gpu_.available());
+    if (L - n_gpu > host_.available()) return PIE_ERR_NOMEM;
+    for (int32_t l = 0; l < L; ++l) {
+        Unit &u = unit(l, block);
+        SlotTag tag;
+        if (l < n_gpu) {
+            u.gpu_slot = gpu_.take(&tag);
+            u.host_slot = -1;
+            u.side = PIE_GPU;
+            u.home_host = 0;
+        } else {
+            u.host_slot = host_.take(&tag);
+            u.gpu_slot = -1;
+            u.side = PIE_HOST;
+            u.home_host = 1;
+        }
+        // a recycled slot whose ticket is open makes the new unit "in flight" on that ticket
+        u.last_q = (uint8_t)tag.queue;
+        u.last_t = tag.ticket;
+        if (tag.queue != PIE_Q_NONE) {
+            int64_t &w = layer_wait_[(size_t)l * 4 + tag.queue];
+            w = std::max(w, tag.ticket);
+        }
+        u.t_stamp = clock_;
+    }
+    allocated_[block] = 1;
+    ++n_allocated_;
+    return PIE_OK;
+}
+
+int Table::free_block(int32_t block) {
+    if (block < 0 || block >= NB) return PIE_ERR_RANGE;
+    if (!allocated_[block]) return PIE_ERR_INVALID;
+    settle();
+    for (int32_t l = 0; l < L; ++l)
+        if (in_flight(unit(l, block))) return PIE_ERR_BUSY;
+    for (int32_t l = 0; l < L; ++l) {
+        Unit &u = unit(l, block);
+        if (u.side == PIE_GPU) {
+            // an attention call issued earlier may still be reading the slot
+            int64_t ct = issued_[PIE_Q_COMPUTE];
+            gpu_.release(u.gpu_slot, ct > done_[PIE_Q_COMPUTE] ? PIE_Q_COMPUTE : PIE_Q_NONE, ct);
+        } else {
+            host_.release(u.host_slot, PIE_Q_NONE, 0);
+        }
+        u = Unit();
+    }
+    allocated_[block] = 0;
+    --n_allocated_;
+    return PIE_OK;
+}
+
+int Table::check_ids(int32_t layer, const int32_t *ids, int64_t n) {
+    if (layer < 0 || layer >= L) return PIE_ERR_RANGE;
+    if (n < 0 || (n > 0 && !ids)) return PIE_ERR_INVALID;
+    if (++seen_stamp_ == 0) {  // wrapped: clear
+        std::fill(seen_.begin(), seen_.end(), 0u);
+        seen_stamp_ = 1;
+    }
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t b = ids[i];
+        if (b < 0 || b >= NB) return PIE_ERR_RANGE;
+        if (seen_[b] == seen_stamp_ || !allocated_[b]) return PIE_ERR_INVALID;
+        seen_[b] = seen_stamp_;
+    }
+    return PIE_OK;
+}
+
+int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int32_t *moved,
+                int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits) {
+    if (queue != PIE_Q_IN && queue != PIE_Q_OUT) return PIE_ERR_INVALID;
+    int st = check_ids(layer, ids, n);
+    if (st != PIE_OK) return st;
+    settle();
+    const uint8_t want = queue == PIE_Q_OUT ? PIE_HOST : PIE_GPU;
+    int64_t movers = 0;
+    for (int64_t i = 0; i < n; ++i)
+        if (unit(layer, ids[i]).side != want) ++movers;
+    SlotPool &dst_pool = queue == PIE_Q_OUT ? host_ : gpu_;
+    SlotPool &src_pool = queue == PIE_Q_OUT ? gpu_ : host_;
+    if (movers > dst_pool.available()) return PIE_ERR_NOMEM;
+    waits[0] = waits[1] = waits[2] = waits[3] = 0;
+    *n_moved = 0;
+    *ticket = 0;
+    if (movers == 0) return PIE_OK;
+    const int64_t tk = ++issued_[queue];
+    ++clock_;
+    int64_t k = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        Unit &u = unit(layer, ids[i]);
+        if (u.side == want) continue;
+        SlotTag tag;
+        int32_t d = dst_pool.take(&tag);
+        if (tag.queue != PIE_Q_NONE) waits[tag.queue] = std::max(waits[tag.queue], tag.ticket);
+        // the copy that is still bringing the unit to where it is now
+        if (in_flight(u)) waits[u.last_q] = std::max(waits[u.last_q], u.last_t);
+        int32_t s;
+        if (queue == PIE_Q_OUT) {
+            s = u.gpu_slot;
+            u.host_slot = d;
+            u.gpu_slot = -1;
+        } else {
+            s = u.host_slot;
+            u.gpu_slot = d;
+            u.host_slot = -1;
+        }
+        src_pool.release(s, queue, tk);
+        u.side = want;
+        u.last_q = (uint8_t)queue;
+        u.last_t = tk;
+        u.t_stamp = clock_;
+        moved[k] = ids[i];
+        src[k] = s;
+        dst[k] = d;
+        ++k;
+    }
+    if (queue == PIE_Q_OUT && last_compute_[layer] > done_[PIE_Q_COMPUTE])
+        // the layer's attention call also appends the new token: copy out only after it
+        waits[PIE_Q_COMPUTE] = std::max(waits[PIE_Q_COMPUTE], last_compute_[layer]);
+    if (queue == PIE_Q_IN) layer_wait_[(size_t)layer * 4 + PIE_Q_IN] = tk;
+    waits[queue] = 0;  // same queue: ordered anyway
+    for (int q = 1; q < 4; ++q)
+        if (waits[q] <= done_[q]) waits[q] = 0;
+    *n_moved = k;
+    *ticket = tk;
+    return PIE_OK;
+}
+
+int Table::attention(int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits) {
+    int st = check_ids(layer, ids, ids ? n : 0);
+    if (st != PIE_OK) return st;
+    settle();
+    waits[0] = waits[1] = waits[2] = waits[3] = 0;
+    if (ids) {
+        for (int64_t i = 0; i < n; ++i)
+            if (unit(layer, ids[i]).side != PIE_GPU) return PIE_ERR_NOT_RESIDENT;
+        for (int64_t i = 0; i < n; ++i) {
+            const Unit &u = unit(layer, ids[i]);
+            if (in_flight(u)) waits[u.last_q] = std::max(waits[u.last_q], u.last_t);
+        }
+    } else {
+        for (int q = 1; q < 4; ++q) waits[q] = layer_wait_[(size_t)layer * 4 + q];
+    }
+    waits[PIE_Q_COMPUTE] = 0;
+    for (int q = 1; q < 4; ++q)
+        if (waits[q] <= done_[q]) waits[q] = 0;
+    *ticket = ++issued_[PIE_Q_COMPUTE];
+    last_compute_[layer] = *ticket;
+    return PIE_OK;
+}
+
+int Table::confirm(int32_t queue, int64_t ticket) {
+    if (queue < 1 || queue > 3) return PIE_ERR_INVALID;
+    if (ticket > issued_[queue]) return PIE_ERR_RANGE;
+    if (ticket > done_[queue]) done_[queue] = ticket;
+    settle();
+    return PIE_OK;
+}
+
+int Table::state(int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot) {
+    if (layer < 0 || layer >= L || block < 0 || block >= NB) return PIE_ERR_RANGE;
+    const Unit &u = unit(layer, block);
+    int32_t s = u.side;
+    if (s != PIE_FREE && in_flight(u)) s = u.side == PIE_GPU ? PIE_TO_GPU : PIE_TO_HOST;
+    if (state) *state = s;
+    if (gpu_slot) *gpu_slot = u.gpu_slot;
+    if (host_slot) *host_slot = u.host_slot;
+    return PIE_OK;
+}
+
+// ---------------------------------------------------------------------------------------- Fifo
+Fifo::Fifo(int32_t n, int32_t gpu_regions, int32_t cpu_regions, const uint8_t *on_cpu)
+    : n_(n), gpu_regions_(gpu_regions), cpu_regions_(cpu_regions), loc_((size_t)n, 0) {
+    for (int32_t l = 0; l < n; ++l) loc_[l] = on_cpu && on_cpu[l] ? 1 : 0;
+}
+
+int Fifo::complete(int32_t dir) {
+    if (dir == PIE_Q_OUT) {
+        if (out_layer_ < 0) return PIE_ERR_INVALID;
+        loc_[out_layer_] = 1;  // now on the CPU: its GPU region is free
+        out_layer_ = -1;
+    } else if (dir == PIE_Q_IN) {
+        if (in_layer_ < 0) return PIE_ERR_INVALID;
+        loc_[in_layer_] = 0;  // usable on the GPU: its CPU region is free
+        in_layer_ = -1;
+    } else {
+        return PIE_ERR_INVALID;
+    }
+    return PIE_OK;
+}
+
+int Fifo::location(int32_t layer) const {
+    if (layer < 0 || layer >= n_) return PIE_ERR_RANGE;
+    return loc_[layer];
+}
+
+int Fifo::layer_start(int32_t k, int32_t *start_out, int32_t *start_in) {
+    if (k < 0 || k >= n_ || !start_out || !start_in) return PIE_ERR_INVALID;
+    *start_out = *start_in = -1;
+    auto dist = [&](int32_t l) { return ((l - k) % n_ + n_) % n_; };  // compute-steps until l is needed
+    int32_t gpu_used = 0, cpu_used = 0;
+    for (int32_t l = 0; l < n_; ++l) {
+        gpu_used += loc_[l] != 1;
+        cpu_used += loc_[l] != 0;
+    }
+    if (out_layer_ < 0 && cpu_used < cpu_regions_) {
+        // coldest GPU layer other than k: next use farthest away (the layer that just finished)
+        int32_t victim = -1;
+        for (int32_t l = 0; l < n_; ++l)
+            if (loc_[l] == 0 && l != k && (victim < 0 || dist(l) > dist(victim))) victim = l;
+        bool hotter_on_cpu = false;
+        if (victim >= 0)
+            for (int32_t l = 0; l < n_; ++l)
+                if (loc_[l] == 1 && dist(l) < dist(victim)) hotter_on_cpu = true;
+        if (hotter_on_cpu) {  // otherwise every CPU layer is colder: no swap-out
+            loc_[victim] = 2;
+            out_layer_ = victim;
+            *start_out = victim;
+            ++cpu_used;
+        }
+    }
+    if (in_layer_ < 0 && gpu_used < gpu_regions_) {
+        int32_t hot = -1;
+        for (int32_t l = 0; l < n_; ++l)
+            if (loc_[l] == 1 && (hot < 0 || dist(l) < dist(hot))) hot = l;
+        if (hot >= 0) {
+            loc_[hot] = 3;
+            in_layer_ = hot;
+            *start_in = hot;
+        }
+    }
+    return PIE_OK;
+}
+
+}  // namespace pie
+
+// ------------------------------------------------------------------------------------ C ABI
+using pie::Fifo;
+using pie::Table;
+
+extern "C" {
+
+pie_table *pie_table_create(int32_t n_layers, int32_t n_logical, int64_t n_gpu_slots, int64_t n_host_slots) {
+    if (n_layers <= 0 || n_logical <= 0 || n_gpu_slots < 0 || n_host_slots < 0) return nullptr;
+    return reinterpret_cast<pie_table *>(new (std::nothrow) Table(n_layers, n_logical, n_gpu_slots, n_host_slots));
+}
+void pie_table_destroy(pie_table *t) { delete reinterpret_cast<Table *>(t); }
+int pie_table_alloc(pie_table *t, int32_t block, int32_t on_host) {
+    return t ? reinterpret_cast<Table *>(t)->alloc(block, on_host != 0) : PIE_ERR_INVALID;
+}
+int pie_table_free(pie_table *t, int32_t block) {
+    return t ? reinterpret_cast<Table *>(t)->free_block(block) : PIE_ERR_INVALID;
+}
+int pie_table_swap(pie_table *t, int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket,
+                   int32_t *moved_ids, int32_t *src_slots, int32_t *dst_slots, int64_t *n_moved, int64_t *waits) {
+    if (!t || !ticket || !moved_ids || !src_slots || !dst_slots || !n_moved || !waits) return PIE_ERR_INVALID;
+    return reinterpret_cast<Table *>(t)->swap(queue, layer, ids, n, ticket, moved_ids, src_slots, dst_slots, n_moved,
+                                              waits);
+}
+int pie_table_attention(pie_table *t, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits) {
+    if (!t || !ticket || !waits) return PIE_ERR_INVALID;
+    return reinterpret_cast<Table *>(t)->attention(layer, ids, n, ticket, waits);
+}
+int pie_table_confirm(pie_table *t, int32_t queue, int64_t ticket) {
+    return t ? reinterpret_cast<Table *>(t)->confirm(queue, ticket) : PIE_ERR_INVALID;
+}
+int pie_table_state(pie_table *t, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot,
+                    int32_t *host_slot) {
+    return t ? reinterpret_cast<Table *>(t)->state(layer, block, state, gpu_slot, host_slot) : PIE_ERR_INVALID;
+}
+
+pie_fifo *pie_fifo_create(int32_t n_layers, int32_t gpu_regions, int32_t cpu_regions, const uint8_t *on_cpu) {
+    if (n_layers <= 0 || gpu_regions <= 0 || cpu_regions < 0) return nullptr;
+    return reinterpret_cast<pie_fifo *>(new (std::nothrow) Fifo(n_layers, gpu_regions, cpu_regions, on_cpu));
+}
+void pie_fifo_destroy(pie_fifo *f) { delete reinterpret_cast<Fifo *>(f); }
+int pie_fifo_complete(pie_fifo *f, int32_t dir) { return f ? reinterpret_cast<Fifo *>(f)->complete(dir) : PIE_ERR_INVALID; }
+int pie_fifo_layer_start(pie_fifo *f, int32_t k, int32_t *start_out, int32_t *start_in) {
+    return f ? reinterpret_cast<Fifo *>(f)->layer_start(k, start_out, start_in) : PIE_ERR_INVALID;
+}
+int pie_fifo_location(pie_fifo *f, int32_t layer) {
+    return f ? reinterpret_cast<Fifo *>(f)->location(layer) : PIE_ERR_INVALID;
+}
+
+// state[0..3]: stalled flags of the last steps (newest last), state[4]: how many are valid.
+// Constants (the paper gives none): eps = 0.02, back off on 2 stalls within 4 steps, grow while the
+// link is busy for less than 0.9 of the compute time.
+double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
+                             double swap_busy) {
+    const double eps = 0.02, u_hi = 0.9;
+    const int window = 4, k_dec = 2;
+    int n = (int)state[4];
+    bool stalled = stall > eps * compute;
+    if (n == window) {
+        for (int i = 1; i < window; ++i) state[i - 1] = state[i];
+        n = window - 1;
+    }
+    state[n++] = stalled ? 1.0 : 0.0;
+    state[4] = n;
+    if (stalled) {
+        int count = 0;
+        for (int i = 0; i < n; ++i) count += state[i] != 0.0;
+        if (count >= k_dec) {
+            ratio = std::max(0.0, ratio - step);
+            state[4] = 0;  // start a fresh window after a change
+        }
+    } else if (swap_busy < u_hi * compute && ratio < 1.0) {
+        ratio = std::min(1.0, ratio + step);
+    }
+    return ratio;
+}
+
+}  // extern "C"

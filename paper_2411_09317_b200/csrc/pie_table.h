@@ -1,0 +1,101 @@
+// Host-side mapping table, slot pools, whole-layer protocol scheduler and controller rule.
+// Pure C++ (no CUDA): pie_pool drives it, and it is exported through the C ABI for CPU tests.
+#pragma once
+#include <cstdint>
+#include <deque>
+#include <vector>
+
+#include "../../include/pie.h"
+
+namespace pie {
+
+struct SlotTag {
+    int32_t queue;
+    int64_t ticket;
+};
+
+// Free slots of one pool.  `ready` is a stack (slot 0 on top at start); `pending` is a queue of slots
+// released by a copy that may not have finished: they can be handed out, but the receiver must wait
+// for the tag's ticket.
+class SlotPool {
+  public:
+    explicit SlotPool(int64_t n);
+    void settle(const int64_t *done);
+    int64_t available() const { return (int64_t)ready_.size() + (int64_t)pending_.size(); }
+    int32_t take(SlotTag *tag);
+    void release(int32_t slot, int32_t queue, int64_t ticket);
+
+  private:
+    struct Pending {
+        int32_t slot;
+        int32_t queue;
+        int64_t ticket;
+    };
+    std::vector<int32_t> ready_;
+    std::deque<Pending> pending_;
+};
+
+struct Unit {
+    uint8_t side = PIE_FREE;  // PIE_FREE / PIE_GPU / PIE_HOST: where the unit is or is heading
+    uint8_t last_q = PIE_Q_NONE;
+    uint8_t home_host = 0;  // belongs to the host-resident set between uses
+    int32_t gpu_slot = -1;
+    int32_t host_slot = -1;
+    int64_t last_t = 0;
+    uint32_t t_stamp = 0;  // the table's timestamp column (Section 3.2)
+};
+
+class Table {
+  public:
+    Table(int32_t n_layers, int32_t n_logical, int64_t n_gpu_slots, int64_t n_host_slots);
+
+    int alloc(int32_t block, bool on_host);
+    int free_block(int32_t block);
+    int swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int32_t *moved,
+             int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits);
+    int attention(int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits);
+    int confirm(int32_t queue, int64_t ticket);
+    int state(int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot);
+
+    bool in_flight(const Unit &u) const { return u.last_q != PIE_Q_NONE && u.last_t > done_[u.last_q]; }
+    Unit &unit(int32_t layer, int32_t block) { return units_[(int64_t)layer * NB + block]; }
+    bool allocated(int32_t block) const { return allocated_[block] != 0; }
+    int64_t gpu_available() { settle(); return gpu_.available(); }
+    int64_t host_available() { settle(); return host_.available(); }
+    int64_t issued(int q) const { return issued_[q]; }
+    int64_t done(int q) const { return done_[q]; }
+    int32_t n_allocated() const { return n_allocated_; }
+    void settle() { gpu_.settle(done_); host_.settle(done_); }
+
+    const int32_t L, NB;
+
+  private:
+    int check_ids(int32_t layer, const int32_t *ids, int64_t n);
+    SlotPool gpu_, host_;
+    std::vector<Unit> units_;
+    std::vector<uint8_t> allocated_;
+    std::vector<uint32_t> seen_;  // duplicate detection: seen_[block] == stamp
+    uint32_t seen_stamp_ = 0;
+    std::vector<int64_t> last_compute_;      // per layer
+    std::vector<int64_t> layer_wait_;        // per layer x 4 queues: newest open ticket among its units
+    int64_t issued_[4] = {0, 0, 0, 0};
+    int64_t done_[4] = {0, 0, 0, 0};
+    uint32_t clock_ = 0;
+    int32_t n_allocated_ = 0;
+};
+
+// Whole-layer protocol of Section 3.3.
+class Fifo {
+  public:
+    Fifo(int32_t n, int32_t gpu_regions, int32_t cpu_regions, const uint8_t *on_cpu);
+    int complete(int32_t dir);
+    int layer_start(int32_t k, int32_t *start_out, int32_t *start_in);
+    int location(int32_t layer) const;
+
+  private:
+    int32_t n_, gpu_regions_, cpu_regions_;
+    std::vector<uint8_t> loc_;  // 0 GPU, 1 CPU, 2 to CPU, 3 to GPU
+    int32_t out_layer_ = -1, in_layer_ = -1;
+};
+
+}  // namespace pie
