@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-swap + paged-decode-attention hot path on B200.
+
+A *step* is one decode step of the whole path over one batch: for each layer, prefetch the next layer's
+host-resident blocks, append the new token's K/V, split-K paged attention + combine, push the layer's share
+back to the host; controller tick at the end.  Workload at N = 1: the Llama-2-7B-shaped configuration
+(32 layers, 32/32 heads, head_dim 128, fp16, batch 64, contexts uniform in [512, 2048], 16-token blocks).
+
+Prints ONE JSON line.  `value` = decode-attention GB/s over whole steps (algorithmic KV + q + out + table bytes
+of all layers / step time) with the swap path running at the controller's transparent ratio; the run "as
+configured" (30 % of blocks host resident, link-bound by construction) and the resident run are reported
+beside it, with the hidden-swap figures, the roofline of the attention kernel and the CPU oracle's time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--scale F]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2411_09317_b200 import synth  # noqa: E402
+
+WORKLOAD = "llama2_7b"
+METRIC = "paged decode-attn GB/s over whole decode steps, swaps hidden at <=2% slowdown"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "200"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# -------------------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample of the same workload
+# -------------------------------------------------------------------------------------------------------
+def oracle_sample(wl, n_seqs_sample=6, min_seconds=10.0, max_seconds=30.0):
+    """Time the oracle's paged attention of layer 0 for the first `n_seqs_sample` sequences (contents from the
+    numpy generator), all host cores, repeated until `min_seconds` of CPU work.  -> dict for the JSON line."""
+    import oracle
+    block_table, nblk, NB = wl.tables()
+    S = min(n_seqs_sample, wl.n_seqs)
+    ctx = (wl.ctx_lens[:S] + 1).astype(np.int32)
+    ids = np.unique(np.concatenate([block_table[s, :nblk[s]] for s in range(S)]))
+    elems = wl.block_bytes // 2
+    pool = np.zeros((len(ids), elems), dtype=np.uint16)
+    slot_of = np.full(NB, -1, dtype=np.int32)
+    for i, b in enumerate(ids):
+        pool[i] = synth.kv_unit_bits(wl.seed, 0, int(b), NB, wl.n_kv_heads, wl.head_dim, wl.dtype).ravel()
+        slot_of[b] = i
+    side = np.zeros(NB, dtype=np.int32)
+    q = synth.tensor_bits(wl.seed, synth.STREAM_Q, (wl.n_seqs, wl.n_q_heads, wl.head_dim), wl.dtype)[:S]
+    cores = os.cpu_count() or 1
+    nbytes = int(ctx.astype(np.int64).sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2 + 2 * S * wl.n_q_heads * wl.head_dim * 2 \
+        + 4 * (int(((ctx + 15) // 16).sum()) + S)
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        oracle.paged_attention(pool, pool, side, np.maximum(slot_of, 0), q, block_table[:S], ctx, wl.n_q_heads,
+                               wl.n_kv_heads, wl.head_dim, wl.dtype, 1.0 / np.sqrt(wl.head_dim), "f32", nthreads=cores)
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds or dt >= max_seconds:
+            break
+    return {"value": nbytes * reps / dt / 1e9, "unit": "GB/s", "cores": min(cores, S), "kind": "oracle",
+            "sample": f"layer 0, first {S} of {wl.n_seqs} sequences ({int(ctx.sum())} tokens), fp32 oracle, "
+                      f"{reps} passes in {dt:.1f} s", "seconds": dt, "bytes_per_pass": nbytes}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same metric and workload, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = synth.workload(WORKLOAD, args.scale)
+    import oracle
+    oracle.build()
+    times, info = [], None
+    for i in range(args.warmup + args.steps):
+        info = oracle_sample(wl, n_seqs_sample=4, min_seconds=0.0, max_seconds=0.0)
+        if i >= args.warmup:
+            times.append(info["seconds"])
+    ms = float(np.mean(times)) * 1e3
+    value = info["bytes_per_pass"] / (ms * 1e-3) / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "gpu_launches": 0,
+            "config": {"workload": f"{WORKLOAD} (Llama-2-7B-shaped KV), CPU oracle on a sample", "scale": args.scale},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": info["cores"], "kind": "oracle", "sample": info["sample"]},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# -------------------------------------------------------------------------------------------------------
+def timed_steps(dw, torch, n, append=True, mode=0):
+    """Run n decode steps back to back; -> (ms total by CUDA events on the compute stream, per-step stats)."""
+    from paper_2411_09317_b200 import binding as pie
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dw.sync()
+    stats = []
+    with torch.cuda.stream(dw.s_compute):
+        e0.record()
+    for _ in range(n):
+        dw.advance_context()
+        dw.decode_step(append=append, mode=mode)
+        stats.append(pie.pie_get_stats(dw.pool))
+    with torch.cuda.stream(dw.s_compute):
+        e1.record()
+    dw.sync()
+    return e0.elapsed_time(e1), stats
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--scale", type=float, default=1.0, help="<1: fewer layers/sequences (smoke runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--split", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--swap-ctas", type=int, default=0)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2411_09317_b200 import binding as pie
+    from paper_2411_09317_b200.harness import DeviceWorkload
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    wl = synth.workload(WORKLOAD, args.scale)
+    L = wl.n_layers
+    # link and HBM probes (this process's GPU)
+    link = {"h2d": pie.pie_probe_link(256 << 20, pie.PIE_H2D, 3), "d2h": pie.pie_probe_link(256 << 20, pie.PIE_D2H, 3),
+            "both": pie.pie_probe_link(256 << 20, 2, 3)}
+    hbm_probe = pie.pie_probe_hbm(1 << 30, 3)
+
+    dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
+                        attn_ctas_per_sm=args.ctas_per_sm)
+    bytes_layer0 = dw.attention_bytes_per_layer()
+
+    def bytes_of_steps(n_steps, ctx_before):
+        """Algorithmic attention bytes of n steps starting from context lengths ctx_before (each step adds a token)."""
+        total = 0
+        ctx = ctx_before.astype(np.int64).copy()
+        for _ in range(n_steps):
+            ctx += 1
+            kv = int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2
+            qo = 2 * wl.n_seqs * wl.n_q_heads * wl.head_dim * 2
+            tab = 4 * (int(((ctx + 15) // 16).sum()) + wl.n_seqs)
+            total += L * (kv + qo + tab)
+        return total
+
+    # ---- phase 1: as configured (30 % of blocks host resident; link-bound by construction) ----------------
+    n_conf = 3
+    timed_steps(dw, torch, 1)  # warm-up: first step fetches layer 0 on demand
+    c0 = dw.ctx_lens.copy()
+    s_before = pie.pie_get_stats(dw.pool)
+    ms_conf, st_conf = timed_steps(dw, torch, n_conf)
+    s_after = pie.pie_get_stats(dw.pool)
+    as_configured = {
+        "host_fraction": wl.host_frac, "steps": n_conf, "ms_per_step": ms_conf / n_conf,
+        "attn_gbs": bytes_of_steps(n_conf, c0) / (ms_conf * 1e-3) / 1e9,
+        "swap_in_gbs": (s_after["bytes_in"] - s_before["bytes_in"]) / (ms_conf * 1e-3) / 1e9,
+        "swap_out_gbs": (s_after["bytes_out"] - s_before["bytes_out"]) / (ms_conf * 1e-3) / 1e9,
+        "stall_frac": st_conf[-1]["last_step_stall_ms"] / max(st_conf[-1]["last_step_ms"], 1e-9),
+    }
+
+    # ---- phase 2: resident baseline (ratio 0: nothing moves) ---------------------------------------------------
+    pie.pie_set_extension_ratio(dw.pool, 0.0)
+    timed_steps(dw, torch, 3)  # drains the host-resident sets back to the GPU
+    c0 = dw.ctx_lens.copy()
+    barrier()
+    ms_res, st_res = timed_steps(dw, torch, args.steps)
+    resident_gbs = bytes_of_steps(args.steps, c0) / (ms_res * 1e-3) / 1e9
+
+    # ---- phase 3: adaptive controller -> transparent ratio; the headline timed region ---------------------------
+    pie.pie_set_controller(dw.pool, 1.0 / 4096.0, 0.0, 0.0)
+    pie.pie_set_extension_ratio(dw.pool, -1.0)
+    ramp = max(args.warmup, 48)
+    timed_steps(dw, torch, ramp)
+    c0 = dw.ctx_lens.copy()
+    s_before = pie.pie_get_stats(dw.pool)
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    ms_run, st_run = timed_steps(dw, torch, args.steps)
+    barrier()
+    clocks = sampler.stop()
+    s_after = pie.pie_get_stats(dw.pool)
+    ms_run = max_over_ranks(ms_run)
+    step_bytes = bytes_of_steps(args.steps, c0)
+    value_1gpu = step_bytes / (ms_run * 1e-3) / 1e9
+    swapped_in = s_after["bytes_in"] - s_before["bytes_in"]
+    swapped_out = s_after["bytes_out"] - s_before["bytes_out"]
+    comp_ms = [s["last_step_compute_ms"] for s in st_run if s["steps_measured"] > 0]
+    attn_ms_layer = float(np.mean(comp_ms)) / L if comp_ms else float("nan")
+    n_launch = int(4 * L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
+                   (s_after["calls_copy_engine"] - s_before["calls_copy_engine"]))
+    slowdown = ms_run / ms_res - 1.0
+    hidden = {
+        "ratio": s_after["ratio"], "swap_in_gbs": swapped_in / (ms_run * 1e-3) / 1e9,
+        "swap_out_gbs": swapped_out / (ms_run * 1e-3) / 1e9, "link_h2d_gbs": link["h2d"], "link_d2h_gbs": link["d2h"],
+        "link_both_gbs_per_dir": link["both"], "slowdown_vs_resident": slowdown,
+        "frac_of_link": (swapped_in / (ms_run * 1e-3) / 1e9) / max(link["h2d"], 1e-9),
+        "stall_frac": st_run[-1]["last_step_stall_ms"] / max(st_run[-1]["last_step_ms"], 1e-9),
+    }
+
+    # ---- e2e: the same step through the host-buffer entry point (inputs H2D, outputs D2H inside the region) -----
+    q_h = torch.empty(dw.q_all.shape, dtype=torch.int16).pin_memory()
+    k_h = torch.empty(dw.k_new.shape, dtype=torch.int16).pin_memory()
+    v_h = torch.empty(dw.v_new.shape, dtype=torch.int16).pin_memory()
+    o_h = torch.empty(dw.q_all.shape, dtype=torch.int16).pin_memory()
+    q_h.copy_(dw.q_all)
+    k_h.copy_(dw.k_new)
+    v_h.copy_(dw.v_new)
+    torch.cuda.synchronize()
+    h2d = q_h.numel() * 2 + k_h.numel() * 2 + v_h.numel() * 2 + dw.block_table.nbytes + dw.ctx_lens.nbytes
+    d2h = o_h.numel() * 2
+
+    def host_step():
+        dw.advance_context()
+        pie.pie_decode_step_host(dw.pool, q_h.data_ptr(), o_h.data_ptr(), dw.block_table, dw.max_blocks, dw.ctx_lens,
+                                 wl.n_seqs, dw.scale, k_h.data_ptr(), v_h.data_ptr())
+
+    for _ in range(3):
+        host_step()
+    c0 = dw.ctx_lens.copy()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        host_step()
+    dw.sync()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
+    e2e_value = bytes_of_steps(args.steps, c0) / (e2e_ms * 1e-3) / 1e9
+
+    peak, peak_kind = measured_peaks()
+    achieved = bytes_layer0 / (attn_ms_layer * 1e-3) / 1e9 if attn_ms_layer == attn_ms_layer else None
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": None, "peak_kind": peak_kind,
+                "kernel": "paged_decode_attn_kernel (+plan, append, combine: per-layer event span)",
+                "alg_bytes_per_launch": bytes_layer0, "ms_per_launch": attn_ms_layer, "hbm_copy_probe_gbs": hbm_probe,
+                "frac_of_nominal_8tbs": (achieved / 8000.0) if achieved else None}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        cpu = oracle_sample(wl)
+        cpu.pop("seconds", None)
+        cpu.pop("bytes_per_pass", None)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value_1gpu * world, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": ramp, "ms_per_step": ms_run / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f16", "data": "synthetic", "gpu_launches": n_launch,
+            "config": {"workload": "llama2_7b: 32 layers, 32q/32kv heads, head_dim 128, fp16, 16-token blocks, batch 64, "
+                                   "contexts U[512,2048] (+1 token per step), per-layer prefetch; host-resident share "
+                                   "chosen by the adaptive controller (the configured 30 % run is under as_configured)",
+                       "scale": args.scale, "n_layers": L, "n_seqs": wl.n_seqs, "l2": "inputs larger than L2 "
+                       f"({bytes_layer0 / 1e9:.2f} GB of distinct KV per layer call)", "parallelism": "replicas only"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value * world, "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "ms_per_step": e2e_ms / args.steps},
+            "roofline": roofline, "cpu_baseline": cpu,
+            "hidden_swap": hidden, "resident": {"attn_gbs": resident_gbs, "ms_per_step": ms_res / args.steps},
+            "as_configured": as_configured,
+        }
+        print(json.dumps(line))
+    dw.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

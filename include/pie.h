@@ -185,6 +185,10 @@ int pie_step_begin(pie_pool *pool);
  * the current one.  Until the first call the host-resident sets are whatever the caller established. */
 int pie_set_extension_ratio(pie_pool *pool, float r);
 int pie_get_extension_ratio(pie_pool *pool, float *r);
+/* Controller constants (the paper gives none): step = ratio change per adjustment (default 1 / n_layers,
+ * "one layer"), eps = stall / compute above which a step counts as stalled (0.02), u_hi = link-busy /
+ * compute below which the ratio may grow (0.9).  A value <= 0 keeps the current setting. */
+int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
 /* The per-layer plan at the start of layer `layer`: in_ids = units of layer (layer+1) mod L to bring in
  * (ascending id, as many as the GPU pool can take), out_ids = units of `layer` to push out once it has
  * computed.  Arrays are host, capacity n_logical_blocks each. */
@@ -235,7 +239,8 @@ int pie_fifo_layer_start(pie_fifo *f, int32_t k, int32_t *start_out, int32_t *st
 int pie_fifo_location(pie_fifo *f, int32_t layer);
 
 /* The controller's decision rule by itself.  state: 8 doubles owned by the caller, zero-initialised
- * (history).  Returns the new ratio for one decode step's measurements (same unit for all three). */
+ * (history in [0..4]; [5] = stall tolerance eps, [6] = link-busy ceiling u_hi, 0 = defaults 0.02 / 0.9).
+ * Returns the new ratio for one decode step's measurements (same unit for all three). */
 double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
                              double swap_busy);
 

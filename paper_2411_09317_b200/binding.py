@@ -29,7 +29,7 @@ EXPORTS = [
     "pie_pool_create", "pie_pool_destroy", "pie_block_bytes", "pie_block_alloc", "pie_block_free", "pie_block_write",
     "pie_block_read", "pie_block_state", "pie_get_placement", "pie_swap_out", "pie_swap_in", "pie_swap_raw",
     "pie_decode_attention", "pie_decode_step", "pie_decode_step_host", "pie_step_begin", "pie_set_extension_ratio",
-    "pie_get_extension_ratio", "pie_plan_layer", "pie_controller_tick", "pie_get_stats", "pie_sync", "pie_status_str",
+    "pie_get_extension_ratio", "pie_set_controller", "pie_plan_layer", "pie_controller_tick", "pie_get_stats", "pie_sync", "pie_status_str",
     "pie_last_cuda_error", "pie_probe_link", "pie_probe_hbm", "pie_table_create", "pie_table_destroy", "pie_table_alloc",
     "pie_table_free", "pie_table_swap", "pie_table_attention", "pie_table_confirm", "pie_table_state", "pie_fifo_create",
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
@@ -86,6 +86,7 @@ _sig = {
     "pie_step_begin": (_i32, [_vp]),
     "pie_set_extension_ratio": (_i32, [_vp, _f32]),
     "pie_get_extension_ratio": (_i32, [_vp, ctypes.POINTER(_f32)]),
+    "pie_set_controller": (_i32, [_vp, _f64, _f64, _f64]),
     "pie_plan_layer": (_i32, [_vp, _i32, _vp, ctypes.POINTER(_i64), _vp, ctypes.POINTER(_i64)]),
     "pie_controller_tick": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "pie_get_stats": (_i32, [_vp, ctypes.POINTER(Stats)]),
@@ -252,6 +253,10 @@ def pie_get_extension_ratio(pool) -> float:
     r = _f32()
     check(lib.pie_get_extension_ratio(pool, ctypes.byref(r)), "pie_get_extension_ratio")
     return r.value
+
+
+def pie_set_controller(pool, step=0.0, eps=0.0, u_hi=0.0) -> None:
+    check(lib.pie_set_controller(pool, step, eps, u_hi), "pie_set_controller")
 
 
 def pie_plan_layer(pool, layer, n_logical):

@@ -488,8 +488,16 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 o[j][3] *= a1;
             }
             // P^T as the B operand of O^T += V^T P^T: transpose the two 8x8 (token x head) blocks
-            const uint32_t pb0 = movmatrix_trans(pack2<BF16>(p0, p1));
-            const uint32_t pb1 = movmatrix_trans(pack2<BF16>(p2, p3));
+            const uint32_t h01 = pack2<BF16>(p0, p1), h23 = pack2<BF16>(p2, p3);
+            const uint32_t pb0 = movmatrix_trans(h01);
+            const uint32_t pb1 = movmatrix_trans(h23);
+            // bf16 keeps 8 significant bits: carry the rounding remainder of P in a second bf16 term so that the
+            // PV product sees ~16 bits (fp16's 11 bits need no correction)
+            uint32_t pl0 = 0, pl1 = 0;
+            if (BF16) {
+                pl0 = movmatrix_trans(pack2<true>(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u)));
+                pl1 = movmatrix_trans(pack2<true>(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xffff0000u)));
+            }
 #pragma unroll
             for (int j = 0; j < D / 16; ++j) {
                 const int chunk = 2 * j + v_csel;
@@ -497,6 +505,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 ldmatrix_x4_trans(
                     tile_u32 + (chunk >> 3) * SM::HALF_BYTES + (16 + v_tok) * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), a);
                 mma_16816<BF16>(o[j], a, pb0, pb1);
+                if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
             }
             __syncwarp();
             if (nvalid < 16) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -72,6 +72,7 @@ struct pie_pool {
     int ratio_mode = 0;  // 0 unset (keep the caller's sets), 1 fixed, 2 adaptive
     double ratio = 0.0;
     double ctrl_state[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
     std::vector<int64_t> home_count;  // per layer: units whose home is the host
     // timing
     std::vector<LayerEvents> lev[2];
@@ -841,6 +842,14 @@ int pie_set_extension_ratio(pie_pool *pool, float r) {
     return PIE_OK;
 }
 
+int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi) {
+    if (!pool || step > 1.0 || eps >= 1.0 || u_hi > 1.0) return PIE_ERR_INVALID;
+    if (step > 0) pool->ctrl_step = step;
+    if (eps > 0) pool->ctrl_state[5] = eps;
+    if (u_hi > 0) pool->ctrl_state[6] = u_hi;
+    return PIE_OK;
+}
+
 int pie_get_extension_ratio(pie_pool *pool, float *r) {
     if (!pool || !r) return PIE_ERR_INVALID;
     if (pool->ratio_mode == 0) {
@@ -911,7 +920,7 @@ int pie_controller_tick(pie_pool *pool, int32_t *changed) {
     }
     pool->stats.steps_measured += 1;
     if (pool->ratio_mode == 2 && compute > 0) {
-        const double step = 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
+        const double step = pool->ctrl_step > 0 ? pool->ctrl_step : 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
         const double r = pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall, compute, std::max(t_in, t_out));
         if (r != pool->ratio) {
             pool->ratio = r;

@@ -339,12 +339,13 @@ int pie_fifo_location(pie_fifo *f, int32_t layer) {
     return f ? reinterpret_cast<Fifo *>(f)->location(layer) : PIE_ERR_INVALID;
 }
 
-// state[0..3]: stalled flags of the last steps (newest last), state[4]: how many are valid.
+// state[0..3]: stalled flags of the last steps (newest last), state[4]: how many are valid,
+// state[5]: eps override, state[6]: u_hi override (0 = default).
 // Constants (the paper gives none): eps = 0.02, back off on 2 stalls within 4 steps, grow while the
 // link is busy for less than 0.9 of the compute time.
 double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
                              double swap_busy) {
-    const double eps = 0.02, u_hi = 0.9;
+    const double eps = state[5] > 0 ? state[5] : 0.02, u_hi = state[6] > 0 ? state[6] : 0.9;
     const int window = 4, k_dec = 2;
     int n = (int)state[4];
     bool stalled = stall > eps * compute;

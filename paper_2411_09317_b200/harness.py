@@ -22,7 +22,7 @@ class DeviceWorkload:
     def __init__(self, wl: synth.Workload, host_frac=None, timing=True, split_tokens=0, swap_ctas=0,
                  attn_ctas_per_sm=0, staging_layers=3, shuffle_table=False, extra_gpu_slots=0, extra_host_slots=0):
         self.wl = wl
-        dev = torch.device("cuda:0")
+        dev = torch.device("cuda", torch.cuda.current_device())
         self.dev = dev
         self.host_frac = wl.host_frac if host_frac is None else host_frac
         self.block_table, self.nblk, self.NB = wl.tables(shuffle=shuffle_table)

@@ -11,7 +11,14 @@ from tests.helpers import Case
 
 pytestmark = pytest.mark.gpu
 F16, BF16 = synth.F16, synth.BF16
-TOL = 2e-3  # max-abs bound on attention outputs for N(0,1) inputs (16-bit output rounding dominates)
+TOL = 2e-3  # max-abs bound on attention outputs for the N(0,1) workloads (contexts of 100+ tokens, |out| << 1)
+
+
+def edge_tol(want, dtype):
+    """Edge cases with very short contexts have |out| of order 1-4, where rounding the output to 16 bits alone
+    costs up to half an ulp: at most 2^-8 |out| in bf16 (8 significant bits), 2^-11 |out| in fp16 (11 bits).
+    The bound is 2e-3 plus that."""
+    return TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
 
 
 # ---------------------------------------------------------------------------------- input generator
@@ -131,12 +138,13 @@ def test_swap_raw_whole_pool_untouched_bytes():
 
 
 # --------------------------------------------------------------------------------------- attention
-def check_attention(case, pc, layer, tol=TOL):
+def check_attention(case, pc, layer, edge=False):
     pc.attention(layer)
     bits, got = pc.result(layer)
     want = oracle_attention(case, layer, "f32")
-    err = np.abs(got - want).max() if got.size else 0.0
-    assert err <= tol, f"max-abs {err}"
+    err = np.abs(got - want)
+    bound = edge_tol(want, case.dtype) if edge else TOL
+    assert np.all(err <= bound), f"max-abs {err.max()}"
     return bits
 
 
@@ -150,7 +158,7 @@ def test_attention_parity_edge_lengths(hq, hkv, d, dtype):
     lens = [1, 15, 16, 17, 31, 32, 33, 255, 256, 257, 511, 512, 513, 0, 100]
     case = Case(1, hq, hkv, d, dtype, lens, seed=21, host_frac=0.0, placement="random", shuffle_table=True)
     pc = PoolCase(case)
-    check_attention(case, pc, 0)
+    check_attention(case, pc, 0, edge=True)
     pc.close()
 
 
@@ -158,7 +166,7 @@ def test_attention_parity_edge_lengths(hq, hkv, d, dtype):
 def test_attention_parity_split_sizes_and_long_context(split):
     case = Case(1, 8, 2, 128, BF16, [4097, 3, 1500], seed=22, placement="reversed")
     pc = PoolCase(case, split_tokens=split)
-    check_attention(case, pc, 0)
+    check_attention(case, pc, 0, edge=True)
     pc.close()
 
 
@@ -166,14 +174,14 @@ def test_attention_parity_batch_128_ragged():
     lens = synth.uniform_lengths(7, 128, 1, 200)
     case = Case(1, 32, 8, 128, BF16, lens, seed=23, placement="random")
     pc = PoolCase(case)
-    check_attention(case, pc, 0)
+    check_attention(case, pc, 0, edge=True)   # contexts from 1 token up
     pc.close()
 
 
 def test_tail_poison_is_excluded():
     case = Case(1, 8, 4, 128, F16, [5, 17, 33, 250], seed=24)
     pc0 = PoolCase(case)
-    clean = check_attention(case, pc0, 0)
+    clean = check_attention(case, pc0, 0, edge=True)
     pc0.close()
     for s in range(case.S):
         ctx = int(case.ctx_lens[s])
@@ -183,7 +191,7 @@ def test_tail_poison_is_excluded():
             unit[:, :, ctx % 16:, :] = 0x7E00          # NaN in K and V tails
             unit[:, 1, ctx % 16:, ::2] = 0x7C00        # +inf
     pc = PoolCase(case)
-    poisoned = check_attention(case, pc, 0)
+    poisoned = check_attention(case, pc, 0, edge=True)
     pc.close()
     assert np.array_equal(clean, poisoned)
 
@@ -196,7 +204,7 @@ def test_large_scores_running_max():
     pc.attention(0)
     bits, got = pc.result(0)
     want = oracle_attention(case, 0, "f32")
-    assert np.all(np.abs(got - want) <= TOL + 2.0 ** -8 * np.abs(want))
+    assert np.all(np.abs(got - want) <= edge_tol(want, BF16))
     pc.close()
 
 
@@ -206,7 +214,7 @@ def test_resident_vs_swapped_bit_identical():
     lens = [100, 231, 300, 17, 513]
     case = Case(2, 8, 4, 64, F16, lens, seed=0, host_frac=0.0)
     res = PoolCase(case, all_on_gpu=True)
-    ref = [check_attention(case, res, l) for l in range(case.L)]
+    ref = [check_attention(case, res, l, edge=True) for l in range(case.L)]
     res.close()
     moved = Case(2, 8, 4, 64, F16, lens, seed=0, host_frac=0.5, placement="random")
     pc = PoolCase(moved)
@@ -215,7 +223,7 @@ def test_resident_vs_swapped_bit_identical():
         others = np.setdiff1d(np.arange(moved.NB), moved.host_ids)[::2]
         pie.pie_swap_out(pc.pool, l, others, pie.PIE_MODE_KERNEL)          # push some residents out ...
         pie.pie_swap_in(pc.pool, l, others, pie.PIE_MODE_COPY_ENGINE)      # ... and back, into other slots
-        got = check_attention(moved, pc, l)
+        got = check_attention(moved, pc, l, edge=True)
         assert np.array_equal(got, ref[l])
     pc.close()
 
@@ -231,7 +239,7 @@ def test_presence_check_and_device_status_word():
         pie.pie_sync(pc.pool)
     assert e.value.status == pie.PIE_ERR_NOT_RESIDENT
     pie.pie_swap_in(pc.pool, 0, case.host_ids)
-    check_attention(case, pc, 0)
+    check_attention(case, pc, 0, edge=True)
     # a context longer than the table is rejected before anything is enqueued
     bad = case.ctx_lens.copy()
     bad[0] = 16 * case.block_table.shape[1] + 1
