@@ -217,8 +217,13 @@ def main():
             "both": pie.pie_probe_link(256 << 20, 2, 3)}
     hbm_probe = pie.pie_probe_hbm(1 << 30, 3)
 
+    # the GPU pool is sized for the fully resident baseline run as well (every unit + 3 layers of staging)
+    ramp = max(args.warmup, 48)
+    total_steps = 1 + 3 + 3 + args.steps + ramp + args.steps + 3 + args.steps   # every phase below appends one token per step
+    n_host_blocks = int(round(wl.host_frac * (int(((wl.ctx_lens.astype(np.int64) + total_steps + 15) // 16).sum()))))
     dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
-                        attn_ctas_per_sm=args.ctas_per_sm)
+                        attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=L * (n_host_blocks + wl.n_seqs),
+                        extra_tokens=total_steps)
     bytes_layer0 = dw.attention_bytes_per_layer()
 
     def bytes_of_steps(n_steps, ctx_before):
@@ -259,12 +264,11 @@ def main():
     # ---- phase 3: adaptive controller -> transparent ratio; the headline timed region ---------------------------
     pie.pie_set_controller(dw.pool, 1.0 / 4096.0, 0.0, 0.0)
     pie.pie_set_extension_ratio(dw.pool, -1.0)
-    ramp = max(args.warmup, 48)
+    sampler = ClockSampler(local)   # started before the ramp (nvidia-smi takes a while to come up); same load throughout
+    sampler.start()
     timed_steps(dw, torch, ramp)
     c0 = dw.ctx_lens.copy()
     s_before = pie.pie_get_stats(dw.pool)
-    sampler = ClockSampler(local)
-    sampler.start()
     barrier()
     ms_run, st_run = timed_steps(dw, torch, args.steps)
     barrier()
@@ -279,7 +283,7 @@ def main():
     attn_ms_layer = float(np.mean(comp_ms)) / L if comp_ms else float("nan")
     n_launch = int(4 * L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
                    (s_after["calls_copy_engine"] - s_before["calls_copy_engine"]))
-    slowdown = ms_run / ms_res - 1.0
+    slowdown = resident_gbs / value_1gpu - 1.0   # in GB/s, since the contexts keep growing between the two runs
     hidden = {
         "ratio": s_after["ratio"], "swap_in_gbs": swapped_in / (ms_run * 1e-3) / 1e9,
         "swap_out_gbs": swapped_out / (ms_run * 1e-3) / 1e9, "link_h2d_gbs": link["h2d"], "link_d2h_gbs": link["d2h"],

@@ -164,7 +164,8 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
 
 /* One decode step: for every layer l, prefetch layer l+1's host-resident units (wrapping to layer 0 of
  * the next token, Section 3.4.2), run layer l's attention, push layer l's share back out (Section 3.3:
- * the layer that just finished is the coldest).  q_all/out_all: device [n_layers][n_seqs][Hq][D];
+ * the layer that just finished is the coldest).  PIE_ERR_NOMEM if the GPU pool cannot take a layer's
+ * host-resident share (the layers before it have been enqueued).  q_all/out_all: device [n_layers][n_seqs][Hq][D];
  * k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D] or NULL.  Runs pie_controller_tick at the end
  * when the ratio is adaptive.  Never blocks the host on the GPU. */
 int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev,

@@ -32,7 +32,7 @@ constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine wh
 struct LayerEvents {
     cudaEvent_t pre = nullptr, go = nullptr, done = nullptr;  // compute stream: before wait, after wait, after layer
     cudaEvent_t in0 = nullptr, in1 = nullptr, out0 = nullptr, out1 = nullptr;
-    bool has_in = false, has_out = false, has_compute = false;
+    bool has_in = false, has_out = false, has_compute = false, waited = false;
 };
 
 struct ListRecord {
@@ -394,7 +394,10 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         st = wait_ticket(p, stream, qd, waits[qd]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
-    if (le) PIE_CUDA(cudaEventRecord(le->go, stream));
+    if (le) {
+        le->waited = waits[1] > p->table->done(1) || waits[2] > p->table->done(2);
+        PIE_CUDA(cudaEventRecord(le->go, stream));
+    }
     pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
                       p->cfg.n_gpu_slots};
     pie::AttnLaunch a{};
@@ -431,7 +434,14 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
 void apply_ratio_to_layer(pie_pool *p, int32_t layer) {
     if (p->ratio_mode == 0) return;
     const int32_t NB = p->cfg.n_logical_blocks;
-    const int64_t target = (int64_t)std::llround(p->ratio * (double)p->table->n_allocated());
+    const int64_t n_alloc = p->table->n_allocated(), L = p->cfg.n_layers;
+    int64_t target = (int64_t)std::llround(p->ratio * (double)n_alloc);
+    // the GPU pool must hold every layer's resident share plus two layers' host share in transit:
+    // L (n - h) + 2 h <= n_gpu_slots bounds the host-resident count h from below
+    if (L > 2) {
+        const int64_t deficit = L * n_alloc - p->cfg.n_gpu_slots;
+        if (deficit > 0) target = std::max(target, std::min(n_alloc, (deficit + L - 3) / (L - 2)));
+    }
     int64_t &count = p->home_count[(size_t)layer];
     if (count < target) {
         for (int32_t b = 0; b < NB && count < target; ++b) {
@@ -457,11 +467,16 @@ int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::ve
     apply_ratio_to_layer(p, next);
     // hottest first: the next layer's host-resident units, as many as the GPU pool can take
     int64_t room = p->table->gpu_available();
-    for (int32_t b = 0; b < NB && room > 0; ++b) {
+    int64_t left_behind = 0;
+    for (int32_t b = 0; b < NB; ++b) {
         if (!p->table->allocated(b)) continue;
         if (p->table->unit(next, b).side == PIE_HOST) {
-            in_ids.push_back(b);
-            --room;
+            if (room > 0) {
+                in_ids.push_back(b);
+                --room;
+            } else {
+                ++left_behind;
+            }
         }
     }
     // coldest: this layer's host-home units go back once it has computed
@@ -470,7 +485,7 @@ int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::ve
         const pie::Unit &u = p->table->unit(layer, b);
         if (u.home_host && u.side == PIE_GPU) out_ids.push_back(b);
     }
-    return PIE_OK;
+    return left_behind == 0 ? PIE_OK : PIE_ERR_NOMEM;
 }
 
 int ensure_stage(pie_pool *p, int32_t n_seqs, int32_t max_blocks) {
@@ -822,7 +837,7 @@ int pie_step_begin(pie_pool *pool) {
         pool->prev_step_valid = pool->step > 0;
         pool->prev_step_ticked = false;
         ++pool->step;
-        for (LayerEvents &e : pool->lev[pool->step & 1]) e.has_in = e.has_out = e.has_compute = false;
+        for (LayerEvents &e : pool->lev[pool->step & 1]) e.has_in = e.has_out = e.has_compute = e.waited = false;
     } else {
         ++pool->step;
     }
@@ -894,8 +909,11 @@ int pie_controller_tick(pie_pool *pool, int32_t *changed) {
         if (e.has_compute) {
             PIE_CUDA(cudaEventElapsedTime(&ms, e.go, e.done));
             compute += ms;
-            PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
-            stall += ms;
+            if (e.waited) {
+                // two back-to-back event records are already ~2-3 us apart: count only what exceeds that
+                PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
+                stall += std::max(0.0, (double)ms - 0.004);
+            }
             if (!first) first = e.pre;
             last = e.done;
         }
@@ -985,7 +1003,8 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
     for (int32_t l = 0; l < L; ++l) {
         st = poll(pool);
         if (st != PIE_OK) return st;
-        plan_layer(pool, l, in_ids, out_ids);
+        st = plan_layer(pool, l, in_ids, out_ids);
+        if (st != PIE_OK) return st;  // the GPU pool cannot take the next layer's share: nothing was enqueued for it
         if (L > 1 && !in_ids.empty()) {
             st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode);
             if (st != PIE_OK) return st;

@@ -20,12 +20,14 @@ class DeviceWorkload:
     allocation time and contents written by the generator kernels (so nothing is moved during set-up)."""
 
     def __init__(self, wl: synth.Workload, host_frac=None, timing=True, split_tokens=0, swap_ctas=0,
-                 attn_ctas_per_sm=0, staging_layers=3, shuffle_table=False, extra_gpu_slots=0, extra_host_slots=0):
+                 attn_ctas_per_sm=0, staging_layers=3, shuffle_table=False, extra_gpu_slots=0, extra_host_slots=0,
+                 extra_tokens=None):
         self.wl = wl
         dev = torch.device("cuda", torch.cuda.current_device())
         self.dev = dev
         self.host_frac = wl.host_frac if host_frac is None else host_frac
-        self.block_table, self.nblk, self.NB = wl.tables(shuffle=shuffle_table)
+        self.extra_tokens = wl.decode_steps if extra_tokens is None else extra_tokens
+        self.block_table, self.nblk, self.NB = wl.tables(shuffle=shuffle_table, extra_tokens=self.extra_tokens)
         self.max_blocks = self.block_table.shape[1]
         self.host_ids = synth.pick_host_blocks(wl.seed, self.block_table, self.nblk, self.host_frac)
         on_host = np.zeros(self.NB, dtype=np.uint8)
@@ -105,6 +107,7 @@ class DeviceWorkload:
     def advance_context(self):
         """One more token per sequence (the step's append position)."""
         self.ctx_lens += 1
+        assert int(self.ctx_lens.max() - self.wl.ctx_lens.max()) <= self.extra_tokens, "block table has no room left"
         with torch.cuda.stream(self.s_compute):
             self.ctx_lens_dev += 1
 

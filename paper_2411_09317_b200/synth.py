@@ -230,8 +230,10 @@ class Workload:
     def block_bytes(self) -> int:
         return 2 * self.block_tokens * self.n_kv_heads * self.head_dim * 2
 
-    def tables(self, shuffle: bool = False):
-        return build_block_table(self.ctx_lens, self.block_tokens, extra_tokens=self.decode_steps,
+    def tables(self, shuffle: bool = False, extra_tokens: int | None = None):
+        """Block table with room for `extra_tokens` decoded tokens per sequence (default: decode_steps)."""
+        return build_block_table(self.ctx_lens, self.block_tokens,
+                                 extra_tokens=self.decode_steps if extra_tokens is None else extra_tokens,
                                  shuffle_seed=self.seed if shuffle else None)
 
 
