@@ -209,6 +209,37 @@ int pie_probe_link(int64_t bytes, int32_t dir, int32_t reps, double *gbps);
 /* HBM probe: device-to-device copy kernel-free cudaMemcpyAsync of `bytes`; *gbps counts read+write. */
 int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps);
 
+/* ---- for callers that must not allocate ------------------------------------------------------------ */
+
+#define PIE_NOALLOC_SCRATCH_BYTES (16ll << 20) /* fixed device scratch held by every GPU that loads the library */
+#define PIE_NOALLOC_MAX_SEQS 4096
+
+/* (No counterpart in the paper: this entry point exists for the library's users.)
+ * Paged decode attention of one layer without any allocation.  pie_decode_attention needs a pie_pool, and
+ * creating a pool calls cudaMalloc / cudaHostAlloc.  Some callers may not do that: code running while another
+ * component owns the device's memory arena, plug-ins that receive fixed buffers and a stream, loops that
+ * cannot afford the device-wide synchronisation an allocation implies.  Here the caller passes everything:
+ *   kv_pool     device memory holding n_slots slots in the slot layout above, 128-byte aligned
+ *   slot_table  device int32 [n_logical_blocks]: GPU slot of each logical block of this layer, -1 if absent
+ *   q, out, block_table_dev, ctx_lens_dev, scale   as for pie_decode_attention (no append)
+ *   ctx_lens_host  host copy of the lengths (required: sizes are checked before anything is enqueued)
+ *   status_dev  optional device int32[4]; word 0 is set to 1 if a referenced block had no slot
+ *   stream      a cudaStream_t
+ * The split-K scratch (chunk offsets, fp32 partials) is a static device array of PIE_NOALLOC_SCRATCH_BYTES
+ * that every GPU loading the library holds until the process exits.  A call whose partials would not fit
+ * (sum over sequences of ceil(ctx / split_tokens), times n_q_heads * (head_dim + 2) * 4 bytes, plus 17 KiB)
+ * or with more than PIE_NOALLOC_MAX_SEQS sequences returns PIE_ERR_NOMEM and enqueues nothing.
+ * All calls on a device share that array and it keeps the previous call's contents: every word a call reads
+ * it has written first, so nothing needs clearing, but two calls that overlap on the GPU (different
+ * streams, no dependency) race - order them.  The first call on each device looks up the array's device
+ * address (cudaGetSymbolAddress) and sets the kernels' shared-memory attribute; make that first call outside
+ * any stream capture.  Calls cudaMalloc, cudaFree or any allocating routine: never. */
+int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots, const int32_t *slot_table,
+                                 int32_t n_logical_blocks, const void *q, void *out, const int32_t *block_table_dev,
+                                 int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, const int32_t *ctx_lens_host,
+                                 int32_t n_seqs, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t dtype,
+                                 int32_t split_tokens, float scale, int32_t *status_dev, void *stream);
+
 /* ---- host-only pieces, usable without a GPU ------------------------------------------------------ */
 
 /* The mapping table by itself (what pie_pool uses inside).  Stream-ordered two-phase semantics:

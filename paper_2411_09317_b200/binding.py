@@ -33,6 +33,7 @@ EXPORTS = [
     "pie_last_cuda_error", "pie_probe_link", "pie_probe_hbm", "pie_table_create", "pie_table_destroy", "pie_table_alloc",
     "pie_table_free", "pie_table_swap", "pie_table_attention", "pie_table_confirm", "pie_table_state", "pie_fifo_create",
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
+    "pie_decode_attention_noalloc",
 ]
 
 
@@ -109,6 +110,8 @@ _sig = {
     "pie_fifo_layer_start": (_i32, [_vp, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pie_fifo_location": (_i32, [_vp, _i32]),
     "pie_controller_decide": (_f64, [_vp, _f64, _f64, _f64, _f64, _f64]),
+    "pie_decode_attention_noalloc": (_i32, [_vp, _i64, _vp, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
+                                            _i32, _f32, _vp, _vp]),
 }
 for _name, (_res, _args) in _sig.items():
     _fn = getattr(lib, _name)
@@ -292,6 +295,18 @@ def pie_probe_hbm(nbytes, reps=3) -> float:
     g = _f64()
     check(lib.pie_probe_hbm(nbytes, reps, ctypes.byref(g)), "pie_probe_hbm")
     return g.value
+
+
+def pie_decode_attention_noalloc(kv_pool, n_slots, slot_table, n_logical_blocks, q, out, block_table_dev,
+                                 max_blocks_per_seq, ctx_lens_dev, ctx_lens_host, n_seqs, n_q_heads, n_kv_heads, head_dim,
+                                 dtype, scale, split_tokens=0, status_dev=None, stream=None) -> None:
+    """Attention for callers that may not allocate: no pool, the split-K scratch is a fixed device array inside
+    the library (see include/pie.h).  All device arguments are raw addresses owned by the caller."""
+    clh = _np_i32(ctx_lens_host)
+    check(lib.pie_decode_attention_noalloc(_ptr(kv_pool), n_slots, _ptr(slot_table), n_logical_blocks, _ptr(q), _ptr(out),
+                                           _ptr(block_table_dev), max_blocks_per_seq, _ptr(ctx_lens_dev), _ptr(clh), n_seqs,
+                                           n_q_heads, n_kv_heads, head_dim, dtype, split_tokens, scale, _ptr(status_dev),
+                                           _ptr(stream)), "pie_decode_attention_noalloc")
 
 
 # ---- host-only pieces ------------------------------------------------------------------------------------------
