@@ -178,6 +178,7 @@ def main():
     ap.add_argument("--split", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--swap-ctas", type=int, default=0)
+    ap.add_argument("--ramp", type=int, default=48, help="controller ramp steps before the timed region")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -218,7 +219,7 @@ def main():
     hbm_probe = pie.pie_probe_hbm(1 << 30, 3)
 
     # the GPU pool is sized for the fully resident baseline run as well (every unit + 3 layers of staging)
-    ramp = max(args.warmup, 48)
+    ramp = max(args.warmup, args.ramp)
     total_steps = 1 + 3 + 3 + args.steps + ramp + args.steps + 3 + args.steps   # every phase below appends one token per step
     n_host_blocks = int(round(wl.host_frac * (int(((wl.ctx_lens.astype(np.int64) + total_steps + 15) // 16).sum()))))
     dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,

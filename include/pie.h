@@ -71,11 +71,11 @@ typedef struct pie_pool_config {
     void *copy_in_stream;
     void *copy_out_stream;
     int32_t own_streams;       /* 1: the library creates three non-blocking streams */
-    int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (256) */
+    int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (512) */
     int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
     int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
     int32_t timing;            /* 1: record per-layer events for pie_controller_tick / pie_get_stats */
-    int32_t reserved[7];
+    int32_t reserved[7];       /* [0]: attention kernel variant for tuning (0 = default); rest 0 */
 } pie_pool_config;
 
 typedef struct pie_stats {
@@ -227,11 +227,12 @@ int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps);
  *   stream      a cudaStream_t
  * The split-K scratch (chunk offsets, fp32 partials) is a static device array of PIE_NOALLOC_SCRATCH_BYTES
  * that every GPU loading the library holds until the process exits.  A call whose partials would not fit
- * (sum over sequences of ceil(ctx / split_tokens), times n_q_heads * (head_dim + 2) * 4 bytes, plus 17 KiB)
+ * (sum over sequences of ceil(ctx / split_tokens), times n_q_heads * (head_dim + 2) * 4 bytes, plus
+ * 4 * n_seqs * n_kv_heads bytes of counters and 17 KiB)
  * or with more than PIE_NOALLOC_MAX_SEQS sequences returns PIE_ERR_NOMEM and enqueues nothing.
- * All calls on a device share that array and it keeps the previous call's contents: every word a call reads
- * it has written first, so nothing needs clearing, but two calls that overlap on the GPU (different
- * streams, no dependency) race - order them.  The first call on each device looks up the array's device
+ * All calls on a device share that array and it keeps the previous call's contents: each call clears the
+ * counters it needs at zero (a memset on `stream`) and writes every other word before reading it; two calls
+ * that overlap on the GPU (different streams, no dependency) race - order them.  The first call on each device looks up the array's device
  * address (cudaGetSymbolAddress) and sets the kernels' shared-memory attribute; make that first call outside
  * any stream capture.  Calls cudaMalloc, cudaFree or any allocating routine: never. */
 int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots, const int32_t *slot_table,

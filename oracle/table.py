@@ -19,10 +19,12 @@ overwritten before the copy reading it has finished, and a unit's bytes are neve
 destination before the copy writing them has finished.
 
 Slot hand-out order (shared rule, so that two implementations can be compared slot by slot):
-``ready`` is a stack that starts as n-1 .. 0 (slot 0 on top); ``pending`` is a queue of released
-slots still waiting for their ticket.  At the start of every call pending slots whose ticket is
-confirmed move to ``ready`` in queue order.  Allocation pops ``ready`` first, then takes
-``pending`` from the front and reports the tickets to wait for.
+``ready`` is a queue that starts as 0 .. n-1; ``pending`` is a queue of released slots still
+waiting for their ticket.  At the start of every call pending slots whose ticket is confirmed
+move to the back of ``ready`` in queue order.  Allocation takes from the front of ``ready``
+first, then from the front of ``pending`` and reports the tickets to wait for.  (First in, first
+out on both keeps slots that were released together next to each other when they are handed out
+again, so lists of swapped blocks stay long runs of consecutive slots.)
 """
 from __future__ import annotations
 
@@ -41,7 +43,7 @@ Q_NONE, Q_IN, Q_OUT, Q_COMPUTE = 0, 1, 2, 3
 
 class _SlotPool:
     def __init__(self, n):
-        self.ready = list(range(n - 1, -1, -1))
+        self.ready = list(range(n))
         self.pending = []  # (slot, queue, ticket)
 
     def settle(self, done):
@@ -61,7 +63,7 @@ class _SlotPool:
         slots, waits, tags = [], {}, []
         for _ in range(n):
             if self.ready:
-                slots.append(self.ready.pop())
+                slots.append(self.ready.pop(0))
                 tags.append((Q_NONE, 0))
             else:
                 slot, qu, tk = self.pending.pop(0)

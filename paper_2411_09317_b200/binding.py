@@ -151,6 +151,7 @@ def pie_pool_create(**kw) -> int:
     kw.setdefault("block_tokens", 16)
     kw.setdefault("own_streams", 1)
     kw.setdefault("max_seqs", 256)
+    cfg.reserved[0] = kw.pop("attn_variant", 0)
     for k, v in kw.items():
         setattr(cfg, k, v)
     out = _vp()

@@ -230,131 +230,229 @@ plan_kernel(const int32_t *__restrict__ ctx_lens, int32_t n_seqs, int32_t max_to
 }
 
 // =====================================================================================================
-// KV append (Section 3.2: each token iteration updates each layer's cache): K and V rows of the new token
-// go to position ctx_len-1 of the sequence's tail block.  grid (S, Hkv), block 2 * D/8 threads.
-// =====================================================================================================
-__global__ void append_kernel(uint4 *__restrict__ pool, const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-                              const int32_t *__restrict__ block_table, int32_t max_blocks,
-                              const int32_t *__restrict__ ctx_lens, const int32_t *__restrict__ slot_table,
-                              int32_t n_kv_heads, int32_t head_dim, int32_t n_logical, int64_t n_gpu_slots,
-                              int32_t *status) {
-    const int s = blockIdx.x, kvh = blockIdx.y;
-    const int vecs = head_dim / 8;
-    const int kv = threadIdx.x / vecs, v = threadIdx.x % vecs;
-    int32_t pos = ctx_lens[s] - 1;
-    if (pos < 0) return;
-    if (pos >= max_blocks * 16) return;  // flagged by the plan kernel
-    const int32_t blk = block_table[(int64_t)s * max_blocks + pos / 16];
-    int32_t slot = (blk >= 0 && blk < n_logical) ? slot_table[blk] : -1;
-    if (slot < 0 || slot >= n_gpu_slots) {
-        if (threadIdx.x == 0) raise_status(status, STATUS_MISSING_UNIT);
-        return;
-    }
-    const uint4 *src = (kv == 0 ? k_new : v_new) + ((int64_t)s * n_kv_heads + kvh) * vecs + v;
-    uint4 *dst = pool + ((((int64_t)slot * n_kv_heads + kvh) * 2 + kv) * 16 + (pos & 15)) * vecs + v;
-    *dst = *src;
-}
-
-// =====================================================================================================
-// Paged decode attention, split-K.
+// Paged decode attention, split-K, one kernel per layer call.
 //
-// Work item = (sequence, KV head, chunk of `split_tokens` tokens); items are dealt round-robin to a
-// persistent grid.  Per item a CTA streams the chunk's 16-token tiles (K rows 0-15 and V rows 16-31 of
-// one head: one contiguous 2*16*D*2-byte piece of the slot) through a ring of shared-memory stages:
-//   - warp NW (producer): resolves block_table -> slot table -> slot for 32 tiles at a time and issues
-//     one TMA tile copy per stage (128-byte swizzle), completion on the stage's "full" mbarrier;
-//   - warps 0..NW-1 (consumers): tile i of an item goes to warp i % NW.  The KV tokens sit on the M axis
-//     of mma.m16n8k16 and the (up to 8) query heads of the KV head's group on the N axis, so a tile costs
-//     D/16 MMAs for S^T = K q^T and D/16 for O^T += V^T P^T whatever the group size.  Online softmax in
-//     fp32 per warp; P^T reaches the B-operand layout with two movmatrix transposes.
-// The NW per-warp partials are merged in warp order through shared memory and written as one fp32 partial
-// (m, l, unnormalised acc) per item; combine_kernel merges a sequence's chunks in chunk order.  Every
-// reduction order depends only on the logical token order and on ctx_len, never on slot ids or timing, so
-// a run with swapped blocks reproduces a resident run bit for bit.
+// Work item = (sequence, KV head, chunk of `split_tokens` tokens).  A persistent grid pulls items from a
+// global counter (so an SM that is slowed down, e.g. by a co-resident copy kernel, simply takes fewer).
+// Per item a CTA streams the chunk's 16-token tiles (K rows 0-15 and V rows 16-31 of one head: one
+// contiguous 2*16*D*2-byte piece of the slot) through a ring of shared-memory stages:
+//   - warp NW (producer): fetches the next item, publishes it to the consumers through a small queue,
+//     resolves block_table -> slot table -> slot for 32 tiles at a time and issues one TMA tile copy per
+//     stage (128-byte swizzle), completion on the stage's "full" mbarrier;
+//   - warps 0..NW-1 (consumers): tile i of an item goes to warp i % NW.  The KV tokens sit on the M axis of
+//     mma.m16n8k16 and the (up to 8) query heads of the KV head's group on the N axis, so a tile costs D/16
+//     MMAs for S^T = K q^T and D/16 for O^T += V^T P^T whatever the group size.  Online softmax in fp32
+//     per warp; P^T reaches the B-operand layout with two movmatrix transposes.
+// Fused into the same kernel:
+//   - the split-K plan: every CTA builds the chunk offsets of the batch in shared memory (exclusive scan of
+//     ceil(ctx / split) over the sequences);
+//   - the KV append (Section 3.2: each token iteration updates each layer's cache): the warp that owns the
+//     tile holding position ctx-1 patches the new token's K and V rows into the staged tile and into the pool;
+//   - the combine: a sequence with one chunk is normalised and written directly; otherwise each item writes
+//     an fp32 partial (m, l, unnormalised acc) and the CTA that completes a (sequence, KV head) last merges
+//     its chunks in chunk order with the log-sum-exp rule, normalises and rounds to 16 bits (nearest even).
+// Every reduction order depends only on the logical token order and on ctx_len (tile -> warp by index, warps
+// merged in warp order, chunks merged in chunk order), never on slot ids, on which CTA ran an item or on
+// timing, so a run with swapped blocks reproduces a resident run bit for bit.
+// All waits are bounded: a wait that runs out raises a status word and the CTA leaves through its barriers.
 // =====================================================================================================
-constexpr int ATT_NW = 4;
-constexpr int ATT_THREADS = (ATT_NW + 1) * 32;
-constexpr int ATT_STAGES = 8;
+constexpr int ATT_QD = 2;           // depth of the producer -> consumer item queue (item id + its query rows)
+constexpr int ATT_SMEM_SEQS = 1024; // largest batch whose chunk offsets are built in shared memory
 
 struct AttnParams {
     const uint16_t *q;
+    uint16_t *out;
     const int32_t *block_table;
     const int32_t *ctx_lens;
     const int32_t *slot_table;
-    const int32_t *chunk_off;
+    const int32_t *chunk_off_global;  // used when n_seqs > ATT_SMEM_SEQS (filled by plan_kernel)
+    const uint4 *k_new, *v_new;       // optional append
+    uint4 *pool;
     float *part_o;
     float *part_ml;
+    int32_t *counters;  // [0] next item, [1] CTAs that have left, [64 + s * Hkv + kvh] chunks done
     int32_t *status;
     int64_t n_gpu_slots;
-    int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d;
+    int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d, max_chunks;
     float scale_log2e;
 };
 
-template <int D>
+template <int D, int STAGES, int NW>
 struct AttnSmem {
     static constexpr int TILE_BYTES = 2 * 16 * D * 2;
     static constexpr int HALF_BYTES = 32 * 128;  // 32 rows x 128 bytes
     static constexpr int MO_STRIDE = D + 4;      // floats per (warp, head) row; +4 keeps the scatter conflict-free
-    static constexpr int OFF_MO = ATT_STAGES * TILE_BYTES;
-    static constexpr int OFF_ML = OFF_MO + ATT_NW * 8 * MO_STRIDE * 4;
-    static constexpr int OFF_BAR = OFF_ML + ATT_NW * 8 * 2 * 4;
-    static constexpr int OFF_ABORT = OFF_BAR + 2 * ATT_STAGES * 8;
-    static constexpr int BYTES = OFF_ABORT + 16;
+    static constexpr int Q_BYTES = 8 * D * 2;    // query rows of one item (up to 8 heads)
+    static constexpr int OFF_Q = STAGES * TILE_BYTES;
+    static constexpr int OFF_MO = OFF_Q + ATT_QD * Q_BYTES;
+    static constexpr int OFF_ML = OFF_MO + NW * 8 * MO_STRIDE * 4;
+    static constexpr int OFF_BAR = OFF_ML + NW * 8 * 2 * 4;              // full[STAGES], empty[STAGES], qfull[QD], qempty[QD]
+    static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 2 * ATT_QD) * 8;  // abort, is_last, q_item[QD]
+    static constexpr int OFF_CO = OFF_MISC + 64;                          // chunk offsets [ATT_SMEM_SEQS + 1]
+    static constexpr int BYTES = OFF_CO + (ATT_SMEM_SEQS + 1) * 4 + 12;
 };
 
 struct ItemInfo {
-    int32_t s, kvh, t0, t1, ntiles;
+    int32_t s, kvh, ctx, t0, t1, ntiles, nchunks, chunk0;
 };
 
-__device__ __forceinline__ ItemInfo decode_item(const AttnParams &p, int32_t item) {
+__device__ __forceinline__ ItemInfo decode_item(const AttnParams &p, const int32_t *co, int32_t item) {
     ItemInfo it;
     const int32_t ci = item / p.n_kv_heads;
     it.kvh = item - ci * p.n_kv_heads;
-    int32_t lo = 0, hi = p.n_seqs;  // largest s with chunk_off[s] <= ci
+    int32_t lo = 0, hi = p.n_seqs;  // largest s with co[s] <= ci
     while (hi - lo > 1) {
         const int32_t mid = (lo + hi) >> 1;
-        if (__ldg(p.chunk_off + mid) <= ci) lo = mid;
+        if (co[mid] <= ci) lo = mid;
         else hi = mid;
     }
     it.s = lo;
-    const int32_t c = ci - __ldg(p.chunk_off + lo);
-    int32_t ctx = __ldg(p.ctx_lens + lo);
-    ctx = min(ctx, p.max_blocks * 16);
+    it.chunk0 = co[lo];
+    it.nchunks = co[lo + 1] - it.chunk0;
+    const int32_t c = ci - it.chunk0;
+    it.ctx = min(__ldg(p.ctx_lens + lo), p.max_blocks * 16);
     it.t0 = c * p.split_tokens;
-    it.t1 = min(ctx, it.t0 + p.split_tokens);
+    it.t1 = min(it.ctx, it.t0 + p.split_tokens);
     it.ntiles = (it.t1 - it.t0 + 15) >> 4;
     return it;
 }
 
-template <int D, bool BF16>
-__global__ void __launch_bounds__(ATT_THREADS)
+// barrier over the consumer warps that also ORs a predicate: every consumer thread gets the same answer
+template <int NTHREADS>
+__device__ __forceinline__ bool consumer_vote(bool pred) {
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(any)
+        : "r"((uint32_t)pred), "n"(NTHREADS)
+        : "memory");
+    return any != 0;
+}
+template <int NTHREADS>
+__device__ __forceinline__ void consumer_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+template <int D, bool BF16, int STAGES, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p) {
-    using SM = AttnSmem<D>;
+    using SM = AttnSmem<D, STAGES, NW>;
+    // A stage must always be consumed by the same warp: tile i goes to warp i % NW and to stage i % STAGES.  If two
+    // warps alternated on a stage, the one running ahead could pass a parity wait on the phase before the one it
+    // needs (an mbarrier waiter may be at most one phase ahead).
+    static_assert(STAGES % NW == 0, "ring stages must be a multiple of the consumer warps");
+    constexpr int ATT_NW = NW;
+    constexpr int ATT_THREADS = (NW + 1) * 32;
+    constexpr int NCONS = NW * 32;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t bar_full = smem_base + SM::OFF_BAR;
-    const uint32_t bar_empty = bar_full + ATT_STAGES * 8;
-    volatile int32_t *abort_flag = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_ABORT);
+    const uint32_t bar_empty = bar_full + STAGES * 8;
+    const uint32_t bar_qfull = bar_empty + STAGES * 8;
+    const uint32_t bar_qempty = bar_qfull + ATT_QD * 8;
+    volatile int32_t *misc = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_MISC);
+    volatile int32_t *abort_flag = misc;      // [0]
+    volatile int32_t *is_last = misc + 1;     // [1]
+    volatile int32_t *q_item = misc + 4;      // [4 .. 4 + QD)
+    int32_t *co_smem = reinterpret_cast<int32_t *>(smem + SM::OFF_CO);
 
     if (tid == 0) {
-        for (int s = 0; s < ATT_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int s = 0; s < ATT_QD; ++s) {
+            mbar_init(bar_qfull + 8 * s, 1);
+            mbar_init(bar_qempty + 8 * s, ATT_NW);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // ---- plan: chunk offsets of the batch (exclusive scan of the per-sequence chunk counts)
+    const bool co_in_smem = p.n_seqs <= ATT_SMEM_SEQS;
+    if (co_in_smem) {
+        for (int32_t s = tid; s < p.n_seqs; s += ATT_THREADS) {
+            int32_t ctx = __ldg(p.ctx_lens + s);
+            if (ctx > p.max_blocks * 16) {
+                ctx = p.max_blocks * 16;
+                if (blockIdx.x == 0) raise_status(p.status, STATUS_CTX_TOO_LONG);
+            }
+            co_smem[s + 1] = ctx > 0 ? (ctx + p.split_tokens - 1) / p.split_tokens : 0;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            int32_t carry = 0;
+            for (int32_t base = 0; base < p.n_seqs; base += 32) {
+                const int32_t s = base + lane;
+                const int32_t v = s < p.n_seqs ? co_smem[s + 1] : 0;
+                int32_t x = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int32_t y = __shfl_up_sync(0xffffffffu, x, o);
+                    if (lane >= o) x += y;
+                }
+                if (s < p.n_seqs) co_smem[s + 1] = carry + x;
+                carry += __shfl_sync(0xffffffffu, x, 31);
+            }
+            if (lane == 0) co_smem[0] = 0;
+        }
+    }
     __syncthreads();
-
-    const int32_t n_items = __ldg(p.chunk_off + p.n_seqs) * p.n_kv_heads;
+    const int32_t *co = co_in_smem ? co_smem : p.chunk_off_global;
+    int32_t n_chunks_total = co[p.n_seqs];
+    if (n_chunks_total > p.max_chunks) {  // more chunks than the partials buffer holds: compute nothing, flag it
+        if (blockIdx.x == 0 && tid == 0) raise_status(p.status, STATUS_CTX_TOO_LONG);
+        n_chunks_total = 0;
+    }
+    const int32_t n_items = n_chunks_total * p.n_kv_heads;
     uint32_t gt = 0;  // tiles this CTA has streamed so far (same count in producer and consumers)
+    uint32_t qn = 0;  // items this CTA has taken so far
 
     if (warp == ATT_NW) {
         // ------------------------------------------------------------------ producer warp
-        for (int32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-            const ItemInfo it = decode_item(p, item);
+        int32_t next = lane == 0 ? atomicAdd(p.counters, 1) : 0;
+        for (;;) {
+            int32_t item = -1;
+            if (lane == 0) {
+                const uint32_t qs = qn % ATT_QD;
+                if (!mbar_wait(bar_qempty + 8 * qs, ((qn / ATT_QD) & 1u) ^ 1u)) {
+                    raise_status(p.status, STATUS_WAIT_TIMEOUT);
+                    *abort_flag = 1;
+                }
+                if (*abort_flag == 0 && next < n_items) item = next;
+                q_item[qs] = item;
+                if (item >= 0) {
+                    // the item's query rows travel with its id: one bulk copy that completes on the same barrier
+                    const int32_t ci = item / p.n_kv_heads, kvh = item - ci * p.n_kv_heads;
+                    int32_t lo = 0, hi = p.n_seqs;
+                    while (hi - lo > 1) {
+                        const int32_t mid = (lo + hi) >> 1;
+                        if (co[mid] <= ci) lo = mid;
+                        else hi = mid;
+                    }
+                    const uint32_t bytes = (uint32_t)p.group * D * 2;
+                    mbar_expect_tx(bar_qfull + 8 * qs, bytes);
+                    bulk_load(smem_base + SM::OFF_Q + qs * SM::Q_BYTES,
+                              p.q + ((int64_t)lo * p.n_q_heads + (int64_t)kvh * p.group) * D, bytes, bar_qfull + 8 * qs);
+                    next = atomicAdd(p.counters, 1);  // the next item's id: its latency hides behind this item's tiles
+                } else {
+                    mbar_arrive(bar_qfull + 8 * qs);
+                }
+            }
+            item = __shfl_sync(0xffffffffu, item, 0);
+            ++qn;
+            if (item < 0) break;
+            const ItemInfo it = decode_item(p, co, item);
             const int32_t *bt = p.block_table + (int64_t)it.s * p.max_blocks + (it.t0 >> 4);
             for (int32_t base = 0; base < it.ntiles; base += 32) {
                 int32_t slot = -1;
@@ -367,8 +465,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 for (int32_t j = 0; j < cnt; ++j, ++gt) {
                     int32_t sl = __shfl_sync(0xffffffffu, slot, j);
                     if (lane == 0) {
-                        const uint32_t stage = gt % ATT_STAGES;
-                        const uint32_t phase = (gt / ATT_STAGES) & 1u;
+                        const uint32_t stage = gt % STAGES;
+                        const uint32_t phase = (gt / STAGES) & 1u;
                         if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u)) {
                             raise_status(p.status, STATUS_WAIT_TIMEOUT);
                             *abort_flag = 1;
@@ -391,7 +489,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                             }
                         }
                     }
-                    if (__shfl_sync(0xffffffffu, (int)*abort_flag, 0)) return;
+                    if (__shfl_sync(0xffffffffu, (int)*abort_flag, 0)) {
+                        // give the copies still in flight a bounded time to land before the CTA's memory goes away
+                        if (lane == 0) {
+                            const uint32_t first = gt > (uint32_t)STAGES ? gt - STAGES : 0u;
+                            for (uint32_t t = first; t < gt; ++t) mbar_wait(bar_full + 8 * (t % STAGES), (t / STAGES) & 1u);
+                        }
+                        return;
+                    }
                 }
             }
         }
@@ -408,18 +513,65 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const int k_tok = lr + (lm & 1) * 8, k_csel = lm >> 1;   // K: matrices {tok 0-7, tok 8-15} x {chunk, chunk+1}
     const int v_tok = lr + (lm >> 1) * 8, v_csel = lm & 1;   // V (transposed): {chunk, chunk+1} x {tok 0-7, tok 8-15}
 
-    for (int32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const ItemInfo it = decode_item(p, item);
+    // sequences without any token get a zero row (nobody else writes them)
+    if (blockIdx.x == 0)
+        for (int32_t s = 0; s < p.n_seqs; ++s)
+            if (co[s + 1] == co[s] || n_items == 0)
+                for (int e = tid; e < p.n_q_heads * D; e += ATT_NW * 32) p.out[(int64_t)s * p.n_q_heads * D + e] = 0;
+
+    // Completion of a (sequence, KV head) is signalled one item late: thread 0 bumps the pair's counter after an
+    // item's last barrier and looks at the answer only when the next item has been computed, so nobody waits
+    // for the atomic's round trip.  prev_* describe the item whose answer is still outstanding.
+    int32_t prev_s = -1, prev_kvh = 0, prev_nchunks = 0, prev_chunk0 = 0, prev_old = 0;
+
+    // merge the chunks of (s, kvh) in chunk order, normalise, round (run by the CTA that completed the pair)
+    auto final_combine = [&](int32_t cs, int32_t ckvh, int32_t nchunks, int32_t chunk0) {
+        const int64_t row0 = ((int64_t)cs * p.n_q_heads + (int64_t)ckvh * p.group) * D;
+        for (int e = tid; e < p.group * D; e += ATT_NW * 32) {
+            const int g = e / D, d = e - g * D;
+            float mm = -INFINITY;
+            for (int32_t c = 0; c < nchunks; ++c)
+                mm = fmaxf(mm, __ldcg(p.part_ml + (((int64_t)(chunk0 + c) * p.n_kv_heads + ckvh) * p.group + g) * 2));
+            float acc = 0.f, ll = 0.f;
+            for (int32_t c = 0; c < nchunks; ++c) {
+                const int64_t idx = ((int64_t)(chunk0 + c) * p.n_kv_heads + ckvh) * p.group + g;
+                const float mc = __ldcg(p.part_ml + idx * 2);
+                const float wt = mc == -INFINITY ? 0.f : fast_exp2(mc - mm);
+                ll += __ldcg(p.part_ml + idx * 2 + 1) * wt;
+                acc += __ldcg(p.part_o + idx * D + d) * wt;
+            }
+            const float r = acc * (ll > 0.f ? 1.f / ll : 0.f);
+            p.out[row0 + e] = BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(r)) : __half_as_ushort(__float2half_rn(r));
+        }
+    };
+    auto publish_prev = [&]() {  // thread 0: was this CTA the last to finish the previous item's pair?
+        int32_t last = 0;
+        if (prev_s >= 0 && prev_nchunks > 1 && prev_old == prev_nchunks - 1) {
+            last = 1;
+            p.counters[64 + prev_s * p.n_kv_heads + prev_kvh] = 0;  // ready for the next launch
+        }
+        *is_last = last;
+    };
+
+    for (;;) {
+        const uint32_t qs = qn % ATT_QD;
+        const bool late = !mbar_wait(bar_qfull + 8 * qs, (qn / ATT_QD) & 1u);
+        if (consumer_vote<NCONS>(late || *abort_flag != 0)) {  // uniform: either every consumer goes on or none does
+            if (late) raise_status(p.status, STATUS_WAIT_TIMEOUT);
+            break;
+        }
+        const int32_t item = q_item[qs];
+        if (item < 0) break;  // end marker: all consumers read the same queue entry
+        const ItemInfo it = decode_item(p, co, item);
         // q as the B operand of S^T = K q^T: b0 = q[g][16 ks + c2 .. +1], b1 = q[g][16 ks + 8 + c2 .. +1], g = lane / 4
         uint32_t bq[D / 16][2];
         {
             const int g = lane >> 2;
-            const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
-                p.q + ((int64_t)it.s * p.n_q_heads + (int64_t)it.kvh * p.group + g) * D);
+            const uint32_t *qrow = reinterpret_cast<const uint32_t *>(smem + SM::OFF_Q + qs * SM::Q_BYTES) + g * (D / 2);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                bq[ks][0] = g < p.group ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
-                bq[ks][1] = g < p.group ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+                bq[ks][0] = g < p.group ? qrow[ks * 8 + (lane & 3)] : 0u;
+                bq[ks][1] = g < p.group ? qrow[ks * 8 + 4 + (lane & 3)] : 0u;
             }
         }
         float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
@@ -429,8 +581,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
         for (int32_t i = warp; i < it.ntiles; i += ATT_NW) {
             const uint32_t tg = gt + (uint32_t)i;
-            const uint32_t stage = tg % ATT_STAGES;
-            const uint32_t phase = (tg / ATT_STAGES) & 1u;
+            const uint32_t stage = tg % STAGES;
+            const uint32_t phase = (tg / STAGES) & 1u;
             if (!mbar_wait(bar_full + 8 * stage, phase)) {
                 raise_status(p.status, STATUS_WAIT_TIMEOUT);
                 *abort_flag = 1;
@@ -440,6 +592,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             uint8_t *tile = smem + stage * SM::TILE_BYTES;
             const uint32_t tile_u32 = smem_base + stage * SM::TILE_BYTES;
             const int nvalid = min(16, it.t1 - (it.t0 + 16 * i));
+            bool touched = false;
             if (nvalid < 16) {
                 // masked tokens are excluded, not multiplied by zero: clear their V rows so that 0 * garbage
                 // (possibly NaN/Inf) never enters the PV product.  A row is 128 contiguous bytes per half.
@@ -450,8 +603,29 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     *reinterpret_cast<uint4 *>(tile + (rem >> 3) * SM::HALF_BYTES + row * 128 + (rem & 7) * 16) =
                         make_uint4(0, 0, 0, 0);
                 }
-                __syncwarp();
+                touched = true;
             }
+            if (p.k_new != nullptr && it.t1 == it.ctx && i == it.ntiles - 1) {
+                // append: this tile holds position ctx-1; put the new token's K and V rows into the staged tile
+                // (lanes 0-15: K, lanes 16-31: V, one 16-byte piece each) and into the pool
+                const int32_t pos = it.ctx - 1, r = pos & 15;
+                int32_t slot = -1;
+                if (lane == 0) {
+                    const int32_t blk = __ldg(p.block_table + (int64_t)it.s * p.max_blocks + (pos >> 4));
+                    if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
+                    if (slot >= p.n_gpu_slots) slot = -1;
+                }
+                slot = __shfl_sync(0xffffffffu, slot, 0);
+                const int kv = lane >> 4, c = lane & 15;
+                if (c < D / 8) {
+                    const uint4 val = __ldg((kv ? p.v_new : p.k_new) + ((int64_t)it.s * p.n_kv_heads + it.kvh) * (D / 8) + c);
+                    *reinterpret_cast<uint4 *>(tile + (c >> 3) * SM::HALF_BYTES + (kv * 16 + r) * 128 + (((c & 7) ^ (r & 7)) << 4)) = val;
+                    if (slot >= 0)
+                        p.pool[((((int64_t)slot * p.n_kv_heads + it.kvh) * 2 + kv) * 16 + r) * (D / 8) + c] = val;
+                }
+                touched = true;
+            }
+            if (touched) __syncwarp();
             // ---- S^T[16 tokens][8 heads] = K[16][D] . q^T[D][8]
             float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -508,7 +682,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
             }
             __syncwarp();
-            if (nvalid < 16) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
         }
         gt += (uint32_t)it.ntiles;
@@ -535,7 +709,9 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 ml[(warp * 8 + c2 + 1) * 2 + 1] = l1;
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(ATT_NW * 32) : "memory");
+        if (tid == 0) publish_prev();
+        consumer_sync<NCONS>();
+        const int64_t out_row0 = ((int64_t)it.s * p.n_q_heads + (int64_t)it.kvh * p.group) * D;
         for (int e = tid; e < p.group * D; e += ATT_NW * 32) {
             const int g = e / D, d = e - g * D;
             float mm = -INFINITY;
@@ -549,62 +725,50 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 acc += mo[(w * 8 + g) * SM::MO_STRIDE + d] * wt;
                 ll += ml[(w * 8 + g) * 2 + 1] * wt;
             }
-            p.part_o[((int64_t)item * p.group + g) * D + d] = acc;
-            if (d == 0) {
-                p.part_ml[((int64_t)item * p.group + g) * 2 + 0] = mm;
-                p.part_ml[((int64_t)item * p.group + g) * 2 + 1] = ll;
+            if (it.nchunks == 1) {
+                // the whole context in one chunk: normalise and round here
+                const float r = acc * (ll > 0.f ? 1.f / ll : 0.f);
+                p.out[out_row0 + e] = BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(r)) : __half_as_ushort(__float2half_rn(r));
+            } else {
+                p.part_o[((int64_t)item * p.group + g) * D + d] = acc;
+                if (d == 0) {
+                    p.part_ml[((int64_t)item * p.group + g) * 2 + 0] = mm;
+                    p.part_ml[((int64_t)item * p.group + g) * 2 + 1] = ll;
+                }
             }
         }
-        // second barrier (partials buffer free again) doubles as a uniform vote on the abort flag
-        uint32_t any_abort;
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\t"
-            "setp.ne.u32 q, %1, 0;\n\t"
-            "bar.red.or.pred p, 1, %2, q;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(any_abort)
-            : "r"((uint32_t)*abort_flag), "n"(ATT_NW * 32)
-            : "memory");
-        if (any_abort) return;
+        if (*is_last) final_combine(prev_s, prev_kvh, prev_nchunks, prev_chunk0);  // the previous item's pair is complete
+        // last barrier of the item (partials buffer free again) doubles as a uniform vote on the abort flag
+        if (consumer_vote<NCONS>(*abort_flag != 0)) {
+            prev_s = -1;
+            break;
+        }
+        // every thread's partial stores precede the barrier above; a release by thread 0 after it covers them all
+        if (tid == 0 && it.nchunks > 1)
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                         : "=r"(prev_old)
+                         : "l"(p.counters + 64 + it.s * p.n_kv_heads + it.kvh)
+                         : "memory");
+        prev_s = it.s;
+        prev_kvh = it.kvh;
+        prev_nchunks = it.nchunks;
+        prev_chunk0 = it.chunk0;
+        if (lane == 0) mbar_arrive(bar_qempty + 8 * qs);
+        ++qn;
     }
-}
-
-// =====================================================================================================
-// Combine: one warp per (sequence, query head) merges that sequence's chunk partials in chunk order with the
-// log-sum-exp rule, normalises and rounds to the 16-bit output type (nearest even).  No chunk -> zeros.
-// =====================================================================================================
-template <int D, bool BF16>
-__global__ void __launch_bounds__(128)
-combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, const int32_t *__restrict__ chunk_off,
-               uint16_t *__restrict__ out, int32_t n_seqs, int32_t n_q_heads, int32_t n_kv_heads, int32_t group) {
-    constexpr int EPL = D / 32;  // elements per lane
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (row >= (int64_t)n_seqs * n_q_heads) return;
-    const int32_t s = (int32_t)(row / n_q_heads), h = (int32_t)(row % n_q_heads);
-    const int32_t kvh = h / group, g = h % group;
-    const int32_t c0 = chunk_off[s], c1 = chunk_off[s + 1];
-    float mm = -INFINITY;
-    for (int32_t c = c0; c < c1; ++c) mm = fmaxf(mm, part_ml[(((int64_t)c * n_kv_heads + kvh) * group + g) * 2]);
-    float acc[EPL];
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    float ll = 0.f;
-    for (int32_t c = c0; c < c1; ++c) {
-        const int64_t idx = ((int64_t)c * n_kv_heads + kvh) * group + g;
-        const float mc = part_ml[idx * 2];
-        const float wt = mc == -INFINITY ? 0.f : fast_exp2(mc - mm);
-        ll += part_ml[idx * 2 + 1] * wt;
-        const float *po = part_o + idx * D + lane * EPL;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) acc[e] += po[e] * wt;
+    // the answer for the last item is still outstanding
+    if (prev_s >= 0 && prev_nchunks > 1) {
+        if (tid == 0) publish_prev();
+        consumer_sync<NCONS>();
+        if (*is_last) final_combine(prev_s, prev_kvh, prev_nchunks, prev_chunk0);
     }
-    const float inv = ll > 0.f ? 1.f / ll : 0.f;
-    uint16_t *dst = out + row * D + lane * EPL;
-#pragma unroll
-    for (int e = 0; e < EPL; e += 2) {
-        const uint32_t v = pack2<BF16>(acc[e] * inv, acc[e + 1] * inv);
-        *reinterpret_cast<uint32_t *>(dst + e) = v;
+    // the last CTA to leave resets the work counter for the next launch (every CTA has drawn its end marker by then)
+    if (tid == 0) {
+        const int32_t old = atomicAdd(p.counters + 1, 1);
+        if (old == (int32_t)gridDim.x - 1) {
+            p.counters[0] = 0;
+            p.counters[1] = 0;
+        }
     }
 }
 
@@ -649,33 +813,90 @@ cudaError_t make_pool_tensor_maps(void *gpu_pool, int64_t n_gpu_slots, int n_kv_
     return cudaSuccess;
 }
 
-int attn_smem_bytes(int head_dim) { return head_dim == 128 ? AttnSmem<128>::BYTES : AttnSmem<64>::BYTES; }
+// Kernel variants (consumer warps, ring stages): more stages keep more bytes in flight per CTA, fewer let a third
+// CTA share the SM.  Variant 0 is the default.
+struct AttnVariant {
+    int nw, stages;
+};
+static const AttnVariant kVariants[] = {{2, 4}, {4, 8}, {2, 12}, {2, 6}, {4, 4}, {2, 8}, {1, 5}, {3, 6}, {1, 7}, {2, 4}, {1, 4}, {3, 3}, {1, 3}, {2, 2}};
+constexpr int kNumVariants = (int)(sizeof(kVariants) / sizeof(kVariants[0]));
 
-template <int D, bool BF16>
-static cudaError_t configure_one(int *ctas_per_sm) {
-    cudaError_t e = cudaFuncSetAttribute(paged_decode_attn_kernel<D, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         AttnSmem<D>::BYTES);
-    if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, paged_decode_attn_kernel<D, BF16>, ATT_THREADS,
-                                                         AttnSmem<D>::BYTES);
+template <typename F>
+static cudaError_t dispatch_variant(int head_dim, int dtype, int variant, F &&f) {
+    if (variant < 0 || variant >= kNumVariants) return cudaErrorInvalidValue;
+#define PIE_VARIANT(NWV, STV)                                                                       \
+    if (kVariants[variant].nw == NWV && kVariants[variant].stages == STV) {                         \
+        if (head_dim == 128) return dtype == PIE_BF16 ? f(paged_decode_attn_kernel<128, true, STV, NWV>, AttnSmem<128, STV, NWV>::BYTES, NWV) \
+                                                      : f(paged_decode_attn_kernel<128, false, STV, NWV>, AttnSmem<128, STV, NWV>::BYTES, NWV); \
+        return dtype == PIE_BF16 ? f(paged_decode_attn_kernel<64, true, STV, NWV>, AttnSmem<64, STV, NWV>::BYTES, NWV)   \
+                                 : f(paged_decode_attn_kernel<64, false, STV, NWV>, AttnSmem<64, STV, NWV>::BYTES, NWV); \
+    }
+    PIE_VARIANT(2, 12)
+    PIE_VARIANT(4, 8)
+    PIE_VARIANT(2, 6)
+    PIE_VARIANT(4, 4)
+    PIE_VARIANT(2, 8)
+    PIE_VARIANT(1, 5)
+    PIE_VARIANT(3, 6)
+    PIE_VARIANT(1, 7)
+    PIE_VARIANT(2, 4)
+    PIE_VARIANT(1, 4)
+    PIE_VARIANT(3, 3)
+    PIE_VARIANT(1, 3)
+    PIE_VARIANT(2, 2)
+#undef PIE_VARIANT
+    return cudaErrorInvalidValue;
 }
 
-cudaError_t attn_configure(int head_dim, int dtype, int *ctas_per_sm) {
-    if (head_dim == 128) return dtype == PIE_BF16 ? configure_one<128, true>(ctas_per_sm) : configure_one<128, false>(ctas_per_sm);
-    return dtype == PIE_BF16 ? configure_one<64, true>(ctas_per_sm) : configure_one<64, false>(ctas_per_sm);
+int attn_smem_bytes(int head_dim) { return head_dim == 128 ? AttnSmem<128, 4, 2>::BYTES : AttnSmem<64, 4, 2>::BYTES; }
+
+// The attention kernel needs the SM's largest shared-memory carve-out.  An SM cannot change its carve-out while
+// any CTA is resident, so every other kernel of the path asks for the same one: otherwise a small kernel that
+// lands on an idle SM first could keep attention CTAs off that SM until it has finished.
+static cudaError_t prefer_max_shared() {
+    const void *fns[] = {(const void *)swap_kernel, (const void *)patch_kernel, (const void *)patch_from_list_kernel,
+                         (const void *)plan_kernel};
+    for (const void *f : fns) {
+        cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
-template <int D, bool BF16>
-static cudaError_t launch_one(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
-                              int use3d, cudaStream_t stream) {
+cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_sm) {
+    cudaError_t e0 = prefer_max_shared();
+    if (e0 != cudaSuccess) return e0;
+    return dispatch_variant(head_dim, dtype, variant, [&](auto kernel, int smem, int nw) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, kernel, (nw + 1) * 32, smem);
+    });
+}
+
+int64_t attn_counter_words(int32_t max_seqs, int32_t n_kv_heads) { return 64 + (int64_t)max_seqs * n_kv_heads; }
+
+cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
+                             int use3d, cudaStream_t stream) {
+    if (a.n_seqs <= 0) return cudaSuccess;
+    if (a.n_seqs > ATT_SMEM_SEQS) {  // batch too large for the in-kernel plan: build the chunk offsets first
+        plan_kernel<<<1, 1024, 0, stream>>>(a.ctx_lens, a.n_seqs, a.max_blocks * 16, a.split_tokens,
+                                            (int32_t)(sc.max_items / sh.n_kv_heads), sc.chunk_off, a.status);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     AttnParams p;
     p.q = (const uint16_t *)a.q;
+    p.out = (uint16_t *)a.out;
     p.block_table = a.block_table;
     p.ctx_lens = a.ctx_lens;
     p.slot_table = a.slot_table;
-    p.chunk_off = sc.chunk_off;
+    p.chunk_off_global = sc.chunk_off;
+    p.k_new = (const uint4 *)a.k_new;
+    p.v_new = (const uint4 *)a.v_new;
+    p.pool = (uint4 *)a.gpu_pool;
     p.part_o = sc.part_o;
     p.part_ml = sc.part_ml;
+    p.counters = sc.counters;
     p.status = a.status;
     p.n_gpu_slots = sh.n_gpu_slots;
     p.max_blocks = a.max_blocks;
@@ -686,38 +907,13 @@ static cudaError_t launch_one(const AttnShape &sh, const AttnScratch &sc, const 
     p.n_logical = sh.n_logical;
     p.split_tokens = a.split_tokens;
     p.use3d = use3d;
+    p.max_chunks = (int32_t)(sc.max_items / sh.n_kv_heads);
     p.scale_log2e = a.scale * 1.4426950408889634f;
-    paged_decode_attn_kernel<D, BF16><<<a.grid, ATT_THREADS, AttnSmem<D>::BYTES, stream>>>(map, p);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const int64_t rows = (int64_t)a.n_seqs * sh.n_q_heads;
-    combine_kernel<D, BF16><<<(unsigned)((rows + 3) / 4), 128, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off,
-                                                                           (uint16_t *)a.out, a.n_seqs, sh.n_q_heads,
-                                                                           sh.n_kv_heads, p.group);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
-                             int use3d, cudaStream_t stream) {
-    if (a.n_seqs <= 0) return cudaSuccess;
-    plan_kernel<<<1, 1024, 0, stream>>>(a.ctx_lens, a.n_seqs, a.max_blocks * 16, a.split_tokens,
-                                        (int32_t)(sc.max_items / sh.n_kv_heads), sc.chunk_off, a.status);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (a.k_new != nullptr && a.v_new != nullptr) {
-        dim3 grid((unsigned)a.n_seqs, (unsigned)sh.n_kv_heads);
-        append_kernel<<<grid, 2 * sh.head_dim / 8, 0, stream>>>((uint4 *)a.gpu_pool, (const uint4 *)a.k_new,
-                                                                (const uint4 *)a.v_new, a.block_table, a.max_blocks,
-                                                                a.ctx_lens, a.slot_table, sh.n_kv_heads, sh.head_dim,
-                                                                sh.n_logical, sh.n_gpu_slots, a.status);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
-    if (sh.head_dim == 128)
-        return sh.dtype == PIE_BF16 ? launch_one<128, true>(sh, sc, a, map, use3d, stream)
-                                    : launch_one<128, false>(sh, sc, a, map, use3d, stream);
-    return sh.dtype == PIE_BF16 ? launch_one<64, true>(sh, sc, a, map, use3d, stream)
-                                : launch_one<64, false>(sh, sc, a, map, use3d, stream);
+    if (a.k_new == nullptr || a.v_new == nullptr) p.k_new = p.v_new = nullptr;
+    return dispatch_variant(sh.head_dim, sh.dtype, a.variant, [&](auto kernel, int smem, int nw) -> cudaError_t {
+        kernel<<<a.grid, (nw + 1) * 32, smem, stream>>>(map, p);
+        return cudaGetLastError();
+    });
 }
 
 }  // namespace pie

@@ -35,7 +35,8 @@ struct AttnShape {
 };
 
 struct AttnScratch {
-    int32_t *chunk_off;  // [max_seqs + 1]
+    int32_t *chunk_off;  // [max_seqs + 1] (used only for batches beyond the in-kernel plan)
+    int32_t *counters;   // attn_counter_words(max_seqs, n_kv_heads) int32, zero before the first launch
     float *part_o;       // [max_items][G][D]
     float *part_ml;      // [max_items][G][2]
     int64_t max_items;   // capacity in items (chunk, kv head)
@@ -55,6 +56,7 @@ struct AttnLaunch {
     void *gpu_pool;
     int32_t split_tokens;
     int32_t grid;               // persistent CTAs
+    int32_t variant;            // kernel variant (0 = default)
     int32_t *status;            // device-visible status word
 };
 
@@ -64,7 +66,8 @@ struct AttnLaunch {
 cudaError_t make_pool_tensor_maps(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, int head_dim, CUtensorMap *map3d,
                                   CUtensorMap *map2d, int *use3d);
 int attn_smem_bytes(int head_dim);
-cudaError_t attn_configure(int head_dim, int dtype, int *ctas_per_sm);
+int64_t attn_counter_words(int32_t max_seqs, int32_t n_kv_heads);
+cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_sm);
 cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
                              int use3d, cudaStream_t stream);
 

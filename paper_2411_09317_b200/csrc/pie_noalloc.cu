@@ -49,7 +49,7 @@ int setup_device(int dev, DeviceSetup **out) {
         if (cudaDeviceGetAttribute(&s.n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PIE_ERR_CUDA;
         for (int d128 = 0; d128 < 2; ++d128)
             for (int dt = 0; dt < 2; ++dt)
-                if (pie::attn_configure(d128 ? 128 : 64, dt, &s.ctas_per_sm[d128][dt]) != cudaSuccess) return PIE_ERR_CUDA;
+                if (pie::attn_configure(d128 ? 128 : 64, dt, 0, &s.ctas_per_sm[d128][dt]) != cudaSuccess) return PIE_ERR_CUDA;
         s.scratch = static_cast<unsigned char *>(ptr);
         s.ready = true;
     }
@@ -70,7 +70,7 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
     if (n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads != 0) return PIE_ERR_INVALID;
     if (dtype != PIE_F16 && dtype != PIE_BF16) return PIE_ERR_INVALID;
     if ((head_dim != 64 && head_dim != 128) || n_q_heads / n_kv_heads > 8) return PIE_ERR_UNSUPPORTED;
-    if (split_tokens == 0) split_tokens = 256;
+    if (split_tokens == 0) split_tokens = 512;
     if (split_tokens < 0 || split_tokens % 16 != 0) return PIE_ERR_INVALID;
     if (((uintptr_t)kv_pool & 127) != 0) return PIE_ERR_INVALID;
     if ((uint64_t)n_slots * (uint64_t)n_kv_heads * 32u > 0x7fffffffull) return PIE_ERR_UNSUPPORTED;
@@ -86,9 +86,10 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
         chunks += (ctx + split_tokens - 1) / split_tokens;
     }
     const int64_t items = chunks * n_kv_heads;
+    const int64_t cnt_bytes = (pie::attn_counter_words(n_seqs, n_kv_heads) * 4 + 255) / 256 * 256;
     const int64_t ml_bytes = (items * group * 2 * 4 + 255) / 256 * 256;
     const int64_t o_bytes = items * group * head_dim * 4;
-    if (OFF_PART + ml_bytes + o_bytes > NOALLOC_SCRATCH_BYTES) return PIE_ERR_NOMEM;
+    if (OFF_PART + cnt_bytes + ml_bytes + o_bytes > NOALLOC_SCRATCH_BYTES) return PIE_ERR_NOMEM;
 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PIE_ERR_CUDA;
@@ -105,8 +106,11 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
     pie::AttnShape sh{head_dim, dtype, n_q_heads, n_kv_heads, n_logical_blocks, n_slots};
     pie::AttnScratch sc{};
     sc.chunk_off = reinterpret_cast<int32_t *>(setup->scratch + OFF_CHUNK);
-    sc.part_ml = reinterpret_cast<float *>(setup->scratch + OFF_PART);
-    sc.part_o = reinterpret_cast<float *>(setup->scratch + OFF_PART + ml_bytes);
+    sc.counters = reinterpret_cast<int32_t *>(setup->scratch + OFF_PART);
+    sc.part_ml = reinterpret_cast<float *>(setup->scratch + OFF_PART + cnt_bytes);
+    sc.part_o = reinterpret_cast<float *>(setup->scratch + OFF_PART + cnt_bytes + ml_bytes);
+    // the array keeps the last call's contents: the work and completion counters must start at zero
+    if (cudaMemsetAsync(sc.counters, 0, (size_t)cnt_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PIE_ERR_CUDA;
     sc.max_items = items;
     sc.max_seqs = NOALLOC_MAX_SEQS;
     pie::AttnLaunch a{};
@@ -122,6 +126,7 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
     a.v_new = nullptr;
     a.gpu_pool = const_cast<void *>(kv_pool);
     a.split_tokens = split_tokens;
+    a.variant = 0;
     a.grid = setup->ctas_per_sm[head_dim == 128][dtype] * setup->n_sms;
     a.status = status_dev ? status_dev : reinterpret_cast<int32_t *>(setup->scratch + OFF_STATUS);
     if (a.grid <= 0) return PIE_ERR_UNSUPPORTED;

@@ -340,6 +340,7 @@ void destroy_pool(pie_pool *p) {
     if (p->list_host) cudaFreeHost(p->list_host);
     if (p->status_host) cudaFreeHost(p->status_host);
     cudaFree(p->scratch.chunk_off);
+    cudaFree(p->scratch.counters);
     cudaFree(p->scratch.part_o);
     cudaFree(p->scratch.part_ml);
     cudaFree(p->stage_q);
@@ -414,6 +415,7 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.gpu_pool = p->gpu_base;
     a.split_tokens = (int32_t)split;
     a.grid = p->attn_grid;
+    a.variant = p->cfg.reserved[0];
     a.status = p->status_dev;
     cudaError_t e = pie::launch_attention(sh, p->scratch, a, p->use3d ? p->map3d : p->map2d, p->use3d, stream);
     if (e != cudaSuccess) {
@@ -576,7 +578,7 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     pie_pool *p = new (std::nothrow) pie_pool();
     if (!p) return PIE_ERR_NOMEM;
     p->cfg = *cfg;
-    if (p->cfg.split_tokens == 0) p->cfg.split_tokens = 256;
+    if (p->cfg.split_tokens == 0) p->cfg.split_tokens = 512;
     p->block_bytes = (int64_t)2 * 16 * cfg->n_kv_heads * cfg->head_dim * 2;
     p->n_sms = prop.multiProcessorCount;
     p->table = new (std::nothrow) pie::Table(cfg->n_layers, cfg->n_logical_blocks, cfg->n_gpu_slots, cfg->n_host_slots);
@@ -643,6 +645,11 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     p->scratch.max_items = max_chunks * cfg->n_kv_heads;
     p->scratch.max_seqs = cfg->max_seqs;
     PIE_TRY(cudaMalloc((void **)&p->scratch.chunk_off, (size_t)(cfg->max_seqs + 1) * 4), PIE_ERR_NOMEM);
+    {
+        const size_t words = (size_t)pie::attn_counter_words(cfg->max_seqs, cfg->n_kv_heads);
+        PIE_TRY(cudaMalloc((void **)&p->scratch.counters, words * 4), PIE_ERR_NOMEM);
+        PIE_TRY(cudaMemset(p->scratch.counters, 0, words * 4), PIE_ERR_CUDA);  // the kernel leaves them at zero again
+    }
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_o, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
     PIE_TRY(pie::make_pool_tensor_maps(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, cfg->head_dim, &p->map3d, &p->map2d,
@@ -651,7 +658,7 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     if (const char *env = std::getenv("PIE_TMA_2D"))
         if (env[0] == '1') p->use3d = 0;
     int per_sm = 0;
-    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, &per_sm), PIE_ERR_CUDA);
+    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, cfg->reserved[0], &per_sm), PIE_ERR_CUDA);
     if (per_sm <= 0) { destroy_pool(p); return PIE_ERR_UNSUPPORTED; }
     if (cfg->attn_ctas_per_sm > 0) per_sm = std::min(per_sm, cfg->attn_ctas_per_sm);
     p->attn_grid = per_sm * p->n_sms;
@@ -675,37 +682,25 @@ int pie_block_alloc(pie_pool *pool, int64_t n, const uint8_t *on_host, int32_t *
     pie::Table *t = pool->table;
     const int32_t NB = pool->cfg.n_logical_blocks, L = pool->cfg.n_layers;
     if (n > NB - t->n_allocated()) return PIE_ERR_NOMEM;
-    // all-or-nothing: check the slot budget first
-    int64_t need_host = 0, need_gpu = 0;
-    {
-        int64_t gpu_left = t->gpu_available();
-        for (int64_t i = 0; i < n; ++i) {
-            if (on_host && on_host[i]) need_host += L;
-            else {
-                const int64_t g = std::min<int64_t>(L, gpu_left - need_gpu);
-                need_gpu += g;
-                need_host += L - g;
-            }
-        }
-        if (need_host > t->host_available()) return PIE_ERR_NOMEM;
-    }
-    std::vector<int32_t> entries;
-    entries.reserve((size_t)(n * L * 2));
+    // ids: the lowest free ones; slots are handed out layer by layer (consecutive slots within a layer)
     int32_t next = 0;
     for (int64_t i = 0; i < n; ++i) {
         while (next < NB && t->allocated(next)) ++next;
-        st = t->alloc(next, on_host && on_host[i]);
-        if (st != PIE_OK) return st;  // cannot happen after the budget check
-        ids_out[i] = next;
+        ids_out[i] = next++;
+    }
+    st = t->alloc_bulk(ids_out, n, on_host);
+    if (st != PIE_OK) return st;  // all or nothing: the table is unchanged
+    std::vector<int32_t> entries;
+    entries.reserve((size_t)(n * L * 2));
+    for (int64_t i = 0; i < n; ++i)
         for (int32_t l = 0; l < L; ++l) {
-            const pie::Unit &u = t->unit(l, next);
+            const pie::Unit &u = t->unit(l, ids_out[i]);
             if (u.home_host) pool->home_count[(size_t)l] += 1;
             if (u.side == PIE_GPU) {
-                entries.push_back(l * NB + next);
+                entries.push_back(l * NB + ids_out[i]);
                 entries.push_back(u.gpu_slot);
             }
         }
-    }
     st = patch_units(pool, entries);
     if (st != PIE_OK) pool->sticky = st;
     return st;

@@ -10,8 +10,7 @@ namespace pie {
 
 // ------------------------------------------------------------------------------------ SlotPool
 SlotPool::SlotPool(int64_t n) {
-    ready_.reserve((size_t)n);
-    for (int64_t s = n - 1; s >= 0; --s) ready_.push_back((int32_t)s);
+    for (int64_t s = 0; s < n; ++s) ready_.push_back((int32_t)s);
 }
 
 void SlotPool::settle(const int64_t *done) {
@@ -27,8 +26,8 @@ void SlotPool::settle(const int64_t *done) {
 
 int32_t SlotPool::take(SlotTag *tag) {
     if (!ready_.empty()) {
-        int32_t s = ready_.back();
-        ready_.pop_back();
+        int32_t s = ready_.front();
+        ready_.pop_front();
         tag->queue = PIE_Q_NONE;
         tag->ticket = 0;
         return s;
@@ -82,6 +81,49 @@ int Table::alloc(int32_t block, bool on_host) {
     }
     allocated_[block] = 1;
     ++n_allocated_;
+    return PIE_OK;
+}
+
+int Table::alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host) {
+    settle();
+    for (int64_t i = 0; i < n; ++i) {
+        if (blocks[i] < 0 || blocks[i] >= NB) return PIE_ERR_RANGE;
+        if (allocated_[blocks[i]]) return PIE_ERR_INVALID;
+    }
+    // budget: a block that is not forced to the host takes GPU slots for its first layers while any are left
+    std::vector<int32_t> n_gpu((size_t)n, 0);
+    int64_t gpu_left = gpu_.available(), need_host = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        n_gpu[(size_t)i] = on_host && on_host[i] ? 0 : (int32_t)std::min<int64_t>(L, gpu_left);
+        gpu_left -= n_gpu[(size_t)i];
+        need_host += L - n_gpu[(size_t)i];
+    }
+    if (need_host > host_.available()) return PIE_ERR_NOMEM;
+    for (int32_t l = 0; l < L; ++l)
+        for (int64_t i = 0; i < n; ++i) {
+            Unit &u = unit(l, blocks[i]);
+            SlotTag tag;
+            if (l < n_gpu[(size_t)i]) {
+                u.gpu_slot = gpu_.take(&tag);
+                u.host_slot = -1;
+                u.side = PIE_GPU;
+                u.home_host = 0;
+            } else {
+                u.host_slot = host_.take(&tag);
+                u.gpu_slot = -1;
+                u.side = PIE_HOST;
+                u.home_host = 1;
+            }
+            u.last_q = (uint8_t)tag.queue;
+            u.last_t = tag.ticket;
+            if (tag.queue != PIE_Q_NONE) {
+                int64_t &w = layer_wait_[(size_t)l * 4 + tag.queue];
+                w = std::max(w, tag.ticket);
+            }
+            u.t_stamp = clock_;
+        }
+    for (int64_t i = 0; i < n; ++i) allocated_[blocks[i]] = 1;
+    n_allocated_ += (int32_t)n;
     return PIE_OK;
 }
 

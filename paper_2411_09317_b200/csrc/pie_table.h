@@ -14,9 +14,10 @@ struct SlotTag {
     int64_t ticket;
 };
 
-// Free slots of one pool.  `ready` is a stack (slot 0 on top at start); `pending` is a queue of slots
+// Free slots of one pool.  `ready` is a queue (0 .. n-1 at start); `pending` is a queue of slots
 // released by a copy that may not have finished: they can be handed out, but the receiver must wait
-// for the tag's ticket.
+// for the tag's ticket.  First in, first out on both: slots released together are handed out together
+// again, so swap lists stay long runs of consecutive slots (few, large copies).
 class SlotPool {
   public:
     explicit SlotPool(int64_t n);
@@ -31,7 +32,7 @@ class SlotPool {
         int32_t queue;
         int64_t ticket;
     };
-    std::vector<int32_t> ready_;
+    std::deque<int32_t> ready_;
     std::deque<Pending> pending_;
 };
 
@@ -50,6 +51,8 @@ class Table {
     Table(int32_t n_layers, int32_t n_logical, int64_t n_gpu_slots, int64_t n_host_slots);
 
     int alloc(int32_t block, bool on_host);
+    // n blocks at once, slots handed out layer by layer so that each layer's units sit in consecutive slots
+    int alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host);
     int free_block(int32_t block);
     int swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int32_t *moved,
              int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits);

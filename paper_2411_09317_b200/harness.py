@@ -21,7 +21,7 @@ class DeviceWorkload:
 
     def __init__(self, wl: synth.Workload, host_frac=None, timing=True, split_tokens=0, swap_ctas=0,
                  attn_ctas_per_sm=0, staging_layers=3, shuffle_table=False, extra_gpu_slots=0, extra_host_slots=0,
-                 extra_tokens=None):
+                 extra_tokens=None, attn_variant=0):
         self.wl = wl
         dev = torch.device("cuda", torch.cuda.current_device())
         self.dev = dev
@@ -49,7 +49,7 @@ class DeviceWorkload:
             gpu_base=self.gpu_pool.data_ptr(), host_base=self.host_pool.data_ptr(), own_streams=0,
             compute_stream=self.s_compute.cuda_stream, copy_in_stream=self.s_in.cuda_stream,
             copy_out_stream=self.s_out.cuda_stream, split_tokens=split_tokens, swap_ctas=swap_ctas,
-            attn_ctas_per_sm=attn_ctas_per_sm, timing=int(timing))
+            attn_ctas_per_sm=attn_ctas_per_sm, timing=int(timing), attn_variant=attn_variant)
         ids = pie.pie_block_alloc(self.pool, self.NB, on_host)
         assert np.array_equal(ids, np.arange(self.NB))
         self.fill_pools()
