@@ -32,6 +32,9 @@ if ROOT not in sys.path:
 from paper_2411_09317_b200 import synth  # noqa: E402
 
 WORKLOAD = "llama2_7b"
+# dram__bytes_read + dram__bytes_write per algorithmic byte of the attention kernel, from the ncu capture summarised in
+# profiles/paged_decode_attn_llama2_7b_quarter.md (quarter-scale case; traffic grows in proportion to the KV bytes)
+TRAFFIC_PER_ALG_BYTE = 1.026
 METRIC = "paged decode-attn GB/s over whole decode steps, swaps hidden at <=2% slowdown"
 
 
@@ -220,7 +223,10 @@ def main():
 
     # the GPU pool is sized for the fully resident baseline run as well (every unit + 3 layers of staging)
     ramp = max(args.warmup, args.ramp)
-    total_steps = 1 + 3 + 3 + args.steps + ramp + args.steps + 3 + args.steps   # every phase below appends one token per step
+    sweep_ratios = [0.0005, 0.001, 0.002, 0.004, 0.008]
+    n_sweep = 8
+    # every phase below appends one token per step
+    total_steps = 1 + 3 + 3 + args.steps + ramp + args.steps + len(sweep_ratios) * (3 + n_sweep) + 3 + n_sweep + 3 + args.steps
     n_host_blocks = int(round(wl.host_frac * (int(((wl.ctx_lens.astype(np.int64) + total_steps + 15) // 16).sum()))))
     dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
                         attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=L * (n_host_blocks + wl.n_seqs),
@@ -282,7 +288,8 @@ def main():
     swapped_out = s_after["bytes_out"] - s_before["bytes_out"]
     comp_ms = [s["last_step_compute_ms"] for s in st_run if s["steps_measured"] > 0]
     attn_ms_layer = float(np.mean(comp_ms)) / L if comp_ms else float("nan")
-    n_launch = int(4 * L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
+    # one attention kernel per layer call, plus one swap kernel (or one table-patch kernel after copy-engine copies) per list
+    n_launch = int(L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
                    (s_after["calls_copy_engine"] - s_before["calls_copy_engine"]))
     slowdown = resident_gbs / value_1gpu - 1.0   # in GB/s, since the contexts keep growing between the two runs
     hidden = {
@@ -292,6 +299,34 @@ def main():
         "frac_of_link": (swapped_in / (ms_run * 1e-3) / 1e9) / max(link["h2d"], 1e-9),
         "stall_frac": st_run[-1]["last_step_stall_ms"] / max(st_run[-1]["last_step_ms"], 1e-9),
     }
+
+    # ---- phase 4: fixed ratios, to place the <= 2 % slow-down point (resident re-measured afterwards: A/B/A) ----------
+    sweep = []
+    for r in sweep_ratios:
+        pie.pie_set_extension_ratio(dw.pool, r)
+        timed_steps(dw, torch, 3)
+        c0 = dw.ctx_lens.copy()
+        sb = pie.pie_get_stats(dw.pool)
+        ms_r, _ = timed_steps(dw, torch, n_sweep)
+        sa = pie.pie_get_stats(dw.pool)
+        sweep.append({"ratio": r, "attn_gbs": bytes_of_steps(n_sweep, c0) / (ms_r * 1e-3) / 1e9,
+                      "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / (ms_r * 1e-3) / 1e9,
+                      "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / (ms_r * 1e-3) / 1e9})
+    pie.pie_set_extension_ratio(dw.pool, 0.0)
+    timed_steps(dw, torch, 3)
+    c0 = dw.ctx_lens.copy()
+    ms_res2, _ = timed_steps(dw, torch, n_sweep)
+    resident2_gbs = bytes_of_steps(n_sweep, c0) / (ms_res2 * 1e-3) / 1e9
+    ref_gbs = 0.5 * (resident_gbs + resident2_gbs)
+    best = None
+    for e in sweep:
+        e["slowdown"] = ref_gbs / e["attn_gbs"] - 1.0
+        e["frac_of_link"] = e["swap_in_gbs"] / max(link["both"], 1e-9)
+        if e["slowdown"] <= 0.02 and (best is None or e["swap_in_gbs"] > best["swap_in_gbs"]):
+            best = e
+    hidden["fixed_ratio_sweep"] = sweep
+    hidden["resident_gbs_after_sweep"] = resident2_gbs
+    hidden["best_within_2pct"] = best
 
     # ---- e2e: the same step through the host-buffer entry point (inputs H2D, outputs D2H inside the region) -----
     q_h = torch.empty(dw.q_all.shape, dtype=torch.int16).pin_memory()
@@ -324,8 +359,9 @@ def main():
     peak, peak_kind = measured_peaks()
     achieved = bytes_layer0 / (attn_ms_layer * 1e-3) / 1e9 if attn_ms_layer == attn_ms_layer else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": None, "peak_kind": peak_kind,
-                "kernel": "paged_decode_attn_kernel (+plan, append, combine: per-layer event span)",
+                "frac": (achieved / peak) if achieved else None, "traffic": int(TRAFFIC_PER_ALG_BYTE * bytes_layer0),
+                "traffic_note": "ncu dram bytes of a quarter-scale launch scaled by the KV bytes read", "peak_kind": peak_kind,
+                "kernel": "paged_decode_attn_kernel (plan, append and combine fused; per-layer event span on the compute stream)",
                 "alg_bytes_per_launch": bytes_layer0, "ms_per_launch": attn_ms_layer, "hbm_copy_probe_gbs": hbm_probe,
                 "frac_of_nominal_8tbs": (achieved / 8000.0) if achieved else None}
 

@@ -88,7 +88,7 @@ typedef struct pie_stats {
     double ratio;                          /* current extension ratio */
     int64_t n_units_gpu, n_units_host, n_units_in_flight;
     int64_t steps_measured;
-    double reserved[8];
+    double reserved[8];                    /* [0]: last step's attention slow-down vs the no-swap record, ms */
 } pie_stats;
 
 /* ---- pool (Section 3.1: the physical pools; Section 3.2: the mapping table) --------------------- */
@@ -164,10 +164,9 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
 
 /* One decode step: for every layer l, prefetch layer l+1's host-resident units (wrapping to layer 0 of
  * the next token, Section 3.4.2), run layer l's attention, push layer l's share back out (Section 3.3:
- * the layer that just finished is the coldest).  PIE_ERR_NOMEM if the GPU pool cannot take a layer's
+ * the layer that just finished is the coldest).  With timing enabled the host runs at most 4 steps ahead.  PIE_ERR_NOMEM if the GPU pool cannot take a layer's
  * host-resident share (the layers before it have been enqueued).  q_all/out_all: device [n_layers][n_seqs][Hq][D];
- * k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D] or NULL.  Runs pie_controller_tick at the end
- * when the ratio is adaptive.  Never blocks the host on the GPU. */
+ * k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D] or NULL.  Runs pie_controller_tick at the end. */
 int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev,
                     int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale,
                     const void *k_new_all, const void *v_new_all, int32_t mode);
@@ -188,14 +187,18 @@ int pie_set_extension_ratio(pie_pool *pool, float r);
 int pie_get_extension_ratio(pie_pool *pool, float *r);
 /* Controller constants (the paper gives none): step = ratio change per adjustment (default 1 / n_layers,
  * "one layer"), eps = stall / compute above which a step counts as stalled (0.02), u_hi = link-busy /
- * compute below which the ratio may grow (0.9).  A value <= 0 keeps the current setting. */
+ * compute below which the ratio may grow (0.9).  A value <= 0 keeps the current setting.
+ * What counts as "stall" is the compute stream's wait for arriving units plus the attention time in excess of
+ * the time-per-token record taken on steps without swap traffic (copies that are hidden can still slow the
+ * attention down through shared HBM bandwidth). */
 int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
 /* The per-layer plan at the start of layer `layer`: in_ids = units of layer (layer+1) mod L to bring in
  * (ascending id, as many as the GPU pool can take), out_ids = units of `layer` to push out once it has
  * computed.  Arrays are host, capacity n_logical_blocks each. */
 int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in, int32_t *out_ids, int64_t *n_out);
-/* Read the previous step's events (no blocking: returns PIE_OK with *changed = 0 if they have not all
- * completed), update the stats, and in adaptive mode adjust the ratio. */
+/* Evaluate, in step order, the event sets of earlier steps that have completed (no blocking), update the
+ * stats, and in adaptive mode adjust the ratio.  The library keeps 4 steps of events: pie_step_begin waits
+ * for the oldest step when the host gets that far ahead of the GPU. */
 int pie_controller_tick(pie_pool *pool, int32_t *changed);
 int pie_get_stats(pie_pool *pool, pie_stats *out);
 /* Wait until everything enqueued so far has completed, at most timeout_us (PIE_ERR_TIMEOUT); applies
@@ -223,7 +226,8 @@ int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps);
  *   slot_table  device int32 [n_logical_blocks]: GPU slot of each logical block of this layer, -1 if absent
  *   q, out, block_table_dev, ctx_lens_dev, scale   as for pie_decode_attention (no append)
  *   ctx_lens_host  host copy of the lengths (required: sizes are checked before anything is enqueued)
- *   status_dev  optional device int32[4]; word 0 is set to 1 if a referenced block had no slot
+ *   status_dev  optional device int32[4]; word 0 is set to 1 if a referenced block had no slot, word 3
+ *               receives the batch's context-token count
  *   stream      a cudaStream_t
  * The split-K scratch (chunk offsets, fp32 partials) is a static device array of PIE_NOALLOC_SCRATCH_BYTES
  * that every GPU loading the library holds until the process exits.  A call whose partials would not fit

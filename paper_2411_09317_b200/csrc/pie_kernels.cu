@@ -381,6 +381,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // ---- plan: chunk offsets of the batch (exclusive scan of the per-sequence chunk counts)
     const bool co_in_smem = p.n_seqs <= ATT_SMEM_SEQS;
     if (co_in_smem) {
+        int32_t my_tokens = 0;
         for (int32_t s = tid; s < p.n_seqs; s += ATT_THREADS) {
             int32_t ctx = __ldg(p.ctx_lens + s);
             if (ctx > p.max_blocks * 16) {
@@ -388,6 +389,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 if (blockIdx.x == 0) raise_status(p.status, STATUS_CTX_TOO_LONG);
             }
             co_smem[s + 1] = ctx > 0 ? (ctx + p.split_tokens - 1) / p.split_tokens : 0;
+            my_tokens += max(ctx, 0);
+        }
+        if (blockIdx.x == 0) {  // the batch's context tokens, for the host's time-per-token record (status word 3)
+            if (tid == 0) misc[2] = 0;
+            __syncthreads();
+            atomicAdd(const_cast<int32_t *>(misc + 2), my_tokens);
+            __syncthreads();
+            if (tid == 0) *reinterpret_cast<volatile int32_t *>(p.status + 3) = misc[2];
         }
         __syncthreads();
         if (warp == 0) {

@@ -18,6 +18,7 @@ thread_local int g_last_cuda_error = 0;
 
 constexpr int EV_RING = 512;       // events per queue: ticket t uses slot t % EV_RING
 constexpr int LIST_EVENTS = 512;   // events guarding regions of the id-list ring
+constexpr int TIMING_RING = 4;     // the host may enqueue at most this many steps ahead of their evaluation
 constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB
 
 #define PIE_CUDA(call)                                  \
@@ -75,9 +76,12 @@ struct pie_pool {
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
     std::vector<int64_t> home_count;  // per layer: units whose home is the host
     // timing
-    std::vector<LayerEvents> lev[2];
+    // per-step event sets: step k uses set k % TIMING_RING; a set is evaluated once, in step order, when complete
+    std::vector<LayerEvents> lev[TIMING_RING];
+    int64_t lev_step[TIMING_RING] = {};      // which step a set holds (0 = none)
+    bool lev_done[TIMING_RING] = {};         // already evaluated
     int64_t step = 0;
-    bool prev_step_valid = false, prev_step_ticked = true;
+    double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
     pie_stats stats{};
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
@@ -178,7 +182,7 @@ int check_status_word(pie_pool *p) {
 
 LayerEvents *timing_slot(pie_pool *p, int32_t layer) {
     if (!p->cfg.timing) return nullptr;
-    return &p->lev[p->step & 1][(size_t)layer];
+    return &p->lev[p->step % TIMING_RING][(size_t)layer];
 }
 
 // ---- one swap call ------------------------------------------------------------------------------------
@@ -326,7 +330,7 @@ void destroy_pool(pie_pool *p) {
             if (p->ticket_ev[q][i]) cudaEventDestroy(p->ticket_ev[q][i]);
     for (int i = 0; i < LIST_EVENTS; ++i)
         if (p->list_events[i]) cudaEventDestroy(p->list_events[i]);
-    for (int k = 0; k < 2; ++k)
+    for (int k = 0; k < TIMING_RING; ++k)
         for (LayerEvents &e : p->lev[k])
             for (cudaEvent_t ev : {e.pre, e.go, e.done, e.in0, e.in1, e.out0, e.out1})
                 if (ev) cudaEventDestroy(ev);
@@ -622,7 +626,7 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
         for (int i = 0; i < EV_RING; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->ticket_ev[q][i], cudaEventDisableTiming), PIE_ERR_CUDA);
     for (int i = 0; i < LIST_EVENTS; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->list_events[i], cudaEventDisableTiming), PIE_ERR_CUDA);
     if (cfg->timing) {
-        for (int k = 0; k < 2; ++k) {
+        for (int k = 0; k < TIMING_RING; ++k) {
             p->lev[k].resize((size_t)cfg->n_layers);
             for (LayerEvents &e : p->lev[k])
                 for (cudaEvent_t *ev : {&e.pre, &e.go, &e.done, &e.in0, &e.in1, &e.out0, &e.out1})
@@ -825,16 +829,106 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
                           ctx_lens_host, n_seqs, scale, k_new, v_new);
 }
 
+// Evaluate one step's event set: per-layer compute, stall and swap times -> stats -> (adaptive mode) the ratio.
+// wait = true blocks until the set's events have completed (used only when the ring is about to wrap).
+static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed) {
+    std::vector<LayerEvents> &ev = pool->lev[k];
+    for (LayerEvents &e : ev) {
+        for (int which = 0; which < 3; ++which) {
+            const bool has = which == 0 ? e.has_compute : which == 1 ? e.has_in : e.has_out;
+            cudaEvent_t evt = which == 0 ? e.done : which == 1 ? e.in1 : e.out1;
+            if (!has) continue;
+            if (wait) PIE_CUDA(cudaEventSynchronize(evt));
+            else if (cudaEventQuery(evt) != cudaSuccess) return 1;  // not complete yet
+        }
+    }
+    double compute = 0, stall = 0, t_in = 0, t_out = 0;
+    cudaEvent_t first = nullptr, last = nullptr;
+    bool any_swap = false;
+    for (LayerEvents &e : ev) {
+        float ms = 0;
+        if (e.has_compute) {
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.go, e.done));
+            compute += ms;
+            if (e.waited) {
+                // two back-to-back event records are already ~2-3 us apart: count only what exceeds that
+                PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
+                stall += std::max(0.0, (double)ms - 0.004);
+            }
+            if (!first) first = e.pre;
+            last = e.done;
+        }
+        if (e.has_in) {
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.in0, e.in1));
+            t_in += ms;
+            any_swap = true;
+        }
+        if (e.has_out) {
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.out0, e.out1));
+            t_out += ms;
+            any_swap = true;
+        }
+    }
+    pool->lev_done[k] = true;
+    pool->stats.last_step_compute_ms = compute;
+    pool->stats.last_step_stall_ms = stall;
+    pool->stats.last_step_swap_in_ms = t_in;
+    pool->stats.last_step_swap_out_ms = t_out;
+    if (first && last) {
+        float ms = 0;
+        PIE_CUDA(cudaEventElapsedTime(&ms, first, last));
+        pool->stats.last_step_ms = ms;
+    }
+    pool->stats.steps_measured += 1;
+    // Performance record (Section 3.4.2): attention time per context token on steps without swap traffic.  Copies
+    // that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
+    // wait, so the controller holds the ratio where wait + slow-down stays within its tolerance.
+    const double tokens = (double)((volatile int32_t *)pool->status_host)[3];
+    double slow = 0.0;
+    if (tokens > 0 && compute > 0) {
+        const double per_token = compute / tokens;
+        if (!any_swap) pool->base_ms_per_token = pool->base_ms_per_token > 0 ? 0.75 * pool->base_ms_per_token + 0.25 * per_token : per_token;
+        else if (pool->base_ms_per_token > 0) slow = std::max(0.0, compute - pool->base_ms_per_token * tokens);
+    }
+    pool->stats.reserved[0] = slow;
+    if (pool->ratio_mode == 2 && compute > 0) {
+        const double step = pool->ctrl_step > 0 ? pool->ctrl_step : 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
+        const double r = pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall + slow, compute, std::max(t_in, t_out));
+        if (r != pool->ratio) {
+            pool->ratio = r;
+            if (changed) *changed = 1;
+        }
+    }
+    return PIE_OK;
+}
+
+// evaluate, in step order, every completed set that has not been evaluated yet
+static int evaluate_completed(pie_pool *pool, int32_t *changed) {
+    for (int64_t st = std::max<int64_t>(1, pool->step - TIMING_RING + 1); st < pool->step; ++st) {
+        const int k = (int)(st % TIMING_RING);
+        if (pool->lev_step[k] != st || pool->lev_done[k]) continue;
+        const int rc = evaluate_step_set(pool, k, false, changed);
+        if (rc < 0) return rc;
+        if (rc == 1) break;  // this one is still running: so are the later ones
+    }
+    return PIE_OK;
+}
+
 int pie_step_begin(pie_pool *pool) {
     if (!pool) return PIE_ERR_INVALID;
+    ++pool->step;
     if (pool->cfg.timing) {
-        // the set about to be reused belongs to step-1's predecessor: it must have been read (or is dropped)
-        pool->prev_step_valid = pool->step > 0;
-        pool->prev_step_ticked = false;
-        ++pool->step;
-        for (LayerEvents &e : pool->lev[pool->step & 1]) e.has_in = e.has_out = e.has_compute = e.waited = false;
-    } else {
-        ++pool->step;
+        int st = evaluate_completed(pool, nullptr);
+        if (st != PIE_OK) return st;
+        const int k = (int)(pool->step % TIMING_RING);
+        if (pool->lev_step[k] != 0 && !pool->lev_done[k]) {
+            // the ring wraps: the host is TIMING_RING steps ahead of the GPU; wait for that step and evaluate it
+            st = evaluate_step_set(pool, k, true, nullptr);
+            if (st < 0) return st;
+        }
+        pool->lev_step[k] = pool->step;
+        pool->lev_done[k] = false;
+        for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = e.waited = false;
     }
     return PIE_OK;
 }
@@ -889,58 +983,8 @@ int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in
 int pie_controller_tick(pie_pool *pool, int32_t *changed) {
     if (!pool) return PIE_ERR_INVALID;
     if (changed) *changed = 0;
-    if (!pool->cfg.timing || !pool->prev_step_valid || pool->prev_step_ticked) return PIE_OK;
-    std::vector<LayerEvents> &ev = pool->lev[(pool->step - 1) & 1];
-    // everything of the previous step must have completed; never block
-    for (LayerEvents &e : ev) {
-        if (e.has_compute && cudaEventQuery(e.done) != cudaSuccess) return PIE_OK;
-        if (e.has_in && cudaEventQuery(e.in1) != cudaSuccess) return PIE_OK;
-        if (e.has_out && cudaEventQuery(e.out1) != cudaSuccess) return PIE_OK;
-    }
-    double compute = 0, stall = 0, t_in = 0, t_out = 0;
-    cudaEvent_t first = nullptr, last = nullptr;
-    for (LayerEvents &e : ev) {
-        float ms = 0;
-        if (e.has_compute) {
-            PIE_CUDA(cudaEventElapsedTime(&ms, e.go, e.done));
-            compute += ms;
-            if (e.waited) {
-                // two back-to-back event records are already ~2-3 us apart: count only what exceeds that
-                PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
-                stall += std::max(0.0, (double)ms - 0.004);
-            }
-            if (!first) first = e.pre;
-            last = e.done;
-        }
-        if (e.has_in) {
-            PIE_CUDA(cudaEventElapsedTime(&ms, e.in0, e.in1));
-            t_in += ms;
-        }
-        if (e.has_out) {
-            PIE_CUDA(cudaEventElapsedTime(&ms, e.out0, e.out1));
-            t_out += ms;
-        }
-    }
-    pool->prev_step_ticked = true;
-    pool->stats.last_step_compute_ms = compute;
-    pool->stats.last_step_stall_ms = stall;
-    pool->stats.last_step_swap_in_ms = t_in;
-    pool->stats.last_step_swap_out_ms = t_out;
-    if (first && last) {
-        float ms = 0;
-        PIE_CUDA(cudaEventElapsedTime(&ms, first, last));
-        pool->stats.last_step_ms = ms;
-    }
-    pool->stats.steps_measured += 1;
-    if (pool->ratio_mode == 2 && compute > 0) {
-        const double step = pool->ctrl_step > 0 ? pool->ctrl_step : 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
-        const double r = pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall, compute, std::max(t_in, t_out));
-        if (r != pool->ratio) {
-            pool->ratio = r;
-            if (changed) *changed = 1;
-        }
-    }
-    return PIE_OK;
+    if (!pool->cfg.timing) return PIE_OK;
+    return evaluate_completed(pool, changed);
 }
 
 int pie_get_stats(pie_pool *pool, pie_stats *out) {
