@@ -190,29 +190,16 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
     from paper_2411_09317_b200 import binding as pie
     from paper_2411_09317_b200.harness import DeviceWorkload
+    from paper_2411_09317_b200.replicas import Replicas
 
-    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    rep = Replicas("nccl")                      # replicas only: one independent pool per GPU, timing combined
+    rank, world, local = rep.rank, rep.world, rep.local_rank
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier, max_over_ranks = rep.barrier, rep.max_over_ranks
 
     wl = synth.workload(WORKLOAD, args.scale)
     L = wl.n_layers
@@ -392,8 +379,7 @@ def main():
         }
         print(json.dumps(line))
     dw.close()
-    if world > 1:
-        dist.destroy_process_group()
+    rep.close()
 
 
 if __name__ == "__main__":

@@ -129,7 +129,10 @@ int pie_get_placement(pie_pool *pool, int32_t *side, int32_t *slot);
  * known complete (observed with cudaEventQuery at any later call) the units read PIE_HOST.
  * Blocks already on, or heading to, the host are skipped.  block_ids: host, n entries, distinct.
  * mode: PIE_MODE_KERNEL = gather/scatter kernel, PIE_MODE_COPY_ENGINE = one cudaMemcpyAsync per run of
- * consecutive slots, PIE_MODE_AUTO = chosen from the run lengths. */
+ * consecutive slots, PIE_MODE_AUTO = copy engine when the list is at most 8 runs or its runs average 1 MiB,
+ * else the kernel (measured: the copy engine reaches the link rate from ~16 MB and disturbs a concurrent
+ * attention kernel several times less than SM-issued host traffic, but one call per scattered 64 KiB block
+ * tops out near 12 GB/s). */
 int pie_swap_out(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode);
 /* The mirror image on the copy-in stream.  The layer's next pie_decode_attention waits for it
  * (Section 3.2: presence check). */
@@ -201,6 +204,11 @@ int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in
  * for the oldest step when the host gets that far ahead of the GPU. */
 int pie_controller_tick(pie_pool *pool, int32_t *changed);
 int pie_get_stats(pie_pool *pool, pie_stats *out);
+/* Per-layer timeline of the most recently evaluated step (timing = 1): ms[l][7] = {compute stream reaches the
+ * layer, presence wait over, layer done, swap-in start, swap-in end, swap-out start, swap-out end} in ms
+ * from the step's first event; -1 where nothing was recorded.  capacity = floats available (>= 7 * n_layers).
+ * PIE_ERR_INVALID if no step has been evaluated yet.  Shows what overlapped with what. */
+int pie_get_step_timeline(pie_pool *pool, float *ms, int64_t capacity);
 /* Wait until everything enqueued so far has completed, at most timeout_us (PIE_ERR_TIMEOUT); applies
  * phase-2 updates and reports a pending device status word (PIE_ERR_NOT_RESIDENT ...). */
 int pie_sync(pie_pool *pool, int64_t timeout_us);

@@ -98,10 +98,11 @@ def simulate_protocol(n_layers, t_swap, gpu_regions, cpu_regions, cpu_layers, n_
 #   - decrease when the computation had to wait for a swap (stall above eps of compute time) in at
 #     least k_dec of the last `window` steps - a single disturbed step is tolerated;
 #   - increase by one step when there was no stall and the link was busy for less than u_hi of the
-#     compute time (the link has slack and nothing on the host was needed late);
+#     compute time (the link has slack and nothing on the host was needed late), but not within
+#     `cooldown` steps of the previous increase (a change has to be observed before the next);
 #   - hold otherwise.
 # The paper gives no constants; these are the build's: step = 1/n_layers ("one layer"), eps = 0.02,
-# k_dec = 2 of window = 4, u_hi = 0.9.
+# k_dec = 2 of window = 4, u_hi = 0.9, cooldown = 3.
 # ---------------------------------------------------------------------------------------------
 
 @dataclasses.dataclass
@@ -112,7 +113,9 @@ class Controller:
     window: int = 4
     u_hi: float = 0.9
     r_max: float = 1.0
+    cooldown: int = 3
     r: float = 0.0
+    wait: int = 0
     history: list = dataclasses.field(default_factory=list)
 
     def tick(self, stall, compute, swap_busy):
@@ -124,8 +127,11 @@ class Controller:
             if sum(self.history) >= self.k_dec:
                 self.r = max(0.0, self.r - self.step)
                 self.history = []
+        elif self.wait > 0:
+            self.wait -= 1
         elif swap_busy < self.u_hi * compute and self.r < self.r_max:
             self.r = min(self.r_max, self.r + self.step)
+            self.wait = self.cooldown
         return self.r
 
 

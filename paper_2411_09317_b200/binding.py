@@ -29,7 +29,7 @@ EXPORTS = [
     "pie_pool_create", "pie_pool_destroy", "pie_block_bytes", "pie_block_alloc", "pie_block_free", "pie_block_write",
     "pie_block_read", "pie_block_state", "pie_get_placement", "pie_swap_out", "pie_swap_in", "pie_swap_raw",
     "pie_decode_attention", "pie_decode_step", "pie_decode_step_host", "pie_step_begin", "pie_set_extension_ratio",
-    "pie_get_extension_ratio", "pie_set_controller", "pie_plan_layer", "pie_controller_tick", "pie_get_stats", "pie_sync", "pie_status_str",
+    "pie_get_extension_ratio", "pie_set_controller", "pie_plan_layer", "pie_controller_tick", "pie_get_stats", "pie_get_step_timeline", "pie_sync", "pie_status_str",
     "pie_last_cuda_error", "pie_probe_link", "pie_probe_hbm", "pie_table_create", "pie_table_destroy", "pie_table_alloc",
     "pie_table_free", "pie_table_swap", "pie_table_attention", "pie_table_confirm", "pie_table_state", "pie_fifo_create",
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
@@ -91,6 +91,7 @@ _sig = {
     "pie_plan_layer": (_i32, [_vp, _i32, _vp, ctypes.POINTER(_i64), _vp, ctypes.POINTER(_i64)]),
     "pie_controller_tick": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "pie_get_stats": (_i32, [_vp, ctypes.POINTER(Stats)]),
+    "pie_get_step_timeline": (_i32, [_vp, _vp, _i64]),
     "pie_sync": (_i32, [_vp, _i64]),
     "pie_status_str": (ctypes.c_char_p, [_i32]),
     "pie_last_cuda_error": (_i32, []),
@@ -280,6 +281,12 @@ def pie_get_stats(pool) -> dict:
     s = Stats()
     check(lib.pie_get_stats(pool, ctypes.byref(s)), "pie_get_stats")
     return s.as_dict()
+
+
+def pie_get_step_timeline(pool, n_layers) -> np.ndarray:
+    out = np.zeros((n_layers, 7), dtype=np.float32)
+    check(lib.pie_get_step_timeline(pool, _ptr(out), out.size), "pie_get_step_timeline")
+    return out
 
 
 def pie_sync(pool, timeout_us=60_000_000) -> None:

@@ -19,7 +19,8 @@ thread_local int g_last_cuda_error = 0;
 constexpr int EV_RING = 512;       // events per queue: ticket t uses slot t % EV_RING
 constexpr int LIST_EVENTS = 512;   // events guarding regions of the id-list ring
 constexpr int TIMING_RING = 4;     // the host may enqueue at most this many steps ahead of their evaluation
-constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB
+constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB ...
+constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list is at most this many runs
 
 #define PIE_CUDA(call)                                  \
     do {                                                \
@@ -82,6 +83,7 @@ struct pie_pool {
     bool lev_done[TIMING_RING] = {};         // already evaluated
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
+    std::vector<float> timeline;     // last evaluated step: [L][7] ms from the step's first event (-1 = not recorded)
     pie_stats stats{};
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
@@ -196,7 +198,10 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         int64_t runs = 1;
         for (int64_t i = 1; i < n; ++i)
             if (src[i] != src[i - 1] + 1 || dst[i] != dst[i - 1] + 1) ++runs;
-        mode = (n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES ? PIE_MODE_COPY_ENGINE : PIE_MODE_KERNEL;
+        // copy engine for long runs or few copies (no SM or L2 footprint next to attention); the kernel for scattered
+        // lists, where one cudaMemcpyAsync per block would be bound by the call rate (~5 us each)
+        mode = ((n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS) ? PIE_MODE_COPY_ENGINE
+                                                                                                   : PIE_MODE_KERNEL;
     }
     const bool need_list = mode == PIE_MODE_KERNEL || slot_table_row != nullptr;
     int64_t off = 0;
@@ -870,6 +875,19 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         }
     }
     pool->lev_done[k] = true;
+    if (first) {
+        pool->timeline.assign(ev.size() * 7, -1.f);
+        for (size_t l = 0; l < ev.size(); ++l) {
+            LayerEvents &e = ev[l];
+            cudaEvent_t list[7] = {e.pre, e.go, e.done, e.in0, e.in1, e.out0, e.out1};
+            const bool has[7] = {e.has_compute, e.has_compute, e.has_compute, e.has_in, e.has_in, e.has_out, e.has_out};
+            for (int j = 0; j < 7; ++j)
+                if (has[j]) {
+                    float ms = 0;
+                    if (cudaEventElapsedTime(&ms, first, list[j]) == cudaSuccess) pool->timeline[l * 7 + j] = ms;
+                }
+        }
+    }
     pool->stats.last_step_compute_ms = compute;
     pool->stats.last_step_stall_ms = stall;
     pool->stats.last_step_swap_in_ms = t_in;
@@ -936,9 +954,15 @@ int pie_step_begin(pie_pool *pool) {
 int pie_set_extension_ratio(pie_pool *pool, float r) {
     if (!pool || r > 1.0f || r != r) return PIE_ERR_INVALID;
     if (r < 0.f) {
-        if (pool->ratio_mode == 0) pool->ratio = 0.0;  // Section 3.4.2: start with everything on the GPU
-        pool->ratio_mode = 2;
         if (!pool->cfg.timing) return PIE_ERR_INVALID;  // the controller needs the per-layer events
+        if (pool->ratio_mode == 0) {
+            // the controller takes over from the sets the caller established (all on the GPU gives 0: the paper's
+            // starting point, Section 3.4.2)
+            float cur = 0.f;
+            pie_get_extension_ratio(pool, &cur);
+            pool->ratio = cur;
+        }
+        pool->ratio_mode = 2;
     } else {
         pool->ratio_mode = 1;
         pool->ratio = r;
@@ -985,6 +1009,13 @@ int pie_controller_tick(pie_pool *pool, int32_t *changed) {
     if (changed) *changed = 0;
     if (!pool->cfg.timing) return PIE_OK;
     return evaluate_completed(pool, changed);
+}
+
+int pie_get_step_timeline(pie_pool *pool, float *ms, int64_t capacity) {
+    if (!pool || !ms) return PIE_ERR_INVALID;
+    if ((int64_t)pool->timeline.size() > capacity || pool->timeline.empty()) return PIE_ERR_INVALID;
+    std::copy(pool->timeline.begin(), pool->timeline.end(), ms);
+    return PIE_OK;
 }
 
 int pie_get_stats(pie_pool *pool, pie_stats *out) {

@@ -382,9 +382,10 @@ int pie_fifo_location(pie_fifo *f, int32_t layer) {
 }
 
 // state[0..3]: stalled flags of the last steps (newest last), state[4]: how many are valid,
-// state[5]: eps override, state[6]: u_hi override (0 = default).
+// state[5]: eps override, state[6]: u_hi override (0 = default), state[7]: steps left before the next increase.
 // Constants (the paper gives none): eps = 0.02, back off on 2 stalls within 4 steps, grow while the
-// link is busy for less than 0.9 of the compute time.
+// link is busy for less than 0.9 of the compute time, and after an increase wait 3 steps before the next one
+// (measurements arrive a few steps late: a change must be seen at work before it is built upon).
 double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
                              double swap_busy) {
     const double eps = state[5] > 0 ? state[5] : 0.02, u_hi = state[6] > 0 ? state[6] : 0.9;
@@ -404,8 +405,11 @@ double pie_controller_decide(double *state, double ratio, double step, double st
             ratio = std::max(0.0, ratio - step);
             state[4] = 0;  // start a fresh window after a change
         }
+    } else if (state[7] > 0) {
+        state[7] -= 1;
     } else if (swap_busy < u_hi * compute && ratio < 1.0) {
         ratio = std::min(1.0, ratio + step);
+        state[7] = 3;
     }
     return ratio;
 }
