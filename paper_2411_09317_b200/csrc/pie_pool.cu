@@ -242,7 +242,10 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
     return PIE_OK;
 }
 
-int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t n, int32_t mode) {
+// not_before: a compute ticket the copy must not start before (0 = none).  The decode loop uses it to start the
+// prefetch of layer l+1 when layer l starts computing (Section 3.3), not as early as the host happens to run ahead:
+// that keeps a unit on the host for as long as possible and the GPU staging share at a few layers' worth.
+int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t n, int32_t mode, int64_t not_before = 0) {
     if (!p) return PIE_ERR_INVALID;
     if (p->sticky != PIE_OK) return p->sticky;
     if (mode < PIE_MODE_AUTO || mode > PIE_MODE_COPY_ENGINE) return PIE_ERR_INVALID;
@@ -271,6 +274,7 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
     cudaStream_t stream = p->stream[queue];
     st = reserve_ticket_event(p, queue, ticket);
     if (st != PIE_OK) return st;
+    waits[PIE_Q_COMPUTE] = std::max(waits[PIE_Q_COMPUTE], not_before);
     for (int q = 1; q <= 3; ++q) {
         st = wait_ticket(p, stream, q, waits[q]);
         if (st != PIE_OK) { p->sticky = st; return st; }
@@ -1076,7 +1080,9 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
         st = plan_layer(pool, l, in_ids, out_ids);
         if (st != PIE_OK) return st;  // the GPU pool cannot take the next layer's share: nothing was enqueued for it
         if (L > 1 && !in_ids.empty()) {
-            st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode);
+            // starts when layer l starts, i.e. once the previous attention call has finished
+            st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode,
+                           pool->table->issued(PIE_Q_COMPUTE));
             if (st != PIE_OK) return st;
         }
         st = attention_call(pool, l, (const uint8_t *)q_all + l * q_stride, (uint8_t *)out_all + l * q_stride, block_table_dev,
