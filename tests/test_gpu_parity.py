@@ -292,3 +292,80 @@ def test_tiny_config_one_decode_step():
     assert stats["bytes_in"] == 3 * len(hs) * case.block_bytes
     assert stats["bytes_out"] == 2 * len(hs) * case.block_bytes
     pc.close()
+
+
+# ------------------------------------------------------------------ more paths: large batch, multi-step, recycling
+def test_large_batch_uses_the_separate_plan_kernel():
+    """More sequences than the in-kernel plan holds (1024): the chunk offsets come from plan_kernel."""
+    lens = synth.uniform_lengths(41, 1100, 0, 40)
+    case = Case(1, 4, 2, 64, F16, lens, seed=41, placement="random")
+    pc = PoolCase(case, split_tokens=16)
+    check_attention(case, pc, 0, edge=True)
+    pc.close()
+
+
+def test_multi_step_decode_with_append_matches_oracle_every_step():
+    """Five decode steps on a small GQA model, 40 % of the blocks host resident: outputs of every step and the final
+    bytes of every unit against the oracle (append, prefetch, write-back, next-token look-ahead)."""
+    lens = np.array([30, 63, 64, 65, 129, 7], dtype=np.int32)
+    steps = 5
+    case = Case(3, 8, 2, 128, BF16, lens, seed=42, host_frac=0.4, placement="random", extra_tokens=steps)
+    pc = PoolCase(case, timing=1)
+    dev = torch.device("cuda:0")
+    cur = lens.copy()
+    ctx_dev = torch.from_numpy(cur).to(dev)
+    for t in range(steps):
+        k_new = synth.tensor_bits(42, synth.STREAM_KNEW, (case.L, case.S, case.Hkv, case.D), case.dtype, offset=t * 10_000_000)
+        v_new = synth.tensor_bits(42, synth.STREAM_VNEW, (case.L, case.S, case.Hkv, case.D), case.dtype, offset=t * 10_000_000)
+        k_dev = torch.from_numpy(k_new.view(np.int16)).to(dev)
+        v_dev = torch.from_numpy(v_new.view(np.int16)).to(dev)
+        cur = cur + 1
+        ctx_dev.copy_(torch.from_numpy(cur))
+        torch.cuda.synchronize()
+        pie.pie_decode_step(pc.pool, pc.q.data_ptr(), pc.out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                            ctx_dev.data_ptr(), case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        pie.pie_sync(pc.pool)
+        case.ctx_lens = cur.copy()
+        for l in range(case.L):
+            oracle.append(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k_new[l], v_new[l],
+                          case.block_table, cur, case.Hkv, case.D)
+            want = oracle_attention(case, l)
+            got = synth.bits16_to_f32(pc.out[l].cpu().numpy().view(np.uint16), case.dtype)
+            assert np.all(np.abs(got - want) <= edge_tol(want, case.dtype)), (t, l)
+    for l in range(case.L):
+        for b in range(case.NB):
+            assert np.array_equal(pc.read_unit(l, b), pc.unit_bits(l, b)), (l, b)
+    pc.close()
+
+
+def test_block_free_and_reuse_and_nomem():
+    case = Case(2, 4, 4, 64, F16, [40, 20], seed=43)
+    pc = PoolCase(case, n_gpu_slots=2 * case.NB + 2, n_host_slots=4)
+    check_attention(case, pc, 0, edge=True)
+    # no room for another block on the GPU side beyond the 2 spare slots + 4 host slots
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_block_alloc(pc.pool, 1)
+    assert e.value.status == pie.PIE_ERR_NOMEM          # the pool has NB logical ids only
+    # free one sequence's blocks, allocate them again: slots are recycled behind the attention call that read them
+    ids = case.block_table[1, :2].copy()
+    pie.pie_block_free(pc.pool, ids)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_block_free(pc.pool, ids)
+    assert e.value.status == pie.PIE_ERR_INVALID
+    again = pie.pie_block_alloc(pc.pool, 2)
+    assert sorted(again.tolist()) == sorted(ids.tolist())
+    for l in range(case.L):
+        for b in again:
+            pie.pie_block_write(pc.pool, l, int(b), pc.unit_bits(l, int(b)))
+    check_attention(case, pc, 1, edge=True)
+    # swap lists: duplicates and unallocated ids are rejected and change nothing
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_swap_out(pc.pool, 0, [int(ids[0]), int(ids[0])])
+    assert e.value.status == pie.PIE_ERR_INVALID
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_swap_out(pc.pool, 0, np.arange(case.NB))   # only 4 host slots
+    assert e.value.status == pie.PIE_ERR_NOMEM
+    assert pie.pie_block_state(pc.pool, 0, 0)[0] == pie.PIE_GPU
+    pie.pie_swap_out(pc.pool, 0, [])                        # empty list: fine
+    pie.pie_sync(pc.pool)
+    pc.close()
