@@ -160,6 +160,9 @@ def timed_steps(dw, torch, n, append=True, mode=0):
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
     dw.sync()
     stats = []
+    # one more untimed step, enqueued right after the synchronisation: the first step on an idle GPU runs ~20 % slow
+    dw.advance_context()
+    dw.decode_step(append=append, mode=mode)
     with torch.cuda.stream(dw.s_compute):
         marks[0].record()
     for i in range(n):
@@ -221,7 +224,7 @@ def main():
     sweep_ratios = [0.0005, 0.001, 0.002, 0.004, 0.008]
     n_sweep = 8
     # every phase below appends one token per step
-    total_steps = (3 + args.steps) + (ramp + args.steps) + (3 + args.steps) + len(sweep_ratios) * 2 * (3 + n_sweep) + (3 + args.steps)
+    total_steps = (4 + args.steps) + (ramp + 2 + args.steps) + (4 + args.steps) + len(sweep_ratios) * 2 * (5 + n_sweep) + (3 + args.steps) + 8
     n_blocks = int(((wl.ctx_lens.astype(np.int64) + total_steps + 15) // 16).sum())
     r_cap = 0.02   # room in both pools for host-resident shares up to this ratio (+ 3 layers of staging)
     dw = DeviceWorkload(wl, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
@@ -360,7 +363,7 @@ def main():
     torch.cuda.empty_cache()
     n_conf = 3
     dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
-                        attn_ctas_per_sm=args.ctas_per_sm, extra_tokens=1 + n_conf)
+                        attn_ctas_per_sm=args.ctas_per_sm, extra_tokens=3 + n_conf)
     timed_steps(dw, torch, 1)  # warm-up: the first step fetches layer 0 on demand
     c0 = dw.ctx_lens.copy()
     s_b = pie.pie_get_stats(dw.pool)

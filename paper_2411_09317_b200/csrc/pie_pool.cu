@@ -32,7 +32,9 @@ constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list
     } while (0)
 
 struct LayerEvents {
-    cudaEvent_t pre = nullptr, go = nullptr, done = nullptr;  // compute stream: before wait, after wait, after layer
+    // compute stream: before the presence wait, after it, after the layer; copy streams: start and end of a list.
+    // pre, go, in0, out0 are owned; done, in1, out1 point at the ticket events of the calls (valid for EV_RING tickets)
+    cudaEvent_t pre = nullptr, go = nullptr, done = nullptr;
     cudaEvent_t in0 = nullptr, in1 = nullptr, out0 = nullptr, out1 = nullptr;
     bool has_in = false, has_out = false, has_compute = false, waited = false;
 };
@@ -284,12 +286,12 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
     st = do_copies(p, queue, p->v_src.data(), p->v_dst.data(), n_moved, p->v_moved.data(),
                    p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream);
     if (st != PIE_OK) { p->sticky = st; return st; }
-    if (le) {
-        PIE_CUDA(cudaEventRecord(queue == PIE_Q_IN ? le->in1 : le->out1, stream));
-        (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
-    }
     st = record_ticket(p, queue, ticket);
     if (st != PIE_OK) { p->sticky = st; return st; }
+    if (le) {
+        (queue == PIE_Q_IN ? le->in1 : le->out1) = p->ticket_ev[queue][ticket % EV_RING];
+        (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
+    }
     (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)n_moved * (double)p->block_bytes;
     return PIE_OK;
 }
@@ -341,7 +343,7 @@ void destroy_pool(pie_pool *p) {
         if (p->list_events[i]) cudaEventDestroy(p->list_events[i]);
     for (int k = 0; k < TIMING_RING; ++k)
         for (LayerEvents &e : p->lev[k])
-            for (cudaEvent_t ev : {e.pre, e.go, e.done, e.in0, e.in1, e.out0, e.out1})
+            for (cudaEvent_t ev : {e.pre, e.go, e.in0, e.out0})
                 if (ev) cudaEventDestroy(ev);
     if (p->own_streams)
         for (int q = 1; q <= 3; ++q)
@@ -403,15 +405,16 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     st = reserve_ticket_event(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) return st;
     LayerEvents *le = timing_slot(p, layer);
-    if (le) PIE_CUDA(cudaEventRecord(le->pre, stream));
+    if (le) {
+        // every record costs the stream about a microsecond: the "before the wait" mark only when there is a wait
+        le->waited = waits[1] > p->table->done(1) || waits[2] > p->table->done(2);
+        if (le->waited) PIE_CUDA(cudaEventRecord(le->pre, stream));
+    }
     for (int qd = 1; qd <= 2; ++qd) {
         st = wait_ticket(p, stream, qd, waits[qd]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
-    if (le) {
-        le->waited = waits[1] > p->table->done(1) || waits[2] > p->table->done(2);
-        PIE_CUDA(cudaEventRecord(le->go, stream));
-    }
+    if (le) PIE_CUDA(cudaEventRecord(le->go, stream));
     pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
                       p->cfg.n_gpu_slots};
     pie::AttnLaunch a{};
@@ -436,12 +439,12 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         p->sticky = PIE_ERR_CUDA;
         return PIE_ERR_CUDA;
     }
-    if (le) {
-        PIE_CUDA(cudaEventRecord(le->done, stream));
-        le->has_compute = true;
-    }
     st = record_ticket(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) p->sticky = st;
+    if (le && st == PIE_OK) {
+        le->done = p->ticket_ev[PIE_Q_COMPUTE][ticket % EV_RING];
+        le->has_compute = true;
+    }
     return st;
 }
 
@@ -632,13 +635,14 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
         p->stream[PIE_Q_OUT] = (cudaStream_t)cfg->copy_out_stream;
     }
     for (int q = 1; q <= 3; ++q)
-        for (int i = 0; i < EV_RING; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->ticket_ev[q][i], cudaEventDisableTiming), PIE_ERR_CUDA);
+        for (int i = 0; i < EV_RING; ++i)  // with timing on, a ticket's event doubles as the "end" mark of its work
+            PIE_TRY(cudaEventCreateWithFlags(&p->ticket_ev[q][i], cfg->timing ? cudaEventDefault : cudaEventDisableTiming), PIE_ERR_CUDA);
     for (int i = 0; i < LIST_EVENTS; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->list_events[i], cudaEventDisableTiming), PIE_ERR_CUDA);
     if (cfg->timing) {
         for (int k = 0; k < TIMING_RING; ++k) {
             p->lev[k].resize((size_t)cfg->n_layers);
             for (LayerEvents &e : p->lev[k])
-                for (cudaEvent_t *ev : {&e.pre, &e.go, &e.done, &e.in0, &e.in1, &e.out0, &e.out1})
+                for (cudaEvent_t *ev : {&e.pre, &e.go, &e.in0, &e.out0})
                     PIE_TRY(cudaEventCreate(ev), PIE_ERR_CUDA);
         }
     }
@@ -864,7 +868,7 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
                 PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
                 stall += std::max(0.0, (double)ms - 0.004);
             }
-            if (!first) first = e.pre;
+            if (!first) first = e.waited ? e.pre : e.go;
             last = e.done;
         }
         if (e.has_in) {
@@ -883,7 +887,7 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         pool->timeline.assign(ev.size() * 7, -1.f);
         for (size_t l = 0; l < ev.size(); ++l) {
             LayerEvents &e = ev[l];
-            cudaEvent_t list[7] = {e.pre, e.go, e.done, e.in0, e.in1, e.out0, e.out1};
+            cudaEvent_t list[7] = {e.waited ? e.pre : e.go, e.go, e.done, e.in0, e.in1, e.out0, e.out1};
             const bool has[7] = {e.has_compute, e.has_compute, e.has_compute, e.has_in, e.has_in, e.has_out, e.has_out};
             for (int j = 0; j < 7; ++j)
                 if (has[j]) {
