@@ -95,58 +95,89 @@ class ClockSampler:
 # -------------------------------------------------------------------------------------------------------
 # CPU baseline: the oracle, as it stands, on a bounded sample of the same workload
 # -------------------------------------------------------------------------------------------------------
-def oracle_sample(wl, n_seqs_sample=6, min_seconds=10.0, max_seconds=30.0):
-    """Time the oracle's paged attention of layer 0 for the first `n_seqs_sample` sequences (contents from the
-    numpy generator), all host cores, repeated until `min_seconds` of CPU work.  -> dict for the JSON line."""
-    import oracle
-    block_table, nblk, NB = wl.tables()
-    S = min(n_seqs_sample, wl.n_seqs)
-    ctx = (wl.ctx_lens[:S] + 1).astype(np.int32)
-    ids = np.unique(np.concatenate([block_table[s, :nblk[s]] for s in range(S)]))
-    elems = wl.block_bytes // 2
-    pool = np.zeros((len(ids), elems), dtype=np.uint16)
-    slot_of = np.full(NB, -1, dtype=np.int32)
-    for i, b in enumerate(ids):
-        pool[i] = synth.kv_unit_bits(wl.seed, 0, int(b), NB, wl.n_kv_heads, wl.head_dim, wl.dtype).ravel()
-        slot_of[b] = i
-    side = np.zeros(NB, dtype=np.int32)
-    q = synth.tensor_bits(wl.seed, synth.STREAM_Q, (wl.n_seqs, wl.n_q_heads, wl.head_dim), wl.dtype)[:S]
-    cores = os.cpu_count() or 1
-    nbytes = int(ctx.astype(np.int64).sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2 + 2 * S * wl.n_q_heads * wl.head_dim * 2 \
-        + 4 * (int(((ctx + 15) // 16).sum()) + S)
-    reps, t0 = 0, time.perf_counter()
-    while True:
-        oracle.paged_attention(pool, pool, side, np.maximum(slot_of, 0), q, block_table[:S], ctx, wl.n_q_heads,
-                               wl.n_kv_heads, wl.head_dim, wl.dtype, 1.0 / np.sqrt(wl.head_dim), "f32", nthreads=cores)
+CONFIG_WORKLOAD = ("llama2_7b: 32 layers, 32q/32kv heads, head_dim 128, fp16, 16-token blocks, batch 64, contexts "
+                   "U[512,2048] (+1 token per step), per-layer prefetch; host-resident share chosen by the adaptive "
+                   "controller (the configured 30 % run is under as_configured)")
+
+
+class OracleSample:
+    """The oracle's paged attention of layer 0 on the first `n_seqs_sample` sequences (contents from the numpy
+    generator): built once, timed as often as asked.  The oracle is used as it stands, all host cores."""
+
+    def __init__(self, wl, n_seqs_sample=6):
+        import oracle
+        self.oracle, self.wl = oracle, wl
+        self.block_table, nblk, NB = wl.tables()
+        S = self.S = min(n_seqs_sample, wl.n_seqs)
+        self.ctx = (wl.ctx_lens[:S] + 1).astype(np.int32)
+        ids = np.unique(np.concatenate([self.block_table[s, :nblk[s]] for s in range(S)]))
+        elems = wl.block_bytes // 2
+        self.pool = np.zeros((len(ids), elems), dtype=np.uint16)
+        slot_of = np.zeros(NB, dtype=np.int32)
+        for i, b in enumerate(ids):
+            self.pool[i] = synth.kv_unit_bits(wl.seed, 0, int(b), NB, wl.n_kv_heads, wl.head_dim, wl.dtype).ravel()
+            slot_of[b] = i
+        self.slot_of, self.side = slot_of, np.zeros(NB, dtype=np.int32)
+        self.q = synth.tensor_bits(wl.seed, synth.STREAM_Q, (wl.n_seqs, wl.n_q_heads, wl.head_dim), wl.dtype)[:S]
+        self.cores = os.cpu_count() or 1
+        ctx64 = self.ctx.astype(np.int64)
+        self.nbytes = int(ctx64.sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2 + 2 * S * wl.n_q_heads * wl.head_dim * 2 \
+            + 4 * (int(((ctx64 + 15) // 16).sum()) + S)
+
+    def run_once(self):
+        wl = self.wl
+        t0 = time.perf_counter()
+        self.oracle.paged_attention(self.pool, self.pool, self.side, self.slot_of, self.q, self.block_table[:self.S], self.ctx,
+                                    wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, 1.0 / np.sqrt(wl.head_dim), "f32",
+                                    nthreads=self.cores)
+        return time.perf_counter() - t0
+
+    def describe(self, reps, seconds):
+        return (f"layer 0, first {self.S} of {self.wl.n_seqs} sequences ({int(self.ctx.sum())} tokens), fp32 oracle, "
+                f"{reps} passes in {seconds:.1f} s")
+
+    def swap_memcpy_gbs(self, n_blocks=512):
+        """The oracle's swap (block memcpy) of a scattered list, for the record."""
+        BB = self.wl.block_bytes
+        src_pool = synth.random_bytes(5, n_blocks * BB).copy()
+        dst_pool = np.zeros(n_blocks * BB, dtype=np.uint8)
+        src = synth.seeded_permutation(5, n_blocks, salt=3).astype(np.int32)
+        dst = synth.seeded_permutation(5, n_blocks, salt=4).astype(np.int32)
+        t0 = time.perf_counter()
+        self.oracle.swap_raw(dst_pool, src_pool, BB, src, dst)
+        return n_blocks * BB / (time.perf_counter() - t0) / 1e9
+
+
+def oracle_sample(wl, min_seconds=10.0):
+    """cpu_baseline: about min_seconds of oracle work on the sample -> dict for the JSON line."""
+    smp = OracleSample(wl)
+    reps, total = 0, 0.0
+    while total < min_seconds:
+        total += smp.run_once()
         reps += 1
-        dt = time.perf_counter() - t0
-        if dt >= min_seconds or dt >= max_seconds:
-            break
-    return {"value": nbytes * reps / dt / 1e9, "unit": "GB/s", "cores": min(cores, S), "kind": "oracle",
-            "sample": f"layer 0, first {S} of {wl.n_seqs} sequences ({int(ctx.sum())} tokens), fp32 oracle, "
-                      f"{reps} passes in {dt:.1f} s", "seconds": dt, "bytes_per_pass": nbytes}
+    return {"value": smp.nbytes * reps / total / 1e9, "unit": "GB/s", "cores": min(smp.cores, smp.S), "kind": "oracle",
+            "sample": smp.describe(reps, total), "swap_memcpy_gbs_1thread": smp.swap_memcpy_gbs()}
 
 
 def run_reference(args):
-    """--impl reference: the CPU oracle on the host cores, same metric and workload, bounded sample per step."""
+    """--impl reference: the CPU oracle on the host cores, same metric and workload, a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     wl = synth.workload(WORKLOAD, args.scale)
     import oracle
     oracle.build()
-    times, info = [], None
-    for i in range(args.warmup + args.steps):
-        info = oracle_sample(wl, n_seqs_sample=4, min_seconds=0.0, max_seconds=0.0)
-        if i >= args.warmup:
-            times.append(info["seconds"])
+    smp = OracleSample(wl, n_seqs_sample=6)
+    times = [smp.run_once() for _ in range(args.warmup + args.steps)][args.warmup:]
     ms = float(np.mean(times)) * 1e3
-    value = info["bytes_per_pass"] / (ms * 1e-3) / 1e9
+    value = smp.nbytes / (ms * 1e-3) / 1e9
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "gpu_launches": 0,
-            "config": {"workload": f"{WORKLOAD} (Llama-2-7B-shaped KV), CPU oracle on a sample", "scale": args.scale},
-            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": info["cores"], "kind": "oracle", "sample": info["sample"]},
+            "config": {"workload": CONFIG_WORKLOAD, "scale": args.scale,
+                       "note": "CPU oracle (test infrastructure, deliberately plain) on a bounded sample of the workload per step"},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": min(smp.cores, smp.S), "kind": "oracle",
+                             "sample": smp.describe(args.steps, sum(times))},
             "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -163,6 +194,8 @@ def timed_steps(dw, torch, n, append=True, mode=0):
     # one more untimed step, enqueued right after the synchronisation: the first step on an idle GPU runs ~20 % slow
     dw.advance_context()
     dw.decode_step(append=append, mode=mode)
+    timed_steps.before = pie.pie_get_stats(dw.pool)      # byte counters at the start of the timed steps
+    timed_steps.ctx_before = dw.ctx_lens.copy()
     with torch.cuda.stream(dw.s_compute):
         marks[0].record()
     for i in range(n):
@@ -172,6 +205,7 @@ def timed_steps(dw, torch, n, append=True, mode=0):
         with torch.cuda.stream(dw.s_compute):
             marks[i + 1].record()
     dw.sync()
+    timed_steps.after = pie.pie_get_stats(dw.pool)
     timed_steps.last_per_step = [marks[i].elapsed_time(marks[i + 1]) for i in range(n)]
     return marks[0].elapsed_time(marks[n]), stats
 
@@ -247,9 +281,9 @@ def main():
     # ---- phase 1: resident baseline (ratio 0: nothing moves) ---------------------------------------------------
     pie.pie_set_extension_ratio(dw.pool, 0.0)
     timed_steps(dw, torch, 3)
-    c0 = dw.ctx_lens.copy()
     barrier()
     ms_res, st_res = timed_steps(dw, torch, args.steps)
+    c0 = timed_steps.ctx_before
     resident_gbs = bytes_of_steps(args.steps, c0) / (ms_res * 1e-3) / 1e9
     resident_med = median_gbs(bytes_of_steps(args.steps, c0), args.steps)
 
@@ -259,13 +293,11 @@ def main():
     sampler = ClockSampler(local)   # started before the ramp (nvidia-smi takes a while to come up); same load throughout
     sampler.start()
     timed_steps(dw, torch, ramp)
-    c0 = dw.ctx_lens.copy()
-    s_before = pie.pie_get_stats(dw.pool)
     barrier()
     ms_run, st_run = timed_steps(dw, torch, args.steps)
+    c0, s_before, s_after = timed_steps.ctx_before, timed_steps.before, timed_steps.after
     barrier()
     clocks = sampler.stop()
-    s_after = pie.pie_get_stats(dw.pool)
     ms_run = max_over_ranks(ms_run)
     step_bytes = bytes_of_steps(args.steps, c0)
     value_med = median_gbs(step_bytes, args.steps)
@@ -281,8 +313,8 @@ def main():
     # slow-down is taken in GB/s against the mean of the resident runs on both sides
     pie.pie_set_extension_ratio(dw.pool, 0.0)
     timed_steps(dw, torch, 3)
-    c0 = dw.ctx_lens.copy()
     ms_res_b, _ = timed_steps(dw, torch, args.steps)
+    c0 = timed_steps.ctx_before
     resident_after_gbs = bytes_of_steps(args.steps, c0) / (ms_res_b * 1e-3) / 1e9
     resident_after_med = median_gbs(bytes_of_steps(args.steps, c0), args.steps)
     slowdown = 0.5 * (resident_med + resident_after_med) / value_med - 1.0
@@ -298,10 +330,8 @@ def main():
     def run_fixed(r, n):
         pie.pie_set_extension_ratio(dw.pool, r)
         timed_steps(dw, torch, 3)
-        c = dw.ctx_lens.copy()
-        sb = pie.pie_get_stats(dw.pool)
         ms, _ = timed_steps(dw, torch, n)
-        sa = pie.pie_get_stats(dw.pool)
+        c, sb, sa = timed_steps.ctx_before, timed_steps.before, timed_steps.after
         return {"ratio": r, "attn_gbs": median_gbs(bytes_of_steps(n, c), n), "attn_gbs_mean": bytes_of_steps(n, c) / (ms * 1e-3) / 1e9,
                 "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / (ms * 1e-3) / 1e9,
                 "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / (ms * 1e-3) / 1e9}
@@ -365,10 +395,8 @@ def main():
     dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
                         attn_ctas_per_sm=args.ctas_per_sm, extra_tokens=3 + n_conf)
     timed_steps(dw, torch, 1)  # warm-up: the first step fetches layer 0 on demand
-    c0 = dw.ctx_lens.copy()
-    s_b = pie.pie_get_stats(dw.pool)
     ms_conf, st_conf = timed_steps(dw, torch, n_conf)
-    s_a = pie.pie_get_stats(dw.pool)
+    c0, s_b, s_a = timed_steps.ctx_before, timed_steps.before, timed_steps.after
     as_configured = {
         "host_fraction": wl.host_frac, "steps": n_conf, "ms_per_step": ms_conf / n_conf,
         "attn_gbs": bytes_of_steps(n_conf, c0) / (ms_conf * 1e-3) / 1e9,
@@ -392,17 +420,13 @@ def main():
         import oracle
         oracle.build()
         cpu = oracle_sample(wl)
-        cpu.pop("seconds", None)
-        cpu.pop("bytes_per_pass", None)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value_1gpu * world, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": ramp, "ms_per_step": ms_run / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16", "data": "synthetic", "gpu_launches": n_launch,
-            "config": {"workload": "llama2_7b: 32 layers, 32q/32kv heads, head_dim 128, fp16, 16-token blocks, batch 64, "
-                                   "contexts U[512,2048] (+1 token per step), per-layer prefetch; host-resident share "
-                                   "chosen by the adaptive controller (the configured 30 % run is under as_configured)",
+            "config": {"workload": CONFIG_WORKLOAD,
                        "scale": args.scale, "n_layers": L, "n_seqs": wl.n_seqs, "l2": "inputs larger than L2 "
                        f"({bytes_layer0 / 1e9:.2f} GB of distinct KV per layer call)", "parallelism": "replicas only"},
             "clocks": clocks,
