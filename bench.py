@@ -306,8 +306,8 @@ def main():
     swapped_out = s_after["bytes_out"] - s_before["bytes_out"]
     comp_ms = [s["last_step_compute_ms"] for s in st_run if s["steps_measured"] > 0]
     attn_ms_layer = float(np.mean(comp_ms)) / L if comp_ms else float("nan")
-    # one attention kernel per layer call, plus one swap kernel (or one table-patch kernel after copy-engine copies) per list
-    n_launch = int(L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
+    # attention + combine kernel per layer call, plus one swap kernel (or one table-patch kernel after copy-engine copies) per list
+    n_launch = int(2 * L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
                    (s_after["calls_copy_engine"] - s_before["calls_copy_engine"]))
     # resident again right after (A/B/A): clocks drift under the power cap and the contexts keep growing, so the
     # slow-down is taken in GB/s against the mean of the resident runs on both sides
@@ -411,7 +411,7 @@ def main():
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "traffic": int(TRAFFIC_PER_ALG_BYTE * bytes_layer0),
                 "traffic_note": "ncu dram bytes of a quarter-scale launch scaled by the KV bytes read", "peak_kind": peak_kind,
-                "kernel": "paged_decode_attn_kernel (plan, append and combine fused; per-layer event span on the compute stream)",
+                "kernel": "paged_decode_attn_kernel (plan and append fused) + combine_kernel: per-layer event span on the compute stream",
                 "alg_bytes_per_launch": bytes_layer0, "ms_per_launch": attn_ms_layer, "hbm_copy_probe_gbs": hbm_probe,
                 "frac_of_nominal_8tbs": (achieved / 8000.0) if achieved else None}
 

@@ -248,9 +248,11 @@ plan_kernel(const int32_t *__restrict__ ctx_lens, int32_t n_seqs, int32_t max_to
 //     ceil(ctx / split) over the sequences);
 //   - the KV append (Section 3.2: each token iteration updates each layer's cache): the warp that owns the
 //     tile holding position ctx-1 patches the new token's K and V rows into the staged tile and into the pool;
-//   - the combine: a sequence with one chunk is normalised and written directly; otherwise each item writes
-//     an fp32 partial (m, l, unnormalised acc) and the CTA that completes a (sequence, KV head) last merges
-//     its chunks in chunk order with the log-sum-exp rule, normalises and rounds to 16 bits (nearest even).
+//   - the combine of single-chunk sequences: normalised and rounded to 16 bits (nearest even) right here.  A
+//     sequence with several chunks gets one fp32 partial (m, l, unnormalised acc) per item, merged in chunk order
+//     by combine_kernel right after.  (A fused "last CTA to finish the pair merges it" variant was measured: its
+//     per-item release/acquire atomics and the serial merges cost more than the extra launch, badly so for 8-head
+//     groups and long contexts.)
 // Every reduction order depends only on the logical token order and on ctx_len (tile -> warp by index, warps
 // merged in warp order, chunks merged in chunk order), never on slot ids, on which CTA ran an item or on
 // timing, so a run with swapped blocks reproduces a resident run bit for bit.
@@ -266,11 +268,12 @@ struct AttnParams {
     const int32_t *ctx_lens;
     const int32_t *slot_table;
     const int32_t *chunk_off_global;  // used when n_seqs > ATT_SMEM_SEQS (filled by plan_kernel)
+    int32_t *chunk_off_out;           // [n_seqs + 1]: the plan, written by CTA 0 for the combine kernel
     const uint4 *k_new, *v_new;       // optional append
     uint4 *pool;
     float *part_o;
     float *part_ml;
-    int32_t *counters;  // [0] next item, [1] CTAs that have left, [64 + s * Hkv + kvh] chunks done
+    int32_t *counters;  // [0] next item, [1] CTAs that have left
     int32_t *status;
     int64_t n_gpu_slots;
     int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d, max_chunks;
@@ -287,7 +290,7 @@ struct AttnSmem {
     static constexpr int OFF_MO = OFF_Q + ATT_QD * Q_BYTES;
     static constexpr int OFF_ML = OFF_MO + NW * 8 * MO_STRIDE * 4;
     static constexpr int OFF_BAR = OFF_ML + NW * 8 * 2 * 4;              // full[STAGES], empty[STAGES], qfull[QD], qempty[QD]
-    static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 2 * ATT_QD) * 8;  // abort, is_last, q_item[QD]
+    static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 2 * ATT_QD) * 8;  // abort, -, token count, -, q_item[QD]
     static constexpr int OFF_CO = OFF_MISC + 64;                          // chunk offsets [ATT_SMEM_SEQS + 1]
     static constexpr int BYTES = OFF_CO + (ATT_SMEM_SEQS + 1) * 4 + 12;
 };
@@ -361,7 +364,6 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const uint32_t bar_qempty = bar_qfull + ATT_QD * 8;
     volatile int32_t *misc = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_MISC);
     volatile int32_t *abort_flag = misc;      // [0]
-    volatile int32_t *is_last = misc + 1;     // [1]
     volatile int32_t *q_item = misc + 4;      // [4 .. 4 + QD)
     int32_t *co_smem = reinterpret_cast<int32_t *>(smem + SM::OFF_CO);
 
@@ -522,45 +524,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const int k_tok = lr + (lm & 1) * 8, k_csel = lm >> 1;   // K: matrices {tok 0-7, tok 8-15} x {chunk, chunk+1}
     const int v_tok = lr + (lm >> 1) * 8, v_csel = lm & 1;   // V (transposed): {chunk, chunk+1} x {tok 0-7, tok 8-15}
 
-    // sequences without any token get a zero row (nobody else writes them)
+    // CTA 0: the chunk offsets for the combine kernel; sequences without any token get a zero row (nobody else writes them)
+    if (blockIdx.x == 0 && co_in_smem)
+        for (int32_t s = tid; s <= p.n_seqs; s += ATT_NW * 32) p.chunk_off_out[s] = n_items == 0 ? 0 : co[s];
     if (blockIdx.x == 0)
         for (int32_t s = 0; s < p.n_seqs; ++s)
             if (co[s + 1] == co[s] || n_items == 0)
                 for (int e = tid; e < p.n_q_heads * D; e += ATT_NW * 32) p.out[(int64_t)s * p.n_q_heads * D + e] = 0;
-
-    // Completion of a (sequence, KV head) is signalled one item late: thread 0 bumps the pair's counter after an
-    // item's last barrier and looks at the answer only when the next item has been computed, so nobody waits
-    // for the atomic's round trip.  prev_* describe the item whose answer is still outstanding.
-    int32_t prev_s = -1, prev_kvh = 0, prev_nchunks = 0, prev_chunk0 = 0, prev_old = 0;
-
-    // merge the chunks of (s, kvh) in chunk order, normalise, round (run by the CTA that completed the pair)
-    auto final_combine = [&](int32_t cs, int32_t ckvh, int32_t nchunks, int32_t chunk0) {
-        const int64_t row0 = ((int64_t)cs * p.n_q_heads + (int64_t)ckvh * p.group) * D;
-        for (int e = tid; e < p.group * D; e += ATT_NW * 32) {
-            const int g = e / D, d = e - g * D;
-            float mm = -INFINITY;
-            for (int32_t c = 0; c < nchunks; ++c)
-                mm = fmaxf(mm, __ldcg(p.part_ml + (((int64_t)(chunk0 + c) * p.n_kv_heads + ckvh) * p.group + g) * 2));
-            float acc = 0.f, ll = 0.f;
-            for (int32_t c = 0; c < nchunks; ++c) {
-                const int64_t idx = ((int64_t)(chunk0 + c) * p.n_kv_heads + ckvh) * p.group + g;
-                const float mc = __ldcg(p.part_ml + idx * 2);
-                const float wt = mc == -INFINITY ? 0.f : fast_exp2(mc - mm);
-                ll += __ldcg(p.part_ml + idx * 2 + 1) * wt;
-                acc += __ldcg(p.part_o + idx * D + d) * wt;
-            }
-            const float r = acc * (ll > 0.f ? 1.f / ll : 0.f);
-            p.out[row0 + e] = BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(r)) : __half_as_ushort(__float2half_rn(r));
-        }
-    };
-    auto publish_prev = [&]() {  // thread 0: was this CTA the last to finish the previous item's pair?
-        int32_t last = 0;
-        if (prev_s >= 0 && prev_nchunks > 1 && prev_old == prev_nchunks - 1) {
-            last = 1;
-            p.counters[64 + prev_s * p.n_kv_heads + prev_kvh] = 0;  // ready for the next launch
-        }
-        *is_last = last;
-    };
 
     for (;;) {
         const uint32_t qs = qn % ATT_QD;
@@ -718,7 +688,6 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 ml[(warp * 8 + c2 + 1) * 2 + 1] = l1;
             }
         }
-        if (tid == 0) publish_prev();
         consumer_sync<NCONS>();
         const int64_t out_row0 = ((int64_t)it.s * p.n_q_heads + (int64_t)it.kvh * p.group) * D;
         for (int e = tid; e < p.group * D; e += ATT_NW * 32) {
@@ -746,30 +715,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 }
             }
         }
-        if (*is_last) final_combine(prev_s, prev_kvh, prev_nchunks, prev_chunk0);  // the previous item's pair is complete
-        // last barrier of the item (partials buffer free again) doubles as a uniform vote on the abort flag
-        if (consumer_vote<NCONS>(*abort_flag != 0)) {
-            prev_s = -1;
-            break;
-        }
-        // every thread's partial stores precede the barrier above; a release by thread 0 after it covers them all
-        if (tid == 0 && it.nchunks > 1)
-            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
-                         : "=r"(prev_old)
-                         : "l"(p.counters + 64 + it.s * p.n_kv_heads + it.kvh)
-                         : "memory");
-        prev_s = it.s;
-        prev_kvh = it.kvh;
-        prev_nchunks = it.nchunks;
-        prev_chunk0 = it.chunk0;
+        // last barrier of the item (merge buffer free again) doubles as a uniform vote on the abort flag
+        if (consumer_vote<NCONS>(*abort_flag != 0)) break;
         if (lane == 0) mbar_arrive(bar_qempty + 8 * qs);
         ++qn;
-    }
-    // the answer for the last item is still outstanding
-    if (prev_s >= 0 && prev_nchunks > 1) {
-        if (tid == 0) publish_prev();
-        consumer_sync<NCONS>();
-        if (*is_last) final_combine(prev_s, prev_kvh, prev_nchunks, prev_chunk0);
     }
     // the last CTA to leave resets the work counter for the next launch (every CTA has drawn its end marker by then)
     if (tid == 0) {
@@ -778,6 +727,94 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             p.counters[0] = 0;
             p.counters[1] = 0;
         }
+    }
+}
+
+// =====================================================================================================
+// Combine: one CTA per (sequence, KV head, 32-wide slice of head_dim) merges the sequence's chunk partials in chunk
+// order with the log-sum-exp rule, normalises and rounds to the 16-bit output type (nearest even).  Sequences with
+// fewer than two chunks were finished by the attention kernel.  The per-(head, chunk) weights are computed once in
+// shared memory; the accumulation keeps eight 16-byte loads in flight per thread.
+// =====================================================================================================
+constexpr int COMB_THREADS = 64;
+constexpr int COMB_CAP = 256;  // chunks per sequence handled through shared memory; beyond that, plain loops
+
+template <int D, bool BF16>
+__global__ void __launch_bounds__(COMB_THREADS)
+combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, const int32_t *__restrict__ chunk_off,
+               uint16_t *__restrict__ out, int32_t n_q_heads, int32_t n_kv_heads, int32_t group) {
+    __shared__ float wbuf[8][COMB_CAP];
+    __shared__ float lbuf[8][COMB_CAP];
+    const int tid = threadIdx.x;
+    const int32_t s = blockIdx.x / n_kv_heads, kvh = blockIdx.x - s * n_kv_heads;
+    const int32_t chunk0 = chunk_off[s], nchunks = chunk_off[s + 1] - chunk0;
+    if (nchunks < 2) return;
+    const int d_lo = blockIdx.y * 32;  // this CTA's slice of head_dim
+    const int64_t row0 = ((int64_t)s * n_q_heads + (int64_t)kvh * group) * D;
+    if (nchunks <= COMB_CAP) {
+        for (int idx = tid; idx < group * nchunks; idx += COMB_THREADS) {
+            const int g = idx / nchunks, c = idx - g * nchunks;
+            const int64_t id = ((int64_t)(chunk0 + c) * n_kv_heads + kvh) * group + g;
+            wbuf[g][c] = part_ml[id * 2];
+            lbuf[g][c] = part_ml[id * 2 + 1];
+        }
+        __syncthreads();
+        if (tid < group) {
+            float *w = wbuf[tid], *l = lbuf[tid];
+            float mm = -INFINITY;
+            for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, w[c]);
+            float ll = 0.f;
+            for (int32_t c = 0; c < nchunks; ++c) {
+                const float wt = w[c] == -INFINITY ? 0.f : fast_exp2(w[c] - mm);
+                ll += l[c] * wt;
+                w[c] = wt;
+            }
+            l[0] = ll > 0.f ? 1.f / ll : 0.f;
+        }
+        __syncthreads();
+        for (int e4 = tid; e4 < group * 8; e4 += COMB_THREADS) {  // 8 float4 pieces per head in a 32-wide slice
+            const int g = e4 >> 3, d = d_lo + (e4 & 7) * 4;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int32_t c0 = 0; c0 < nchunks; c0 += 8) {
+                float4 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (c0 + j < nchunks) {
+                        const int64_t id = ((int64_t)(chunk0 + c0 + j) * n_kv_heads + kvh) * group + g;
+                        v[j] = *reinterpret_cast<const float4 *>(part_o + id * D + d);
+                    }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (c0 + j < nchunks) {
+                        const float wt = wbuf[g][c0 + j];
+                        acc.x += v[j].x * wt;
+                        acc.y += v[j].y * wt;
+                        acc.z += v[j].z * wt;
+                        acc.w += v[j].w * wt;
+                    }
+            }
+            const float inv = lbuf[g][0];
+            uint2 r;
+            r.x = pack2<BF16>(acc.x * inv, acc.y * inv);
+            r.y = pack2<BF16>(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2 *>(out + row0 + g * D + d) = r;
+        }
+        return;
+    }
+    for (int e = tid; e < group * 32; e += COMB_THREADS) {  // very many chunks: plain loops
+        const int g = e >> 5, d = d_lo + (e & 31);
+        float mm = -INFINITY;
+        for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, part_ml[(((int64_t)(chunk0 + c) * n_kv_heads + kvh) * group + g) * 2]);
+        float acc = 0.f, ll = 0.f;
+        for (int32_t c = 0; c < nchunks; ++c) {
+            const int64_t idx = ((int64_t)(chunk0 + c) * n_kv_heads + kvh) * group + g;
+            const float mc = part_ml[idx * 2];
+            const float wt = mc == -INFINITY ? 0.f : fast_exp2(mc - mm);
+            ll += part_ml[idx * 2 + 1] * wt;
+            acc += part_o[idx * D + d] * wt;
+        }
+        const float r = acc * (ll > 0.f ? 1.f / ll : 0.f);
+        out[row0 + g * D + d] = BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(r)) : __half_as_ushort(__float2half_rn(r));
     }
 }
 
@@ -864,7 +901,8 @@ int attn_smem_bytes(int head_dim) { return head_dim == 128 ? AttnSmem<128, 4, 2>
 // lands on an idle SM first could keep attention CTAs off that SM until it has finished.
 static cudaError_t prefer_max_shared() {
     const void *fns[] = {(const void *)swap_kernel, (const void *)patch_kernel, (const void *)patch_from_list_kernel,
-                         (const void *)plan_kernel};
+                         (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
+                         (const void *)combine_kernel<64, true>, (const void *)combine_kernel<64, false>};
     for (const void *f : fns) {
         cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
@@ -882,7 +920,7 @@ cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_s
     });
 }
 
-int64_t attn_counter_words(int32_t max_seqs, int32_t n_kv_heads) { return 64 + (int64_t)max_seqs * n_kv_heads; }
+int64_t attn_counter_words(int32_t, int32_t) { return 64; }  // [0] next item, [1] CTAs that have left
 
 cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
                              int use3d, cudaStream_t stream) {
@@ -900,6 +938,7 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.ctx_lens = a.ctx_lens;
     p.slot_table = a.slot_table;
     p.chunk_off_global = sc.chunk_off;
+    p.chunk_off_out = sc.chunk_off;
     p.k_new = (const uint4 *)a.k_new;
     p.v_new = (const uint4 *)a.v_new;
     p.pool = (uint4 *)a.gpu_pool;
@@ -919,10 +958,26 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.max_chunks = (int32_t)(sc.max_items / sh.n_kv_heads);
     p.scale_log2e = a.scale * 1.4426950408889634f;
     if (a.k_new == nullptr || a.v_new == nullptr) p.k_new = p.v_new = nullptr;
-    return dispatch_variant(sh.head_dim, sh.dtype, a.variant, [&](auto kernel, int smem, int nw) -> cudaError_t {
+    cudaError_t e = dispatch_variant(sh.head_dim, sh.dtype, a.variant, [&](auto kernel, int smem, int nw) -> cudaError_t {
         kernel<<<a.grid, (nw + 1) * 32, smem, stream>>>(map, p);
         return cudaGetLastError();
     });
+    if (e != cudaSuccess) return e;
+    // merge the partials of sequences that span several chunks (CTAs of single-chunk sequences return at once)
+    const dim3 cgrid((unsigned)(a.n_seqs * sh.n_kv_heads), (unsigned)(sh.head_dim / 32));
+    uint16_t *out = (uint16_t *)a.out;
+    if (sh.head_dim == 128) {
+        if (sh.dtype == PIE_BF16)
+            combine_kernel<128, true><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
+        else
+            combine_kernel<128, false><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
+    } else {
+        if (sh.dtype == PIE_BF16)
+            combine_kernel<64, true><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
+        else
+            combine_kernel<64, false><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
+    }
+    return cudaGetLastError();
 }
 
 }  // namespace pie
