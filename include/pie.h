@@ -239,8 +239,7 @@ int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps);
  *   stream      a cudaStream_t
  * The split-K scratch (chunk offsets, fp32 partials) is a static device array of PIE_NOALLOC_SCRATCH_BYTES
  * that every GPU loading the library holds until the process exits.  A call whose partials would not fit
- * (sum over sequences of ceil(ctx / split_tokens), times n_q_heads * (head_dim + 2) * 4 bytes, plus
- * 4 * n_seqs * n_kv_heads bytes of counters and 17 KiB)
+ * (sum over sequences of ceil(ctx / split_tokens), times n_q_heads * (head_dim + 2) * 4 bytes, plus 17 KiB)
  * or with more than PIE_NOALLOC_MAX_SEQS sequences returns PIE_ERR_NOMEM and enqueues nothing.
  * All calls on a device share that array and it keeps the previous call's contents: each call clears the
  * counters it needs at zero (a memset on `stream`) and writes every other word before reading it; two calls
