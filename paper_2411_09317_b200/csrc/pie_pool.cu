@@ -216,7 +216,10 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
             h[3 * i + 1] = dst[i];
             h[3 * i + 2] = blocks ? blocks[i] : 0;
         }
-        PIE_CUDA(cudaMemcpyAsync(p->list_dev + off, h, (size_t)(3 * n) * 4, cudaMemcpyHostToDevice, stream));
+        // the swap kernel wants its indices in device memory (no link latency per item); the table patch after
+        // copy-engine copies reads the few entries straight from the pinned list and saves a copy-engine operation
+        if (mode == PIE_MODE_KERNEL)
+            PIE_CUDA(cudaMemcpyAsync(p->list_dev + off, h, (size_t)(3 * n) * 4, cudaMemcpyHostToDevice, stream));
     }
     const int table_mode = slot_table_row ? (dir_queue == PIE_Q_IN ? 1 : 2) : 0;
     if (mode == PIE_MODE_KERNEL) {
@@ -234,7 +237,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
                                      kind, stream));
             i = j;
         }
-        if (slot_table_row) PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_dev + off, n, table_mode, stream));
+        if (slot_table_row) PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_host + off, n, table_mode, stream));
         p->stats.calls_copy_engine += 1;
     }
     if (need_list) {
@@ -273,16 +276,17 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
                 p->home_count[(size_t)layer] += 1;
             }
         }
+    // from here on the table has been updated: a failure leaves the pool unusable (sticky) rather than inconsistent
     cudaStream_t stream = p->stream[queue];
     st = reserve_ticket_event(p, queue, ticket);
-    if (st != PIE_OK) return st;
+    if (st != PIE_OK) { p->sticky = st; return st; }
     waits[PIE_Q_COMPUTE] = std::max(waits[PIE_Q_COMPUTE], not_before);
     for (int q = 1; q <= 3; ++q) {
         st = wait_ticket(p, stream, q, waits[q]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
     LayerEvents *le = timing_slot(p, layer);
-    if (le) PIE_CUDA(cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream));
+    if (le && cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream) != cudaSuccess) le = nullptr;
     st = do_copies(p, queue, p->v_src.data(), p->v_dst.data(), n_moved, p->v_moved.data(),
                    p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream);
     if (st != PIE_OK) { p->sticky = st; return st; }
@@ -403,18 +407,18 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     if (st != PIE_OK) return st;
     cudaStream_t stream = p->stream[PIE_Q_COMPUTE];
     st = reserve_ticket_event(p, PIE_Q_COMPUTE, ticket);
-    if (st != PIE_OK) return st;
+    if (st != PIE_OK) { p->sticky = st; return st; }
     LayerEvents *le = timing_slot(p, layer);
     if (le) {
         // every record costs the stream about a microsecond: the "before the wait" mark only when there is a wait
         le->waited = waits[1] > p->table->done(1) || waits[2] > p->table->done(2);
-        if (le->waited) PIE_CUDA(cudaEventRecord(le->pre, stream));
+        if (le->waited && cudaEventRecord(le->pre, stream) != cudaSuccess) le = nullptr;  // timing is best effort
     }
     for (int qd = 1; qd <= 2; ++qd) {
         st = wait_ticket(p, stream, qd, waits[qd]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
-    if (le) PIE_CUDA(cudaEventRecord(le->go, stream));
+    if (le && cudaEventRecord(le->go, stream) != cudaSuccess) le = nullptr;
     pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
                       p->cfg.n_gpu_slots};
     pie::AttnLaunch a{};
