@@ -178,6 +178,18 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
 int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_host, const int32_t *block_table_host,
                          int32_t max_blocks_per_seq, const int32_t *ctx_lens_host, int32_t n_seqs, float scale,
                          const void *k_new_all_host, const void *v_new_all_host, int32_t mode);
+/* The paper's whole-layer protocol on the GPU (Section 3.3), as a variant of the block-granular plan.  After this
+ * call pie_decode_step moves whole layers: when layer k starts, confirmed completions are applied, the coldest
+ * GPU layer is swapped out unless every CPU layer is colder or no CPU region is free, and the hottest CPU layer is
+ * swapped in unless no GPU region is free; one swap in flight per direction; a layer that is still on the CPU when
+ * its turn comes is waited for.  The host keeps step with the device, layer by layer (it waits for the previous
+ * layer's attention before deciding), as the paper's per-layer control loop does.  A region is one layer's units.
+ * Every layer must be wholly on one side (PIE_ERR_INVALID otherwise); gpu_regions + cpu_regions >= n_layers;
+ * the pools must hold that many layers' units.  gpu_regions <= 0 and cpu_regions <= 0: back to the block plan. */
+int pie_set_layer_policy(pie_pool *pool, int32_t gpu_regions, int32_t cpu_regions);
+/* The decisions taken so far in whole-layer mode: int32 quadruples {step, layer starting, layer whose swap-out
+ * started or -1, layer whose swap-in started or -1}.  log may be NULL to ask for the count only. */
+int pie_get_layer_log(pie_pool *pool, int32_t *log, int64_t capacity, int64_t *n_entries);
 /* Marks a step boundary for the per-step timing sets (pie_decode_step calls it itself). */
 int pie_step_begin(pie_pool *pool);
 

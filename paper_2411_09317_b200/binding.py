@@ -33,7 +33,7 @@ EXPORTS = [
     "pie_last_cuda_error", "pie_probe_link", "pie_probe_hbm", "pie_table_create", "pie_table_destroy", "pie_table_alloc",
     "pie_table_free", "pie_table_swap", "pie_table_attention", "pie_table_confirm", "pie_table_state", "pie_fifo_create",
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
-    "pie_decode_attention_noalloc",
+    "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
 ]
 
 
@@ -85,6 +85,8 @@ _sig = {
     "pie_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _i32, _f32, _vp, _vp, _i32]),
     "pie_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _i32, _f32, _vp, _vp, _i32]),
     "pie_step_begin": (_i32, [_vp]),
+    "pie_set_layer_policy": (_i32, [_vp, _i32, _i32]),
+    "pie_get_layer_log": (_i32, [_vp, _vp, _i64, ctypes.POINTER(_i64)]),
     "pie_set_extension_ratio": (_i32, [_vp, _f32]),
     "pie_get_extension_ratio": (_i32, [_vp, ctypes.POINTER(_f32)]),
     "pie_set_controller": (_i32, [_vp, _f64, _f64, _f64]),
@@ -243,6 +245,18 @@ def pie_decode_step_host(pool, q_all_host, out_all_host, block_table_host, max_b
     check(lib.pie_decode_step_host(pool, _ptr(q_all_host), _ptr(out_all_host), _ptr(block_table_host), max_blocks_per_seq,
                                    _ptr(ctx_lens_host), n_seqs, scale, _ptr(k_new_all_host), _ptr(v_new_all_host), mode),
           "pie_decode_step_host")
+
+
+def pie_set_layer_policy(pool, gpu_regions, cpu_regions) -> None:
+    check(lib.pie_set_layer_policy(pool, gpu_regions, cpu_regions), "pie_set_layer_policy")
+
+
+def pie_get_layer_log(pool) -> np.ndarray:
+    n = _i64()
+    check(lib.pie_get_layer_log(pool, None, 0, ctypes.byref(n)), "pie_get_layer_log")
+    log = np.zeros((max(n.value, 1), 4), dtype=np.int32)
+    check(lib.pie_get_layer_log(pool, _ptr(log), log.size, ctypes.byref(n)), "pie_get_layer_log")
+    return log[:n.value]
 
 
 def pie_step_begin(pool) -> None:

@@ -78,6 +78,10 @@ struct pie_pool {
     double ctrl_state[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
     std::vector<int64_t> home_count;  // per layer: units whose home is the host
+    // whole-layer protocol (Section 3.3): when set, pie_decode_step moves whole layers as the scheduler says
+    pie::Fifo *fifo = nullptr;
+    int64_t fifo_ticket[3] = {0, 0, 0};        // ticket of the layer swap in flight, per queue (0 = none)
+    std::vector<int32_t> fifo_log;             // {step, layer starting, swap-out started or -1, swap-in started or -1} x n
     // timing
     // per-step event sets: step k uses set k % TIMING_RING; a set is evaluated once, in step order, when complete
     std::vector<LayerEvents> lev[TIMING_RING];
@@ -368,6 +372,7 @@ void destroy_pool(pie_pool *p) {
     cudaFree(p->stage_v);
     cudaFree(p->stage_bt);
     cudaFree(p->stage_ctx);
+    delete p->fifo;
     delete p->table;
     delete p;
 }
@@ -1060,11 +1065,140 @@ int pie_sync(pie_pool *pool, int64_t timeout_us) {
     return check_status_word(pool);
 }
 
+// ---- whole-layer protocol on the GPU ------------------------------------------------------------------------
+static void all_block_ids(pie_pool *pool, std::vector<int32_t> &ids) {
+    ids.clear();
+    for (int32_t b = 0; b < pool->cfg.n_logical_blocks; ++b)
+        if (pool->table->allocated(b)) ids.push_back(b);
+}
+
+int pie_set_layer_policy(pie_pool *pool, int32_t gpu_regions, int32_t cpu_regions) {
+    if (!pool) return PIE_ERR_INVALID;
+    if (gpu_regions <= 0 && cpu_regions <= 0) {  // back to the block-granular plan
+        delete pool->fifo;
+        pool->fifo = nullptr;
+        return PIE_OK;
+    }
+    const int32_t L = pool->cfg.n_layers;
+    if (gpu_regions <= 0 || cpu_regions < 0 || gpu_regions + cpu_regions < L) return PIE_ERR_INVALID;
+    int st = sync_all(pool, 30 * 1000 * 1000);  // layers must be settled, each wholly on one side
+    if (st != PIE_OK) return st;
+    std::vector<uint8_t> on_cpu((size_t)L, 0);
+    int32_t n_gpu = 0, n_cpu = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        int64_t g = 0, h = 0;
+        for (int32_t b = 0; b < pool->cfg.n_logical_blocks; ++b) {
+            if (!pool->table->allocated(b)) continue;
+            (pool->table->unit(l, b).side == PIE_GPU ? g : h) += 1;
+        }
+        if (g > 0 && h > 0) return PIE_ERR_INVALID;  // a layer split between the sides: not a whole-layer state
+        on_cpu[(size_t)l] = h > 0;
+        (h > 0 ? n_cpu : n_gpu) += 1;
+    }
+    if (n_gpu > gpu_regions || n_cpu > cpu_regions) return PIE_ERR_NOMEM;
+    delete pool->fifo;
+    pool->fifo = new (std::nothrow) pie::Fifo(L, gpu_regions, cpu_regions, on_cpu.data());
+    if (!pool->fifo) return PIE_ERR_NOMEM;
+    pool->fifo_ticket[PIE_Q_IN] = pool->fifo_ticket[PIE_Q_OUT] = 0;
+    pool->fifo_log.clear();
+    return PIE_OK;
+}
+
+int pie_get_layer_log(pie_pool *pool, int32_t *log, int64_t capacity, int64_t *n_entries) {
+    if (!pool || !n_entries) return PIE_ERR_INVALID;
+    const int64_t n = (int64_t)pool->fifo_log.size() / 4;
+    *n_entries = n;
+    if (log) {
+        if (capacity < n * 4) return PIE_ERR_INVALID;
+        std::copy(pool->fifo_log.begin(), pool->fifo_log.end(), log);
+    }
+    return PIE_OK;
+}
+
+// confirmed completions -> scheduler (a finished swap-out frees its GPU region, a finished swap-in its CPU region)
+static int fifo_apply_completions(pie_pool *pool) {
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    for (int q : {PIE_Q_OUT, PIE_Q_IN})
+        if (pool->fifo_ticket[q] > 0 && pool->fifo_ticket[q] <= pool->table->done(q)) {
+            pool->fifo->complete(q);
+            pool->fifo_ticket[q] = 0;
+        }
+    return PIE_OK;
+}
+
+// the protocol's step at the instant layer k starts: start the swaps the scheduler asks for
+static int fifo_start_swaps(pie_pool *pool, int32_t k, int32_t mode, std::vector<int32_t> &ids) {
+    int32_t so = -1, si = -1;
+    int st = pool->fifo->layer_start(k, &so, &si);
+    if (st != PIE_OK) return st;
+    pool->fifo_log.insert(pool->fifo_log.end(), {(int32_t)pool->step, k, so, si});
+    for (int which = 0; which < 2; ++which) {
+        const int32_t layer = which == 0 ? so : si;
+        const int q = which == 0 ? PIE_Q_OUT : PIE_Q_IN;
+        if (layer < 0) continue;
+        all_block_ids(pool, ids);
+        const int64_t before = pool->table->issued(q);
+        st = pool_swap(pool, q, layer, ids.data(), (int64_t)ids.size(), mode);
+        if (st != PIE_OK) return st;
+        // an empty layer moves nothing and is complete at once
+        if (pool->table->issued(q) == before) pool->fifo->complete(q);
+        else pool->fifo_ticket[q] = pool->table->issued(q);
+    }
+    return PIE_OK;
+}
+
+static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev,
+                              int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale,
+                              const void *k_new_all, const void *v_new_all, int32_t mode) {
+    const int32_t L = pool->cfg.n_layers;
+    const int64_t q_stride = (int64_t)n_seqs * pool->cfg.n_q_heads * pool->cfg.head_dim * 2;
+    const int64_t kv_stride = (int64_t)n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;
+    int st = pie_step_begin(pool);
+    if (st != PIE_OK) return st;
+    std::vector<int32_t> ids;
+    for (int32_t k = 0; k < L; ++k) {
+        // the control logic runs when layer k starts, i.e. when layer k-1 has finished: the host keeps step with
+        // the device here (as the paper's per-layer control loop does), so completions are what they really are
+        const int64_t prev = pool->table->issued(PIE_Q_COMPUTE);
+        if (prev > pool->table->done(PIE_Q_COMPUTE)) PIE_CUDA(cudaEventSynchronize(pool->ticket_ev[PIE_Q_COMPUTE][prev % EV_RING]));
+        st = fifo_apply_completions(pool);
+        if (st != PIE_OK) return st;
+        st = fifo_start_swaps(pool, k, mode, ids);
+        if (st != PIE_OK) return st;
+        // presence check (Section 3.2): a layer still on the CPU with no copy under way has to be fetched first
+        for (int guard = 0; pool->fifo->location(k) == 1; ++guard) {
+            if (guard > 4 * L) return PIE_ERR_TIMEOUT;
+            bool waited = false;
+            for (int q : {PIE_Q_OUT, PIE_Q_IN})
+                if (pool->fifo_ticket[q] > 0) {
+                    PIE_CUDA(cudaEventSynchronize(pool->ticket_ev[q][pool->fifo_ticket[q] % EV_RING]));
+                    waited = true;
+                }
+            if (!waited) return PIE_ERR_NOMEM;  // nothing in flight and still no GPU region for layer k
+            st = fifo_apply_completions(pool);
+            if (st != PIE_OK) return st;
+            st = fifo_start_swaps(pool, k, mode, ids);
+            if (st != PIE_OK) return st;
+        }
+        // in transit to the GPU: the attention call waits for the copy's event on the device
+        st = attention_call(pool, k, (const uint8_t *)q_all + k * q_stride, (uint8_t *)out_all + k * q_stride, block_table_dev,
+                            max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
+                            k_new_all ? (const uint8_t *)k_new_all + k * kv_stride : nullptr,
+                            v_new_all ? (const uint8_t *)v_new_all + k * kv_stride : nullptr);
+        if (st != PIE_OK) return st;
+    }
+    return pie_controller_tick(pool, nullptr);
+}
+
 int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev, int32_t max_blocks_per_seq,
                     const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new_all, const void *v_new_all,
                     int32_t mode) {
     if (!pool || !q_all || !out_all) return PIE_ERR_INVALID;
     if (pool->sticky != PIE_OK) return pool->sticky;
+    if (pool->fifo)
+        return decode_step_layers(pool, q_all, out_all, block_table_dev, max_blocks_per_seq, ctx_lens_dev, n_seqs, scale,
+                                  k_new_all, v_new_all, mode);
     const int32_t L = pool->cfg.n_layers;
     const int64_t q_stride = (int64_t)n_seqs * pool->cfg.n_q_heads * pool->cfg.head_dim * 2;
     const int64_t kv_stride = (int64_t)n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;

@@ -369,3 +369,73 @@ def test_block_free_and_reuse_and_nomem():
     pie.pie_swap_out(pc.pool, 0, [])                        # empty list: fine
     pie.pie_sync(pc.pool)
     pc.close()
+
+
+# ---------------------------------------------------------------- the paper's whole-layer protocol on the GPU
+def test_whole_layer_protocol_nine_layers():
+    """Nine layers, layers 8 and 9 on the CPU at the start, seven GPU regions and four CPU regions (the paper's worked
+    example, Section 3.3), real copies and real attention.  Swap durations are whatever the link gives, so the
+    schedule is not the figure's; what must hold at any timing: outputs and bytes match the oracle, whole layers
+    move, one swap per direction at a time, layers leave in the order they finished (first in, first out), and the
+    first decisions - which depend on no completion - are the narrated ones."""
+    lens = np.array([200, 333, 90, 17], dtype=np.int32)
+    steps = 4
+    L = 9
+    case = Case(L, 8, 4, 64, F16, lens, seed=51, host_frac=0.0, placement="identity", extra_tokens=steps)
+    NB = case.NB
+    pool = pie.pie_pool_create(n_layers=L, n_q_heads=8, n_kv_heads=4, head_dim=64, dtype=F16, n_logical_blocks=NB,
+                               max_seqs=case.S, n_gpu_slots=7 * NB, n_host_slots=9 * NB, timing=1)
+    pie.pie_block_alloc(pool, NB, np.ones(NB, np.uint8))    # everything on the host first ...
+    for l in range(L):
+        for b in range(NB):
+            pie.pie_block_write(pool, l, b, case.gpu_pool[case.unit_slot[l, b]])
+    for l in range(7):                                      # ... then layers 1-7 wholly onto the GPU: 8 and 9 stay on the CPU
+        pie.pie_swap_in(pool, l, np.arange(NB))
+    pie.pie_sync(pool)
+    side, _ = pie.pie_get_placement(pool, L, NB)
+    assert np.all(side[:7] == pie.PIE_GPU) and np.all(side[7:] == pie.PIE_HOST)
+    pie.pie_set_layer_policy(pool, 7, 4)
+    dev = torch.device("cuda:0")
+    q = torch.from_numpy(case.q.view(np.int16)).to(dev)
+    out = torch.zeros_like(q)
+    bt = torch.from_numpy(case.block_table).to(dev)
+    cur = lens.copy()
+    ctx_dev = torch.from_numpy(cur).to(dev)
+    for t in range(steps):
+        k_new = synth.tensor_bits(51, synth.STREAM_KNEW, (L, case.S, case.Hkv, case.D), F16, offset=t * 1_000_000)
+        v_new = synth.tensor_bits(51, synth.STREAM_VNEW, (L, case.S, case.Hkv, case.D), F16, offset=t * 1_000_000)
+        k_dev = torch.from_numpy(k_new.view(np.int16)).to(dev)
+        v_dev = torch.from_numpy(v_new.view(np.int16)).to(dev)
+        cur = cur + 1
+        ctx_dev.copy_(torch.from_numpy(cur))
+        torch.cuda.synchronize()
+        pie.pie_decode_step(pool, q.data_ptr(), out.data_ptr(), bt.data_ptr(), case.block_table.shape[1], ctx_dev.data_ptr(),
+                            case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        pie.pie_sync(pool)
+        case.ctx_lens = cur.copy()
+        for l in range(L):
+            oracle.append(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k_new[l], v_new[l],
+                          case.block_table, cur, case.Hkv, case.D)
+            want = oracle_attention(case, l)
+            got = synth.bits16_to_f32(out[l].cpu().numpy().view(np.uint16), F16)
+            assert np.all(np.abs(got - want) <= edge_tol(want, F16)), (t, l)
+    for l in range(L):
+        for b in range(NB):
+            assert np.array_equal(pie.pie_block_read(pool, l, b).view(np.uint16), case.gpu_pool[case.unit_slot[l, b]]), (l, b)
+    side, _ = pie.pie_get_placement(pool, L, NB)
+    for l in range(L):                                     # whole layers only
+        assert len(set(side[l].tolist())) == 1
+    assert int((side[:, 0] == pie.PIE_GPU).sum()) <= 7
+    log = pie.pie_get_layer_log(pool)
+    first = {int(r[1]): (int(r[2]), int(r[3])) for r in log if r[0] == 1}
+    assert first[0] == (-1, -1)          # layer 1 starts: the CPU layers are colder, the GPU is full
+    assert first[1] == (0, -1)           # layer 2 starts: layer 1 goes out, no room yet for a swap-in
+    outs = [int(r[2]) for r in log if r[2] >= 0]
+    ins = [int(r[3]) for r in log if r[3] >= 0]
+    assert outs[0] == 0 and ins[0] == 7   # layer 1 leaves first; layer 8, the hottest CPU layer, comes in first
+    # first in, first out: layers come back in the order they left (after the two that started on the CPU)
+    assert ins[2:] == outs[:len(ins) - 2]
+    stats = pie.pie_get_stats(pool)
+    assert stats["bytes_out"] == len(outs) * NB * case.block_bytes
+    assert stats["bytes_in"] == (len(ins) + 7) * NB * case.block_bytes   # + the seven layers brought in during set-up
+    pie.pie_pool_destroy(pool)
