@@ -41,6 +41,10 @@ def main(argv=None):
     ap.add_argument("--ctx", type=int, default=4096)
     ap.add_argument("--swap-ctas", type=int, default=0)
     ap.add_argument("--part", default="12")
+    ap.add_argument("--q-heads", type=int, default=32)
+    ap.add_argument("--kv-heads", type=int, default=8)
+    ap.add_argument("--fp16", action="store_true", help="fp16 instead of bf16")
+    ap.add_argument("--blocks", default="", help="comma list of blocks per launch for part 2")
     args = ap.parse_args(argv)
     out = open(args.out, "w") if args.out else sys.stdout
 
@@ -49,7 +53,8 @@ def main(argv=None):
         out.flush()
 
     n_swap_slots = 16384 if not args.quick else 2048
-    wl = synth.Workload("swap_attn", 4, 1, 32, 8, 128, synth.BF16, np.full(args.seqs, args.ctx, dtype=np.int32), 0, 0.0)
+    wl = synth.Workload("swap_attn", 4, 1, args.q_heads, args.kv_heads, 128, synth.F16 if args.fp16 else synth.BF16,
+                        np.full(args.seqs, args.ctx, dtype=np.int32), 0, 0.0)
     dw = DeviceWorkload(wl, host_frac=0.0, timing=False, extra_gpu_slots=n_swap_slots, extra_host_slots=n_swap_slots,
                         swap_ctas=args.swap_ctas, extra_tokens=0)
     BB = wl.block_bytes
@@ -127,6 +132,8 @@ def main(argv=None):
         kv_bytes = dw.attention_bytes_per_layer()
         emit({"part": "attention_alone", "ms_per_launch": t0, "gbs": kv_bytes / (t0 * 1e-3) / 1e9, "runs": base})
         blocks = [8, 16, 32, 64, 128, 192, 256, 384] if not args.quick else [32, 128]
+        if args.blocks:
+            blocks = [int(x) for x in args.blocks.split(",")]
         for pattern in ("contiguous", "scattered"):
             for mode, mname in ((pie.PIE_MODE_KERNEL, "kernel"), (pie.PIE_MODE_COPY_ENGINE, "copy_engine")):
                 for direction in ("h2d", "d2h", "both"):

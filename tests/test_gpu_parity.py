@@ -260,7 +260,7 @@ def test_tiny_config_one_decode_step():
     lens = wl.ctx_lens
     case = Case(wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, lens, seed=0, host_frac=0.5,
                 placement="random", extra_tokens=1)
-    # Q17-style pool sizes: 64 blocks x 2 layers of slots per side
+    # pool sizes of the tiny configuration: 64 blocks x 2 layers of slots per side
     pc = PoolCase(case, n_gpu_slots=128, n_host_slots=128, timing=1)
     k_new = synth.tensor_bits(0, synth.STREAM_KNEW, (case.L, case.S, case.Hkv, case.D), case.dtype)
     v_new = synth.tensor_bits(0, synth.STREAM_VNEW, (case.L, case.S, case.Hkv, case.D), case.dtype)
