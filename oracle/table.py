@@ -80,8 +80,10 @@ class _SlotPool:
 
 
 class MappingTable:
-    def __init__(self, n_layers, n_logical, n_gpu_slots, n_host_slots):
+    def __init__(self, n_layers, n_logical, n_gpu_slots, n_host_slots, capacity=None):
         self.L, self.NB = n_layers, n_logical
+        if capacity is not None and not 0 < capacity <= n_logical:
+            raise ValueError("capacity")
         self.gpu = _SlotPool(n_gpu_slots)
         self.host = _SlotPool(n_host_slots)
         n = n_layers * n_logical
@@ -96,6 +98,12 @@ class MappingTable:
         self.clock = 0
         self.t_last = [0] * n           # the table's timestamp column
         self.last_compute = [0] * n_layers  # ticket of the newest attention call on each layer
+        # run-time resize (Section 4.1): ids below `capacity` are visible to the block manager; `target` is the
+        # size a resize in progress is heading to; `moved` holds the layers that have gone through a swap pass
+        # since the resize was triggered
+        self.capacity = n_logical if capacity is None else capacity
+        self.target = None
+        self.moved = set()
 
     # ---- helpers -------------------------------------------------------------------
     def _u(self, layer, block):
@@ -124,6 +132,37 @@ class MappingTable:
         self._settle()
         return OK
 
+    # ---- run-time resize of the per-layer cache (Section 4.1) ---------------------------
+    def alloc_limit(self):
+        """Ids below this may be handed out now.  Growing: the old size until every layer has moved (the new
+        space is prepared first, made visible afterwards).  Shrinking: the new size from the trigger on (nothing
+        is scheduled onto blocks that are about to go)."""
+        return self.capacity if self.target is None else min(self.capacity, self.target)
+
+    def resize_begin(self, new_size):
+        """Trigger a change of the per-layer size, in blocks.  NB (the table's physical width) bounds it."""
+        if not 0 < new_size <= self.NB:
+            return ERR_RANGE
+        if self.target is not None:
+            return ERR_BUSY
+        if new_size != self.capacity:
+            self.target = new_size
+            self.moved = set()
+        return OK
+
+    def layer_pass(self, layer):
+        """The layer goes through a swap pass (its space is re-established at the new size).  Once every layer
+        has done so the new size takes effect: grown ids become allocatable; shrunk ids leave the free list
+        for good (blocks still in use beyond the new size stay accessible until they are freed).
+        -> True when this call completed a resize."""
+        if not 0 <= layer < self.L or self.target is None:
+            return False
+        self.moved.add(layer)
+        if len(self.moved) < self.L:
+            return False
+        self.capacity, self.target, self.moved = self.target, None, set()
+        return True
+
     # ---- logical block allocation ----------------------------------------------------
     def alloc(self, block, on_host=False):
         """One unit per layer: a GPU slot while any is available (never, if on_host), else a host slot.  A recycled slot
@@ -131,6 +170,8 @@ class MappingTable:
         touches the unit next waits for it."""
         if not 0 <= block < self.NB:
             return ERR_RANGE
+        if block >= self.alloc_limit():
+            return ERR_NOMEM    # beyond the size visible now
         if self.allocated[block]:
             return ERR_INVALID
         self._settle()
@@ -202,6 +243,7 @@ class MappingTable:
         src_pool = self.gpu if direction == Q_OUT else self.host
         if len(movers) > dst_pool.available():
             return ERR_NOMEM, 0, [], {}
+        self.layer_pass(layer)
         if not movers:
             return OK, 0, [], {}
         slots, waits, _ = dst_pool.take(len(movers))

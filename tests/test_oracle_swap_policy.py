@@ -229,6 +229,112 @@ def test_table_random_long_runs():
 
 
 # ------------------------------------------------------------------------- protocol golden trace
+# ---- run-time resize of the per-layer size (Section 4.1) --------------------------------------------------
+def test_resize_grow_is_prepared_first_and_visible_only_after_every_layer_moved():
+    L = 3
+    t = table.MappingTable(L, 6, 12, 12, capacity=4)
+    for b in range(3):
+        assert t.alloc(b) == table.OK
+    assert t.alloc(4) == table.ERR_NOMEM               # beyond the size: not there yet
+    assert t.resize_begin(6) == table.OK
+    assert t.alloc(3) == table.OK                      # blocks within the previous size stay usable meanwhile
+    assert t.alloc(4) == table.ERR_NOMEM
+    assert not t.layer_pass(0) and not t.layer_pass(1)
+    assert not t.layer_pass(0)                         # the same layer again is not another layer
+    assert t.alloc(4) == table.ERR_NOMEM and t.capacity == 4
+    assert t.layer_pass(2)                             # the last layer: the new size takes effect
+    assert t.capacity == 6 and t.target is None
+    assert t.alloc(4) == table.OK and t.alloc(5) == table.OK
+    t.check_invariants()
+
+
+def test_resize_shrink_stops_handing_out_doomed_blocks_at_once_and_keeps_them_accessible():
+    L = 2
+    t = table.MappingTable(L, 6, 12, 12)
+    for b in range(6):
+        assert t.alloc(b) == table.OK
+    assert t.free(4) == table.OK
+    assert t.resize_begin(3) == table.OK
+    assert t.alloc(4) == table.ERR_NOMEM               # from the trigger on, before any layer has passed
+    assert t.capacity == 6                             # ... although the size itself has not changed yet
+    # a block in use beyond the new size is still swapped and attended to
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [5, 1])
+    assert st == table.OK and [p[0] for p in pairs] == [5, 1]
+    assert t.confirm(table.Q_OUT, tk) == table.OK
+    assert t.state(0, 5) == table.HOST
+    assert t.target == 3 and t.moved == {0}            # the swap call was layer 0's pass
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [5])
+    assert st == table.OK and t.attention(0, [5, 1])[0] == table.ERR_NOT_RESIDENT
+    assert t.swap(table.Q_IN, 0, [1])[0] == table.OK and t.attention(0, [5, 1])[0] == table.OK
+    assert t.target == 3
+    assert t.layer_pass(1) and t.capacity == 3 and t.target is None
+    for q in (table.Q_IN, table.Q_OUT, table.Q_COMPUTE):
+        t.confirm(q, t.issued[q])
+    assert t.attention(1, [5])[0] == table.OK          # still accessible after the size took effect
+    t.confirm(table.Q_COMPUTE, t.issued[table.Q_COMPUTE])
+    assert t.free(5) == table.OK and t.alloc(5) == table.ERR_NOMEM and t.alloc(3) == table.ERR_NOMEM
+    assert t.free(2) == table.OK and t.alloc(2) == table.OK
+    t.check_invariants()
+
+
+def test_resize_argument_checks_and_one_at_a_time():
+    t = table.MappingTable(2, 5, 10, 10, capacity=3)
+    assert t.resize_begin(0) == table.ERR_RANGE and t.resize_begin(6) == table.ERR_RANGE
+    assert t.resize_begin(3) == table.OK and t.target is None      # same size: nothing to do
+    assert t.resize_begin(5) == table.OK and t.resize_begin(4) == table.ERR_BUSY
+    assert not t.layer_pass(7) and not t.layer_pass(-1)            # no such layer: no mark
+    assert not t.layer_pass(1) and t.layer_pass(0)
+    assert t.resize_begin(4) == table.OK
+    with pytest.raises(ValueError):
+        table.MappingTable(2, 5, 10, 10, capacity=6)
+
+
+def test_resize_never_exposes_an_id_outside_both_sizes_under_random_traffic():
+    """Whatever the interleaving: an id handed out is below the old size and, when shrinking, below the new one too; the
+    size changes exactly when the last of the L layers has passed since the trigger."""
+    rng = random.Random(5)
+    for trial in range(200):
+        L, NB = rng.randint(1, 4), rng.randint(2, 8)
+        t = table.MappingTable(L, NB, L * NB, L * NB, capacity=rng.randint(1, NB))
+        passed, old = set(), t.capacity
+        for _ in range(60):
+            k = rng.random()
+            if k < 0.15:
+                new = rng.randint(1, NB)
+                busy = t.target is not None
+                assert t.resize_begin(new) == (table.ERR_BUSY if busy else table.OK)
+                if not busy and new != t.capacity:
+                    passed, old = set(), t.capacity
+            elif k < 0.45:
+                layer = rng.randrange(L)
+                in_progress, target = t.target is not None, t.target
+                if rng.random() < 0.5:
+                    done = t.layer_pass(layer)
+                else:
+                    ids = [b for b in range(NB) if t.allocated[b]][:2]
+                    before = t.capacity
+                    assert t.swap(rng.choice([table.Q_IN, table.Q_OUT]), layer, ids)[0] == table.OK
+                    done = in_progress and t.target is None
+                    for q in (table.Q_IN, table.Q_OUT):
+                        t.confirm(q, t.issued[q])
+                if in_progress:
+                    passed.add(layer)
+                    assert done == (len(passed) == L)
+                    assert t.capacity == (target if done else old)
+                else:
+                    assert not done
+            elif k < 0.8:
+                b = rng.randrange(NB)
+                limit = t.capacity if t.target is None else min(t.capacity, t.target)
+                st = t.alloc(b, rng.random() < 0.5)
+                assert (st == table.ERR_NOMEM) == (b >= limit)
+                assert st in (table.OK, table.ERR_INVALID, table.ERR_NOMEM)
+            else:
+                b = rng.randrange(NB)
+                t.free(b)
+        t.check_invariants()
+
+
 def read_golden():
     rows, totals = [], {}
     for line in open(os.path.join(GOLD, "fifo_9layer.txt")):
