@@ -74,8 +74,11 @@ typedef struct pie_pool_config {
     int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (512) */
     int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
     int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
-    int32_t timing;            /* 1: record per-layer events for pie_controller_tick / pie_get_stats */
-    int32_t reserved[7];       /* [0]: attention kernel variant for tuning (0 = default); rest 0 */
+    int32_t timing;            /* 1: record per-layer events for pie_controller_tick / pie_get_stats;
+                                * 2: also keep the per-layer timeline for pie_get_step_timeline */
+    int32_t reserved[7];       /* [0]: attention kernel variant for tuning (0 = default);
+                                * [1]: per-layer size visible to allocation at creation, in blocks (0 = n_logical_blocks;
+                                *      see pie_resize_begin); rest 0 */
 } pie_pool_config;
 
 typedef struct pie_stats {
@@ -88,7 +91,9 @@ typedef struct pie_stats {
     double ratio;                          /* current extension ratio */
     int64_t n_units_gpu, n_units_host, n_units_in_flight;
     int64_t steps_measured;
-    double reserved[8];                    /* [0]: last step's attention slow-down vs the no-swap record, ms */
+    double reserved[8];                    /* [0]: last step's attention slow-down vs the no-swap record, ms;
+                                            * [1]: the smallest extension ratio the GPU pool's size allows with the
+                                            *      blocks allocated now (the controller never goes below it) */
 } pie_stats;
 
 /* ---- pool (Section 3.1: the physical pools; Section 3.2: the mapping table) --------------------- */
@@ -207,6 +212,22 @@ int pie_get_extension_ratio(pie_pool *pool, float *r);
  * the time-per-token record taken on steps without swap traffic (copies that are hidden can still slow the
  * attention down through shared HBM bandwidth). */
 int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
+/* ---- run-time resize of the per-layer cache size (Section 4.1) -----------------------------------
+ * n_logical_blocks is the physical width of the per-layer tables; the size visible to allocation is
+ * reserved[1] of the configuration at creation (0: the full width) and changes in two phases:
+ *   grow:   pie_resize_begin(new) starts it; ids in [old, new) become allocatable only after every layer has
+ *           gone through a swap pass (pie_plan_layer / pie_decode_step on that layer, or a swap call on it) -
+ *           the space is prepared first and made visible afterwards;
+ *   shrink: ids >= new are not handed out from the moment of the call; blocks still in use up there stay
+ *           accessible; the new size takes effect once every layer has passed, and freed ids beyond it are
+ *           never handed out again.
+ * Slots come from the shared pools, so no region is physically moved: what the paper re-allocates per layer
+ * is here the layer's row of the slot table, which already has the full width.
+ * PIE_ERR_RANGE: new_blocks <= 0 or > n_logical_blocks; PIE_ERR_BUSY: a resize is in progress. */
+int pie_resize_begin(pie_pool *pool, int32_t new_blocks);
+/* Any pointer may be NULL.  target = -1 when no resize is in progress. */
+int pie_resize_status(pie_pool *pool, int32_t *visible, int32_t *alloc_limit, int32_t *target, int32_t *layers_moved);
+
 /* The per-layer plan at the start of layer `layer`: in_ids = units of layer (layer+1) mod L to bring in
  * (ascending id, as many as the GPU pool can take), out_ids = units of `layer` to push out once it has
  * computed.  Arrays are host, capacity n_logical_blocks each. */
@@ -216,7 +237,8 @@ int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in
  * for the oldest step when the host gets that far ahead of the GPU. */
 int pie_controller_tick(pie_pool *pool, int32_t *changed);
 int pie_get_stats(pie_pool *pool, pie_stats *out);
-/* Per-layer timeline of the most recently evaluated step (timing = 1): ms[l][7] = {compute stream reaches the
+/* Per-layer timeline of the most recently evaluated step (timing = 2 in the configuration; timing = 1 keeps the
+ * statistics and the controller but not this table, which costs a few hundred event queries per step): ms[l][7] = {compute stream reaches the
  * layer, presence wait over, layer done, swap-in start, swap-in end, swap-out start, swap-out end} in ms
  * from the step's first event; -1 where nothing was recorded.  capacity = floats available (>= 7 * n_layers).
  * PIE_ERR_INVALID if no step has been evaluated yet.  Shows what overlapped with what. */
@@ -282,6 +304,13 @@ int pie_table_swap(pie_table *t, int32_t queue, int32_t layer, const int32_t *id
 int pie_table_attention(pie_table *t, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits);
 int pie_table_confirm(pie_table *t, int32_t queue, int64_t ticket);
 int pie_table_state(pie_table *t, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot);
+/* Run-time resize on the bare table: see pie_resize_begin.  pie_table_init_capacity sets the visible size
+ * before anything is allocated; pie_table_layer_pass returns 1 when the call completed a resize, else 0
+ * (pie_table_swap makes the same mark for its layer). */
+int pie_table_init_capacity(pie_table *t, int32_t size);
+int pie_table_resize_begin(pie_table *t, int32_t new_size);
+int pie_table_layer_pass(pie_table *t, int32_t layer);
+int pie_table_capacity(pie_table *t, int32_t *visible, int32_t *alloc_limit, int32_t *target, int32_t *layers_moved);
 
 /* The whole-layer swap protocol of Section 3.3 as a scheduler object.  on_cpu: n_layers flags. */
 pie_fifo *pie_fifo_create(int32_t n_layers, int32_t gpu_regions, int32_t cpu_regions, const uint8_t *on_cpu);

@@ -34,6 +34,8 @@ EXPORTS = [
     "pie_table_free", "pie_table_swap", "pie_table_attention", "pie_table_confirm", "pie_table_state", "pie_fifo_create",
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
+    "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
+    "pie_table_capacity",
 ]
 
 
@@ -62,7 +64,9 @@ class Stats(ctypes.Structure):
     ]
 
     def as_dict(self):
-        return {k: getattr(self, k) for k, _ in self._fields_ if k != "reserved"}
+        d = {k: getattr(self, k) for k, _ in self._fields_ if k != "reserved"}
+        d["reserved"] = list(self.reserved)
+        return d
 
 
 lib = ctypes.CDLL(LIB_PATH)
@@ -107,6 +111,12 @@ _sig = {
     "pie_table_attention": (_i32, [_vp, _i32, _vp, _i64, ctypes.POINTER(_i64), _vp]),
     "pie_table_confirm": (_i32, [_vp, _i32, _i64]),
     "pie_table_state": (_i32, [_vp, _i32, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "pie_table_init_capacity": (_i32, [_vp, _i32]),
+    "pie_table_resize_begin": (_i32, [_vp, _i32]),
+    "pie_table_layer_pass": (_i32, [_vp, _i32]),
+    "pie_table_capacity": (_i32, [_vp] + [ctypes.POINTER(_i32)] * 4),
+    "pie_resize_begin": (_i32, [_vp, _i32]),
+    "pie_resize_status": (_i32, [_vp] + [ctypes.POINTER(_i32)] * 4),
     "pie_fifo_create": (_vp, [_i32, _i32, _i32, _vp]),
     "pie_fifo_destroy": (None, [_vp]),
     "pie_fifo_complete": (_i32, [_vp, _i32]),
@@ -155,6 +165,7 @@ def pie_pool_create(**kw) -> int:
     kw.setdefault("own_streams", 1)
     kw.setdefault("max_seqs", 256)
     cfg.reserved[0] = kw.pop("attn_variant", 0)
+    cfg.reserved[1] = kw.pop("visible_blocks", 0)
     for k, v in kw.items():
         setattr(cfg, k, v)
     out = _vp()
@@ -164,6 +175,16 @@ def pie_pool_create(**kw) -> int:
 
 def pie_pool_destroy(pool) -> None:
     check(lib.pie_pool_destroy(pool), "pie_pool_destroy")
+
+
+def pie_resize_begin(pool, new_blocks) -> None:
+    check(lib.pie_resize_begin(pool, new_blocks), "pie_resize_begin")
+
+
+def pie_resize_status(pool) -> dict:
+    v = [_i32() for _ in range(4)]
+    check(lib.pie_resize_status(pool, *[ctypes.byref(x) for x in v]), "pie_resize_status")
+    return dict(zip(("visible", "alloc_limit", "target", "layers_moved"), (x.value for x in v)))
 
 
 def pie_block_bytes(pool) -> int:
@@ -380,6 +401,21 @@ class Table:
         s, g, h = _i32(), _i32(), _i32()
         st = lib.pie_table_state(self.h, layer, block, ctypes.byref(s), ctypes.byref(g), ctypes.byref(h))
         return st, s.value, g.value, h.value
+
+
+    def init_capacity(self, size):
+        return lib.pie_table_init_capacity(self.h, size)
+
+    def resize_begin(self, new_size):
+        return lib.pie_table_resize_begin(self.h, new_size)
+
+    def layer_pass(self, layer):
+        return lib.pie_table_layer_pass(self.h, layer)
+
+    def capacity(self):
+        v = [_i32() for _ in range(4)]
+        st = lib.pie_table_capacity(self.h, *[ctypes.byref(x) for x in v])
+        return st, dict(zip(("visible", "alloc_limit", "target", "layers_moved"), (x.value for x in v)))
 
 
 class Fifo:

@@ -745,6 +745,10 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
                uint16_t *__restrict__ out, int32_t n_q_heads, int32_t n_kv_heads, int32_t group) {
     __shared__ float wbuf[8][COMB_CAP];
     __shared__ float lbuf[8][COMB_CAP];
+    // Launched with programmatic stream serialization: CTAs may become resident while the attention kernel's last
+    // CTAs are still running (which hides the launch latency); nothing that kernel wrote is read before this wait,
+    // which returns once the attention grid has completed and its writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int tid = threadIdx.x;
     const int32_t s = blockIdx.x / n_kv_heads, kvh = blockIdx.x - s * n_kv_heads;
     const int32_t chunk0 = chunk_off[s], nchunks = chunk_off[s + 1] - chunk0;
@@ -964,20 +968,25 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     });
     if (e != cudaSuccess) return e;
     // merge the partials of sequences that span several chunks (CTAs of single-chunk sequences return at once)
-    const dim3 cgrid((unsigned)(a.n_seqs * sh.n_kv_heads), (unsigned)(sh.head_dim / 32));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(a.n_seqs * sh.n_kv_heads), (unsigned)(sh.head_dim / 32));
+    cfg.blockDim = dim3(COMB_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     uint16_t *out = (uint16_t *)a.out;
-    if (sh.head_dim == 128) {
-        if (sh.dtype == PIE_BF16)
-            combine_kernel<128, true><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
-        else
-            combine_kernel<128, false><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
-    } else {
-        if (sh.dtype == PIE_BF16)
-            combine_kernel<64, true><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
-        else
-            combine_kernel<64, false><<<cgrid, COMB_THREADS, 0, stream>>>(sc.part_o, sc.part_ml, sc.chunk_off, out, sh.n_q_heads, sh.n_kv_heads, p.group);
-    }
-    return cudaGetLastError();
+    const float *po = sc.part_o, *pml = sc.part_ml;
+    const int32_t *co = sc.chunk_off;
+    const int32_t hq = sh.n_q_heads, hkv = sh.n_kv_heads, group = p.group;
+    if (sh.head_dim == 128)
+        return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<128, true>, po, pml, co, out, hq, hkv, group)
+                                    : cudaLaunchKernelEx(&cfg, combine_kernel<128, false>, po, pml, co, out, hq, hkv, group);
+    return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<64, true>, po, pml, co, out, hq, hkv, group)
+                                : cudaLaunchKernelEx(&cfg, combine_kernel<64, false>, po, pml, co, out, hq, hkv, group);
 }
 
 }  // namespace pie

@@ -33,15 +33,20 @@ constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list
 
 struct LayerEvents {
     // compute stream: before the presence wait, after it, after the layer; copy streams: start and end of a list.
+    // Every record costs the stream about a microsecond between two kernels, so a layer records only what it needs:
+    // `pre` for the first layer of a step, `go` when there is a wait to measure.
     // pre, go, in0, out0 are owned; done, in1, out1 point at the ticket events of the calls (valid for EV_RING tickets)
     cudaEvent_t pre = nullptr, go = nullptr, done = nullptr;
+    cudaEvent_t start = nullptr;  // where the layer's time starts: the previous layer's `done` within a step, else `pre`
     cudaEvent_t in0 = nullptr, in1 = nullptr, out0 = nullptr, out1 = nullptr;
     bool has_in = false, has_out = false, has_compute = false, waited = false;
 };
 
 struct ListRecord {
     int64_t start, end;
-    int ev;  // index into list_events
+    int ev;          // index into list_events, or -1: guarded by a ticket of a queue (its event is recorded by the caller)
+    int queue;
+    int64_t ticket;
 };
 
 }  // namespace
@@ -77,7 +82,12 @@ struct pie_pool {
     double ratio = 0.0;
     double ctrl_state[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
+    cudaEvent_t last_compute_ev = nullptr;  // the newest attention call's ticket event and the step it belongs to
+    int64_t last_compute_step = -1;
+    bool poll_hold = false;  // a decode step is polling once per layer: nested calls skip theirs
     std::vector<int64_t> home_count;  // per layer: units whose home is the host
+    std::vector<std::vector<int32_t>> home_list;  // per layer: ids the planner looks at (see candidate_ids)
+    std::vector<uint8_t> home_dirty;              // per layer: home_list must be rebuilt
     // whole-layer protocol (Section 3.3): when set, pie_decode_step moves whole layers as the scheduler says
     pie::Fifo *fifo = nullptr;
     int64_t fifo_ticket[3] = {0, 0, 0};        // ticket of the layer swap in flight, per queue (0 = none)
@@ -87,6 +97,7 @@ struct pie_pool {
     std::vector<LayerEvents> lev[TIMING_RING];
     int64_t lev_step[TIMING_RING] = {};      // which step a set holds (0 = none)
     bool lev_done[TIMING_RING] = {};         // already evaluated
+    cudaEvent_t lev_last[TIMING_RING][4] = {};  // the set's newest event on each queue's stream (its streams complete in order)
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
     std::vector<float> timeline;     // last evaluated step: [L][7] ms from the step's first event (-1 = not recorded)
@@ -98,7 +109,10 @@ struct pie_pool {
 
 namespace {
 
-int poll(pie_pool *p) {
+// Phase 2 of the table update (Section 3.2): learn which copies and attention calls have completed.  While a
+// decode step holds the poll (one forced poll per layer there), the calls inside it skip their own.
+int poll(pie_pool *p, bool force = false) {
+    if (p->poll_hold && !force) return PIE_OK;
     for (int q = 1; q <= 3; ++q) {
         int64_t d = p->table->done(q);
         const int64_t issued = p->recorded[q];  // a ticket whose event is not recorded yet cannot be queried
@@ -129,7 +143,7 @@ int reserve_ticket_event(pie_pool *p, int q, int64_t t) {
     const int64_t prev = t - EV_RING;
     if (prev > 0 && prev > p->table->done(q)) {
         PIE_CUDA(cudaEventSynchronize(p->ticket_ev[q][prev % EV_RING]));
-        poll(p);
+        poll(p, true);
     }
     return PIE_OK;
 }
@@ -146,14 +160,20 @@ int list_alloc(pie_pool *p, int64_t words, int64_t *offset) {
     if (words > p->list_words) return PIE_ERR_INVALID;
     if (p->list_head + words > p->list_words) p->list_head = 0;
     const int64_t a = p->list_head, b = a + words;
-    while (!p->list_live.empty() && cudaEventQuery(p->list_events[p->list_live.front().ev]) == cudaSuccess)
-        p->list_live.pop_front();
+    auto consumed = [&](const ListRecord &r) {
+        if (r.ev < 0) return r.ticket <= p->table->done(r.queue);  // as of the last poll: no driver call
+        return cudaEventQuery(p->list_events[r.ev]) == cudaSuccess;
+    };
+    auto wait_for = [&](const ListRecord &r) {
+        return cudaEventSynchronize(r.ev < 0 ? p->ticket_ev[r.queue][r.ticket % EV_RING] : p->list_events[r.ev]);
+    };
+    while (!p->list_live.empty() && consumed(p->list_live.front())) p->list_live.pop_front();
     for (;;) {
         bool clash = false;
         for (size_t i = 0; i < p->list_live.size(); ++i) {
-            const ListRecord &r = p->list_live[i];
+            const ListRecord r = p->list_live[i];
             if (r.start < b && a < r.end) {
-                PIE_CUDA(cudaEventSynchronize(p->list_events[r.ev]));
+                if (!consumed(r)) PIE_CUDA(wait_for(r));
                 p->list_live.erase(p->list_live.begin() + (long)i);
                 clash = true;
                 break;
@@ -162,7 +182,7 @@ int list_alloc(pie_pool *p, int64_t words, int64_t *offset) {
         if (!clash) break;
     }
     if ((int)p->list_live.size() >= LIST_EVENTS - 1) {
-        PIE_CUDA(cudaEventSynchronize(p->list_events[p->list_live.front().ev]));
+        PIE_CUDA(wait_for(p->list_live.front()));
         p->list_live.pop_front();
     }
     *offset = a;
@@ -176,8 +196,15 @@ int list_commit(pie_pool *p, int64_t offset, int64_t words, cudaStream_t stream)
     const int ev = p->list_ev_next;
     p->list_ev_next = (p->list_ev_next + 1) % LIST_EVENTS;
     PIE_CUDA(cudaEventRecord(p->list_events[ev], stream));
-    p->list_live.push_back({offset, offset + words, ev});
+    p->list_live.push_back({offset, offset + words, ev, 0, 0});
     return PIE_OK;
+}
+
+// the same for a list consumed by work that belongs to ticket t of queue q: the ticket's event, which the caller
+// records right after that work, guards the list and no event of its own is needed
+void list_commit_ticket(pie_pool *p, int64_t offset, int64_t words, int q, int64_t t) {
+    words = (words + 3) & ~int64_t(3);
+    p->list_live.push_back({offset, offset + words, -1, q, t});
 }
 
 int check_status_word(pie_pool *p) {
@@ -195,7 +222,7 @@ LayerEvents *timing_slot(pie_pool *p, int32_t layer) {
 
 // ---- one swap call ------------------------------------------------------------------------------------
 int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst, int64_t n, const int32_t *blocks,
-              int32_t *slot_table_row, int mode, cudaStream_t stream) {
+              int32_t *slot_table_row, int mode, cudaStream_t stream, int64_t ticket = 0) {
     // dir_queue PIE_Q_IN: host -> GPU; PIE_Q_OUT: GPU -> host
     const uint8_t *src_pool = dir_queue == PIE_Q_IN ? p->host_base : p->gpu_base;
     uint8_t *dst_pool = dir_queue == PIE_Q_IN ? p->gpu_base : p->host_base;
@@ -245,8 +272,12 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         p->stats.calls_copy_engine += 1;
     }
     if (need_list) {
-        int st = list_commit(p, off, 3 * n, stream);
-        if (st != PIE_OK) return st;
+        if (ticket > 0) {
+            list_commit_ticket(p, off, 3 * n, dir_queue, ticket);
+        } else {
+            int st = list_commit(p, off, 3 * n, stream);
+            if (st != PIE_OK) return st;
+        }
     }
     return PIE_OK;
 }
@@ -278,6 +309,7 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
             if (!u.home_host) {
                 u.home_host = 1;
                 p->home_count[(size_t)layer] += 1;
+                p->home_dirty[(size_t)layer] = 1;
             }
         }
     // from here on the table has been updated: a failure leaves the pool unusable (sticky) rather than inconsistent
@@ -292,13 +324,14 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
     LayerEvents *le = timing_slot(p, layer);
     if (le && cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream) != cudaSuccess) le = nullptr;
     st = do_copies(p, queue, p->v_src.data(), p->v_dst.data(), n_moved, p->v_moved.data(),
-                   p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream);
+                   p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream, ticket);
     if (st != PIE_OK) { p->sticky = st; return st; }
     st = record_ticket(p, queue, ticket);
     if (st != PIE_OK) { p->sticky = st; return st; }
     if (le) {
         (queue == PIE_Q_IN ? le->in1 : le->out1) = p->ticket_ev[queue][ticket % EV_RING];
         (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
+        p->lev_last[p->step % TIMING_RING][queue] = p->ticket_ev[queue][ticket % EV_RING];
     }
     (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)n_moved * (double)p->block_bytes;
     return PIE_OK;
@@ -415,15 +448,19 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     if (st != PIE_OK) { p->sticky = st; return st; }
     LayerEvents *le = timing_slot(p, layer);
     if (le) {
-        // every record costs the stream about a microsecond: the "before the wait" mark only when there is a wait
         le->waited = waits[1] > p->table->done(1) || waits[2] > p->table->done(2);
-        if (le->waited && cudaEventRecord(le->pre, stream) != cudaSuccess) le = nullptr;  // timing is best effort
+        if (p->last_compute_ev && p->last_compute_step == p->step) {
+            le->start = p->last_compute_ev;
+        } else {
+            le->start = le->pre;
+            if (cudaEventRecord(le->pre, stream) != cudaSuccess) le = nullptr;  // timing is best effort
+        }
     }
     for (int qd = 1; qd <= 2; ++qd) {
         st = wait_ticket(p, stream, qd, waits[qd]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
-    if (le && cudaEventRecord(le->go, stream) != cudaSuccess) le = nullptr;
+    if (le && le->waited && cudaEventRecord(le->go, stream) != cudaSuccess) le = nullptr;
     pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
                       p->cfg.n_gpu_slots};
     pie::AttnLaunch a{};
@@ -453,23 +490,36 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     if (le && st == PIE_OK) {
         le->done = p->ticket_ev[PIE_Q_COMPUTE][ticket % EV_RING];
         le->has_compute = true;
+        p->lev_last[p->step % TIMING_RING][PIE_Q_COMPUTE] = le->done;
+        p->last_compute_ev = le->done;
+        p->last_compute_step = p->step;
     }
     return st;
 }
 
 // the host-resident set of `layer` follows the ratio: mark / unmark units in id order
+// The GPU pool must hold every layer's resident share plus two layers' host share in transit:
+// L (n - h) + 2 h <= n_gpu_slots bounds the host-resident count h of a layer from below.
+int64_t min_home_count(const pie_pool *p) {
+    const int64_t n_alloc = p->table->n_allocated(), L = p->cfg.n_layers;
+    if (L <= 2) return 0;
+    const int64_t deficit = L * n_alloc - p->cfg.n_gpu_slots;
+    return deficit > 0 ? std::min(n_alloc, (deficit + L - 3) / (L - 2)) : 0;
+}
+
+// the smallest extension ratio the GPU pool's size allows with the blocks allocated now
+double ratio_floor(const pie_pool *p) {
+    const int64_t n_alloc = p->table->n_allocated();
+    return n_alloc > 0 ? (double)min_home_count(p) / (double)n_alloc : 0.0;
+}
+
 void apply_ratio_to_layer(pie_pool *p, int32_t layer) {
     if (p->ratio_mode == 0) return;
     const int32_t NB = p->cfg.n_logical_blocks;
-    const int64_t n_alloc = p->table->n_allocated(), L = p->cfg.n_layers;
-    int64_t target = (int64_t)std::llround(p->ratio * (double)n_alloc);
-    // the GPU pool must hold every layer's resident share plus two layers' host share in transit:
-    // L (n - h) + 2 h <= n_gpu_slots bounds the host-resident count h from below
-    if (L > 2) {
-        const int64_t deficit = L * n_alloc - p->cfg.n_gpu_slots;
-        if (deficit > 0) target = std::max(target, std::min(n_alloc, (deficit + L - 3) / (L - 2)));
-    }
+    const int64_t n_alloc = p->table->n_allocated();
+    const int64_t target = std::max((int64_t)std::llround(p->ratio * (double)n_alloc), min_home_count(p));
     int64_t &count = p->home_count[(size_t)layer];
+    if (count != target) p->home_dirty[(size_t)layer] = 1;
     if (count < target) {
         for (int32_t b = 0; b < NB && count < target; ++b) {
             if (!p->table->allocated(b)) continue;
@@ -485,30 +535,51 @@ void apply_ratio_to_layer(pie_pool *p, int32_t layer) {
     }
 }
 
+// The units of `layer` that a plan has to look at, in ascending id: members of the host-resident set and units
+// that are on the host for any other reason.  Rebuilt by one scan only after the set changed (an allocation, a
+// free, a ratio change, a caller's own swap-out), so that a steady decode loop does not walk every block of
+// every layer on every step.
+const std::vector<int32_t> &candidate_ids(pie_pool *p, int32_t layer) {
+    std::vector<int32_t> &v = p->home_list[(size_t)layer];
+    if (p->home_dirty[(size_t)layer]) {
+        v.clear();
+        const int32_t NB = p->cfg.n_logical_blocks;
+        for (int32_t b = 0; b < NB; ++b) {
+            if (!p->table->allocated(b)) continue;
+            const pie::Unit &u = p->table->unit(layer, b);
+            if (u.home_host || u.side == PIE_HOST) v.push_back(b);
+        }
+        p->home_dirty[(size_t)layer] = 0;
+    }
+    return v;
+}
+
 int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::vector<int32_t> &out_ids) {
-    const int32_t L = p->cfg.n_layers, NB = p->cfg.n_logical_blocks;
+    const int32_t L = p->cfg.n_layers;
     const int32_t next = (layer + 1) % L;
     in_ids.clear();
     out_ids.clear();
+    p->table->layer_pass(layer);  // a resize in progress takes effect once every layer has been here (Section 4.1)
     apply_ratio_to_layer(p, layer);
     apply_ratio_to_layer(p, next);
     // hottest first: the next layer's host-resident units, as many as the GPU pool can take
     int64_t room = p->table->gpu_available();
     int64_t left_behind = 0;
-    for (int32_t b = 0; b < NB; ++b) {
-        if (!p->table->allocated(b)) continue;
-        if (p->table->unit(next, b).side == PIE_HOST) {
+    for (int32_t b : candidate_ids(p, next)) {
+        const pie::Unit &u = p->table->unit(next, b);
+        if (u.side == PIE_HOST) {
             if (room > 0) {
                 in_ids.push_back(b);
                 --room;
             } else {
                 ++left_behind;
             }
+        } else if (!u.home_host) {
+            p->home_dirty[(size_t)next] = 1;  // left the set and is back on the GPU: drop it at the next rebuild
         }
     }
     // coldest: this layer's host-home units go back once it has computed
-    for (int32_t b = 0; b < NB; ++b) {
-        if (!p->table->allocated(b)) continue;
+    for (int32_t b : candidate_ids(p, layer)) {
         const pie::Unit &u = p->table->unit(layer, b);
         if (u.home_host && u.side == PIE_GPU) out_ids.push_back(b);
     }
@@ -608,7 +679,10 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     p->n_sms = prop.multiProcessorCount;
     p->table = new (std::nothrow) pie::Table(cfg->n_layers, cfg->n_logical_blocks, cfg->n_gpu_slots, cfg->n_host_slots);
     if (!p->table) { destroy_pool(p); return PIE_ERR_NOMEM; }
+    if (cfg->reserved[1] != 0 && p->table->init_capacity(cfg->reserved[1]) != PIE_OK) { destroy_pool(p); return PIE_ERR_INVALID; }
     p->home_count.assign((size_t)cfg->n_layers, 0);
+    p->home_list.assign((size_t)cfg->n_layers, std::vector<int32_t>());
+    p->home_dirty.assign((size_t)cfg->n_layers, 1);
 
 #define PIE_TRY(call, code)                            \
     do {                                               \
@@ -707,15 +781,18 @@ int pie_block_alloc(pie_pool *pool, int64_t n, const uint8_t *on_host, int32_t *
     if (st != PIE_OK) return st;
     pie::Table *t = pool->table;
     const int32_t NB = pool->cfg.n_logical_blocks, L = pool->cfg.n_layers;
-    if (n > NB - t->n_allocated()) return PIE_ERR_NOMEM;
-    // ids: the lowest free ones; slots are handed out layer by layer (consecutive slots within a layer)
+    // ids: the lowest free ones below the size visible now (a resize in progress: Section 4.1); slots are
+    // handed out layer by layer (consecutive slots within a layer)
+    const int32_t limit = t->alloc_limit();
     int32_t next = 0;
     for (int64_t i = 0; i < n; ++i) {
-        while (next < NB && t->allocated(next)) ++next;
+        while (next < limit && t->allocated(next)) ++next;
+        if (next >= limit) return PIE_ERR_NOMEM;
         ids_out[i] = next++;
     }
     st = t->alloc_bulk(ids_out, n, on_host);
     if (st != PIE_OK) return st;  // all or nothing: the table is unchanged
+    std::fill(pool->home_dirty.begin(), pool->home_dirty.end(), (uint8_t)1);
     std::vector<int32_t> entries;
     entries.reserve((size_t)(n * L * 2));
     for (int64_t i = 0; i < n; ++i)
@@ -748,6 +825,7 @@ int pie_block_free(pie_pool *pool, const int32_t *ids, int64_t n) {
             if (t->in_flight(t->unit(l, ids[i]))) return PIE_ERR_BUSY;
     }
     std::vector<int32_t> entries;
+    std::fill(pool->home_dirty.begin(), pool->home_dirty.end(), (uint8_t)1);
     for (int64_t i = 0; i < n; ++i) {
         for (int32_t l = 0; l < L; ++l) {
             const pie::Unit &u = t->unit(l, ids[i]);
@@ -855,14 +933,13 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
 // wait = true blocks until the set's events have completed (used only when the ring is about to wrap).
 static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed) {
     std::vector<LayerEvents> &ev = pool->lev[k];
-    for (LayerEvents &e : ev) {
-        for (int which = 0; which < 3; ++which) {
-            const bool has = which == 0 ? e.has_compute : which == 1 ? e.has_in : e.has_out;
-            cudaEvent_t evt = which == 0 ? e.done : which == 1 ? e.in1 : e.out1;
-            if (!has) continue;
-            if (wait) PIE_CUDA(cudaEventSynchronize(evt));
-            else if (cudaEventQuery(evt) != cudaSuccess) return 1;  // not complete yet
-        }
+    // every event of the set sits on one of three streams and a stream completes in order: the newest event of
+    // each stream tells whether the whole set is complete
+    for (int q = 1; q <= 3; ++q) {
+        cudaEvent_t evt = pool->lev_last[k][q];
+        if (!evt) continue;
+        if (wait) PIE_CUDA(cudaEventSynchronize(evt));
+        else if (cudaEventQuery(evt) != cudaSuccess) return 1;  // not complete yet
     }
     double compute = 0, stall = 0, t_in = 0, t_out = 0;
     cudaEvent_t first = nullptr, last = nullptr;
@@ -870,14 +947,19 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     for (LayerEvents &e : ev) {
         float ms = 0;
         if (e.has_compute) {
-            PIE_CUDA(cudaEventElapsedTime(&ms, e.go, e.done));
-            compute += ms;
+            // the layer's time runs from the end of the previous layer; what the stream spent in the presence wait
+            // is the stall (two back-to-back stream operations are already ~2-3 us apart: only the excess counts),
+            // the rest - launch gap included, with or without swaps - is compute
+            PIE_CUDA(cudaEventElapsedTime(&ms, e.start, e.done));
+            double layer_stall = 0.0;
             if (e.waited) {
-                // two back-to-back event records are already ~2-3 us apart: count only what exceeds that
-                PIE_CUDA(cudaEventElapsedTime(&ms, e.pre, e.go));
-                stall += std::max(0.0, (double)ms - 0.004);
+                float w = 0;
+                PIE_CUDA(cudaEventElapsedTime(&w, e.start, e.go));
+                layer_stall = std::max(0.0, (double)w - 0.004);
             }
-            if (!first) first = e.waited ? e.pre : e.go;
+            stall += layer_stall;
+            compute += std::max(0.0, (double)ms - layer_stall);
+            if (!first) first = e.start;
             last = e.done;
         }
         if (e.has_in) {
@@ -892,11 +974,11 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         }
     }
     pool->lev_done[k] = true;
-    if (first) {
+    if (first && pool->cfg.timing >= 2) {
         pool->timeline.assign(ev.size() * 7, -1.f);
         for (size_t l = 0; l < ev.size(); ++l) {
             LayerEvents &e = ev[l];
-            cudaEvent_t list[7] = {e.waited ? e.pre : e.go, e.go, e.done, e.in0, e.in1, e.out0, e.out1};
+            cudaEvent_t list[7] = {e.start, e.waited ? e.go : e.start, e.done, e.in0, e.in1, e.out0, e.out1};
             const bool has[7] = {e.has_compute, e.has_compute, e.has_compute, e.has_in, e.has_in, e.has_out, e.has_out};
             for (int j = 0; j < 7; ++j)
                 if (has[j]) {
@@ -926,9 +1008,13 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         else if (pool->base_ms_per_token > 0) slow = std::max(0.0, compute - pool->base_ms_per_token * tokens);
     }
     pool->stats.reserved[0] = slow;
+    pool->stats.reserved[1] = ratio_floor(pool);
     if (pool->ratio_mode == 2 && compute > 0) {
         const double step = pool->ctrl_step > 0 ? pool->ctrl_step : 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
-        const double r = pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall + slow, compute, std::max(t_in, t_out));
+        // the rule never asks for less than the GPU pool's size allows: below that floor the number would drift
+        // away from what the layers actually keep on the host
+        const double r = std::max(ratio_floor(pool),
+                                  pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall + slow, compute, std::max(t_in, t_out)));
         if (r != pool->ratio) {
             pool->ratio = r;
             if (changed) *changed = 1;
@@ -964,6 +1050,7 @@ int pie_step_begin(pie_pool *pool) {
         pool->lev_step[k] = pool->step;
         pool->lev_done[k] = false;
         for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = e.waited = false;
+        for (int q = 0; q < 4; ++q) pool->lev_last[k][q] = nullptr;
     }
     return PIE_OK;
 }
@@ -1005,6 +1092,21 @@ int pie_get_extension_ratio(pie_pool *pool, float *r) {
     } else {
         *r = (float)pool->ratio;
     }
+    return PIE_OK;
+}
+
+int pie_resize_begin(pie_pool *pool, int32_t new_blocks) {
+    if (!pool) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    return pool->table->resize_begin(new_blocks);
+}
+
+int pie_resize_status(pie_pool *pool, int32_t *visible, int32_t *alloc_limit, int32_t *target, int32_t *layers_moved) {
+    if (!pool) return PIE_ERR_INVALID;
+    if (visible) *visible = pool->table->capacity();
+    if (alloc_limit) *alloc_limit = pool->table->alloc_limit();
+    if (target) *target = pool->table->resize_target();
+    if (layers_moved) *layers_moved = pool->table->layers_moved();
     return PIE_OK;
 }
 
@@ -1205,10 +1307,15 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
     int st = pie_step_begin(pool);
     if (st != PIE_OK) return st;
     // layer 0 has no predecessor in the first step: fetch what it needs now (later steps prefetch it from layer L-1)
+    struct PollHold {
+        pie_pool *p;
+        ~PollHold() { p->poll_hold = false; }
+    } hold{pool};
+    pool->poll_hold = true;
     {
         pool->v_in.clear();
-        for (int32_t b = 0; b < pool->cfg.n_logical_blocks; ++b)
-            if (pool->table->allocated(b) && pool->table->unit(0, b).side == PIE_HOST) pool->v_in.push_back(b);
+        for (int32_t b : candidate_ids(pool, 0))
+            if (pool->table->unit(0, b).side == PIE_HOST) pool->v_in.push_back(b);
         if (!pool->v_in.empty()) {
             std::vector<int32_t> ids(pool->v_in);
             st = pool_swap(pool, PIE_Q_IN, 0, ids.data(), (int64_t)ids.size(), mode);
@@ -1217,8 +1324,12 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
     }
     std::vector<int32_t> in_ids, out_ids;
     for (int32_t l = 0; l < L; ++l) {
-        st = poll(pool);
-        if (st != PIE_OK) return st;
+        // completions are learnt every few layers: a stale view only means a wait on an event that has already
+        // completed, or a slot that stays "pending" a little longer
+        if (l % 8 == 0) {
+            st = poll(pool, true);
+            if (st != PIE_OK) return st;
+        }
         st = plan_layer(pool, l, in_ids, out_ids);
         if (st != PIE_OK) return st;  // the GPU pool cannot take the next layer's share: nothing was enqueued for it
         if (L > 1 && !in_ids.empty()) {

@@ -48,10 +48,43 @@ void SlotPool::release(int32_t slot, int32_t queue, int64_t ticket) {
 Table::Table(int32_t n_layers, int32_t n_logical, int64_t n_gpu_slots, int64_t n_host_slots)
     : L(n_layers), NB(n_logical), gpu_(n_gpu_slots), host_(n_host_slots),
       units_((size_t)n_layers * (size_t)n_logical), allocated_((size_t)n_logical, 0), seen_((size_t)n_logical, 0),
-      last_compute_((size_t)n_layers, 0), layer_wait_((size_t)n_layers * 4, 0) {}
+      last_compute_((size_t)n_layers, 0), layer_wait_((size_t)n_layers * 4, 0), capacity_(n_logical),
+      moved_((size_t)n_layers, 0) {}
+
+int Table::init_capacity(int32_t size) {
+    if (size <= 0 || size > NB) return PIE_ERR_RANGE;
+    if (n_allocated_ != 0 || target_ >= 0) return PIE_ERR_BUSY;
+    capacity_ = size;
+    return PIE_OK;
+}
+
+int Table::resize_begin(int32_t new_size) {
+    if (new_size <= 0 || new_size > NB) return PIE_ERR_RANGE;
+    if (target_ >= 0) return PIE_ERR_BUSY;
+    if (new_size != capacity_) {
+        target_ = new_size;
+        n_moved_ = 0;
+        std::fill(moved_.begin(), moved_.end(), (uint8_t)0);
+    }
+    return PIE_OK;
+}
+
+bool Table::layer_pass(int32_t layer) {
+    if (target_ < 0 || layer < 0 || layer >= L) return false;
+    if (!moved_[(size_t)layer]) {
+        moved_[(size_t)layer] = 1;
+        ++n_moved_;
+    }
+    if (n_moved_ < L) return false;
+    capacity_ = target_;
+    target_ = -1;
+    n_moved_ = 0;
+    return true;
+}
 
 int Table::alloc(int32_t block, bool on_host) {
     if (block < 0 || block >= NB) return PIE_ERR_RANGE;
+    if (block >= alloc_limit()) return PIE_ERR_NOMEM;  // beyond the size visible now
     if (allocated_[block]) return PIE_ERR_INVALID;
     settle();
     int64_t n_gpu = on_host ? 0 : std::min<int64_t>(L, gpu_.available());
@@ -88,6 +121,7 @@ int Table::alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host) 
     settle();
     for (int64_t i = 0; i < n; ++i) {
         if (blocks[i] < 0 || blocks[i] >= NB) return PIE_ERR_RANGE;
+        if (blocks[i] >= alloc_limit()) return PIE_ERR_NOMEM;
         if (allocated_[blocks[i]]) return PIE_ERR_INVALID;
     }
     // budget: a block that is not forced to the host takes GPU slots for its first layers while any are left
@@ -178,6 +212,7 @@ int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int
     SlotPool &dst_pool = queue == PIE_Q_OUT ? host_ : gpu_;
     SlotPool &src_pool = queue == PIE_Q_OUT ? gpu_ : host_;
     if (movers > dst_pool.available()) return PIE_ERR_NOMEM;
+    layer_pass(layer);
     waits[0] = waits[1] = waits[2] = waits[3] = 0;
     *n_moved = 0;
     *ticket = 0;
@@ -366,6 +401,27 @@ int pie_table_confirm(pie_table *t, int32_t queue, int64_t ticket) {
 int pie_table_state(pie_table *t, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot,
                     int32_t *host_slot) {
     return t ? reinterpret_cast<Table *>(t)->state(layer, block, state, gpu_slot, host_slot) : PIE_ERR_INVALID;
+}
+int pie_table_init_capacity(pie_table *t, int32_t size) {
+    return t ? reinterpret_cast<Table *>(t)->init_capacity(size) : PIE_ERR_INVALID;
+}
+int pie_table_resize_begin(pie_table *t, int32_t new_size) {
+    return t ? reinterpret_cast<Table *>(t)->resize_begin(new_size) : PIE_ERR_INVALID;
+}
+int pie_table_layer_pass(pie_table *t, int32_t layer) {
+    if (!t) return PIE_ERR_INVALID;
+    Table *tb = reinterpret_cast<Table *>(t);
+    if (layer < 0 || layer >= tb->L) return PIE_ERR_RANGE;
+    return tb->layer_pass(layer) ? 1 : 0;
+}
+int pie_table_capacity(pie_table *t, int32_t *visible, int32_t *alloc_limit, int32_t *target, int32_t *layers_moved) {
+    if (!t) return PIE_ERR_INVALID;
+    Table *tb = reinterpret_cast<Table *>(t);
+    if (visible) *visible = tb->capacity();
+    if (alloc_limit) *alloc_limit = tb->alloc_limit();
+    if (target) *target = tb->resize_target();
+    if (layers_moved) *layers_moved = tb->layers_moved();
+    return PIE_OK;
 }
 
 pie_fifo *pie_fifo_create(int32_t n_layers, int32_t gpu_regions, int32_t cpu_regions, const uint8_t *on_cpu) {

@@ -1,6 +1,7 @@
 // Host-side mapping table, slot pools, whole-layer protocol scheduler and controller rule.
 // Pure C++ (no CUDA): pie_pool drives it, and it is exported through the C ABI for CPU tests.
 #pragma once
+#include <algorithm>
 #include <cstdint>
 #include <deque>
 #include <vector>
@@ -58,6 +59,18 @@ class Table {
              int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits);
     int attention(int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits);
     int confirm(int32_t queue, int64_t ticket);
+
+    // Run-time resize of the per-layer size (Section 4.1).  NB is the physical width; ids below capacity()
+    // are visible.  Growing: new ids become allocatable once every layer has gone through a swap pass;
+    // shrinking: ids at or above the new size stop being handed out at once and the size takes effect
+    // once every layer has passed (blocks still in use up there stay accessible until freed).
+    int init_capacity(int32_t size);  // before anything is allocated
+    int resize_begin(int32_t new_size);
+    bool layer_pass(int32_t layer);  // true when this call completed a resize
+    int32_t capacity() const { return capacity_; }
+    int32_t resize_target() const { return target_; }  // -1: none in progress
+    int32_t layers_moved() const { return n_moved_; }
+    int32_t alloc_limit() const { return target_ < 0 ? capacity_ : std::min(capacity_, target_); }
     int state(int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot);
 
     bool in_flight(const Unit &u) const { return u.last_q != PIE_Q_NONE && u.last_t > done_[u.last_q]; }
@@ -68,7 +81,13 @@ class Table {
     int64_t issued(int q) const { return issued_[q]; }
     int64_t done(int q) const { return done_[q]; }
     int32_t n_allocated() const { return n_allocated_; }
-    void settle() { gpu_.settle(done_); host_.settle(done_); }
+    // a slot goes to `pending` only with a ticket that is still open, so nothing can move while `done_` stands still
+    void settle() {
+        if (settled_[1] == done_[1] && settled_[2] == done_[2] && settled_[3] == done_[3]) return;
+        gpu_.settle(done_);
+        host_.settle(done_);
+        for (int q = 0; q < 4; ++q) settled_[q] = done_[q];
+    }
 
     const int32_t L, NB;
 
@@ -83,8 +102,11 @@ class Table {
     std::vector<int64_t> layer_wait_;        // per layer x 4 queues: newest open ticket among its units
     int64_t issued_[4] = {0, 0, 0, 0};
     int64_t done_[4] = {0, 0, 0, 0};
+    int64_t settled_[4] = {0, 0, 0, 0};  // done_ as of the last settle()
     uint32_t clock_ = 0;
     int32_t n_allocated_ = 0;
+    int32_t capacity_, target_ = -1, n_moved_ = 0;
+    std::vector<uint8_t> moved_;  // per layer
 };
 
 // Whole-layer protocol of Section 3.3.

@@ -1,0 +1,133 @@
+"""Ratio sweep and controller trajectory on the larger workload shapes (the synthetic counterpart of the paper's
+throughput-versus-expansion and adaptive-expansion experiments, Section 5.2 and 5.4; no request stream here, so
+what is reported is the decode step itself).
+
+    python -m paper_2411_09317_b200.sweep --workload llama3_8b  --mode ratios   [--layers N] [--steps K]
+    python -m paper_2411_09317_b200.sweep --workload llama3_70b --mode adaptive [--layers N] [--steps K]
+
+ratios:   the extension ratio is set to 0, 0.1, ... 1.0 (fraction of every layer's blocks kept host resident
+          between uses); per ratio: median step time, attention GB/s, swap GB/s per direction, share of the step
+          the computation spent waiting for blocks.
+adaptive: the controller owns the ratio.  --host-frac 0.5 (default): half of the blocks start host resident and the GPU
+          pool holds only the other half, so the ratio has a floor; --host-frac 0: everything starts on the GPU and the
+          ratio climbs from 0 until waits or slow-down appear.  Per step: ratio, floor, step time, wait share.
+Prints one JSON object per line.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import sys
+
+import numpy as np
+import torch
+
+from . import binding as pie
+from . import synth
+from .harness import DeviceWorkload
+
+
+def run_steps(dw, n):
+    """n decode steps; -> (per-step ms by CUDA events, stats before, stats after, context lengths before)"""
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    dw.sync()
+    dw.advance_context()
+    dw.decode_step()
+    before, ctx0 = pie.pie_get_stats(dw.pool), dw.ctx_lens.copy()
+    with torch.cuda.stream(dw.s_compute):
+        marks[0].record()
+    per_stats = []
+    for i in range(n):
+        dw.advance_context()
+        dw.decode_step()
+        per_stats.append(pie.pie_get_stats(dw.pool))
+        with torch.cuda.stream(dw.s_compute):
+            marks[i + 1].record()
+    dw.sync()
+    pie.pie_controller_tick(dw.pool)
+    return [marks[i].elapsed_time(marks[i + 1]) for i in range(n)], before, pie.pie_get_stats(dw.pool), ctx0, per_stats
+
+
+def attention_bytes(wl, ctx):
+    ctx = ctx.astype(np.int64)
+    return wl.n_layers * (int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2 + 2 * wl.n_seqs * wl.n_q_heads * wl.head_dim * 2
+                          + 4 * (int(((ctx + 15) // 16).sum()) + wl.n_seqs))
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="llama3_8b")
+    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive"])
+    ap.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller pools)")
+    ap.add_argument("--steps", type=int, default=6)
+    ap.add_argument("--ratios", default="", help="ratios: comma list instead of 0, 0.1, ... 1.0")
+    ap.add_argument("--host-frac", type=float, default=0.5, help="adaptive: share of the blocks that starts host resident")
+    ap.add_argument("--ctrl-step", type=float, default=1.0 / 64.0, help="adaptive: the controller's ratio step")
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args(argv)
+    out = open(args.out, "w") if args.out else sys.stdout
+
+    def emit(obj):
+        out.write(json.dumps(obj) + "\n")
+        out.flush()
+
+    wl = synth.workload(args.workload)
+    if args.layers:
+        wl = dataclasses.replace(wl, n_layers=args.layers)
+    L = wl.n_layers
+    link = {"h2d": pie.pie_probe_link(256 << 20, pie.PIE_H2D, 3), "d2h": pie.pie_probe_link(256 << 20, pie.PIE_D2H, 3),
+            "both_per_dir": pie.pie_probe_link(256 << 20, 2, 3)}
+    if args.mode == "ratios":
+        ratios = [float(x) for x in args.ratios.split(",")] if args.ratios else [round(0.1 * i, 1) for i in range(11)]
+        total = len(ratios) * (args.steps + 4) + 4
+        wl = dataclasses.replace(wl, decode_steps=total)
+        _, _, nb = wl.tables()
+        # both pools can hold everything: ratio 0 needs it on the GPU side, ratio 1 on the host side
+        dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(L + 3) * nb + 64)
+        emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
+              "kv_gb": L * nb * wl.block_bytes / 1e9, "link": link})
+        for r in ratios:
+            pie.pie_set_extension_ratio(dw.pool, r)
+            run_steps(dw, 2)
+            per, sb, sa, ctx0, _ = run_steps(dw, args.steps)
+            ms = float(np.median(per))
+            tot = sum(per) * 1e-3
+            by = attention_bytes(wl, ctx0 + (args.steps + 1) // 2)
+            emit({"ratio": r, "expansion": None if r >= 1.0 else 1.0 / (1.0 - r), "ms_per_step": ms,
+                  "attn_gbs": by / (ms * 1e-3) / 1e9, "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9,
+                  "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
+                  "wait_share": sa["last_step_stall_ms"] / max(sa["last_step_ms"], 1e-9),
+                  "last_step": {k: sa[k] for k in ("last_step_ms", "last_step_compute_ms", "last_step_stall_ms",
+                                                   "last_step_swap_in_ms", "last_step_swap_out_ms")},
+                  "calls_kernel": sa["calls_kernel"] - sb["calls_kernel"],
+                  "calls_copy_engine": sa["calls_copy_engine"] - sb["calls_copy_engine"],
+                  "swap_frac_of_link": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9 / link["both_per_dir"]})
+    else:
+        wl = dataclasses.replace(wl, decode_steps=args.steps + 8)
+        _, _, nb = wl.tables()
+        # host_frac > 0: the GPU pool is sized for the GPU-resident share only (the ratio cannot go below that share);
+        # host_frac = 0: everything fits, the host pool has room for a quarter of the blocks and the ratio climbs from 0
+        extra_host = 0 if args.host_frac > 0 else (L // 4 + 3) * nb
+        dw = DeviceWorkload(wl, host_frac=args.host_frac, timing=True, extra_host_slots=extra_host,
+                            extra_gpu_slots=0 if args.host_frac > 0 else 3 * nb)
+        emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
+              "kv_gb": L * nb * wl.block_bytes / 1e9, "gpu_pool_gb": dw.n_gpu_slots * wl.block_bytes / 1e9,
+              "host_pool_gb": dw.n_host_slots * wl.block_bytes / 1e9, "host_frac": args.host_frac,
+              "ctrl_step": args.ctrl_step, "link": link})
+        pie.pie_set_controller(dw.pool, args.ctrl_step, 0.0, 0.0)
+        pie.pie_set_extension_ratio(dw.pool, -1.0)
+        per, sb, sa, ctx0, per_stats = run_steps(dw, args.steps)
+        for i, (ms, st) in enumerate(zip(per, per_stats)):
+            emit({"step": i, "ratio": st["ratio"], "ratio_floor": st["reserved"][1], "ms_per_step": ms,
+                  "wait_share_of_last_measured_step": st["last_step_stall_ms"] / max(st["last_step_ms"], 1e-9),
+                  "slowdown_share_of_last_measured_step": st["reserved"][0] / max(st["last_step_compute_ms"], 1e-9)})
+        tot = sum(per) * 1e-3
+        emit({"summary": True, "final_ratio": sa["ratio"], "ratio_floor": sa["reserved"][1], "median_ms_per_step": float(np.median(per)),
+              "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9, "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
+              "attn_gbs": attention_bytes(wl, ctx0 + args.steps // 2) / (float(np.median(per)) * 1e-3) / 1e9})
+    dw.close()
+
+
+if __name__ == "__main__":
+    main()

@@ -66,7 +66,14 @@ def both_apply(o, t, op):
         q, frac = op[1], op[2]
         tk = int(o.issued[q] * frac)
         a, b = o.confirm(q, tk), t.confirm(q, tk)
+    elif kind == "resize":
+        a, b = o.resize_begin(op[1]), t.resize_begin(op[1])
+    elif kind == "pass":
+        a, b = int(o.layer_pass(op[1])), t.layer_pass(op[1])
     assert a == b, (op, a, b)
+    st, cap = t.capacity()
+    assert cap == {"visible": o.capacity, "alloc_limit": o.alloc_limit(), "target": -1 if o.target is None else o.target,
+                   "layers_moved": len(o.moved)}, op
     for l in range(o.L):
         for blk in range(o.NB):
             u = o._u(l, blk)
@@ -102,11 +109,30 @@ def test_table_matches_oracle_random_long():
             if rng.random() < 0.05:
                 ids = ids + (ids[0],) if rng.random() < 0.5 else ids + (NB + 3,)
             layer = rng.randrange(L) if rng.random() > 0.03 else L
+            if rng.random() < 0.06:
+                both_apply(o, t, ("resize", rng.randint(0, NB + 1)) if rng.random() < 0.5 else ("pass", rng.randrange(L)))
             op = (("alloc", rng.randrange(NB), rng.random() < 0.3) if k < 0.15 else ("free", rng.randrange(NB)) if k < 0.2
                   else ("out", layer, ids) if k < 0.45 else ("in", layer, ids) if k < 0.7
                   else ("attn", layer, ids) if k < 0.85 else ("confirm", rng.choice([1, 2, 3]), rng.random()))
             both_apply(o, t, op)
         o.check_invariants()
+
+
+def test_table_resize_matches_oracle_exhaustive_tiny():
+    """Every sequence of up to 5 calls over resize / layer pass / alloc / free / swap on a 2-layer table of width 3."""
+    alphabet = [("resize", 3), ("resize", 1), ("resize", 2), ("pass", 0), ("pass", 1), ("alloc", 0, False), ("alloc", 2, True),
+                ("free", 2), ("out", 0, (0,)), ("in", 1, (2,))]
+    n = 0
+    for length in range(1, 6):
+        for seq in itertools.product(alphabet, repeat=length):
+            if seq[0][0] not in ("resize", "alloc"):
+                continue
+            o, t = otable.MappingTable(2, 3, 4, 4, capacity=2), pie.Table(2, 3, 4, 4)
+            assert t.init_capacity(2) == pie.PIE_OK
+            for op in seq:
+                both_apply(o, t, op)
+            n += 1
+    assert n > 20000
 
 
 def test_table_attention_without_ids_waits_for_every_arriving_unit():
