@@ -45,6 +45,7 @@ def main(argv=None):
     ap.add_argument("--kv-heads", type=int, default=8)
     ap.add_argument("--fp16", action="store_true", help="fp16 instead of bf16")
     ap.add_argument("--blocks", default="", help="comma list of blocks per launch for part 2")
+    ap.add_argument("--every", type=int, default=1, help="part 2: one swap call per this many launches, carrying as many times the blocks")
     args = ap.parse_args(argv)
     out = open(args.out, "w") if args.out else sys.stdout
 
@@ -138,9 +139,11 @@ def main(argv=None):
             for mode, mname in ((pie.PIE_MODE_KERNEL, "kernel"), (pie.PIE_MODE_COPY_ENGINE, "copy_engine")):
                 for direction in ("h2d", "d2h", "both"):
                     for n in blocks:
-                        src, dst = swap_lists(n, pattern, n_swap_slots, 200 + n)
+                        src, dst = swap_lists(n * args.every, pattern, n_swap_slots, 200 + n)
 
                         def per_launch(i):
+                            if i % args.every:
+                                return
                             if direction in ("h2d", "both"):
                                 do_swap("h2d", src, dst, mode)
                             if direction in ("d2h", "both"):
@@ -152,6 +155,7 @@ def main(argv=None):
                         gbs = n * BB / (max(t1, t_swap) * 1e-3) / 1e9
                         lref = link["both_per_dir"] if direction == "both" else link[direction]
                         emit({"part": "behind_attention", "pattern": pattern, "mode": mname, "dir": direction, "blocks_per_launch": n,
+                              "swap_call_every": args.every,
                               "attn_ms": t1, "attn_ms_alone": ref, "slowdown": t1 / ref - 1.0, "swap_gbs_per_dir": gbs,
                               "frac_of_link": gbs / lref, "swap_keeps_up": t_swap <= t1 * 1.02})
     dw.close()

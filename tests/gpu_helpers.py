@@ -10,7 +10,8 @@ from paper_2411_09317_b200 import synth
 
 
 class PoolCase:
-    def __init__(self, case, n_gpu_slots=None, n_host_slots=None, split_tokens=0, timing=0, all_on_gpu=False):
+    def __init__(self, case, n_gpu_slots=None, n_host_slots=None, split_tokens=0, timing=0, all_on_gpu=False,
+                 visible_blocks=0):
         self.c = case
         L, NB = case.L, case.NB
         on_host = np.zeros(NB, dtype=np.uint8) if all_on_gpu else case.unit_side[0].astype(np.uint8)
@@ -20,18 +21,22 @@ class PoolCase:
         self.pool = pie.pie_pool_create(n_layers=L, n_q_heads=case.Hq, n_kv_heads=case.Hkv, head_dim=case.D,
                                         dtype=case.dtype, n_logical_blocks=NB, max_seqs=max(case.S, 1),
                                         n_gpu_slots=self.n_gpu_slots, n_host_slots=self.n_host_slots,
-                                        split_tokens=split_tokens, timing=timing)
-        ids = pie.pie_block_alloc(self.pool, NB, on_host)
-        assert np.array_equal(ids, np.arange(NB))
-        for l in range(L):
-            for b in range(NB):
-                pie.pie_block_write(self.pool, l, b, self.unit_bits(l, b))
+                                        split_tokens=split_tokens, timing=timing, visible_blocks=visible_blocks)
+        n0 = visible_blocks or NB          # with a smaller visible size only that many blocks exist at first
+        ids = pie.pie_block_alloc(self.pool, n0, on_host[:n0])
+        assert np.array_equal(ids, np.arange(n0))
+        self.write_blocks(range(n0))
         dev = torch.device("cuda:0")
         self.q = torch.from_numpy(case.q.view(np.int16)).to(dev)              # [L][S][Hq][D]
         self.out = torch.zeros_like(self.q)
         self.bt = torch.from_numpy(case.block_table).to(dev)
         self.ctx = torch.from_numpy(case.ctx_lens.astype(np.int32)).to(dev)
         torch.cuda.synchronize()
+
+    def write_blocks(self, ids):
+        for l in range(self.c.L):
+            for b in ids:
+                pie.pie_block_write(self.pool, l, int(b), self.unit_bits(l, int(b)))
 
     def unit_bits(self, l, b):
         c = self.c

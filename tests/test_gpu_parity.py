@@ -371,6 +371,70 @@ def test_block_free_and_reuse_and_nomem():
     pc.close()
 
 
+# ---------------------------------------------------------------- run-time resize (Section 4.1) on a live pool
+def test_resize_grow_then_shrink_while_serving():
+    """The per-layer size grows from 8 to 11 blocks and shrinks back while attention calls keep running: new ids appear
+    only after every layer has gone through a swap pass, doomed ids stop being handed out at once, blocks in use beyond
+    the new size stay readable, and every attention result along the way matches the oracle."""
+    full = np.array([40, 70, 33], dtype=np.int32)                  # 3 + 5 + 3 blocks
+    case = Case(3, 8, 4, 64, F16, full, seed=51)
+    assert case.NB == 11 and list(case.block_table[2, :3]) == [8, 9, 10]
+    pc = PoolCase(case, n_gpu_slots=3 * 11 + 4, n_host_slots=8, visible_blocks=8)
+    two = np.array([40, 70, 0], dtype=np.int32)                    # the third sequence has nothing yet
+
+    def check(layer, lens):
+        case.ctx_lens = lens
+        pc.ctx.copy_(torch.from_numpy(lens).cuda())
+        check_attention(case, pc, layer, edge=True)
+
+    def nomem():
+        with pytest.raises(pie.PieError) as e:
+            pie.pie_block_alloc(pc.pool, 1)
+        assert e.value.status == pie.PIE_ERR_NOMEM
+
+    assert pie.pie_resize_status(pc.pool) == {"visible": 8, "alloc_limit": 8, "target": -1, "layers_moved": 0}
+    nomem()
+    check(0, two)
+    pie.pie_resize_begin(pc.pool, 11)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_resize_begin(pc.pool, 10)
+    assert e.value.status == pie.PIE_ERR_BUSY
+    nomem()                                                        # prepared first, visible later
+    pie.pie_plan_layer(pc.pool, 0, case.NB)
+    pie.pie_plan_layer(pc.pool, 1, case.NB)
+    assert pie.pie_resize_status(pc.pool) == {"visible": 8, "alloc_limit": 8, "target": 11, "layers_moved": 2}
+    nomem()
+    check(1, two)                                                  # blocks within the old size stay usable meanwhile
+    pie.pie_swap_out(pc.pool, 2, [0, 5])                           # a swap call on the last layer is its pass
+    assert pie.pie_resize_status(pc.pool) == {"visible": 11, "alloc_limit": 11, "target": -1, "layers_moved": 0}
+    pie.pie_swap_in(pc.pool, 2, [0, 5])
+    ids = pie.pie_block_alloc(pc.pool, 3)
+    assert ids.tolist() == [8, 9, 10]
+    pc.write_blocks(ids)
+    for l in range(3):
+        check(l, full)
+    # shrink back: nothing new is handed out beyond 8 from this moment, the blocks in use up there still serve
+    pie.pie_resize_begin(pc.pool, 8)
+    assert pie.pie_resize_status(pc.pool)["alloc_limit"] == 8
+    pie.pie_sync(pc.pool)
+    pie.pie_block_free(pc.pool, [10])
+    nomem()
+    shorter = np.array([40, 70, 32], dtype=np.int32)               # the third sequence without its last block
+    check(0, shorter)
+    for l in range(3):
+        pie.pie_plan_layer(pc.pool, l, case.NB)
+    assert pie.pie_resize_status(pc.pool) == {"visible": 8, "alloc_limit": 8, "target": -1, "layers_moved": 0}
+    check(2, shorter)                                              # still accessible after the size took effect
+    pie.pie_sync(pc.pool)
+    pie.pie_block_free(pc.pool, [8, 9])
+    nomem()
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_resize_begin(pc.pool, 12)
+    assert e.value.status == pie.PIE_ERR_RANGE
+    check(1, two)
+    pc.close()
+
+
 # ---------------------------------------------------------------- the paper's whole-layer protocol on the GPU
 def test_whole_layer_protocol_nine_layers():
     """Nine layers, layers 8 and 9 on the CPU at the start, seven GPU regions and four CPU regions (the paper's worked
