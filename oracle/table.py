@@ -80,8 +80,12 @@ class _SlotPool:
 
 
 class MappingTable:
-    def __init__(self, n_layers, n_logical, n_gpu_slots, n_host_slots, capacity=None):
+    def __init__(self, n_layers, n_logical, n_gpu_slots, n_host_slots, capacity=None, retain=False):
         self.L, self.NB = n_layers, n_logical
+        # Variant beyond the paper (which gives the CPU region up after a swap-in, Section 3.2): with `retain` a unit
+        # that is brought in keeps its host slot, and pushing it out again copies nothing unless it was written
+        # meanwhile (`mark_dirty`: the append of the new token goes into one block per sequence).
+        self.retain = retain
         if capacity is not None and not 0 < capacity <= n_logical:
             raise ValueError("capacity")
         self.gpu = _SlotPool(n_gpu_slots)
@@ -93,6 +97,8 @@ class MappingTable:
         self.last_q = [Q_NONE] * n      # queue and ticket of the last copy issued on the unit
         self.last_t = [0] * n
         self.allocated = [False] * n_logical
+        self.dirty = [False] * n        # written on the GPU since the host copy was taken (meaningful with a kept host slot)
+        self.last_elided = []           # per pair of the last swap(): True where no bytes need to move
         self.issued = {Q_IN: 0, Q_OUT: 0, Q_COMPUTE: 0}
         self.done = {Q_NONE: 0, Q_IN: 0, Q_OUT: 0, Q_COMPUTE: 0}
         self.clock = 0
@@ -186,6 +192,7 @@ class MappingTable:
             self.gpu_slot[u] = slot if side == GPU else -1
             self.host_slot[u] = slot if side == HOST else -1
             self.last_q[u], self.last_t[u] = tag
+            self.dirty[u] = False
         self.allocated[block] = True
         return OK
 
@@ -205,6 +212,8 @@ class MappingTable:
             if self.side[u] == GPU:
                 ct = self.issued[Q_COMPUTE]
                 self.gpu.release(self.gpu_slot[u], Q_COMPUTE if ct > self.done[Q_COMPUTE] else Q_NONE, ct)
+                if self.host_slot[u] >= 0:          # a kept host copy goes with the unit
+                    self.host.release(self.host_slot[u], Q_NONE, 0)
             else:
                 self.host.release(self.host_slot[u], Q_NONE, 0)
             self.side[u], self.gpu_slot[u], self.host_slot[u] = FREE, -1, -1
@@ -241,36 +250,60 @@ class MappingTable:
         movers = [b for b in ids if self.side[self._u(layer, b)] != want]
         dst_pool = self.host if direction == Q_OUT else self.gpu
         src_pool = self.gpu if direction == Q_OUT else self.host
-        if len(movers) > dst_pool.available():
+        # a unit that kept its host slot goes back into it: only the others need a new one
+        need = [b for b in movers if direction == Q_IN or self.host_slot[self._u(layer, b)] < 0]
+        if len(need) > dst_pool.available():
             return ERR_NOMEM, 0, [], {}
         self.layer_pass(layer)
+        self.last_elided = []
         if not movers:
             return OK, 0, [], {}
-        slots, waits, _ = dst_pool.take(len(movers))
+        slots, waits, _ = dst_pool.take(len(need))
+        slots = iter(slots)
         self.issued[direction] += 1
         ticket = self.issued[direction]
         self.clock += 1
         pairs = []
-        for b, dst in zip(movers, slots):
+        for b in movers:
             u = self._u(layer, b)
             if self._in_flight(u):  # the copy that is still bringing the unit to where it is now
                 waits[self.last_q[u]] = max(waits.get(self.last_q[u], 0), self.last_t[u])
             if direction == Q_OUT:
                 src = self.gpu_slot[u]
+                if self.host_slot[u] >= 0:
+                    dst, elide = self.host_slot[u], not self.dirty[u]   # the kept copy is still good unless written
+                else:
+                    dst, elide = next(slots), False
                 self.host_slot[u], self.gpu_slot[u] = dst, -1
+                self.dirty[u] = False
+                src_pool.release(src, direction, ticket)
             else:
-                src = self.host_slot[u]
-                self.gpu_slot[u], self.host_slot[u] = dst, -1
-            src_pool.release(src, direction, ticket)
+                src, dst, elide = self.host_slot[u], next(slots), False
+                self.gpu_slot[u] = dst
+                if not self.retain:
+                    self.host_slot[u] = -1
+                    src_pool.release(src, direction, ticket)
+                # with `retain` the host slot stays the unit's; `dirty` keeps whatever it was: a mark made before the
+                # unit came in (the step's append is declared up front) must survive until the next copy out
             self.side[u] = want
             self.last_q[u], self.last_t[u] = direction, ticket
             self.t_last[u] = self.clock
             pairs.append((b, src, dst))
+            self.last_elided.append(elide)
         if direction == Q_OUT and self.last_compute[layer] > self.done[Q_COMPUTE]:
             # the layer's attention call also appends the new token: copy out only after it
             waits[Q_COMPUTE] = max(waits.get(Q_COMPUTE, 0), self.last_compute[layer])
         waits.pop(direction, None)  # same queue: ordered anyway
         return OK, ticket, pairs, waits
+
+    def mark_dirty(self, layer, ids):
+        """The layer's next attention call appends into these blocks: their host copies, where kept, go stale."""
+        st = self._check_ids(layer, ids)
+        if st != OK:
+            return st
+        for b in ids:
+            self.dirty[self._u(layer, b)] = True
+        return OK
 
     # ---- presence check (Section 3.2: computation may start only on units present on the GPU) ----
     def attention(self, layer, ids):
@@ -301,7 +334,7 @@ class MappingTable:
             assert len(set(free)) == len(free), f"{n}: a slot is free twice"
         for u, side in enumerate(self.side):
             if side == GPU:
-                assert self.gpu_slot[u] >= 0 and self.host_slot[u] < 0
+                assert self.gpu_slot[u] >= 0   # a host slot may be kept beside it (retain)
             elif side == HOST:
                 assert self.host_slot[u] >= 0 and self.gpu_slot[u] < 0
             else:

@@ -50,17 +50,19 @@ class Executor:
 
     def __init__(self, tbl, rng):
         self.t, self.rng = tbl, rng
-        self.g = {}   # gpu slot -> tag
+        self.g = {}   # gpu slot -> tag = (layer, block, version); an append bumps the version where the unit then lives
         self.h = {}
+        self.version = {}   # (layer, block) -> number of appends the device has run on it
         self.ops = {table.Q_IN: [], table.Q_OUT: [], table.Q_COMPUTE: []}
         self.ran = {table.Q_IN: 0, table.Q_OUT: 0, table.Q_COMPUTE: 0}
 
     def write_unit(self, layer, block):  # host-side initial fill at alloc time (synchronous)
         u = self.t._u(layer, block)
+        self.version[(layer, block)] = 0
         if self.t.side[u] == table.GPU:
-            self.g[self.t.gpu_slot[u]] = (layer, block)
+            self.g[self.t.gpu_slot[u]] = (layer, block, 0)
         else:
-            self.h[self.t.host_slot[u]] = (layer, block)
+            self.h[self.t.host_slot[u]] = (layer, block, 0)
 
     def issue(self, queue, ticket, waits, body):
         assert ticket == len(self.ops[queue]) + 1
@@ -103,24 +105,37 @@ def apply_op(tbl, ex, op):
         q = table.Q_OUT if kind == "out" else table.Q_IN
         st, ticket, pairs, waits = tbl.swap(q, op[1], list(op[2]))
         if st == table.OK and ticket:
-            layer = op[1]
+            layer, elided = op[1], list(tbl.last_elided)
+            assert len(elided) == len(pairs) and (tbl.retain or not any(elided))
 
-            def body(pairs=pairs, layer=layer, q=q):
+            def body(pairs=pairs, layer=layer, q=q, elided=elided):
                 src, dst = (ex.g, ex.h) if q == table.Q_OUT else (ex.h, ex.g)
-                for b, s, d in pairs:
-                    assert src.get(s) == (layer, b), f"copy read slot {s}: {src.get(s)} != {(layer, b)}"
-                    dst[d] = src[s]
+                for (b, s, d), skip in zip(pairs, elided):
+                    want = (layer, b, ex.version[(layer, b)])
+                    assert src.get(s) == want, f"copy read slot {s}: {src.get(s)} != {want}"
+                    if skip:    # no bytes move: the destination must already hold exactly what the copy would bring
+                        assert dst.get(d) == want, f"elided copy, but slot {d} holds {dst.get(d)} != {want}"
+                    else:
+                        dst[d] = src[s]
             ex.issue(q, ticket, waits, body)
         return st
-    if kind == "attn":
-        st, ticket, waits = tbl.attention(op[1], list(op[2]))
+    if kind in ("attn", "attn_append"):
+        ids = list(op[2])
+        appended = [b for b in ids if b in op[3]] if kind == "attn_append" else []
+        if appended and tbl.mark_dirty(op[1], appended) != table.OK:
+            appended = []   # the attention call below fails on the same ids
+        st, ticket, waits = tbl.attention(op[1], ids)
         if st == table.OK:
-            layer, ids = op[1], list(op[2])
+            layer = op[1]
             slots = [tbl.gpu_slot[tbl._u(layer, b)] for b in ids]
 
             def body():
                 for b, s in zip(ids, slots):
-                    assert ex.g.get(s) == (layer, b), f"attention read slot {s}: {ex.g.get(s)}"
+                    want = (layer, b, ex.version[(layer, b)])
+                    assert ex.g.get(s) == want, f"attention read slot {s}: {ex.g.get(s)} != {want}"
+                    if b in appended:   # the new token's K/V rows land in this block
+                        ex.version[(layer, b)] += 1
+                        ex.g[s] = (layer, b, ex.version[(layer, b)])
             ex.issue(table.Q_COMPUTE, ticket, waits, body)
         return st
     if kind == "confirm":  # the host learns how far the device got
@@ -141,9 +156,9 @@ def final_check(tbl, ex):
         for b in range(tbl.NB):
             u = tbl._u(l, b)
             if tbl.side[u] == table.GPU:
-                assert ex.g.get(tbl.gpu_slot[u]) == (l, b)
+                assert ex.g.get(tbl.gpu_slot[u]) == (l, b, ex.version[(l, b)])
             elif tbl.side[u] == table.HOST:
-                assert ex.h.get(tbl.host_slot[u]) == (l, b)
+                assert ex.h.get(tbl.host_slot[u]) == (l, b, ex.version[(l, b)])   # the newest bytes, also after elided copies
     tbl.check_invariants()
 
 
@@ -169,6 +184,70 @@ def test_table_exhaustive_tiny():
             final_check(tbl, ex)
             n_seq += 1
     assert n_seq > 10000
+
+
+def test_table_exhaustive_tiny_with_kept_host_copies():
+    """The same enumeration with host copies kept after a swap-in and appends that write into blocks: an elided copy
+    out never leaves stale bytes on the host, whatever the order the device runs things in."""
+    alphabet = [("alloc", 0), ("alloc", 1), ("free", 0), ("out", 0, (0,)), ("out", 1, (0, 1)), ("in", 0, (0,)),
+                ("in", 1, (1, 0)), ("attn", 0, (0,)), ("attn_append", 0, (0,), (0,)), ("attn_append", 1, (0, 1), (1,)),
+                ("confirm", True), ("run", 1)]
+    n_seq = n_elided = 0
+    # from a warm state: both blocks allocated and every unit once out and back in, so that host copies are kept
+    warm = [("alloc", 0), ("alloc", 1), ("out", 0, (0, 1)), ("out", 1, (0, 1)), ("in", 0, (0, 1)), ("in", 1, (0, 1)), ("confirm", True)]
+    for length in range(1, 5):
+        for seq in itertools.product(alphabet, repeat=length):
+            tbl = table.MappingTable(2, 2, 4, 4, retain=True)
+            ex = Executor(tbl, random.Random(n_seq))
+            for op in warm:
+                assert apply_op(tbl, ex, op) == table.OK
+            for op in seq:
+                snap = (list(tbl.side), list(tbl.gpu_slot), list(tbl.host_slot), list(tbl.gpu.ready), list(tbl.host.ready))
+                st = apply_op(tbl, ex, op)
+                if st != table.OK and op[0] != "attn_append":   # (a failed attention call may have left its dirty marks)
+                    assert snap == (list(tbl.side), list(tbl.gpu_slot), list(tbl.host_slot), list(tbl.gpu.ready),
+                                    list(tbl.host.ready)), f"failed call {op} changed the table"
+                if st == table.OK and op[0] == "out":
+                    n_elided += sum(tbl.last_elided)
+                tbl.check_invariants()
+            final_check(tbl, ex)
+            n_seq += 1
+    assert n_seq > 10000 and n_elided > 500
+
+
+def test_kept_host_copy_is_reused_and_written_blocks_are_copied():
+    t = table.MappingTable(1, 3, 3, 3, retain=True)
+    assert [t.alloc(b, on_host=True) for b in range(3)] == [table.OK] * 3
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [0, 1, 2])
+    assert st == table.OK and t.last_elided == [False] * 3
+    home = [p[1] for p in pairs]
+    assert [t.host_slot[u] for u in range(3)] == home and t.host.available() == 0     # the host slots stay the units'
+    t.confirm(table.Q_IN, tk)
+    assert t.mark_dirty(0, [2]) == table.OK                                            # the step's append goes into block 2
+    assert t.attention(0, [0, 1, 2])[0] == table.OK
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [0, 1, 2])
+    assert st == table.OK and t.last_elided == [True, True, False]                     # only the written block is copied
+    assert [p[2] for p in pairs] == home                                               # ... and everyone returns to its slot
+    assert waits == {table.Q_COMPUTE: 1}                                               # after the attention call, as ever
+    assert t.gpu.available() == 3                                                      # the GPU slots are given up (pending)
+    t.confirm(table.Q_COMPUTE, 1); t.confirm(table.Q_OUT, tk)
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [2])
+    t.confirm(table.Q_IN, tk)
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [2])                                 # not written since: nothing to copy
+    assert t.last_elided == [True]
+    # a mark made while the unit is still on the host (the step's appends are declared up front) survives the swap-in
+    t.confirm(table.Q_OUT, tk)
+    assert t.mark_dirty(0, [2]) == table.OK
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [2]); t.confirm(table.Q_IN, tk)
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [2])
+    assert t.last_elided == [False]
+    # without the option every copy out moves bytes and takes a fresh host slot
+    t2 = table.MappingTable(1, 1, 1, 2)
+    t2.alloc(0, on_host=True)
+    st, tk, pairs, _ = t2.swap(table.Q_IN, 0, [0]); t2.confirm(table.Q_IN, tk)
+    assert t2.host_slot[0] == -1
+    st, tk, pairs, _ = t2.swap(table.Q_OUT, 0, [0])
+    assert t2.last_elided == [False] and pairs[0][2] == 1                              # FIFO: the other host slot
 
 
 def test_table_error_codes_and_two_phase_states():
@@ -210,11 +289,13 @@ def test_table_nomem_and_slot_recycling_waits():
     assert st == table.OK and pairs[0][2] == 0 and waits == {table.Q_OUT: 1}
 
 
-def test_table_random_long_runs():
+@pytest.mark.parametrize("retain", [False, True])
+def test_table_random_long_runs(retain):
     rng = random.Random(5)
     for trial in range(60):
         L, NB = rng.choice([(1, 6), (3, 4), (2, 8)])
-        tbl = table.MappingTable(L, NB, rng.randint(NB, L * NB), rng.randint(NB, L * NB))
+        tbl = table.MappingTable(L, NB, rng.randint(NB, L * NB), rng.randint(NB, L * NB) + (L * NB if retain else 0),
+                                 retain=retain)
         ex = Executor(tbl, rng)
         for _ in range(120):
             k = rng.random()
@@ -222,7 +303,8 @@ def test_table_random_long_runs():
             layer = rng.randrange(L)
             op = (("alloc", rng.randrange(NB)) if k < 0.15 else ("free", rng.randrange(NB)) if k < 0.2 else
                   ("out", layer, ids) if k < 0.45 else ("in", layer, ids) if k < 0.7 else
-                  ("attn", layer, ids) if k < 0.85 else ("confirm", rng.random() < 0.3) if k < 0.93 else ("run", 2))
+                  ("attn", layer, ids) if k < 0.78 else ("attn_append", layer, ids, set(rng.sample(ids, 1))) if k < 0.85 else
+                  ("confirm", rng.random() < 0.3) if k < 0.93 else ("run", 2))
             apply_op(tbl, ex, op)
             tbl.check_invariants()
         final_check(tbl, ex)
