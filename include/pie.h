@@ -74,7 +74,8 @@ typedef struct pie_pool_config {
     int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (512) */
     int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
     int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
-    int32_t timing;            /* 1: record per-layer events for pie_controller_tick / pie_get_stats;
+    int32_t timing;            /* 1: per-layer timing for pie_controller_tick / pie_get_stats (the attention kernel notes
+                                *    the GPU's timer in host-visible memory; timing events only on the copy streams);
                                 * 2: also keep the per-layer timeline for pie_get_step_timeline */
     int32_t reserved[7];       /* [0]: attention kernel variant for tuning (0 = default);
                                 * [1]: per-layer size visible to allocation at creation, in blocks (0 = n_logical_blocks;
@@ -84,14 +85,17 @@ typedef struct pie_pool_config {
 typedef struct pie_stats {
     double bytes_in, bytes_out;            /* swapped so far, per direction */
     double calls_kernel, calls_copy_engine;
-    double last_step_compute_ms;           /* sum over layers: attention (+append, combine) time */
-    double last_step_stall_ms;             /* sum over layers: compute stream waiting for swap-in */
+    double last_step_compute_ms;           /* sum over layers: end of the previous layer's attention kernel to the end
+                                            * of this one's (append, combine and launch gap included), minus the stall */
+    double last_step_stall_ms;             /* sum over layers that had units brought in: what the gap before the layer's
+                                            * attention kernel exceeds the step's usual gap by (the presence wait) */
     double last_step_swap_in_ms, last_step_swap_out_ms;
     double last_step_ms;                   /* first layer's start to last layer's end */
     double ratio;                          /* current extension ratio */
     int64_t n_units_gpu, n_units_host, n_units_in_flight;
     int64_t steps_measured;
     double reserved[8];                    /* [0]: last step's attention slow-down vs the no-swap record, ms;
+                                            * [2]: bytes of swap-out traffic elided so far (pie_set_retention);
                                             * [1]: the smallest extension ratio the GPU pool's size allows with the
                                             *      blocks allocated now (the controller never goes below it) */
 } pie_stats;
@@ -212,6 +216,20 @@ int pie_get_extension_ratio(pie_pool *pool, float *r);
  * the time-per-token record taken on steps without swap traffic (copies that are hidden can still slow the
  * attention down through shared HBM bandwidth). */
 int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
+/* ---- kept host copies and write-back elision (a variant the paper does not have: Section 3.2 gives the
+ * CPU region up once a unit has been swapped in) ---------------------------------------------------------
+ * on != 0: a unit that is swapped in keeps its host slot; when it is swapped out again it returns to that slot, and
+ * no bytes are copied unless the unit was written on the GPU meanwhile.  In decode only the block that receives
+ * the new token is written per sequence, so nearly all of the device-to-host traffic of Section 3.3's protocol
+ * disappears; the price is host memory for every unit of the host-resident set even while it is on the GPU.
+ * Which blocks an attention call with k_new/v_new writes: derived from block_table_host / ctx_lens_host when the
+ * call gets them; otherwise the ids given to pie_declare_append_blocks (host, n ids; valid until replaced; the
+ * caller vouches for them - a block that is written but not listed would leave a stale host copy); with
+ * neither (n < 0 or never declared), every block of the layer counts as written and nothing is elided.
+ * Switching off takes effect unit by unit at its next swap-in.  pie_stats.reserved[2] counts the bytes elided. */
+int pie_set_retention(pie_pool *pool, int32_t on);
+int pie_declare_append_blocks(pie_pool *pool, const int32_t *ids, int64_t n);
+
 /* ---- run-time resize of the per-layer cache size (Section 4.1) -----------------------------------
  * n_logical_blocks is the physical width of the per-layer tables; the size visible to allocation is
  * reserved[1] of the configuration at creation (0: the full width) and changes in two phases:
@@ -238,10 +256,12 @@ int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in
 int pie_controller_tick(pie_pool *pool, int32_t *changed);
 int pie_get_stats(pie_pool *pool, pie_stats *out);
 /* Per-layer timeline of the most recently evaluated step (timing = 2 in the configuration; timing = 1 keeps the
- * statistics and the controller but not this table, which costs a few hundred event queries per step): ms[l][7] = {compute stream reaches the
- * layer, presence wait over, layer done, swap-in start, swap-in end, swap-out start, swap-out end} in ms
- * from the step's first event; -1 where nothing was recorded.  capacity = floats available (>= 7 * n_layers).
- * PIE_ERR_INVALID if no step has been evaluated yet.  Shows what overlapped with what. */
+ * statistics and the controller but not this table): ms[l][7] = {end of the previous layer's attention kernel,
+ * start of this layer's, its end, swap-in list start, end, swap-out list start, end} in ms from the start of the
+ * step's first attention kernel; -1 where nothing was recorded.  The compute columns are the kernels' own GPU-timer
+ * stamps; the copy columns are copy-stream events tied to them through one event recorded just before the step's
+ * first kernel (a few us of slack).  capacity = floats available (>= 7 * n_layers).  PIE_ERR_INVALID if no step has
+ * been evaluated yet.  Shows what overlapped with what. */
 int pie_get_step_timeline(pie_pool *pool, float *ms, int64_t capacity);
 /* Wait until everything enqueued so far has completed, at most timeout_us (PIE_ERR_TIMEOUT); applies
  * phase-2 updates and reports a pending device status word (PIE_ERR_NOT_RESIDENT ...). */
@@ -304,6 +324,14 @@ int pie_table_swap(pie_table *t, int32_t queue, int32_t layer, const int32_t *id
 int pie_table_attention(pie_table *t, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits);
 int pie_table_confirm(pie_table *t, int32_t queue, int64_t ticket);
 int pie_table_state(pie_table *t, int32_t layer, int32_t block, int32_t *state, int32_t *gpu_slot, int32_t *host_slot);
+/* pie_table_swap with one more output: elided[i] = 1 where pair i needs no bytes moved (see pie_set_retention). */
+int pie_table_swap_ex(pie_table *t, int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket,
+                      int32_t *moved_ids, int32_t *src_slots, int32_t *dst_slots, uint8_t *elided, int64_t *n_moved,
+                      int64_t *waits);
+int pie_table_set_retention(pie_table *t, int32_t on);
+int pie_table_mark_dirty(pie_table *t, int32_t layer, const int32_t *ids, int64_t n);
+/* A unit that lives on the GPU gives its kept host slot up (no-op otherwise). */
+int pie_table_drop_host_copy(pie_table *t, int32_t layer, int32_t block);
 /* Run-time resize on the bare table: see pie_resize_begin.  pie_table_init_capacity sets the visible size
  * before anything is allocated; pie_table_layer_pass returns 1 when the call completed a resize, else 0
  * (pie_table_swap makes the same mark for its layer). */

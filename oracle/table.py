@@ -296,6 +296,21 @@ class MappingTable:
         waits.pop(direction, None)  # same queue: ordered anyway
         return OK, ticket, pairs, waits
 
+    def drop_host_copy(self, layer, block):
+        """A unit that lives on the GPU gives its kept host slot up (it left the host-resident set).  The slot may
+        still be read by the copy that is bringing the unit in: whoever gets it next waits for that copy."""
+        if not 0 <= layer < self.L or not 0 <= block < self.NB:
+            return ERR_RANGE
+        if not self.allocated[block]:
+            return ERR_INVALID
+        self._settle()
+        u = self._u(layer, block)
+        if self.side[u] == GPU and self.host_slot[u] >= 0:
+            tag = (self.last_q[u], self.last_t[u]) if self._in_flight(u) else (Q_NONE, 0)
+            self.host.release(self.host_slot[u], *tag)
+            self.host_slot[u] = -1
+        return OK
+
     def mark_dirty(self, layer, ids):
         """The layer's next attention call appends into these blocks: their host copies, where kept, go stale."""
         st = self._check_ids(layer, ids)

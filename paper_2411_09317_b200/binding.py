@@ -35,7 +35,8 @@ EXPORTS = [
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
-    "pie_table_capacity",
+    "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
+    "pie_declare_append_blocks",
 ]
 
 
@@ -111,6 +112,12 @@ _sig = {
     "pie_table_attention": (_i32, [_vp, _i32, _vp, _i64, ctypes.POINTER(_i64), _vp]),
     "pie_table_confirm": (_i32, [_vp, _i32, _i64]),
     "pie_table_state": (_i32, [_vp, _i32, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "pie_table_swap_ex": (_i32, [_vp, _i32, _i32, _vp, _i64, ctypes.POINTER(_i64), _vp, _vp, _vp, _vp, ctypes.POINTER(_i64), _vp]),
+    "pie_table_set_retention": (_i32, [_vp, _i32]),
+    "pie_table_mark_dirty": (_i32, [_vp, _i32, _vp, _i64]),
+    "pie_table_drop_host_copy": (_i32, [_vp, _i32, _i32]),
+    "pie_set_retention": (_i32, [_vp, _i32]),
+    "pie_declare_append_blocks": (_i32, [_vp, _vp, _i64]),
     "pie_table_init_capacity": (_i32, [_vp, _i32]),
     "pie_table_resize_begin": (_i32, [_vp, _i32]),
     "pie_table_layer_pass": (_i32, [_vp, _i32]),
@@ -175,6 +182,18 @@ def pie_pool_create(**kw) -> int:
 
 def pie_pool_destroy(pool) -> None:
     check(lib.pie_pool_destroy(pool), "pie_pool_destroy")
+
+
+def pie_set_retention(pool, on) -> None:
+    check(lib.pie_set_retention(pool, int(on)), "pie_set_retention")
+
+
+def pie_declare_append_blocks(pool, ids) -> None:
+    if ids is None:
+        check(lib.pie_declare_append_blocks(pool, None, -1), "pie_declare_append_blocks")
+    else:
+        ids = _np_i32(ids)
+        check(lib.pie_declare_append_blocks(pool, _ptr(ids), len(ids)), "pie_declare_append_blocks")
 
 
 def pie_resize_begin(pool, new_blocks) -> None:
@@ -376,13 +395,25 @@ class Table:
         ids = _np_i32(ids)
         n = max(len(ids), 1)
         moved, src, dst = np.zeros(n, np.int32), np.zeros(n, np.int32), np.zeros(n, np.int32)
+        elided = np.zeros(n, np.uint8)
         waits = np.zeros(4, np.int64)
         ticket, n_moved = _i64(), _i64()
-        st = lib.pie_table_swap(self.h, queue, layer, _ptr(ids), len(ids), ctypes.byref(ticket), _ptr(moved), _ptr(src),
-                                _ptr(dst), ctypes.byref(n_moved), _ptr(waits))
+        st = lib.pie_table_swap_ex(self.h, queue, layer, _ptr(ids), len(ids), ctypes.byref(ticket), _ptr(moved), _ptr(src),
+                                   _ptr(dst), _ptr(elided), ctypes.byref(n_moved), _ptr(waits))
         k = n_moved.value if st == PIE_OK else 0
         pairs = [(int(moved[i]), int(src[i]), int(dst[i])) for i in range(k)]
+        self.last_elided = [bool(elided[i]) for i in range(k)]   # pairs that need no bytes moved (kept host copies)
         return st, (ticket.value if st == PIE_OK else 0), pairs, {q: int(waits[q]) for q in range(1, 4) if waits[q]}
+
+    def set_retention(self, on):
+        return lib.pie_table_set_retention(self.h, int(on))
+
+    def mark_dirty(self, layer, ids):
+        ids = _np_i32(ids)
+        return lib.pie_table_mark_dirty(self.h, layer, _ptr(ids), len(ids))
+
+    def drop_host_copy(self, layer, block):
+        return lib.pie_table_drop_host_copy(self.h, layer, block)
 
     def attention(self, layer, ids):
         waits = np.zeros(4, np.int64)

@@ -18,6 +18,14 @@ constexpr int SWAP_THREADS = 256;
 constexpr int SWAP_UNROLL = 8;
 constexpr int SWAP_CHUNK_VECS = SWAP_THREADS * SWAP_UNROLL;  // 16-byte vectors per chunk
 
+// Time stamps: kernels note the GPU's nanosecond timer in host-visible memory instead of the host putting timing
+// events between the kernels of the compute stream (a timing event there costs the stream 2-3 us per record).
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
 __global__ void __launch_bounds__(SWAP_THREADS)
 swap_kernel(const uint4 *__restrict__ src_pool, uint4 *__restrict__ dst_pool, const int32_t *__restrict__ list,
             int64_t n, int32_t vecs_per_block, int32_t chunks_per_block, int32_t *slot_table, int table_mode) {
@@ -274,6 +282,7 @@ struct AttnParams {
     float *part_o;
     float *part_ml;
     int32_t *counters;  // [0] next item, [1] CTAs that have left
+    uint64_t *stamps;   // optional, host visible: [0] when CTA 0 started, [1] when the last CTA left (globaltimer ns)
     int32_t *status;
     int64_t n_gpu_slots;
     int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d, max_chunks;
@@ -368,6 +377,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     int32_t *co_smem = reinterpret_cast<int32_t *>(smem + SM::OFF_CO);
 
     if (tid == 0) {
+        if (p.stamps != nullptr && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps) = globaltimer_ns();
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
@@ -726,6 +736,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (old == (int32_t)gridDim.x - 1) {
             p.counters[0] = 0;
             p.counters[1] = 0;
+            if (p.stamps != nullptr) *reinterpret_cast<volatile uint64_t *>(p.stamps + 1) = globaltimer_ns();
         }
     }
 }
@@ -949,6 +960,7 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.part_o = sc.part_o;
     p.part_ml = sc.part_ml;
     p.counters = sc.counters;
+    p.stamps = a.stamps;
     p.status = a.status;
     p.n_gpu_slots = sh.n_gpu_slots;
     p.max_blocks = a.max_blocks;

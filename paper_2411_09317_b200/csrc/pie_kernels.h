@@ -58,6 +58,7 @@ struct AttnLaunch {
     int32_t grid;               // persistent CTAs
     int32_t variant;            // kernel variant (0 = default)
     int32_t *status;            // device-visible status word
+    uint64_t *stamps = nullptr; // optional, device-visible: [0] start, [1] end of the attention kernel (GPU timer, ns)
 };
 
 // Build the TMA descriptors of the HBM pool: map3d covers a whole K+V tile in one copy

@@ -21,6 +21,7 @@ constexpr int LIST_EVENTS = 512;   // events guarding regions of the id-list rin
 constexpr int TIMING_RING = 4;     // the host may enqueue at most this many steps ahead of their evaluation
 constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB ...
 constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list is at most this many runs
+constexpr int64_t PATCH_DMA_MAX_RUNS = 16;               // table entries by small copies up to this many runs of ids, else a kernel
 
 #define PIE_CUDA(call)                                  \
     do {                                                \
@@ -32,15 +33,17 @@ constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list
     } while (0)
 
 struct LayerEvents {
-    // compute stream: before the presence wait, after it, after the layer; copy streams: start and end of a list.
-    // Every record costs the stream about a microsecond between two kernels, so a layer records only what it needs:
-    // `pre` for the first layer of a step, `go` when there is a wait to measure.
-    // pre, go, in0, out0 are owned; done, in1, out1 point at the ticket events of the calls (valid for EV_RING tickets)
-    cudaEvent_t pre = nullptr, go = nullptr, done = nullptr;
-    cudaEvent_t start = nullptr;  // where the layer's time starts: the previous layer's `done` within a step, else `pre`
+    // Copy streams: timing events at the start of a list (in0, out0, owned) and its ticket's event at the end (in1,
+    // out1: valid for EV_RING tickets).  The compute stream carries no timing events at all - a record there costs
+    // 2-3 us between two kernels; the attention kernel notes the GPU timer itself (stamps, below).  For the per-layer
+    // timeline (timing = 2) one timing event per step on the compute stream, recorded right before the step's first
+    // attention kernel, ties the copy streams' events to the stamps (to within the few us between that record and
+    // the kernel's start).
     cudaEvent_t in0 = nullptr, in1 = nullptr, out0 = nullptr, out1 = nullptr;
-    bool has_in = false, has_out = false, has_compute = false, waited = false;
+    bool has_in = false, has_out = false, has_compute = false;
 };
+// per layer of a step: GPU-timer stamps in mapped pinned memory
+enum { STAMP_START = 0, STAMP_END = 1, STAMP_WORDS = 2 };
 
 struct ListRecord {
     int64_t start, end;
@@ -59,6 +62,12 @@ struct pie_pool {
     bool own_gpu = false, own_host = false, own_streams = false;
     cudaStream_t stream[4] = {nullptr, nullptr, nullptr, nullptr};  // indexed by queue id
     cudaEvent_t ticket_ev[4][EV_RING] = {};
+    // Compute tickets have two sets of events; ticket_ev[PIE_Q_COMPUTE][i] points at the one its newest record used.
+    // A record without a time stamp is ~2.5 us cheaper between two kernels, but when another stream waits on such an
+    // event the recording stream loses ~5 us instead (measured on this part and driver): so plain events while
+    // nothing is being swapped, time-stamped ones while swap lists, which wait on compute tickets, are in flight.
+    cudaEvent_t compute_ev_plain[EV_RING] = {}, compute_ev_stamped[EV_RING] = {};
+    int64_t last_swap_step = -2;   // the step in which the newest swap list was issued
     int64_t recorded[4] = {0, 0, 0, 0};  // newest ticket of each queue whose event has been recorded
     int32_t *slot_table_dev = nullptr;  // [L][NB]
     // id lists: pinned ring + device mirror at the same offsets
@@ -69,6 +78,10 @@ struct pie_pool {
     int list_ev_next = 0;
     // device status word (mapped pinned memory)
     int32_t *status_host = nullptr, *status_dev = nullptr;
+    uint64_t *stamps_host = nullptr, *stamps_dev = nullptr;  // [TIMING_RING][n_layers][STAMP_WORDS]
+    uint64_t prev_step_end = 0;   // GPU-timer stamp of the end of the last layer of the newest evaluated step
+    int64_t prev_step_id = -1;
+    bool prev_step_prefetched0 = false;  // that step issued a prefetch of layer 0 for the step after it
     // attention
     pie::AttnScratch scratch{};
     CUtensorMap map3d{}, map2d{};
@@ -82,8 +95,6 @@ struct pie_pool {
     double ratio = 0.0;
     double ctrl_state[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
-    cudaEvent_t last_compute_ev = nullptr;  // the newest attention call's ticket event and the step it belongs to
-    int64_t last_compute_step = -1;
     bool poll_hold = false;  // a decode step is polling once per layer: nested calls skip theirs
     std::vector<int64_t> home_count;  // per layer: units whose home is the host
     std::vector<std::vector<int32_t>> home_list;  // per layer: ids the planner looks at (see candidate_ids)
@@ -97,6 +108,8 @@ struct pie_pool {
     std::vector<LayerEvents> lev[TIMING_RING];
     int64_t lev_step[TIMING_RING] = {};      // which step a set holds (0 = none)
     bool lev_done[TIMING_RING] = {};         // already evaluated
+    cudaEvent_t lev_anchor[TIMING_RING] = {};   // timing = 2: recorded on the compute stream before the step's first attention kernel
+    bool lev_anchored[TIMING_RING] = {};
     cudaEvent_t lev_last[TIMING_RING][4] = {};  // the set's newest event on each queue's stream (its streams complete in order)
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
@@ -104,6 +117,9 @@ struct pie_pool {
     pie_stats stats{};
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
+    std::vector<uint8_t> v_elide;
+    std::vector<int32_t> append_ids;  // blocks the coming appends write (pie_declare_append_blocks)
+    bool append_declared = false;
     int sticky = PIE_OK;
 };
 
@@ -149,6 +165,8 @@ int reserve_ticket_event(pie_pool *p, int q, int64_t t) {
 }
 
 int record_ticket(pie_pool *p, int q, int64_t t) {
+    if (q == PIE_Q_COMPUTE)
+        p->ticket_ev[q][t % EV_RING] = p->last_swap_step >= p->step - 1 ? p->compute_ev_stamped[t % EV_RING] : p->compute_ev_plain[t % EV_RING];
     PIE_CUDA(cudaEventRecord(p->ticket_ev[q][t % EV_RING], p->stream[q]));
     p->recorded[q] = t;
     return PIE_OK;
@@ -220,13 +238,26 @@ LayerEvents *timing_slot(pie_pool *p, int32_t layer) {
     return &p->lev[p->step % TIMING_RING][(size_t)layer];
 }
 
+// device-visible address of one stamp of the current step's set (nullptr with timing off)
+uint64_t *stamp_dev(pie_pool *p, int32_t layer, int which) {
+    if (!p->cfg.timing) return nullptr;
+    return p->stamps_dev + ((size_t)(p->step % TIMING_RING) * (size_t)p->cfg.n_layers + (size_t)layer) * STAMP_WORDS + which;
+}
+
 // ---- one swap call ------------------------------------------------------------------------------------
+// elide (optional): pairs flagged 1 move no bytes (a kept, unwritten host copy); they still get their table entry
+// patched, and they force the copy-engine path: the gather/scatter kernel takes the whole list.
 int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst, int64_t n, const int32_t *blocks,
-              int32_t *slot_table_row, int mode, cudaStream_t stream, int64_t ticket = 0) {
+              int32_t *slot_table_row, int mode, cudaStream_t stream, int64_t ticket = 0, const uint8_t *elide = nullptr) {
     // dir_queue PIE_Q_IN: host -> GPU; PIE_Q_OUT: GPU -> host
     const uint8_t *src_pool = dir_queue == PIE_Q_IN ? p->host_base : p->gpu_base;
     uint8_t *dst_pool = dir_queue == PIE_Q_IN ? p->gpu_base : p->host_base;
     const int64_t BB = p->block_bytes;
+    bool any_elided = false;
+    if (elide)
+        for (int64_t i = 0; i < n && !any_elided; ++i) any_elided = elide[i] != 0;
+    if (!any_elided) elide = nullptr;
+    if (elide) mode = PIE_MODE_COPY_ENGINE;
     if (mode == PIE_MODE_AUTO) {
         int64_t runs = 1;
         for (int64_t i = 1; i < n; ++i)
@@ -236,10 +267,28 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         mode = ((n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS) ? PIE_MODE_COPY_ENGINE
                                                                                                    : PIE_MODE_KERNEL;
     }
+    // Table entries after copy-engine copies.  The persistent attention kernel leaves no room for another CTA on any
+    // SM, so a patch kernel on a copy stream only gets to run in the gap between two attention launches - and the next
+    // layer, which waits for that swap's ticket, starts late by as much.  When the moved ids form a few runs of
+    // consecutive blocks (the usual case: lists are in ascending id), the new entries are written to the pinned list
+    // ring instead and one small host-to-device copy per run puts them into the layer's row: no SM is involved.
+    bool dma_patch = false;
+    if (mode == PIE_MODE_COPY_ENGINE && slot_table_row != nullptr && blocks != nullptr) {
+        int64_t id_runs = 1;
+        for (int64_t i = 1; i < n && id_runs <= PATCH_DMA_MAX_RUNS; ++i)
+            if (blocks[i] != blocks[i - 1] + 1) ++id_runs;
+        dma_patch = id_runs <= PATCH_DMA_MAX_RUNS;
+    }
     const bool need_list = mode == PIE_MODE_KERNEL || slot_table_row != nullptr;
+    const int64_t list_len = dma_patch ? n : 3 * n;
     int64_t off = 0;
-    if (need_list) {
-        int st = list_alloc(p, 3 * n, &off);
+    if (need_list && dma_patch) {
+        int st = list_alloc(p, list_len, &off);
+        if (st != PIE_OK) return st;
+        int32_t *h = p->list_host + off;
+        for (int64_t i = 0; i < n; ++i) h[i] = dir_queue == PIE_Q_IN ? dst[i] : -1;
+    } else if (need_list) {
+        int st = list_alloc(p, list_len, &off);
         if (st != PIE_OK) return st;
         int32_t *h = p->list_host + off;
         for (int64_t i = 0; i < n; ++i) {
@@ -262,20 +311,34 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         const cudaMemcpyKind kind = dir_queue == PIE_Q_IN ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
         int64_t i = 0;
         while (i < n) {
+            if (elide && elide[i]) {
+                ++i;
+                continue;
+            }
             int64_t j = i + 1;
-            while (j < n && src[j] == src[j - 1] + 1 && dst[j] == dst[j - 1] + 1) ++j;
+            while (j < n && !(elide && elide[j]) && src[j] == src[j - 1] + 1 && dst[j] == dst[j - 1] + 1) ++j;
             PIE_CUDA(cudaMemcpyAsync(dst_pool + (int64_t)dst[i] * BB, src_pool + (int64_t)src[i] * BB, (size_t)((j - i) * BB),
                                      kind, stream));
             i = j;
         }
-        if (slot_table_row) PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_host + off, n, table_mode, stream));
+        if (dma_patch) {
+            const int32_t *h = p->list_host + off;
+            for (int64_t a = 0; a < n;) {
+                int64_t b = a + 1;
+                while (b < n && blocks[b] == blocks[b - 1] + 1) ++b;
+                PIE_CUDA(cudaMemcpyAsync(slot_table_row + blocks[a], h + a, (size_t)(b - a) * 4, cudaMemcpyHostToDevice, stream));
+                a = b;
+            }
+        } else if (slot_table_row) {
+            PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_host + off, n, table_mode, stream));
+        }
         p->stats.calls_copy_engine += 1;
     }
     if (need_list) {
         if (ticket > 0) {
-            list_commit_ticket(p, off, 3 * n, dir_queue, ticket);
+            list_commit_ticket(p, off, list_len, dir_queue, ticket);
         } else {
-            int st = list_commit(p, off, 3 * n, stream);
+            int st = list_commit(p, off, list_len, stream);
             if (st != PIE_OK) return st;
         }
     }
@@ -297,10 +360,15 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
         p->v_moved.resize((size_t)n);
         p->v_src.resize((size_t)n);
         p->v_dst.resize((size_t)n);
+        p->v_elide.resize((size_t)n);
     }
+    p->last_swap_step = p->step;
     int64_t ticket = 0, n_moved = 0, waits[4];
-    st = p->table->swap(queue, layer, ids, n, &ticket, p->v_moved.data(), p->v_src.data(), p->v_dst.data(), &n_moved, waits);
+    st = p->table->swap(queue, layer, ids, n, &ticket, p->v_moved.data(), p->v_src.data(), p->v_dst.data(), &n_moved, waits,
+                        p->v_elide.data());
     if (st != PIE_OK || n_moved == 0) return st;
+    int64_t n_elided = 0;
+    for (int64_t i = 0; i < n_moved; ++i) n_elided += p->v_elide[(size_t)i];
     // a unit that is pushed out belongs to the host-resident set from now on; bringing it in for a layer's
     // turn does not take it out of the set (only a lower ratio does)
     if (queue == PIE_Q_OUT)
@@ -324,7 +392,7 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
     LayerEvents *le = timing_slot(p, layer);
     if (le && cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream) != cudaSuccess) le = nullptr;
     st = do_copies(p, queue, p->v_src.data(), p->v_dst.data(), n_moved, p->v_moved.data(),
-                   p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream, ticket);
+                   p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream, ticket, p->v_elide.data());
     if (st != PIE_OK) { p->sticky = st; return st; }
     st = record_ticket(p, queue, ticket);
     if (st != PIE_OK) { p->sticky = st; return st; }
@@ -333,7 +401,8 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
         (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
         p->lev_last[p->step % TIMING_RING][queue] = p->ticket_ev[queue][ticket % EV_RING];
     }
-    (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)n_moved * (double)p->block_bytes;
+    (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)(n_moved - n_elided) * (double)p->block_bytes;
+    p->stats.reserved[2] += (double)n_elided * (double)p->block_bytes;
     return PIE_OK;
 }
 
@@ -377,15 +446,21 @@ int patch_units(pie_pool *p, const std::vector<int32_t> &entries) {
 
 void destroy_pool(pie_pool *p) {
     if (!p) return;
-    for (int q = 1; q <= 3; ++q)
+    for (int q = 1; q <= 2; ++q)
         for (int i = 0; i < EV_RING; ++i)
             if (p->ticket_ev[q][i]) cudaEventDestroy(p->ticket_ev[q][i]);
+    for (int i = 0; i < EV_RING; ++i) {
+        if (p->compute_ev_plain[i]) cudaEventDestroy(p->compute_ev_plain[i]);
+        if (p->compute_ev_stamped[i]) cudaEventDestroy(p->compute_ev_stamped[i]);
+    }
     for (int i = 0; i < LIST_EVENTS; ++i)
         if (p->list_events[i]) cudaEventDestroy(p->list_events[i]);
     for (int k = 0; k < TIMING_RING; ++k)
         for (LayerEvents &e : p->lev[k])
-            for (cudaEvent_t ev : {e.pre, e.go, e.in0, e.out0})
+            for (cudaEvent_t ev : {e.in0, e.out0})
                 if (ev) cudaEventDestroy(ev);
+    for (int k = 0; k < TIMING_RING; ++k)
+        if (p->lev_anchor[k]) cudaEventDestroy(p->lev_anchor[k]);
     if (p->own_streams)
         for (int q = 1; q <= 3; ++q)
             if (p->stream[q]) cudaStreamDestroy(p->stream[q]);
@@ -395,6 +470,7 @@ void destroy_pool(pie_pool *p) {
     cudaFree(p->list_dev);
     if (p->list_host) cudaFreeHost(p->list_host);
     if (p->status_host) cudaFreeHost(p->status_host);
+    if (p->stamps_host) cudaFreeHost(p->stamps_host);
     cudaFree(p->scratch.chunk_off);
     cudaFree(p->scratch.counters);
     cudaFree(p->scratch.part_o);
@@ -443,24 +519,29 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         st = p->table->attention(layer, nullptr, 0, &ticket, waits);
     }
     if (st != PIE_OK) return st;
+    if (k_new && p->table->retain()) {
+        // kept host copies of the blocks this call's append writes go stale
+        const int32_t NB = p->cfg.n_logical_blocks;
+        auto mark = [&](int32_t b) {
+            if (b >= 0 && b < NB && p->table->allocated(b)) p->table->unit(layer, b).dirty = 1;
+        };
+        if (bt_host) {
+            for (int32_t s = 0; s < n_seqs; ++s)
+                if (ctx_host[s] > 0) mark(bt_host[(int64_t)s * max_blocks + (ctx_host[s] - 1) / 16]);
+        } else if (p->append_declared) {
+            for (int32_t b : p->append_ids) mark(b);
+        } else {
+            p->table->mark_layer_dirty(layer);
+        }
+    }
     cudaStream_t stream = p->stream[PIE_Q_COMPUTE];
     st = reserve_ticket_event(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) { p->sticky = st; return st; }
     LayerEvents *le = timing_slot(p, layer);
-    if (le) {
-        le->waited = waits[1] > p->table->done(1) || waits[2] > p->table->done(2);
-        if (p->last_compute_ev && p->last_compute_step == p->step) {
-            le->start = p->last_compute_ev;
-        } else {
-            le->start = le->pre;
-            if (cudaEventRecord(le->pre, stream) != cudaSuccess) le = nullptr;  // timing is best effort
-        }
-    }
     for (int qd = 1; qd <= 2; ++qd) {
         st = wait_ticket(p, stream, qd, waits[qd]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
-    if (le && le->waited && cudaEventRecord(le->go, stream) != cudaSuccess) le = nullptr;
     pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
                       p->cfg.n_gpu_slots};
     pie::AttnLaunch a{};
@@ -479,6 +560,11 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.grid = p->attn_grid;
     a.variant = p->cfg.reserved[0];
     a.status = p->status_dev;
+    a.stamps = le ? stamp_dev(p, layer, STAMP_START) : nullptr;
+    if (le && p->cfg.timing >= 2 && !p->lev_anchored[p->step % TIMING_RING]) {
+        const int k = (int)(p->step % TIMING_RING);
+        if (cudaEventRecord(p->lev_anchor[k], stream) == cudaSuccess) p->lev_anchored[k] = true;
+    }
     cudaError_t e = pie::launch_attention(sh, p->scratch, a, p->use3d ? p->map3d : p->map2d, p->use3d, stream);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
@@ -488,11 +574,8 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     st = record_ticket(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) p->sticky = st;
     if (le && st == PIE_OK) {
-        le->done = p->ticket_ev[PIE_Q_COMPUTE][ticket % EV_RING];
         le->has_compute = true;
-        p->lev_last[p->step % TIMING_RING][PIE_Q_COMPUTE] = le->done;
-        p->last_compute_ev = le->done;
-        p->last_compute_step = p->step;
+        p->lev_last[p->step % TIMING_RING][PIE_Q_COMPUTE] = p->ticket_ev[PIE_Q_COMPUTE][ticket % EV_RING];
     }
     return st;
 }
@@ -530,7 +613,11 @@ void apply_ratio_to_layer(pie_pool *p, int32_t layer) {
         for (int32_t b = NB - 1; b >= 0 && count > target; --b) {
             if (!p->table->allocated(b)) continue;
             pie::Unit &u = p->table->unit(layer, b);
-            if (u.home_host) { u.home_host = 0; --count; }
+            if (u.home_host) {
+                u.home_host = 0;
+                --count;
+                p->table->drop_host_copy(layer, b);  // a kept host slot is only for members of the set
+            }
         }
     }
 }
@@ -576,6 +663,7 @@ int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::ve
             }
         } else if (!u.home_host) {
             p->home_dirty[(size_t)next] = 1;  // left the set and is back on the GPU: drop it at the next rebuild
+            p->table->drop_host_copy(next, b);
         }
     }
     // coldest: this layer's host-home units go back once it has computed
@@ -717,17 +805,28 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
         p->stream[PIE_Q_IN] = (cudaStream_t)cfg->copy_in_stream;
         p->stream[PIE_Q_OUT] = (cudaStream_t)cfg->copy_out_stream;
     }
-    for (int q = 1; q <= 3; ++q)
-        for (int i = 0; i < EV_RING; ++i)  // with timing on, a ticket's event doubles as the "end" mark of its work
+    for (int q = 1; q <= 2; ++q)
+        for (int i = 0; i < EV_RING; ++i)  // with timing on, a copy ticket's event doubles as the "end" mark of its list
             PIE_TRY(cudaEventCreateWithFlags(&p->ticket_ev[q][i], cfg->timing ? cudaEventDefault : cudaEventDisableTiming), PIE_ERR_CUDA);
+    for (int i = 0; i < EV_RING; ++i) {
+        PIE_TRY(cudaEventCreateWithFlags(&p->compute_ev_plain[i], cudaEventDisableTiming), PIE_ERR_CUDA);
+        PIE_TRY(cudaEventCreateWithFlags(&p->compute_ev_stamped[i], cudaEventDefault), PIE_ERR_CUDA);
+        p->ticket_ev[PIE_Q_COMPUTE][i] = p->compute_ev_plain[i];
+    }
     for (int i = 0; i < LIST_EVENTS; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->list_events[i], cudaEventDisableTiming), PIE_ERR_CUDA);
     if (cfg->timing) {
         for (int k = 0; k < TIMING_RING; ++k) {
             p->lev[k].resize((size_t)cfg->n_layers);
             for (LayerEvents &e : p->lev[k])
-                for (cudaEvent_t *ev : {&e.pre, &e.go, &e.in0, &e.out0})
+                for (cudaEvent_t *ev : {&e.in0, &e.out0})
                     PIE_TRY(cudaEventCreate(ev), PIE_ERR_CUDA);
         }
+        if (cfg->timing >= 2)
+            for (int k = 0; k < TIMING_RING; ++k) PIE_TRY(cudaEventCreate(&p->lev_anchor[k]), PIE_ERR_CUDA);
+        const size_t stamp_bytes = (size_t)TIMING_RING * (size_t)cfg->n_layers * STAMP_WORDS * 8;
+        PIE_TRY(cudaHostAlloc((void **)&p->stamps_host, stamp_bytes, cudaHostAllocMapped), PIE_ERR_NOMEM);
+        std::memset(p->stamps_host, 0, stamp_bytes);
+        PIE_TRY(cudaHostGetDevicePointer((void **)&p->stamps_dev, p->stamps_host, 0), PIE_ERR_CUDA);
     }
     const size_t table_bytes = (size_t)cfg->n_layers * (size_t)cfg->n_logical_blocks * 4;
     PIE_TRY(cudaMalloc((void **)&p->slot_table_dev, table_bytes), PIE_ERR_NOMEM);
@@ -942,60 +1041,102 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         else if (cudaEventQuery(evt) != cudaSuccess) return 1;  // not complete yet
     }
     double compute = 0, stall = 0, t_in = 0, t_out = 0;
-    cudaEvent_t first = nullptr, last = nullptr;
     bool any_swap = false;
-    for (LayerEvents &e : ev) {
+    const size_t L = ev.size();
+    const volatile uint64_t *stamps = pool->stamps_host + (size_t)k * L * STAMP_WORDS;
+    std::vector<float> dur_in(L, -1.f), dur_out(L, -1.f);
+    for (size_t l = 0; l < L; ++l) {
+        LayerEvents &e = ev[l];
         float ms = 0;
-        if (e.has_compute) {
-            // the layer's time runs from the end of the previous layer; what the stream spent in the presence wait
-            // is the stall (two back-to-back stream operations are already ~2-3 us apart: only the excess counts),
-            // the rest - launch gap included, with or without swaps - is compute
-            PIE_CUDA(cudaEventElapsedTime(&ms, e.start, e.done));
-            double layer_stall = 0.0;
-            if (e.waited) {
-                float w = 0;
-                PIE_CUDA(cudaEventElapsedTime(&w, e.start, e.go));
-                layer_stall = std::max(0.0, (double)w - 0.004);
-            }
-            stall += layer_stall;
-            compute += std::max(0.0, (double)ms - layer_stall);
-            if (!first) first = e.start;
-            last = e.done;
-        }
         if (e.has_in) {
             PIE_CUDA(cudaEventElapsedTime(&ms, e.in0, e.in1));
             t_in += ms;
+            dur_in[l] = ms;
             any_swap = true;
         }
         if (e.has_out) {
             PIE_CUDA(cudaEventElapsedTime(&ms, e.out0, e.out1));
             t_out += ms;
+            dur_out[l] = ms;
             any_swap = true;
         }
     }
+    // Compute stream, from the GPU-timer stamps.  A layer's time runs from the end of the previous layer's attention
+    // kernel to the end of its own (combine and launch gap included, with or without swaps).  What the gap before a
+    // layer that had units brought in exceeds the usual gap by is the stall: the stream sat in the presence wait.  The
+    // usual gap is the smallest one of the step, but no more than 20 us, so that a step in which every layer waits
+    // still shows it.
+    const bool chained = pool->prev_step_id == pool->lev_step[k] - 1 && pool->prev_step_end != 0;
+    uint64_t prev_end = chained ? pool->prev_step_end : 0, first = 0, last = 0;
+    uint64_t usual_gap = 20000;
+    double first_stall = 0.0;
+    {
+        uint64_t pe = 0;
+        for (size_t l = 0; l < L; ++l) {
+            const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
+            if (!ev[l].has_compute || !S || !E) continue;
+            if (pe && S > pe) usual_gap = std::min(usual_gap, S - pe);
+            pe = E;
+        }
+    }
+    for (size_t l = 0; l < L; ++l) {
+        const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
+        if (!ev[l].has_compute || !S || !E || E < S) continue;
+        // units were brought in for this layer: by a list of this step for layers >= 1, by the previous step's
+        // look-ahead across the token boundary for layer 0
+        const bool fetched = l > 0 ? ev[l].has_in : (chained && pool->prev_step_prefetched0);
+        double layer_stall = 0.0;
+        if (fetched && prev_end && S > prev_end + usual_gap) layer_stall = (double)(S - prev_end - usual_gap) * 1e-6;
+        stall += layer_stall;
+        if (!first) {
+            // the step's first layer: its time starts with its own kernel (whatever the caller did between two steps
+            // is not the layer's); a wait before it still counts as stall, and as part of the step
+            first = S;
+            first_stall = layer_stall;
+            compute += (double)(E - S) * 1e-6;
+        } else {
+            compute += std::max(0.0, (double)(E - prev_end) * 1e-6 - layer_stall);
+        }
+        prev_end = last = E;
+    }
+    if (last) {
+        pool->prev_step_end = last;
+        pool->prev_step_id = pool->lev_step[k];
+        pool->prev_step_prefetched0 = L > 1 && ev[0].has_in;
+    }
     pool->lev_done[k] = true;
     if (first && pool->cfg.timing >= 2) {
-        pool->timeline.assign(ev.size() * 7, -1.f);
-        for (size_t l = 0; l < ev.size(); ++l) {
-            LayerEvents &e = ev[l];
-            cudaEvent_t list[7] = {e.start, e.waited ? e.go : e.start, e.done, e.in0, e.in1, e.out0, e.out1};
-            const bool has[7] = {e.has_compute, e.has_compute, e.has_compute, e.has_in, e.has_in, e.has_out, e.has_out};
-            for (int j = 0; j < 7; ++j)
-                if (has[j]) {
-                    float ms = 0;
-                    if (cudaEventElapsedTime(&ms, first, list[j]) == cudaSuccess) pool->timeline[l * 7 + j] = ms;
-                }
+        // compute columns from the stamps, relative to the first kernel's start; copy columns from the copy streams'
+        // events relative to the step's anchor event, which was recorded just before that kernel
+        pool->timeline.assign(L * 7, -1.f);
+        auto rel = [&](uint64_t t) { return (float)(((double)t - (double)first) * 1e-6); };
+        uint64_t before = first;
+        for (size_t l = 0; l < L; ++l) {
+            const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
+            float *row = pool->timeline.data() + l * 7;
+            if (ev[l].has_compute && S && E) {
+                row[0] = rel(before);
+                row[1] = rel(S);
+                row[2] = rel(E);
+                before = E;
+            }
+            if (!pool->lev_anchored[k]) continue;
+            float ms = 0;
+            if (ev[l].has_in && cudaEventElapsedTime(&ms, pool->lev_anchor[k], ev[l].in0) == cudaSuccess) {
+                row[3] = ms;
+                row[4] = ms + dur_in[l];
+            }
+            if (ev[l].has_out && cudaEventElapsedTime(&ms, pool->lev_anchor[k], ev[l].out0) == cudaSuccess) {
+                row[5] = ms;
+                row[6] = ms + dur_out[l];
+            }
         }
     }
     pool->stats.last_step_compute_ms = compute;
     pool->stats.last_step_stall_ms = stall;
     pool->stats.last_step_swap_in_ms = t_in;
     pool->stats.last_step_swap_out_ms = t_out;
-    if (first && last) {
-        float ms = 0;
-        PIE_CUDA(cudaEventElapsedTime(&ms, first, last));
-        pool->stats.last_step_ms = ms;
-    }
+    if (first && last) pool->stats.last_step_ms = (double)(last - first) * 1e-6 + first_stall;
     pool->stats.steps_measured += 1;
     // Performance record (Section 3.4.2): attention time per context token on steps without swap traffic.  Copies
     // that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
@@ -1049,8 +1190,12 @@ int pie_step_begin(pie_pool *pool) {
         }
         pool->lev_step[k] = pool->step;
         pool->lev_done[k] = false;
-        for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = e.waited = false;
+        for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = false;
         for (int q = 0; q < 4; ++q) pool->lev_last[k][q] = nullptr;
+        pool->lev_anchored[k] = false;
+        // the set's kernels are launched after this point, and the previous user of the set has completed
+        std::memset(pool->stamps_host + (size_t)k * (size_t)pool->cfg.n_layers * STAMP_WORDS, 0,
+                    (size_t)pool->cfg.n_layers * STAMP_WORDS * 8);
     }
     return PIE_OK;
 }
@@ -1092,6 +1237,26 @@ int pie_get_extension_ratio(pie_pool *pool, float *r) {
     } else {
         *r = (float)pool->ratio;
     }
+    return PIE_OK;
+}
+
+int pie_set_retention(pie_pool *pool, int32_t on) {
+    if (!pool) return PIE_ERR_INVALID;
+    pool->table->set_retain(on != 0);
+    return PIE_OK;
+}
+
+int pie_declare_append_blocks(pie_pool *pool, const int32_t *ids, int64_t n) {
+    if (!pool || (n > 0 && !ids)) return PIE_ERR_INVALID;
+    if (n < 0) {
+        pool->append_declared = false;
+        pool->append_ids.clear();
+        return PIE_OK;
+    }
+    for (int64_t i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= pool->cfg.n_logical_blocks) return PIE_ERR_RANGE;
+    pool->append_ids.assign(ids, ids + n);
+    pool->append_declared = true;
     return PIE_OK;
 }
 
@@ -1370,8 +1535,22 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
     }
     PIE_CUDA(cudaMemcpyAsync(pool->stage_bt, block_table_host, (size_t)n_seqs * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, s));
     PIE_CUDA(cudaMemcpyAsync(pool->stage_ctx, ctx_lens_host, (size_t)n_seqs * 4, cudaMemcpyHostToDevice, s));
+    // the host tables say which block of each sequence the append writes: kept host copies of the others stay good
+    std::vector<int32_t> saved_ids;
+    const bool saved_declared = pool->append_declared;
+    if (k_new_all_host && pool->table->retain()) {
+        saved_ids.swap(pool->append_ids);
+        for (int32_t sq = 0; sq < n_seqs; ++sq)
+            if (ctx_lens_host[sq] > 0 && ctx_lens_host[sq] <= max_blocks_per_seq * 16)
+                pool->append_ids.push_back(block_table_host[(int64_t)sq * max_blocks_per_seq + (ctx_lens_host[sq] - 1) / 16]);
+        pool->append_declared = true;
+    }
     st = pie_decode_step(pool, pool->stage_q, pool->stage_out, pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
                          k_new_all_host ? pool->stage_k : nullptr, k_new_all_host ? pool->stage_v : nullptr, mode);
+    if (k_new_all_host && pool->table->retain()) {
+        pool->append_ids.swap(saved_ids);
+        pool->append_declared = saved_declared;
+    }
     if (st != PIE_OK) return st;
     PIE_CUDA(cudaMemcpyAsync(out_all_host, pool->stage_out, (size_t)qb, cudaMemcpyDeviceToHost, s));
     PIE_CUDA(cudaStreamSynchronize(s));

@@ -173,6 +173,7 @@ int Table::free_block(int32_t block) {
             // an attention call issued earlier may still be reading the slot
             int64_t ct = issued_[PIE_Q_COMPUTE];
             gpu_.release(u.gpu_slot, ct > done_[PIE_Q_COMPUTE] ? PIE_Q_COMPUTE : PIE_Q_NONE, ct);
+            if (u.host_slot >= 0) host_.release(u.host_slot, PIE_Q_NONE, 0);  // a kept host copy goes with the unit
         } else {
             host_.release(u.host_slot, PIE_Q_NONE, 0);
         }
@@ -199,19 +200,50 @@ int Table::check_ids(int32_t layer, const int32_t *ids, int64_t n) {
     return PIE_OK;
 }
 
+int Table::drop_host_copy(int32_t layer, int32_t block) {
+    if (layer < 0 || layer >= L || block < 0 || block >= NB) return PIE_ERR_RANGE;
+    if (!allocated_[block]) return PIE_ERR_INVALID;
+    settle();
+    Unit &u = unit(layer, block);
+    if (u.side == PIE_GPU && u.host_slot >= 0) {
+        // the copy that is bringing the unit in may still be reading the slot: its next owner waits for that copy
+        if (in_flight(u)) host_.release(u.host_slot, u.last_q, u.last_t);
+        else host_.release(u.host_slot, PIE_Q_NONE, 0);
+        u.host_slot = -1;
+    }
+    return PIE_OK;
+}
+
+int Table::mark_dirty(int32_t layer, const int32_t *ids, int64_t n) {
+    int st = check_ids(layer, ids, n);
+    if (st != PIE_OK) return st;
+    for (int64_t i = 0; i < n; ++i) unit(layer, ids[i]).dirty = 1;
+    return PIE_OK;
+}
+
+void Table::mark_layer_dirty(int32_t layer) {
+    for (int32_t b = 0; b < NB; ++b)
+        if (allocated_[b]) unit(layer, b).dirty = 1;
+}
+
 int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int32_t *moved,
-                int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits) {
+                int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits, uint8_t *elide) {
     if (queue != PIE_Q_IN && queue != PIE_Q_OUT) return PIE_ERR_INVALID;
     int st = check_ids(layer, ids, n);
     if (st != PIE_OK) return st;
     settle();
     const uint8_t want = queue == PIE_Q_OUT ? PIE_HOST : PIE_GPU;
-    int64_t movers = 0;
-    for (int64_t i = 0; i < n; ++i)
-        if (unit(layer, ids[i]).side != want) ++movers;
+    // a unit that kept its host slot goes back into it: only the others need a new one
+    int64_t movers = 0, need = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        const Unit &u = unit(layer, ids[i]);
+        if (u.side == want) continue;
+        ++movers;
+        if (queue == PIE_Q_IN || u.host_slot < 0) ++need;
+    }
     SlotPool &dst_pool = queue == PIE_Q_OUT ? host_ : gpu_;
     SlotPool &src_pool = queue == PIE_Q_OUT ? gpu_ : host_;
-    if (movers > dst_pool.available()) return PIE_ERR_NOMEM;
+    if (need > dst_pool.available()) return PIE_ERR_NOMEM;
     layer_pass(layer);
     waits[0] = waits[1] = waits[2] = waits[3] = 0;
     *n_moved = 0;
@@ -223,22 +255,34 @@ int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int
     for (int64_t i = 0; i < n; ++i) {
         Unit &u = unit(layer, ids[i]);
         if (u.side == want) continue;
-        SlotTag tag;
-        int32_t d = dst_pool.take(&tag);
-        if (tag.queue != PIE_Q_NONE) waits[tag.queue] = std::max(waits[tag.queue], tag.ticket);
+        const bool kept = queue == PIE_Q_OUT && u.host_slot >= 0;
+        int32_t d = u.host_slot;
+        if (!kept) {
+            SlotTag tag;
+            d = dst_pool.take(&tag);
+            if (tag.queue != PIE_Q_NONE) waits[tag.queue] = std::max(waits[tag.queue], tag.ticket);
+        }
         // the copy that is still bringing the unit to where it is now
         if (in_flight(u)) waits[u.last_q] = std::max(waits[u.last_q], u.last_t);
         int32_t s;
+        bool skip = false;
         if (queue == PIE_Q_OUT) {
             s = u.gpu_slot;
+            skip = kept && !u.dirty;  // the kept copy is still good unless the unit was written
             u.host_slot = d;
             u.gpu_slot = -1;
+            u.dirty = 0;
+            src_pool.release(s, queue, tk);
         } else {
             s = u.host_slot;
             u.gpu_slot = d;
-            u.host_slot = -1;
+            if (!retain_) {
+                u.host_slot = -1;
+                src_pool.release(s, queue, tk);
+            }
+            // with retain_ the host slot stays the unit's, and a dirty mark made before the unit came in survives
         }
-        src_pool.release(s, queue, tk);
+        if (elide) elide[k] = skip ? 1 : 0;
         u.side = want;
         u.last_q = (uint8_t)queue;
         u.last_t = tk;
@@ -390,6 +434,24 @@ int pie_table_swap(pie_table *t, int32_t queue, int32_t layer, const int32_t *id
     if (!t || !ticket || !moved_ids || !src_slots || !dst_slots || !n_moved || !waits) return PIE_ERR_INVALID;
     return reinterpret_cast<Table *>(t)->swap(queue, layer, ids, n, ticket, moved_ids, src_slots, dst_slots, n_moved,
                                               waits);
+}
+int pie_table_swap_ex(pie_table *t, int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket,
+                      int32_t *moved_ids, int32_t *src_slots, int32_t *dst_slots, uint8_t *elided, int64_t *n_moved,
+                      int64_t *waits) {
+    if (!t || !ticket || !moved_ids || !src_slots || !dst_slots || !elided || !n_moved || !waits) return PIE_ERR_INVALID;
+    return reinterpret_cast<Table *>(t)->swap(queue, layer, ids, n, ticket, moved_ids, src_slots, dst_slots, n_moved,
+                                              waits, elided);
+}
+int pie_table_set_retention(pie_table *t, int32_t on) {
+    if (!t) return PIE_ERR_INVALID;
+    reinterpret_cast<Table *>(t)->set_retain(on != 0);
+    return PIE_OK;
+}
+int pie_table_drop_host_copy(pie_table *t, int32_t layer, int32_t block) {
+    return t ? reinterpret_cast<Table *>(t)->drop_host_copy(layer, block) : PIE_ERR_INVALID;
+}
+int pie_table_mark_dirty(pie_table *t, int32_t layer, const int32_t *ids, int64_t n) {
+    return t ? reinterpret_cast<Table *>(t)->mark_dirty(layer, ids, n) : PIE_ERR_INVALID;
 }
 int pie_table_attention(pie_table *t, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits) {
     if (!t || !ticket || !waits) return PIE_ERR_INVALID;

@@ -41,6 +41,7 @@ struct Unit {
     uint8_t side = PIE_FREE;  // PIE_FREE / PIE_GPU / PIE_HOST: where the unit is or is heading
     uint8_t last_q = PIE_Q_NONE;
     uint8_t home_host = 0;  // belongs to the host-resident set between uses
+    uint8_t dirty = 0;      // written on the GPU since its host copy was taken (matters while a host slot is kept)
     int32_t gpu_slot = -1;
     int32_t host_slot = -1;
     int64_t last_t = 0;
@@ -55,8 +56,16 @@ class Table {
     // n blocks at once, slots handed out layer by layer so that each layer's units sit in consecutive slots
     int alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host);
     int free_block(int32_t block);
+    // elide (optional, capacity n): 1 where the pair needs no bytes moved (a kept, unwritten host copy)
     int swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int32_t *moved,
-             int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits);
+             int32_t *src, int32_t *dst, int64_t *n_moved, int64_t *waits, uint8_t *elide = nullptr);
+    // Variant beyond the paper (Section 3.2 gives the CPU region up after a swap-in): a unit that comes in keeps
+    // its host slot, and going out again copies nothing unless it was marked written meanwhile.
+    void set_retain(bool on) { retain_ = on; }
+    bool retain() const { return retain_; }
+    int mark_dirty(int32_t layer, const int32_t *ids, int64_t n);
+    int drop_host_copy(int32_t layer, int32_t block);  // a GPU-resident unit gives its kept host slot up
+    void mark_layer_dirty(int32_t layer);
     int attention(int32_t layer, const int32_t *ids, int64_t n, int64_t *ticket, int64_t *waits);
     int confirm(int32_t queue, int64_t ticket);
 
@@ -106,6 +115,7 @@ class Table {
     uint32_t clock_ = 0;
     int32_t n_allocated_ = 0;
     int32_t capacity_, target_ = -1, n_moved_ = 0;
+    bool retain_ = false;
     std::vector<uint8_t> moved_;  // per layer
 };
 

@@ -104,12 +104,23 @@ class DeviceWorkload:
         return out
 
     # ---- running ---------------------------------------------------------------------------------------
+    def set_retention(self, on: bool):
+        """Kept host copies + write-back elision (pie_set_retention); the blocks each step's append writes are
+        declared from the host mirror of the context lengths."""
+        self.retention = bool(on)
+        pie.pie_set_retention(self.pool, int(on))
+        if not on:
+            pie.pie_declare_append_blocks(self.pool, None)
+
     def advance_context(self):
         """One more token per sequence (the step's append position)."""
         self.ctx_lens += 1
         assert int(self.ctx_lens.max() - self.wl.ctx_lens.max()) <= self.extra_tokens, "block table has no room left"
         with torch.cuda.stream(self.s_compute):
             self.ctx_lens_dev += 1
+        if getattr(self, "retention", False):
+            tails = self.block_table[np.arange(self.wl.n_seqs), (self.ctx_lens - 1) // 16]
+            pie.pie_declare_append_blocks(self.pool, tails)
 
     def decode_step(self, append=True, mode=pie.PIE_MODE_AUTO):
         pie.pie_decode_step(self.pool, self.q_all.data_ptr(), self.out_all.data_ptr(), self.block_table_dev.data_ptr(),

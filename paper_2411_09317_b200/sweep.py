@@ -64,6 +64,8 @@ def main(argv=None):
     ap.add_argument("--ratios", default="", help="ratios: comma list instead of 0, 0.1, ... 1.0")
     ap.add_argument("--host-frac", type=float, default=0.5, help="adaptive: share of the blocks that starts host resident")
     ap.add_argument("--ctrl-step", type=float, default=1.0 / 64.0, help="adaptive: the controller's ratio step")
+    ap.add_argument("--kept-copies", action="store_true",
+                    help="host copies are kept after a swap-in and the write-back of unwritten blocks is skipped (pie_set_retention)")
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
     out = open(args.out, "w") if args.out else sys.stdout
@@ -85,8 +87,9 @@ def main(argv=None):
         _, _, nb = wl.tables()
         # both pools can hold everything: ratio 0 needs it on the GPU side, ratio 1 on the host side
         dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(L + 3) * nb + 64)
+        dw.set_retention(args.kept_copies)
         emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
-              "kv_gb": L * nb * wl.block_bytes / 1e9, "link": link})
+              "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "link": link})
         for r in ratios:
             pie.pie_set_extension_ratio(dw.pool, r)
             run_steps(dw, 2)
@@ -100,6 +103,7 @@ def main(argv=None):
                   "wait_share": sa["last_step_stall_ms"] / max(sa["last_step_ms"], 1e-9),
                   "last_step": {k: sa[k] for k in ("last_step_ms", "last_step_compute_ms", "last_step_stall_ms",
                                                    "last_step_swap_in_ms", "last_step_swap_out_ms")},
+                  "elided_out_gbs": (sa["reserved"][2] - sb["reserved"][2]) / tot / 1e9,
                   "calls_kernel": sa["calls_kernel"] - sb["calls_kernel"],
                   "calls_copy_engine": sa["calls_copy_engine"] - sb["calls_copy_engine"],
                   "swap_frac_of_link": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9 / link["both_per_dir"]})
@@ -115,6 +119,7 @@ def main(argv=None):
               "kv_gb": L * nb * wl.block_bytes / 1e9, "gpu_pool_gb": dw.n_gpu_slots * wl.block_bytes / 1e9,
               "host_pool_gb": dw.n_host_slots * wl.block_bytes / 1e9, "host_frac": args.host_frac,
               "ctrl_step": args.ctrl_step, "link": link})
+        dw.set_retention(args.kept_copies)
         pie.pie_set_controller(dw.pool, args.ctrl_step, 0.0, 0.0)
         pie.pie_set_extension_ratio(dw.pool, -1.0)
         per, sb, sa, ctx0, per_stats = run_steps(dw, args.steps)

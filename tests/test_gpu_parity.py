@@ -304,13 +304,19 @@ def test_large_batch_uses_the_separate_plan_kernel():
     pc.close()
 
 
-def test_multi_step_decode_with_append_matches_oracle_every_step():
+@pytest.mark.parametrize("retention", ["off", "declared", "undeclared", "host_tables"])
+def test_multi_step_decode_with_append_matches_oracle_every_step(retention):
     """Five decode steps on a small GQA model, 40 % of the blocks host resident: outputs of every step and the final
-    bytes of every unit against the oracle (append, prefetch, write-back, next-token look-ahead)."""
+    bytes of every unit against the oracle (append, prefetch, write-back, next-token look-ahead).  With kept host
+    copies, write-backs of blocks the step did not write are skipped: the bytes must come out the same, with the
+    written blocks declared by the caller, not declared at all (nothing may be skipped then), or derived by the
+    library from host tables."""
     lens = np.array([30, 63, 64, 65, 129, 7], dtype=np.int32)
     steps = 5
     case = Case(3, 8, 2, 128, BF16, lens, seed=42, host_frac=0.4, placement="random", extra_tokens=steps)
     pc = PoolCase(case, timing=1)
+    if retention != "off":
+        pie.pie_set_retention(pc.pool, 1)
     dev = torch.device("cuda:0")
     cur = lens.copy()
     ctx_dev = torch.from_numpy(cur).to(dev)
@@ -322,8 +328,17 @@ def test_multi_step_decode_with_append_matches_oracle_every_step():
         cur = cur + 1
         ctx_dev.copy_(torch.from_numpy(cur))
         torch.cuda.synchronize()
-        pie.pie_decode_step(pc.pool, pc.q.data_ptr(), pc.out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
-                            ctx_dev.data_ptr(), case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        if retention == "declared":     # the block of each sequence that receives this step's token
+            pie.pie_declare_append_blocks(pc.pool, case.block_table[np.arange(case.S), (cur - 1) // 16])
+        if retention == "host_tables":
+            out_host = np.zeros(tuple(pc.q.shape), dtype=np.int16)
+            pie.pie_decode_step_host(pc.pool, np.ascontiguousarray(case.q.view(np.int16)), out_host, case.block_table,
+                                     case.block_table.shape[1], cur.astype(np.int32), case.S, case.scale,
+                                     np.ascontiguousarray(k_new.view(np.int16)), np.ascontiguousarray(v_new.view(np.int16)))
+            pc.out.copy_(torch.from_numpy(out_host))
+        else:
+            pie.pie_decode_step(pc.pool, pc.q.data_ptr(), pc.out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                                ctx_dev.data_ptr(), case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
         pie.pie_sync(pc.pool)
         case.ctx_lens = cur.copy()
         for l in range(case.L):
@@ -335,6 +350,15 @@ def test_multi_step_decode_with_append_matches_oracle_every_step():
     for l in range(case.L):
         for b in range(case.NB):
             assert np.array_equal(pc.read_unit(l, b), pc.unit_bits(l, b)), (l, b)
+    stats = pie.pie_get_stats(pc.pool)
+    elided = stats["reserved"][2]
+    n_home = len(case.host_ids)
+    if retention in ("off", "undeclared"):
+        assert elided == 0
+    else:
+        # per step and layer every host-resident unit goes out once; only the written ones are copied
+        assert elided > 0 and elided + stats["bytes_out"] == steps * case.L * n_home * case.block_bytes
+        assert stats["bytes_out"] <= steps * case.L * case.S * case.block_bytes
     pc.close()
 
 

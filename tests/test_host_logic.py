@@ -58,6 +58,8 @@ def both_apply(o, t, op):
     elif kind in ("out", "in"):
         q = otable.Q_OUT if kind == "out" else otable.Q_IN
         a, b = o.swap(q, op[1], list(op[2])), t.swap(q, op[1], list(op[2]))
+        if a[0] == otable.OK:
+            assert list(o.last_elided) == list(t.last_elided), op
     elif kind == "attn":
         ra, rb = o.attention(op[1], list(op[2])), t.attention(op[1], list(op[2]))
         ra[2].pop(otable.Q_COMPUTE, None)  # same stream as the call itself: the library drops it
@@ -66,6 +68,10 @@ def both_apply(o, t, op):
         q, frac = op[1], op[2]
         tk = int(o.issued[q] * frac)
         a, b = o.confirm(q, tk), t.confirm(q, tk)
+    elif kind == "dirty":
+        a, b = o.mark_dirty(op[1], list(op[2])), t.mark_dirty(op[1], list(op[2]))
+    elif kind == "drop":
+        a, b = o.drop_host_copy(op[1], op[2]), t.drop_host_copy(op[1], op[2])
     elif kind == "resize":
         a, b = o.resize_begin(op[1]), t.resize_begin(op[1])
     elif kind == "pass":
@@ -97,14 +103,35 @@ def test_table_matches_oracle_exhaustive_tiny():
     assert n > 3000
 
 
-def test_table_matches_oracle_random_long():
+def test_table_with_kept_host_copies_matches_oracle_exhaustive_tiny():
+    alphabet = [("alloc", 1, True), ("free", 0), ("out", 0, (0,)), ("out", 1, (0, 1)), ("in", 0, (0,)), ("in", 1, (1, 0)),
+                ("attn", 0, (0,)), ("dirty", 0, (0,)), ("dirty", 1, (1, 0)), ("drop", 0, 0), ("confirm", otable.Q_OUT, 1.0),
+                ("confirm", otable.Q_IN, 1.0), ("confirm", otable.Q_COMPUTE, 1.0)]
+    n = 0
+    for length in range(1, 5):
+        for seq in itertools.product(alphabet, repeat=length):
+            o, t = otable.MappingTable(2, 2, 4, 4, retain=True), pie.Table(2, 2, 4, 4)
+            assert t.set_retention(True) == pie.PIE_OK
+            for op in [("alloc", 0, True), ("in", 0, (0,)), ("in", 1, (0,)), ("confirm", otable.Q_IN, 1.0)] + list(seq):
+                both_apply(o, t, op)
+            n += 1
+    assert n > 20000
+
+
+@pytest.mark.parametrize("retain", [False, True])
+def test_table_matches_oracle_random_long(retain):
     rng = random.Random(11)
     for trial in range(40):
         L, NB = rng.choice([(1, 6), (3, 5), (2, 9)])
-        ng, nh = rng.randint(NB, L * NB), rng.randint(NB, L * NB)
-        o, t = otable.MappingTable(L, NB, ng, nh), pie.Table(L, NB, ng, nh)
+        ng, nh = rng.randint(NB, L * NB), rng.randint(NB, L * NB) + (L * NB if retain else 0)
+        o, t = otable.MappingTable(L, NB, ng, nh, retain=retain), pie.Table(L, NB, ng, nh)
+        t.set_retention(retain)
         for _ in range(150):
             k = rng.random()
+            if retain and rng.random() < 0.15:
+                both_apply(o, t, ("dirty", rng.randrange(L), tuple(rng.sample(range(NB), rng.randint(1, NB)))))
+            if retain and rng.random() < 0.05:
+                both_apply(o, t, ("drop", rng.randrange(L), rng.randrange(NB)))
             ids = tuple(rng.sample(range(NB), rng.randint(1, NB)))
             if rng.random() < 0.05:
                 ids = ids + (ids[0],) if rng.random() < 0.5 else ids + (NB + 3,)

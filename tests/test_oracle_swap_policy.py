@@ -138,6 +138,8 @@ def apply_op(tbl, ex, op):
                         ex.g[s] = (layer, b, ex.version[(layer, b)])
             ex.issue(table.Q_COMPUTE, ticket, waits, body)
         return st
+    if kind == "drop":
+        return tbl.drop_host_copy(op[1], op[2])
     if kind == "confirm":  # the host learns how far the device got
         ex.drain() if op[1] else None
         for q in ex.ran:
@@ -191,7 +193,7 @@ def test_table_exhaustive_tiny_with_kept_host_copies():
     out never leaves stale bytes on the host, whatever the order the device runs things in."""
     alphabet = [("alloc", 0), ("alloc", 1), ("free", 0), ("out", 0, (0,)), ("out", 1, (0, 1)), ("in", 0, (0,)),
                 ("in", 1, (1, 0)), ("attn", 0, (0,)), ("attn_append", 0, (0,), (0,)), ("attn_append", 1, (0, 1), (1,)),
-                ("confirm", True), ("run", 1)]
+                ("drop", 0, 0), ("confirm", True), ("run", 1)]
     n_seq = n_elided = 0
     # from a warm state: both blocks allocated and every unit once out and back in, so that host copies are kept
     warm = [("alloc", 0), ("alloc", 1), ("out", 0, (0, 1)), ("out", 1, (0, 1)), ("in", 0, (0, 1)), ("in", 1, (0, 1)), ("confirm", True)]
@@ -303,7 +305,8 @@ def test_table_random_long_runs(retain):
             layer = rng.randrange(L)
             op = (("alloc", rng.randrange(NB)) if k < 0.15 else ("free", rng.randrange(NB)) if k < 0.2 else
                   ("out", layer, ids) if k < 0.45 else ("in", layer, ids) if k < 0.7 else
-                  ("attn", layer, ids) if k < 0.78 else ("attn_append", layer, ids, set(rng.sample(ids, 1))) if k < 0.85 else
+                  ("attn", layer, ids) if k < 0.76 else ("drop", layer, ids[0]) if k < 0.78 else
+                  ("attn_append", layer, ids, set(rng.sample(ids, 1))) if k < 0.85 else
                   ("confirm", rng.random() < 0.3) if k < 0.93 else ("run", 2))
             apply_op(tbl, ex, op)
             tbl.check_invariants()
