@@ -267,9 +267,9 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         mode = ((n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS) ? PIE_MODE_COPY_ENGINE
                                                                                                    : PIE_MODE_KERNEL;
     }
-    // Table entries after copy-engine copies.  The persistent attention kernel leaves no room for another CTA on any
-    // SM, so a patch kernel on a copy stream only gets to run in the gap between two attention launches - and the next
-    // layer, which waits for that swap's ticket, starts late by as much.  When the moved ids form a few runs of
+    // Table entries after copy-engine copies.  A patch kernel on a copy stream, launched while the persistent
+    // attention grid owns the SMs, was measured to lengthen the gap between two attention launches, and it puts an
+    // SM-side kernel on the path of the ticket the next layer waits for.  When the moved ids form a few runs of
     // consecutive blocks (the usual case: lists are in ascending id), the new entries are written to the pinned list
     // ring instead and one small host-to-device copy per run puts them into the layer's row: no SM is involved.
     bool dma_patch = false;
