@@ -134,3 +134,57 @@ def test_llama3_70b_shape_long_context_adaptive_controller():
     short = int(np.argmin(wl.ctx_lens))
     check_samples(dw, [(0, short), (15, short)], steps)
     free(dw)
+
+
+def test_step_timing_from_gpu_timer_stamps_and_timeline():
+    """The per-step statistics come from time stamps the attention kernel writes itself (no timing events on the
+    compute stream): they must agree with CUDA events around the same step, report no stall while nothing is swapped
+    and a dominant one once half of every layer has to cross the link, and the per-layer timeline must be ordered."""
+    lens = np.full(16, 4096, dtype=np.int32)
+    wl = synth.Workload("timing", 7, 4, 8, 8, 128, synth.F16, lens, 12, 0.0)
+    nb = int(((lens.astype(np.int64) + 12 + 15) // 16).sum())
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=2, extra_gpu_slots=3 * nb, extra_host_slots=5 * nb)
+    L = wl.n_layers
+
+    def one_measured_step():
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dw.advance_context()
+        dw.decode_step()                       # warm, so that the timed one follows a step directly
+        with torch.cuda.stream(dw.s_compute):
+            e0.record()
+        dw.advance_context()
+        dw.decode_step()
+        with torch.cuda.stream(dw.s_compute):
+            e1.record()
+        dw.sync()
+        pie.pie_controller_tick(dw.pool)
+        return e0.elapsed_time(e1), pie.pie_get_stats(dw.pool), pie.pie_get_step_timeline(dw.pool, L)
+
+    pie.pie_set_extension_ratio(dw.pool, 0.0)
+    ms, st, tl = one_measured_step()
+    assert st["steps_measured"] >= 1 and st["last_step_stall_ms"] == 0.0
+    assert 0.5 * ms <= st["last_step_ms"] <= ms + 0.01          # first kernel's start to last kernel's end
+    assert 0.8 * st["last_step_ms"] <= st["last_step_compute_ms"] <= st["last_step_ms"] + 1e-6
+    for l in range(L):
+        assert tl[l, 1] <= tl[l, 2] and tl[l, 0] <= tl[l, 1] + 1e-6, tl[l]
+        if l:
+            assert tl[l, 0] == tl[l - 1, 2]                      # a layer's time starts where the previous one ended
+        assert tl[l, 3] == -1 and tl[l, 5] == -1                 # no swap lists
+    # algorithmic bytes of the step / its compute time must be a plausible HBM rate
+    gbs = L * dw.attention_bytes_per_layer() / (st["last_step_compute_ms"] * 1e-3) / 1e9
+    assert 1000 < gbs < 8000, gbs
+
+    pie.pie_set_extension_ratio(dw.pool, 0.5)
+    one_measured_step()
+    ms, st, tl = one_measured_step()
+    assert st["last_step_stall_ms"] > 0.5 * st["last_step_ms"] > 0, st   # 134 MB per layer and direction behind a ~50 us layer
+    assert abs(st["last_step_ms"] - ms) < 0.25 * ms
+    assert st["last_step_swap_in_ms"] > 0 and st["last_step_swap_out_ms"] > 0
+    for l in range(1, L):
+        assert tl[l, 3] >= -1 and tl[l, 4] > tl[l, 3]            # swap-in list of the layer: start before end
+        assert tl[l, 1] >= tl[l, 4] - 0.05                       # the layer starts once its units have arrived (50 us slack
+                                                                 # between the anchor event and the first kernel's stamp)
+    dw.close()
+    del dw
+    gc.collect()
+    torch.cuda.empty_cache()
