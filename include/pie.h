@@ -351,9 +351,10 @@ int pie_fifo_layer_start(pie_fifo *f, int32_t k, int32_t *start_out, int32_t *st
 /* 0 GPU, 1 CPU, 2 in transit to the CPU, 3 in transit to the GPU */
 int pie_fifo_location(pie_fifo *f, int32_t layer);
 
-/* The controller's decision rule by itself.  state: 8 doubles owned by the caller, zero-initialised
- * (history in [0..4]; [5] = stall tolerance eps, [6] = link-busy ceiling u_hi, 0 = defaults 0.02 / 0.9).
- * Returns the new ratio for one decode step's measurements (same unit for all three). */
+/* The controller's decision rule by itself.  state: 16 doubles owned by the caller, zero-initialised
+ * (history in [0..4]; [5] = stall tolerance eps, [6] = link-busy ceiling u_hi, 0 = defaults 0.02 / 0.9; [7..11] the
+ * cooldown and the performance record: the lowest ratio known to stall and how long to leave it alone, which doubles
+ * with every failed probe).  Returns the new ratio for one decode step's measurements (same unit for all three). */
 double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
                              double swap_busy);
 

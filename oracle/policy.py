@@ -114,24 +114,43 @@ class Controller:
     u_hi: float = 0.9
     r_max: float = 1.0
     cooldown: int = 3
+    hold_max: int = 96
     r: float = 0.0
     wait: int = 0
     history: list = dataclasses.field(default_factory=list)
+    # performance record (Section 3.4.2): the lowest ratio known to make the computation wait, how long to leave it
+    # alone before probing it again (doubles with every failed probe), steps since the last back-off, and unstalled
+    # steps spent at or above that ratio (enough of them clear the record)
+    r_bad: float = -1.0
+    hold: int = 3
+    since_dec: int = 0
+    ok_at_bad: int = 0
 
     def tick(self, stall, compute, swap_busy):
         """One decode step's measurements (same time unit) -> new ratio."""
         stalled = stall > self.eps * compute
         self.history.append(stalled)
         self.history = self.history[-self.window:]
+        self.since_dec += 1
+        if self.r_bad >= 0:
+            self.ok_at_bad = self.ok_at_bad + 1 if (not stalled and self.r >= self.r_bad - 1e-12) else 0
+            if self.ok_at_bad >= self.window:           # the ratio that used to stall is fine now: forget the record
+                self.r_bad, self.hold, self.ok_at_bad = -1.0, self.cooldown, 0
         if stalled:
             if sum(self.history) >= self.k_dec:
+                # backing off from the known bad ratio (or below it) again: the next probe waits twice as long
+                again = self.r_bad >= 0 and self.r <= self.r_bad + 1e-12
+                self.hold = min(2 * self.hold, self.hold_max) if again else self.cooldown
+                self.r_bad, self.since_dec, self.ok_at_bad = self.r, 0, 0
                 self.r = max(0.0, self.r - self.step)
                 self.history = []
         elif self.wait > 0:
             self.wait -= 1
         elif swap_busy < self.u_hi * compute and self.r < self.r_max:
-            self.r = min(self.r_max, self.r + self.step)
-            self.wait = self.cooldown
+            target = min(self.r_max, self.r + self.step)
+            if not (self.r_bad >= 0 and target >= self.r_bad - 1e-12 and self.since_dec < self.hold):
+                self.r = target
+                self.wait = self.cooldown
         return self.r
 
 

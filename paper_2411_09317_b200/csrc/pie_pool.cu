@@ -93,7 +93,7 @@ struct pie_pool {
     // policy / controller
     int ratio_mode = 0;  // 0 unset (keep the caller's sets), 1 fixed, 2 adaptive
     double ratio = 0.0;
-    double ctrl_state[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    double ctrl_state[16] = {};
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
     bool poll_hold = false;  // a decode step is polling once per layer: nested calls skip theirs
     std::vector<int64_t> home_count;  // per layer: units whose home is the host

@@ -504,10 +504,15 @@ int pie_fifo_location(pie_fifo *f, int32_t layer) {
 // Constants (the paper gives none): eps = 0.02, back off on 2 stalls within 4 steps, grow while the
 // link is busy for less than 0.9 of the compute time, and after an increase wait 3 steps before the next one
 // (measurements arrive a few steps late: a change must be seen at work before it is built upon).
+// Performance record (Section 3.4.2): the lowest ratio known to make the computation wait is remembered; a probe
+// back up to it waits 3 steps after the back-off the first time and twice as long after every failed probe (at most
+// 96); four unstalled steps at or above that ratio clear the record.
+// state: [0..3] stall flags of the window, [4] their count, [5] eps, [6] u_hi, [7] steps left before the next increase,
+// [8] 1 + the bad ratio (0: none), [9] hold, [10] steps since the last back-off, [11] unstalled steps at or above it.
 double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
                              double swap_busy) {
     const double eps = state[5] > 0 ? state[5] : 0.02, u_hi = state[6] > 0 ? state[6] : 0.9;
-    const int window = 4, k_dec = 2;
+    const int window = 4, k_dec = 2, cooldown = 3, hold_max = 96;
     int n = (int)state[4];
     bool stalled = stall > eps * compute;
     if (n == window) {
@@ -516,18 +521,39 @@ double pie_controller_decide(double *state, double ratio, double step, double st
     }
     state[n++] = stalled ? 1.0 : 0.0;
     state[4] = n;
+    bool has_bad = state[8] > 0;
+    double r_bad = state[8] - 1.0;
+    if (state[9] <= 0) state[9] = cooldown;
+    state[10] += 1;
+    if (has_bad) {
+        state[11] = (!stalled && ratio >= r_bad - 1e-12) ? state[11] + 1 : 0;
+        if (state[11] >= window) {
+            state[8] = 0;
+            state[9] = cooldown;
+            state[11] = 0;
+            has_bad = false;
+        }
+    }
     if (stalled) {
         int count = 0;
         for (int i = 0; i < n; ++i) count += state[i] != 0.0;
         if (count >= k_dec) {
+            const bool again = has_bad && ratio <= r_bad + 1e-12;
+            state[9] = again ? std::min(2.0 * state[9], (double)hold_max) : (double)cooldown;
+            state[8] = 1.0 + ratio;
+            state[10] = 0;
+            state[11] = 0;
             ratio = std::max(0.0, ratio - step);
             state[4] = 0;  // start a fresh window after a change
         }
     } else if (state[7] > 0) {
         state[7] -= 1;
     } else if (swap_busy < u_hi * compute && ratio < 1.0) {
-        ratio = std::min(1.0, ratio + step);
-        state[7] = 3;
+        const double target = std::min(1.0, ratio + step);
+        if (!(has_bad && target >= r_bad - 1e-12 && state[10] < state[9])) {
+            ratio = target;
+            state[7] = cooldown;
+        }
     }
     return ratio;
 }

@@ -11,6 +11,7 @@ ratios:   the extension ratio is set to 0, 0.1, ... 1.0 (fraction of every layer
 adaptive: the controller owns the ratio.  --host-frac 0.5 (default): half of the blocks start host resident and the GPU
           pool holds only the other half, so the ratio has a floor; --host-frac 0: everything starts on the GPU and the
           ratio climbs from 0 until waits or slow-down appear.  Per step: ratio, floor, step time, wait share.
+interference: adaptive, with foreign pinned-memory traffic on the host link during the middle third of the run.
 Prints one JSON object per line.
 """
 from __future__ import annotations
@@ -58,7 +59,9 @@ def attention_bytes(wl, ctx):
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="llama3_8b")
-    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive"])
+    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive", "interference"])
+    ap.add_argument("--background-mb", type=int, default=256,
+                    help="interference: pinned-memory traffic per step and direction on two other streams, MB")
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller pools)")
     ap.add_argument("--steps", type=int, default=6)
     ap.add_argument("--ratios", default="", help="ratios: comma list instead of 0, 0.1, ... 1.0")
@@ -80,6 +83,9 @@ def main(argv=None):
     L = wl.n_layers
     link = {"h2d": pie.pie_probe_link(256 << 20, pie.PIE_H2D, 3), "d2h": pie.pie_probe_link(256 << 20, pie.PIE_D2H, 3),
             "both_per_dir": pie.pie_probe_link(256 << 20, 2, 3)}
+    if args.mode == "interference":
+        interference(args, wl, link, emit)
+        return
     if args.mode == "ratios":
         ratios = [float(x) for x in args.ratios.split(",")] if args.ratios else [round(0.1 * i, 1) for i in range(11)]
         total = len(ratios) * (args.steps + 4) + 4
@@ -131,6 +137,63 @@ def main(argv=None):
         emit({"summary": True, "final_ratio": sa["ratio"], "ratio_floor": sa["reserved"][1], "median_ms_per_step": float(np.median(per)),
               "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9, "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
               "attn_gbs": attention_bytes(wl, ctx0 + args.steps // 2) / (float(np.median(per)) * 1e-3) / 1e9})
+    dw.close()
+
+
+def interference(args, wl, link, emit):
+    """Section 3.4.2, last paragraph: other traffic on the host link takes bandwidth away; the controller is expected
+    to notice (waits or slow-down appear) and give ground, and to come back when the traffic stops.  Three phases of
+    --steps decode steps each: quiet, with --background-mb of pinned copies per step in each direction on two streams
+    of their own, quiet again."""
+    L = wl.n_layers
+    wl = dataclasses.replace(wl, decode_steps=3 * args.steps + 16)
+    _, _, nb = wl.tables()
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_host_slots=(L // 4 + 3) * nb, extra_gpu_slots=3 * nb)
+    dw.set_retention(args.kept_copies)
+    pie.pie_set_controller(dw.pool, args.ctrl_step, 0.0, 0.0)
+    pie.pie_set_extension_ratio(dw.pool, -1.0)
+    n = args.background_mb << 20
+    h_src = torch.empty(n, dtype=torch.uint8).pin_memory()
+    h_dst = torch.empty(n, dtype=torch.uint8).pin_memory()
+    d_a = torch.empty(n, dtype=torch.uint8, device=dw.dev)
+    d_b = torch.empty(n, dtype=torch.uint8, device=dw.dev)
+    s_bg_in, s_bg_out = torch.cuda.Stream(device=dw.dev), torch.cuda.Stream(device=dw.dev)
+    emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "ctrl_step": args.ctrl_step,
+          "background_mb_per_step_and_direction": args.background_mb, "kept_copies": args.kept_copies, "link": link})
+    run_steps(dw, 2)
+    for phase in ("quiet", "background", "quiet_again"):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        with torch.cuda.stream(dw.s_compute):
+            marks[0].record()
+        sb = pie.pie_get_stats(dw.pool)
+        ratios, slow = [], []
+        for i in range(args.steps):
+            if phase == "background":
+                # one step's worth of foreign traffic, released when the step starts
+                s_bg_in.wait_event(marks[i])
+                s_bg_out.wait_event(marks[i])
+                with torch.cuda.stream(s_bg_in):
+                    d_a.copy_(h_src, non_blocking=True)
+                with torch.cuda.stream(s_bg_out):
+                    h_dst.copy_(d_b, non_blocking=True)
+            dw.advance_context()
+            dw.decode_step()
+            st = pie.pie_get_stats(dw.pool)
+            ratios.append(st["ratio"])
+            slow.append((st["last_step_stall_ms"] + st["reserved"][0]) / max(st["last_step_compute_ms"], 1e-9))
+            with torch.cuda.stream(dw.s_compute):
+                marks[i + 1].record()
+        dw.sync()
+        torch.cuda.synchronize()
+        sa = pie.pie_get_stats(dw.pool)
+        per = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
+        tot = sum(per) * 1e-3
+        emit({"phase": phase, "median_ms_per_step": float(np.median(per)), "ratio_first": ratios[0], "ratio_last": ratios[-1],
+              "ratio_mean": float(np.mean(ratios)), "ratio_max": float(np.max(ratios)),
+              "wait_plus_slowdown_share_mean": float(np.mean(slow)),
+              "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9, "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
+              "background_gbs_per_dir": (args.background_mb * 2**20 * args.steps / tot / 1e9) if phase == "background" else 0.0,
+              "ratios": [round(r, 4) for r in ratios]})
     dw.close()
 
 

@@ -238,11 +238,11 @@ def test_fifo_matches_oracle_protocol(n, t_swap, g, c, cpu):
 @pytest.mark.parametrize("bw,tc,bytes_layer,L", [(50e9, 200e-6, 400e6, 32), (400e9, 300e-6, 400e6, 32), (1e12, 1e-3, 1e8, 8)])
 def test_controller_rule_matches_oracle(bw, tc, bytes_layer, L):
     c = policy.Controller(step=1.0 / L)
-    state = np.zeros(8)
+    state = np.zeros(16)
     r = 0.0
     rng = random.Random(3)
-    for i in range(300):
-        b = bw * (0.4 if 100 <= i < 110 or i > 200 else 1.0) * (1.0 + 0.2 * (rng.random() - 0.5))
+    for i in range(600):
+        b = bw * (0.4 if 100 <= i < 110 or 200 < i < 400 else 1.0) * (1.0 + 0.2 * (rng.random() - 0.5))
         m = policy.fake_clock_step(r, bytes_layer, b, tc, L)
         want = c.tick(*m)
         r = pie.pie_controller_decide(state, r, 1.0 / L, *m)

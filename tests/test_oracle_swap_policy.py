@@ -488,6 +488,28 @@ def test_controller_settles_at_the_transparent_ratio(bw, tc, bytes_layer, L):
     assert all(abs(r - r2) <= c.step + 0.1 * r2 + 1e-9 for r in trace[-40:])
 
 
+def test_controller_probes_a_ratio_that_keeps_stalling_less_and_less_often():
+    """Performance record (Section 3.4.2): at the transparent ratio the next step up always stalls.  Without a record
+    the rule would try it again every few steps; with it the probes thin out (the wait doubles after every failed one),
+    so that in steady state the computation rarely waits - and when conditions improve the record is dropped."""
+    bw, tc, bytes_layer, L = 50e9, 200e-6, 400e6, 32
+    c = policy.Controller(step=1.0 / L)
+    stalled = []
+    for _ in range(600):
+        m = policy.fake_clock_step(c.r, bytes_layer, bw, tc, L)
+        stalled.append(m[0] > c.eps * m[1])
+        c.tick(*m)
+    # stalled steps come in pairs (two of four trigger the back-off); their spacing grows up to the cap
+    first, last = sum(stalled[:100]), sum(stalled[-200:])
+    assert first >= 6 and last <= 6, (first, last)
+    assert c.hold == c.hold_max and c.r_bad > 0
+    # twice the bandwidth: the old bad ratio is fine now; the record must not hold the ratio down for long
+    r_star2 = min(1.0, 2 * bw * tc / bytes_layer)
+    for _ in range(c.hold_max + 8 * int(r_star2 * L + 2)):
+        c.tick(*policy.fake_clock_step(c.r, bytes_layer, 2 * bw, tc, L))
+    assert abs(c.r - r_star2) <= c.step + 0.1 * r_star2
+
+
 def test_controller_tolerates_one_disturbed_step():
     c = policy.Controller(step=0.1)
     for _ in range(3):
