@@ -68,6 +68,31 @@ def append(gpu_pool, host_pool, unit_side, unit_slot, k_new, v_new, block_table,
                             _p(block_table), block_table.shape[1], _p(_i32(ctx_lens)), len(ctx_lens), n_kv_heads, head_dim)
 
 
+def kv_write(gpu_pool, host_pool, unit_side, unit_slot, k, v, token_seq, token_pos, block_table, n_kv_heads, head_dim):
+    """Prefill-side write of a flat batch of tokens into the paged KV cache (the prompt's keys and values, Section 2.2):
+    token t is position token_pos[t] of sequence token_seq[t]; k[t], v[t] are [Hkv][D] 16-bit rows.  Its K row of head
+    h lands in row pos % 16 of the K half of head h's tile in the block that holds the position, its V row in the V
+    half - in whichever pool the unit lives (slot layout [Hkv][2][16][D]).  Plain loops: the definition.
+    Returns -1 (nothing written) if a position is beyond the table or a block id out of range."""
+    block_table = _i32(block_table)
+    k = np.ascontiguousarray(k, dtype=np.uint16).reshape(-1, n_kv_heads, head_dim)
+    v = np.ascontiguousarray(v, dtype=np.uint16).reshape(-1, n_kv_heads, head_dim)
+    for t in range(len(token_seq)):
+        s, pos = int(token_seq[t]), int(token_pos[t])
+        if not (0 <= s < block_table.shape[0] and 0 <= pos < 16 * block_table.shape[1]):
+            return -1
+        if not 0 <= block_table[s, pos // 16] < len(unit_slot):
+            return -1
+    for t in range(len(token_seq)):
+        s, pos = int(token_seq[t]), int(token_pos[t])
+        b = int(block_table[s, pos // 16])
+        pool = host_pool if unit_side[b] else gpu_pool
+        tile = pool[int(unit_slot[b])].reshape(n_kv_heads, 2, 16, head_dim)
+        tile[:, 0, pos % 16, :] = k[t]
+        tile[:, 1, pos % 16, :] = v[t]
+    return 0
+
+
 def paged_attention(gpu_pool, host_pool, unit_side, unit_slot, q, block_table, ctx_lens, n_q_heads, n_kv_heads,
                     head_dim, dtype, scale, precision="f32", nthreads=1, split_tokens=None):
     """Paged decode attention of one layer.  Pools are uint16 arrays (slot layout [Hkv][2][16][D]);

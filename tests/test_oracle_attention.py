@@ -176,3 +176,52 @@ def test_append_writes_position_ctx_minus_one():
         K, V = c.dense_kv(0, s)
         assert np.array_equal(K[-1], synth.bits16_to_f32(k_new[s], F16))
         assert np.array_equal(V[-1], synth.bits16_to_f32(v_new[s], F16))
+
+
+# ---- prefill-side write of many tokens (the oracle's definition against an independent reader) ----------------
+def test_kv_write_then_paged_attention_equals_dense_attention_on_the_source_arrays():
+    """The writer is tied to the reader, which is itself pinned against the dense brute force: a prompt written token
+    by token from dense K/V arrays must attend exactly like those arrays (a swapped K/V half, a transposed head/row
+    index or an off-by-one position fails)."""
+    rng = np.random.default_rng(5)
+    c = Case(1, 8, 4, 64, F16, [1, 16, 17, 45], seed=21, host_frac=0.5, placement="random", shuffle_table=True)
+    c.gpu_pool[:] = 0x7e00          # NaN everywhere: whatever is not written must not be read
+    c.host_pool[:] = 0x7e00
+    dense = {}
+    seqs, poss, ks, vs = [], [], [], []
+    for s in range(c.S):
+        ctx = int(c.ctx_lens[s])
+        K = rng.standard_normal((ctx, c.Hkv, c.D)).astype(np.float16)
+        V = rng.standard_normal((ctx, c.Hkv, c.D)).astype(np.float16)
+        dense[s] = (K, V)
+        for t in range(ctx):
+            seqs.append(s); poss.append(t); ks.append(K[t].view(np.uint16)); vs.append(V[t].view(np.uint16))
+    order = rng.permutation(len(seqs))         # any order of the flat batch
+    st = oracle.kv_write(c.gpu_pool, c.host_pool, c.unit_side[0], c.unit_slot[0], np.stack(ks)[order], np.stack(vs)[order],
+                         np.array(seqs)[order], np.array(poss)[order], c.block_table, c.Hkv, c.D)
+    assert st == 0
+    out = run(c, 0, "f64")
+    for s in range(c.S):
+        K, V = dense[s]
+        want = dense_attention(c.q_f(0)[s], K.astype(np.float64), V.astype(np.float64), c.scale)
+        assert np.abs(out[s] - want).max() < 1e-12
+
+
+def test_kv_write_of_one_token_per_sequence_is_the_append_and_touches_nothing_else():
+    c = Case(1, 4, 2, 64, F16, [16, 17, 1, 40], seed=12, host_frac=0.5, placement="random", extra_tokens=1)
+    k_new = synth.tensor_bits(12, synth.STREAM_KNEW, (c.S, c.Hkv, c.D), F16)
+    v_new = synth.tensor_bits(12, synth.STREAM_VNEW, (c.S, c.Hkv, c.D), F16)
+    g1, h1 = c.gpu_pool.copy(), c.host_pool.copy()
+    lens = c.ctx_lens + 1
+    oracle.append(g1, h1, c.unit_side[0], c.unit_slot[0], k_new, v_new, c.block_table, lens, c.Hkv, c.D)
+    g2, h2 = c.gpu_pool.copy(), c.host_pool.copy()
+    assert oracle.kv_write(g2, h2, c.unit_side[0], c.unit_slot[0], k_new, v_new, np.arange(c.S), lens - 1, c.block_table,
+                           c.Hkv, c.D) == 0
+    assert np.array_equal(g1, g2) and np.array_equal(h1, h2)
+    assert int((g2 != c.gpu_pool).sum() + (h2 != c.host_pool).sum()) <= c.S * c.Hkv * c.D * 2
+    # a position beyond the table, a sequence that does not exist: nothing is written
+    g3, h3 = c.gpu_pool.copy(), c.host_pool.copy()
+    for seq, pos in ((0, 16 * c.block_table.shape[1]), (c.S, 0), (0, -1)):
+        assert oracle.kv_write(g3, h3, c.unit_side[0], c.unit_slot[0], k_new[:2], v_new[:2], [1, seq], [3, pos],
+                               c.block_table, c.Hkv, c.D) == -1
+    assert np.array_equal(g3, c.gpu_pool) and np.array_equal(h3, c.host_pool)
