@@ -216,6 +216,20 @@ int pie_get_extension_ratio(pie_pool *pool, float *r);
  * the time-per-token record taken on steps without swap traffic (copies that are hidden can still slow the
  * attention down through shared HBM bandwidth). */
 int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
+/* ---- prefill-side KV write (Section 2.2: the prompt's keys and values enter the cache; the decode path above
+ * appends one token per sequence, this call writes any number) ---------------------------------------------
+ * k, v: device [n_tokens][n_kv_heads][head_dim] in the pool's 16-bit type.  Token t is position
+ * token_pos_dev[t] (0-based) of sequence token_seq_dev[t] (row of block_table_dev, n_seqs rows of
+ * max_blocks_per_seq ids): its rows go to row pos % 16 of the K and V halves of every head's tile in the block that
+ * holds the position.  Enqueued on the compute stream behind every copy that is still bringing a unit of the layer
+ * in; swap-outs of the layer issued afterwards wait for it.  Every unit written must be GPU resident: a token whose
+ * block is not (or whose position or sequence is out of range) is skipped and the next call that checks the device
+ * status word returns PIE_ERR_NOT_RESIDENT / PIE_ERR_INVALID.  Two tokens of one call must not name the same
+ * position.  With kept host copies every block of the layer counts as written. */
+int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, const int32_t *token_seq_dev,
+                 const int32_t *token_pos_dev, int64_t n_tokens, const int32_t *block_table_dev, int32_t max_blocks_per_seq,
+                 int32_t n_seqs);
+
 /* ---- kept host copies and write-back elision (a variant the paper does not have: Section 3.2 gives the
  * CPU region up once a unit has been swapped in) ---------------------------------------------------------
  * on != 0: a unit that is swapped in keeps its host slot; when it is swapped out again it returns to that slot, and

@@ -78,6 +78,56 @@ cudaError_t launch_patch(int32_t *table, const int32_t *entries, int64_t n, cuda
     return cudaGetLastError();
 }
 
+__device__ __forceinline__ void raise_status(int32_t *status, int32_t flag);  // defined with the other helpers below
+
+// Prefill-side write: a CTA takes a few consecutive tokens of a flat batch (about 16 KiB of rows) and copies each
+// token's K and V rows of every KV head into the block that holds its position (slot layout [Hkv][2][16][D], 16-byte
+// vectors).  A token whose block is not on the GPU, or whose position lies beyond the table, is skipped and flagged.
+__global__ void __launch_bounds__(256)
+kv_write_kernel(const uint4 *__restrict__ k, const uint4 *__restrict__ v, const int32_t *__restrict__ token_seq,
+                const int32_t *__restrict__ token_pos, int64_t n_tokens, int32_t tokens_per_cta,
+                const int32_t *__restrict__ block_table, int32_t max_blocks, int32_t n_seqs,
+                const int32_t *__restrict__ slot_table, int32_t n_logical, int64_t n_gpu_slots, uint4 *__restrict__ pool,
+                int32_t n_kv_heads, int32_t vecs_per_row, int32_t *status) {
+    const int32_t per_token = n_kv_heads * vecs_per_row;                  // vectors of K (and of V) per token
+    const int64_t slot_vecs = (int64_t)n_kv_heads * 2 * 16 * vecs_per_row;
+    const int64_t t0 = (int64_t)blockIdx.x * tokens_per_cta;
+    for (int32_t i = threadIdx.x; i < tokens_per_cta * 2 * per_token; i += blockDim.x) {
+        const int32_t tt = i / (2 * per_token), r = i - tt * 2 * per_token;
+        const int64_t t = t0 + tt;
+        if (t >= n_tokens) break;
+        const int32_t s = token_seq[t], pos = token_pos[t];
+        if (s < 0 || s >= n_seqs || pos < 0 || pos >= max_blocks * 16) {
+            if (r == 0) raise_status(status, STATUS_CTX_TOO_LONG);
+            continue;
+        }
+        const int32_t b = block_table[(int64_t)s * max_blocks + (pos >> 4)];
+        const int32_t slot = (b >= 0 && b < n_logical) ? slot_table[b] : -1;
+        if (slot < 0 || slot >= n_gpu_slots) {
+            if (r == 0) raise_status(status, STATUS_MISSING_UNIT);
+            continue;
+        }
+        const int32_t kv = r >= per_token, j = r - kv * per_token;
+        const int32_t h = j / vecs_per_row, c = j - h * vecs_per_row;
+        const uint4 val = (kv ? v : k)[t * per_token + j];
+        pool[(int64_t)slot * slot_vecs + (((int64_t)h * 2 + kv) * 16 + (pos & 15)) * vecs_per_row + c] = val;
+    }
+}
+
+cudaError_t launch_kv_write(const void *k, const void *v, const int32_t *token_seq, const int32_t *token_pos, int64_t n_tokens,
+                            const int32_t *block_table, int32_t max_blocks, int32_t n_seqs, const int32_t *slot_table,
+                            int32_t n_logical, int64_t n_gpu_slots, void *gpu_pool, int32_t n_kv_heads, int32_t head_dim,
+                            int32_t *status, cudaStream_t stream) {
+    if (n_tokens <= 0) return cudaSuccess;
+    const int32_t vecs_per_row = head_dim * 2 / 16;
+    const int32_t per_cta = std::max(1, 1024 / (2 * n_kv_heads * vecs_per_row));   // ~1024 vectors = 4 per thread
+    const int64_t grid = (n_tokens + per_cta - 1) / per_cta;
+    kv_write_kernel<<<(unsigned)grid, 256, 0, stream>>>((const uint4 *)k, (const uint4 *)v, token_seq, token_pos, n_tokens, per_cta,
+                                                       block_table, max_blocks, n_seqs, slot_table, n_logical, n_gpu_slots,
+                                                       (uint4 *)gpu_pool, n_kv_heads, vecs_per_row, status);
+    return cudaGetLastError();
+}
+
 __global__ void patch_from_list_kernel(int32_t *slot_table, const int32_t *__restrict__ list, int64_t n, int mode) {
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         slot_table[list[3 * i + 2]] = mode == 1 ? list[3 * i + 1] : -1;
@@ -916,7 +966,7 @@ int attn_smem_bytes(int head_dim) { return head_dim == 128 ? AttnSmem<128, 4, 2>
 // lands on an idle SM first could keep attention CTAs off that SM until it has finished.
 static cudaError_t prefer_max_shared() {
     const void *fns[] = {(const void *)swap_kernel, (const void *)patch_kernel, (const void *)patch_from_list_kernel,
-                         (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
+                         (const void *)kv_write_kernel, (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
                          (const void *)combine_kernel<64, true>, (const void *)combine_kernel<64, false>};
     for (const void *f : fns) {
         cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);

@@ -25,6 +25,13 @@ cudaError_t launch_patch(int32_t *table, const int32_t *entries, int64_t n, cuda
 cudaError_t launch_patch_from_list(int32_t *slot_table, const int32_t *list, int64_t n, int table_mode,
                                    cudaStream_t stream);
 
+// ---- prefill-side KV write -------------------------------------------------------------------------
+// k, v: device [n_tokens][n_kv_heads][head_dim] 16-bit; token t is position token_pos[t] of sequence token_seq[t].
+cudaError_t launch_kv_write(const void *k, const void *v, const int32_t *token_seq, const int32_t *token_pos, int64_t n_tokens,
+                            const int32_t *block_table, int32_t max_blocks, int32_t n_seqs, const int32_t *slot_table,
+                            int32_t n_logical, int64_t n_gpu_slots, void *gpu_pool, int32_t n_kv_heads, int32_t head_dim,
+                            int32_t *status, cudaStream_t stream);
+
 // ---- attention -----------------------------------------------------------------------------------
 struct AttnShape {
     int head_dim;      // 64 or 128

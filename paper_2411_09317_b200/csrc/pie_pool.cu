@@ -1240,6 +1240,44 @@ int pie_get_extension_ratio(pie_pool *pool, float *r) {
     return PIE_OK;
 }
 
+int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, const int32_t *token_seq_dev,
+                 const int32_t *token_pos_dev, int64_t n_tokens, const int32_t *block_table_dev, int32_t max_blocks_per_seq,
+                 int32_t n_seqs) {
+    if (!pool || n_tokens < 0 || max_blocks_per_seq <= 0 || n_seqs <= 0) return PIE_ERR_INVALID;
+    if (n_tokens > 0 && (!k || !v || !token_seq_dev || !token_pos_dev || !block_table_dev)) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    if (layer < 0 || layer >= pool->cfg.n_layers) return PIE_ERR_RANGE;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    st = check_status_word(pool);
+    if (st != PIE_OK) return st;
+    if (n_tokens == 0) return PIE_OK;
+    // like an attention call: a compute ticket, behind every copy that is still bringing a unit of the layer in
+    int64_t ticket = 0, waits[4];
+    st = pool->table->attention(layer, nullptr, 0, &ticket, waits);
+    if (st != PIE_OK) return st;
+    if (pool->table->retain()) pool->table->mark_layer_dirty(layer);  // which blocks are written is on the device only
+    cudaStream_t stream = pool->stream[PIE_Q_COMPUTE];
+    st = reserve_ticket_event(pool, PIE_Q_COMPUTE, ticket);
+    if (st != PIE_OK) { pool->sticky = st; return st; }
+    for (int qd = 1; qd <= 2; ++qd) {
+        st = wait_ticket(pool, stream, qd, waits[qd]);
+        if (st != PIE_OK) { pool->sticky = st; return st; }
+    }
+    cudaError_t e = pie::launch_kv_write(k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs,
+                                         pool->slot_table_dev + (int64_t)layer * pool->cfg.n_logical_blocks,
+                                         pool->cfg.n_logical_blocks, pool->cfg.n_gpu_slots, pool->gpu_base, pool->cfg.n_kv_heads,
+                                         pool->cfg.head_dim, pool->status_dev, stream);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        pool->sticky = PIE_ERR_CUDA;
+        return PIE_ERR_CUDA;
+    }
+    st = record_ticket(pool, PIE_Q_COMPUTE, ticket);
+    if (st != PIE_OK) pool->sticky = st;
+    return st;
+}
+
 int pie_set_retention(pie_pool *pool, int32_t on) {
     if (!pool) return PIE_ERR_INVALID;
     pool->table->set_retain(on != 0);

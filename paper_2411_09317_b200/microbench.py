@@ -158,6 +158,34 @@ def main(argv=None):
                               "swap_call_every": args.every,
                               "attn_ms": t1, "attn_ms_alone": ref, "slowdown": t1 / ref - 1.0, "swap_gbs_per_dir": gbs,
                               "frac_of_link": gbs / lref, "swap_keeps_up": t_swap <= t1 * 1.02})
+    # ---------------------------------------------------------------- part 3: prefill-side KV write
+    if "3" in args.part:
+        # every position of every sequence of the attention workload, one layer, in one call: reads the K/V rows once
+        # and writes them once (HBM-bound scatter of 2 * head_dim * 2-byte pieces)
+        ctx = dw.ctx_lens.astype(np.int64)
+        seq = np.repeat(np.arange(wl.n_seqs, dtype=np.int32), ctx)
+        pos = np.concatenate([np.arange(c, dtype=np.int32) for c in ctx])
+        T = len(seq)
+        k = torch.empty((T, wl.n_kv_heads, wl.head_dim), dtype=torch.int16, device=dw.dev)
+        v = torch.empty_like(k)
+        lib = pie.synth_lib()
+        for t_, stream in ((k, synth.STREAM_KNEW), (v, synth.STREAM_VNEW)):
+            base = int(synth.stream_base(wl.seed, stream)) & 0xFFFFFFFFFFFFFFFF
+            assert lib.pie_synth_fill_tensor(t_.data_ptr(), t_.numel(), base, 0, wl.dtype, 1.0, None) == 0
+        seq_d, pos_d = torch.from_numpy(seq).to(dw.dev), torch.from_numpy(pos).to(dw.dev)
+        torch.cuda.synchronize()
+        times = []
+        for r in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(s_c)
+            pie.pie_kv_write(dw.pool, r % wl.n_layers, k.data_ptr(), v.data_ptr(), seq_d.data_ptr(), pos_d.data_ptr(), T,
+                             dw.block_table_dev.data_ptr(), dw.max_blocks, wl.n_seqs)
+            e1.record(s_c)
+            dw.sync()
+            times.append(e0.elapsed_time(e1))
+        ms = float(np.median(times[1:]))
+        nbytes = 2 * 2 * T * wl.n_kv_heads * wl.head_dim * 2     # K and V, read once and written once
+        emit({"part": "kv_write", "tokens": T, "ms": ms, "gbs_read_plus_write": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes})
     dw.close()
 
 

@@ -395,6 +395,63 @@ def test_block_free_and_reuse_and_nomem():
     pc.close()
 
 
+# ---------------------------------------------------------------- prefill-side KV write
+@pytest.mark.parametrize("hq,hkv,d,dtype", [(8, 4, 64, F16), (8, 8, 128, BF16), (8, 1, 128, F16)])
+def test_kv_write_bit_exact_and_then_attention(hq, hkv, d, dtype):
+    """Whole prompts are written token by token (flat batch, shuffled order) into pools that start as poison: every byte
+    of every unit equals the oracle's write, and decode attention over what was written matches the oracle."""
+    lens = np.array([1, 16, 17, 100, 45], dtype=np.int32)
+    case = Case(2, hq, hkv, d, dtype, lens, seed=61)
+    expect_gpu = case.gpu_pool.copy()                 # the contents the generator defines: the source of the K/V rows
+    seqs, poss = [], []
+    for s in range(case.S):
+        for t in range(int(lens[s])):
+            seqs.append(s); poss.append(t)
+    order = synth.seeded_permutation(61, len(seqs), salt=9)
+    seqs, poss = np.array(seqs, np.int32)[order], np.array(poss, np.int32)[order]
+    case.gpu_pool[:] = 0x7e00                         # poison: NaN in both 16-bit formats
+    pc = PoolCase(case)                               # the pool now holds poison in every unit
+    dev = torch.device("cuda:0")
+    seq_dev, pos_dev = torch.from_numpy(seqs).to(dev), torch.from_numpy(poss).to(dev)
+    for l in range(case.L):
+        k = np.zeros((len(seqs), hkv, d), np.uint16)
+        v = np.zeros((len(seqs), hkv, d), np.uint16)
+        for i, (s_, p_) in enumerate(zip(seqs, poss)):
+            b = case.block_table[s_, p_ // 16]
+            tile = expect_gpu[case.unit_slot[l, b]].reshape(hkv, 2, 16, d)
+            k[i], v[i] = tile[:, 0, p_ % 16, :], tile[:, 1, p_ % 16, :]
+        k_dev, v_dev = torch.from_numpy(k.view(np.int16)).to(dev), torch.from_numpy(v.view(np.int16)).to(dev)
+        torch.cuda.synchronize()
+        pie.pie_kv_write(pc.pool, l, k_dev.data_ptr(), v_dev.data_ptr(), seq_dev.data_ptr(), pos_dev.data_ptr(), len(seqs),
+                         pc.bt.data_ptr(), case.block_table.shape[1], case.S)
+        assert oracle.kv_write(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k, v, seqs, poss,
+                               case.block_table, hkv, d) == 0
+    pie.pie_sync(pc.pool)
+    for l in range(case.L):
+        for b in range(case.NB):
+            assert np.array_equal(pc.read_unit(l, b), pc.unit_bits(l, b)), (l, b)     # written rows and untouched poison alike
+        check_attention(case, pc, l, edge=True)
+    # a token beyond the table, and a block that is not on the GPU: skipped and reported, nothing else touched
+    bad_pos = torch.tensor([16 * case.block_table.shape[1]], dtype=torch.int32, device=dev)
+    one = torch.zeros(1, dtype=torch.int32, device=dev)
+    pie.pie_kv_write(pc.pool, 0, k_dev.data_ptr(), v_dev.data_ptr(), one.data_ptr(), bad_pos.data_ptr(), 1, pc.bt.data_ptr(),
+                     case.block_table.shape[1], case.S)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_sync(pc.pool)
+    assert e.value.status == pie.PIE_ERR_INVALID
+    pie.pie_swap_out(pc.pool, 0, [int(case.block_table[3, 0])])
+    zero_pos = torch.zeros(1, dtype=torch.int32, device=dev)
+    three = torch.full((1,), 3, dtype=torch.int32, device=dev)
+    pie.pie_kv_write(pc.pool, 0, k_dev.data_ptr(), v_dev.data_ptr(), three.data_ptr(), zero_pos.data_ptr(), 1, pc.bt.data_ptr(),
+                     case.block_table.shape[1], case.S)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_sync(pc.pool)
+    assert e.value.status == pie.PIE_ERR_NOT_RESIDENT
+    for b in range(case.NB):
+        assert np.array_equal(pc.read_unit(0, b), pc.unit_bits(0, b)), b
+    pc.close()
+
+
 # ---------------------------------------------------------------- run-time resize (Section 4.1) on a live pool
 def test_resize_grow_then_shrink_while_serving():
     """The per-layer size grows from 8 to 11 blocks and shrinks back while attention calls keep running: new ids appear
