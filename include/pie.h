@@ -71,7 +71,8 @@ typedef struct pie_pool_config {
     void *copy_in_stream;
     void *copy_out_stream;
     int32_t own_streams;       /* 1: the library creates three non-blocking streams */
-    int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (512) */
+    int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (512; 1024 where the pool is laid
+                                * out for long sequences: n_logical_blocks * 16 / max_seqs >= 6144) */
     int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
     int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
     int32_t timing;            /* 1: per-layer timing for pie_controller_tick / pie_get_stats (the attention kernel notes

@@ -762,7 +762,11 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     pie_pool *p = new (std::nothrow) pie_pool();
     if (!p) return PIE_ERR_NOMEM;
     p->cfg = *cfg;
-    if (p->cfg.split_tokens == 0) p->cfg.split_tokens = 512;
+    // Split-K chunk: 512 tokens balances the persistent grid best on batches of many short sequences; where the pool
+    // is laid out for few long ones (>= 6144 tokens per sequence on average) 1024 halves the partials and the merge
+    // (measured: +6.5 % on 17 sequences of 4k-32k tokens with 8-head groups, -1.5 % on the batched shapes).
+    if (p->cfg.split_tokens == 0)
+        p->cfg.split_tokens = (int64_t)cfg->n_logical_blocks * 16 / std::max(cfg->max_seqs, 1) >= 6144 ? 1024 : 512;
     p->block_bytes = (int64_t)2 * 16 * cfg->n_kv_heads * cfg->head_dim * 2;
     p->n_sms = prop.multiProcessorCount;
     p->table = new (std::nothrow) pie::Table(cfg->n_layers, cfg->n_logical_blocks, cfg->n_gpu_slots, cfg->n_host_slots);

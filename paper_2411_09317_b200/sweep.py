@@ -69,6 +69,7 @@ def main(argv=None):
     ap.add_argument("--ctrl-step", type=float, default=1.0 / 64.0, help="adaptive: the controller's ratio step")
     ap.add_argument("--kept-copies", action="store_true",
                     help="host copies are kept after a swap-in and the write-back of unwritten blocks is skipped (pie_set_retention)")
+    ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
     out = open(args.out, "w") if args.out else sys.stdout
@@ -92,7 +93,8 @@ def main(argv=None):
         wl = dataclasses.replace(wl, decode_steps=total)
         _, _, nb = wl.tables()
         # both pools can hold everything: ratio 0 needs it on the GPU side, ratio 1 on the host side
-        dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(L + 3) * nb + 64)
+        dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(L + 3) * nb + 64,
+                            split_tokens=args.split)
         dw.set_retention(args.kept_copies)
         emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
               "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "link": link})
