@@ -183,6 +183,15 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
 int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev,
                     int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale,
                     const void *k_new_all, const void *v_new_all, int32_t mode);
+/* One layer of pie_decode_step by itself, for callers that run other work between the layers (Section 4.2: supporting
+ * a model means adding this control loop to its forward pass): fetches whatever the layer still lacks, starts the
+ * prefetch of layer (layer+1) mod n_layers, runs the attention (and the append, if k_new / v_new are given) and
+ * pushes this layer's host-resident share out behind it.  q / out / k_new / v_new are this layer's device arrays
+ * ([n_seqs][n_q_heads][head_dim], [n_seqs][n_kv_heads][head_dim]).  Call pie_step_begin before layer 0 and
+ * pie_controller_tick after the last layer when timing is on.  PIE_ERR_UNSUPPORTED under pie_set_layer_policy. */
+int pie_decode_layer(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
+                     int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new,
+                     const void *v_new, int32_t mode);
 /* The same with q / k_new / v_new / out in HOST memory (pinned for full speed): copies the inputs in,
  * runs the step, copies out_all back and waits for it.  ctx_lens_host/block_table_host are uploaded too. */
 int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_host, const int32_t *block_table_host,

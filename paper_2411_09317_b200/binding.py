@@ -36,7 +36,7 @@ EXPORTS = [
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
-    "pie_declare_append_blocks", "pie_kv_write",
+    "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer",
 ]
 
 
@@ -117,6 +117,7 @@ _sig = {
     "pie_table_mark_dirty": (_i32, [_vp, _i32, _vp, _i64]),
     "pie_table_drop_host_copy": (_i32, [_vp, _i32, _i32]),
     "pie_set_retention": (_i32, [_vp, _i32]),
+    "pie_decode_layer": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _i32, _f32, _vp, _vp, _i32]),
     "pie_kv_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i64, _vp, _i32, _i32]),
     "pie_declare_append_blocks": (_i32, [_vp, _vp, _i64]),
     "pie_table_init_capacity": (_i32, [_vp, _i32]),
@@ -284,6 +285,12 @@ def pie_decode_step(pool, q_all, out_all, block_table_dev, max_blocks_per_seq, c
                     k_new_all=None, v_new_all=None, mode=PIE_MODE_AUTO) -> None:
     check(lib.pie_decode_step(pool, _ptr(q_all), _ptr(out_all), _ptr(block_table_dev), max_blocks_per_seq,
                               _ptr(ctx_lens_dev), n_seqs, scale, _ptr(k_new_all), _ptr(v_new_all), mode), "pie_decode_step")
+
+
+def pie_decode_layer(pool, layer, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, n_seqs, scale, k_new=None,
+                     v_new=None, mode=PIE_MODE_AUTO) -> None:
+    check(lib.pie_decode_layer(pool, layer, _ptr(q), _ptr(out), _ptr(block_table_dev), max_blocks_per_seq, _ptr(ctx_lens_dev),
+                               n_seqs, scale, _ptr(k_new), _ptr(v_new), mode), "pie_decode_layer")
 
 
 def pie_decode_step_host(pool, q_all_host, out_all_host, block_table_host, max_blocks_per_seq, ctx_lens_host, n_seqs,

@@ -79,6 +79,7 @@ struct pie_pool {
     // device status word (mapped pinned memory)
     int32_t *status_host = nullptr, *status_dev = nullptr;
     uint64_t *stamps_host = nullptr, *stamps_dev = nullptr;  // [TIMING_RING][n_layers][STAMP_WORDS]
+    uint64_t free_step_gap_ns = 0;   // smallest gap between two layers' attention kernels in the newest step without swaps
     uint64_t prev_step_end = 0;   // GPU-timer stamp of the end of the last layer of the newest evaluated step
     int64_t prev_step_id = -1;
     bool prev_step_prefetched0 = false;  // that step issued a prefetch of layer 0 for the step after it
@@ -118,6 +119,7 @@ struct pie_pool {
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
     std::vector<uint8_t> v_elide;
+    std::vector<int32_t> v_plan_in, v_plan_out;  // one layer's plan inside the decode loop
     std::vector<int32_t> append_ids;  // blocks the coming appends write (pie_declare_append_blocks)
     bool append_declared = false;
     int sticky = PIE_OK;
@@ -1069,19 +1071,24 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     // kernel to the end of its own (combine and launch gap included, with or without swaps).  What the gap before a
     // layer that had units brought in exceeds the usual gap by is the stall: the stream sat in the presence wait.  The
     // usual gap is the smallest one of the step, but no more than 20 us, so that a step in which every layer waits
-    // still shows it.
+    // still shows it - or the smallest gap of the newest swap-free step, where that is larger.
     const bool chained = pool->prev_step_id == pool->lev_step[k] - 1 && pool->prev_step_end != 0;
     uint64_t prev_end = chained ? pool->prev_step_end : 0, first = 0, last = 0;
     uint64_t usual_gap = 20000;
     double first_stall = 0.0;
     {
-        uint64_t pe = 0;
+        uint64_t pe = 0, step_min = ~uint64_t(0);
         for (size_t l = 0; l < L; ++l) {
             const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
             if (!ev[l].has_compute || !S || !E) continue;
-            if (pe && S > pe) usual_gap = std::min(usual_gap, S - pe);
+            if (pe && S > pe) step_min = std::min(step_min, S - pe);
             pe = E;
         }
+        // A caller that runs other kernels between the layers has long gaps without any waiting: the smallest gap of
+        // the newest step that moved nothing is the better yardstick where one has been seen.
+        if (!any_swap && step_min != ~uint64_t(0)) pool->free_step_gap_ns = step_min;
+        if (pool->free_step_gap_ns) usual_gap = std::max(pool->free_step_gap_ns, std::min(usual_gap, step_min));
+        else usual_gap = std::min(usual_gap, step_min);
     }
     for (size_t l = 0; l < L; ++l) {
         const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
@@ -1500,6 +1507,54 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
     return pie_controller_tick(pool, nullptr);
 }
 
+// One layer of the control loop (Section 3.2; Section 4.2: what a model's forward pass calls per layer): fetch what the
+// layer still lacks, start the prefetch of the next layer, attend (and append), push this layer's host-resident share out.
+static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, const int32_t *block_table_dev,
+                        int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new,
+                        const void *v_new, int32_t mode) {
+    const int32_t L = pool->cfg.n_layers;
+    struct PollHold {
+        pie_pool *p;
+        bool was;
+        ~PollHold() { p->poll_hold = was; }
+    } hold{pool, pool->poll_hold};
+    // completions are learnt every few layers: a stale view only means a wait on an event that has already
+    // completed, or a slot that stays "pending" a little longer
+    if (l % 8 == 0) {
+        int st = poll(pool, true);
+        if (st != PIE_OK) return st;
+    }
+    pool->poll_hold = true;
+    // units of this layer that nobody prefetched (the very first layer of a run, a caller that skipped a layer):
+    // fetch them now; the attention call waits for the copy
+    {
+        pool->v_in.clear();
+        for (int32_t b : candidate_ids(pool, l))
+            if (pool->table->unit(l, b).side == PIE_HOST) pool->v_in.push_back(b);
+        if (!pool->v_in.empty()) {
+            std::vector<int32_t> ids(pool->v_in);
+            int st = pool_swap(pool, PIE_Q_IN, l, ids.data(), (int64_t)ids.size(), mode);
+            if (st != PIE_OK) return st;
+        }
+    }
+    std::vector<int32_t> &in_ids = pool->v_plan_in, &out_ids = pool->v_plan_out;
+    int st = plan_layer(pool, l, in_ids, out_ids);
+    if (st != PIE_OK) return st;  // the GPU pool cannot take the next layer's share: nothing was enqueued for it
+    if (L > 1 && !in_ids.empty()) {
+        // starts when layer l starts, i.e. once the previous attention call has finished
+        st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode, pool->table->issued(PIE_Q_COMPUTE));
+        if (st != PIE_OK) return st;
+    }
+    st = attention_call(pool, l, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
+                        k_new, v_new);
+    if (st != PIE_OK) return st;
+    if (L > 1 && !out_ids.empty()) {
+        st = pool_swap(pool, PIE_Q_OUT, l, out_ids.data(), (int64_t)out_ids.size(), mode);
+        if (st != PIE_OK) return st;
+    }
+    return PIE_OK;
+}
+
 int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev, int32_t max_blocks_per_seq,
                     const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new_all, const void *v_new_all,
                     int32_t mode) {
@@ -1513,49 +1568,24 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
     const int64_t kv_stride = (int64_t)n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;
     int st = pie_step_begin(pool);
     if (st != PIE_OK) return st;
-    // layer 0 has no predecessor in the first step: fetch what it needs now (later steps prefetch it from layer L-1)
-    struct PollHold {
-        pie_pool *p;
-        ~PollHold() { p->poll_hold = false; }
-    } hold{pool};
-    pool->poll_hold = true;
-    {
-        pool->v_in.clear();
-        for (int32_t b : candidate_ids(pool, 0))
-            if (pool->table->unit(0, b).side == PIE_HOST) pool->v_in.push_back(b);
-        if (!pool->v_in.empty()) {
-            std::vector<int32_t> ids(pool->v_in);
-            st = pool_swap(pool, PIE_Q_IN, 0, ids.data(), (int64_t)ids.size(), mode);
-            if (st != PIE_OK) return st;
-        }
-    }
-    std::vector<int32_t> in_ids, out_ids;
     for (int32_t l = 0; l < L; ++l) {
-        // completions are learnt every few layers: a stale view only means a wait on an event that has already
-        // completed, or a slot that stays "pending" a little longer
-        if (l % 8 == 0) {
-            st = poll(pool, true);
-            if (st != PIE_OK) return st;
-        }
-        st = plan_layer(pool, l, in_ids, out_ids);
-        if (st != PIE_OK) return st;  // the GPU pool cannot take the next layer's share: nothing was enqueued for it
-        if (L > 1 && !in_ids.empty()) {
-            // starts when layer l starts, i.e. once the previous attention call has finished
-            st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode,
-                           pool->table->issued(PIE_Q_COMPUTE));
-            if (st != PIE_OK) return st;
-        }
-        st = attention_call(pool, l, (const uint8_t *)q_all + l * q_stride, (uint8_t *)out_all + l * q_stride, block_table_dev,
-                            max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
-                            k_new_all ? (const uint8_t *)k_new_all + l * kv_stride : nullptr,
-                            v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr);
+        st = decode_layer(pool, l, (const uint8_t *)q_all + l * q_stride, (uint8_t *)out_all + l * q_stride, block_table_dev,
+                          max_blocks_per_seq, ctx_lens_dev, n_seqs, scale,
+                          k_new_all ? (const uint8_t *)k_new_all + l * kv_stride : nullptr,
+                          v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr, mode);
         if (st != PIE_OK) return st;
-        if (L > 1 && !out_ids.empty()) {
-            st = pool_swap(pool, PIE_Q_OUT, l, out_ids.data(), (int64_t)out_ids.size(), mode);
-            if (st != PIE_OK) return st;
-        }
     }
     return pie_controller_tick(pool, nullptr);
+}
+
+int pie_decode_layer(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
+                     int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new,
+                     const void *v_new, int32_t mode) {
+    if (!pool || !q || !out) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    if (pool->fifo) return PIE_ERR_UNSUPPORTED;  // the whole-layer protocol is driven by pie_decode_step
+    if (layer < 0 || layer >= pool->cfg.n_layers) return PIE_ERR_RANGE;
+    return decode_layer(pool, layer, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, n_seqs, scale, k_new, v_new, mode);
 }
 
 int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_host, const int32_t *block_table_host,

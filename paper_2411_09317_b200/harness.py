@@ -122,10 +122,23 @@ class DeviceWorkload:
             tails = self.block_table[np.arange(self.wl.n_seqs), (self.ctx_lens - 1) // 16]
             pie.pie_declare_append_blocks(self.pool, tails)
 
-    def decode_step(self, append=True, mode=pie.PIE_MODE_AUTO):
-        pie.pie_decode_step(self.pool, self.q_all.data_ptr(), self.out_all.data_ptr(), self.block_table_dev.data_ptr(),
-                            self.max_blocks, self.ctx_lens_dev.data_ptr(), self.wl.n_seqs, self.scale,
-                            self.k_new.data_ptr() if append else None, self.v_new.data_ptr() if append else None, mode)
+    def decode_step(self, append=True, mode=pie.PIE_MODE_AUTO, between_layers=None):
+        """One decode step.  between_layers(l), if given, is called after every layer's attention has been enqueued (the
+        place of a model's projections and MLP): the step then goes layer by layer through pie_decode_layer."""
+        if between_layers is None:
+            pie.pie_decode_step(self.pool, self.q_all.data_ptr(), self.out_all.data_ptr(), self.block_table_dev.data_ptr(),
+                                self.max_blocks, self.ctx_lens_dev.data_ptr(), self.wl.n_seqs, self.scale,
+                                self.k_new.data_ptr() if append else None, self.v_new.data_ptr() if append else None, mode)
+            return
+        pie.pie_step_begin(self.pool)
+        for l in range(self.wl.n_layers):
+            pie.pie_decode_layer(self.pool, l, self.q_all[l].data_ptr(), self.out_all[l].data_ptr(),
+                                 self.block_table_dev.data_ptr(), self.max_blocks, self.ctx_lens_dev.data_ptr(), self.wl.n_seqs,
+                                 self.scale, self.k_new[l].data_ptr() if append else None,
+                                 self.v_new[l].data_ptr() if append else None, mode)
+            with torch.cuda.stream(self.s_compute):
+                between_layers(l)
+        pie.pie_controller_tick(self.pool)
 
     def attention(self, layer, append=False, host_tables=False):
         pie.pie_decode_attention(

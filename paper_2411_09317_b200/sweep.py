@@ -29,19 +29,22 @@ from . import synth
 from .harness import DeviceWorkload
 
 
+OTHER = {"fn": None}   # stand-in for a model's other per-layer work (--other-mb): called after every layer's attention
+
+
 def run_steps(dw, n):
     """n decode steps; -> (per-step ms by CUDA events, stats before, stats after, context lengths before)"""
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
     dw.sync()
     dw.advance_context()
-    dw.decode_step()
+    dw.decode_step(between_layers=OTHER["fn"])
     before, ctx0 = pie.pie_get_stats(dw.pool), dw.ctx_lens.copy()
     with torch.cuda.stream(dw.s_compute):
         marks[0].record()
     per_stats = []
     for i in range(n):
         dw.advance_context()
-        dw.decode_step()
+        dw.decode_step(between_layers=OTHER["fn"])
         per_stats.append(pie.pie_get_stats(dw.pool))
         with torch.cuda.stream(dw.s_compute):
             marks[i + 1].record()
@@ -69,6 +72,10 @@ def main(argv=None):
     ap.add_argument("--ctrl-step", type=float, default=1.0 / 64.0, help="adaptive: the controller's ratio step")
     ap.add_argument("--kept-copies", action="store_true",
                     help="host copies are kept after a swap-in and the write-back of unwritten blocks is skipped (pie_set_retention)")
+    ap.add_argument("--other-mb", type=int, default=0,
+                    help="ratios / adaptive: after every layer's attention, an elementwise kernel that reads and writes this many MB "
+                         "on the compute stream stands in for the model's projections and MLP (weights streamed from HBM); the "
+                         "step then runs layer by layer through pie_decode_layer")
     ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
@@ -78,6 +85,12 @@ def main(argv=None):
         out.write(json.dumps(obj) + "\n")
         out.flush()
 
+    if args.other_mb > 0:
+        # an elementwise kernel, not a memcpy: a device-to-device cudaMemcpyAsync may be served by the copy engines,
+        # which the swaps need
+        w_src = torch.zeros((args.other_mb << 20) // 4, dtype=torch.float32, device="cuda")
+        w_dst = torch.empty_like(w_src)
+        OTHER["fn"] = lambda l: torch.add(w_src, 1.0, out=w_dst)
     wl = synth.workload(args.workload)
     if args.layers:
         wl = dataclasses.replace(wl, n_layers=args.layers)
@@ -97,7 +110,8 @@ def main(argv=None):
                             split_tokens=args.split)
         dw.set_retention(args.kept_copies)
         emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
-              "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "link": link})
+              "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "other_mb_per_layer": args.other_mb,
+              "link": link})
         for r in ratios:
             pie.pie_set_extension_ratio(dw.pool, r)
             run_steps(dw, 2)

@@ -395,6 +395,38 @@ def test_block_free_and_reuse_and_nomem():
     pc.close()
 
 
+# ---------------------------------------------------------------- the control loop layer by layer (Section 4.2)
+def test_layer_by_layer_loop_with_other_work_in_between_equals_the_whole_step():
+    """pie_decode_layer per layer, with another kernel on the compute stream after every layer, gives bit for bit what
+    pie_decode_step gives - outputs, every unit's bytes, placement and byte counters - over several steps."""
+    from paper_2411_09317_b200.harness import DeviceWorkload
+    lens = synth.uniform_lengths(71, 6, 40, 300)
+    wl = synth.Workload("loop", 71, 4, 8, 2, 128, BF16, lens, 6, 0.4)
+    runs = []
+    for manual in (False, True):
+        dw = DeviceWorkload(wl, timing=True)
+        scratch = torch.zeros(1 << 20, dtype=torch.float32, device=dw.dev)
+        outs = []
+        for step in range(4):
+            dw.advance_context()
+            dw.decode_step(between_layers=(lambda l: scratch.add_(1.0)) if manual else None)
+            dw.sync()
+            outs.append(dw.out_bits().copy())
+        units = [pie.pie_block_read(dw.pool, l, b).copy() for l in range(wl.n_layers) for b in range(dw.NB)]
+        side, slot = pie.pie_get_placement(dw.pool, wl.n_layers, dw.NB)
+        st = pie.pie_get_stats(dw.pool)
+        runs.append((outs, units, side.copy(), st["bytes_in"], st["bytes_out"]))
+        if manual:
+            assert float(scratch[0]) == 4 * wl.n_layers
+        dw.close()
+    a, b = runs
+    for x, y in zip(a[0], b[0]):
+        assert np.array_equal(x, y)
+    for x, y in zip(a[1], b[1]):
+        assert np.array_equal(x, y)
+    assert np.array_equal(a[2], b[2]) and a[3] == b[3] > 0 and a[4] == b[4] > 0
+
+
 # ---------------------------------------------------------------- prefill-side KV write
 @pytest.mark.parametrize("hq,hkv,d,dtype", [(8, 4, 64, F16), (8, 8, 128, BF16), (8, 1, 128, F16)])
 def test_kv_write_bit_exact_and_then_attention(hq, hkv, d, dtype):
