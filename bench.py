@@ -306,9 +306,10 @@ def main():
     swapped_out = s_after["bytes_out"] - s_before["bytes_out"]
     comp_ms = [s["last_step_compute_ms"] for s in st_run if s["steps_measured"] > 0]
     attn_ms_layer = float(np.mean(comp_ms)) / L if comp_ms else float("nan")
-    # attention + combine kernel per layer call, plus one swap kernel (or one table-patch kernel after copy-engine copies) per list
+    # attention + combine kernel per layer call, plus one swap kernel per list that took the kernel path and one table-patch
+    # kernel per copy-engine list of many id runs (lists of few runs patch the table by copy: no kernel)
     n_launch = int(2 * L * args.steps + (s_after["calls_kernel"] - s_before["calls_kernel"]) +
-                   (s_after["calls_copy_engine"] - s_before["calls_copy_engine"]))
+                   (s_after["reserved"][3] - s_before["reserved"][3]))
     # resident again right after (A/B/A): clocks drift under the power cap and the contexts keep growing, so the
     # slow-down is taken in GB/s against the mean of the resident runs on both sides
     pie.pie_set_extension_ratio(dw.pool, 0.0)

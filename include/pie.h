@@ -97,6 +97,8 @@ typedef struct pie_stats {
     int64_t steps_measured;
     double reserved[8];                    /* [0]: last step's attention slow-down vs the no-swap record, ms;
                                             * [2]: bytes of swap-out traffic elided so far (pie_set_retention);
+                                            * [3]: table-patch kernels launched after copy-engine lists (lists of few
+                                            *      id runs patch the table by copy and launch none);
                                             * [1]: the smallest extension ratio the GPU pool's size allows with the
                                             *      blocks allocated now (the controller never goes below it) */
 } pie_stats;

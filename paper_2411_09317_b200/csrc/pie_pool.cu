@@ -333,6 +333,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
             }
         } else if (slot_table_row) {
             PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_host + off, n, table_mode, stream));
+            p->stats.reserved[3] += 1;
         }
         p->stats.calls_copy_engine += 1;
     }
