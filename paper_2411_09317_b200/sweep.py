@@ -11,6 +11,7 @@ ratios:   the extension ratio is set to 0, 0.1, ... 1.0 (fraction of every layer
 adaptive: the controller owns the ratio.  --host-frac 0.5 (default): half of the blocks start host resident and the GPU
           pool holds only the other half, so the ratio has a floor; --host-frac 0: everything starts on the GPU and the
           ratio climbs from 0 until waits or slow-down appear.  Per step: ratio, floor, step time, wait share.
+layers:   whole layers on the CPU (the paper's protocol, Section 3.3) against the same share of every layer's blocks.
 interference: adaptive, with foreign pinned-memory traffic on the host link during the middle third of the run.
 Prints one JSON object per line.
 """
@@ -62,7 +63,8 @@ def attention_bytes(wl, ctx):
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="llama3_8b")
-    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive", "interference"])
+    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive", "interference", "layers"])
+    ap.add_argument("--cpu-layers", default="1,2,4", help="layers: numbers of layers kept on the CPU, comma list")
     ap.add_argument("--background-mb", type=int, default=256,
                     help="interference: pinned-memory traffic per step and direction on two other streams, MB")
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller pools)")
@@ -99,6 +101,9 @@ def main(argv=None):
             "both_per_dir": pie.pie_probe_link(256 << 20, 2, 3)}
     if args.mode == "interference":
         interference(args, wl, link, emit)
+        return
+    if args.mode == "layers":
+        layers_vs_blocks(args, wl, link, emit)
         return
     if args.mode == "ratios":
         ratios = [float(x) for x in args.ratios.split(",")] if args.ratios else [round(0.1 * i, 1) for i in range(11)]
@@ -153,6 +158,46 @@ def main(argv=None):
         emit({"summary": True, "final_ratio": sa["ratio"], "ratio_floor": sa["reserved"][1], "median_ms_per_step": float(np.median(per)),
               "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9, "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
               "attn_gbs": attention_bytes(wl, ctx0 + args.steps // 2) / (float(np.median(per)) * 1e-3) / 1e9})
+    dw.close()
+
+
+def layers_vs_blocks(args, wl, link, emit):
+    """The paper's unit against this build's: m whole layers live on the CPU and rotate through n - m GPU regions and
+    m + 2 CPU regions first in, first out (Section 3.3, pie_set_layer_policy) - against the same share m / n of every
+    layer's blocks (the block-granular plan at extension ratio m / n).  Same bytes per token either way."""
+    L = wl.n_layers
+    ms_list = [int(x) for x in args.cpu_layers.split(",")]
+    wl = dataclasses.replace(wl, decode_steps=len(ms_list) * 2 * (args.steps + 6) + 8)
+    _, _, nb = wl.tables()
+    m_max = max(ms_list)
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(2 * m_max + 6) * nb + 64)   # room for the change-over between the two plans
+    emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
+          "kv_gb": L * nb * wl.block_bytes / 1e9, "link": link})
+    ids = np.arange(nb, dtype=np.int32)
+    for m in ms_list:
+        # whole layers: the last m layers wholly onto the host, then the protocol takes over
+        pie.pie_set_extension_ratio(dw.pool, 0.0)
+        run_steps(dw, 2)                      # everything back on the GPU
+        for l in range(L - m, L):
+            pie.pie_swap_out(dw.pool, l, ids)
+        dw.sync()
+        pie.pie_set_layer_policy(dw.pool, L - m, m + 2)
+        run_steps(dw, 2)
+        per, sb, sa, ctx0, _ = run_steps(dw, args.steps)
+        tot = sum(per) * 1e-3
+        row = {"cpu_layers": m, "ratio": m / L, "whole_layers": {
+            "ms_per_step": float(np.median(per)), "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9,
+            "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
+            "gb_in_per_step": (sa["bytes_in"] - sb["bytes_in"]) / args.steps / 1e9}}
+        pie.pie_set_layer_policy(dw.pool, 0, 0)
+        pie.pie_set_extension_ratio(dw.pool, m / L)
+        run_steps(dw, 3)                      # the block plan redistributes: every layer keeps m / n of its blocks out
+        per, sb, sa, ctx0, _ = run_steps(dw, args.steps)
+        tot = sum(per) * 1e-3
+        row["blocks"] = {"ms_per_step": float(np.median(per)), "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9,
+                         "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
+                         "gb_in_per_step": (sa["bytes_in"] - sb["bytes_in"]) / args.steps / 1e9}
+        emit(row)
     dw.close()
 
 
