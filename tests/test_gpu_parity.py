@@ -427,6 +427,74 @@ def test_layer_by_layer_loop_with_other_work_in_between_equals_the_whole_step():
     assert np.array_equal(a[2], b[2]) and a[3] == b[3] > 0 and a[4] == b[4] > 0
 
 
+def test_kept_host_slots_are_given_back_when_units_leave_the_host_resident_set():
+    """Kept host copies hold host slots while their units are on the GPU.  When the ratio drops, the units that leave the
+    host-resident set must give those slots up: afterwards the whole host pool can be allocated again."""
+    from paper_2411_09317_b200.harness import DeviceWorkload
+    lens = synth.uniform_lengths(73, 5, 60, 200)
+    wl = synth.Workload("kept", 73, 3, 8, 4, 64, F16, lens, 12, 0.0)
+    _, _, nb = wl.tables(extra_tokens=12)
+    extra_ids = 8                                            # logical ids beyond the workload's, for the final allocation
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=2 * nb, extra_host_slots=3 * nb)
+    n_host = dw.n_host_slots
+    dw.set_retention(True)
+    pie.pie_set_extension_ratio(dw.pool, 0.5)
+    for _ in range(3):
+        dw.advance_context(); dw.decode_step()
+    dw.sync()
+    st = pie.pie_get_stats(dw.pool)
+    assert st["reserved"][2] > 0 and st["n_units_host"] > 0   # something was elided, something lives on the host
+    pie.pie_set_extension_ratio(dw.pool, 0.0)
+    for _ in range(3):
+        dw.advance_context(); dw.decode_step()
+    dw.sync()
+    st = pie.pie_get_stats(dw.pool)
+    assert st["n_units_host"] == 0
+    # every host slot is free again: swapping out as many units as the host pool has slots succeeds, one more does not
+    ids = np.arange(dw.NB, dtype=np.int32)
+    moved = 0
+    for l in range(wl.n_layers):
+        take = min(dw.NB, n_host - moved)
+        if take > 0:
+            pie.pie_swap_out(dw.pool, l, ids[:take])
+            moved += take
+    dw.sync()
+    assert moved == min(n_host, wl.n_layers * dw.NB)
+    assert pie.pie_get_stats(dw.pool)["n_units_host"] == moved
+    dw.close()
+
+
+def test_argument_checks_of_the_newer_entry_points():
+    case = Case(3, 8, 4, 64, F16, [40, 20], seed=77)
+    pc = PoolCase(case, n_gpu_slots=3 * case.NB + 4, n_host_slots=3 * case.NB)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_declare_append_blocks(pc.pool, [0, case.NB])
+    assert e.value.status == pie.PIE_ERR_RANGE
+    pie.pie_declare_append_blocks(pc.pool, [0, 1])
+    pie.pie_declare_append_blocks(pc.pool, None)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_kv_write(pc.pool, 7, pc.q.data_ptr(), pc.q.data_ptr(), pc.ctx.data_ptr(), pc.ctx.data_ptr(), 1, pc.bt.data_ptr(),
+                         case.block_table.shape[1], case.S)
+    assert e.value.status == pie.PIE_ERR_RANGE
+    pie.pie_kv_write(pc.pool, 0, None, None, None, None, 0, None, case.block_table.shape[1], case.S)   # nothing to write: fine
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_decode_layer(pc.pool, 3, pc.q[0].data_ptr(), pc.out[0].data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                             pc.ctx.data_ptr(), case.S, case.scale)
+    assert e.value.status == pie.PIE_ERR_RANGE
+    pie.pie_set_layer_policy(pc.pool, 3, 2)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_decode_layer(pc.pool, 0, pc.q[0].data_ptr(), pc.out[0].data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                             pc.ctx.data_ptr(), case.S, case.scale)
+    assert e.value.status == pie.PIE_ERR_UNSUPPORTED
+    pie.pie_set_layer_policy(pc.pool, 0, 0)
+    pie.pie_decode_layer(pc.pool, 0, pc.q[0].data_ptr(), pc.out[0].data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                         pc.ctx.data_ptr(), case.S, case.scale)
+    bits, got = pc.result(0)
+    want = oracle_attention(case, 0, "f32")
+    assert np.all(np.abs(got - want) <= edge_tol(want, case.dtype))
+    pc.close()
+
+
 # ---------------------------------------------------------------- prefill-side KV write
 @pytest.mark.parametrize("hq,hkv,d,dtype", [(8, 4, 64, F16), (8, 8, 128, BF16), (8, 1, 128, F16)])
 def test_kv_write_bit_exact_and_then_attention(hq, hkv, d, dtype):
