@@ -335,7 +335,10 @@ def main():
         c, sb, sa = timed_steps.ctx_before, timed_steps.before, timed_steps.after
         return {"ratio": r, "attn_gbs": median_gbs(bytes_of_steps(n, c), n), "attn_gbs_mean": bytes_of_steps(n, c) / (ms * 1e-3) / 1e9,
                 "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / (ms * 1e-3) / 1e9,
-                "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / (ms * 1e-3) / 1e9}
+                "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / (ms * 1e-3) / 1e9,
+                "lists_by_kernel": sa["calls_kernel"] - sb["calls_kernel"],
+                "lists_by_copy_engine": sa["calls_copy_engine"] - sb["calls_copy_engine"],
+                "wait_share_last_step": sa["last_step_stall_ms"] / max(sa["last_step_ms"], 1e-9)}
 
     def run_sweep(before):
         sweep, best = [], None

@@ -228,6 +228,13 @@ int pie_get_extension_ratio(pie_pool *pool, float *r);
  * the time-per-token record taken on steps without swap traffic (copies that are hidden can still slow the
  * attention down through shared HBM bandwidth). */
 int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
+/* Look-ahead depth of the decode loop (pie_decode_step / pie_decode_layer): while layer l computes, the host-resident
+ * shares of layers l+1 .. l+layers are on their way (wrapping into the next token).  1 is the paper's look-ahead
+ * (Section 3.4.2).  A deeper one gives each copy several layers' time to arrive - the copy stream then only has to
+ * keep up on average, not layer by layer - at the price of as many more layers' shares of GPU staging slots.
+ * 1 <= layers <= 8 (PIE_ERR_INVALID otherwise). */
+int pie_set_lookahead(pie_pool *pool, int32_t layers);
+
 /* ---- prefill-side KV write (Section 2.2: the prompt's keys and values enter the cache; the decode path above
  * appends one token per sequence, this call writes any number) ---------------------------------------------
  * k, v: device [n_tokens][n_kv_heads][head_dim] in the pool's 16-bit type.  Token t is position

@@ -19,14 +19,19 @@ overwritten before the copy reading it has finished, and a unit's bytes are neve
 destination before the copy writing them has finished.
 
 Slot hand-out order (shared rule, so that two implementations can be compared slot by slot):
-``ready`` is a queue that starts as 0 .. n-1; ``pending`` is a queue of released slots still
-waiting for their ticket.  At the start of every call pending slots whose ticket is confirmed
-move to the back of ``ready`` in queue order.  Allocation takes from the front of ``ready``
-first, then from the front of ``pending`` and reports the tickets to wait for.  (First in, first
-out on both keeps slots that were released together next to each other when they are handed out
-again, so lists of swapped blocks stay long runs of consecutive slots.)
+``ready`` holds the slots that are free for certain; ``pending`` is a queue of released slots still
+waiting for their ticket.  At the start of every call pending slots whose ticket is confirmed move to
+``ready``.  A request for n slots takes the first n of the lowest run of consecutive ready slots that
+has at least n; failing that, whole runs, longest first (lowest first among equals), until it is
+served; what ``ready`` cannot give comes from the front of ``pending``, and the tickets to wait for
+are reported.  (Lists of swapped blocks thus land in consecutive slots whenever the pool has room for
+that, however the set of free slots came about; a first-in-first-out hand-out keeps whatever order
+the slots were released in, and that order degrades once the host-resident sets change one block at
+a time.)
 """
 from __future__ import annotations
+
+import bisect
 
 FREE, GPU, TO_HOST, HOST, TO_GPU = 0, 1, 2, 3, 4
 STATE_NAMES = {FREE: "FREE", GPU: "GPU", TO_HOST: "TO_HOST", HOST: "HOST", TO_GPU: "TO_GPU"}
@@ -43,14 +48,17 @@ Q_NONE, Q_IN, Q_OUT, Q_COMPUTE = 0, 1, 2, 3
 
 class _SlotPool:
     def __init__(self, n):
-        self.ready = list(range(n))
+        self.ready = list(range(n))   # kept in ascending order
         self.pending = []  # (slot, queue, ticket)
+
+    def _add_ready(self, slot):
+        bisect.insort(self.ready, slot)
 
     def settle(self, done):
         keep = []
         for slot, qu, tk in self.pending:
             if tk <= done[qu]:
-                self.ready.append(slot)
+                self._add_ready(slot)
             else:
                 keep.append((slot, qu, tk))
         self.pending = keep
@@ -58,23 +66,42 @@ class _SlotPool:
     def available(self):
         return len(self.ready) + len(self.pending)
 
+    def _runs(self):
+        """maximal runs of consecutive ready slots -> [(start, length)] in ascending order"""
+        runs = []
+        for s in self.ready:
+            if runs and runs[-1][0] + runs[-1][1] == s:
+                runs[-1][1] += 1
+            else:
+                runs.append([s, 1])
+        return runs
+
     def take(self, n):
         """-> (slots, {queue: max ticket to wait for}, per-slot (queue, ticket) tags)"""
         slots, waits, tags = [], {}, []
-        for _ in range(n):
-            if self.ready:
-                slots.append(self.ready.pop(0))
-                tags.append((Q_NONE, 0))
+        while len(slots) < n and self.ready:
+            want = n - len(slots)
+            runs = self._runs()
+            fit = [r for r in runs if r[1] >= want]
+            if fit:
+                start, length = fit[0]                       # the lowest run that serves the rest of the request
             else:
-                slot, qu, tk = self.pending.pop(0)
-                slots.append(slot)
-                tags.append((qu, tk))
-                waits[qu] = max(waits.get(qu, 0), tk)
+                start, length = max(runs, key=lambda r: (r[1], -r[0]))   # else whole runs, longest first, lowest among equals
+            got = list(range(start, start + min(want, length)))
+            for s in got:
+                self.ready.remove(s)
+            slots += got
+            tags += [(Q_NONE, 0)] * len(got)
+        while len(slots) < n:
+            slot, qu, tk = self.pending.pop(0)
+            slots.append(slot)
+            tags.append((qu, tk))
+            waits[qu] = max(waits.get(qu, 0), tk)
         return slots, waits, tags
 
     def release(self, slot, queue, ticket):
         if queue == Q_NONE:
-            self.ready.append(slot)
+            self._add_ready(slot)
         else:
             self.pending.append((slot, queue, ticket))
 

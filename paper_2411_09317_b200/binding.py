@@ -36,7 +36,7 @@ EXPORTS = [
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
-    "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer",
+    "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead",
 ]
 
 
@@ -117,6 +117,7 @@ _sig = {
     "pie_table_mark_dirty": (_i32, [_vp, _i32, _vp, _i64]),
     "pie_table_drop_host_copy": (_i32, [_vp, _i32, _i32]),
     "pie_set_retention": (_i32, [_vp, _i32]),
+    "pie_set_lookahead": (_i32, [_vp, _i32]),
     "pie_decode_layer": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _i32, _f32, _vp, _vp, _i32]),
     "pie_kv_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i64, _vp, _i32, _i32]),
     "pie_declare_append_blocks": (_i32, [_vp, _vp, _i64]),
@@ -189,6 +190,10 @@ def pie_pool_destroy(pool) -> None:
 def pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs) -> None:
     check(lib.pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq,
                            n_seqs), "pie_kv_write")
+
+
+def pie_set_lookahead(pool, layers) -> None:
+    check(lib.pie_set_lookahead(pool, layers), "pie_set_lookahead")
 
 
 def pie_set_retention(pool, on) -> None:

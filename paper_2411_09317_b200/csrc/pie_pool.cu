@@ -21,6 +21,8 @@ constexpr int LIST_EVENTS = 512;   // events guarding regions of the id-list rin
 constexpr int TIMING_RING = 4;     // the host may enqueue at most this many steps ahead of their evaluation
 constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB ...
 constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list is at most this many runs
+constexpr int64_t AUTO_COPY_ENGINE_PIECE_BYTES = 256 << 10;  // ... or runs of this size, up to
+constexpr int64_t AUTO_COPY_ENGINE_MAX_PIECES = 32;          //     this many of them
 constexpr int64_t PATCH_DMA_MAX_RUNS = 16;               // table entries by small copies up to this many runs of ids, else a kernel
 
 #define PIE_CUDA(call)                                  \
@@ -82,7 +84,7 @@ struct pie_pool {
     uint64_t free_step_gap_ns = 0;   // smallest gap between two layers' attention kernels in the newest step without swaps
     uint64_t prev_step_end = 0;   // GPU-timer stamp of the end of the last layer of the newest evaluated step
     int64_t prev_step_id = -1;
-    bool prev_step_prefetched0 = false;  // that step issued a prefetch of layer 0 for the step after it
+    uint32_t prev_step_prefetched = 0;   // bit l: that step issued a swap-in list for layer l (l < 8)
     // attention
     pie::AttnScratch scratch{};
     CUtensorMap map3d{}, map2d{};
@@ -96,6 +98,7 @@ struct pie_pool {
     double ratio = 0.0;
     double ctrl_state[16] = {};
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
+    int32_t lookahead = 1;   // how many layers ahead the decode loop prefetches (Section 3.4.2 uses 1)
     bool poll_hold = false;  // a decode step is polling once per layer: nested calls skip theirs
     std::vector<int64_t> home_count;  // per layer: units whose home is the host
     std::vector<std::vector<int32_t>> home_list;  // per layer: ids the planner looks at (see candidate_ids)
@@ -265,9 +268,15 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         for (int64_t i = 1; i < n; ++i)
             if (src[i] != src[i - 1] + 1 || dst[i] != dst[i - 1] + 1) ++runs;
         // copy engine for long runs or few copies (no SM or L2 footprint next to attention); the kernel for scattered
-        // lists, where one cudaMemcpyAsync per block would be bound by the call rate (~5 us each)
-        mode = ((n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS) ? PIE_MODE_COPY_ENGINE
-                                                                                                   : PIE_MODE_KERNEL;
+        // lists of small pieces, where one cudaMemcpyAsync per piece would be bound by the call rate (~2-5 us each).
+        // Pieces of 256 KiB and more still move at most of the link's rate one by one, and host traffic issued by SMs
+        // disturbs a concurrent attention kernel several times more than the copy engine's: up to 32 such pieces per
+        // list go by copy engine too (slot lists get scattered when the host-resident sets change one block at a time).
+        const int64_t avg_run = (n * BB) / runs;
+        mode = (avg_run >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS ||
+                (avg_run >= AUTO_COPY_ENGINE_PIECE_BYTES && runs <= AUTO_COPY_ENGINE_MAX_PIECES))
+                   ? PIE_MODE_COPY_ENGINE
+                   : PIE_MODE_KERNEL;
     }
     // Table entries after copy-engine copies.  A patch kernel on a copy stream, launched while the persistent
     // attention grid owns the SMs, was measured to lengthen the gap between two attention launches, and it puts an
@@ -584,13 +593,15 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
 }
 
 // the host-resident set of `layer` follows the ratio: mark / unmark units in id order
-// The GPU pool must hold every layer's resident share plus two layers' host share in transit:
-// L (n - h) + 2 h <= n_gpu_slots bounds the host-resident count h of a layer from below.
+// The GPU pool must hold every layer's resident share plus the host shares in transit (the layer computing and the
+// `lookahead` layers being prefetched): L (n - h) + (1 + lookahead) h <= n_gpu_slots bounds the host-resident count h
+// of a layer from below.
 int64_t min_home_count(const pie_pool *p) {
     const int64_t n_alloc = p->table->n_allocated(), L = p->cfg.n_layers;
-    if (L <= 2) return 0;
+    const int64_t transit = 1 + std::min<int64_t>(p->lookahead, L - 1);  // this layer's share + the layers being prefetched
+    if (L <= transit) return 0;
     const int64_t deficit = L * n_alloc - p->cfg.n_gpu_slots;
-    return deficit > 0 ? std::min(n_alloc, (deficit + L - 3) / (L - 2)) : 0;
+    return deficit > 0 ? std::min(n_alloc, (deficit + L - transit - 1) / (L - transit)) : 0;
 }
 
 // the smallest extension ratio the GPU pool's size allows with the blocks allocated now
@@ -644,19 +655,14 @@ const std::vector<int32_t> &candidate_ids(pie_pool *p, int32_t layer) {
     return v;
 }
 
-int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::vector<int32_t> &out_ids) {
-    const int32_t L = p->cfg.n_layers;
-    const int32_t next = (layer + 1) % L;
+// the units of `target` that are still on the host, as many as the GPU pool can take: hottest first (Section 3.3)
+int plan_in(pie_pool *p, int32_t target, std::vector<int32_t> &in_ids) {
     in_ids.clear();
-    out_ids.clear();
-    p->table->layer_pass(layer);  // a resize in progress takes effect once every layer has been here (Section 4.1)
-    apply_ratio_to_layer(p, layer);
-    apply_ratio_to_layer(p, next);
-    // hottest first: the next layer's host-resident units, as many as the GPU pool can take
+    apply_ratio_to_layer(p, target);
     int64_t room = p->table->gpu_available();
     int64_t left_behind = 0;
-    for (int32_t b : candidate_ids(p, next)) {
-        const pie::Unit &u = p->table->unit(next, b);
+    for (int32_t b : candidate_ids(p, target)) {
+        const pie::Unit &u = p->table->unit(target, b);
         if (u.side == PIE_HOST) {
             if (room > 0) {
                 in_ids.push_back(b);
@@ -665,16 +671,27 @@ int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::ve
                 ++left_behind;
             }
         } else if (!u.home_host) {
-            p->home_dirty[(size_t)next] = 1;  // left the set and is back on the GPU: drop it at the next rebuild
-            p->table->drop_host_copy(next, b);
+            p->home_dirty[(size_t)target] = 1;  // left the set and is back on the GPU: drop it at the next rebuild
+            p->table->drop_host_copy(target, b);
         }
     }
-    // coldest: this layer's host-home units go back once it has computed
+    return left_behind == 0 ? PIE_OK : PIE_ERR_NOMEM;
+}
+
+// coldest: this layer's host-home units go back once it has computed
+void plan_out(pie_pool *p, int32_t layer, std::vector<int32_t> &out_ids) {
+    out_ids.clear();
+    p->table->layer_pass(layer);  // a resize in progress takes effect once every layer has been here (Section 4.1)
+    apply_ratio_to_layer(p, layer);
     for (int32_t b : candidate_ids(p, layer)) {
         const pie::Unit &u = p->table->unit(layer, b);
         if (u.home_host && u.side == PIE_GPU) out_ids.push_back(b);
     }
-    return left_behind == 0 ? PIE_OK : PIE_ERR_NOMEM;
+}
+
+int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::vector<int32_t> &out_ids) {
+    plan_out(p, layer, out_ids);
+    return plan_in(p, (layer + 1) % p->cfg.n_layers, in_ids);
 }
 
 int ensure_stage(pie_pool *p, int32_t n_seqs, int32_t max_blocks) {
@@ -1094,9 +1111,9 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     for (size_t l = 0; l < L; ++l) {
         const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
         if (!ev[l].has_compute || !S || !E || E < S) continue;
-        // units were brought in for this layer: by a list of this step for layers >= 1, by the previous step's
-        // look-ahead across the token boundary for layer 0
-        const bool fetched = l > 0 ? ev[l].has_in : (chained && pool->prev_step_prefetched0);
+        // units were brought in for this layer: by a list of this step, or - for the first layers - by the previous
+        // step's look-ahead across the token boundary
+        const bool fetched = ev[l].has_in || (chained && l < 8 && ((pool->prev_step_prefetched >> l) & 1u));
         double layer_stall = 0.0;
         if (fetched && prev_end && S > prev_end + usual_gap) layer_stall = (double)(S - prev_end - usual_gap) * 1e-6;
         stall += layer_stall;
@@ -1114,7 +1131,9 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     if (last) {
         pool->prev_step_end = last;
         pool->prev_step_id = pool->lev_step[k];
-        pool->prev_step_prefetched0 = L > 1 && ev[0].has_in;
+        pool->prev_step_prefetched = 0;   // lists this step issued for the first layers: they serve the next step
+        for (size_t l = 0; l < std::min<size_t>(8, L); ++l)
+            if (L > 1 && ev[l].has_in) pool->prev_step_prefetched |= 1u << l;
     }
     pool->lev_done[k] = true;
     if (first && pool->cfg.timing >= 2) {
@@ -1288,6 +1307,12 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
     st = record_ticket(pool, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) pool->sticky = st;
     return st;
+}
+
+int pie_set_lookahead(pie_pool *pool, int32_t layers) {
+    if (!pool || layers < 1 || layers > 8) return PIE_ERR_INVALID;
+    pool->lookahead = layers;
+    return PIE_OK;
 }
 
 int pie_set_retention(pie_pool *pool, int32_t on) {
@@ -1539,11 +1564,18 @@ static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, con
         }
     }
     std::vector<int32_t> &in_ids = pool->v_plan_in, &out_ids = pool->v_plan_out;
-    int st = plan_layer(pool, l, in_ids, out_ids);
-    if (st != PIE_OK) return st;  // the GPU pool cannot take the next layer's share: nothing was enqueued for it
-    if (L > 1 && !in_ids.empty()) {
-        // starts when layer l starts, i.e. once the previous attention call has finished
-        st = pool_swap(pool, PIE_Q_IN, (l + 1) % L, in_ids.data(), (int64_t)in_ids.size(), mode, pool->table->issued(PIE_Q_COMPUTE));
+    plan_out(pool, l, out_ids);
+    // prefetch: the layers up to `lookahead` ahead (wrapping into the next token) that still have units on the host;
+    // in a steady loop only the farthest one does.  The copies start when layer l starts, i.e. once the previous
+    // attention call has finished, and run back to back on the copy-in stream.
+    int st = PIE_OK;
+    const int64_t start_with = pool->table->issued(PIE_Q_COMPUTE);
+    for (int32_t d = 1; d <= std::min(pool->lookahead, L - 1); ++d) {
+        const int32_t target = (l + d) % L;
+        st = plan_in(pool, target, in_ids);
+        if (st != PIE_OK) return st;  // the GPU pool cannot take that layer's share: nothing was enqueued for it
+        if (in_ids.empty()) continue;
+        st = pool_swap(pool, PIE_Q_IN, target, in_ids.data(), (int64_t)in_ids.size(), mode, start_with);
         if (st != PIE_OK) return st;
     }
     st = attention_call(pool, l, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,

@@ -10,7 +10,34 @@ namespace pie {
 
 // ------------------------------------------------------------------------------------ SlotPool
 SlotPool::SlotPool(int64_t n) {
-    for (int64_t s = 0; s < n; ++s) ready_.push_back((int32_t)s);
+    if (n > 0) runs_[0] = (int32_t)n;
+    n_ready_ = n;
+}
+
+void SlotPool::add_ready(int32_t slot) {
+    auto next = runs_.lower_bound(slot);
+    bool joined = false;
+    if (next != runs_.begin()) {
+        auto prev = std::prev(next);
+        if (prev->first + prev->second == slot) {  // extends the run before it
+            prev->second += 1;
+            joined = true;
+            if (next != runs_.end() && next->first == slot + 1) {  // ... and closes the gap to the run after it
+                prev->second += next->second;
+                runs_.erase(next);
+            }
+        }
+    }
+    if (!joined) {
+        if (next != runs_.end() && next->first == slot + 1) {  // extends the run after it downwards
+            const int32_t len = next->second + 1;
+            runs_.erase(next);
+            runs_[slot] = len;
+        } else {
+            runs_[slot] = 1;
+        }
+    }
+    ++n_ready_;
 }
 
 void SlotPool::settle(const int64_t *done) {
@@ -18,29 +45,49 @@ void SlotPool::settle(const int64_t *done) {
     size_t keep = 0;
     for (size_t i = 0; i < pending_.size(); ++i) {
         const Pending p = pending_[i];
-        if (p.ticket <= done[p.queue]) ready_.push_back(p.slot);
+        if (p.ticket <= done[p.queue]) add_ready(p.slot);
         else pending_[keep++] = p;
     }
     pending_.resize(keep);
 }
 
-int32_t SlotPool::take(SlotTag *tag) {
-    if (!ready_.empty()) {
-        int32_t s = ready_.front();
-        ready_.pop_front();
-        tag->queue = PIE_Q_NONE;
-        tag->ticket = 0;
-        return s;
+void SlotPool::take_n(int64_t n, int32_t *slots, SlotTag *tags) {
+    int64_t k = 0;
+    while (k < n && !runs_.empty()) {
+        const int64_t want = n - k;
+        auto pick = runs_.end(), longest = runs_.begin();
+        for (auto it = runs_.begin(); it != runs_.end(); ++it) {
+            if (it->second >= want) {
+                pick = it;  // the lowest run that serves the rest of the request
+                break;
+            }
+            if (it->second > longest->second) longest = it;
+        }
+        if (pick == runs_.end()) pick = longest;
+        const int32_t start = pick->first, len = pick->second;
+        const int32_t m = (int32_t)std::min<int64_t>(want, len);
+        for (int32_t i = 0; i < m; ++i) {
+            slots[k] = start + i;
+            tags[k].queue = PIE_Q_NONE;
+            tags[k].ticket = 0;
+            ++k;
+        }
+        runs_.erase(pick);
+        if (m < len) runs_[start + m] = len - m;
+        n_ready_ -= m;
     }
-    Pending p = pending_.front();
-    pending_.pop_front();
-    tag->queue = p.queue;
-    tag->ticket = p.ticket;
-    return p.slot;
+    while (k < n) {
+        Pending p = pending_.front();
+        pending_.pop_front();
+        slots[k] = p.slot;
+        tags[k].queue = p.queue;
+        tags[k].ticket = p.ticket;
+        ++k;
+    }
 }
 
 void SlotPool::release(int32_t slot, int32_t queue, int64_t ticket) {
-    if (queue == PIE_Q_NONE) ready_.push_back(slot);
+    if (queue == PIE_Q_NONE) add_ready(slot);
     else pending_.push_back({slot, queue, ticket});
 }
 
@@ -133,17 +180,31 @@ int Table::alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host) 
         need_host += L - n_gpu[(size_t)i];
     }
     if (need_host > host_.available()) return PIE_ERR_NOMEM;
-    for (int32_t l = 0; l < L; ++l)
+    std::vector<int32_t> host_slots;
+    std::vector<SlotTag> host_tags;
+    for (int32_t l = 0; l < L; ++l) {
+        // one request per layer and side: a layer's units sit in consecutive slots where the pools allow
+        int64_t want_gpu = 0;
+        for (int64_t i = 0; i < n; ++i) want_gpu += l < n_gpu[(size_t)i];
+        take_slots_.resize((size_t)want_gpu);
+        take_tags_.resize((size_t)want_gpu);
+        host_slots.resize((size_t)(n - want_gpu));
+        host_tags.resize((size_t)(n - want_gpu));
+        if (want_gpu > 0) gpu_.take_n(want_gpu, take_slots_.data(), take_tags_.data());
+        if (n - want_gpu > 0) host_.take_n(n - want_gpu, host_slots.data(), host_tags.data());
+        int64_t ig = 0, ih = 0;
         for (int64_t i = 0; i < n; ++i) {
             Unit &u = unit(l, blocks[i]);
             SlotTag tag;
             if (l < n_gpu[(size_t)i]) {
-                u.gpu_slot = gpu_.take(&tag);
+                tag = take_tags_[(size_t)ig];
+                u.gpu_slot = take_slots_[(size_t)ig++];
                 u.host_slot = -1;
                 u.side = PIE_GPU;
                 u.home_host = 0;
             } else {
-                u.host_slot = host_.take(&tag);
+                tag = host_tags[(size_t)ih];
+                u.host_slot = host_slots[(size_t)ih++];
                 u.gpu_slot = -1;
                 u.side = PIE_HOST;
                 u.home_host = 1;
@@ -156,6 +217,7 @@ int Table::alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host) 
             }
             u.t_stamp = clock_;
         }
+    }
     for (int64_t i = 0; i < n; ++i) allocated_[blocks[i]] = 1;
     n_allocated_ += (int32_t)n;
     return PIE_OK;
@@ -251,15 +313,19 @@ int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int
     if (movers == 0) return PIE_OK;
     const int64_t tk = ++issued_[queue];
     ++clock_;
-    int64_t k = 0;
+    // the new slots of the whole list in one request, so that they are consecutive where the pool allows
+    take_slots_.resize((size_t)need);
+    take_tags_.resize((size_t)need);
+    if (need > 0) dst_pool.take_n(need, take_slots_.data(), take_tags_.data());
+    int64_t k = 0, taken = 0;
     for (int64_t i = 0; i < n; ++i) {
         Unit &u = unit(layer, ids[i]);
         if (u.side == want) continue;
         const bool kept = queue == PIE_Q_OUT && u.host_slot >= 0;
         int32_t d = u.host_slot;
         if (!kept) {
-            SlotTag tag;
-            d = dst_pool.take(&tag);
+            const SlotTag tag = take_tags_[(size_t)taken];
+            d = take_slots_[(size_t)taken++];
             if (tag.queue != PIE_Q_NONE) waits[tag.queue] = std::max(waits[tag.queue], tag.ticket);
         }
         // the copy that is still bringing the unit to where it is now

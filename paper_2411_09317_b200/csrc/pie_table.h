@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cstdint>
 #include <deque>
+#include <map>
 #include <vector>
 
 #include "../../include/pie.h"
@@ -15,16 +16,25 @@ struct SlotTag {
     int64_t ticket;
 };
 
-// Free slots of one pool.  `ready` is a queue (0 .. n-1 at start); `pending` is a queue of slots
-// released by a copy that may not have finished: they can be handed out, but the receiver must wait
-// for the tag's ticket.  First in, first out on both: slots released together are handed out together
-// again, so swap lists stay long runs of consecutive slots (few, large copies).
+// Free slots of one pool.  `ready` holds slots that are free for certain, as runs of consecutive numbers; `pending`
+// is a queue of slots released by a copy that may not have finished: they can be handed out, but the receiver must
+// wait for the tag's ticket.  Hand-out rule (shared with the oracle, so that the two can be compared slot by slot):
+// a request for n slots takes the first n of the lowest ready run that has at least n; failing that, whole runs,
+// longest first (lowest first among equals), until it is served; what ready cannot give comes from the front of
+// pending.  Lists of swapped blocks thus land in consecutive slots whenever the pool has room for that, however the
+// set of free slots came about - which is what lets a few large copies move them.
 class SlotPool {
   public:
     explicit SlotPool(int64_t n);
     void settle(const int64_t *done);
-    int64_t available() const { return (int64_t)ready_.size() + (int64_t)pending_.size(); }
-    int32_t take(SlotTag *tag);
+    int64_t available() const { return n_ready_ + (int64_t)pending_.size(); }
+    // n slots into slots[0..n), their tags into tags[0..n); the caller has checked available() >= n
+    void take_n(int64_t n, int32_t *slots, SlotTag *tags);
+    int32_t take(SlotTag *tag) {
+        int32_t s;
+        take_n(1, &s, tag);
+        return s;
+    }
     void release(int32_t slot, int32_t queue, int64_t ticket);
 
   private:
@@ -33,7 +43,9 @@ class SlotPool {
         int32_t queue;
         int64_t ticket;
     };
-    std::deque<int32_t> ready_;
+    void add_ready(int32_t slot);
+    std::map<int32_t, int32_t> runs_;  // start -> length of a run of ready slots
+    int64_t n_ready_ = 0;
     std::deque<Pending> pending_;
 };
 
@@ -117,6 +129,8 @@ class Table {
     int32_t capacity_, target_ = -1, n_moved_ = 0;
     bool retain_ = false;
     std::vector<uint8_t> moved_;  // per layer
+    std::vector<int32_t> take_slots_;  // scratch of swap() / alloc_bulk()
+    std::vector<SlotTag> take_tags_;
 };
 
 // Whole-layer protocol of Section 3.3.

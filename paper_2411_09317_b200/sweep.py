@@ -78,6 +78,7 @@ def main(argv=None):
                     help="ratios / adaptive: after every layer's attention, an elementwise kernel that reads and writes this many MB "
                          "on the compute stream stands in for the model's projections and MLP (weights streamed from HBM); the "
                          "step then runs layer by layer through pie_decode_layer")
+    ap.add_argument("--lookahead", type=int, default=1, help="layers prefetched ahead (pie_set_lookahead)")
     ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
@@ -114,8 +115,10 @@ def main(argv=None):
         dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(L + 3) * nb + 64,
                             split_tokens=args.split)
         dw.set_retention(args.kept_copies)
+        pie.pie_set_lookahead(dw.pool, args.lookahead)
         emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
               "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "other_mb_per_layer": args.other_mb,
+              "lookahead": args.lookahead,
               "link": link})
         for r in ratios:
             pie.pie_set_extension_ratio(dw.pool, r)

@@ -304,8 +304,9 @@ def test_large_batch_uses_the_separate_plan_kernel():
     pc.close()
 
 
-@pytest.mark.parametrize("retention", ["off", "declared", "undeclared", "host_tables"])
-def test_multi_step_decode_with_append_matches_oracle_every_step(retention):
+@pytest.mark.parametrize("retention,lookahead", [("off", 1), ("declared", 1), ("undeclared", 1), ("host_tables", 1), ("off", 2),
+                                                 ("declared", 3)])
+def test_multi_step_decode_with_append_matches_oracle_every_step(retention, lookahead):
     """Five decode steps on a small GQA model, 40 % of the blocks host resident: outputs of every step and the final
     bytes of every unit against the oracle (append, prefetch, write-back, next-token look-ahead).  With kept host
     copies, write-backs of blocks the step did not write are skipped: the bytes must come out the same, with the
@@ -314,9 +315,11 @@ def test_multi_step_decode_with_append_matches_oracle_every_step(retention):
     lens = np.array([30, 63, 64, 65, 129, 7], dtype=np.int32)
     steps = 5
     case = Case(3, 8, 2, 128, BF16, lens, seed=42, host_frac=0.4, placement="random", extra_tokens=steps)
-    pc = PoolCase(case, timing=1)
+    nh = len(case.host_ids)                                       # staging: the computing layer's share + the look-ahead's
+    pc = PoolCase(case, timing=1, n_gpu_slots=case.L * (case.NB - nh) + (lookahead + 2) * nh + 2)
     if retention != "off":
         pie.pie_set_retention(pc.pool, 1)
+    pie.pie_set_lookahead(pc.pool, lookahead)      # deeper look-ahead: more layers' shares in flight, same bytes and results
     dev = torch.device("cuda:0")
     cur = lens.copy()
     ctx_dev = torch.from_numpy(cur).to(dev)

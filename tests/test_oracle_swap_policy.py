@@ -249,7 +249,30 @@ def test_kept_host_copy_is_reused_and_written_blocks_are_copied():
     st, tk, pairs, _ = t2.swap(table.Q_IN, 0, [0]); t2.confirm(table.Q_IN, tk)
     assert t2.host_slot[0] == -1
     st, tk, pairs, _ = t2.swap(table.Q_OUT, 0, [0])
-    assert t2.last_elided == [False] and pairs[0][2] == 1                              # FIFO: the other host slot
+    assert t2.last_elided == [False] and pairs[0][2] == 0 and t2.host_slot[0] == 0     # a slot from the pool (the lowest free run)
+
+
+def test_slot_hand_out_prefers_runs_of_consecutive_slots():
+    """The shared hand-out rule by hand: the lowest run that serves the request; else whole runs, longest first; pending
+    slots (with their tickets) only when nothing else is left."""
+    p = table._SlotPool(10)
+    assert p.take(3)[0] == [0, 1, 2]
+    assert p.take(1)[0] == [3]
+    p.release(1, table.Q_NONE, 0)                      # ready: {1} and {4..9}
+    assert p.take(2)[0] == [4, 5]                      # the single slot cannot serve two: the next run does, and 1 stays
+    assert p.take(1)[0] == [1]
+    for s in (0, 2):                                   # ready: {0}, {2}, {6..9}
+        p.release(s, table.Q_NONE, 0)
+    p.release(3, table.Q_OUT, 7)                       # pending behind out-ticket 7
+    slots, waits, tags = p.take(7)                     # no run of 7: the longest first, then the lowest, then pending
+    assert slots == [6, 7, 8, 9, 0, 2, 3] and waits == {table.Q_OUT: 7} and tags[-1] == (table.Q_OUT, 7)
+    assert p.available() == 0
+    # a pool whose free set was scrambled one slot at a time still serves a list from one run if it has one
+    q = table._SlotPool(64)
+    q.take(64)
+    for s in (5, 40, 41, 42, 43, 9, 44, 45, 13, 46, 47):
+        q.release(s, table.Q_NONE, 0)
+    assert q.take(6)[0] == [40, 41, 42, 43, 44, 45]
 
 
 def test_table_error_codes_and_two_phase_states():
