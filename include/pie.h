@@ -141,10 +141,11 @@ int pie_get_placement(pie_pool *pool, int32_t *side, int32_t *slot);
  * known complete (observed with cudaEventQuery at any later call) the units read PIE_HOST.
  * Blocks already on, or heading to, the host are skipped.  block_ids: host, n entries, distinct.
  * mode: PIE_MODE_KERNEL = gather/scatter kernel, PIE_MODE_COPY_ENGINE = one cudaMemcpyAsync per run of
- * consecutive slots, PIE_MODE_AUTO = copy engine when the list is at most 8 runs or its runs average 1 MiB,
- * else the kernel (measured: the copy engine reaches the link rate from ~16 MB and disturbs a concurrent
- * attention kernel several times less than SM-issued host traffic, but one call per scattered 64 KiB block
- * tops out near 12 GB/s). */
+ * consecutive slots, PIE_MODE_AUTO = copy engine when the list is at most 8 runs, or its runs average 1 MiB, or it
+ * is at most 32 runs averaging 256 KiB, else the kernel (measured: the copy engine reaches the link rate from
+ * ~16 MB and disturbs a concurrent attention kernel several times less than SM-issued host traffic, but one call
+ * per scattered 64 KiB block tops out near 12 GB/s).  The slot table follows the data in stream order: written by
+ * the kernel, or by one small copy per run of consecutive block ids (a patch kernel beyond 16 such runs). */
 int pie_swap_out(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode);
 /* The mirror image on the copy-in stream.  The layer's next pie_decode_attention waits for it
  * (Section 3.2: presence check). */
