@@ -258,7 +258,7 @@ def main():
     sweep_ratios = [0.0005, 0.001, 0.002, 0.004, 0.006, 0.008]
     n_sweep = 8
     # every phase below appends one token per step
-    total_steps = (4 + args.steps) + (ramp + 2 + args.steps) + (4 + args.steps) + 2 * len(sweep_ratios) * 2 * (5 + n_sweep) + (3 + args.steps) + 8
+    total_steps = (4 + args.steps) + (ramp + 2 + args.steps) + (4 + args.steps) + 2 * len(sweep_ratios) * 2 * (5 + n_sweep) + (8 + args.steps) + 8
     n_blocks = int(((wl.ctx_lens.astype(np.int64) + total_steps + 15) // 16).sum())
     r_cap = 0.02   # room in both pools for host-resident shares up to this ratio (+ 3 layers of staging)
     dw = DeviceWorkload(wl, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
@@ -367,7 +367,7 @@ def main():
     hidden["note"] = ("slow-downs compare median steps (GB/s) with the mean of the resident runs measured right before and "
                       "right after; attn_gbs_mean is the plain total over the same steps")
 
-    pie.pie_set_extension_ratio(dw.pool, float(hidden["ratio"]))   # e2e runs at the ratio the controller chose
+    pie.pie_set_extension_ratio(dw.pool, -1.0)   # e2e runs like the headline region: the controller owns the ratio
     # ---- e2e: the same step through the host-buffer entry point (inputs H2D, outputs D2H inside the region) -----
     q_h = torch.empty(dw.q_all.shape, dtype=torch.int16).pin_memory()
     k_h = torch.empty(dw.k_new.shape, dtype=torch.int16).pin_memory()
@@ -385,9 +385,10 @@ def main():
         pie.pie_decode_step_host(dw.pool, q_h.data_ptr(), o_h.data_ptr(), dw.block_table, dw.max_blocks, dw.ctx_lens,
                                  wl.n_seqs, dw.scale, k_h.data_ptr(), v_h.data_ptr())
 
-    for _ in range(3):
+    for _ in range(8):
         host_step()
     c0 = dw.ctx_lens.copy()
+    e2e_before = pie.pie_get_stats(dw.pool)
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
@@ -395,6 +396,8 @@ def main():
     dw.sync()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
     e2e_value = bytes_of_steps(args.steps, c0) / (e2e_ms * 1e-3) / 1e9
+    e2e_after = pie.pie_get_stats(dw.pool)
+    e2e_swap_gbs = (e2e_after["bytes_in"] - e2e_before["bytes_in"]) / (e2e_ms * 1e-3) / 1e9
 
     # ---- as configured: a seeded 30 % of every sequence's blocks host resident (link-bound by construction) --------
     dw.close()
@@ -456,7 +459,8 @@ def main():
                        f"({bytes_layer0 / 1e9:.2f} GB of distinct KV per layer call)", "parallelism": "replicas only"},
             "clocks": clocks,
             "e2e": {"value": e2e_value * world, "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "ms_per_step": e2e_ms / args.steps},
+                    "ms_per_step": e2e_ms / args.steps, "swap_in_gbs": e2e_swap_gbs, "ratio_at_end": e2e_after["ratio"],
+                    "note": "pie_decode_step_host with pinned host buffers, adaptive controller running as in the headline region"},
             "roofline": roofline, "cpu_baseline": cpu,
             "hidden_swap": hidden, "resident": {"attn_gbs": resident_gbs, "attn_gbs_after": resident_after_gbs,
                                                 "attn_gbs_median_step": resident_med,

@@ -196,7 +196,9 @@ int pie_decode_layer(pie_pool *pool, int32_t layer, const void *q, void *out, co
                      int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new,
                      const void *v_new, int32_t mode);
 /* The same with q / k_new / v_new / out in HOST memory (pinned for full speed): copies the inputs in,
- * runs the step, copies out_all back and waits for it.  ctx_lens_host/block_table_host are uploaded too. */
+ * runs the step, copies out_all back and waits for it.  ctx_lens_host/block_table_host are uploaded too.
+ * Inputs and results move in groups of four layers on two streams of the library's own, so that a group's
+ * upload and download overlap the other groups' attention; when the call returns nothing is in flight. */
 int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_host, const int32_t *block_table_host,
                          int32_t max_blocks_per_seq, const int32_t *ctx_lens_host, int32_t n_seqs, float scale,
                          const void *k_new_all_host, const void *v_new_all_host, int32_t mode);

@@ -23,6 +23,7 @@ constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine wh
 constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list is at most this many runs
 constexpr int64_t AUTO_COPY_ENGINE_PIECE_BYTES = 256 << 10;  // ... or runs of this size, up to
 constexpr int64_t AUTO_COPY_ENGINE_MAX_PIECES = 32;          //     this many of them
+constexpr int IO_GROUP_LAYERS = 4;   // pie_decode_step_host moves inputs and results in groups of this many layers
 constexpr int64_t PATCH_DMA_MAX_RUNS = 16;               // table entries by small copies up to this many runs of ids, else a kernel
 
 #define PIE_CUDA(call)                                  \
@@ -122,6 +123,8 @@ struct pie_pool {
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
     std::vector<uint8_t> v_elide;
+    cudaStream_t io_stream[2] = {nullptr, nullptr};  // pie_decode_step_host: inputs up / results down
+    std::vector<cudaEvent_t> io_up;                   // one per group of layers: its inputs have arrived
     std::vector<int32_t> v_plan_in, v_plan_out;  // one layer's plan inside the decode loop
     std::vector<int32_t> append_ids;  // blocks the coming appends write (pie_declare_append_blocks)
     bool append_declared = false;
@@ -473,6 +476,10 @@ void destroy_pool(pie_pool *p) {
                 if (ev) cudaEventDestroy(ev);
     for (int k = 0; k < TIMING_RING; ++k)
         if (p->lev_anchor[k]) cudaEventDestroy(p->lev_anchor[k]);
+    for (cudaEvent_t ev : p->io_up)
+        if (ev) cudaEventDestroy(ev);
+    for (int i = 0; i < 2; ++i)
+        if (p->io_stream[i]) cudaStreamDestroy(p->io_stream[i]);
     if (p->own_streams)
         for (int q = 1; q <= 3; ++q)
             if (p->stream[q]) cudaStreamDestroy(p->stream[q]);
@@ -692,6 +699,17 @@ void plan_out(pie_pool *p, int32_t layer, std::vector<int32_t> &out_ids) {
 int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::vector<int32_t> &out_ids) {
     plan_out(p, layer, out_ids);
     return plan_in(p, (layer + 1) % p->cfg.n_layers, in_ids);
+}
+
+// streams and events of the host-buffer entry point's pipeline (created at its first use)
+int ensure_io(pie_pool *p) {
+    if (p->io_stream[0]) return PIE_OK;
+    PIE_CUDA(cudaStreamCreateWithFlags(&p->io_stream[0], cudaStreamNonBlocking));
+    PIE_CUDA(cudaStreamCreateWithFlags(&p->io_stream[1], cudaStreamNonBlocking));
+    const int n_groups = (p->cfg.n_layers + IO_GROUP_LAYERS - 1) / IO_GROUP_LAYERS;
+    p->io_up.assign((size_t)n_groups, nullptr);
+    for (cudaEvent_t &ev : p->io_up) PIE_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    return PIE_OK;
 }
 
 int ensure_stage(pie_pool *p, int32_t n_seqs, int32_t max_blocks) {
@@ -1631,34 +1649,93 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
     int st = ensure_stage(pool, n_seqs, max_blocks_per_seq);
     if (st != PIE_OK) return st;
     cudaStream_t s = pool->stream[PIE_Q_COMPUTE];
-    const int64_t qb = (int64_t)pool->cfg.n_layers * n_seqs * pool->cfg.n_q_heads * pool->cfg.head_dim * 2;
-    const int64_t kb = (int64_t)pool->cfg.n_layers * n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;
-    PIE_CUDA(cudaMemcpyAsync(pool->stage_q, q_all_host, (size_t)qb, cudaMemcpyHostToDevice, s));
-    if (k_new_all_host) {
-        PIE_CUDA(cudaMemcpyAsync(pool->stage_k, k_new_all_host, (size_t)kb, cudaMemcpyHostToDevice, s));
-        PIE_CUDA(cudaMemcpyAsync(pool->stage_v, v_new_all_host, (size_t)kb, cudaMemcpyHostToDevice, s));
-    }
-    PIE_CUDA(cudaMemcpyAsync(pool->stage_bt, block_table_host, (size_t)n_seqs * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, s));
-    PIE_CUDA(cudaMemcpyAsync(pool->stage_ctx, ctx_lens_host, (size_t)n_seqs * 4, cudaMemcpyHostToDevice, s));
+    const int32_t L = pool->cfg.n_layers;
+    const int64_t q_layer = (int64_t)n_seqs * pool->cfg.n_q_heads * pool->cfg.head_dim * 2;
+    const int64_t kv_layer = (int64_t)n_seqs * pool->cfg.n_kv_heads * pool->cfg.head_dim * 2;
+    const int64_t qb = L * q_layer, kb = L * kv_layer;
     // the host tables say which block of each sequence the append writes: kept host copies of the others stay good
-    std::vector<int32_t> saved_ids;
-    const bool saved_declared = pool->append_declared;
+    struct AppendGuard {
+        pie_pool *p;
+        std::vector<int32_t> saved;
+        bool declared, active = false;
+        ~AppendGuard() {
+            if (!active) return;
+            p->append_ids.swap(saved);
+            p->append_declared = declared;
+        }
+    } guard{pool, {}, pool->append_declared};
     if (k_new_all_host && pool->table->retain()) {
-        saved_ids.swap(pool->append_ids);
+        guard.saved.swap(pool->append_ids);
+        guard.active = true;
         for (int32_t sq = 0; sq < n_seqs; ++sq)
             if (ctx_lens_host[sq] > 0 && ctx_lens_host[sq] <= max_blocks_per_seq * 16)
                 pool->append_ids.push_back(block_table_host[(int64_t)sq * max_blocks_per_seq + (ctx_lens_host[sq] - 1) / 16]);
         pool->append_declared = true;
     }
-    st = pie_decode_step(pool, pool->stage_q, pool->stage_out, pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
-                         k_new_all_host ? pool->stage_k : nullptr, k_new_all_host ? pool->stage_v : nullptr, mode);
-    if (k_new_all_host && pool->table->retain()) {
-        pool->append_ids.swap(saved_ids);
-        pool->append_declared = saved_declared;
+    PIE_CUDA(cudaMemcpyAsync(pool->stage_bt, block_table_host, (size_t)n_seqs * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, s));
+    PIE_CUDA(cudaMemcpyAsync(pool->stage_ctx, ctx_lens_host, (size_t)n_seqs * 4, cudaMemcpyHostToDevice, s));
+    if (pool->fifo) {
+        // whole-layer protocol: the step is driven as a whole; inputs go up first, results come down last
+        PIE_CUDA(cudaMemcpyAsync(pool->stage_q, q_all_host, (size_t)qb, cudaMemcpyHostToDevice, s));
+        if (k_new_all_host) {
+            PIE_CUDA(cudaMemcpyAsync(pool->stage_k, k_new_all_host, (size_t)kb, cudaMemcpyHostToDevice, s));
+            PIE_CUDA(cudaMemcpyAsync(pool->stage_v, v_new_all_host, (size_t)kb, cudaMemcpyHostToDevice, s));
+        }
+        st = pie_decode_step(pool, pool->stage_q, pool->stage_out, pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs,
+                             scale, k_new_all_host ? pool->stage_k : nullptr, k_new_all_host ? pool->stage_v : nullptr, mode);
+        if (st != PIE_OK) return st;
+        PIE_CUDA(cudaMemcpyAsync(out_all_host, pool->stage_out, (size_t)qb, cudaMemcpyDeviceToHost, s));
+        PIE_CUDA(cudaStreamSynchronize(s));
+        return check_status_word(pool);
     }
+    // Pipelined by groups of layers on two streams of their own (not the swap streams: a prefetch must not queue
+    // behind an upload): a group's inputs go up while the groups before it compute, its results come down while the
+    // groups after it compute.  The previous call ended with a synchronisation, so the staging buffers are free.
+    st = ensure_io(pool);
     if (st != PIE_OK) return st;
-    PIE_CUDA(cudaMemcpyAsync(out_all_host, pool->stage_out, (size_t)qb, cudaMemcpyDeviceToHost, s));
-    PIE_CUDA(cudaStreamSynchronize(s));
+    const int32_t G = IO_GROUP_LAYERS, n_groups = (L + G - 1) / G;
+    for (int32_t g = 0; g < n_groups; ++g) {
+        const int32_t l0 = g * G, nl = std::min(G, L - l0);
+        PIE_CUDA(cudaMemcpyAsync((uint8_t *)pool->stage_q + l0 * q_layer, (const uint8_t *)q_all_host + l0 * q_layer,
+                                 (size_t)(nl * q_layer), cudaMemcpyHostToDevice, pool->io_stream[0]));
+        if (k_new_all_host) {
+            PIE_CUDA(cudaMemcpyAsync((uint8_t *)pool->stage_k + l0 * kv_layer, (const uint8_t *)k_new_all_host + l0 * kv_layer,
+                                     (size_t)(nl * kv_layer), cudaMemcpyHostToDevice, pool->io_stream[0]));
+            PIE_CUDA(cudaMemcpyAsync((uint8_t *)pool->stage_v + l0 * kv_layer, (const uint8_t *)v_new_all_host + l0 * kv_layer,
+                                     (size_t)(nl * kv_layer), cudaMemcpyHostToDevice, pool->io_stream[0]));
+        }
+        PIE_CUDA(cudaEventRecord(pool->io_up[(size_t)g], pool->io_stream[0]));
+    }
+    st = pie_step_begin(pool);
+    if (st != PIE_OK) return st;
+    for (int32_t l = 0; l < L; ++l) {
+        if (l % G == 0) PIE_CUDA(cudaStreamWaitEvent(s, pool->io_up[(size_t)(l / G)], 0));
+        st = decode_layer(pool, l, (const uint8_t *)pool->stage_q + l * q_layer, (uint8_t *)pool->stage_out + l * q_layer,
+                          pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
+                          k_new_all_host ? (const uint8_t *)pool->stage_k + l * kv_layer : nullptr,
+                          k_new_all_host ? (const uint8_t *)pool->stage_v + l * kv_layer : nullptr, mode);
+        if (st != PIE_OK) break;
+        if ((l + 1) % G == 0 || l + 1 == L) {
+            // the group's results: behind the compute ticket of its last layer
+            const int32_t l0 = (l / G) * G, nl = l + 1 - l0;
+            const int64_t t = pool->table->issued(PIE_Q_COMPUTE);
+            PIE_CUDA(cudaStreamWaitEvent(pool->io_stream[1], pool->ticket_ev[PIE_Q_COMPUTE][t % EV_RING], 0));
+            PIE_CUDA(cudaMemcpyAsync((uint8_t *)out_all_host + l0 * q_layer, (const uint8_t *)pool->stage_out + l0 * q_layer,
+                                     (size_t)(nl * q_layer), cudaMemcpyDeviceToHost, pool->io_stream[1]));
+        }
+    }
+    // whatever happened, nothing of this call may still be in flight when it returns (the caller owns the host buffers)
+    cudaError_t e1 = cudaStreamSynchronize(pool->io_stream[0]);
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    cudaError_t e3 = cudaStreamSynchronize(pool->io_stream[1]);
+    if (st != PIE_OK) return st;
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+        g_last_cuda_error = (int)(e1 != cudaSuccess ? e1 : e2 != cudaSuccess ? e2 : e3);
+        pool->sticky = PIE_ERR_CUDA;
+        return PIE_ERR_CUDA;
+    }
+    st = pie_controller_tick(pool, nullptr);
+    if (st != PIE_OK) return st;
     return check_status_word(pool);
 }
 
