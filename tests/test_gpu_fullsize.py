@@ -91,6 +91,39 @@ def test_llama2_7b_full_size_swapped_matches_oracle_and_resident_run():
     free(dw2)
 
 
+def test_llama2_7b_full_size_kept_host_copies_layer_by_layer_matches_resident_run():
+    """The benchmark workload as configured (30 % host resident), with host copies kept and the write-back of unwritten
+    blocks skipped, driven layer by layer through pie_decode_layer with another kernel between the layers, look-ahead 2:
+    the outputs are bit for bit those of a run that never swapped, and only the written blocks went back."""
+    wl = synth.workload("llama2_7b")
+    steps = 3
+    dw = DeviceWorkload(wl, host_frac=wl.host_frac, timing=True, staging_layers=4)
+    dw.set_retention(True)
+    pie.pie_set_lookahead(dw.pool, 2)
+    scratch = torch.zeros(1 << 22, dtype=torch.float32, device=dw.dev)
+    for _ in range(steps):
+        dw.advance_context()
+        dw.decode_step(between_layers=lambda l: scratch.add_(1.0))
+    dw.sync()
+    short = int(np.argmin(wl.ctx_lens))
+    check_samples(dw, [(0, short), (wl.n_layers - 1, short)], steps)
+    stats = pie.pie_get_stats(dw.pool)
+    n_host = len(set(dw.host_ids.tolist()))
+    moved_out = steps * wl.n_layers * n_host * wl.block_bytes          # what the paper's protocol would write back
+    assert stats["bytes_out"] + stats["reserved"][2] == moved_out
+    # the first time a unit goes out it has no kept copy yet; after that only the blocks that received a token go back
+    assert stats["bytes_out"] <= (wl.n_layers * n_host + (steps - 1) * wl.n_layers * wl.n_seqs) * wl.block_bytes
+    swapped = dw.out_all.cpu().numpy().copy()
+    free(dw)
+    dw2 = DeviceWorkload(wl, host_frac=0.0, timing=False)
+    for _ in range(steps):
+        dw2.advance_context()
+        dw2.decode_step()
+    dw2.sync()
+    assert np.array_equal(swapped, dw2.out_all.cpu().numpy())
+    free(dw2)
+
+
 def test_llama3_8b_full_size_gqa_bf16_fixed_ratio():
     wl = synth.workload("llama3_8b")
     wl = dataclasses.replace(wl, decode_steps=4)            # room for the steps run here (the config decodes 256)
