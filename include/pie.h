@@ -41,7 +41,7 @@ typedef enum pie_status {
 } pie_status;
 
 enum { PIE_F16 = 0, PIE_BF16 = 1 };
-enum { PIE_MODE_AUTO = 0, PIE_MODE_KERNEL = 1, PIE_MODE_COPY_ENGINE = 2 };
+enum { PIE_MODE_AUTO = 0, PIE_MODE_KERNEL = 1, PIE_MODE_COPY_ENGINE = 2, PIE_MODE_KERNEL_BULK = 3 };
 enum { PIE_H2D = 0, PIE_D2H = 1 };
 /* unit states of the two-phase mapping table (Section 3.2) */
 enum { PIE_FREE = 0, PIE_GPU = 1, PIE_TO_HOST = 2, PIE_HOST = 3, PIE_TO_GPU = 4 };
@@ -140,11 +140,13 @@ int pie_get_placement(pie_pool *pool, int32_t *side, int32_t *slot);
  * call, and the GPU slots are released tagged with this copy's ticket.  Phase 2: once the copy is
  * known complete (observed with cudaEventQuery at any later call) the units read PIE_HOST.
  * Blocks already on, or heading to, the host are skipped.  block_ids: host, n entries, distinct.
- * mode: PIE_MODE_KERNEL = gather/scatter kernel, PIE_MODE_COPY_ENGINE = one cudaMemcpyAsync per run of
+ * mode: PIE_MODE_KERNEL = gather/scatter kernel (16-byte loads and stores), PIE_MODE_KERNEL_BULK = the same lists
+ * moved by bulk (TMA) copies through small shared-memory stages, PIE_MODE_COPY_ENGINE = one cudaMemcpyAsync per run of
  * consecutive slots, PIE_MODE_AUTO = copy engine when the list is at most 8 runs, or its runs average 1 MiB, or it
- * is at most 32 runs averaging 256 KiB, else the kernel (measured: the copy engine reaches the link rate from
+ * is at most 32 runs averaging 256 KiB, else the bulk-copy kernel (measured: the copy engine reaches the link rate from
  * ~16 MB and disturbs a concurrent attention kernel several times less than SM-issued host traffic, but one call
- * per scattered 64 KiB block tops out near 12 GB/s).  The slot table follows the data in stream order: written by
+ * per scattered 64 KiB block tops out near 12 GB/s; both kernels reach 0.92 of the link on scattered lists, the
+ * bulk-copy one at a third of the load/store kernel's cost to the attention).  The slot table follows the data in stream order: written by
  * the kernel, or by one small copy per run of consecutive block ids (a patch kernel beyond 16 such runs). */
 int pie_swap_out(pie_pool *pool, int32_t layer, const int32_t *block_ids, int64_t n, int32_t mode);
 /* The mirror image on the copy-in stream.  The layer's next pie_decode_attention waits for it

@@ -20,7 +20,7 @@ PIE_OK = 0
 PIE_ERR_INVALID, PIE_ERR_RANGE, PIE_ERR_NOMEM, PIE_ERR_BUSY = -1, -2, -3, -4
 PIE_ERR_NOT_RESIDENT, PIE_ERR_TIMEOUT, PIE_ERR_CUDA, PIE_ERR_UNSUPPORTED = -5, -6, -7, -8
 PIE_F16, PIE_BF16 = 0, 1
-PIE_MODE_AUTO, PIE_MODE_KERNEL, PIE_MODE_COPY_ENGINE = 0, 1, 2
+PIE_MODE_AUTO, PIE_MODE_KERNEL, PIE_MODE_COPY_ENGINE, PIE_MODE_KERNEL_BULK = 0, 1, 2, 3
 PIE_H2D, PIE_D2H = 0, 1
 PIE_FREE, PIE_GPU, PIE_TO_HOST, PIE_HOST, PIE_TO_GPU = 0, 1, 2, 3, 4
 PIE_Q_NONE, PIE_Q_IN, PIE_Q_OUT, PIE_Q_COMPUTE = 0, 1, 2, 3

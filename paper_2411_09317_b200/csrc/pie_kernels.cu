@@ -288,6 +288,115 @@ plan_kernel(const int32_t *__restrict__ ctx_lens, int32_t n_seqs, int32_t max_to
 }
 
 // =====================================================================================================
+// Swap by bulk copies: the same lists as swap_kernel, moved by the TMA unit instead of by loads and stores.  One
+// thread per CTA drives a ring of 4 KiB shared-memory stages: a bulk copy brings a chunk of a source slot in
+// (host memory or HBM, completing on the stage's mbarrier), a bulk copy sends it on to the destination slot, and
+// a stage is loaded again once the store that last used it has finished reading it.  No registers hold data and
+// no load/store unit is kept busy: the SM footprint is one warp and the stages.
+// =====================================================================================================
+// Small stages on purpose: the persistent attention kernel leaves about 24 KiB of shared memory per SM, and a swap
+// CTA that does not fit beside it would only run between two attention launches.
+constexpr int BULK_STAGES = 4;
+constexpr int BULK_CHUNK_BYTES = 4 * 1024;
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+
+__global__ void __launch_bounds__(32)
+swap_bulk_kernel(const uint8_t *__restrict__ src_pool, uint8_t *__restrict__ dst_pool, const int32_t *__restrict__ list,
+                 int64_t n, int64_t block_bytes, int32_t chunks_per_block, int32_t *slot_table, int table_mode,
+                 int32_t *status) {
+    extern __shared__ __align__(128) uint8_t bulk_smem[];
+    __shared__ __align__(8) uint64_t bars[BULK_STAGES];
+    if (threadIdx.x != 0) return;  // one thread drives the copies
+    const uint32_t smem_base = smem_u32(bulk_smem), bar0 = smem_u32(bars);
+    for (int s = 0; s < BULK_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    const int64_t n_items = n * chunks_per_block;
+    const int64_t mine = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    auto chunk_of = [&](int64_t k, const uint8_t *&sp, uint8_t *&dp, uint32_t &bytes, int32_t &pair_block, int32_t &d_slot, bool &last) {
+        const int64_t item = blockIdx.x + k * gridDim.x;
+        const int64_t pair = item / chunks_per_block;
+        const int32_t chunk = (int32_t)(item - pair * chunks_per_block);
+        const int32_t s_slot = list[3 * pair + 0];
+        d_slot = list[3 * pair + 1];
+        pair_block = list[3 * pair + 2];
+        const int64_t off = (int64_t)chunk * BULK_CHUNK_BYTES;
+        bytes = (uint32_t)min((int64_t)BULK_CHUNK_BYTES, block_bytes - off);
+        sp = src_pool + (int64_t)s_slot * block_bytes + off;
+        dp = dst_pool + (int64_t)d_slot * block_bytes + off;
+        last = chunk == chunks_per_block - 1;
+    };
+    bool ok = true;
+    // loads run BULK_STAGES - 1 chunks ahead of the stores
+    for (int64_t k = 0; k < mine + BULK_STAGES - 1 && ok; ++k) {
+        if (k < mine) {
+            const uint32_t stage = (uint32_t)(k % BULK_STAGES);
+            // the store that last used this stage (chunk k - BULK_STAGES) is the newest one issued: wait for its reads
+            if (k >= BULK_STAGES) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            const uint8_t *sp;
+            uint8_t *dp;
+            uint32_t bytes;
+            int32_t blk, d_slot;
+            bool last;
+            chunk_of(k, sp, dp, bytes, blk, d_slot, last);
+            mbar_expect_tx(bar0 + 8 * stage, bytes);
+            bulk_load(smem_base + stage * BULK_CHUNK_BYTES, sp, bytes, bar0 + 8 * stage);
+        }
+        const int64_t j = k - (BULK_STAGES - 1);
+        if (j >= 0) {
+            const uint32_t stage = (uint32_t)(j % BULK_STAGES);
+            if (!mbar_wait(bar0 + 8 * stage, (uint32_t)((j / BULK_STAGES) & 1))) {
+                raise_status(status, STATUS_WAIT_TIMEOUT);
+                ok = false;
+                break;
+            }
+            const uint8_t *sp;
+            uint8_t *dp;
+            uint32_t bytes;
+            int32_t blk, d_slot;
+            bool last;
+            chunk_of(j, sp, dp, bytes, blk, d_slot, last);
+            bulk_store(dp, smem_base + stage * BULK_CHUNK_BYTES, bytes);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            if (slot_table != nullptr && last) slot_table[blk] = table_mode == 1 ? d_slot : -1;
+        }
+    }
+    // everything this CTA stored must have landed before the kernel counts as complete; after a wait that ran out the
+    // loads still in flight get their (bounded) time to arrive before the stages go away
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (!ok) {
+        const int64_t issued = min(mine, (int64_t)BULK_STAGES);
+        for (int64_t t = 0; t < issued; ++t) mbar_wait(bar0 + 8 * (uint32_t)(t % BULK_STAGES), 0);
+    }
+}
+
+cudaError_t launch_swap_bulk(const void *src_pool, void *dst_pool, const int32_t *list, int64_t n, int64_t block_bytes,
+                             int32_t *slot_table, int table_mode, int n_ctas, int32_t *status, cudaStream_t stream) {
+    if (n <= 0) return cudaSuccess;
+    if (block_bytes % 16 != 0) return cudaErrorInvalidValue;
+    const int32_t chunks = (int32_t)((block_bytes + BULK_CHUNK_BYTES - 1) / BULK_CHUNK_BYTES);
+    const int64_t items = n * chunks;
+    const int grid = (int)(items < n_ctas ? items : n_ctas);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(swap_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGES * BULK_CHUNK_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    swap_bulk_kernel<<<grid, 32, BULK_STAGES * BULK_CHUNK_BYTES, stream>>>((const uint8_t *)src_pool, (uint8_t *)dst_pool, list, n,
+                                                                          block_bytes, chunks, slot_table, table_mode, status);
+    return cudaGetLastError();
+}
+
+// =====================================================================================================
 // Paged decode attention, split-K, one kernel per layer call.
 //
 // Work item = (sequence, KV head, chunk of `split_tokens` tokens).  A persistent grid pulls items from a
@@ -396,11 +505,6 @@ __device__ __forceinline__ bool consumer_vote(bool pred) {
 template <int NTHREADS>
 __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
 }
 
 template <int D, bool BF16, int STAGES, int NW>
@@ -966,7 +1070,7 @@ int attn_smem_bytes(int head_dim) { return head_dim == 128 ? AttnSmem<128, 4, 2>
 // lands on an idle SM first could keep attention CTAs off that SM until it has finished.
 static cudaError_t prefer_max_shared() {
     const void *fns[] = {(const void *)swap_kernel, (const void *)patch_kernel, (const void *)patch_from_list_kernel,
-                         (const void *)kv_write_kernel, (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
+                         (const void *)kv_write_kernel, (const void *)swap_bulk_kernel, (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
                          (const void *)combine_kernel<64, true>, (const void *)combine_kernel<64, false>};
     for (const void *f : fns) {
         cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);

@@ -19,6 +19,10 @@ enum : int32_t {
 // table_mode 1: slot_table[block] = dst_slot (swap-in), 2: slot_table[block] = -1 (swap-out).
 cudaError_t launch_swap(const void *src_pool, void *dst_pool, const int32_t *list, int64_t n, int64_t block_bytes,
                         int32_t *slot_table, int table_mode, int n_ctas, cudaStream_t stream);
+// the same lists moved by bulk (TMA) copies through shared-memory stages: one warp per CTA, no data in registers.
+// status: device-visible status words (a bounded wait that runs out raises STATUS_WAIT_TIMEOUT).
+cudaError_t launch_swap_bulk(const void *src_pool, void *dst_pool, const int32_t *list, int64_t n, int64_t block_bytes,
+                             int32_t *slot_table, int table_mode, int n_ctas, int32_t *status, cudaStream_t stream);
 // table update only (copy-engine path, alloc/free): entries = device int32 pairs {index, value} x n.
 cudaError_t launch_patch(int32_t *table, const int32_t *entries, int64_t n, cudaStream_t stream);
 // same, from triples {src, dst, block} as launch_swap

@@ -279,7 +279,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         mode = (avg_run >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS ||
                 (avg_run >= AUTO_COPY_ENGINE_PIECE_BYTES && runs <= AUTO_COPY_ENGINE_MAX_PIECES))
                    ? PIE_MODE_COPY_ENGINE
-                   : PIE_MODE_KERNEL;
+                   : PIE_MODE_KERNEL_BULK;  // same rate as the load/store kernel, a third of its cost to a concurrent attention kernel
     }
     // Table entries after copy-engine copies.  A patch kernel on a copy stream, launched while the persistent
     // attention grid owns the SMs, was measured to lengthen the gap between two attention launches, and it puts an
@@ -293,7 +293,8 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
             if (blocks[i] != blocks[i - 1] + 1) ++id_runs;
         dma_patch = id_runs <= PATCH_DMA_MAX_RUNS;
     }
-    const bool need_list = mode == PIE_MODE_KERNEL || slot_table_row != nullptr;
+    const bool by_kernel = mode == PIE_MODE_KERNEL || mode == PIE_MODE_KERNEL_BULK;
+    const bool need_list = by_kernel || slot_table_row != nullptr;
     const int64_t list_len = dma_patch ? n : 3 * n;
     int64_t off = 0;
     if (need_list && dma_patch) {
@@ -312,13 +313,17 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         }
         // the swap kernel wants its indices in device memory (no link latency per item); the table patch after
         // copy-engine copies reads the few entries straight from the pinned list and saves a copy-engine operation
-        if (mode == PIE_MODE_KERNEL)
+        if (by_kernel)
             PIE_CUDA(cudaMemcpyAsync(p->list_dev + off, h, (size_t)(3 * n) * 4, cudaMemcpyHostToDevice, stream));
     }
     const int table_mode = slot_table_row ? (dir_queue == PIE_Q_IN ? 1 : 2) : 0;
-    if (mode == PIE_MODE_KERNEL) {
-        const int ctas = p->cfg.swap_ctas > 0 ? p->cfg.swap_ctas : 16;
-        PIE_CUDA(pie::launch_swap(src_pool, dst_pool, p->list_dev + off, n, BB, slot_table_row, table_mode, ctas, stream));
+    if (by_kernel) {
+        const int ctas = p->cfg.swap_ctas > 0 ? p->cfg.swap_ctas : (mode == PIE_MODE_KERNEL ? 16 : 32);
+        if (mode == PIE_MODE_KERNEL)
+            PIE_CUDA(pie::launch_swap(src_pool, dst_pool, p->list_dev + off, n, BB, slot_table_row, table_mode, ctas, stream));
+        else
+            PIE_CUDA(pie::launch_swap_bulk(src_pool, dst_pool, p->list_dev + off, n, BB, slot_table_row, table_mode, ctas,
+                                           p->status_dev, stream));
         p->stats.calls_kernel += 1;
     } else {
         // copy engine: one cudaMemcpyAsync per run of consecutive (src, dst) slots
@@ -366,7 +371,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
 int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t n, int32_t mode, int64_t not_before = 0) {
     if (!p) return PIE_ERR_INVALID;
     if (p->sticky != PIE_OK) return p->sticky;
-    if (mode < PIE_MODE_AUTO || mode > PIE_MODE_COPY_ENGINE) return PIE_ERR_INVALID;
+    if (mode < PIE_MODE_AUTO || mode > PIE_MODE_KERNEL_BULK) return PIE_ERR_INVALID;
     if (n < 0 || (n > 0 && !ids)) return PIE_ERR_INVALID;
     int st = poll(p);
     if (st != PIE_OK) return st;
@@ -1045,7 +1050,7 @@ int pie_swap_raw(pie_pool *pool, int32_t dir, const int32_t *src_slots, const in
     if (!pool || n < 0 || (n > 0 && (!src_slots || !dst_slots))) return PIE_ERR_INVALID;
     if (pool->sticky != PIE_OK) return pool->sticky;
     if (dir != PIE_H2D && dir != PIE_D2H) return PIE_ERR_INVALID;
-    if (mode < PIE_MODE_AUTO || mode > PIE_MODE_COPY_ENGINE) return PIE_ERR_INVALID;
+    if (mode < PIE_MODE_AUTO || mode > PIE_MODE_KERNEL_BULK) return PIE_ERR_INVALID;
     const int64_t n_src = dir == PIE_H2D ? pool->cfg.n_host_slots : pool->cfg.n_gpu_slots;
     const int64_t n_dst = dir == PIE_H2D ? pool->cfg.n_gpu_slots : pool->cfg.n_host_slots;
     for (int64_t i = 0; i < n; ++i)

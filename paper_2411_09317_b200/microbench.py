@@ -79,7 +79,8 @@ def main(argv=None):
             sizes = [1, 16, 256, 2048]
         for pattern in ("contiguous", "scattered"):
             for direction in ("h2d", "d2h", "both"):
-                for mode, mname in ((pie.PIE_MODE_KERNEL, "kernel"), (pie.PIE_MODE_COPY_ENGINE, "copy_engine")):
+                for mode, mname in ((pie.PIE_MODE_KERNEL, "kernel"), (pie.PIE_MODE_KERNEL_BULK, "bulk_kernel"),
+                                    (pie.PIE_MODE_COPY_ENGINE, "copy_engine")):
                     for n in sizes:
                         if n > n_swap_slots:
                             continue
@@ -136,7 +137,8 @@ def main(argv=None):
         if args.blocks:
             blocks = [int(x) for x in args.blocks.split(",")]
         for pattern in ("contiguous", "scattered"):
-            for mode, mname in ((pie.PIE_MODE_KERNEL, "kernel"), (pie.PIE_MODE_COPY_ENGINE, "copy_engine")):
+            for mode, mname in ((pie.PIE_MODE_KERNEL, "kernel"), (pie.PIE_MODE_KERNEL_BULK, "bulk_kernel"),
+                                (pie.PIE_MODE_COPY_ENGINE, "copy_engine")):
                 for direction in ("h2d", "d2h", "both"):
                     for n in blocks:
                         src, dst = swap_lists(n * args.every, pattern, n_swap_slots, 200 + n)

@@ -56,7 +56,7 @@ def make_raw_pool(block_kv_heads=8, head_dim=128, n_slots=96):
     return pool
 
 
-@pytest.mark.parametrize("mode", [pie.PIE_MODE_KERNEL, pie.PIE_MODE_COPY_ENGINE, pie.PIE_MODE_AUTO])
+@pytest.mark.parametrize("mode", [pie.PIE_MODE_KERNEL, pie.PIE_MODE_COPY_ENGINE, pie.PIE_MODE_AUTO, pie.PIE_MODE_KERNEL_BULK])
 @pytest.mark.parametrize("kvh,d", [(8, 128), (4, 64), (1, 64)])
 def test_swap_raw_bit_exact_both_directions(mode, kvh, d):
     n_slots = 96
@@ -113,7 +113,7 @@ def test_swap_raw_whole_pool_untouched_bytes():
     torch.cuda.synchronize()
     pool = pie.pie_pool_create(n_layers=1, n_q_heads=kvh, n_kv_heads=kvh, head_dim=d, dtype=F16, n_logical_blocks=n,
                                n_gpu_slots=n, n_host_slots=n, gpu_base=g_t.data_ptr(), host_base=h_t.data_ptr())
-    for mode in (pie.PIE_MODE_KERNEL, pie.PIE_MODE_COPY_ENGINE):
+    for mode in (pie.PIE_MODE_KERNEL, pie.PIE_MODE_COPY_ENGINE, pie.PIE_MODE_KERNEL_BULK):
         src = synth.seeded_permutation(mode, n)[:17].astype(np.int32)
         dst = synth.seeded_permutation(mode + 5, n)[:17].astype(np.int32)
         pie.pie_swap_raw(pool, pie.PIE_D2H, src, dst, mode)
