@@ -142,8 +142,8 @@ int pie_get_placement(pie_pool *pool, int32_t *side, int32_t *slot);
  * Blocks already on, or heading to, the host are skipped.  block_ids: host, n entries, distinct.
  * mode: PIE_MODE_KERNEL = gather/scatter kernel (16-byte loads and stores), PIE_MODE_KERNEL_BULK = the same lists
  * moved by bulk (TMA) copies through small shared-memory stages, PIE_MODE_COPY_ENGINE = one cudaMemcpyAsync per run of
- * consecutive slots, PIE_MODE_AUTO = copy engine when the list is at most 8 runs, or its runs average 1 MiB, or it
- * is at most 32 runs averaging 256 KiB, else the bulk-copy kernel (measured: the copy engine reaches the link rate from
+ * consecutive slots, PIE_MODE_AUTO = copy engine when the list is at most 8 runs or its runs average 1 MiB, else
+ * the bulk-copy kernel (measured: the copy engine reaches the link rate from
  * ~16 MB and disturbs a concurrent attention kernel several times less than SM-issued host traffic, but one call
  * per scattered 64 KiB block tops out near 12 GB/s; both kernels reach 0.92 of the link on scattered lists, the
  * bulk-copy one at a third of the load/store kernel's cost to the attention).  The slot table follows the data in stream order: written by

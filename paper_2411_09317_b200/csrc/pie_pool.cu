@@ -21,8 +21,6 @@ constexpr int LIST_EVENTS = 512;   // events guarding regions of the id-list rin
 constexpr int TIMING_RING = 4;     // the host may enqueue at most this many steps ahead of their evaluation
 constexpr int64_t AUTO_COPY_ENGINE_RUN_BYTES = 1 << 20;  // AUTO: copy engine when runs average >= 1 MiB ...
 constexpr int64_t AUTO_COPY_ENGINE_MAX_RUNS = 8;         // ... or when the list is at most this many runs
-constexpr int64_t AUTO_COPY_ENGINE_PIECE_BYTES = 256 << 10;  // ... or runs of this size, up to
-constexpr int64_t AUTO_COPY_ENGINE_MAX_PIECES = 32;          //     this many of them
 constexpr int IO_GROUP_LAYERS = 4;   // pie_decode_step_host moves inputs and results in groups of this many layers
 constexpr int64_t PATCH_DMA_MAX_RUNS = 16;               // table entries by small copies up to this many runs of ids, else a kernel
 
@@ -270,16 +268,13 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         int64_t runs = 1;
         for (int64_t i = 1; i < n; ++i)
             if (src[i] != src[i - 1] + 1 || dst[i] != dst[i - 1] + 1) ++runs;
-        // copy engine for long runs or few copies (no SM or L2 footprint next to attention); the kernel for scattered
-        // lists of small pieces, where one cudaMemcpyAsync per piece would be bound by the call rate (~2-5 us each).
-        // Pieces of 256 KiB and more still move at most of the link's rate one by one, and host traffic issued by SMs
-        // disturbs a concurrent attention kernel several times more than the copy engine's: up to 32 such pieces per
-        // list go by copy engine too (slot lists get scattered when the host-resident sets change one block at a time).
-        const int64_t avg_run = (n * BB) / runs;
-        mode = (avg_run >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS ||
-                (avg_run >= AUTO_COPY_ENGINE_PIECE_BYTES && runs <= AUTO_COPY_ENGINE_MAX_PIECES))
-                   ? PIE_MODE_COPY_ENGINE
-                   : PIE_MODE_KERNEL_BULK;  // same rate as the load/store kernel, a third of its cost to a concurrent attention kernel
+        // copy engine for long runs or few copies (no SM or L2 footprint next to attention); the bulk-copy kernel for
+        // scattered lists, where one cudaMemcpyAsync per piece is bound by the call rate (~2-5 us each) and every
+        // separate device-to-host copy costs a concurrent attention kernel a fixed 1-2 % (measured: 21 pieces of
+        // 256 KiB per list by copy engine cost 18 %, by kernel far less).  The bulk kernel moves scattered lists at
+        // the same rate as the load/store kernel and costs the attention a third of what that one does.
+        mode = ((n * BB) / runs >= AUTO_COPY_ENGINE_RUN_BYTES || runs <= AUTO_COPY_ENGINE_MAX_RUNS) ? PIE_MODE_COPY_ENGINE
+                                                                                                   : PIE_MODE_KERNEL_BULK;
     }
     // Table entries after copy-engine copies.  A patch kernel on a copy stream, launched while the persistent
     // attention grid owns the SMs, was measured to lengthen the gap between two attention launches, and it puts an
