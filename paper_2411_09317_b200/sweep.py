@@ -31,6 +31,7 @@ from .harness import DeviceWorkload
 
 
 OTHER = {"fn": None}   # stand-in for a model's other per-layer work (--other-mb): called after every layer's attention
+SWAP_MODE = {"mode": pie.PIE_MODE_AUTO}   # --swap-mode: how swap lists are moved
 
 
 def run_steps(dw, n):
@@ -38,14 +39,14 @@ def run_steps(dw, n):
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
     dw.sync()
     dw.advance_context()
-    dw.decode_step(between_layers=OTHER["fn"])
+    dw.decode_step(between_layers=OTHER["fn"], mode=SWAP_MODE["mode"])
     before, ctx0 = pie.pie_get_stats(dw.pool), dw.ctx_lens.copy()
     with torch.cuda.stream(dw.s_compute):
         marks[0].record()
     per_stats = []
     for i in range(n):
         dw.advance_context()
-        dw.decode_step(between_layers=OTHER["fn"])
+        dw.decode_step(between_layers=OTHER["fn"], mode=SWAP_MODE["mode"])
         per_stats.append(pie.pie_get_stats(dw.pool))
         with torch.cuda.stream(dw.s_compute):
             marks[i + 1].record()
@@ -78,6 +79,8 @@ def main(argv=None):
                     help="ratios / adaptive: after every layer's attention, an elementwise kernel that reads and writes this many MB "
                          "on the compute stream stands in for the model's projections and MLP (weights streamed from HBM); the "
                          "step then runs layer by layer through pie_decode_layer")
+    ap.add_argument("--swap-mode", default="auto", choices=["auto", "kernel", "copy_engine", "bulk_kernel"],
+                    help="how swap lists are moved (PIE_MODE_*)")
     ap.add_argument("--lookahead", type=int, default=1, help="layers prefetched ahead (pie_set_lookahead)")
     ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
     ap.add_argument("--out", default=None)
@@ -88,6 +91,8 @@ def main(argv=None):
         out.write(json.dumps(obj) + "\n")
         out.flush()
 
+    SWAP_MODE["mode"] = {"auto": pie.PIE_MODE_AUTO, "kernel": pie.PIE_MODE_KERNEL, "copy_engine": pie.PIE_MODE_COPY_ENGINE,
+                         "bulk_kernel": pie.PIE_MODE_KERNEL_BULK}[args.swap_mode]
     if args.other_mb > 0:
         # an elementwise kernel, not a memcpy: a device-to-device cudaMemcpyAsync may be served by the copy engines,
         # which the swaps need
