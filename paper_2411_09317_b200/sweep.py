@@ -125,6 +125,7 @@ def main(argv=None):
               "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "other_mb_per_layer": args.other_mb,
               "lookahead": args.lookahead,
               "link": link})
+        first_gbs = None
         for r in ratios:
             pie.pie_set_extension_ratio(dw.pool, r)
             run_steps(dw, 2)
@@ -132,7 +133,10 @@ def main(argv=None):
             ms = float(np.median(per))
             tot = sum(per) * 1e-3
             by = attention_bytes(wl, ctx0 + (args.steps + 1) // 2)
-            emit({"ratio": r, "expansion": None if r >= 1.0 else 1.0 / (1.0 - r), "ms_per_step": ms,
+            first_gbs = first_gbs or by / (ms * 1e-3) / 1e9
+            emit({"ratio": r,
+                  # the context grows a token per sequence per step: rows are comparable in bytes per second, not in ms
+                  "slowdown_vs_first_row_at_equal_context": first_gbs / (by / (ms * 1e-3) / 1e9) - 1.0, "expansion": None if r >= 1.0 else 1.0 / (1.0 - r), "ms_per_step": ms,
                   "attn_gbs": by / (ms * 1e-3) / 1e9, "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9,
                   "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
                   "wait_share": sa["last_step_stall_ms"] / max(sa["last_step_ms"], 1e-9),
