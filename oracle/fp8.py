@@ -84,8 +84,10 @@ def paged_attention(gpu_pool8, host_pool8, unit_side, unit_slot, q, block_table,
 def append(gpu_pool8, host_pool8, unit_side, unit_slot, k_new, v_new, block_table, ctx_lens, n_kv_heads, head_dim, dtype,
            k_scale, v_scale):
     """The new token of every sequence (16-bit rows [S][Hkv][D]) is quantised and written at position ctx_len - 1."""
-    kf = _bits16_to_f64(k_new, dtype) / k_scale
-    vf = _bits16_to_f64(v_new, dtype) / v_scale
+    # the division is a single-precision one (the precision the kernel takes this decision in); the rounding to E4M3
+    # then starts from that fp32 quotient
+    kf = _bits16_to_f64(k_new, dtype).astype(np.float32) / np.float32(k_scale)
+    vf = _bits16_to_f64(v_new, dtype).astype(np.float32) / np.float32(v_scale)
     kq, vq = quantize(kf), quantize(vf)
     for s, ctx in enumerate(np.asarray(ctx_lens)):
         if ctx <= 0:
