@@ -266,13 +266,13 @@ def main():
                         extra_host_slots=(L + 3) * int(r_cap * n_blocks) + 64, extra_tokens=total_steps)
     bytes_layer0 = dw.attention_bytes_per_layer()
 
-    def bytes_of_steps(n_steps, ctx_before):
+    def bytes_of_steps(n_steps, ctx_before, kv_elem_bytes=2):
         """Algorithmic attention bytes of n steps starting from context lengths ctx_before (each step adds a token)."""
         total = 0
         ctx = ctx_before.astype(np.int64).copy()
         for _ in range(n_steps):
             ctx += 1
-            kv = int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2
+            kv = int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * kv_elem_bytes
             qo = 2 * wl.n_seqs * wl.n_q_heads * wl.head_dim * 2
             tab = 4 * (int(((ctx + 15) // 16).sum()) + wl.n_seqs)
             total += L * (kv + qo + tab)
@@ -434,6 +434,39 @@ def main():
         "frac_of_h2d_link": (s_a["bytes_in"] - s_b["bytes_in"]) / (ms_k * 1e-3) / 1e9 / max(link["h2d"], 1e-9),
     }
 
+    # ---- the 8-bit KV variant (blocks of E4M3 bytes) on the same shape: resident, then a hidden swap with kept host copies
+    dw.close()
+    for name in ("gpu_pool", "host_pool", "q_all", "out_all", "k_new", "v_new"):
+        setattr(dw, name, None)
+    gc.collect()
+    torch.cuda.empty_cache()
+    kv_fp8 = None
+    if wl.head_dim == 128:
+        import dataclasses
+        wl8 = dataclasses.replace(wl, kv_fp8=True)
+        n8, r8 = 8, 0.01
+        dw = DeviceWorkload(wl8, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
+                            attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=3 * int(r_cap * n_blocks) + 64,
+                            extra_host_slots=(L + 3) * int(r_cap * n_blocks) + 64, extra_tokens=6 * (n8 + 2))
+        timed_steps(dw, torch, 3)
+        ms8, _ = timed_steps(dw, torch, n8)
+        by8 = bytes_of_steps(n8, timed_steps.ctx_before, 1)
+        kv_fp8 = {"resident": {"ms_per_step": ms8 / n8, "attn_gbs": median_gbs(by8, n8),
+                               "tokens_per_s_vs_16bit": None}}
+        dw.set_retention(True)
+        pie.pie_set_extension_ratio(dw.pool, r8)
+        timed_steps(dw, torch, 3)
+        ms8s, _ = timed_steps(dw, torch, n8)
+        c8, sb8, sa8 = timed_steps.ctx_before, timed_steps.before, timed_steps.after
+        g8 = median_gbs(bytes_of_steps(n8, c8, 1), n8)
+        kv_fp8["hidden_swap_kept_copies"] = {
+            "ratio": r8, "ms_per_step": ms8s / n8, "attn_gbs": g8, "slowdown": kv_fp8["resident"]["attn_gbs"] / g8 - 1.0,
+            "swap_in_gbs": (sa8["bytes_in"] - sb8["bytes_in"]) / (ms8s * 1e-3) / 1e9,
+            "swap_out_gbs": (sa8["bytes_out"] - sb8["bytes_out"]) / (ms8s * 1e-3) / 1e9,
+            "frac_of_h2d_link": (sa8["bytes_in"] - sb8["bytes_in"]) / (ms8s * 1e-3) / 1e9 / max(link["h2d"], 1e-9)}
+        # the same tokens take half the bytes: time per step against the 16-bit resident run at (nearly) the same context
+        kv_fp8["resident"]["tokens_per_s_vs_16bit"] = (ms_res / args.steps) / (ms8 / n8)
+
     peak, peak_kind = measured_peaks()
     achieved = bytes_layer0 / (attn_ms_layer * 1e-3) / 1e9 if attn_ms_layer == attn_ms_layer else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -465,7 +498,7 @@ def main():
             "hidden_swap": hidden, "resident": {"attn_gbs": resident_gbs, "attn_gbs_after": resident_after_gbs,
                                                 "attn_gbs_median_step": resident_med,
                                                 "ms_per_step": ms_res / args.steps},
-            "as_configured": as_configured,
+            "as_configured": as_configured, "kv_fp8": kv_fp8,
         }
         print(json.dumps(line))
     dw.close()

@@ -80,7 +80,9 @@ typedef struct pie_pool_config {
                                 * 2: also keep the per-layer timeline for pie_get_step_timeline */
     int32_t reserved[7];       /* [0]: attention kernel variant for tuning (0 = default);
                                 * [1]: per-layer size visible to allocation at creation, in blocks (0 = n_logical_blocks;
-                                *      see pie_resize_begin); rest 0 */
+                                *      see pie_resize_begin);
+                                * [2]: 1 = the blocks hold K and V as FP8 E4M3 bytes (see pie_set_kv_scales): head_dim 128
+                                *      and variants 0, 1 only (PIE_ERR_UNSUPPORTED otherwise), block_bytes halves; rest 0 */
 } pie_pool_config;
 
 typedef struct pie_stats {
@@ -239,6 +241,20 @@ int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
  * keep up on average, not layer by layer - at the price of as many more layers' shares of GPU staging slots.
  * 1 <= layers <= 8 (PIE_ERR_INVALID otherwise). */
 int pie_set_lookahead(pie_pool *pool, int32_t layers);
+
+/* ---- 8-bit blocks (a variant beyond the paper, whose blocks are 16-bit: a token costs half the bytes in HBM, in the
+ * host pool and on the link, so the same link hides twice the tokens per layer - Section 3.1's condition in bytes) ----
+ * A pool created with reserved[2] = 1 stores a block as [n_kv_heads][K|V][16 tokens][128] bytes of E4M3 (1-4-3 bits,
+ * bias 7, no infinities, largest value 448); a stored byte b stands for decode(b) * k_scale (keys) or * v_scale
+ * (values), one pair of scales for the pool (default 1, 1).  q, out and the new token's k_new / v_new stay in the pool's
+ * 16-bit type.  pie_decode_attention computes attention over the decoded values (scores and sums in fp32 as for 16-bit
+ * pools; the key scale enters the softmax scale, the value scale the result); its append stores
+ * E4M3(fp32(x) / scale), rounded to nearest (ties to the even code), magnitudes beyond 448 saturating, NaN -> 0x7f, and
+ * the step's own attention already sees the stored (rounded) token.  A NaN byte (0x7f, 0xff) among the valid tokens is
+ * outside the contract: the kernel reads it as +-480 (bytes beyond a sequence's length may hold anything).  Swapping, the table and the controller are
+ * unchanged (they move block_bytes).  pie_kv_write returns PIE_ERR_UNSUPPORTED on such a pool.
+ * PIE_ERR_INVALID unless both scales are finite and > 0; PIE_ERR_UNSUPPORTED on a 16-bit pool. */
+int pie_set_kv_scales(pie_pool *pool, float k_scale, float v_scale);
 
 /* ---- prefill-side KV write (Section 2.2: the prompt's keys and values enter the cache; the decode path above
  * appends one token per sequence, this call writes any number) ---------------------------------------------

@@ -36,7 +36,7 @@ EXPORTS = [
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
-    "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead",
+    "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
 ]
 
 
@@ -118,6 +118,7 @@ _sig = {
     "pie_table_drop_host_copy": (_i32, [_vp, _i32, _i32]),
     "pie_set_retention": (_i32, [_vp, _i32]),
     "pie_set_lookahead": (_i32, [_vp, _i32]),
+    "pie_set_kv_scales": (_i32, [_vp, ctypes.c_float, ctypes.c_float]),
     "pie_decode_layer": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _i32, _f32, _vp, _vp, _i32]),
     "pie_kv_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i64, _vp, _i32, _i32]),
     "pie_declare_append_blocks": (_i32, [_vp, _vp, _i64]),
@@ -176,6 +177,7 @@ def pie_pool_create(**kw) -> int:
     kw.setdefault("max_seqs", 256)
     cfg.reserved[0] = kw.pop("attn_variant", 0)
     cfg.reserved[1] = kw.pop("visible_blocks", 0)
+    cfg.reserved[2] = int(kw.pop("kv_fp8", 0))
     for k, v in kw.items():
         setattr(cfg, k, v)
     out = _vp()
@@ -194,6 +196,10 @@ def pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, bloc
 
 def pie_set_lookahead(pool, layers) -> None:
     check(lib.pie_set_lookahead(pool, layers), "pie_set_lookahead")
+
+
+def pie_set_kv_scales(pool, k_scale, v_scale) -> None:
+    check(lib.pie_set_kv_scales(pool, k_scale, v_scale), "pie_set_kv_scales")
 
 
 def pie_set_retention(pool, on) -> None:
@@ -508,6 +514,8 @@ def synth_lib():
         _synth = ctypes.CDLL(SYNTH_LIB_PATH)
         _synth.pie_synth_fill_slots.restype = _i32
         _synth.pie_synth_fill_slots.argtypes = [_vp, _vp, _i64, _i64, ctypes.c_uint64, _i32, _f32, _vp]
+        _synth.pie_synth_fill_slots_bytes.restype = _i32
+        _synth.pie_synth_fill_slots_bytes.argtypes = [_vp, _vp, _i64, _i64, ctypes.c_uint64, _vp]
         _synth.pie_synth_fill_tensor.restype = _i32
         _synth.pie_synth_fill_tensor.argtypes = [_vp, _i64, ctypes.c_uint64, ctypes.c_uint64, _i32, _f32, _vp]
     return _synth

@@ -445,16 +445,21 @@ struct AttnParams {
     int32_t *status;
     int64_t n_gpu_slots;
     int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d, max_chunks;
-    float scale_log2e;
+    float scale_log2e;      // softmax scale * log2(e) (* the key scale of an 8-bit pool)
+    float out_scale = 1.f;  // 8-bit pools: the value scale (times what the kernel's 16-bit images of the bytes leave out)
+    float k_scale = 1.f, v_scale = 1.f;  // 8-bit pools: the append stores E4M3(x / scale)
 };
 
-template <int D, int STAGES, int NW>
+// KV8: the pool holds E4M3 bytes; a ring stage is then the 4 KiB byte tile as the TMA unit delivers it, and the consumer
+// warps build their tensor-core operands from those bytes in registers.
+template <int D, int STAGES, int NW, bool KV8 = false>
 struct AttnSmem {
     static constexpr int TILE_BYTES = 2 * 16 * D * 2;
+    static constexpr int RING_BYTES = KV8 ? 2 * 16 * D : TILE_BYTES;       // one ring stage
     static constexpr int HALF_BYTES = 32 * 128;  // 32 rows x 128 bytes
     static constexpr int MO_STRIDE = D + 4;      // floats per (warp, head) row; +4 keeps the scatter conflict-free
     static constexpr int Q_BYTES = 8 * D * 2;    // query rows of one item (up to 8 heads)
-    static constexpr int OFF_Q = STAGES * TILE_BYTES;
+    static constexpr int OFF_Q = STAGES * RING_BYTES;
     static constexpr int OFF_MO = OFF_Q + ATT_QD * Q_BYTES;
     static constexpr int OFF_ML = OFF_MO + NW * 8 * MO_STRIDE * 4;
     static constexpr int OFF_BAR = OFF_ML + NW * 8 * 2 * 4;              // full[STAGES], empty[STAGES], qfull[QD], qempty[QD]
@@ -507,10 +512,57 @@ __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
 }
 
-template <int D, bool BF16, int STAGES, int NW>
-__global__ void __launch_bounds__((NW + 1) * 32)
+// Two E4M3 bytes -> two 16-bit values of the compute type, by moving bits instead of converting: E4M3's four exponent
+// bits become the low bits of the wider exponent field and its three mantissa bits the top of the wider mantissa;
+// subnormals stay subnormals of the same shape.  The result is the value times 2^-8 (fp16: the exponent bias goes from 7
+// to 15) or 2^-120 (bf16: 7 to 127).  bf16 multiplies the factor back at once (exact); fp16 leaves it in -
+// KV8_F16_FACTOR - and the launch folds 2^8 into the softmax scale and the value scale: every such value, down to the
+// smallest subnormal 2^-9 * 2^-8, is still an exact fp16 number.  The byte 0x7f / 0xff (E4M3's NaN) comes out as +-480.
+// Two forms, so that the integer work is shared between the ALU and the multiply-add pipe:
+//   hi: the bytes sit in the upper byte of each 16-bit half (what the lower bytes hold does not matter): shift right;
+//   lo: the bytes sit in the lower byte of each half, the upper bytes are zero: multiply up, then move the sign bit one
+//       place (fp16) or four places (bf16) further up by adding it again.
+constexpr float KV8_F16_FACTOR = 256.f;
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_times_2_120(uint32_t r) {
+    uint32_t o;
+    asm("mul.bf16x2 %0, %1, %2;" : "=r"(o) : "r"(r), "r"(0x7b807b80u));
+    return o;
+}
+template <bool BF16>
+__device__ __forceinline__ uint32_t e4m3x2_hi_to_16x2(uint32_t t) {
+    if (BF16) return bf16x2_times_2_120((t & 0x80008000u) | ((t >> 4) & 0x07f007f0u));
+    return (t & 0x80008000u) | ((t >> 1) & 0x3f803f80u);
+}
+template <bool BF16>
+__device__ __forceinline__ uint32_t e4m3x2_lo_to_16x2(uint32_t x) {
+    if (BF16) {
+        const uint32_t y = mad_u32(x, 16u, 0u);                       // sign at bit 11 of each half: 15 more of it -> bit 15
+        return bf16x2_times_2_120(mad_u32(y & 0x08000800u, 15u, y));
+    }
+    const uint32_t y = mad_u32(x, 128u, 0u);                          // sign at bit 14 of each half
+    return mad_u32(y & 0x40004000u, 1u, y);
+}
+// two floats -> two E4M3 bytes (lo in the low byte): nearest even, saturating to +-448
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// The second launch bound: for 16-bit pools it only tells the assembler that it need not hold registers back for more
+// CTAs per SM than shared memory lets in anyway (three; without it some instantiations were capped at 96 registers and
+// spilled).  The 8-bit kernel is bound by instruction latency, not by bytes in flight, and its CTAs need a third of
+// the shared memory: five per SM (128 registers) measured 3-6 % faster than four.
+template <int D, bool BF16, int STAGES, int NW, bool KV8 = false>
+__global__ void __launch_bounds__((NW + 1) * 32, KV8 ? 5 : 1)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p) {
-    using SM = AttnSmem<D, STAGES, NW>;
+    using SM = AttnSmem<D, STAGES, NW, KV8>;
+    static_assert(!KV8 || D == 128, "8-bit blocks: head_dim 128 (one 128-byte row per token)");
     // A stage must always be consumed by the same warp: tile i goes to warp i % NW and to stage i % STAGES.  If two
     // warps alternated on a stage, the one running ahead could pass a parity wait on the phase before the one it
     // needs (an mbarrier waiter may be at most one phase ahead).
@@ -651,11 +703,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                             sl = 0;
                         }
                         if (*abort_flag == 0) {
-                            const uint32_t dst = smem_base + stage * SM::TILE_BYTES;
+                            const uint32_t dst = smem_base + stage * SM::RING_BYTES;
                             const uint32_t bar = bar_full + 8 * stage;
                             const int32_t row0 = (sl * p.n_kv_heads + it.kvh) * 32;
-                            mbar_expect_tx(bar, SM::TILE_BYTES);
-                            if (p.use3d) {
+                            mbar_expect_tx(bar, SM::RING_BYTES);
+                            if (KV8) {
+                                tma_load_2d(dst, &tmap, 0, row0, bar);  // 32 rows (16 K, 16 V) of 128 bytes
+                            } else if (p.use3d) {
                                 tma_load_3d(dst, &tmap, 0, row0, 0, bar);
                             } else {
 #pragma unroll
@@ -713,8 +767,15 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(smem + SM::OFF_Q + qs * SM::Q_BYTES) + g * (D / 2);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                bq[ks][0] = g < p.group ? qrow[ks * 8 + (lane & 3)] : 0u;
-                bq[ks][1] = g < p.group ? qrow[ks * 8 + 4 + (lane & 3)] : 0u;
+                if (KV8) {  // step 4 j + s reads d0 = 16 (4 j + t) + 4 s .. + 3 as k = d0, d0 + 2 | d0 + 1, d0 + 3: the K bytes' order below
+                    const int w = 8 * (4 * (ks >> 2) + (lane & 3)) + 2 * (ks & 3);
+                    const uint32_t qa = g < p.group ? qrow[w] : 0u, qb = g < p.group ? qrow[w + 1] : 0u;
+                    bq[ks][0] = __byte_perm(qa, qb, 0x5410u);
+                    bq[ks][1] = __byte_perm(qa, qb, 0x7632u);
+                } else {
+                    bq[ks][0] = g < p.group ? qrow[ks * 8 + (lane & 3)] : 0u;
+                    bq[ks][1] = g < p.group ? qrow[ks * 8 + 4 + (lane & 3)] : 0u;
+                }
             }
         }
         float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
@@ -732,52 +793,136 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             }
             __syncwarp();
             if (*abort_flag) break;  // leave through the item's barriers so that no warp is left waiting
-            uint8_t *tile = smem + stage * SM::TILE_BYTES;
-            const uint32_t tile_u32 = smem_base + stage * SM::TILE_BYTES;
             const int nvalid = min(16, it.t1 - (it.t0 + 16 * i));
             bool touched = false;
-            if (nvalid < 16) {
-                // masked tokens are excluded, not multiplied by zero: clear their V rows so that 0 * garbage
-                // (possibly NaN/Inf) never enters the PV product.  A row is 128 contiguous bytes per half.
-                const int nvec = (16 - nvalid) * (D / 64) * 8;
-                for (int e = lane; e < nvec; e += 32) {
-                    const int row = 16 + nvalid + e / ((D / 64) * 8);
-                    const int rem = e % ((D / 64) * 8);
-                    *reinterpret_cast<uint4 *>(tile + (rem >> 3) * SM::HALF_BYTES + row * 128 + (rem & 7) * 16) =
-                        make_uint4(0, 0, 0, 0);
-                }
-                touched = true;
-            }
-            if (p.k_new != nullptr && it.t1 == it.ctx && i == it.ntiles - 1) {
-                // append: this tile holds position ctx-1; put the new token's K and V rows into the staged tile
-                // (lanes 0-15: K, lanes 16-31: V, one 16-byte piece each) and into the pool
-                const int32_t pos = it.ctx - 1, r = pos & 15;
-                int32_t slot = -1;
-                if (lane == 0) {
-                    const int32_t blk = __ldg(p.block_table + (int64_t)it.s * p.max_blocks + (pos >> 4));
-                    if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
-                    if (slot >= p.n_gpu_slots) slot = -1;
-                }
-                slot = __shfl_sync(0xffffffffu, slot, 0);
-                const int kv = lane >> 4, c = lane & 15;
-                if (c < D / 8) {
-                    const uint4 val = __ldg((kv ? p.v_new : p.k_new) + ((int64_t)it.s * p.n_kv_heads + it.kvh) * (D / 8) + c);
-                    *reinterpret_cast<uint4 *>(tile + (c >> 3) * SM::HALF_BYTES + (kv * 16 + r) * 128 + (((c & 7) ^ (r & 7)) << 4)) = val;
-                    if (slot >= 0)
-                        p.pool[((((int64_t)slot * p.n_kv_heads + it.kvh) * 2 + kv) * 16 + r) * (D / 8) + c] = val;
-                }
-                touched = true;
-            }
-            if (touched) __syncwarp();
-            // ---- S^T[16 tokens][8 heads] = K[16][D] . q^T[D][8]
             float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+            [[maybe_unused]] uint4 vv[4];  // 8-bit path: this lane's 16 bytes of the V rows of tokens 2t, 2t+1, 2t+8, 2t+9
+            if constexpr (KV8) {
+                // The stage holds the tile as bytes: 32 rows (16 K, 16 V) of 128, 16-byte pieces swizzled by the row.  The
+                // operands are built in registers, straight from the bytes.  The sums over head_dim (scores) and over the
+                // tokens (output) do not care in which order their terms are fed to the tensor core, and neither does the
+                // output care which accumulator row holds which d, so every lane reads whole 16-byte pieces:
+                //   K: lane (g, t) reads pieces t and 4 + t of rows g and g + 8; word s of piece 4 j + t feeds step 4 j + s,
+                //      bytes 0, 2 as k = 2t, 2t+1 and bytes 1, 3 as k = 2t+8, 2t+9 (q is read with the same assignment);
+                //   V: lane (g, t) reads piece g of the rows of tokens 2t, 2t+1, 2t+8, 2t+9; byte 2i (2i+1) of the piece is
+                //      accumulator row g (g + 8) of product i, that is d = 16 g + 2 i (+ 1).
+                uint8_t *ring = smem + stage * SM::RING_BYTES;
+                if (p.k_new != nullptr && it.t1 == it.ctx && i == it.ntiles - 1) {
+                    // append: quantise the new token's rows (fp32 quotient by the scale, nearest-even E4M3, saturating) and
+                    // put the bytes into the pool and into the staged tile (lanes 0-15: K, 16-31: V, eight values each)
+                    const int32_t pos = it.ctx - 1, r = pos & 15;
+                    int32_t slot = -1;
+                    if (lane == 0) {
+                        const int32_t blk = __ldg(p.block_table + (int64_t)it.s * p.max_blocks + (pos >> 4));
+                        if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
+                        if (slot >= p.n_gpu_slots) slot = -1;
+                    }
+                    slot = __shfl_sync(0xffffffffu, slot, 0);
+                    const int kv = lane >> 4, c = lane & 15;
+                    const uint4 val = __ldg((kv ? p.v_new : p.k_new) + ((int64_t)it.s * p.n_kv_heads + it.kvh) * (D / 8) + c);
+                    const float sc = kv ? p.v_scale : p.k_scale;
+                    const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+                    uint32_t b[4];
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const int chunk = 2 * ks + k_csel;
-                uint32_t a[4];
-                ldmatrix_x4(tile_u32 + (chunk >> 3) * SM::HALF_BYTES + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), a);
-                if (ks & 1) mma_16816<BF16>(sb, a, bq[ks][0], bq[ks][1]);
-                else mma_16816<BF16>(sa, a, bq[ks][0], bq[ks][1]);
+                    for (int j = 0; j < 4; ++j) {
+                        float lo, hi;
+                        if (BF16) {
+                            lo = __uint_as_float(w[j] << 16);
+                            hi = __uint_as_float(w[j] & 0xffff0000u);
+                        } else {
+                            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[j]));
+                            lo = f.x;
+                            hi = f.y;
+                        }
+                        b[j] = f32x2_to_e4m3x2(__fdiv_rn(lo, sc), __fdiv_rn(hi, sc));
+                    }
+                    const uint2 bytes = make_uint2(b[0] | (b[1] << 16), b[2] | (b[3] << 16));
+                    if (slot >= 0)
+                        *reinterpret_cast<uint2 *>(reinterpret_cast<uint8_t *>(p.pool) +
+                                                   ((((int64_t)slot * p.n_kv_heads + it.kvh) * 2 + kv) * 16 + r) * D + 8 * c) = bytes;
+                    *reinterpret_cast<uint2 *>(ring + (kv * 16 + r) * 128 + (((c >> 1) ^ (r & 7)) << 4) + (c & 1) * 8) = bytes;
+                    touched = true;
+                    __syncwarp();
+                }
+                const int g = lane >> 2, t = lane & 3;
+                uint4 kg[2], kh[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int off = ((4 * j + t) ^ g) << 4;  // rows g and g + 8 are swizzled alike
+                    kg[j] = *reinterpret_cast<const uint4 *>(ring + g * 128 + off);
+                    kh[j] = *reinterpret_cast<const uint4 *>(ring + (g + 8) * 128 + off);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int tok = 2 * t + (j & 1) + 8 * (j >> 1);
+                    vv[j] = *reinterpret_cast<const uint4 *>(ring + (16 + tok) * 128 + ((g ^ (tok & 7)) << 4));
+                }
+                __syncwarp();
+                if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                if (lane == 0) mbar_arrive(bar_empty + 8 * stage);  // everything is in registers: the stage may be refilled
+                // ---- S^T[16 tokens][8 heads] = K . q^T
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint32_t wg[4] = {kg[j].x, kg[j].y, kg[j].z, kg[j].w};
+                    const uint32_t wh[4] = {kh[j].x, kh[j].y, kh[j].z, kh[j].w};
+#pragma unroll
+                    for (int s4 = 0; s4 < 4; ++s4) {
+                        const int ks = 4 * j + s4;
+                        uint32_t a[4];
+                        a[0] = e4m3x2_lo_to_16x2<BF16>(wg[s4] & 0x00ff00ffu);
+                        a[1] = e4m3x2_lo_to_16x2<BF16>(wh[s4] & 0x00ff00ffu);
+                        a[2] = e4m3x2_hi_to_16x2<BF16>(wg[s4]);
+                        a[3] = e4m3x2_hi_to_16x2<BF16>(wh[s4]);
+                        if (ks & 1) mma_16816<BF16>(sb, a, bq[ks][0], bq[ks][1]);
+                        else mma_16816<BF16>(sa, a, bq[ks][0], bq[ks][1]);
+                    }
+                }
+            } else {
+                uint8_t *tile = smem + stage * SM::RING_BYTES;
+                const uint32_t tile_u32 = smem_base + stage * SM::RING_BYTES;
+                if (nvalid < 16) {
+                    // masked tokens are excluded, not multiplied by zero: clear their V rows so that 0 * garbage
+                    // (possibly NaN/Inf) never enters the PV product.  A row is 128 contiguous bytes per half.
+                    const int nvec = (16 - nvalid) * (D / 64) * 8;
+                    for (int e = lane; e < nvec; e += 32) {
+                        const int row = 16 + nvalid + e / ((D / 64) * 8);
+                        const int rem = e % ((D / 64) * 8);
+                        *reinterpret_cast<uint4 *>(tile + (rem >> 3) * SM::HALF_BYTES + row * 128 + (rem & 7) * 16) =
+                            make_uint4(0, 0, 0, 0);
+                    }
+                    touched = true;
+                }
+                if (p.k_new != nullptr && it.t1 == it.ctx && i == it.ntiles - 1) {
+                    // append: this tile holds position ctx-1; put the new token's K and V rows into the staged tile
+                    // (lanes 0-15: K, lanes 16-31: V, one 16-byte piece each) and into the pool
+                    const int32_t pos = it.ctx - 1, r = pos & 15;
+                    int32_t slot = -1;
+                    if (lane == 0) {
+                        const int32_t blk = __ldg(p.block_table + (int64_t)it.s * p.max_blocks + (pos >> 4));
+                        if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
+                        if (slot >= p.n_gpu_slots) slot = -1;
+                    }
+                    slot = __shfl_sync(0xffffffffu, slot, 0);
+                    const int kv = lane >> 4, c = lane & 15;
+                    if (c < D / 8) {
+                        const uint4 val = __ldg((kv ? p.v_new : p.k_new) + ((int64_t)it.s * p.n_kv_heads + it.kvh) * (D / 8) + c);
+                        if (slot >= 0) {
+                            p.pool[((((int64_t)slot * p.n_kv_heads + it.kvh) * 2 + kv) * 16 + r) * (D / 8) + c] = val;
+                        }
+                        *reinterpret_cast<uint4 *>(tile + (c >> 3) * SM::HALF_BYTES + (kv * 16 + r) * 128 + (((c & 7) ^ (r & 7)) << 4)) = val;
+                    }
+                    touched = true;
+                }
+                if (touched) __syncwarp();
+                // ---- S^T[16 tokens][8 heads] = K[16][D] . q^T[D][8]
+    #pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const int chunk = 2 * ks + k_csel;
+                    uint32_t a[4];
+                    ldmatrix_x4(tile_u32 + (chunk >> 3) * SM::HALF_BYTES + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), a);
+                    if (ks & 1) mma_16816<BF16>(sb, a, bq[ks][0], bq[ks][1]);
+                    else mma_16816<BF16>(sa, a, bq[ks][0], bq[ks][1]);
+                }
             }
             float v0 = (sa[0] + sb[0]) * p.scale_log2e, v1 = (sa[1] + sb[1]) * p.scale_log2e;
             float v2 = (sa[2] + sb[2]) * p.scale_log2e, v3 = (sa[3] + sb[3]) * p.scale_log2e;
@@ -815,18 +960,39 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 pl0 = movmatrix_trans(pack2<true>(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u)));
                 pl1 = movmatrix_trans(pack2<true>(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xffff0000u)));
             }
+            if constexpr (KV8) {
+                // the bytes of masked tokens need no clearing: every byte decodes to a finite number and their P is exactly 0
+                const uint32_t v0w[4] = {vv[0].x, vv[0].y, vv[0].z, vv[0].w}, v1w[4] = {vv[1].x, vv[1].y, vv[1].z, vv[1].w};
+                const uint32_t v2w[4] = {vv[2].x, vv[2].y, vv[2].z, vv[2].w}, v3w[4] = {vv[3].x, vv[3].y, vv[3].z, vv[3].w};
 #pragma unroll
-            for (int j = 0; j < D / 16; ++j) {
-                const int chunk = 2 * j + v_csel;
-                uint32_t a[4];
-                ldmatrix_x4_trans(
-                    tile_u32 + (chunk >> 3) * SM::HALF_BYTES + (16 + v_tok) * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), a);
-                mma_16816<BF16>(o[j], a, pb0, pb1);
-                if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
+                for (int j = 0; j < D / 16; ++j) {
+                    const int w = j >> 1;
+                    const uint32_t sel = (j & 1) ? 0x7632u : 0x5410u;  // bytes 2j, 2j+1 (mod 4) of the first, then of the second
+                    const uint32_t z01 = __byte_perm(v0w[w], v1w[w], sel), z23 = __byte_perm(v2w[w], v3w[w], sel);
+                    uint32_t a[4];
+                    a[0] = e4m3x2_lo_to_16x2<BF16>(z01 & 0x00ff00ffu);  // d = 16 g + 2 j of both tokens
+                    a[1] = e4m3x2_hi_to_16x2<BF16>(z01);                // d = 16 g + 2 j + 1
+                    a[2] = e4m3x2_lo_to_16x2<BF16>(z23 & 0x00ff00ffu);
+                    a[3] = e4m3x2_hi_to_16x2<BF16>(z23);
+                    mma_16816<BF16>(o[j], a, pb0, pb1);
+                    if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
+                }
+                __syncwarp();
+            } else {
+                const uint32_t tile_u32 = smem_base + stage * SM::RING_BYTES;
+#pragma unroll
+                for (int j = 0; j < D / 16; ++j) {
+                    const int chunk = 2 * j + v_csel;
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(
+                        tile_u32 + (chunk >> 3) * SM::HALF_BYTES + (16 + v_tok) * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), a);
+                    mma_16816<BF16>(o[j], a, pb0, pb1);
+                    if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
+                }
+                __syncwarp();
+                if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
             }
-            __syncwarp();
-            if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
         }
         gt += (uint32_t)it.ntiles;
 
@@ -840,10 +1006,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             float *w = mo + warp * 8 * SM::MO_STRIDE;
 #pragma unroll
             for (int j = 0; j < D / 16; ++j) {
-                w[c2 * SM::MO_STRIDE + 16 * j + r0] = o[j][0];
-                w[(c2 + 1) * SM::MO_STRIDE + 16 * j + r0] = o[j][1];
-                w[c2 * SM::MO_STRIDE + 16 * j + 8 + r0] = o[j][2];
-                w[(c2 + 1) * SM::MO_STRIDE + 16 * j + 8 + r0] = o[j][3];
+                // accumulator rows r0 and r0 + 8 of product j: d = 16 j + r0 (+ 8); 8-bit path: d = 16 r0 + 2 j (+ 1)
+                const int d0 = KV8 ? 16 * r0 + 2 * j : 16 * j + r0, d1 = KV8 ? d0 + 1 : d0 + 8;
+                w[c2 * SM::MO_STRIDE + d0] = o[j][0];
+                w[(c2 + 1) * SM::MO_STRIDE + d0] = o[j][1];
+                w[c2 * SM::MO_STRIDE + d1] = o[j][2];
+                w[(c2 + 1) * SM::MO_STRIDE + d1] = o[j][3];
             }
             if (lane < 4) {
                 ml[(warp * 8 + c2) * 2 + 0] = m0;
@@ -867,6 +1035,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 acc += mo[(w * 8 + g) * SM::MO_STRIDE + d] * wt;
                 ll += ml[(w * 8 + g) * 2 + 1] * wt;
             }
+            acc *= p.out_scale;  // 1 for 16-bit pools
             if (it.nchunks == 1) {
                 // the whole context in one chunk: normalise and round here
                 const float r = acc * (ll > 0.f ? 1.f / ll : 0.f);
@@ -1028,6 +1197,23 @@ cudaError_t make_pool_tensor_maps(void *gpu_pool, int64_t n_gpu_slots, int n_kv_
     return cudaSuccess;
 }
 
+// 8-bit pools: rows of 128 bytes (one token's K or V of one head, head_dim 128), 32 rows per tile.
+cudaError_t make_pool_tensor_map_fp8(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, CUtensorMap *map2d) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+    cuuint64_t dims[2] = {128, (cuuint64_t)n_gpu_slots * (cuuint64_t)n_kv_heads * 32u};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t box[2] = {128, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(map2d, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, gpu_pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 // Kernel variants (consumer warps, ring stages): more stages keep more bytes in flight per CTA, fewer let a third
 // CTA share the SM.  Variant 0 is the default.
 struct AttnVariant {
@@ -1035,10 +1221,22 @@ struct AttnVariant {
 };
 static const AttnVariant kVariants[] = {{2, 4}, {4, 8}, {2, 12}, {2, 6}, {4, 4}, {2, 8}, {1, 5}, {3, 6}, {1, 7}, {2, 4}, {1, 4}, {3, 3}, {1, 3}, {2, 2}};
 constexpr int kNumVariants = (int)(sizeof(kVariants) / sizeof(kVariants[0]));
+constexpr int kNumVariants8 = 2;
 
 template <typename F>
-static cudaError_t dispatch_variant(int head_dim, int dtype, int variant, F &&f) {
+static cudaError_t dispatch_variant(int head_dim, int dtype, int variant, int kv_fp8, F &&f) {
     if (variant < 0 || variant >= kNumVariants) return cudaErrorInvalidValue;
+    if (kv_fp8) {  // 8-bit blocks: head_dim 128; variants (consumer warps, stages of 4 KiB)
+        if (head_dim != 128 || variant >= kNumVariants8) return cudaErrorInvalidValue;
+#define PIE_VARIANT8(IDX, NWV, STV)                                                                                                      \
+    if (variant == IDX)                                                                                                                  \
+        return dtype == PIE_BF16 ? f(paged_decode_attn_kernel<128, true, STV, NWV, true>, AttnSmem<128, STV, NWV, true>::BYTES, NWV)   \
+                                 : f(paged_decode_attn_kernel<128, false, STV, NWV, true>, AttnSmem<128, STV, NWV, true>::BYTES, NWV);
+        PIE_VARIANT8(0, 2, 4)
+        PIE_VARIANT8(1, 2, 8)
+#undef PIE_VARIANT8
+        return cudaErrorInvalidValue;
+    }
 #define PIE_VARIANT(NWV, STV)                                                                       \
     if (kVariants[variant].nw == NWV && kVariants[variant].stages == STV) {                         \
         if (head_dim == 128) return dtype == PIE_BF16 ? f(paged_decode_attn_kernel<128, true, STV, NWV>, AttnSmem<128, STV, NWV>::BYTES, NWV) \
@@ -1079,10 +1277,10 @@ static cudaError_t prefer_max_shared() {
     return cudaSuccess;
 }
 
-cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_sm) {
+cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_sm, int kv_fp8) {
     cudaError_t e0 = prefer_max_shared();
     if (e0 != cudaSuccess) return e0;
-    return dispatch_variant(head_dim, dtype, variant, [&](auto kernel, int smem, int nw) -> cudaError_t {
+    return dispatch_variant(head_dim, dtype, variant, kv_fp8, [&](auto kernel, int smem, int nw) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, kernel, (nw + 1) * 32, smem);
@@ -1127,8 +1325,17 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.use3d = use3d;
     p.max_chunks = (int32_t)(sc.max_items / sh.n_kv_heads);
     p.scale_log2e = a.scale * 1.4426950408889634f;
+    if (sh.kv_fp8) {
+        p.k_scale = a.k_scale;
+        p.v_scale = p.out_scale = a.v_scale;
+        p.scale_log2e *= a.k_scale;  // scores over the stored keys are scores over the keys / k_scale
+        if (sh.dtype == PIE_F16) {   // the kernel's fp16 images of the bytes are the values / 256
+            p.scale_log2e *= KV8_F16_FACTOR;
+            p.out_scale *= KV8_F16_FACTOR;
+        }
+    }
     if (a.k_new == nullptr || a.v_new == nullptr) p.k_new = p.v_new = nullptr;
-    cudaError_t e = dispatch_variant(sh.head_dim, sh.dtype, a.variant, [&](auto kernel, int smem, int nw) -> cudaError_t {
+    cudaError_t e = dispatch_variant(sh.head_dim, sh.dtype, a.variant, sh.kv_fp8, [&](auto kernel, int smem, int nw) -> cudaError_t {
         kernel<<<a.grid, (nw + 1) * 32, smem, stream>>>(map, p);
         return cudaGetLastError();
     });

@@ -43,6 +43,7 @@ struct AttnShape {
     int n_q_heads, n_kv_heads;
     int n_logical;
     int64_t n_gpu_slots;
+    int kv_fp8 = 0;    // blocks hold E4M3 bytes (head_dim 128 only)
 };
 
 struct AttnScratch {
@@ -70,6 +71,7 @@ struct AttnLaunch {
     int32_t variant;            // kernel variant (0 = default)
     int32_t *status;            // device-visible status word
     uint64_t *stamps = nullptr; // optional, device-visible: [0] start, [1] end of the attention kernel (GPU timer, ns)
+    float k_scale = 1.f, v_scale = 1.f;  // 8-bit pools: a stored byte stands for decode(byte) * scale
 };
 
 // Build the TMA descriptors of the HBM pool: map3d covers a whole K+V tile in one copy
@@ -79,7 +81,8 @@ cudaError_t make_pool_tensor_maps(void *gpu_pool, int64_t n_gpu_slots, int n_kv_
                                   CUtensorMap *map2d, int *use3d);
 int attn_smem_bytes(int head_dim);
 int64_t attn_counter_words(int32_t max_seqs, int32_t n_kv_heads);
-cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_sm);
+cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_sm, int kv_fp8 = 0);
+cudaError_t make_pool_tensor_map_fp8(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, CUtensorMap *map2d);
 cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
                              int use3d, cudaStream_t stream);
 

@@ -58,6 +58,8 @@ struct ListRecord {
 struct pie_pool {
     pie_pool_config cfg{};
     int64_t block_bytes = 0;
+    int kv_fp8 = 0;                       // blocks hold E4M3 bytes (cfg.reserved[2])
+    float k_scale = 1.f, v_scale = 1.f;   // a stored byte stands for decode(byte) * scale
     pie::Table *table = nullptr;
     uint8_t *gpu_base = nullptr, *host_base = nullptr;
     bool own_gpu = false, own_host = false, own_streams = false;
@@ -562,8 +564,10 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
     pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
-                      p->cfg.n_gpu_slots};
+                      p->cfg.n_gpu_slots, p->kv_fp8};
     pie::AttnLaunch a{};
+    a.k_scale = p->k_scale;
+    a.v_scale = p->v_scale;
     a.q = q;
     a.out = out;
     a.block_table = bt_dev;
@@ -781,6 +785,8 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     if (cfg->dtype != PIE_F16 && cfg->dtype != PIE_BF16) return PIE_ERR_INVALID;
     if (cfg->block_tokens != 16 || (cfg->head_dim != 64 && cfg->head_dim != 128)) return PIE_ERR_UNSUPPORTED;
     if (cfg->n_q_heads / cfg->n_kv_heads > 8) return PIE_ERR_UNSUPPORTED;
+    if (cfg->reserved[2] != 0 && cfg->reserved[2] != 1) return PIE_ERR_INVALID;
+    if (cfg->reserved[2] == 1 && (cfg->head_dim != 128 || cfg->reserved[0] < 0 || cfg->reserved[0] > 1)) return PIE_ERR_UNSUPPORTED;
     if (cfg->split_tokens < 0 || cfg->split_tokens % 16 != 0) return PIE_ERR_INVALID;
     if (cfg->gpu_base && ((uintptr_t)cfg->gpu_base & 127)) return PIE_ERR_INVALID;
     if ((uint64_t)cfg->n_gpu_slots * (uint64_t)cfg->n_kv_heads * 32u > 0x7fffffffull) return PIE_ERR_UNSUPPORTED;
@@ -805,7 +811,8 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     // (measured: +6.5 % on 17 sequences of 4k-32k tokens with 8-head groups, -1.5 % on the batched shapes).
     if (p->cfg.split_tokens == 0)
         p->cfg.split_tokens = (int64_t)cfg->n_logical_blocks * 16 / std::max(cfg->max_seqs, 1) >= 6144 ? 1024 : 512;
-    p->block_bytes = (int64_t)2 * 16 * cfg->n_kv_heads * cfg->head_dim * 2;
+    p->kv_fp8 = cfg->reserved[2];
+    p->block_bytes = (int64_t)2 * 16 * cfg->n_kv_heads * cfg->head_dim * (p->kv_fp8 ? 1 : 2);
     p->n_sms = prop.multiProcessorCount;
     p->table = new (std::nothrow) pie::Table(cfg->n_layers, cfg->n_logical_blocks, cfg->n_gpu_slots, cfg->n_host_slots);
     if (!p->table) { destroy_pool(p); return PIE_ERR_NOMEM; }
@@ -893,13 +900,18 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     }
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_o, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
-    PIE_TRY(pie::make_pool_tensor_maps(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, cfg->head_dim, &p->map3d, &p->map2d,
-                                       &p->use3d),
-            PIE_ERR_CUDA);
-    if (const char *env = std::getenv("PIE_TMA_2D"))
-        if (env[0] == '1') p->use3d = 0;
+    if (p->kv_fp8) {
+        PIE_TRY(pie::make_pool_tensor_map_fp8(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, &p->map2d), PIE_ERR_CUDA);
+        p->use3d = 0;
+    } else {
+        PIE_TRY(pie::make_pool_tensor_maps(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, cfg->head_dim, &p->map3d, &p->map2d,
+                                           &p->use3d),
+                PIE_ERR_CUDA);
+        if (const char *env = std::getenv("PIE_TMA_2D"))
+            if (env[0] == '1') p->use3d = 0;
+    }
     int per_sm = 0;
-    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, cfg->reserved[0], &per_sm), PIE_ERR_CUDA);
+    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, cfg->reserved[0], &per_sm, p->kv_fp8), PIE_ERR_CUDA);
     if (per_sm <= 0) { destroy_pool(p); return PIE_ERR_UNSUPPORTED; }
     if (cfg->attn_ctas_per_sm > 0) per_sm = std::min(per_sm, cfg->attn_ctas_per_sm);
     p->attn_grid = per_sm * p->n_sms;
@@ -1295,6 +1307,7 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
     if (!pool || n_tokens < 0 || max_blocks_per_seq <= 0 || n_seqs <= 0) return PIE_ERR_INVALID;
     if (n_tokens > 0 && (!k || !v || !token_seq_dev || !token_pos_dev || !block_table_dev)) return PIE_ERR_INVALID;
     if (pool->sticky != PIE_OK) return pool->sticky;
+    if (pool->kv_fp8) return PIE_ERR_UNSUPPORTED;  // the scatter moves 16-bit vectors as they are
     if (layer < 0 || layer >= pool->cfg.n_layers) return PIE_ERR_RANGE;
     int st = poll(pool);
     if (st != PIE_OK) return st;
@@ -1325,6 +1338,14 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
     st = record_ticket(pool, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) pool->sticky = st;
     return st;
+}
+
+int pie_set_kv_scales(pie_pool *pool, float k_scale, float v_scale) {
+    if (!pool || !(k_scale > 0.f) || !(v_scale > 0.f) || !std::isfinite(k_scale) || !std::isfinite(v_scale)) return PIE_ERR_INVALID;
+    if (!pool->kv_fp8) return PIE_ERR_UNSUPPORTED;
+    pool->k_scale = k_scale;
+    pool->v_scale = v_scale;
+    return PIE_OK;
 }
 
 int pie_set_lookahead(pie_pool *pool, int32_t layers) {

@@ -55,6 +55,28 @@ __global__ void fill_slots_kernel(uint16_t *pool, const int64_t *__restrict__ sl
     }
 }
 
+// 8-bit pools: a byte with a random sign and mantissa and an exponent field of 3 .. 10 (never the all-ones one)
+__device__ __forceinline__ uint8_t draw_byte(uint64_t base, uint64_t idx) {
+    const uint64_t h = mix64(base + GOLDEN * (idx + 1ull));
+    return (uint8_t)(((h >> 32) & 0x87u) | ((((h >> 40) & 7u) + 3u) << 3));
+}
+
+__global__ void fill_slots_bytes_kernel(uint8_t *pool, const int64_t *__restrict__ slot_unit, int64_t n_slots, int64_t elems,
+                                        uint64_t base) {
+    const int64_t vec_per_slot = elems / 16;
+    const int64_t total = n_slots * vec_per_slot;
+    for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < total; v += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t slot = v / vec_per_slot;
+        const int64_t unit = slot_unit[slot];
+        if (unit < 0) continue;
+        const int64_t e0 = (v - slot * vec_per_slot) * 16;
+        uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int k = 0; k < 16; ++k) w[k >> 2] |= (uint32_t)draw_byte(base, (uint64_t)(unit * elems + e0 + k)) << (8 * (k & 3));
+        *reinterpret_cast<uint4 *>(pool + slot * elems + e0) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 __global__ void fill_tensor_kernel(uint16_t *dst, int64_t n, uint64_t base, uint64_t offset, int dtype, float gain) {
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         dst[i] = draw(base, offset + (uint64_t)i, dtype, gain);
@@ -71,6 +93,17 @@ PIE_SYNTH_API int pie_synth_fill_slots(void *pool, const int64_t *slot_unit, int
     const int64_t total = n_slots * (elems_per_slot / 8);
     const int grid = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     fill_slots_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((uint16_t *)pool, slot_unit, n_slots, elems_per_slot, base, dtype, gain);
+    return (int)cudaGetLastError();
+}
+
+// the same for pools whose elements are bytes (8-bit blocks)
+PIE_SYNTH_API int pie_synth_fill_slots_bytes(void *pool, const int64_t *slot_unit, int64_t n_slots, int64_t elems_per_slot,
+                                             uint64_t base, void *stream) {
+    if (n_slots <= 0) return 0;
+    if (elems_per_slot % 16 != 0) return (int)cudaErrorInvalidValue;
+    const int64_t total = n_slots * (elems_per_slot / 16);
+    const int grid = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    fill_slots_bytes_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((uint8_t *)pool, slot_unit, n_slots, elems_per_slot, base);
     return (int)cudaGetLastError();
 }
 

@@ -19,6 +19,8 @@ class DeviceWorkload:
     """A pool holding one workload's KV blocks, with the seeded host-resident choice established at
     allocation time and contents written by the generator kernels (so nothing is moved during set-up)."""
 
+    K_SCALE, V_SCALE = 0.25, 0.125    # scales of an 8-bit pool: the generator's bytes (|decoded| < 15) then stand for |k| < 4, |v| < 2
+
     def __init__(self, wl: synth.Workload, host_frac=None, timing=True, split_tokens=0, swap_ctas=0,
                  attn_ctas_per_sm=0, staging_layers=3, shuffle_table=False, extra_gpu_slots=0, extra_host_slots=0,
                  extra_tokens=None, attn_variant=0):
@@ -49,7 +51,9 @@ class DeviceWorkload:
             gpu_base=self.gpu_pool.data_ptr(), host_base=self.host_pool.data_ptr(), own_streams=0,
             compute_stream=self.s_compute.cuda_stream, copy_in_stream=self.s_in.cuda_stream,
             copy_out_stream=self.s_out.cuda_stream, split_tokens=split_tokens, swap_ctas=swap_ctas,
-            attn_ctas_per_sm=attn_ctas_per_sm, timing=int(timing), attn_variant=attn_variant)
+            attn_ctas_per_sm=attn_ctas_per_sm, timing=int(timing), attn_variant=attn_variant, kv_fp8=int(wl.kv_fp8))
+        if wl.kv_fp8:
+            pie.pie_set_kv_scales(self.pool, self.K_SCALE, self.V_SCALE)
         ids = pie.pie_block_alloc(self.pool, self.NB, on_host)
         assert np.array_equal(ids, np.arange(self.NB))
         self.fill_pools()
@@ -71,7 +75,7 @@ class DeviceWorkload:
     def fill_pools(self):
         wl = self.wl
         side, slot = pie.pie_get_placement(self.pool, wl.n_layers, self.NB)
-        elems = wl.block_bytes // 2
+        elems = wl.block_bytes // (1 if wl.kv_fp8 else 2)
         base = _u64(synth.stream_base(wl.seed, synth.STREAM_KV))
         units = np.arange(wl.n_layers * self.NB, dtype=np.int64).reshape(wl.n_layers, self.NB)
         lib = pie.synth_lib()
@@ -81,7 +85,10 @@ class DeviceWorkload:
             m = side == which
             slot_unit[slot[m]] = units[m]
             su = torch.from_numpy(slot_unit).to(self.dev)
-            rc = lib.pie_synth_fill_slots(ptr, su.data_ptr(), n_slots, elems, base, wl.dtype, 1.0, None)
+            if wl.kv_fp8:
+                rc = lib.pie_synth_fill_slots_bytes(ptr, su.data_ptr(), n_slots, elems, base, None)
+            else:
+                rc = lib.pie_synth_fill_slots(ptr, su.data_ptr(), n_slots, elems, base, wl.dtype, 1.0, None)
             assert rc == 0, f"fill_slots: cudaError {rc}"
             torch.cuda.synchronize()
 
@@ -158,7 +165,7 @@ class DeviceWorkload:
         """Algorithmic bytes of one layer call: valid KV tokens + q + out + table and lengths."""
         wl = self.wl
         ctx = self.ctx_lens.astype(np.int64)
-        kv = int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2
+        kv = int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * (1 if wl.kv_fp8 else 2)
         qo = 2 * wl.n_seqs * wl.n_q_heads * wl.head_dim * 2
         tab = 4 * (int(((ctx + 15) // 16).sum()) + wl.n_seqs)
         return kv + qo + tab

@@ -57,7 +57,7 @@ def run_steps(dw, n):
 
 def attention_bytes(wl, ctx):
     ctx = ctx.astype(np.int64)
-    return wl.n_layers * (int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * 2 + 2 * wl.n_seqs * wl.n_q_heads * wl.head_dim * 2
+    return wl.n_layers * (int(ctx.sum()) * 2 * wl.n_kv_heads * wl.head_dim * (1 if wl.kv_fp8 else 2) + 2 * wl.n_seqs * wl.n_q_heads * wl.head_dim * 2
                           + 4 * (int(((ctx + 15) // 16).sum()) + wl.n_seqs))
 
 
@@ -83,6 +83,8 @@ def main(argv=None):
                     help="how swap lists are moved (PIE_MODE_*)")
     ap.add_argument("--lookahead", type=int, default=1, help="layers prefetched ahead (pie_set_lookahead)")
     ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
+    ap.add_argument("--attn-variant", type=int, default=0, help="attention kernel variant (tuning)")
+    ap.add_argument("--kv-fp8", action="store_true", help="blocks of E4M3 bytes (half the bytes per token; head_dim 128)")
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
     out = open(args.out, "w") if args.out else sys.stdout
@@ -100,6 +102,8 @@ def main(argv=None):
         w_dst = torch.empty_like(w_src)
         OTHER["fn"] = lambda l: torch.add(w_src, 1.0, out=w_dst)
     wl = synth.workload(args.workload)
+    if args.kv_fp8:
+        wl = dataclasses.replace(wl, kv_fp8=True)
     if args.layers:
         wl = dataclasses.replace(wl, n_layers=args.layers)
     L = wl.n_layers
@@ -118,7 +122,7 @@ def main(argv=None):
         _, _, nb = wl.tables()
         # both pools can hold everything: ratio 0 needs it on the GPU side, ratio 1 on the host side
         dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb + 64, extra_host_slots=(L + 3) * nb + 64,
-                            split_tokens=args.split)
+                            split_tokens=args.split, attn_variant=args.attn_variant)
         dw.set_retention(args.kept_copies)
         pie.pie_set_lookahead(dw.pool, args.lookahead)
         emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,

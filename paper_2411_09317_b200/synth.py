@@ -123,6 +123,17 @@ def kv_unit_bits(seed: int, layer: int, block: int, n_logical_blocks: int, n_kv_
     return normal_bits(seed, STREAM_KV, idx, dtype, gain).reshape(n_kv_heads, 2, 16, head_dim)
 
 
+def kv_unit_bytes(seed: int, layer: int, block: int, n_logical_blocks: int, n_kv_heads: int, head_dim: int) -> np.ndarray:
+    """uint8 [Hkv][2][16][D] contents of one (layer, logical block) unit of an 8-bit pool: bytes with a random sign bit,
+    a random 3-bit mantissa and an exponent field of 3 .. 10 (so never the all-ones exponent)."""
+    idx = kv_unit_indices(layer, block, n_logical_blocks, n_kv_heads, head_dim)
+    base = stream_base(seed, STREAM_KV)
+    with np.errstate(over="ignore"):
+        h = mix64(base + GOLDEN * (idx + np.uint64(1)))
+    b = ((h >> np.uint64(32)) & np.uint64(0x87)) | ((((h >> np.uint64(40)) & np.uint64(7)) + np.uint64(3)) << np.uint64(3))
+    return b.astype(np.uint8).reshape(n_kv_heads, 2, 16, head_dim)
+
+
 def tensor_bits(seed: int, stream: int, shape, dtype: int, gain: float = 1.0, offset: int = 0) -> np.ndarray:
     n = int(np.prod(shape))
     idx = np.arange(n, dtype=np.uint64) + np.uint64(offset)
@@ -221,6 +232,7 @@ class Workload:
     decode_steps: int
     host_frac: float
     block_tokens: int = 16
+    kv_fp8: bool = False          # blocks hold one byte per element (an 8-bit variant) instead of the 16-bit type
 
     @property
     def n_seqs(self) -> int:
@@ -228,7 +240,7 @@ class Workload:
 
     @property
     def block_bytes(self) -> int:
-        return 2 * self.block_tokens * self.n_kv_heads * self.head_dim * 2
+        return 2 * self.block_tokens * self.n_kv_heads * self.head_dim * (1 if self.kv_fp8 else 2)
 
     def tables(self, shuffle: bool = False, extra_tokens: int | None = None):
         """Block table with room for `extra_tokens` decoded tokens per sequence (default: decode_steps)."""

@@ -21,7 +21,10 @@ class PoolCase:
         self.pool = pie.pie_pool_create(n_layers=L, n_q_heads=case.Hq, n_kv_heads=case.Hkv, head_dim=case.D,
                                         dtype=case.dtype, n_logical_blocks=NB, max_seqs=max(case.S, 1),
                                         n_gpu_slots=self.n_gpu_slots, n_host_slots=self.n_host_slots,
-                                        split_tokens=split_tokens, timing=timing, visible_blocks=visible_blocks)
+                                        split_tokens=split_tokens, timing=timing, visible_blocks=visible_blocks,
+                                        kv_fp8=int(getattr(case, "kv_fp8", False)))
+        if getattr(case, "kv_fp8", False):
+            pie.pie_set_kv_scales(self.pool, case.k_scale, case.v_scale)
         n0 = visible_blocks or NB          # with a smaller visible size only that many blocks exist at first
         ids = pie.pie_block_alloc(self.pool, n0, on_host[:n0])
         assert np.array_equal(ids, np.arange(n0))
@@ -58,7 +61,8 @@ class PoolCase:
         return bits, synth.bits16_to_f32(bits, self.c.dtype)
 
     def read_unit(self, l, b):
-        return pie.pie_block_read(self.pool, l, b).view(np.uint16)
+        raw = pie.pie_block_read(self.pool, l, b)
+        return raw if getattr(self.c, "kv_fp8", False) else raw.view(np.uint16)
 
     def close(self):
         if self.pool:
@@ -67,6 +71,11 @@ class PoolCase:
 
 
 def oracle_attention(case, layer, precision="f32"):
+    if getattr(case, "kv_fp8", False):
+        from oracle import fp8
+        return fp8.paged_attention(case.gpu_pool, case.host_pool, case.unit_side[layer], case.unit_slot[layer], case.q[layer],
+                                   case.block_table, case.ctx_lens, case.Hq, case.Hkv, case.D, case.dtype, case.scale,
+                                   case.k_scale, case.v_scale, precision=precision)
     return oracle.paged_attention(case.gpu_pool, case.host_pool, case.unit_side[layer], case.unit_slot[layer], case.q[layer],
                                   case.block_table, case.ctx_lens, case.Hq, case.Hkv, case.D, case.dtype, case.scale,
                                   precision=precision)

@@ -11,7 +11,9 @@ class Case:
 
     def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, dtype, ctx_lens, seed=0, host_frac=0.0,
                  placement="identity", n_gpu_slots=None, n_host_slots=None, gain=1.0, q_gain=1.0,
-                 shuffle_table=False, extra_tokens=0):
+                 shuffle_table=False, extra_tokens=0, kv_fp8=False, k_scale=0.25, v_scale=0.5):
+        # kv_fp8: the pools hold one byte per element (the 8-bit variant); a byte stands for its value times the scale
+        self.kv_fp8, self.k_scale, self.v_scale = kv_fp8, k_scale, v_scale
         self.L, self.Hq, self.Hkv, self.D, self.dtype = n_layers, n_q_heads, n_kv_heads, head_dim, dtype
         self.seed = seed
         self.ctx_lens = np.asarray(ctx_lens, dtype=np.int32)
@@ -20,7 +22,7 @@ class Case:
             self.ctx_lens, 16, extra_tokens=extra_tokens, shuffle_seed=seed if shuffle_table else None)
         self.NB = max(self.NB, 1)
         self.slot_elems = n_kv_heads * 2 * 16 * head_dim
-        self.block_bytes = self.slot_elems * 2
+        self.block_bytes = self.slot_elems * (1 if kv_fp8 else 2)
         host_ids = synth.pick_host_blocks(seed, self.block_table, self.nblk, host_frac)
         self.host_ids = host_ids
         on_host = np.zeros(self.NB, dtype=bool)
@@ -28,8 +30,8 @@ class Case:
         n_units = self.L * self.NB
         self.n_gpu_slots = n_gpu_slots or n_units
         self.n_host_slots = n_host_slots or max(1, n_units)
-        self.gpu_pool = np.zeros((self.n_gpu_slots, self.slot_elems), dtype=np.uint16)
-        self.host_pool = np.zeros((self.n_host_slots, self.slot_elems), dtype=np.uint16)
+        self.gpu_pool = np.zeros((self.n_gpu_slots, self.slot_elems), dtype=np.uint8 if kv_fp8 else np.uint16)
+        self.host_pool = np.zeros((self.n_host_slots, self.slot_elems), dtype=np.uint8 if kv_fp8 else np.uint16)
         self.unit_side = np.zeros((self.L, self.NB), dtype=np.int32)
         self.unit_slot = np.zeros((self.L, self.NB), dtype=np.int32)
         g_order = self._order(self.n_gpu_slots, placement, 11)
@@ -37,7 +39,10 @@ class Case:
         gi = hi = 0
         for l in range(self.L):
             for b in range(self.NB):
-                bits = synth.kv_unit_bits(seed, l, b, self.NB, n_kv_heads, head_dim, dtype, gain).ravel()
+                if kv_fp8:
+                    bits = synth.kv_unit_bytes(seed, l, b, self.NB, n_kv_heads, head_dim).ravel()
+                else:
+                    bits = synth.kv_unit_bits(seed, l, b, self.NB, n_kv_heads, head_dim, dtype, gain).ravel()
                 if on_host[b]:
                     slot = int(h_order[hi]); hi += 1
                     self.host_pool[slot] = bits

@@ -145,6 +145,48 @@ def test_llama3_8b_full_size_gqa_bf16_fixed_ratio():
     free(dw)
 
 
+def test_llama3_8b_full_size_8bit_blocks_hidden_swap_with_kept_copies():
+    """The 8-bit variant at full size: blocks of E4M3 bytes, 1.5 % of every layer's blocks host resident between uses with
+    their host copies kept; sampled outputs against the 8-bit oracle (append included), and the swapped bytes."""
+    from oracle import fp8
+    wl = dataclasses.replace(synth.workload("llama3_8b"), decode_steps=4, kv_fp8=True)
+    _, _, nb = wl.tables()
+    m = int(0.015 * nb)
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * m + 64, extra_host_slots=(wl.n_layers + 3) * m + 64)
+    assert pie.pie_block_bytes(dw.pool) == wl.block_bytes == 2 * 16 * wl.n_kv_heads * 128
+    dw.set_retention(True)
+    pie.pie_set_extension_ratio(dw.pool, 0.015)
+    steps = 3
+    for _ in range(steps):
+        dw.advance_context()
+        dw.decode_step()
+    dw.sync()
+    stats = pie.pie_get_stats(dw.pool)
+    assert stats["bytes_in"] >= (steps - 1) * wl.n_layers * m * wl.block_bytes
+    assert stats["reserved"][2] > 0                                   # unwritten blocks were not written back
+    got_all = dw.out_all.cpu().numpy().view(np.uint16)
+    order = np.argsort(wl.ctx_lens)
+    worst = 0.0
+    for layer, s in [(0, int(order[0])), (13, int(order[2])), (31, int(order[len(order) // 2]))]:
+        ctx = int(wl.ctx_lens[s]) + steps
+        nblk = (ctx + 15) // 16
+        pool = np.zeros((nblk, wl.block_bytes), dtype=np.uint8)
+        for i, b in enumerate(dw.block_table[s, :nblk]):
+            pool[i] = synth.kv_unit_bytes(wl.seed, layer, int(b), dw.NB, wl.n_kv_heads, wl.head_dim).ravel()
+        q, k_new, v_new = dw.step_inputs_host(0, layer)
+        side, slot = np.zeros(nblk, np.int32), np.arange(nblk, dtype=np.int32)
+        table = np.arange(nblk, dtype=np.int32)[None, :]
+        for t in range(1, steps + 1):
+            fp8.append(pool, pool, side, slot, k_new[s:s + 1], v_new[s:s + 1], table, np.array([int(wl.ctx_lens[s]) + t], np.int32),
+                       wl.n_kv_heads, wl.head_dim, wl.dtype, dw.K_SCALE, dw.V_SCALE)
+        want = fp8.paged_attention(pool, pool, side, slot, q[s:s + 1], table, np.array([ctx], np.int32), wl.n_q_heads,
+                                   wl.n_kv_heads, wl.head_dim, wl.dtype, 1.0 / np.sqrt(wl.head_dim), dw.K_SCALE, dw.V_SCALE)[0]
+        got = synth.bits16_to_f32(got_all[layer, s], wl.dtype)
+        worst = max(worst, float(np.abs(got - want).max()))
+        assert np.all(np.abs(got - want) <= TOL + 2.0 ** -8 * np.abs(want)), (layer, s, worst)
+    free(dw)
+
+
 def test_llama3_70b_shape_long_context_adaptive_controller():
     """GQA-8, contexts of 4k-32k tokens, half of the blocks host resident at the start (KV = 2x the HBM pool share),
     16 of the 80 layers to keep the pinned pool small; the adaptive controller owns the ratio."""

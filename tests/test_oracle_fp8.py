@@ -95,3 +95,14 @@ def test_append_quantises_and_writes_position_ctx_minus_one():
         # the stored value times the scale is within half an E4M3 step of the input (relative 2^-4, absolute 2^-10 * scale)
         assert np.all(np.abs(fp8.decode(tile[:, 0, pos % 16, :]) * 0.25 - kf) <= np.maximum(np.abs(kf) * 2.0 ** -4, 0.25 * 2.0 ** -10))
         assert np.all(np.abs(fp8.decode(tile[:, 1, pos % 16, :]) * 4.0 - vf) <= np.maximum(np.abs(vf) * 2.0 ** -4, 4.0 * 2.0 ** -10))
+
+
+def test_generated_bytes_are_finite_values_of_both_signs():
+    from paper_2411_09317_b200 import synth
+    b = synth.kv_unit_bytes(3, 1, 2, 10, 4, 128)
+    assert b.shape == (4, 2, 16, 128) and b.dtype == np.uint8
+    v = fp8.decode(b)
+    assert np.all(np.isfinite(v)) and (v < 0).any() and (v > 0).any()
+    assert 2.0 ** -4 <= np.abs(v).min() and np.abs(v).max() <= 15.0
+    assert len(np.unique(b)) > 100                       # signs, mantissas and eight exponents all occur
+    assert not np.array_equal(b, synth.kv_unit_bytes(3, 1, 3, 10, 4, 128))
