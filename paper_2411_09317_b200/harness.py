@@ -23,7 +23,7 @@ class DeviceWorkload:
 
     def __init__(self, wl: synth.Workload, host_frac=None, timing=True, split_tokens=0, swap_ctas=0,
                  attn_ctas_per_sm=0, staging_layers=3, shuffle_table=False, extra_gpu_slots=0, extra_host_slots=0,
-                 extra_tokens=None, attn_variant=0):
+                 extra_tokens=None, attn_variant=0, gpu_slots_override=0, host_slots_override=0, initial_host_blocks=0):
         self.wl = wl
         dev = torch.device("cuda", torch.cuda.current_device())
         self.dev = dev
@@ -32,6 +32,8 @@ class DeviceWorkload:
         self.block_table, self.nblk, self.NB = wl.tables(shuffle=shuffle_table, extra_tokens=self.extra_tokens)
         self.max_blocks = self.block_table.shape[1]
         self.host_ids = synth.pick_host_blocks(wl.seed, self.block_table, self.nblk, self.host_frac)
+        if initial_host_blocks:      # a given number of blocks starts on the host (a GPU pool smaller than the batch)
+            self.host_ids = synth.seeded_permutation(wl.seed, self.NB, salt=5)[:initial_host_blocks].astype(np.int32)
         on_host = np.zeros(self.NB, dtype=np.uint8)
         on_host[self.host_ids] = 1
         L, S = wl.n_layers, wl.n_seqs
@@ -39,6 +41,10 @@ class DeviceWorkload:
         staging = staging_layers * max(n_host_blocks, 1)
         self.n_gpu_slots = L * (self.NB - n_host_blocks) + staging + extra_gpu_slots
         self.n_host_slots = L * n_host_blocks + staging + extra_host_slots
+        if gpu_slots_override:
+            self.n_gpu_slots = max(gpu_slots_override, L * (self.NB - n_host_blocks) + 2)
+        if host_slots_override:
+            self.n_host_slots = max(host_slots_override, L * n_host_blocks + 2)
         BB = wl.block_bytes
         self.gpu_pool = torch.empty(self.n_gpu_slots * BB, dtype=torch.uint8, device=dev)
         self.host_pool = torch.empty(self.n_host_slots * BB, dtype=torch.uint8, pin_memory=True)

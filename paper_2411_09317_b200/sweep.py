@@ -11,6 +11,7 @@ ratios:   the extension ratio is set to 0, 0.1, ... 1.0 (fraction of every layer
 adaptive: the controller owns the ratio.  --host-frac 0.5 (default): half of the blocks start host resident and the GPU
           pool holds only the other half, so the ratio has a floor; --host-frac 0: everything starts on the GPU and the
           ratio climbs from 0 until waits or slow-down appear.  Per step: ratio, floor, step time, wait share.
+expansion: tokens per second against expansion (the batch grows, the GPU pool does not; --ratios lists expansions).
 layers:   whole layers on the CPU (the paper's protocol, Section 3.3) against the same share of every layer's blocks.
 interference: adaptive, with foreign pinned-memory traffic on the host link during the middle third of the run.
 Prints one JSON object per line.
@@ -64,7 +65,7 @@ def attention_bytes(wl, ctx):
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="llama3_8b")
-    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive", "interference", "layers"])
+    ap.add_argument("--mode", default="ratios", choices=["ratios", "adaptive", "interference", "layers", "expansion"])
     ap.add_argument("--cpu-layers", default="1,2,4", help="layers: numbers of layers kept on the CPU, comma list")
     ap.add_argument("--background-mb", type=int, default=256,
                     help="interference: pinned-memory traffic per step and direction on two other streams, MB")
@@ -111,6 +112,11 @@ def main(argv=None):
             "both_per_dir": pie.pie_probe_link(256 << 20, 2, 3)}
     if args.mode == "interference":
         interference(args, wl, link, emit)
+        return
+    if args.mode == "expansion":
+        emit({"workload": args.workload, "layers": L, "base_seqs": wl.n_seqs, "block_bytes": wl.block_bytes, "kept_copies": args.kept_copies,
+              "other_mb_per_layer": args.other_mb, "link": link})
+        expansion_throughput(args, wl, link, emit)
         return
     if args.mode == "layers":
         layers_vs_blocks(args, wl, link, emit)
@@ -215,6 +221,50 @@ def layers_vs_blocks(args, wl, link, emit):
                          "gb_in_per_step": (sa["bytes_in"] - sb["bytes_in"]) / args.steps / 1e9}
         emit(row)
     dw.close()
+
+
+def expansion_throughput(args, wl, link, emit):
+    """The paper's throughput-versus-expansion experiment (Section 5.4) in this build's terms: the GPU pool is fixed at what
+    the base batch needs; at expansion e the batch is e times as large (more sequences of the same length mix), the
+    surplus share r = 1 - 1/e of every layer's blocks lives on the host between uses, and what is reported is tokens per
+    second of the decode step (sequences / step time).  No request stream: the batch is full and steady, which is the
+    regime the paper's curves flatten into."""
+    base = wl.n_seqs
+    exps = [float(x) for x in args.ratios.split(",")] if args.ratios else [1.0, 1.02, 1.05, 1.1, 1.25, 1.5, 2.0]
+    _, _, nb_base = dataclasses.replace(wl, decode_steps=args.steps + 8).tables()
+    first = None
+    for e in exps:
+        n = max(base, int(round(base * e)))
+        big = dataclasses.replace(synth.workload(args.workload, scale=n / base), n_layers=wl.n_layers, decode_steps=args.steps + 8,
+                                  kv_fp8=wl.kv_fp8)
+        _, _, nb = big.tables()
+        r = max(0.0, 1.0 - nb_base / nb)
+        h = int(np.ceil(r * nb)) + 1
+        # GPU side: the base batch's blocks per layer, plus three layers' shares in transit; host side: the surplus
+        dw = DeviceWorkload(big, host_frac=0.0, timing=True, split_tokens=args.split, extra_gpu_slots=0, extra_host_slots=0,
+                            gpu_slots_override=wl.n_layers * nb_base + 3 * h + 64, host_slots_override=(wl.n_layers + 3) * h + 64,
+                            initial_host_blocks=h if r > 0 else 0)
+        dw.set_retention(args.kept_copies)
+        pie.pie_set_lookahead(dw.pool, args.lookahead)
+        pie.pie_set_extension_ratio(dw.pool, r)
+        run_steps(dw, 2)
+        per, sb, sa, ctx0, _ = run_steps(dw, args.steps)
+        ms = float(np.median(per))
+        tot = sum(per) * 1e-3
+        tps = big.n_seqs / (ms * 1e-3)
+        first = first or tps
+        emit({"expansion": nb / nb_base, "ratio": r, "seqs": big.n_seqs, "blocks_per_layer": nb, "ms_per_step": ms,
+              "tokens_per_s": tps, "vs_expansion_1": tps / first, "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9,
+              "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
+              "wait_share": sa["last_step_stall_ms"] / max(sa["last_step_ms"], 1e-9),
+              "gpu_pool_gb": dw.n_gpu_slots * big.block_bytes / 1e9, "host_pool_gb": dw.n_host_slots * big.block_bytes / 1e9})
+        dw.close()
+        for name in ("gpu_pool", "host_pool", "q_all", "out_all", "k_new", "v_new"):
+            setattr(dw, name, None)
+        del dw
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
 
 
 def interference(args, wl, link, emit):
