@@ -250,8 +250,9 @@ int pie_set_lookahead(pie_pool *pool, int32_t layers);
  * 16-bit type.  pie_decode_attention computes attention over the decoded values (scores and sums in fp32 as for 16-bit
  * pools; the key scale enters the softmax scale, the value scale the result); its append stores
  * E4M3(fp32(x) / scale), rounded to nearest (ties to the even code), magnitudes beyond 448 saturating, NaN -> 0x7f, and
- * the step's own attention already sees the stored (rounded) token.  A NaN byte (0x7f, 0xff) among the valid tokens is
- * outside the contract: the kernel reads it as +-480 (bytes beyond a sequence's length may hold anything).  Swapping, the table and the controller are
+ * the step's own attention already sees the stored (rounded) token.  Bytes beyond a sequence's length may hold anything.
+ * The products run in fp16 for both 16-bit types (every E4M3 value is an fp16 number); a bf16 query is scaled into
+ * fp16's range by a power of two per (sequence, KV head), exactly, so no finite query overflows.  Swapping, the table and the controller are
  * unchanged (they move block_bytes).  pie_kv_write returns PIE_ERR_UNSUPPORTED on such a pool.
  * PIE_ERR_INVALID unless both scales are finite and > 0; PIE_ERR_UNSUPPORTED on a 16-bit pool. */
 int pie_set_kv_scales(pie_pool *pool, float k_scale, float v_scale);

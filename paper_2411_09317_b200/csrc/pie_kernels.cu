@@ -512,40 +512,18 @@ __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
 }
 
-// Two E4M3 bytes -> two 16-bit values of the compute type, by moving bits instead of converting: E4M3's four exponent
-// bits become the low bits of the wider exponent field and its three mantissa bits the top of the wider mantissa;
-// subnormals stay subnormals of the same shape.  The result is the value times 2^-8 (fp16: the exponent bias goes from 7
-// to 15) or 2^-120 (bf16: 7 to 127).  bf16 multiplies the factor back at once (exact); fp16 leaves it in -
-// KV8_F16_FACTOR - and the launch folds 2^8 into the softmax scale and the value scale: every such value, down to the
-// smallest subnormal 2^-9 * 2^-8, is still an exact fp16 number.  The byte 0x7f / 0xff (E4M3's NaN) comes out as +-480.
-// Two forms, so that the integer work is shared between the ALU and the multiply-add pipe:
-//   hi: the bytes sit in the upper byte of each 16-bit half (what the lower bytes hold does not matter): shift right;
-//   lo: the bytes sit in the lower byte of each half, the upper bytes are zero: multiply up, then move the sign bit one
-//       place (fp16) or four places (bf16) further up by adding it again.
-constexpr float KV8_F16_FACTOR = 256.f;
-__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-__device__ __forceinline__ uint32_t bf16x2_times_2_120(uint32_t r) {
-    uint32_t o;
-    asm("mul.bf16x2 %0, %1, %2;" : "=r"(o) : "r"(r), "r"(0x7b807b80u));
-    return o;
-}
-template <bool BF16>
-__device__ __forceinline__ uint32_t e4m3x2_hi_to_16x2(uint32_t t) {
-    if (BF16) return bf16x2_times_2_120((t & 0x80008000u) | ((t >> 4) & 0x07f007f0u));
-    return (t & 0x80008000u) | ((t >> 1) & 0x3f803f80u);
-}
-template <bool BF16>
-__device__ __forceinline__ uint32_t e4m3x2_lo_to_16x2(uint32_t x) {
-    if (BF16) {
-        const uint32_t y = mad_u32(x, 16u, 0u);                       // sign at bit 11 of each half: 15 more of it -> bit 15
-        return bf16x2_times_2_120(mad_u32(y & 0x08000800u, 15u, y));
-    }
-    const uint32_t y = mad_u32(x, 128u, 0u);                          // sign at bit 14 of each half
-    return mad_u32(y & 0x40004000u, 1u, y);
+// The two low (HI = false) or high bytes of a word -> fp16 x 2 (exact) by the conversion instruction.  The 8-bit kernel
+// computes in fp16 whatever the pool's 16-bit type is: every E4M3 value is an fp16 number, the conversion has a pipe of
+// its own, and fp16 keeps 11 bits of P where bf16 needs a second product for P's rounding remainder.  A bf16 query is
+// brought into fp16's range by a power of two per work item (exact; undone in the softmax scale).  Measured on the way:
+// decoding by bit moves (shift exponent and mantissa into place, fix the bias by a factor) in the ALU 3.5-3.8 TB/s on the
+// fp16 MHA shape against 4.35-4.5 TB/s with the conversion instruction; bf16 operands built that way 3.0 TB/s.
+template <bool HI>
+__device__ __forceinline__ uint32_t e4m3x2_cvt_f16x2(uint32_t w) {
+    uint32_t r;
+    if (HI) asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, hi;\n\t}" : "=r"(r) : "r"(w));
+    else asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, lo;\n\t}" : "=r"(r) : "r"(w));
+    return r;
 }
 // two floats -> two E4M3 bytes (lo in the low byte): nearest even, saturating to +-448
 __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
@@ -562,6 +540,7 @@ template <int D, bool BF16, int STAGES, int NW, bool KV8 = false>
 __global__ void __launch_bounds__((NW + 1) * 32, KV8 ? 5 : 1)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p) {
     using SM = AttnSmem<D, STAGES, NW, KV8>;
+    constexpr bool MB = BF16 && !KV8;  // the tensor-core products run in bf16 (else fp16: always so for 8-bit pools)
     static_assert(!KV8 || D == 128, "8-bit blocks: head_dim 128 (one 128-byte row per token)");
     // A stage must always be consumed by the same warp: tile i goes to warp i % NW and to stage i % STAGES.  If two
     // warps alternated on a stage, the one running ahead could pass a parity wait on the phase before the one it
@@ -767,16 +746,38 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(smem + SM::OFF_Q + qs * SM::Q_BYTES) + g * (D / 2);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                if (KV8) {  // step 4 j + s reads d0 = 16 (4 j + t) + 4 s .. + 3 as k = d0, d0 + 2 | d0 + 1, d0 + 3: the K bytes' order below
+                if (KV8) {  // step 4 j + s reads d0 = 16 (4 j + t) + 4 s .. + 3 as k = d0, d0 + 1 | d0 + 2, d0 + 3: the K bytes' order below
                     const int w = 8 * (4 * (ks >> 2) + (lane & 3)) + 2 * (ks & 3);
-                    const uint32_t qa = g < p.group ? qrow[w] : 0u, qb = g < p.group ? qrow[w + 1] : 0u;
-                    bq[ks][0] = __byte_perm(qa, qb, 0x5410u);
-                    bq[ks][1] = __byte_perm(qa, qb, 0x7632u);
+                    bq[ks][0] = g < p.group ? qrow[w] : 0u;
+                    bq[ks][1] = g < p.group ? qrow[w + 1] : 0u;
                 } else {
                     bq[ks][0] = g < p.group ? qrow[ks * 8 + (lane & 3)] : 0u;
                     bq[ks][1] = g < p.group ? qrow[ks * 8 + 4 + (lane & 3)] : 0u;
                 }
             }
+        }
+        float sl2e = p.scale_log2e;
+        if constexpr (KV8 && BF16) {
+            // bf16 query, fp16 products: scale the item's query rows by the power of two that puts their largest magnitude
+            // into [2^14, 2^15) (exact; what falls below fp16's subnormals is 2^-38 of the largest and cannot show in an
+            // fp32 sum), convert, and give the factor back through the softmax scale
+            float mx = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    mx = fmaxf(mx, fmaxf(fabsf(__uint_as_float(bq[ks][h] << 16)), fabsf(__uint_as_float(bq[ks][h] & 0xffff0000u))));
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+            int sh = mx > 0.f ? (int)((__float_as_uint(mx) >> 23) & 0xffu) - 127 - 14 : 0;
+            sh = max(-100, min(100, sh));
+            const float down = __uint_as_float((uint32_t)(127 - sh) << 23);
+            sl2e *= __uint_as_float((uint32_t)(127 + sh) << 23);
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    bq[ks][h] = pack2<false>(__uint_as_float(bq[ks][h] << 16) * down, __uint_as_float(bq[ks][h] & 0xffff0000u) * down);
         }
         float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
         float o[D / 16][4];
@@ -803,7 +804,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 // tokens (output) do not care in which order their terms are fed to the tensor core, and neither does the
                 // output care which accumulator row holds which d, so every lane reads whole 16-byte pieces:
                 //   K: lane (g, t) reads pieces t and 4 + t of rows g and g + 8; word s of piece 4 j + t feeds step 4 j + s,
-                //      bytes 0, 2 as k = 2t, 2t+1 and bytes 1, 3 as k = 2t+8, 2t+9 (q is read with the same assignment);
+                //      bytes 0, 1 as k = 2t, 2t+1 and bytes 2, 3 as k = 2t+8, 2t+9 (q is read with the same assignment);
                 //   V: lane (g, t) reads piece g of the rows of tokens 2t, 2t+1, 2t+8, 2t+9; byte 2i (2i+1) of the piece is
                 //      accumulator row g (g + 8) of product i, that is d = 16 g + 2 i (+ 1).
                 uint8_t *ring = smem + stage * SM::RING_BYTES;
@@ -857,6 +858,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     const int tok = 2 * t + (j & 1) + 8 * (j >> 1);
                     vv[j] = *reinterpret_cast<const uint4 *>(ring + (16 + tok) * 128 + ((g ^ (tok & 7)) << 4));
                 }
+                if (nvalid < 16) {
+                    // masked tokens are excluded, not multiplied by zero (a NaN byte stays a NaN): clear their V bytes
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (2 * t + (j & 1) + 8 * (j >> 1) >= nvalid) vv[j] = make_uint4(0u, 0u, 0u, 0u);
+                }
                 __syncwarp();
                 if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 if (lane == 0) mbar_arrive(bar_empty + 8 * stage);  // everything is in registers: the stage may be refilled
@@ -869,12 +876,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     for (int s4 = 0; s4 < 4; ++s4) {
                         const int ks = 4 * j + s4;
                         uint32_t a[4];
-                        a[0] = e4m3x2_lo_to_16x2<BF16>(wg[s4] & 0x00ff00ffu);
-                        a[1] = e4m3x2_lo_to_16x2<BF16>(wh[s4] & 0x00ff00ffu);
-                        a[2] = e4m3x2_hi_to_16x2<BF16>(wg[s4]);
-                        a[3] = e4m3x2_hi_to_16x2<BF16>(wh[s4]);
-                        if (ks & 1) mma_16816<BF16>(sb, a, bq[ks][0], bq[ks][1]);
-                        else mma_16816<BF16>(sa, a, bq[ks][0], bq[ks][1]);
+                        a[0] = e4m3x2_cvt_f16x2<false>(wg[s4]);
+                        a[1] = e4m3x2_cvt_f16x2<false>(wh[s4]);
+                        a[2] = e4m3x2_cvt_f16x2<true>(wg[s4]);
+                        a[3] = e4m3x2_cvt_f16x2<true>(wh[s4]);
+                        if (ks & 1) mma_16816<MB>(sb, a, bq[ks][0], bq[ks][1]);
+                        else mma_16816<MB>(sa, a, bq[ks][0], bq[ks][1]);
                     }
                 }
             } else {
@@ -920,12 +927,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     const int chunk = 2 * ks + k_csel;
                     uint32_t a[4];
                     ldmatrix_x4(tile_u32 + (chunk >> 3) * SM::HALF_BYTES + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), a);
-                    if (ks & 1) mma_16816<BF16>(sb, a, bq[ks][0], bq[ks][1]);
-                    else mma_16816<BF16>(sa, a, bq[ks][0], bq[ks][1]);
+                    if (ks & 1) mma_16816<MB>(sb, a, bq[ks][0], bq[ks][1]);
+                    else mma_16816<MB>(sa, a, bq[ks][0], bq[ks][1]);
                 }
             }
-            float v0 = (sa[0] + sb[0]) * p.scale_log2e, v1 = (sa[1] + sb[1]) * p.scale_log2e;
-            float v2 = (sa[2] + sb[2]) * p.scale_log2e, v3 = (sa[3] + sb[3]) * p.scale_log2e;
+            float v0 = (sa[0] + sb[0]) * sl2e, v1 = (sa[1] + sb[1]) * sl2e;
+            float v2 = (sa[2] + sb[2]) * sl2e, v3 = (sa[3] + sb[3]) * sl2e;
             if (r0 >= nvalid) v0 = v1 = -INFINITY;
             if (r0 + 8 >= nvalid) v2 = v3 = -INFINITY;
             float x0 = fmaxf(v0, v2), x1 = fmaxf(v1, v3);
@@ -950,32 +957,31 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 o[j][3] *= a1;
             }
             // P^T as the B operand of O^T += V^T P^T: transpose the two 8x8 (token x head) blocks
-            const uint32_t h01 = pack2<BF16>(p0, p1), h23 = pack2<BF16>(p2, p3);
+            const uint32_t h01 = pack2<MB>(p0, p1), h23 = pack2<MB>(p2, p3);
             const uint32_t pb0 = movmatrix_trans(h01);
             const uint32_t pb1 = movmatrix_trans(h23);
             // bf16 keeps 8 significant bits: carry the rounding remainder of P in a second bf16 term so that the
             // PV product sees ~16 bits (fp16's 11 bits need no correction)
             uint32_t pl0 = 0, pl1 = 0;
-            if (BF16) {
+            if (MB) {
                 pl0 = movmatrix_trans(pack2<true>(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u)));
                 pl1 = movmatrix_trans(pack2<true>(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xffff0000u)));
             }
             if constexpr (KV8) {
-                // the bytes of masked tokens need no clearing: every byte decodes to a finite number and their P is exactly 0
                 const uint32_t v0w[4] = {vv[0].x, vv[0].y, vv[0].z, vv[0].w}, v1w[4] = {vv[1].x, vv[1].y, vv[1].z, vv[1].w};
                 const uint32_t v2w[4] = {vv[2].x, vv[2].y, vv[2].z, vv[2].w}, v3w[4] = {vv[3].x, vv[3].y, vv[3].z, vv[3].w};
 #pragma unroll
                 for (int j = 0; j < D / 16; ++j) {
                     const int w = j >> 1;
-                    const uint32_t sel = (j & 1) ? 0x7632u : 0x5410u;  // bytes 2j, 2j+1 (mod 4) of the first, then of the second
+                    const uint32_t sel = (j & 1) ? 0x7362u : 0x5140u;  // byte 2j (mod 4) of both tokens, then byte 2j+1 of both
                     const uint32_t z01 = __byte_perm(v0w[w], v1w[w], sel), z23 = __byte_perm(v2w[w], v3w[w], sel);
                     uint32_t a[4];
-                    a[0] = e4m3x2_lo_to_16x2<BF16>(z01 & 0x00ff00ffu);  // d = 16 g + 2 j of both tokens
-                    a[1] = e4m3x2_hi_to_16x2<BF16>(z01);                // d = 16 g + 2 j + 1
-                    a[2] = e4m3x2_lo_to_16x2<BF16>(z23 & 0x00ff00ffu);
-                    a[3] = e4m3x2_hi_to_16x2<BF16>(z23);
-                    mma_16816<BF16>(o[j], a, pb0, pb1);
-                    if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
+                    a[0] = e4m3x2_cvt_f16x2<false>(z01);  // d = 16 g + 2 j of tokens 2t, 2t+1
+                    a[1] = e4m3x2_cvt_f16x2<true>(z01);   // d = 16 g + 2 j + 1
+                    a[2] = e4m3x2_cvt_f16x2<false>(z23);  // the same of tokens 2t+8, 2t+9
+                    a[3] = e4m3x2_cvt_f16x2<true>(z23);
+                    mma_16816<MB>(o[j], a, pb0, pb1);
+                    if (MB) mma_16816<MB>(o[j], a, pl0, pl1);
                 }
                 __syncwarp();
             } else {
@@ -986,8 +992,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     uint32_t a[4];
                     ldmatrix_x4_trans(
                         tile_u32 + (chunk >> 3) * SM::HALF_BYTES + (16 + v_tok) * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), a);
-                    mma_16816<BF16>(o[j], a, pb0, pb1);
-                    if (BF16) mma_16816<BF16>(o[j], a, pl0, pl1);
+                    mma_16816<MB>(o[j], a, pb0, pb1);
+                    if (MB) mma_16816<MB>(o[j], a, pl0, pl1);
                 }
                 __syncwarp();
                 if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1329,10 +1335,6 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
         p.k_scale = a.k_scale;
         p.v_scale = p.out_scale = a.v_scale;
         p.scale_log2e *= a.k_scale;  // scores over the stored keys are scores over the keys / k_scale
-        if (sh.dtype == PIE_F16) {   // the kernel's fp16 images of the bytes are the values / 256
-            p.scale_log2e *= KV8_F16_FACTOR;
-            p.out_scale *= KV8_F16_FACTOR;
-        }
     }
     if (a.k_new == nullptr || a.v_new == nullptr) p.k_new = p.v_new = nullptr;
     cudaError_t e = dispatch_variant(sh.head_dim, sh.dtype, a.variant, sh.kv_fp8, [&](auto kernel, int smem, int nw) -> cudaError_t {
