@@ -444,7 +444,7 @@ def main():
     if wl.head_dim == 128:
         import dataclasses
         wl8 = dataclasses.replace(wl, kv_fp8=True)
-        n8, r8 = 8, 0.01
+        n8, r8 = 8, 0.0075
         dw = DeviceWorkload(wl8, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
                             attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=3 * int(r_cap * n_blocks) + 64,
                             extra_host_slots=(L + 3) * int(r_cap * n_blocks) + 64, extra_tokens=6 * (n8 + 2))
