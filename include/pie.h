@@ -51,6 +51,7 @@ enum { PIE_Q_NONE = 0, PIE_Q_IN = 1, PIE_Q_OUT = 2, PIE_Q_COMPUTE = 3 };
 typedef struct pie_pool pie_pool;
 typedef struct pie_table pie_table;
 typedef struct pie_fifo pie_fifo;
+typedef struct pie_governor pie_governor;
 
 typedef struct pie_pool_config {
     int32_t n_layers;
@@ -102,7 +103,9 @@ typedef struct pie_stats {
                                             * [3]: table-patch kernels launched after copy-engine lists (lists of few
                                             *      id runs patch the table by copy and launch none);
                                             * [1]: the smallest extension ratio the GPU pool's size allows with the
-                                            *      blocks allocated now (the controller never goes below it) */
+                                            *      blocks allocated now (the controller never goes below it);
+                                            * [4]: the throughput governor's cap on the ratio (1 = none; 0 before the
+                                            *      first pie_report_throughput), [5]: its state */
 } pie_stats;
 
 /* ---- pool (Section 3.1: the physical pools; Section 3.2: the mapping table) --------------------- */
@@ -412,6 +415,28 @@ int pie_fifo_location(pie_fifo *f, int32_t layer);
  * with every failed probe).  Returns the new ratio for one decode step's measurements (same unit for all three). */
 double pie_controller_decide(double *state, double ratio, double step, double stall, double compute,
                              double swap_busy);
+
+/* ---- performance records against throughput (Section 3.4.2, last paragraph) ------------------------------
+ * The stall-driven controller above cannot see whether a larger host-resident share buys anything: that shows only
+ * in the serving system's throughput.  The governor takes one report per window - the throughput seen at the ratio
+ * then in force, any unit - keeps the newest report per ratio (in units of `step`) and answers with a cap on the ratio
+ * (1.0 = none), which the controller respects.  NORMAL: no cap, until a report shows no gain (within tol) over the record
+ * one step below: the workload has stopped scaling with expansion, so stop increasing and test one step lower.
+ * TEST_DOWN: a report at the lowered cap that is not worse than the reference (within tol) keeps it and tries lower
+ * still; a worse one goes one step back up -> HOLD.  HOLD: every `period` reports, probe one step up.  PROBE_UP: better
+ * than the reference by more than tol -> NORMAL again; else back down -> HOLD.  Reports at a ratio other than the cap only
+ * update the records; `patience` of them in a row end a test at the ratio reported.
+ * Constants are this build's (the paper gives none): tol 0.02, period 8, patience 6 where the argument is <= 0.
+ * Host only, no CUDA.  pie_governor_state: *state 0 NORMAL, 1 TEST_DOWN, 2 HOLD, 3 PROBE_UP; *cap_steps -1 = no cap. */
+pie_governor *pie_governor_create(double step, double tol, int32_t period, int32_t patience);
+void pie_governor_destroy(pie_governor *g);
+double pie_governor_report(pie_governor *g, double ratio, double throughput);
+int pie_governor_state(const pie_governor *g, int32_t *state, int32_t *cap_steps);
+/* The same inside a pool in adaptive mode: report the window's throughput (e.g. tokens per second); the pool's ratio is
+ * held at or below the governor's cap from the next controller tick on (and never below what the GPU pool's size
+ * allows).  The governor's step is the controller's (pie_set_controller).  pie_stats.reserved[4] = the cap (1 = none),
+ * reserved[5] = the governor's state.  PIE_ERR_INVALID for a throughput that is not finite or negative. */
+int pie_report_throughput(pie_pool *pool, double throughput);
 
 #ifdef __cplusplus
 }

@@ -160,3 +160,77 @@ def fake_clock_step(r, bytes_layer, bw, t_compute_layer, n_layers):
     t_in = r * bytes_layer / bw
     stall_per_layer = max(0.0, t_in - t_compute_layer)
     return stall_per_layer * n_layers, t_compute_layer * n_layers, t_in * n_layers
+
+
+# ---------------------------------------------------------------------------------------------
+# Performance records against throughput (Section 3.4.2, last paragraph).  The serving system reports the
+# throughput it saw over a window at the ratio then in force; the governor keeps the newest report per ratio
+# (in units of the controller's step) and turns the paragraph's three sentences into a cap on the ratio,
+# which the stall-driven controller above then respects (it may stay below the cap, never above):
+#   NORMAL   no cap.  When a report at ratio k shows no gain over the record one step below
+#            (T[k] <= T[k-1] (1 + tol)), the workload has stopped scaling with expansion: stop increasing and
+#            test whether decreasing has any adverse effect -> TEST_DOWN with the cap one step lower.
+#   TEST_DOWN a report at the lowered cap: not worse than the reference (>= ref (1 - tol)) -> no adverse effect,
+#            keep it and try one step lower still (at 0: HOLD); worse -> one step back up, HOLD.
+#   HOLD     the cap stays.  Every `period` reports (low demand, spare bandwidth) -> PROBE_UP: cap one step up.
+#   PROBE_UP a report at the raised cap: better than the reference by more than tol -> the workload scales
+#            again: NORMAL; else one step back down, HOLD ("reduces it if the workload remains low").
+# Reports at a ratio other than the cap (the controller has not got there, or was pushed below it by stalls)
+# only update the records; `patience` such reports in a row end a test (TEST_DOWN, PROBE_UP -> HOLD at the
+# ratio reported).  Constants are the build's: tol = 0.02, period = 8, patience = 6.
+# ---------------------------------------------------------------------------------------------
+
+NORMAL, TEST_DOWN, HOLD, PROBE_UP = 0, 1, 2, 3
+
+
+@dataclasses.dataclass
+class Governor:
+    step: float
+    tol: float = 0.02
+    period: int = 8
+    patience: int = 6
+    k_max: int = 1 << 30
+    state: int = NORMAL
+    cap: int = 1 << 30            # in steps; k_max = no cap
+    ref: float = 0.0              # throughput the running test compares with
+    since: int = 0                # reports since HOLD began
+    off: int = 0                  # reports in a row at a ratio other than the cap during a test
+    rec: dict = dataclasses.field(default_factory=dict)
+
+    def cap_ratio(self):
+        return 1.0 if self.cap >= self.k_max else self.cap * self.step
+
+    def report(self, ratio, throughput):
+        """One window's throughput at `ratio` -> the cap (as a ratio; 1.0 = none)."""
+        k = int(round(ratio / self.step))
+        self.rec[k] = throughput
+        if self.state == NORMAL:
+            if k > 0 and (k - 1) in self.rec and throughput <= self.rec[k - 1] * (1 + self.tol):
+                self.state, self.cap, self.ref, self.off = TEST_DOWN, k - 1, throughput, 0
+        elif self.state == TEST_DOWN:
+            if k != self.cap:
+                self.off += 1
+                if self.off >= self.patience:
+                    self.state, self.cap, self.since, self.off = HOLD, k, 0, 0
+            elif throughput >= self.ref * (1 - self.tol):
+                self.ref, self.off = max(self.ref, throughput), 0
+                if self.cap > 0:
+                    self.cap -= 1
+                else:
+                    self.state, self.since = HOLD, 0
+            else:
+                self.state, self.cap, self.since, self.off = HOLD, self.cap + 1, 0, 0
+        elif self.state == HOLD:
+            self.since += 1
+            if self.since >= self.period:
+                self.state, self.ref, self.cap, self.off = PROBE_UP, throughput, self.cap + 1, 0
+        else:  # PROBE_UP
+            if k != self.cap:
+                self.off += 1
+                if self.off >= self.patience:
+                    self.state, self.cap, self.since, self.off = HOLD, k, 0, 0
+            elif throughput > self.ref * (1 + self.tol):
+                self.state, self.cap, self.rec = NORMAL, self.k_max, {k: throughput}
+            else:
+                self.state, self.cap, self.since, self.off = HOLD, self.cap - 1, 0, 0
+        return self.cap_ratio()

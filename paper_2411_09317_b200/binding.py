@@ -37,6 +37,7 @@ EXPORTS = [
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
     "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
+    "pie_governor_create", "pie_governor_destroy", "pie_governor_report", "pie_governor_state", "pie_report_throughput",
 ]
 
 
@@ -119,6 +120,11 @@ _sig = {
     "pie_set_retention": (_i32, [_vp, _i32]),
     "pie_set_lookahead": (_i32, [_vp, _i32]),
     "pie_set_kv_scales": (_i32, [_vp, ctypes.c_float, ctypes.c_float]),
+    "pie_governor_create": (_vp, [_f64, _f64, _i32, _i32]),
+    "pie_governor_destroy": (None, [_vp]),
+    "pie_governor_report": (_f64, [_vp, _f64, _f64]),
+    "pie_governor_state": (_i32, [_vp, _vp, _vp]),
+    "pie_report_throughput": (_i32, [_vp, _f64]),
     "pie_decode_layer": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _i32, _f32, _vp, _vp, _i32]),
     "pie_kv_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i64, _vp, _i32, _i32]),
     "pie_declare_append_blocks": (_i32, [_vp, _vp, _i64]),
@@ -200,6 +206,31 @@ def pie_set_lookahead(pool, layers) -> None:
 
 def pie_set_kv_scales(pool, k_scale, v_scale) -> None:
     check(lib.pie_set_kv_scales(pool, k_scale, v_scale), "pie_set_kv_scales")
+
+
+def pie_report_throughput(pool, throughput) -> None:
+    check(lib.pie_report_throughput(pool, throughput), "pie_report_throughput")
+
+
+class Governor:
+    """Throughput records (host only): report(ratio, throughput) -> cap on the ratio (1.0 = none)."""
+
+    def __init__(self, step, tol=0.0, period=0, patience=0):
+        self.h = lib.pie_governor_create(step, tol, period, patience)
+        assert self.h
+
+    def report(self, ratio, throughput) -> float:
+        return lib.pie_governor_report(self.h, ratio, throughput)
+
+    def state(self):
+        s, c = np.zeros(1, np.int32), np.zeros(1, np.int32)
+        check(lib.pie_governor_state(self.h, _ptr(s), _ptr(c)), "pie_governor_state")
+        return int(s[0]), int(c[0])
+
+    def close(self):
+        if self.h:
+            lib.pie_governor_destroy(self.h)
+            self.h = None
 
 
 def pie_set_retention(pool, on) -> None:

@@ -98,6 +98,8 @@ struct pie_pool {
     int ratio_mode = 0;  // 0 unset (keep the caller's sets), 1 fixed, 2 adaptive
     double ratio = 0.0;
     double ctrl_state[16] = {};
+    pie_governor *governor = nullptr;   // throughput records (pie_report_throughput); created at the first report
+    double ratio_cap = 1.0;
     double ctrl_step = 0.0;  // 0: one layer's worth, 1 / n_layers
     int32_t lookahead = 1;   // how many layers ahead the decode loop prefetches (Section 3.4.2 uses 1)
     bool poll_hold = false;  // a decode step is polling once per layer: nested calls skip theirs
@@ -492,6 +494,7 @@ void destroy_pool(pie_pool *p) {
     if (p->list_host) cudaFreeHost(p->list_host);
     if (p->status_host) cudaFreeHost(p->status_host);
     if (p->stamps_host) cudaFreeHost(p->stamps_host);
+    if (p->governor) pie_governor_destroy(p->governor);
     cudaFree(p->scratch.chunk_off);
     cudaFree(p->scratch.counters);
     cudaFree(p->scratch.part_o);
@@ -1216,7 +1219,8 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         // the rule never asks for less than the GPU pool's size allows: below that floor the number would drift
         // away from what the layers actually keep on the host
         const double r = std::max(ratio_floor(pool),
-                                  pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall + slow, compute, std::max(t_in, t_out)));
+                                  std::min(pool->ratio_cap, pie_controller_decide(pool->ctrl_state, pool->ratio, step, stall + slow,
+                                                                                  compute, std::max(t_in, t_out))));
         if (r != pool->ratio) {
             pool->ratio = r;
             if (changed) *changed = 1;
@@ -1338,6 +1342,21 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
     st = record_ticket(pool, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) pool->sticky = st;
     return st;
+}
+
+int pie_report_throughput(pie_pool *pool, double throughput) {
+    if (!pool || !std::isfinite(throughput) || throughput < 0) return PIE_ERR_INVALID;
+    const double step = pool->ctrl_step > 0 ? pool->ctrl_step : 1.0 / (double)pool->cfg.n_layers;
+    if (!pool->governor) {
+        pool->governor = pie_governor_create(step, 0, 0, 0);
+        if (!pool->governor) return PIE_ERR_NOMEM;
+    }
+    pool->ratio_cap = pie_governor_report(pool->governor, pool->ratio, throughput);
+    int32_t state = 0;
+    pie_governor_state(pool->governor, &state, nullptr);
+    pool->stats.reserved[4] = pool->ratio_cap;
+    pool->stats.reserved[5] = state;
+    return PIE_OK;
 }
 
 int pie_set_kv_scales(pie_pool *pool, float k_scale, float v_scale) {

@@ -3,7 +3,9 @@
 #include "pie_table.h"
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
+#include <map>
 #include <new>
 
 namespace pie {
@@ -625,3 +627,98 @@ double pie_controller_decide(double *state, double ratio, double step, double st
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Performance records against throughput (Section 3.4.2, last paragraph): a cap on the ratio from the
+// throughput the serving system reports per window.  NORMAL: no cap, until a report shows no gain over the
+// record one step below (the workload has stopped scaling): stop increasing and test one step lower.
+// TEST_DOWN: not worse than the reference -> keep it and try lower still; worse -> one step back up, HOLD.
+// HOLD: every `period` reports probe one step up.  PROBE_UP: better by more than tol -> NORMAL again, else back
+// down and HOLD.  Reports at a ratio other than the cap only update the records; `patience` of them in a row
+// end a test at the ratio reported.
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct Governor {
+    enum { NORMAL = 0, TEST_DOWN = 1, HOLD = 2, PROBE_UP = 3 };
+    static constexpr int K_MAX = 1 << 30;
+    double step, tol;
+    int period, patience;
+    int state = NORMAL, cap = K_MAX, since = 0, off = 0;
+    double ref = 0.0;
+    std::map<int, double> rec;
+    double cap_ratio() const { return cap >= K_MAX ? 1.0 : cap * step; }
+    double report(double ratio, double throughput) {
+        const int k = (int)std::llround(ratio / step);
+        rec[k] = throughput;
+        switch (state) {
+        case NORMAL: {
+            auto below = rec.find(k - 1);
+            if (k > 0 && below != rec.end() && throughput <= below->second * (1 + tol)) {
+                state = TEST_DOWN;
+                cap = k - 1;
+                ref = throughput;
+                off = 0;
+            }
+            break;
+        }
+        case TEST_DOWN:
+            if (k != cap) {
+                if (++off >= patience) { state = HOLD; cap = k; since = 0; off = 0; }
+            } else if (throughput >= ref * (1 - tol)) {
+                ref = std::max(ref, throughput);
+                off = 0;
+                if (cap > 0) --cap;
+                else { state = HOLD; since = 0; }
+            } else {
+                state = HOLD;
+                cap = cap + 1;
+                since = 0;
+                off = 0;
+            }
+            break;
+        case HOLD:
+            if (++since >= period) { state = PROBE_UP; ref = throughput; cap = cap + 1; off = 0; }
+            break;
+        default:  // PROBE_UP
+            if (k != cap) {
+                if (++off >= patience) { state = HOLD; cap = k; since = 0; off = 0; }
+            } else if (throughput > ref * (1 + tol)) {
+                state = NORMAL;
+                cap = K_MAX;
+                rec.clear();
+                rec[k] = throughput;
+            } else {
+                state = HOLD;
+                cap = cap - 1;
+                since = 0;
+                off = 0;
+            }
+        }
+        return cap_ratio();
+    }
+};
+}  // namespace
+
+extern "C" {
+pie_governor *pie_governor_create(double step, double tol, int32_t period, int32_t patience) {
+    if (!(step > 0)) return nullptr;
+    Governor *g = new (std::nothrow) Governor();
+    if (!g) return nullptr;
+    g->step = step;
+    g->tol = tol > 0 ? tol : 0.02;
+    g->period = period > 0 ? period : 8;
+    g->patience = patience > 0 ? patience : 6;
+    return reinterpret_cast<pie_governor *>(g);
+}
+void pie_governor_destroy(pie_governor *g) { delete reinterpret_cast<Governor *>(g); }
+double pie_governor_report(pie_governor *g, double ratio, double throughput) {
+    return g ? reinterpret_cast<Governor *>(g)->report(ratio, throughput) : 1.0;
+}
+int pie_governor_state(const pie_governor *g, int32_t *state, int32_t *cap_steps) {
+    if (!g) return PIE_ERR_INVALID;
+    const Governor *gg = reinterpret_cast<const Governor *>(g);
+    if (state) *state = gg->state;
+    if (cap_steps) *cap_steps = gg->cap >= Governor::K_MAX ? -1 : gg->cap;
+    return PIE_OK;
+}
+}

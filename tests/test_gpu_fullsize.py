@@ -263,3 +263,37 @@ def test_step_timing_from_gpu_timer_stamps_and_timeline():
     del dw
     gc.collect()
     torch.cuda.empty_cache()
+
+
+def test_throughput_reports_cap_the_ratio_when_expansion_buys_nothing():
+    """Adaptive mode on a workload that fits: with no reports the stall-driven controller lets the ratio climb while the
+    link has slack; once the caller reports a throughput that does not grow with the ratio, the governor's cap walks it
+    back down and holds it there, with a probe one step up per period (Section 3.4.2, last paragraph)."""
+    lens = np.full(16, 4096, dtype=np.int32)
+    steps_a, steps_b = 14, 40
+    wl = synth.Workload("governed", 9, 4, 8, 8, 128, synth.F16, lens, steps_a + steps_b + 4, 0.0)
+    nb = int(((lens.astype(np.int64) + wl.decode_steps + 15) // 16).sum())
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb, extra_host_slots=5 * nb)
+    step = 1.0 / 1024                                      # four blocks of every layer per step
+    pie.pie_set_controller(dw.pool, step, 0.5, 0.0)       # a tolerant stall rule: these layers take only 50 us
+    pie.pie_set_extension_ratio(dw.pool, -1.0)
+    for _ in range(steps_a):
+        dw.advance_context()
+        dw.decode_step()
+    climbed = pie.pie_get_extension_ratio(dw.pool)
+    assert climbed >= 3 * step - 1e-9, climbed
+    ratios = []
+    for _ in range(steps_b):
+        dw.advance_context()
+        dw.decode_step()
+        pie.pie_report_throughput(dw.pool, 1000.0)            # the same whatever the ratio
+        ratios.append(pie.pie_get_extension_ratio(dw.pool))
+    dw.sync()
+    stats = pie.pie_get_stats(dw.pool)
+    assert max(ratios[-12:]) <= step + 1e-9, ratios
+    assert stats["reserved"][4] <= step + 1e-9 and stats["reserved"][5] in (2.0, 3.0)
+    with pytest.raises(pie.PieError) as e:
+        pie.pie_report_throughput(dw.pool, float("nan"))
+    assert e.value.status == pie.PIE_ERR_INVALID
+    check_samples(dw, [(0, 0), (3, 5)], steps_a + steps_b)
+    free(dw)

@@ -247,3 +247,31 @@ def test_controller_rule_matches_oracle(bw, tc, bytes_layer, L):
         want = c.tick(*m)
         r = pie.pie_controller_decide(state, r, 1.0 / L, *m)
         assert r == pytest.approx(want, abs=1e-12), i
+
+
+# ------------------------------------------------------------------- throughput governor: C++ against the oracle
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_governor_matches_oracle_on_random_reports(seed):
+    """Random walks of (ratio, throughput) reports - rising, flat, falling and noisy stretches, ratios that follow the
+    cap and ratios that do not: state and cap agree after every report."""
+    from oracle.policy import Governor
+    rng = np.random.default_rng(seed)
+    step = [0.01, 1.0 / 32, 0.002, 0.05][seed]
+    og, cg = Governor(step), pie.Governor(step)
+    k, base, slope, sat = 0, 100.0, 800.0, int(rng.integers(0, 12))
+    for i in range(600):
+        if i % 97 == 96:                                   # the workload changes
+            sat, slope = int(rng.integers(0, 12)), float(rng.choice([0.0, 300.0, 3000.0]))
+        t = (base + slope * step * min(k, sat)) * (1 + float(rng.uniform(-0.01, 0.01)))
+        want = og.report(k * step, t)
+        got = cg.report(k * step, t)
+        state, cap = cg.state()
+        assert (state, cap) == (og.state, -1 if og.cap >= og.k_max else og.cap), i
+        assert got == want
+        move = rng.integers(0, 4)
+        target = og.cap if move else int(rng.integers(0, 14))     # mostly follow the cap, sometimes not
+        if k < min(target, 20):
+            k += 1
+        elif k > target:
+            k -= 1
+    cg.close()

@@ -541,3 +541,75 @@ def test_controller_tolerates_one_disturbed_step():
     assert c.tick(0.5, 1.0, 0.5) == r           # a single stall: no change
     assert c.tick(0.0, 1.0, 0.95) == r          # quiet again, link nearly full: hold
     assert c.tick(0.5, 1.0, 0.5) == pytest.approx(r - 0.1)  # second stall within the window: back off
+
+
+# ------------------------------------------------------------------- throughput records (Section 3.4.2, last paragraph)
+def _drive_governor(T, n, step=0.01, stuck_at=None, g=None, k=0):
+    """Reports of a synthetic throughput curve T(ratio, i) to a governor; between reports the ratio moves one step
+    toward the cap, as a stall-free controller would (or stays at `stuck_at` steps where stalls hold it)."""
+    from oracle.policy import Governor
+    g = g or Governor(step)
+    trace = []
+    for i in range(n):
+        g.report(k * step, T(k * step, i))
+        target = g.cap if stuck_at is None else min(g.cap, stuck_at)
+        if k < min(target, 100):
+            k += 1
+        elif k > target:
+            k = target
+        trace.append((k, g.state, g.cap))
+    return g, k, trace
+
+
+def test_governor_stops_where_the_workload_stops_scaling():
+    from oracle.policy import HOLD
+    # throughput grows with the ratio up to 0.05, flat beyond: the paragraph's "stops scaling"
+    g, k, trace = _drive_governor(lambda r, i: 100 + 1000 * min(r, 0.05), 12)
+    # climbed to 6 steps, saw no gain over 5, tested 5 (no adverse effect), tested 4 (worse), back to 5
+    assert [t[0] for t in trace[:9]] == [1, 2, 3, 4, 5, 6, 5, 4, 5]
+    assert (k, g.state, g.cap) == (5, HOLD, 5)
+
+
+def test_governor_walks_down_when_expansion_buys_nothing_and_probes_periodically():
+    from oracle.policy import HOLD, PROBE_UP
+    g, k, trace = _drive_governor(lambda r, i: 100.0, 40)
+    assert (k, g.cap) == (0, 0) and g.state in (HOLD, PROBE_UP)
+    probes = [i for i, t in enumerate(trace) if t[1] == PROBE_UP]
+    assert len(probes) >= 3 and all(b - a == g.period + 1 for a, b in zip(probes, probes[1:]))   # one probe per period
+    assert max(t[0] for t in trace[3:]) == 1                                                     # never more than one step up
+
+
+def test_governor_follows_demand_that_comes_back():
+    from oracle.policy import HOLD
+    g, k, trace = _drive_governor(lambda r, i: 100.0 if i < 30 else 100 + 1000 * min(r, 0.08), 90)
+    assert all(t[0] <= 1 for t in trace[3:30])
+    assert (k, g.cap) == (8, 8) or (k, g.cap) == (9, 9)        # at the new saturation point (or on a probe one above it)
+    assert max(t[0] for t in trace) == 9
+
+
+def test_governor_ignores_noise_within_its_tolerance():
+    import numpy as np
+    rng = np.random.default_rng(3)
+    noise = rng.uniform(-0.004, 0.004, 400)
+    # 10 % more throughput per step up to 0.05: far above the tolerance; +-0.4 % noise: far below
+    g, k, trace = _drive_governor(lambda r, i: (100 + 1000 * min(r, 0.05)) * (1 + noise[i]), 400)
+    assert all(4 <= t[0] <= 6 for t in trace[10:])
+
+
+def test_governor_ends_a_test_the_controller_cannot_follow():
+    from oracle.policy import Governor, HOLD, PROBE_UP, NORMAL
+    # a ratio that stalls hold at 2 steps while throughput still grows with it: nothing to compare above 2, no cap
+    g, k, _ = _drive_governor(lambda r, i: 100.0 + 1000 * r, 60, stuck_at=2)
+    assert k == 2 and g.state == NORMAL and g.cap_ratio() == 1.0
+    # flat throughput: down to 0 and HOLD; then the probe one step up cannot be followed (the ratio stays at 0):
+    # after `patience` reports away from the cap the test ends where the ratio is
+    g = Governor(0.01)
+    g, k, _ = _drive_governor(lambda r, i: 100.0, 4, g=g)
+    assert (k, g.state, g.cap) == (0, HOLD, 0)
+    seen = []
+    for i in range(g.period + g.patience):
+        g.report(0.0, 100.0)
+        seen.append((g.state, g.cap))
+    first = seen.index((PROBE_UP, 1))
+    assert first in (g.period - 2, g.period - 1)                      # one probe per period of reports in HOLD
+    assert seen[first + g.patience - 1] == (PROBE_UP, 1) and seen[first + g.patience] == (HOLD, 0)
