@@ -949,12 +949,16 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             m1 = n1;
             l0 = l0 * a0 + (p0 + p2);
             l1 = l1 * a1 + (p1 + p3);
+            // (8-bit kernel, bound by its instruction stream: once the running maxima have settled both factors are exactly 1
+            // in every lane and the 32 multiplications can go - the same bits either way)
+            if (!KV8 || __any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {
 #pragma unroll
-            for (int j = 0; j < D / 16; ++j) {
-                o[j][0] *= a0;
-                o[j][1] *= a1;
-                o[j][2] *= a0;
-                o[j][3] *= a1;
+                for (int j = 0; j < D / 16; ++j) {
+                    o[j][0] *= a0;
+                    o[j][1] *= a1;
+                    o[j][2] *= a0;
+                    o[j][3] *= a1;
+                }
             }
             // P^T as the B operand of O^T += V^T P^T: transpose the two 8x8 (token x head) blocks
             const uint32_t h01 = pack2<MB>(p0, p1), h23 = pack2<MB>(p2, p3);
