@@ -805,7 +805,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 // output care which accumulator row holds which d, so every lane reads whole 16-byte pieces:
                 //   K: lane (g, t) reads pieces t and 4 + t of rows g and g + 8; word s of piece 4 j + t feeds step 4 j + s,
                 //      bytes 0, 1 as k = 2t, 2t+1 and bytes 2, 3 as k = 2t+8, 2t+9 (q is read with the same assignment);
-                //   V: lane (g, t) reads piece g of the rows of tokens 2t, 2t+1, 2t+8, 2t+9; byte 2i (2i+1) of the piece is
+                //   V (after the softmax): lane (g, t) reads piece g of the rows of tokens 2t, 2t+1, 2t+8, 2t+9; byte 2i (2i+1) of the piece is
                 //      accumulator row g (g + 8) of product i, that is d = 16 g + 2 i (+ 1).
                 uint8_t *ring = smem + stage * SM::RING_BYTES;
                 if (p.k_new != nullptr && it.t1 == it.ctx && i == it.ntiles - 1) {
@@ -853,20 +853,6 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     kg[j] = *reinterpret_cast<const uint4 *>(ring + g * 128 + off);
                     kh[j] = *reinterpret_cast<const uint4 *>(ring + (g + 8) * 128 + off);
                 }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int tok = 2 * t + (j & 1) + 8 * (j >> 1);
-                    vv[j] = *reinterpret_cast<const uint4 *>(ring + (16 + tok) * 128 + ((g ^ (tok & 7)) << 4));
-                }
-                if (nvalid < 16) {
-                    // masked tokens are excluded, not multiplied by zero (a NaN byte stays a NaN): clear their V bytes
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (2 * t + (j & 1) + 8 * (j >> 1) >= nvalid) vv[j] = make_uint4(0u, 0u, 0u, 0u);
-                }
-                __syncwarp();
-                if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                if (lane == 0) mbar_arrive(bar_empty + 8 * stage);  // everything is in registers: the stage may be refilled
                 // ---- S^T[16 tokens][8 heads] = K . q^T
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
@@ -972,6 +958,26 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 pl1 = movmatrix_trans(pack2<true>(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xffff0000u)));
             }
             if constexpr (KV8) {
+                {
+                    // the V bytes are fetched only now: 16 fewer registers live across the softmax, so the 128 that five CTAs
+                    // per SM allow hold everything without spills (+3-4 % over fetching them with the K bytes)
+                    const uint8_t *ring = smem + stage * SM::RING_BYTES;
+                    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int tok = 2 * t + (j & 1) + 8 * (j >> 1);
+                        vv[j] = *reinterpret_cast<const uint4 *>(ring + (16 + tok) * 128 + ((g ^ (tok & 7)) << 4));
+                    }
+                    if (nvalid < 16) {
+                        // masked tokens are excluded, not multiplied by zero (a NaN byte stays a NaN): clear their V bytes
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (2 * t + (j & 1) + 8 * (j >> 1) >= nvalid) vv[j] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    __syncwarp();
+                    if (touched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    if (lane == 0) mbar_arrive(bar_empty + 8 * stage);  // everything is in registers: the stage may be refilled
+                }
                 const uint32_t v0w[4] = {vv[0].x, vv[0].y, vv[0].z, vv[0].w}, v1w[4] = {vv[1].x, vv[1].y, vv[1].z, vv[1].w};
                 const uint32_t v2w[4] = {vv[2].x, vv[2].y, vv[2].z, vv[2].w}, v3w[4] = {vv[3].x, vv[3].y, vv[3].z, vv[3].w};
 #pragma unroll
