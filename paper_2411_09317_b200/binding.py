@@ -547,6 +547,8 @@ def synth_lib():
         _synth.pie_synth_fill_slots.argtypes = [_vp, _vp, _i64, _i64, ctypes.c_uint64, _i32, _f32, _vp]
         _synth.pie_synth_fill_slots_bytes.restype = _i32
         _synth.pie_synth_fill_slots_bytes.argtypes = [_vp, _vp, _i64, _i64, ctypes.c_uint64, _vp]
+        _synth.pie_synth_fill_rows.restype = _i32
+        _synth.pie_synth_fill_rows.argtypes = [_vp, _vp, _i64, _i64, ctypes.c_uint64, _i32, _f32, _vp]
         _synth.pie_synth_fill_tensor.restype = _i32
         _synth.pie_synth_fill_tensor.argtypes = [_vp, _i64, ctypes.c_uint64, ctypes.c_uint64, _i32, _f32, _vp]
     return _synth

@@ -82,6 +82,16 @@ __global__ void fill_tensor_kernel(uint16_t *dst, int64_t n, uint64_t base, uint
         dst[i] = draw(base, offset + (uint64_t)i, dtype, gain);
 }
 
+// row r of dst (row_elems values) = the generator's values at indices row_offset[r] .. + row_elems
+__global__ void fill_rows_kernel(uint16_t *dst, const int64_t *__restrict__ row_offset, int64_t n_rows, int64_t row_elems,
+                                 uint64_t base, int dtype, float gain) {
+    const int64_t total = n_rows * row_elems;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / row_elems;
+        dst[i] = draw(base, (uint64_t)(row_offset[r] + (i - r * row_elems)), dtype, gain);
+    }
+}
+
 }  // namespace
 
 // pool: device-accessible memory (HBM, or pinned host memory through its device pointer); slot_unit: device
@@ -111,5 +121,15 @@ PIE_SYNTH_API int pie_synth_fill_tensor(void *dst, int64_t n, uint64_t base, uin
     if (n <= 0) return 0;
     const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
     fill_tensor_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((uint16_t *)dst, n, base, offset, dtype, gain);
+    return (int)cudaGetLastError();
+}
+
+// dst: device [n_rows][row_elems] 16-bit; row_offset: device int64 [n_rows]
+PIE_SYNTH_API int pie_synth_fill_rows(void *dst, const int64_t *row_offset, int64_t n_rows, int64_t row_elems, uint64_t base,
+                                      int dtype, float gain, void *stream) {
+    if (n_rows <= 0 || row_elems <= 0) return 0;
+    const int64_t total = n_rows * row_elems;
+    const int grid = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    fill_rows_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((uint16_t *)dst, row_offset, n_rows, row_elems, base, dtype, gain);
     return (int)cudaGetLastError();
 }

@@ -297,3 +297,51 @@ def test_throughput_reports_cap_the_ratio_when_expansion_buys_nothing():
     assert e.value.status == pie.PIE_ERR_INVALID
     check_samples(dw, [(0, 0), (3, 5)], steps_a + steps_b)
     free(dw)
+
+
+@pytest.mark.parametrize("kept", [False, True])
+def test_arrival_driver_serves_every_request_and_sampled_outputs_match_the_oracle(kept):
+    """A Poisson stream of requests through admission, prompt writes (pie_kv_write), continuous-batch decode steps with
+    the adaptive controller and the throughput governor, block growth and release: every request completes, every block
+    comes back, and the last output of sampled requests equals the oracle's attention over keys and values rebuilt from
+    the generator (they entered partly through the prompt write, partly token by token through the append, and were
+    swapped while the request ran)."""
+    from paper_2411_09317_b200 import arrivals
+    sh = arrivals.Shape(n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, dtype=synth.BF16)
+    n_req = 40
+    reqs = arrivals.make_requests(3, n_req, mean_gap=0.0004, prompt_median=300.0, prompt_sigma=0.5, out_mean=40.0)
+    sample = [0, 7, 19, 33]
+    d = arrivals.Driver(sh, gpu_blocks_per_layer=420, host_blocks_per_layer=400, max_seqs=32, kept_copies=kept,
+                        ctrl_step=1.0 / 64, window=8, sample_ids=sample)
+    pie.pie_set_controller(d.pool, 1.0 / 64, 0.5, 0.0)            # tolerant: the layers of this tiny model take microseconds
+    res = arrivals.run(d, reqs, max_steps=5000)
+    assert res["done"] == n_req and res["left_waiting"] == 0 and res["left_running"] == 0
+    assert res["tokens"] == sum(r.out_len for r in reqs)
+    assert max(row["running"] for row in d.log) > 8                # the batch did fill up
+    assert {rid for rid, _, _ in d.samples} == set(sample)
+    ke, qe = sh.n_kv_heads * sh.head_dim, sh.n_q_heads * sh.head_dim
+    worst = 0.0
+    for rid, ctx, out_bits in d.samples:
+        for l in (0, sh.n_layers - 1):
+            k = synth.tensor_bits(d.seed, synth.STREAM_KNEW, (ctx, sh.n_kv_heads, sh.head_dim), sh.dtype,
+                                  offset=arrivals.element_offset(sh, rid, l, 0, ke))
+            v = synth.tensor_bits(d.seed, synth.STREAM_VNEW, (ctx, sh.n_kv_heads, sh.head_dim), sh.dtype,
+                                  offset=arrivals.element_offset(sh, rid, l, 0, ke))
+            q = synth.tensor_bits(d.seed, synth.STREAM_Q, (1, sh.n_q_heads, sh.head_dim), sh.dtype,
+                                  offset=arrivals.element_offset(sh, rid, l, ctx - 1, qe))
+            nb = (ctx + 15) // 16
+            pool = np.zeros((nb, sh.n_kv_heads, 2, 16, sh.head_dim), dtype=np.uint16)
+            for t in range(ctx):
+                pool[t // 16, :, 0, t % 16, :] = k[t]
+                pool[t // 16, :, 1, t % 16, :] = v[t]
+            pool = pool.reshape(nb, -1)
+            ident = np.arange(nb, dtype=np.int32)
+            want = oracle.paged_attention(pool, pool, np.zeros(nb, np.int32), ident, q, ident[None, :], np.array([ctx], np.int32),
+                                          sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.dtype, 1.0 / np.sqrt(sh.head_dim))[0]
+            got = synth.bits16_to_f32(out_bits[l].reshape(sh.n_q_heads, sh.head_dim), sh.dtype)
+            worst = max(worst, float(np.abs(got - want).max()))
+            assert np.all(np.abs(got - want) <= TOL + 2.0 ** -8 * np.abs(want)), (rid, l, worst)
+    # every block came back: the whole id space can be handed out again
+    ids = pie.pie_block_alloc(d.pool, d.n_logical)
+    assert len(set(ids.tolist())) == d.n_logical
+    d.close()
