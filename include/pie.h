@@ -387,6 +387,9 @@ int pie_table_swap_ex(pie_table *t, int32_t queue, int32_t layer, const int32_t 
                       int32_t *moved_ids, int32_t *src_slots, int32_t *dst_slots, uint8_t *elided, int64_t *n_moved,
                       int64_t *waits);
 int pie_table_set_retention(pie_table *t, int32_t on);
+/* GPU-resident units that hold a kept host copy.  While there are any, a writer has to mark what it writes
+ * (pie_table_mark_dirty) even after the switch went off: switching off takes effect unit by unit at the next swap-in. */
+int64_t pie_table_kept_copies(const pie_table *t);
 int pie_table_mark_dirty(pie_table *t, int32_t layer, const int32_t *ids, int64_t n);
 /* A unit that lives on the GPU gives its kept host slot up (no-op otherwise). */
 int pie_table_drop_host_copy(pie_table *t, int32_t layer, int32_t block);

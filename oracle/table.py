@@ -338,6 +338,12 @@ class MappingTable:
             self.host_slot[u] = -1
         return OK
 
+    def kept_copies(self):
+        """GPU-resident units that hold a kept host copy.  While there are any, a writer has to mark what it writes even
+        after `retain` went off: switching off takes effect unit by unit at the next swap-in."""
+        return sum(1 for u in range(self.L * self.NB)
+                   if self.allocated[u % self.NB] and self.side[u] == GPU and self.host_slot[u] >= 0)
+
     def mark_dirty(self, layer, ids):
         """The layer's next attention call appends into these blocks: their host copies, where kept, go stale."""
         st = self._check_ids(layer, ids)

@@ -35,7 +35,7 @@ EXPORTS = [
     "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
-    "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
+    "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_kept_copies", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
     "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
     "pie_governor_create", "pie_governor_destroy", "pie_governor_report", "pie_governor_state", "pie_report_throughput",
 ]
@@ -115,6 +115,7 @@ _sig = {
     "pie_table_state": (_i32, [_vp, _i32, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pie_table_swap_ex": (_i32, [_vp, _i32, _i32, _vp, _i64, ctypes.POINTER(_i64), _vp, _vp, _vp, _vp, ctypes.POINTER(_i64), _vp]),
     "pie_table_set_retention": (_i32, [_vp, _i32]),
+    "pie_table_kept_copies": (_i64, [_vp]),
     "pie_table_mark_dirty": (_i32, [_vp, _i32, _vp, _i64]),
     "pie_table_drop_host_copy": (_i32, [_vp, _i32, _i32]),
     "pie_set_retention": (_i32, [_vp, _i32]),
@@ -462,6 +463,9 @@ class Table:
 
     def set_retention(self, on):
         return lib.pie_table_set_retention(self.h, int(on))
+
+    def kept_copies(self):
+        return int(lib.pie_table_kept_copies(self.h))
 
     def mark_dirty(self, layer, ids):
         ids = _np_i32(ids)

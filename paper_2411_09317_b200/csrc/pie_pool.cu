@@ -543,7 +543,7 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         st = p->table->attention(layer, nullptr, 0, &ticket, waits);
     }
     if (st != PIE_OK) return st;
-    if (k_new && p->table->retain()) {
+    if (k_new && p->table->tracks_writes()) {
         // kept host copies of the blocks this call's append writes go stale
         const int32_t NB = p->cfg.n_logical_blocks;
         auto mark = [&](int32_t b) {
@@ -1322,7 +1322,7 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
     int64_t ticket = 0, waits[4];
     st = pool->table->attention(layer, nullptr, 0, &ticket, waits);
     if (st != PIE_OK) return st;
-    if (pool->table->retain()) pool->table->mark_layer_dirty(layer);  // which blocks are written is on the device only
+    if (pool->table->tracks_writes()) pool->table->mark_layer_dirty(layer);  // which blocks are written is on the device only
     cudaStream_t stream = pool->stream[PIE_Q_COMPUTE];
     st = reserve_ticket_event(pool, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) { pool->sticky = st; return st; }
@@ -1704,7 +1704,7 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
             p->append_declared = declared;
         }
     } guard{pool, {}, pool->append_declared};
-    if (k_new_all_host && pool->table->retain()) {
+    if (k_new_all_host && pool->table->tracks_writes()) {
         guard.saved.swap(pool->append_ids);
         guard.active = true;
         for (int32_t sq = 0; sq < n_seqs; ++sq)

@@ -237,7 +237,10 @@ int Table::free_block(int32_t block) {
             // an attention call issued earlier may still be reading the slot
             int64_t ct = issued_[PIE_Q_COMPUTE];
             gpu_.release(u.gpu_slot, ct > done_[PIE_Q_COMPUTE] ? PIE_Q_COMPUTE : PIE_Q_NONE, ct);
-            if (u.host_slot >= 0) host_.release(u.host_slot, PIE_Q_NONE, 0);  // a kept host copy goes with the unit
+            if (u.host_slot >= 0) {  // a kept host copy goes with the unit
+                host_.release(u.host_slot, PIE_Q_NONE, 0);
+                --n_kept_;
+            }
         } else {
             host_.release(u.host_slot, PIE_Q_NONE, 0);
         }
@@ -274,6 +277,7 @@ int Table::drop_host_copy(int32_t layer, int32_t block) {
         if (in_flight(u)) host_.release(u.host_slot, u.last_q, u.last_t);
         else host_.release(u.host_slot, PIE_Q_NONE, 0);
         u.host_slot = -1;
+        --n_kept_;
     }
     return PIE_OK;
 }
@@ -337,6 +341,7 @@ int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int
         if (queue == PIE_Q_OUT) {
             s = u.gpu_slot;
             skip = kept && !u.dirty;  // the kept copy is still good unless the unit was written
+            if (kept) --n_kept_;
             u.host_slot = d;
             u.gpu_slot = -1;
             u.dirty = 0;
@@ -347,6 +352,8 @@ int Table::swap(int32_t queue, int32_t layer, const int32_t *ids, int64_t n, int
             if (!retain_) {
                 u.host_slot = -1;
                 src_pool.release(s, queue, tk);
+            } else {
+                ++n_kept_;
             }
             // with retain_ the host slot stays the unit's, and a dirty mark made before the unit came in survives
         }
@@ -515,6 +522,7 @@ int pie_table_set_retention(pie_table *t, int32_t on) {
     reinterpret_cast<Table *>(t)->set_retain(on != 0);
     return PIE_OK;
 }
+int64_t pie_table_kept_copies(const pie_table *t) { return t ? reinterpret_cast<const Table *>(t)->kept_copies() : 0; }
 int pie_table_drop_host_copy(pie_table *t, int32_t layer, int32_t block) {
     return t ? reinterpret_cast<Table *>(t)->drop_host_copy(layer, block) : PIE_ERR_INVALID;
 }

@@ -75,6 +75,10 @@ class Table {
     // its host slot, and going out again copies nothing unless it was marked written meanwhile.
     void set_retain(bool on) { retain_ = on; }
     bool retain() const { return retain_; }
+    // GPU-resident units that hold a kept host copy: while there are any, whoever writes a unit has to mark it dirty,
+    // whether or not the switch is still on (switching it off takes effect unit by unit at the next swap-in)
+    int64_t kept_copies() const { return n_kept_; }
+    bool tracks_writes() const { return retain_ || n_kept_ > 0; }
     int mark_dirty(int32_t layer, const int32_t *ids, int64_t n);
     int drop_host_copy(int32_t layer, int32_t block);  // a GPU-resident unit gives its kept host slot up
     void mark_layer_dirty(int32_t layer);
@@ -128,6 +132,7 @@ class Table {
     int32_t n_allocated_ = 0;
     int32_t capacity_, target_ = -1, n_moved_ = 0;
     bool retain_ = false;
+    int64_t n_kept_ = 0;
     std::vector<uint8_t> moved_;  // per layer
     std::vector<int32_t> take_slots_;  // scratch of swap() / alloc_bulk()
     std::vector<SlotTag> take_tags_;

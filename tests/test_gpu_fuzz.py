@@ -91,3 +91,54 @@ def test_random_case_matches_oracle(seed):
     bound = TOL + (2.0 ** -8 if case.dtype == BF16 else 2.0 ** -11) * np.abs(want)
     assert np.all(np.abs(got - want) <= bound), (c, float(np.abs(got - want).max()))
     pc.close()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_decode_steps_with_changing_ratio_match_oracle(seed):
+    """Several decode steps on a small model while the extension ratio, the look-ahead and the kept-copies switch change
+    at random between steps: every step's outputs within tolerance, and at the end every unit's bytes equal the oracle's."""
+    rng = np.random.default_rng(5000 + seed)
+    kv8 = bool(seed % 3 == 1)
+    dtype = int(rng.choice([F16, BF16]))
+    L, hkv, group = int(rng.integers(2, 5)), int(rng.choice([1, 2, 4])), int(rng.choice([1, 2, 4]))
+    d = 128 if kv8 else int(rng.choice([64, 128]))
+    lens = rng.integers(1, 400, int(rng.integers(2, 9))).astype(np.int32)
+    steps = 6
+    kw = dict(kv_fp8=True, k_scale=0.25, v_scale=0.125) if kv8 else {}
+    case = Case(L, hkv * group, hkv, d, dtype, lens, seed=seed, host_frac=float(rng.choice([0.0, 0.4])), placement="random",
+                extra_tokens=steps, **kw)
+    nh = len(case.host_ids)
+    pc = PoolCase(case, timing=1, n_gpu_slots=L * case.NB + 6 * case.NB + 8, n_host_slots=L * case.NB + 6 * case.NB + 8)
+    dev = torch.device("cuda:0")
+    cur = lens.copy()
+    ctx_dev = torch.from_numpy(cur).to(dev)
+    for t in range(steps):
+        pie.pie_set_extension_ratio(pc.pool, float(rng.choice([0.0, 0.1, 0.3, 0.6, 1.0])))
+        pie.pie_set_lookahead(pc.pool, int(rng.integers(1, 4)))
+        pie.pie_set_retention(pc.pool, int(rng.integers(0, 2)))
+        k_new = synth.tensor_bits(seed, synth.STREAM_KNEW, (L, case.S, case.Hkv, case.D), dtype, offset=t * 10_000_000)
+        v_new = synth.tensor_bits(seed, synth.STREAM_VNEW, (L, case.S, case.Hkv, case.D), dtype, gain=0.5, offset=t * 10_000_000)
+        k_dev = torch.from_numpy(k_new.view(np.int16)).to(dev)
+        v_dev = torch.from_numpy(v_new.view(np.int16)).to(dev)
+        cur = cur + 1
+        ctx_dev.copy_(torch.from_numpy(cur))
+        torch.cuda.synchronize()
+        pie.pie_decode_step(pc.pool, pc.q.data_ptr(), pc.out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                            ctx_dev.data_ptr(), case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        pie.pie_sync(pc.pool)
+        case.ctx_lens = cur.copy()
+        for l in range(L):
+            if kv8:
+                fp8.append(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k_new[l], v_new[l], case.block_table,
+                           cur, case.Hkv, case.D, dtype, case.k_scale, case.v_scale)
+            else:
+                oracle.append(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k_new[l], v_new[l],
+                              case.block_table, cur, case.Hkv, case.D)
+            want = oracle_attention(case, l)
+            got = synth.bits16_to_f32(pc.out[l].cpu().numpy().view(np.uint16), dtype)
+            bound = TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
+            assert np.all(np.abs(got - want) <= bound), (seed, t, l, float(np.abs(got - want).max()))
+    for l in range(L):
+        for b in range(case.NB):
+            assert np.array_equal(pc.read_unit(l, b), pc.unit_bits(l, b)), (seed, l, b)
+    pc.close()

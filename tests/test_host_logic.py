@@ -72,11 +72,15 @@ def both_apply(o, t, op):
         a, b = o.mark_dirty(op[1], list(op[2])), t.mark_dirty(op[1], list(op[2]))
     elif kind == "drop":
         a, b = o.drop_host_copy(op[1], op[2]), t.drop_host_copy(op[1], op[2])
+    elif kind == "retain":
+        o.retain = bool(op[1])
+        a, b = 0, t.set_retention(op[1])
     elif kind == "resize":
         a, b = o.resize_begin(op[1]), t.resize_begin(op[1])
     elif kind == "pass":
         a, b = int(o.layer_pass(op[1])), t.layer_pass(op[1])
     assert a == b, (op, a, b)
+    assert t.kept_copies() == o.kept_copies(), op
     st, cap = t.capacity()
     assert cap == {"visible": o.capacity, "alloc_limit": o.alloc_limit(), "target": -1 if o.target is None else o.target,
                    "layers_moved": len(o.moved)}, op
@@ -132,6 +136,8 @@ def test_table_matches_oracle_random_long(retain):
                 both_apply(o, t, ("dirty", rng.randrange(L), tuple(rng.sample(range(NB), rng.randint(1, NB)))))
             if retain and rng.random() < 0.05:
                 both_apply(o, t, ("drop", rng.randrange(L), rng.randrange(NB)))
+            if retain and rng.random() < 0.04:
+                both_apply(o, t, ("retain", rng.random() < 0.5))      # the switch itself, while copies are kept
             ids = tuple(rng.sample(range(NB), rng.randint(1, NB)))
             if rng.random() < 0.05:
                 ids = ids + (ids[0],) if rng.random() < 0.5 else ids + (NB + 3,)

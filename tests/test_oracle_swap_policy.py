@@ -106,7 +106,9 @@ def apply_op(tbl, ex, op):
         st, ticket, pairs, waits = tbl.swap(q, op[1], list(op[2]))
         if st == table.OK and ticket:
             layer, elided = op[1], list(tbl.last_elided)
-            assert len(elided) == len(pairs) and (tbl.retain or not any(elided))
+            # (copies kept before the switch went off may still be used: what matters is that kept copies ever existed)
+            ex.kept_ever = getattr(ex, "kept_ever", False) or tbl.retain
+            assert len(elided) == len(pairs) and (ex.kept_ever or not any(elided))
 
             def body(pairs=pairs, layer=layer, q=q, elided=elided):
                 src, dst = (ex.g, ex.h) if q == table.Q_OUT else (ex.h, ex.g)
@@ -331,9 +333,33 @@ def test_table_random_long_runs(retain):
                   ("attn", layer, ids) if k < 0.76 else ("drop", layer, ids[0]) if k < 0.78 else
                   ("attn_append", layer, ids, set(rng.sample(ids, 1))) if k < 0.85 else
                   ("confirm", rng.random() < 0.3) if k < 0.93 else ("run", 2))
+            if retain and rng.random() < 0.04:
+                # the switch itself, while copies are kept: writers go on marking what they write (the executor always
+                # does), so a unit that still holds a copy from before is written back when it next goes out
+                tbl.retain = rng.random() < 0.5
             apply_op(tbl, ex, op)
             tbl.check_invariants()
         final_check(tbl, ex)
+
+
+def test_switching_kept_copies_off_does_not_orphan_a_stale_copy():
+    """A unit comes in with its copy kept, the switch goes off, the unit is written, goes out, comes back: the write-back
+    must have happened (the copy from before the switch is stale), and the table still reports the copy as kept until then."""
+    t = table.MappingTable(1, 2, 2, 4, retain=True)
+    assert t.alloc(0, True) == table.OK
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [0])
+    t.confirm(table.Q_IN, tk)
+    assert t.kept_copies() == 1
+    t.retain = False                                   # off: takes effect at the unit's next swap-in
+    assert t.kept_copies() == 1
+    assert t.mark_dirty(0, [0]) == table.OK            # the writer still marks: there is a kept copy
+    st, tk, pairs, waits = t.swap(table.Q_OUT, 0, [0])
+    assert list(t.last_elided) == [False]              # copied, not skipped
+    t.confirm(table.Q_OUT, tk)
+    st, tk, pairs, waits = t.swap(table.Q_IN, 0, [0])
+    t.confirm(table.Q_IN, tk)
+    assert t.kept_copies() == 0                        # now the host slot is gone
+    t.check_invariants()
 
 
 # ------------------------------------------------------------------------- protocol golden trace
