@@ -42,7 +42,7 @@ def random_case(seed):
                 placement=placement, append=append, shuffle=bool(rng.integers(0, 2)))
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("PIE_FUZZ_CASES", "24"))))
 def test_random_case_matches_oracle(seed):
     c = random_case(seed)
     kw = dict(kv_fp8=True, k_scale=0.25, v_scale=0.125) if c["kv8"] else {}
@@ -93,7 +93,7 @@ def test_random_case_matches_oracle(seed):
     pc.close()
 
 
-@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("PIE_FUZZ_SEEDS", "12"))))
 def test_random_decode_steps_with_changing_ratio_match_oracle(seed):
     """Several decode steps on a small model while the extension ratio, the look-ahead and the kept-copies switch change
     at random between steps: every step's outputs within tolerance, and at the end every unit's bytes equal the oracle's."""
@@ -142,3 +142,90 @@ def test_random_decode_steps_with_changing_ratio_match_oracle(seed):
         for b in range(case.NB):
             assert np.array_equal(pc.read_unit(l, b), pc.unit_bits(l, b)), (seed, l, b)
     pc.close()
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("PIE_FUZZ_OPS", "6"))))
+def test_random_pool_operations_keep_every_unit_and_attend_correctly(seed):
+    """A random walk over the pool's calls - allocate (either side) and fill, free, swap lists out and in by any of the
+    copy paths, read back, attend over sequences made of whatever blocks exist - against a plain dictionary of what every
+    (layer, block) should hold.  Nothing is synchronised unless a call needs it."""
+    rng = np.random.default_rng(9000 + seed)
+    L, hkv, hq, d, dtype = int(rng.integers(1, 4)), 2, 4, 128, int(rng.choice([F16, BF16]))
+    NB = 48
+    elems = hkv * 2 * 16 * d
+    pool = pie.pie_pool_create(n_layers=L, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, dtype=dtype, n_logical_blocks=NB, max_seqs=8,
+                               n_gpu_slots=int(rng.integers(NB // 2, L * NB)) + 4, n_host_slots=L * NB + 8)
+    content = {}                                   # (layer, block) -> uint16 [elems]
+    live = []
+    dev = torch.device("cuda:0")
+    modes = [pie.PIE_MODE_AUTO, pie.PIE_MODE_KERNEL, pie.PIE_MODE_COPY_ENGINE, pie.PIE_MODE_KERNEL_BULK]
+    fills = 0
+    for step in range(120):
+        k = rng.random()
+        if k < 0.2 and len(live) < NB:
+            n = int(rng.integers(1, min(6, NB - len(live)) + 1))
+            try:
+                ids = pie.pie_block_alloc(pool, n, rng.integers(0, 2, n).astype(np.uint8))
+            except pie.PieError as e:
+                assert e.status == pie.PIE_ERR_NOMEM
+                continue
+            for b in ids:
+                for l in range(L):
+                    bits = synth.normal_bits(seed, synth.STREAM_KV, np.arange(elems, dtype=np.uint64) + np.uint64(fills * elems), dtype)
+                    fills += 1
+                    pie.pie_block_write(pool, l, int(b), bits)
+                    content[(l, int(b))] = bits
+                live.append(int(b))
+        elif k < 0.3 and live:
+            gone = [live.pop(int(rng.integers(0, len(live)))) for _ in range(min(len(live), int(rng.integers(1, 4))))]
+            pie.pie_sync(pool)                      # a block with a copy in flight cannot be freed
+            pie.pie_block_free(pool, gone)
+            for b in gone:
+                for l in range(L):
+                    del content[(l, b)]
+        elif k < 0.65 and live:
+            ids = rng.choice(live, int(rng.integers(1, len(live) + 1)), replace=False).astype(np.int32)
+            layer, mode = int(rng.integers(0, L)), modes[int(rng.integers(0, 4))]
+            try:
+                (pie.pie_swap_out if rng.random() < 0.5 else pie.pie_swap_in)(pool, layer, ids, mode)
+            except pie.PieError as e:
+                assert e.status == pie.PIE_ERR_NOMEM
+        elif k < 0.8 and live:
+            l, b = int(rng.integers(0, L)), int(rng.choice(live))
+            assert np.array_equal(pie.pie_block_read(pool, l, b).view(np.uint16), content[(l, b)]), (step, l, b)
+        elif live:
+            # attention over up to four sequences cut from a random order of the live blocks
+            layer = int(rng.integers(0, L))
+            order = rng.permutation(live)
+            S = int(rng.integers(1, min(4, len(order)) + 1))
+            parts = np.array_split(order, S)
+            max_blocks = max(len(p) for p in parts)
+            bt = np.full((S, max_blocks), -1, dtype=np.int32)
+            lens = np.zeros(S, dtype=np.int32)
+            for s, p in enumerate(parts):
+                bt[s, :len(p)] = p
+                lens[s] = 16 * len(p) - int(rng.integers(0, 16))
+            try:
+                pie.pie_swap_in(pool, layer, order.astype(np.int32), modes[int(rng.integers(0, 4))])
+            except pie.PieError as e:
+                assert e.status == pie.PIE_ERR_NOMEM
+                continue
+            q = synth.tensor_bits(seed, synth.STREAM_Q, (S, hq, d), dtype, offset=step * 100_000)
+            q_dev = torch.from_numpy(q.view(np.int16)).to(dev)
+            out_dev = torch.zeros_like(q_dev)
+            bt_dev, len_dev = torch.from_numpy(bt).to(dev), torch.from_numpy(lens).to(dev)
+            torch.cuda.synchronize()
+            pie.pie_decode_attention(pool, layer, q_dev.data_ptr(), out_dev.data_ptr(), bt_dev.data_ptr(), max_blocks,
+                                     len_dev.data_ptr(), S, 1.0 / np.sqrt(d), block_table_host=bt, ctx_lens_host=lens)
+            pie.pie_sync(pool)
+            store = np.stack([content[(layer, int(b))] for b in order])
+            slot_of = np.full(NB, -1, dtype=np.int32)
+            slot_of[order] = np.arange(len(order))
+            want = oracle.paged_attention(store, store, np.zeros(NB, np.int32), slot_of, q, bt, lens, hq, hkv, d, dtype, 1.0 / np.sqrt(d))
+            got = synth.bits16_to_f32(out_dev.cpu().numpy().view(np.uint16), dtype)
+            bound = TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
+            assert np.all(np.abs(got - want) <= bound), (seed, step, float(np.abs(got - want).max()))
+    pie.pie_sync(pool)
+    for (l, b), bits in content.items():
+        assert np.array_equal(pie.pie_block_read(pool, l, b).view(np.uint16), bits), (l, b)
+    pie.pie_pool_destroy(pool)
