@@ -123,8 +123,22 @@ def test_random_decode_steps_with_changing_ratio_match_oracle(seed):
         cur = cur + 1
         ctx_dev.copy_(torch.from_numpy(cur))
         torch.cuda.synchronize()
-        pie.pie_decode_step(pc.pool, pc.q.data_ptr(), pc.out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
-                            ctx_dev.data_ptr(), case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        api = int(rng.integers(0, 3))        # the whole step, the same layer by layer, or from host buffers
+        if api == 0:
+            pie.pie_decode_step(pc.pool, pc.q.data_ptr(), pc.out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                                ctx_dev.data_ptr(), case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        elif api == 1:
+            pie.pie_step_begin(pc.pool)
+            for l in range(L):
+                pie.pie_decode_layer(pc.pool, l, pc.q[l].data_ptr(), pc.out[l].data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                                     ctx_dev.data_ptr(), case.S, case.scale, k_dev[l].data_ptr(), v_dev[l].data_ptr())
+            pie.pie_controller_tick(pc.pool)
+        else:
+            out_host = np.zeros(tuple(pc.q.shape), dtype=np.int16)
+            pie.pie_decode_step_host(pc.pool, np.ascontiguousarray(case.q.view(np.int16)), out_host, case.block_table,
+                                     case.block_table.shape[1], cur.astype(np.int32), case.S, case.scale,
+                                     np.ascontiguousarray(k_new.view(np.int16)), np.ascontiguousarray(v_new.view(np.int16)))
+            pc.out.copy_(torch.from_numpy(out_host))
         pie.pie_sync(pc.pool)
         case.ctx_lens = cur.copy()
         for l in range(L):
