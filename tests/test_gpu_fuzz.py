@@ -243,3 +243,59 @@ def test_random_pool_operations_keep_every_unit_and_attend_correctly(seed):
     for (l, b), bits in content.items():
         assert np.array_equal(pie.pie_block_read(pool, l, b).view(np.uint16), bits), (l, b)
     pie.pie_pool_destroy(pool)
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("PIE_FUZZ_LAYERS", "6"))))
+def test_random_whole_layer_protocol_configurations_match_oracle(seed):
+    """The paper's whole-layer protocol (Section 3.3) with a random number of layers, of layers that start on the CPU and
+    of spare regions on either side: outputs of every step and the final bytes of every unit against the oracle."""
+    rng = np.random.default_rng(7000 + seed)
+    L = int(rng.integers(3, 11))
+    m = int(rng.integers(1, L - 1))                       # layers on the CPU at the start: the last m
+    gpu_regions = L - m + int(rng.integers(0, 2))
+    cpu_regions = m + int(rng.integers(1, 4))
+    dtype = int(rng.choice([F16, BF16]))
+    hkv, group, d = int(rng.choice([1, 2, 4])), int(rng.choice([1, 2])), int(rng.choice([64, 128]))
+    lens = rng.integers(1, 300, int(rng.integers(1, 6))).astype(np.int32)
+    steps = 4
+    case = Case(L, hkv * group, hkv, d, dtype, lens, seed=seed, host_frac=0.0, placement="identity", extra_tokens=steps)
+    NB = case.NB
+    pool = pie.pie_pool_create(n_layers=L, n_q_heads=case.Hq, n_kv_heads=hkv, head_dim=d, dtype=dtype, n_logical_blocks=NB,
+                               max_seqs=case.S, n_gpu_slots=gpu_regions * NB, n_host_slots=max(cpu_regions, L) * NB, timing=1)
+    pie.pie_block_alloc(pool, NB, np.ones(NB, np.uint8))
+    for l in range(L):
+        for b in range(NB):
+            pie.pie_block_write(pool, l, b, case.gpu_pool[case.unit_slot[l, b]])
+    for l in range(L - m):
+        pie.pie_swap_in(pool, l, np.arange(NB))
+    pie.pie_sync(pool)
+    pie.pie_set_layer_policy(pool, gpu_regions, cpu_regions)
+    dev = torch.device("cuda:0")
+    q = torch.from_numpy(case.q.view(np.int16)).to(dev)
+    out = torch.zeros_like(q)
+    bt = torch.from_numpy(case.block_table).to(dev)
+    cur = lens.copy()
+    ctx_dev = torch.from_numpy(cur).to(dev)
+    for t in range(steps):
+        k_new = synth.tensor_bits(seed, synth.STREAM_KNEW, (L, case.S, case.Hkv, case.D), dtype, offset=t * 1_000_000)
+        v_new = synth.tensor_bits(seed, synth.STREAM_VNEW, (L, case.S, case.Hkv, case.D), dtype, offset=t * 1_000_000)
+        k_dev = torch.from_numpy(k_new.view(np.int16)).to(dev)
+        v_dev = torch.from_numpy(v_new.view(np.int16)).to(dev)
+        cur = cur + 1
+        ctx_dev.copy_(torch.from_numpy(cur))
+        torch.cuda.synchronize()
+        pie.pie_decode_step(pool, q.data_ptr(), out.data_ptr(), bt.data_ptr(), case.block_table.shape[1], ctx_dev.data_ptr(),
+                            case.S, case.scale, k_dev.data_ptr(), v_dev.data_ptr())
+        pie.pie_sync(pool)
+        case.ctx_lens = cur.copy()
+        for l in range(L):
+            oracle.append(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k_new[l], v_new[l],
+                          case.block_table, cur, case.Hkv, case.D)
+            want = oracle_attention(case, l)
+            got = synth.bits16_to_f32(out[l].cpu().numpy().view(np.uint16), dtype)
+            bound = TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
+            assert np.all(np.abs(got - want) <= bound), (seed, L, m, gpu_regions, cpu_regions, t, l)
+    for l in range(L):
+        for b in range(NB):
+            assert np.array_equal(pie.pie_block_read(pool, l, b).view(np.uint16), case.gpu_pool[case.unit_slot[l, b]]), (seed, l, b)
+    pie.pie_pool_destroy(pool)
