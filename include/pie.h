@@ -256,7 +256,7 @@ int pie_set_lookahead(pie_pool *pool, int32_t layers);
  * the step's own attention already sees the stored (rounded) token.  Bytes beyond a sequence's length may hold anything.
  * The products run in fp16 for both 16-bit types (every E4M3 value is an fp16 number); a bf16 query is scaled into
  * fp16's range by a power of two per (sequence, KV head), exactly, so no finite query overflows.  Swapping, the table and the controller are
- * unchanged (they move block_bytes).  pie_kv_write returns PIE_ERR_UNSUPPORTED on such a pool.
+ * unchanged (they move block_bytes).  pie_kv_write quantises its rows with the append's rule.
  * PIE_ERR_INVALID unless both scales are finite and > 0; PIE_ERR_UNSUPPORTED on a 16-bit pool. */
 int pie_set_kv_scales(pie_pool *pool, float k_scale, float v_scale);
 

@@ -98,3 +98,30 @@ def append(gpu_pool8, host_pool8, unit_side, unit_slot, k_new, v_new, block_tabl
         tile = pool[int(unit_slot[b])].reshape(n_kv_heads, 2, 16, head_dim)
         tile[:, 0, pos % 16, :] = kq[s]
         tile[:, 1, pos % 16, :] = vq[s]
+
+
+def kv_write(gpu_pool8, host_pool8, unit_side, unit_slot, k, v, token_seq, token_pos, block_table, n_kv_heads, head_dim, dtype,
+             k_scale, v_scale):
+    """Prefill-side write into an 8-bit pool: token t is position token_pos[t] of sequence token_seq[t]; its 16-bit rows
+    k[t], v[t] ([Hkv][D]) are quantised like the append's (fp32 quotient by the scale, nearest E4M3, ties to the even code,
+    saturating) and land in row pos % 16 of the K and V halves of every head's tile in the block that holds the position.
+    Returns -1 (nothing written) if a position is beyond the table or a block id out of range."""
+    block_table = np.asarray(block_table, dtype=np.int32)
+    k = np.ascontiguousarray(k, dtype=np.uint16).reshape(-1, n_kv_heads, head_dim)
+    v = np.ascontiguousarray(v, dtype=np.uint16).reshape(-1, n_kv_heads, head_dim)
+    for t in range(len(token_seq)):
+        s, pos = int(token_seq[t]), int(token_pos[t])
+        if not (0 <= s < block_table.shape[0] and 0 <= pos < 16 * block_table.shape[1]):
+            return -1
+        if not 0 <= block_table[s, pos // 16] < len(unit_slot):
+            return -1
+    kq = quantize(_bits16_to_f64(k, dtype).astype(np.float32) / np.float32(k_scale))
+    vq = quantize(_bits16_to_f64(v, dtype).astype(np.float32) / np.float32(v_scale))
+    for t in range(len(token_seq)):
+        s, pos = int(token_seq[t]), int(token_pos[t])
+        b = int(block_table[s, pos // 16])
+        pool = host_pool8 if unit_side[b] else gpu_pool8
+        tile = pool[int(unit_slot[b])].reshape(n_kv_heads, 2, 16, head_dim)
+        tile[:, 0, pos % 16, :] = kq[t]
+        tile[:, 1, pos % 16, :] = vq[t]
+    return 0

@@ -38,6 +38,7 @@ class Shape:
     n_kv_heads: int = 8
     head_dim: int = 128
     dtype: int = synth.BF16
+    kv_fp8: bool = False      # 8-bit blocks (head_dim 128): prompts and appended tokens are quantised by the library
 
 
 @dataclasses.dataclass
@@ -64,6 +65,8 @@ def make_requests(seed: int, n: int, mean_gap: float, prompt_median=600.0, promp
 
 
 class Driver:
+    K_SCALE, V_SCALE = 0.25, 0.125     # scales of an 8-bit pool
+
     def __init__(self, sh: Shape, gpu_blocks_per_layer: int, host_blocks_per_layer: int, max_seqs=128, seed=11,
                  kept_copies=False, ctrl_step=1.0 / 512, window=16, sample_ids=()):
         self.sh, self.seed, self.window, self.max_seqs = sh, seed, window, max_seqs
@@ -76,7 +79,9 @@ class Driver:
         self.pool = pie.pie_pool_create(
             n_layers=L, n_q_heads=sh.n_q_heads, n_kv_heads=sh.n_kv_heads, head_dim=sh.head_dim, dtype=sh.dtype,
             n_logical_blocks=self.n_logical, max_seqs=max_seqs, n_gpu_slots=L * gpu_blocks_per_layer + staging,
-            n_host_slots=L * host_blocks_per_layer + staging, timing=1)
+            n_host_slots=L * host_blocks_per_layer + staging, timing=1, kv_fp8=int(sh.kv_fp8))
+        if sh.kv_fp8:
+            pie.pie_set_kv_scales(self.pool, self.K_SCALE, self.V_SCALE)
         pie.pie_set_controller(self.pool, ctrl_step, 0.0, 0.0)
         pie.pie_set_extension_ratio(self.pool, -1.0)             # adaptive
         pie.pie_set_retention(self.pool, int(kept_copies))
@@ -262,6 +267,7 @@ def main(argv=None):
     ap.add_argument("--kv-gb", type=float, default=2.0, help="size of the GPU pool")
     ap.add_argument("--host-frac", type=float, default=0.25, help="host pool as a fraction of the GPU pool")
     ap.add_argument("--kept-copies", action="store_true")
+    ap.add_argument("--kv-fp8", action="store_true", help="8-bit KV blocks")
     ap.add_argument("--max-steps", type=int, default=4000)
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
@@ -271,13 +277,13 @@ def main(argv=None):
         out.write(json.dumps(o) + "\n")
         out.flush()
 
-    sh = Shape()
-    block_bytes = 2 * 16 * sh.n_kv_heads * sh.head_dim * 2
+    sh = Shape(kv_fp8=args.kv_fp8)
+    block_bytes = 2 * 16 * sh.n_kv_heads * sh.head_dim * (1 if sh.kv_fp8 else 2)
     gpu_blocks = int(args.kv_gb * 1e9 / (sh.n_layers * block_bytes))
     # service capacity, roughly: a full pool holds gpu_blocks * 16 tokens; a request holds prompt + out/2 tokens for out steps
     mean_tokens, mean_out = 600 * np.exp(0.6 ** 2 / 2) + 48, 96.0
     conc = min(128, gpu_blocks * 16 / mean_tokens)
-    step_s = 40e-6 * sh.n_layers + conc * mean_tokens * sh.n_layers * 2 * sh.n_kv_heads * sh.head_dim * 2 / 5.5e12
+    step_s = 40e-6 * sh.n_layers + conc * mean_tokens * sh.n_layers * 2 * sh.n_kv_heads * sh.head_dim * (1 if sh.kv_fp8 else 2) / 5.5e12
     capacity = conc / (mean_out * step_s)                  # requests per GPU second
     reqs = make_requests(5, args.requests, 1.0 / (args.rate * capacity))
     d = Driver(sh, gpu_blocks, int(args.host_frac * gpu_blocks), kept_copies=args.kept_copies)

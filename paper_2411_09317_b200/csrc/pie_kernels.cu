@@ -532,6 +532,76 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
     return r;
 }
 
+// Prefill-side write into an 8-bit pool: as kv_write_kernel, but every 16-byte vector of 16-bit values becomes eight
+// E4M3 bytes (fp32 quotient by the scale, nearest even, saturating - the append's rule); rows are 128 bytes.
+template <bool BF16>
+__global__ void __launch_bounds__(256)
+kv_write8_kernel(const uint4 *__restrict__ k, const uint4 *__restrict__ v, const int32_t *__restrict__ token_seq,
+                 const int32_t *__restrict__ token_pos, int64_t n_tokens, int32_t tokens_per_cta,
+                 const int32_t *__restrict__ block_table, int32_t max_blocks, int32_t n_seqs,
+                 const int32_t *__restrict__ slot_table, int32_t n_logical, int64_t n_gpu_slots, uint8_t *__restrict__ pool,
+                 int32_t n_kv_heads, float k_scale, float v_scale, int32_t *status) {
+    constexpr int32_t vecs_per_row = 16;                                  // head_dim 128: 16 vectors of eight values
+    const int32_t per_token = n_kv_heads * vecs_per_row;
+    const int64_t slot_bytes = (int64_t)n_kv_heads * 2 * 16 * 128;
+    const int64_t t0 = (int64_t)blockIdx.x * tokens_per_cta;
+    for (int32_t i = threadIdx.x; i < tokens_per_cta * 2 * per_token; i += blockDim.x) {
+        const int32_t tt = i / (2 * per_token), r = i - tt * 2 * per_token;
+        const int64_t t = t0 + tt;
+        if (t >= n_tokens) break;
+        const int32_t s = token_seq[t], pos = token_pos[t];
+        if (s < 0 || s >= n_seqs || pos < 0 || pos >= max_blocks * 16) {
+            if (r == 0) raise_status(status, STATUS_CTX_TOO_LONG);
+            continue;
+        }
+        const int32_t b = block_table[(int64_t)s * max_blocks + (pos >> 4)];
+        const int32_t slot = (b >= 0 && b < n_logical) ? slot_table[b] : -1;
+        if (slot < 0 || slot >= n_gpu_slots) {
+            if (r == 0) raise_status(status, STATUS_MISSING_UNIT);
+            continue;
+        }
+        const int32_t kv = r >= per_token, j = r - kv * per_token;
+        const int32_t h = j / vecs_per_row, c = j - h * vecs_per_row;
+        const uint4 val = (kv ? v : k)[t * per_token + j];
+        const float sc = kv ? v_scale : k_scale;
+        const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float lo, hi;
+            if (BF16) {
+                lo = __uint_as_float(w[q] << 16);
+                hi = __uint_as_float(w[q] & 0xffff0000u);
+            } else {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[q]));
+                lo = f.x;
+                hi = f.y;
+            }
+            o[q] = f32x2_to_e4m3x2(__fdiv_rn(lo, sc), __fdiv_rn(hi, sc));
+        }
+        *reinterpret_cast<uint2 *>(pool + (int64_t)slot * slot_bytes + (((int64_t)h * 2 + kv) * 16 + (pos & 15)) * 128 + 8 * c) =
+            make_uint2(o[0] | (o[1] << 16), o[2] | (o[3] << 16));
+    }
+}
+
+cudaError_t launch_kv_write8(const void *k, const void *v, const int32_t *token_seq, const int32_t *token_pos, int64_t n_tokens,
+                             const int32_t *block_table, int32_t max_blocks, int32_t n_seqs, const int32_t *slot_table,
+                             int32_t n_logical, int64_t n_gpu_slots, void *gpu_pool, int32_t n_kv_heads, int32_t dtype,
+                             float k_scale, float v_scale, int32_t *status, cudaStream_t stream) {
+    if (n_tokens <= 0) return cudaSuccess;
+    const int32_t per_cta = std::max(1, 1024 / (2 * n_kv_heads * 16));
+    const int64_t grid = (n_tokens + per_cta - 1) / per_cta;
+    if (dtype == PIE_BF16)
+        kv_write8_kernel<true><<<(unsigned)grid, 256, 0, stream>>>((const uint4 *)k, (const uint4 *)v, token_seq, token_pos, n_tokens,
+                                                                  per_cta, block_table, max_blocks, n_seqs, slot_table, n_logical,
+                                                                  n_gpu_slots, (uint8_t *)gpu_pool, n_kv_heads, k_scale, v_scale, status);
+    else
+        kv_write8_kernel<false><<<(unsigned)grid, 256, 0, stream>>>((const uint4 *)k, (const uint4 *)v, token_seq, token_pos, n_tokens,
+                                                                   per_cta, block_table, max_blocks, n_seqs, slot_table, n_logical,
+                                                                   n_gpu_slots, (uint8_t *)gpu_pool, n_kv_heads, k_scale, v_scale, status);
+    return cudaGetLastError();
+}
+
 // The second launch bound: for 16-bit pools it only tells the assembler that it need not hold registers back for more
 // CTAs per SM than shared memory lets in anyway (three; without it some instantiations were capped at 96 registers and
 // spilled).  The 8-bit kernel is bound by instruction latency, not by bytes in flight, and its CTAs need a third of
@@ -1284,7 +1354,7 @@ int attn_smem_bytes(int head_dim) { return head_dim == 128 ? AttnSmem<128, 4, 2>
 // lands on an idle SM first could keep attention CTAs off that SM until it has finished.
 static cudaError_t prefer_max_shared() {
     const void *fns[] = {(const void *)swap_kernel, (const void *)patch_kernel, (const void *)patch_from_list_kernel,
-                         (const void *)kv_write_kernel, (const void *)swap_bulk_kernel, (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
+                         (const void *)kv_write_kernel, (const void *)kv_write8_kernel<true>, (const void *)kv_write8_kernel<false>, (const void *)swap_bulk_kernel, (const void *)plan_kernel, (const void *)combine_kernel<128, true>, (const void *)combine_kernel<128, false>,
                          (const void *)combine_kernel<64, true>, (const void *)combine_kernel<64, false>};
     for (const void *f : fns) {
         cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);

@@ -35,6 +35,11 @@ cudaError_t launch_kv_write(const void *k, const void *v, const int32_t *token_s
                             const int32_t *block_table, int32_t max_blocks, int32_t n_seqs, const int32_t *slot_table,
                             int32_t n_logical, int64_t n_gpu_slots, void *gpu_pool, int32_t n_kv_heads, int32_t head_dim,
                             int32_t *status, cudaStream_t stream);
+// the same into an 8-bit pool (head_dim 128): rows are quantised to E4M3 with the append's rule
+cudaError_t launch_kv_write8(const void *k, const void *v, const int32_t *token_seq, const int32_t *token_pos, int64_t n_tokens,
+                             const int32_t *block_table, int32_t max_blocks, int32_t n_seqs, const int32_t *slot_table,
+                             int32_t n_logical, int64_t n_gpu_slots, void *gpu_pool, int32_t n_kv_heads, int32_t dtype,
+                             float k_scale, float v_scale, int32_t *status, cudaStream_t stream);
 
 // ---- attention -----------------------------------------------------------------------------------
 struct AttnShape {

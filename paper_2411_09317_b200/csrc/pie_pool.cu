@@ -1311,7 +1311,6 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
     if (!pool || n_tokens < 0 || max_blocks_per_seq <= 0 || n_seqs <= 0) return PIE_ERR_INVALID;
     if (n_tokens > 0 && (!k || !v || !token_seq_dev || !token_pos_dev || !block_table_dev)) return PIE_ERR_INVALID;
     if (pool->sticky != PIE_OK) return pool->sticky;
-    if (pool->kv_fp8) return PIE_ERR_UNSUPPORTED;  // the scatter moves 16-bit vectors as they are
     if (layer < 0 || layer >= pool->cfg.n_layers) return PIE_ERR_RANGE;
     int st = poll(pool);
     if (st != PIE_OK) return st;
@@ -1330,10 +1329,14 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
         st = wait_ticket(pool, stream, qd, waits[qd]);
         if (st != PIE_OK) { pool->sticky = st; return st; }
     }
-    cudaError_t e = pie::launch_kv_write(k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs,
-                                         pool->slot_table_dev + (int64_t)layer * pool->cfg.n_logical_blocks,
-                                         pool->cfg.n_logical_blocks, pool->cfg.n_gpu_slots, pool->gpu_base, pool->cfg.n_kv_heads,
-                                         pool->cfg.head_dim, pool->status_dev, stream);
+    const int32_t *slots = pool->slot_table_dev + (int64_t)layer * pool->cfg.n_logical_blocks;
+    cudaError_t e = pool->kv_fp8
+                        ? pie::launch_kv_write8(k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs,
+                                                slots, pool->cfg.n_logical_blocks, pool->cfg.n_gpu_slots, pool->gpu_base,
+                                                pool->cfg.n_kv_heads, pool->cfg.dtype, pool->k_scale, pool->v_scale, pool->status_dev, stream)
+                        : pie::launch_kv_write(k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs,
+                                               slots, pool->cfg.n_logical_blocks, pool->cfg.n_gpu_slots, pool->gpu_base,
+                                               pool->cfg.n_kv_heads, pool->cfg.head_dim, pool->status_dev, stream);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
         pool->sticky = PIE_ERR_CUDA;

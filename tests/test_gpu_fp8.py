@@ -236,8 +236,37 @@ def test_argument_checks():
             pie.pie_set_kv_scales(p8, ks, vs)
         assert e.value.status == pie.PIE_ERR_INVALID
     pie.pie_set_kv_scales(p8, 0.5, 0.25)
-    z = torch.zeros(16, dtype=torch.int32, device="cuda")
-    with pytest.raises(pie.PieError) as e:
-        pie.pie_kv_write(p8, 0, z.data_ptr(), z.data_ptr(), z.data_ptr(), z.data_ptr(), 1, z.data_ptr(), 1, 1)
-    assert e.value.status == pie.PIE_ERR_UNSUPPORTED
     pie.pie_pool_destroy(p8)
+
+
+@pytest.mark.parametrize("hq,hkv,dtype", [(8, 8, BF16), (8, 1, F16), (16, 4, F16)])
+def test_prompt_write_quantises_like_the_append_and_attention_reads_it(hq, hkv, dtype):
+    """Whole prompts written token by token (flat batch, shuffled order) into an 8-bit pool that starts as a fill
+    pattern: every byte of every unit equals the oracle's quantised write, and attention over them matches the oracle."""
+    lens = np.array([1, 16, 17, 100, 45], dtype=np.int32)
+    case = fp8_case(2, hq, hkv, 128, dtype, lens, seed=61)
+    seqs, poss = [], []
+    for s in range(case.S):
+        for t in range(int(lens[s])):
+            seqs.append(s); poss.append(t)
+    order = synth.seeded_permutation(61, len(seqs), salt=9)
+    seqs, poss = np.array(seqs, np.int32)[order], np.array(poss, np.int32)[order]
+    case.gpu_pool[:] = 0x55
+    pc = PoolCase(case)
+    dev = torch.device("cuda:0")
+    seq_dev, pos_dev = torch.from_numpy(seqs).to(dev), torch.from_numpy(poss).to(dev)
+    for l in range(case.L):
+        k = synth.tensor_bits(61, synth.STREAM_KNEW, (len(seqs), hkv, 128), dtype, offset=l * 1_000_000)
+        v = synth.tensor_bits(61, synth.STREAM_VNEW, (len(seqs), hkv, 128), dtype, gain=0.5, offset=l * 1_000_000)
+        k_dev, v_dev = torch.from_numpy(k.view(np.int16)).to(dev), torch.from_numpy(v.view(np.int16)).to(dev)
+        torch.cuda.synchronize()
+        pie.pie_kv_write(pc.pool, l, k_dev.data_ptr(), v_dev.data_ptr(), seq_dev.data_ptr(), pos_dev.data_ptr(), len(seqs),
+                         pc.bt.data_ptr(), case.block_table.shape[1], case.S)
+        assert fp8.kv_write(case.gpu_pool, case.host_pool, case.unit_side[l], case.unit_slot[l], k, v, seqs, poss,
+                            case.block_table, hkv, 128, dtype, case.k_scale, case.v_scale) == 0
+    pie.pie_sync(pc.pool)
+    for l in range(case.L):
+        for b in range(case.NB):
+            assert np.array_equal(pc.read_unit(l, b), pc.unit_bits(l, b)), (l, b)     # written rows and the untouched fill alike
+        check(case, pc, l)
+    pc.close()

@@ -299,15 +299,15 @@ def test_throughput_reports_cap_the_ratio_when_expansion_buys_nothing():
     free(dw)
 
 
-@pytest.mark.parametrize("kept", [False, True])
-def test_arrival_driver_serves_every_request_and_sampled_outputs_match_the_oracle(kept):
+@pytest.mark.parametrize("kept,kv8", [(False, False), (True, False), (True, True)])
+def test_arrival_driver_serves_every_request_and_sampled_outputs_match_the_oracle(kept, kv8):
     """A Poisson stream of requests through admission, prompt writes (pie_kv_write), continuous-batch decode steps with
     the adaptive controller and the throughput governor, block growth and release: every request completes, every block
     comes back, and the last output of sampled requests equals the oracle's attention over keys and values rebuilt from
     the generator (they entered partly through the prompt write, partly token by token through the append, and were
     swapped while the request ran)."""
     from paper_2411_09317_b200 import arrivals
-    sh = arrivals.Shape(n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, dtype=synth.BF16)
+    sh = arrivals.Shape(n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, dtype=synth.BF16, kv_fp8=kv8)
     n_req = 40
     reqs = arrivals.make_requests(3, n_req, mean_gap=0.0004, prompt_median=300.0, prompt_sigma=0.5, out_mean=40.0)
     sample = [0, 7, 19, 33]
@@ -336,8 +336,21 @@ def test_arrival_driver_serves_every_request_and_sampled_outputs_match_the_oracl
                 pool[t // 16, :, 1, t % 16, :] = v[t]
             pool = pool.reshape(nb, -1)
             ident = np.arange(nb, dtype=np.int32)
-            want = oracle.paged_attention(pool, pool, np.zeros(nb, np.int32), ident, q, ident[None, :], np.array([ctx], np.int32),
-                                          sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.dtype, 1.0 / np.sqrt(sh.head_dim))[0]
+            if kv8:
+                from oracle import fp8
+                pool8 = np.zeros((nb, sh.n_kv_heads, 2, 16, sh.head_dim), dtype=np.uint8)
+                kq = fp8.quantize(synth.bits16_to_f32(k, sh.dtype) / np.float32(d.K_SCALE))
+                vq = fp8.quantize(synth.bits16_to_f32(v, sh.dtype) / np.float32(d.V_SCALE))
+                for t in range(ctx):
+                    pool8[t // 16, :, 0, t % 16, :] = kq[t]
+                    pool8[t // 16, :, 1, t % 16, :] = vq[t]
+                pool8 = pool8.reshape(nb, -1)
+                want = fp8.paged_attention(pool8, pool8, np.zeros(nb, np.int32), ident, q, ident[None, :], np.array([ctx], np.int32),
+                                           sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.dtype, 1.0 / np.sqrt(sh.head_dim),
+                                           d.K_SCALE, d.V_SCALE)[0]
+            else:
+                want = oracle.paged_attention(pool, pool, np.zeros(nb, np.int32), ident, q, ident[None, :], np.array([ctx], np.int32),
+                                              sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.dtype, 1.0 / np.sqrt(sh.head_dim))[0]
             got = synth.bits16_to_f32(out_bits[l].reshape(sh.n_q_heads, sh.head_dim), sh.dtype)
             worst = max(worst, float(np.abs(got - want).max()))
             assert np.all(np.abs(got - want) <= TOL + 2.0 ** -8 * np.abs(want)), (rid, l, worst)

@@ -106,3 +106,28 @@ def test_generated_bytes_are_finite_values_of_both_signs():
     assert 2.0 ** -4 <= np.abs(v).min() and np.abs(v).max() <= 15.0
     assert len(np.unique(b)) > 100                       # signs, mantissas and eight exponents all occur
     assert not np.array_equal(b, synth.kv_unit_bytes(3, 1, 3, 10, 4, 128))
+
+
+def test_prompt_write_equals_token_by_token_append_and_reads_back_through_attention():
+    """The prefill-side write of a whole prompt leaves the bytes the append leaves when the same tokens arrive one by one,
+    touches nothing else, and rejects positions beyond the table."""
+    rng = np.random.default_rng(4)
+    hkv, d, n_tok = 2, 128, 37
+    nb = (n_tok + 15) // 16
+    k = rng.normal(0, 2.0, (n_tok, hkv, d)).astype(np.float16).view(np.uint16)
+    v = rng.normal(0, 1.0, (n_tok, hkv, d)).astype(np.float16).view(np.uint16)
+    table = np.arange(nb, dtype=np.int32)[::-1].copy()[None, :]          # blocks in reverse order
+    side, slot = np.zeros(nb, np.int32), np.arange(nb, dtype=np.int32)
+    a = np.full((nb, hkv * 2 * 16 * d), 0x55, dtype=np.uint8)
+    b = a.copy()
+    order = rng.permutation(n_tok)
+    assert fp8.kv_write(a, a, side, slot, k[order], v[order], np.zeros(n_tok, np.int32), order.astype(np.int32), table, hkv, d,
+                        fp8.F16, 0.25, 0.5) == 0
+    for t in range(n_tok):
+        fp8.append(b, b, side, slot, k[t:t + 1], v[t:t + 1], table, np.array([t + 1], np.int32), hkv, d, fp8.F16, 0.25, 0.5)
+    assert np.array_equal(a, b)
+    tail = a[slot[table[0, nb - 1]]].reshape(hkv, 2, 16, d)[:, :, n_tok % 16:, :]
+    assert np.all(tail == 0x55)                                            # rows beyond the prompt untouched
+    assert fp8.kv_write(a, a, side, slot, k[:1], v[:1], np.zeros(1, np.int32), np.array([16 * nb], np.int32), table, hkv, d,
+                        fp8.F16, 0.25, 0.5) == -1
+    assert np.array_equal(a, b)
