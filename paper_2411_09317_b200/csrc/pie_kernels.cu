@@ -603,9 +603,9 @@ cudaError_t launch_kv_write8(const void *k, const void *v, const int32_t *token_
 }
 
 // The second launch bound: for 16-bit pools it only tells the assembler that it need not hold registers back for more
-// CTAs per SM than shared memory lets in anyway (three; without it some instantiations were capped at 96 registers and
-// spilled).  The 8-bit kernel is bound by instruction latency, not by bytes in flight, and its CTAs need a third of
-// the shared memory: five per SM (128 registers) measured 3-6 % faster than four.
+// CTAs per SM than shared memory lets in anyway (four of 50 KiB; without it some instantiations were capped at 96
+// registers and spilled).  The 8-bit kernel is bound by instruction latency, not by bytes in flight, and its CTAs need
+// less than half of the shared memory: five per SM (128 registers) measured 3-6 % faster than four.
 template <int D, bool BF16, int STAGES, int NW, bool KV8 = false>
 __global__ void __launch_bounds__((NW + 1) * 32, KV8 ? 5 : 1)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p) {
