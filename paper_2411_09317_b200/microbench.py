@@ -44,6 +44,7 @@ def main(argv=None):
     ap.add_argument("--q-heads", type=int, default=32)
     ap.add_argument("--kv-heads", type=int, default=8)
     ap.add_argument("--fp16", action="store_true", help="fp16 instead of bf16")
+    ap.add_argument("--kv-fp8", action="store_true", help="8-bit KV blocks (the attention beside the swaps, and part 3's write)")
     ap.add_argument("--blocks", default="", help="comma list of blocks per launch for part 2")
     ap.add_argument("--every", type=int, default=1, help="part 2: one swap call per this many launches, carrying as many times the blocks")
     args = ap.parse_args(argv)
@@ -55,7 +56,7 @@ def main(argv=None):
 
     n_swap_slots = 16384 if not args.quick else 2048
     wl = synth.Workload("swap_attn", 4, 1, args.q_heads, args.kv_heads, 128, synth.F16 if args.fp16 else synth.BF16,
-                        np.full(args.seqs, args.ctx, dtype=np.int32), 0, 0.0)
+                        np.full(args.seqs, args.ctx, dtype=np.int32), 0, 0.0, kv_fp8=args.kv_fp8)
     dw = DeviceWorkload(wl, host_frac=0.0, timing=False, extra_gpu_slots=n_swap_slots, extra_host_slots=n_swap_slots,
                         swap_ctas=args.swap_ctas, extra_tokens=0)
     BB = wl.block_bytes
@@ -186,7 +187,8 @@ def main(argv=None):
             dw.sync()
             times.append(e0.elapsed_time(e1))
         ms = float(np.median(times[1:]))
-        nbytes = 2 * 2 * T * wl.n_kv_heads * wl.head_dim * 2     # K and V, read once and written once
+        # K and V rows read once (16-bit) and written once (16-bit, or one byte per value into an 8-bit pool)
+        nbytes = 2 * T * wl.n_kv_heads * wl.head_dim * (2 + (1 if wl.kv_fp8 else 2))
         emit({"part": "kv_write", "tokens": T, "ms": ms, "gbs_read_plus_write": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes})
     dw.close()
 
