@@ -281,3 +281,17 @@ def test_governor_matches_oracle_on_random_reports(seed):
         elif k > target:
             k -= 1
     cg.close()
+
+
+def test_header_is_plain_c_and_cxx(tmp_path):
+    """include/pie.h must stand on its own for a C99 and a C++17 caller (no torch, no CUDA types in the signatures)."""
+    import os
+    import shutil
+    import subprocess
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    for comp, name, std in (("gcc", "t.c", "-std=c99"), ("g++", "t.cpp", "-std=c++17")):
+        if shutil.which(comp) is None:
+            pytest.skip(f"{comp} not installed")
+        src = tmp_path / name
+        src.write_text('#include "pie.h"\nint main(void) { pie_pool_config c; (void)c; return sizeof(pie_stats) > 0 ? 0 : 1; }\n')
+        subprocess.check_call([comp, std, "-Wall", "-Werror", "-pedantic", "-I", inc, "-fsyntax-only", str(src)])
