@@ -358,3 +358,23 @@ def test_arrival_driver_serves_every_request_and_sampled_outputs_match_the_oracl
     ids = pie.pie_block_alloc(d.pool, d.n_logical)
     assert len(set(ids.tolist())) == d.n_logical
     d.close()
+
+
+def test_bench_runs_at_reduced_scale_and_prints_the_contract_line():
+    """bench.py end to end on a fraction of the workload: one JSON line with the keys the measurement contract names."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--scale", "0.25", "--steps", "4", "--warmup", "3", "--ramp", "8",
+                        "--no-cpu-baseline"], capture_output=True, text=True, cwd=root, timeout=900)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline",
+                "dtype", "data", "config", "clocks", "e2e", "gpu_launches", "roofline", "cpu_baseline", "kv_fp8"):
+        assert key in line, key
+    assert line["value"] > 1000 and line["gpu_launches"] > 0 and line["config"]["workload"].startswith("llama2_7b")
+    assert set(line["roofline"]) >= {"bound", "achieved", "peak", "unit", "frac", "traffic"} and 0.3 < line["roofline"]["frac"] < 1.2
+    assert set(line["e2e"]) >= {"value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step"} and line["e2e"]["h2d_bytes_per_step"] > 0
+    assert line["kv_fp8"]["resident"]["attn_gbs"] > 500
