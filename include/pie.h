@@ -83,7 +83,7 @@ typedef struct pie_pool_config {
                                 * [1]: per-layer size visible to allocation at creation, in blocks (0 = n_logical_blocks;
                                 *      see pie_resize_begin);
                                 * [2]: 1 = the blocks hold K and V as FP8 E4M3 bytes (see pie_set_kv_scales): head_dim 128
-                                *      and variants 0, 1 only (PIE_ERR_UNSUPPORTED otherwise), block_bytes halves; rest 0 */
+                                *      and variants 0 - 2 only (PIE_ERR_UNSUPPORTED otherwise), block_bytes halves; rest 0 */
 } pie_pool_config;
 
 typedef struct pie_stats {

@@ -1307,7 +1307,7 @@ struct AttnVariant {
 };
 static const AttnVariant kVariants[] = {{2, 4}, {4, 8}, {2, 12}, {2, 6}, {4, 4}, {2, 8}, {1, 5}, {3, 6}, {1, 7}, {2, 4}, {1, 4}, {3, 3}, {1, 3}, {2, 2}};
 constexpr int kNumVariants = (int)(sizeof(kVariants) / sizeof(kVariants[0]));
-constexpr int kNumVariants8 = 2;
+constexpr int kNumVariants8 = 3;
 
 template <typename F>
 static cudaError_t dispatch_variant(int head_dim, int dtype, int variant, int kv_fp8, F &&f) {
@@ -1318,8 +1318,9 @@ static cudaError_t dispatch_variant(int head_dim, int dtype, int variant, int kv
     if (variant == IDX)                                                                                                                  \
         return dtype == PIE_BF16 ? f(paged_decode_attn_kernel<128, true, STV, NWV, true>, AttnSmem<128, STV, NWV, true>::BYTES, NWV)   \
                                  : f(paged_decode_attn_kernel<128, false, STV, NWV, true>, AttnSmem<128, STV, NWV, true>::BYTES, NWV);
-        PIE_VARIANT8(0, 2, 4)
-        PIE_VARIANT8(1, 2, 8)
+        PIE_VARIANT8(0, 2, 6)  // the most stages that still let five CTAs share an SM's shared memory
+        PIE_VARIANT8(1, 2, 4)
+        PIE_VARIANT8(2, 2, 8)
 #undef PIE_VARIANT8
         return cudaErrorInvalidValue;
     }

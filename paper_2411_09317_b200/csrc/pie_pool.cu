@@ -789,7 +789,7 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     if (cfg->block_tokens != 16 || (cfg->head_dim != 64 && cfg->head_dim != 128)) return PIE_ERR_UNSUPPORTED;
     if (cfg->n_q_heads / cfg->n_kv_heads > 8) return PIE_ERR_UNSUPPORTED;
     if (cfg->reserved[2] != 0 && cfg->reserved[2] != 1) return PIE_ERR_INVALID;
-    if (cfg->reserved[2] == 1 && (cfg->head_dim != 128 || cfg->reserved[0] < 0 || cfg->reserved[0] > 1)) return PIE_ERR_UNSUPPORTED;
+    if (cfg->reserved[2] == 1 && (cfg->head_dim != 128 || cfg->reserved[0] < 0 || cfg->reserved[0] > 2)) return PIE_ERR_UNSUPPORTED;
     if (cfg->split_tokens < 0 || cfg->split_tokens % 16 != 0) return PIE_ERR_INVALID;
     if (cfg->gpu_base && ((uintptr_t)cfg->gpu_base & 127)) return PIE_ERR_INVALID;
     if ((uint64_t)cfg->n_gpu_slots * (uint64_t)cfg->n_kv_heads * 32u > 0x7fffffffull) return PIE_ERR_UNSUPPORTED;

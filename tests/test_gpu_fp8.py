@@ -219,7 +219,7 @@ def test_argument_checks():
         pie.pie_pool_create(head_dim=64, kv_fp8=1, **kw)
     assert e.value.status == pie.PIE_ERR_UNSUPPORTED
     with pytest.raises(pie.PieError) as e:
-        pie.pie_pool_create(head_dim=128, kv_fp8=1, attn_variant=2, **kw)
+        pie.pie_pool_create(head_dim=128, kv_fp8=1, attn_variant=3, **kw)
     assert e.value.status == pie.PIE_ERR_UNSUPPORTED
     with pytest.raises(pie.PieError) as e:
         pie.pie_pool_create(head_dim=128, kv_fp8=2, **kw)
