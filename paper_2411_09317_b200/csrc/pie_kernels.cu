@@ -10,7 +10,7 @@
 namespace pie {
 
 // =====================================================================================================
-// Swap kernel (Section 4: "a CUDA kernel for efficient per-layer KV cache swapping"; here per block list)
+// Swap kernel (the per-layer swap kernel of Section 4, here per block list)
 // One work item = one 32 KiB chunk of one block.  Each thread issues UNROLL 16-byte loads before its
 // stores so that a CTA keeps 32 KiB in flight on the host link; a warp touches 512 contiguous bytes.
 // =====================================================================================================
@@ -226,6 +226,18 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
         return *reinterpret_cast<uint32_t *>(&v);
     }
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may become resident while
+// the kernel before it in the stream still runs; nothing that kernel wrote may be touched before this wait, which
+// returns once it has completed (at once for an ordinary launch).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long *p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+// slot-table entries are written by the copy streams while kernels run: read them from L2, never from a stale L1 line
+__device__ __forceinline__ int32_t ld_slot(const int32_t *p) { return __ldcg(p); }
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -441,8 +453,19 @@ struct AttnParams {
     float *part_o;
     float *part_ml;
     int32_t *counters;  // [0] next item, [1] CTAs that have left
-    uint64_t *stamps;   // optional, host visible: [0] when CTA 0 started, [1] when the last CTA left (globaltimer ns)
+    uint64_t *stamps;   // optional, host visible: [0] when CTA 0 started its main work, [1] when the last CTA left
+                        // (globaltimer ns), [2] how long CTA 0 waited for the layer's arriving units (ns), [3] the
+                        // batch's context tokens
     int32_t *status;
+    // Presence wait inside the kernel (Section 3.2): the copy-in stream stores a list's ticket into *arrive once the
+    // list's blocks and table entries have landed; no slot-table entry is read before *arrive >= arrive_need.
+    int32_t *tokens_out;               // optional: receives the batch's context-token count
+    // Completion word: the last CTA to leave stores done_value there once every CTA's writes (the appended rows among
+    // them) are visible; the copy streams wait for it by value instead of by an event on the compute stream.
+    unsigned long long *done_word;     // device memory, or NULL
+    unsigned long long done_value;
+    const unsigned long long *arrive;  // device word of this layer, or NULL
+    unsigned long long arrive_need;    // 0: nothing to wait for
     int64_t n_gpu_slots;
     int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d, max_chunks;
     float scale_log2e;      // softmax scale * log2(e) (* the key scale of an 8-bit pool)
@@ -631,8 +654,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     volatile int32_t *q_item = misc + 4;      // [4 .. 4 + QD)
     int32_t *co_smem = reinterpret_cast<int32_t *>(smem + SM::OFF_CO);
 
+    // The combine kernel that follows may become resident at once (its CTAs wait for this grid to complete before they
+    // read anything): its launch then costs nothing at the end of this kernel.
+    grid_launch_dependents();
+    // Everything up to the dependency wait below touches only shared memory and the call's own inputs (lengths and
+    // tables, which no kernel of the path writes): under a programmatic dependent launch it overlaps the tail of the
+    // kernel before it in the stream.
     if (tid == 0) {
-        if (p.stamps != nullptr && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps) = globaltimer_ns();
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
@@ -663,7 +691,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             __syncthreads();
             atomicAdd(const_cast<int32_t *>(misc + 2), my_tokens);
             __syncthreads();
-            if (tid == 0) *reinterpret_cast<volatile int32_t *>(p.status + 3) = misc[2];
+            if (tid == 0) {
+                if (p.tokens_out != nullptr) *reinterpret_cast<volatile int32_t *>(p.tokens_out) = misc[2];
+                if (p.stamps != nullptr) *reinterpret_cast<volatile uint64_t *>(p.stamps + 3) = (uint64_t)misc[2];
+            }
         }
         __syncthreads();
         if (warp == 0) {
@@ -684,6 +715,11 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
     }
     __syncthreads();
+    grid_dependency_wait();
+    if (tid == 0 && p.stamps != nullptr && blockIdx.x == 0) {
+        *reinterpret_cast<volatile uint64_t *>(p.stamps) = globaltimer_ns();
+        if (p.arrive_need == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = 0;   // every launch writes all its stamps
+    }
     const int32_t *co = co_in_smem ? co_smem : p.chunk_off_global;
     int32_t n_chunks_total = co[p.n_seqs];
     if (n_chunks_total > p.max_chunks) {  // more chunks than the partials buffer holds: compute nothing, flag it
@@ -696,7 +732,30 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     if (warp == ATT_NW) {
         // ------------------------------------------------------------------ producer warp
-        int32_t next = lane == 0 ? atomicAdd(p.counters, 1) : 0;
+        // presence wait (Section 3.2): no slot-table entry of this layer is read before the list that brings the
+        // layer's units has landed.  Bounded (about half a second of polling): then the CTA flags it and leaves.
+        if (p.arrive_need != 0) {
+            if (lane == 0) {
+                const uint64_t t_begin = globaltimer_ns();
+                bool there = false;
+                for (uint32_t i = 0; i < (1u << 21); ++i) {
+                    if (ld_acquire_u64(p.arrive) >= p.arrive_need) {
+                        there = true;
+                        break;
+                    }
+                    if (i > 16) __nanosleep(250);
+                }
+                if (!there) {
+                    raise_status(p.status, STATUS_WAIT_TIMEOUT);
+                    *abort_flag = 1;
+                }
+                if (p.stamps != nullptr && blockIdx.x == 0)
+                    *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = globaltimer_ns() - t_begin;
+            }
+            __syncwarp();
+        }
+        // the first item is the CTA's own number, the later ones come from the global counter
+        int32_t next = lane == 0 ? (int32_t)blockIdx.x : 0;
         for (;;) {
             int32_t item = -1;
             if (lane == 0) {
@@ -720,7 +779,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     mbar_expect_tx(bar_qfull + 8 * qs, bytes);
                     bulk_load(smem_base + SM::OFF_Q + qs * SM::Q_BYTES,
                               p.q + ((int64_t)lo * p.n_q_heads + (int64_t)kvh * p.group) * D, bytes, bar_qfull + 8 * qs);
-                    next = atomicAdd(p.counters, 1);  // the next item's id: its latency hides behind this item's tiles
+                    next = (int32_t)gridDim.x + atomicAdd(p.counters, 1);  // the next item's id: its latency hides behind this item's tiles
                 } else {
                     mbar_arrive(bar_qfull + 8 * qs);
                 }
@@ -734,7 +793,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 int32_t slot = -1;
                 if (base + lane < it.ntiles) {
                     const int32_t blk = __ldg(bt + base + lane);
-                    if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
+                    if (blk >= 0 && blk < p.n_logical) slot = ld_slot(p.slot_table + blk);
                     if (slot >= p.n_gpu_slots) slot = -1;
                 }
                 const int32_t cnt = min(32, it.ntiles - base);
@@ -885,7 +944,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     int32_t slot = -1;
                     if (lane == 0) {
                         const int32_t blk = __ldg(p.block_table + (int64_t)it.s * p.max_blocks + (pos >> 4));
-                        if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
+                        if (blk >= 0 && blk < p.n_logical) slot = ld_slot(p.slot_table + blk);
                         if (slot >= p.n_gpu_slots) slot = -1;
                     }
                     slot = __shfl_sync(0xffffffffu, slot, 0);
@@ -962,7 +1021,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     int32_t slot = -1;
                     if (lane == 0) {
                         const int32_t blk = __ldg(p.block_table + (int64_t)it.s * p.max_blocks + (pos >> 4));
-                        if (blk >= 0 && blk < p.n_logical) slot = __ldg(p.slot_table + blk);
+                        if (blk >= 0 && blk < p.n_logical) slot = ld_slot(p.slot_table + blk);
                         if (slot >= p.n_gpu_slots) slot = -1;
                     }
                     slot = __shfl_sync(0xffffffffu, slot, 0);
@@ -1140,21 +1199,31 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         ++qn;
     }
     // the last CTA to leave resets the work counter for the next launch (every CTA has drawn its end marker by then)
+    if (p.done_word != nullptr) {
+        consumer_sync<NCONS>();   // the CTA's consumer warps have issued all their writes
+    }
     if (tid == 0) {
+        if (p.done_word != nullptr) __threadfence();   // ... and they are visible before this CTA counts as gone
         const int32_t old = atomicAdd(p.counters + 1, 1);
         if (old == (int32_t)gridDim.x - 1) {
             p.counters[0] = 0;
             p.counters[1] = 0;
             if (p.stamps != nullptr) *reinterpret_cast<volatile uint64_t *>(p.stamps + 1) = globaltimer_ns();
+            if (p.done_word != nullptr) {
+                __threadfence();
+                *reinterpret_cast<volatile unsigned long long *>(p.done_word) = p.done_value;
+            }
         }
     }
 }
 
 // =====================================================================================================
-// Combine: one CTA per (sequence, KV head, 32-wide slice of head_dim) merges the sequence's chunk partials in chunk
-// order with the log-sum-exp rule, normalises and rounds to the 16-bit output type (nearest even).  Sequences with
-// fewer than two chunks were finished by the attention kernel.  The per-(head, chunk) weights are computed once in
-// shared memory; the accumulation keeps eight 16-byte loads in flight per thread.
+// Combine: one CTA per (sequence, KV head, slice of head_dim) merges the sequence's chunk partials in chunk order with
+// the log-sum-exp rule, normalises and rounds to the 16-bit output type (nearest even).  Sequences with fewer than two
+// chunks were finished by the attention kernel.  The per-(head, chunk) weights are computed once in shared memory (sized
+// by the launch for the longest sequence the table allows, so that the whole grid is resident at once: the kernel sits
+// between two layers' attention kernels and every wave of it is dead time); the accumulation keeps eight 16-byte loads
+// in flight per thread.  The slice is the whole head_dim for batches of many (sequence, head) pairs and 32 for few.
 // =====================================================================================================
 constexpr int COMB_THREADS = 64;
 constexpr int COMB_CAP = 256;  // chunks per sequence handled through shared memory; beyond that, plain loops
@@ -1162,29 +1231,32 @@ constexpr int COMB_CAP = 256;  // chunks per sequence handled through shared mem
 template <int D, bool BF16>
 __global__ void __launch_bounds__(COMB_THREADS)
 combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, const int32_t *__restrict__ chunk_off,
-               uint16_t *__restrict__ out, int32_t n_q_heads, int32_t n_kv_heads, int32_t group) {
-    __shared__ float wbuf[8][COMB_CAP];
-    __shared__ float lbuf[8][COMB_CAP];
-    // Launched with programmatic stream serialization: CTAs may become resident while the attention kernel's last
-    // CTAs are still running (which hides the launch latency); nothing that kernel wrote is read before this wait,
-    // which returns once the attention grid has completed and its writes are visible.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+               uint16_t *__restrict__ out, int32_t n_q_heads, int32_t n_kv_heads, int32_t group, int32_t cap) {
+    extern __shared__ __align__(16) float comb_smem[];   // wbuf[group][cap], lbuf[group][cap]
+    float *wbuf = comb_smem, *lbuf = comb_smem + group * cap;
+    // Launched with programmatic stream serialization: CTAs may become resident while the attention kernel still runs
+    // (which hides the launch); nothing that kernel wrote is read before the wait, which returns once the attention
+    // grid has completed and its writes are visible.  The kernel after this one may be launched the same way: let its
+    // CTAs become resident as soon as this grid's have started (it touches nothing of ours before its own wait).
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int tid = threadIdx.x;
     const int32_t s = blockIdx.x / n_kv_heads, kvh = blockIdx.x - s * n_kv_heads;
     const int32_t chunk0 = chunk_off[s], nchunks = chunk_off[s + 1] - chunk0;
     if (nchunks < 2) return;
-    const int d_lo = blockIdx.y * 32;  // this CTA's slice of head_dim
+    const int width = D / (int)gridDim.y;  // this CTA's slice of head_dim
+    const int d_lo = blockIdx.y * width;
     const int64_t row0 = ((int64_t)s * n_q_heads + (int64_t)kvh * group) * D;
-    if (nchunks <= COMB_CAP) {
+    if (nchunks <= cap) {
         for (int idx = tid; idx < group * nchunks; idx += COMB_THREADS) {
             const int g = idx / nchunks, c = idx - g * nchunks;
             const int64_t id = ((int64_t)(chunk0 + c) * n_kv_heads + kvh) * group + g;
-            wbuf[g][c] = part_ml[id * 2];
-            lbuf[g][c] = part_ml[id * 2 + 1];
+            wbuf[g * cap + c] = part_ml[id * 2];
+            lbuf[g * cap + c] = part_ml[id * 2 + 1];
         }
         __syncthreads();
         if (tid < group) {
-            float *w = wbuf[tid], *l = lbuf[tid];
+            float *w = wbuf + tid * cap, *l = lbuf + tid * cap;
             float mm = -INFINITY;
             for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, w[c]);
             float ll = 0.f;
@@ -1196,8 +1268,9 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
             l[0] = ll > 0.f ? 1.f / ll : 0.f;
         }
         __syncthreads();
-        for (int e4 = tid; e4 < group * 8; e4 += COMB_THREADS) {  // 8 float4 pieces per head in a 32-wide slice
-            const int g = e4 >> 3, d = d_lo + (e4 & 7) * 4;
+        const int per_head = width / 4;   // float4 pieces per head in the slice
+        for (int e4 = tid; e4 < group * per_head; e4 += COMB_THREADS) {
+            const int g = e4 / per_head, d = d_lo + (e4 - g * per_head) * 4;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int32_t c0 = 0; c0 < nchunks; c0 += 8) {
                 float4 v[8];
@@ -1210,14 +1283,14 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (c0 + j < nchunks) {
-                        const float wt = wbuf[g][c0 + j];
+                        const float wt = wbuf[g * cap + c0 + j];
                         acc.x += v[j].x * wt;
                         acc.y += v[j].y * wt;
                         acc.z += v[j].z * wt;
                         acc.w += v[j].w * wt;
                     }
             }
-            const float inv = lbuf[g][0];
+            const float inv = lbuf[g * cap];
             uint2 r;
             r.x = pack2<BF16>(acc.x * inv, acc.y * inv);
             r.y = pack2<BF16>(acc.z * inv, acc.w * inv);
@@ -1225,8 +1298,8 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
         }
         return;
     }
-    for (int e = tid; e < group * 32; e += COMB_THREADS) {  // very many chunks: plain loops
-        const int g = e >> 5, d = d_lo + (e & 31);
+    for (int e = tid; e < group * width; e += COMB_THREADS) {  // very many chunks: plain loops
+        const int g = e / width, d = d_lo + (e - g * width);
         float mm = -INFINITY;
         for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, part_ml[(((int64_t)(chunk0 + c) * n_kv_heads + kvh) * group + g) * 2]);
         float acc = 0.f, ll = 0.f;
@@ -1401,6 +1474,11 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.counters = sc.counters;
     p.stamps = a.stamps;
     p.status = a.status;
+    p.tokens_out = a.tokens_out;
+    p.done_word = a.done_word;
+    p.done_value = a.done_value;
+    p.arrive = a.arrive;
+    p.arrive_need = a.arrive != nullptr ? a.arrive_need : 0ull;
     p.n_gpu_slots = sh.n_gpu_slots;
     p.max_blocks = a.max_blocks;
     p.n_seqs = a.n_seqs;
@@ -1419,15 +1497,35 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     }
     if (a.k_new == nullptr || a.v_new == nullptr) p.k_new = p.v_new = nullptr;
     cudaError_t e = dispatch_variant(sh.head_dim, sh.dtype, a.variant, sh.kv_fp8, [&](auto kernel, int smem, int nw) -> cudaError_t {
-        kernel<<<a.grid, (nw + 1) * 32, smem, stream>>>(map, p);
-        return cudaGetLastError();
+        if (!a.dependent_launch) {
+            kernel<<<a.grid, (nw + 1) * 32, smem, stream>>>(map, p);
+            return cudaGetLastError();
+        }
+        // behind the previous layer's combine kernel: the CTAs may become resident, set their barriers up and scan the
+        // batch's lengths while that kernel drains; they wait for it before anything else
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)a.grid);
+        lc.blockDim = dim3((unsigned)((nw + 1) * 32));
+        lc.dynamicSmemBytes = (size_t)smem;
+        lc.stream = stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+        return cudaLaunchKernelEx(&lc, kernel, map, p);
     });
     if (e != cudaSuccess) return e;
     // merge the partials of sequences that span several chunks (CTAs of single-chunk sequences return at once)
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(a.n_seqs * sh.n_kv_heads), (unsigned)(sh.head_dim / 32));
+    // chunks of the longest sequence the table allows (rounded up to a multiple of 8: the loads go in eights)
+    const int64_t longest = ((int64_t)a.max_blocks * 16 + a.split_tokens - 1) / a.split_tokens;
+    const int32_t cap = (int32_t)std::min<int64_t>(COMB_CAP, (longest + 7) / 8 * 8);
+    // whole head_dim per CTA where there are enough (sequence, head) pairs to fill the GPU; 32-wide slices otherwise
+    const int64_t pairs = (int64_t)a.n_seqs * sh.n_kv_heads;
+    cfg.gridDim = dim3((unsigned)pairs, (unsigned)(pairs >= 1024 ? 1 : sh.head_dim / 32));
     cfg.blockDim = dim3(COMB_THREADS);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = (size_t)(2 * p.group * cap) * sizeof(float);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1439,10 +1537,10 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     const int32_t *co = sc.chunk_off;
     const int32_t hq = sh.n_q_heads, hkv = sh.n_kv_heads, group = p.group;
     if (sh.head_dim == 128)
-        return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<128, true>, po, pml, co, out, hq, hkv, group)
-                                    : cudaLaunchKernelEx(&cfg, combine_kernel<128, false>, po, pml, co, out, hq, hkv, group);
-    return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<64, true>, po, pml, co, out, hq, hkv, group)
-                                : cudaLaunchKernelEx(&cfg, combine_kernel<64, false>, po, pml, co, out, hq, hkv, group);
+        return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<128, true>, po, pml, co, out, hq, hkv, group, cap)
+                                    : cudaLaunchKernelEx(&cfg, combine_kernel<128, false>, po, pml, co, out, hq, hkv, group, cap);
+    return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<64, true>, po, pml, co, out, hq, hkv, group, cap)
+                                : cudaLaunchKernelEx(&cfg, combine_kernel<64, false>, po, pml, co, out, hq, hkv, group, cap);
 }
 
 }  // namespace pie

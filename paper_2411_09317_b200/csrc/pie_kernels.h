@@ -75,7 +75,15 @@ struct AttnLaunch {
     int32_t grid;               // persistent CTAs
     int32_t variant;            // kernel variant (0 = default)
     int32_t *status;            // device-visible status word
-    uint64_t *stamps = nullptr; // optional, device-visible: [0] start, [1] end of the attention kernel (GPU timer, ns)
+    uint64_t *stamps = nullptr; // optional, device-visible: [0] start, [1] end of the attention kernel (GPU timer, ns),
+                                // [2] ns CTA 0 waited for arriving units, [3] the batch's context tokens
+    unsigned long long *done_word = nullptr;  // optional, device memory: the kernel's last CTA stores done_value there
+    unsigned long long done_value = 0;        // (the call's compute ticket: copy streams wait for it by value)
+    int32_t *tokens_out = nullptr;  // optional, device-visible: receives the batch's context-token count
+    const unsigned long long *arrive = nullptr;  // presence wait inside the kernel: wait until *arrive >= arrive_need
+    unsigned long long arrive_need = 0;          // (the copy-in stream stores a list's ticket there behind its copies)
+    bool dependent_launch = false;  // launch with programmatic stream serialization: only where the kernel before it in
+                                    // the stream writes none of this call's lengths and tables
     float k_scale = 1.f, v_scale = 1.f;  // 8-bit pools: a stored byte stands for decode(byte) * scale
 };
 

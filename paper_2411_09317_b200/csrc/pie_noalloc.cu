@@ -129,6 +129,7 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
     a.variant = 0;
     a.grid = setup->ctas_per_sm[head_dim == 128][dtype] * setup->n_sms;
     a.status = status_dev ? status_dev : reinterpret_cast<int32_t *>(setup->scratch + OFF_STATUS);
+    a.tokens_out = a.status + 3;
     if (a.grid <= 0) return PIE_ERR_UNSUPPORTED;
     if (pie::launch_attention(sh, sc, a, use3d ? map3d : map2d, use3d, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return PIE_ERR_CUDA;

@@ -42,15 +42,29 @@ struct LayerEvents {
     // the kernel's start).
     cudaEvent_t in0 = nullptr, in1 = nullptr, out0 = nullptr, out1 = nullptr;
     bool has_in = false, has_out = false, has_compute = false;
+    bool stream_wait = false;   // the layer's attention call made the compute stream wait for a copy's event
 };
 // per layer of a step: GPU-timer stamps in mapped pinned memory
-enum { STAMP_START = 0, STAMP_END = 1, STAMP_WORDS = 2 };
+// START: CTA 0 begins its main work (after the dependency wait), END: the last CTA leaves, WAIT: ns CTA 0's producer
+// spent in the presence wait, TOKENS: the batch's context tokens
+enum { STAMP_START = 0, STAMP_END = 1, STAMP_WAIT = 2, STAMP_TOKENS = 3, STAMP_WORDS = 4 };
+constexpr int MAX_GROUP_LAYERS = 8;  // layers whose swap lists are issued together (pie_set_lookahead)
 
 struct ListRecord {
     int64_t start, end;
     int ev;          // index into list_events, or -1: guarded by a ticket of a queue (its event is recorded by the caller)
     int queue;
     int64_t ticket;
+};
+
+// One swap list after phase 1 of the table update (Section 3.2): destination slots chosen and recorded, source slots
+// released under the list's ticket; nothing enqueued yet.
+struct SwapList {
+    int32_t layer = 0;
+    int64_t ticket = 0, n_moved = 0, n_elided = 0;
+    std::vector<int32_t> moved, src, dst;
+    std::vector<uint8_t> elide;
+    int64_t waits[4] = {0, 0, 0, 0};
 };
 
 }  // namespace
@@ -65,11 +79,40 @@ struct pie_pool {
     bool own_gpu = false, own_host = false, own_streams = false;
     cudaStream_t stream[4] = {nullptr, nullptr, nullptr, nullptr};  // indexed by queue id
     cudaEvent_t ticket_ev[4][EV_RING] = {};
-    // Compute tickets have two sets of events; ticket_ev[PIE_Q_COMPUTE][i] points at the one its newest record used.
+    // Marks on the compute stream come from two rings of events (compute_mark picks per record).
     // A record without a time stamp is ~2.5 us cheaper between two kernels, but when another stream waits on such an
     // event the recording stream loses ~5 us instead (measured on this part and driver): so plain events while
     // nothing is being swapped, time-stamped ones while swap lists, which wait on compute tickets, are in flight.
     cudaEvent_t compute_ev_plain[EV_RING] = {}, compute_ev_stamped[EV_RING] = {};
+    // An event on the compute stream between two layers costs every layer a few microseconds (and keeps the next
+    // attention kernel from being launched as a dependent of the previous one), so compute tickets get an event only
+    // where somebody has to wait for one: a mark is recorded at the stream's tail and covers every ticket enqueued so far.
+    struct ComputeMark {
+        int64_t ticket;
+        cudaEvent_t ev;
+    };
+    // Where the driver offers stream waits by value, the copy streams do not need a mark either: the attention kernel's
+    // last CTA stores its call's ticket in a device word and a copy stream waits until the word has reached the ticket
+    // it needs.  A mark between two layers serialises the next kernel's launch behind it, and that launch is slow while
+    // swap lists are crossing the host link; the word costs the compute stream nothing.
+    unsigned long long *done_dev = nullptr;   // newest compute ticket whose attention kernel has completed
+    int64_t last_attn_ticket = 0;             // newest compute ticket an attention kernel will store there
+    CUresult (*wait_value64)(CUstream, CUdeviceptr, cuuint64_t, unsigned int) = nullptr;
+    std::deque<ComputeMark> compute_marks;   // recorded, not yet known complete; tickets ascending
+    int compute_ev_next = 0;                 // next slot of the two event rings
+    int64_t compute_marked = 0;              // newest compute ticket that a recorded mark covers
+    // Presence wait inside the attention kernel: per layer a device word that the copy-in stream sets to a list's ticket
+    // (a small copy behind the list's blocks and table entries).  Lists moved or patched by an SM kernel are waited for
+    // with a stream-level event wait instead: a kernel that polls while it owns the SMs must not wait for another kernel.
+    unsigned long long *arrive_dev = nullptr;   // [n_layers]
+    std::vector<int64_t> layer_in_sm;           // per layer: newest in-ticket that involved an SM kernel
+    std::vector<int64_t> layer_in_last;         // per layer: newest in-ticket whose list sets the layer's arrival word
+    // Swap lists are issued for a group of consecutive layers at a time: while a group computes, the next group's shares
+    // arrive and the previous group's leave; one mark on the compute stream per group.
+    int32_t group_setting = 0;                  // 0: chosen per group from the staging the GPU pool can afford
+    int32_t group_first = 0, group_len = 0;     // the group in progress (group_len 0: none)
+    std::vector<int32_t> group_done;            // its layers that have computed and whose share has yet to go out
+    int32_t group_mode = PIE_MODE_AUTO;
     int64_t last_swap_step = -2;   // the step in which the newest swap list was issued
     int64_t recorded[4] = {0, 0, 0, 0};  // newest ticket of each queue whose event has been recorded
     int32_t *slot_table_dev = nullptr;  // [L][NB]
@@ -81,11 +124,10 @@ struct pie_pool {
     int list_ev_next = 0;
     // device status word (mapped pinned memory)
     int32_t *status_host = nullptr, *status_dev = nullptr;
-    uint64_t *stamps_host = nullptr, *stamps_dev = nullptr;  // [TIMING_RING][n_layers][STAMP_WORDS]
+    uint64_t *stamps_host = nullptr, *stamps_dev = nullptr;  // [TIMING_RING][n_layers][STAMP_WORDS]: pinned copy, device original
     uint64_t free_step_gap_ns = 0;   // smallest gap between two layers' attention kernels in the newest step without swaps
     uint64_t prev_step_end = 0;   // GPU-timer stamp of the end of the last layer of the newest evaluated step
     int64_t prev_step_id = -1;
-    uint32_t prev_step_prefetched = 0;   // bit l: that step issued a swap-in list for layer l (l < 8)
     // attention
     pie::AttnScratch scratch{};
     CUtensorMap map3d{}, map2d{};
@@ -115,15 +157,20 @@ struct pie_pool {
     std::vector<LayerEvents> lev[TIMING_RING];
     int64_t lev_step[TIMING_RING] = {};      // which step a set holds (0 = none)
     bool lev_done[TIMING_RING] = {};         // already evaluated
+    bool lev_closed[TIMING_RING] = {};       // the step's last compute ticket has its mark (or needs none)
     cudaEvent_t lev_anchor[TIMING_RING] = {};   // timing = 2: recorded on the compute stream before the step's first attention kernel
     bool lev_anchored[TIMING_RING] = {};
     cudaEvent_t lev_last[TIMING_RING][4] = {};  // the set's newest event on each queue's stream (its streams complete in order)
+    cudaStream_t aux_stream = nullptr;          // brings a step's stamps to the host without touching the compute stream
+    cudaEvent_t lev_close_ev[TIMING_RING] = {}; // recorded there behind the copy
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
     std::vector<float> timeline;     // last evaluated step: [L][7] ms from the step's first event (-1 = not recorded)
     pie_stats stats{};
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
+    SwapList one_list;                  // the list of a single swap call
+    std::vector<SwapList> group_lists;  // the lists of a group of layers (decode loop)
     std::vector<uint8_t> v_elide;
     cudaStream_t io_stream[2] = {nullptr, nullptr};  // pie_decode_step_host: inputs up / results down
     std::vector<cudaEvent_t> io_up;                   // one per group of layers: its inputs have arrived
@@ -139,7 +186,22 @@ namespace {
 // decode step holds the poll (one forced poll per layer there), the calls inside it skip their own.
 int poll(pie_pool *p, bool force = false) {
     if (p->poll_hold && !force) return PIE_OK;
-    for (int q = 1; q <= 3; ++q) {
+    {
+        int64_t d = p->table->done(PIE_Q_COMPUTE);
+        while (!p->compute_marks.empty()) {
+            cudaError_t e = cudaEventQuery(p->compute_marks.front().ev);
+            if (e == cudaErrorNotReady) break;
+            if (e != cudaSuccess) {
+                g_last_cuda_error = (int)e;
+                p->sticky = PIE_ERR_CUDA;
+                return PIE_ERR_CUDA;
+            }
+            d = std::max(d, p->compute_marks.front().ticket);
+            p->compute_marks.pop_front();
+        }
+        if (d > p->table->done(PIE_Q_COMPUTE)) p->table->confirm(PIE_Q_COMPUTE, d);
+    }
+    for (int q = 1; q <= 2; ++q) {
         int64_t d = p->table->done(q);
         const int64_t issued = p->recorded[q];  // a ticket whose event is not recorded yet cannot be queried
         while (d < issued) {
@@ -157,15 +219,62 @@ int poll(pie_pool *p, bool force = false) {
     return PIE_OK;
 }
 
+// Record a mark at the compute stream's tail: it covers every compute ticket enqueued so far.
+int push_mark(pie_pool *p, cudaEvent_t *ev) {
+    if ((int)p->compute_marks.size() >= EV_RING - 1) {  // the ring is full: its oldest mark must complete first
+        PIE_CUDA(cudaEventSynchronize(p->compute_marks.front().ev));
+        int st = poll(p, true);
+        if (st != PIE_OK) return st;
+    }
+    const int slot = p->compute_ev_next;
+    p->compute_ev_next = (slot + 1) % EV_RING;
+    // (a time-stamped event is the cheaper one for the recording stream when other streams wait on it)
+    cudaEvent_t e = p->last_swap_step >= p->step - 1 ? p->compute_ev_stamped[slot] : p->compute_ev_plain[slot];
+    PIE_CUDA(cudaEventRecord(e, p->stream[PIE_Q_COMPUTE]));
+    p->compute_marked = p->recorded[PIE_Q_COMPUTE];
+    p->compute_marks.push_back({p->compute_marked, e});
+    *ev = e;
+    return PIE_OK;
+}
+
+// The mark that covers compute ticket t: the oldest recorded one at or after it; recorded now, at the stream's tail,
+// if there is none yet.  *ev stays null when the ticket is already known complete.
+int compute_mark(pie_pool *p, int64_t t, cudaEvent_t *ev) {
+    *ev = nullptr;
+    if (t <= 0 || t <= p->table->done(PIE_Q_COMPUTE)) return PIE_OK;
+    if (t > p->compute_marked) return push_mark(p, ev);
+    for (const pie_pool::ComputeMark &m : p->compute_marks)
+        if (m.ticket >= t) {
+            *ev = m.ev;
+            break;
+        }
+    return PIE_OK;
+}
+
 // make `stream` wait for ticket t of queue q (no-op if already known complete)
 int wait_ticket(pie_pool *p, cudaStream_t stream, int q, int64_t t) {
     if (t <= 0 || t <= p->table->done(q)) return PIE_OK;
+    if (q == PIE_Q_COMPUTE && p->wait_value64 && t <= p->last_attn_ticket && stream != p->stream[PIE_Q_COMPUTE]) {
+        if (p->wait_value64((CUstream)stream, (CUdeviceptr)(uintptr_t)p->done_dev, (cuuint64_t)t, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS) {
+            g_last_cuda_error = (int)cudaErrorUnknown;
+            return PIE_ERR_CUDA;
+        }
+        return PIE_OK;
+    }
+    if (q == PIE_Q_COMPUTE) {
+        cudaEvent_t ev = nullptr;
+        int st = compute_mark(p, t, &ev);
+        if (st != PIE_OK) return st;
+        if (ev) PIE_CUDA(cudaStreamWaitEvent(stream, ev, 0));
+        return PIE_OK;
+    }
     PIE_CUDA(cudaStreamWaitEvent(stream, p->ticket_ev[q][t % EV_RING], 0));
     return PIE_OK;
 }
 
 // before ticket t of queue q records its event: the slot's previous user (t - EV_RING) must be done
 int reserve_ticket_event(pie_pool *p, int q, int64_t t) {
+    if (q == PIE_Q_COMPUTE) return PIE_OK;  // compute tickets share marks (compute_mark)
     const int64_t prev = t - EV_RING;
     if (prev > 0 && prev > p->table->done(q)) {
         PIE_CUDA(cudaEventSynchronize(p->ticket_ev[q][prev % EV_RING]));
@@ -175,8 +284,10 @@ int reserve_ticket_event(pie_pool *p, int q, int64_t t) {
 }
 
 int record_ticket(pie_pool *p, int q, int64_t t) {
-    if (q == PIE_Q_COMPUTE)
-        p->ticket_ev[q][t % EV_RING] = p->last_swap_step >= p->step - 1 ? p->compute_ev_stamped[t % EV_RING] : p->compute_ev_plain[t % EV_RING];
+    if (q == PIE_Q_COMPUTE) {  // enqueued; an event follows only if somebody has to wait for it (compute_mark)
+        p->recorded[q] = t;
+        return PIE_OK;
+    }
     PIE_CUDA(cudaEventRecord(p->ticket_ev[q][t % EV_RING], p->stream[q]));
     p->recorded[q] = t;
     return PIE_OK;
@@ -257,8 +368,11 @@ uint64_t *stamp_dev(pie_pool *p, int32_t layer, int which) {
 // ---- one swap call ------------------------------------------------------------------------------------
 // elide (optional): pairs flagged 1 move no bytes (a kept, unwritten host copy); they still get their table entry
 // patched, and they force the copy-engine path: the gather/scatter kernel takes the whole list.
+// arrive (optional, device): behind the list's copies and table entries the ticket is stored there by one small copy -
+// the word the layer's attention kernel waits for; *used_sm tells whether an SM kernel moved or patched the list.
 int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst, int64_t n, const int32_t *blocks,
-              int32_t *slot_table_row, int mode, cudaStream_t stream, int64_t ticket = 0, const uint8_t *elide = nullptr) {
+              int32_t *slot_table_row, int mode, cudaStream_t stream, int64_t ticket = 0, const uint8_t *elide = nullptr,
+              unsigned long long *arrive = nullptr, bool *used_sm = nullptr) {
     // dir_queue PIE_Q_IN: host -> GPU; PIE_Q_OUT: GPU -> host
     const uint8_t *src_pool = dir_queue == PIE_Q_IN ? p->host_base : p->gpu_base;
     uint8_t *dst_pool = dir_queue == PIE_Q_IN ? p->gpu_base : p->host_base;
@@ -293,8 +407,11 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         dma_patch = id_runs <= PATCH_DMA_MAX_RUNS;
     }
     const bool by_kernel = mode == PIE_MODE_KERNEL || mode == PIE_MODE_KERNEL_BULK;
-    const bool need_list = by_kernel || slot_table_row != nullptr;
-    const int64_t list_len = dma_patch ? n : 3 * n;
+    if (arrive != nullptr && ticket <= 0) arrive = nullptr;
+    const bool need_list = by_kernel || slot_table_row != nullptr || arrive != nullptr;
+    const int64_t body_len = ((dma_patch ? n : 3 * n) + 3) & ~int64_t(3);
+    const int64_t list_len = body_len + (arrive ? 4 : 0);   // the ticket for the arrival word sits behind the list
+    if (used_sm) *used_sm = by_kernel || (mode == PIE_MODE_COPY_ENGINE && slot_table_row != nullptr && !dma_patch);
     int64_t off = 0;
     if (need_list && dma_patch) {
         int st = list_alloc(p, list_len, &off);
@@ -305,7 +422,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         int st = list_alloc(p, list_len, &off);
         if (st != PIE_OK) return st;
         int32_t *h = p->list_host + off;
-        for (int64_t i = 0; i < n; ++i) {
+        for (int64_t i = 0; i < n && (by_kernel || slot_table_row != nullptr); ++i) {
             h[3 * i + 0] = src[i];
             h[3 * i + 1] = dst[i];
             h[3 * i + 2] = blocks ? blocks[i] : 0;
@@ -353,6 +470,11 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
         }
         p->stats.calls_copy_engine += 1;
     }
+    if (arrive) {
+        unsigned long long *h = reinterpret_cast<unsigned long long *>(p->list_host + off + body_len);
+        *h = (unsigned long long)ticket;
+        PIE_CUDA(cudaMemcpyAsync(arrive, h, 8, cudaMemcpyHostToDevice, stream));
+    }
     if (need_list) {
         if (ticket > 0) {
             list_commit_ticket(p, off, list_len, dir_queue, ticket);
@@ -364,9 +486,178 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
     return PIE_OK;
 }
 
-// not_before: a compute ticket the copy must not start before (0 = none).  The decode loop uses it to start the
-// prefetch of layer l+1 when layer l starts computing (Section 3.3), not as early as the host happens to run ahead:
-// that keeps a unit on the host for as long as possible and the GPU staging share at a few layers' worth.
+int swap_prepare(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t n, SwapList *out) {
+    out->layer = layer;
+    out->ticket = out->n_moved = out->n_elided = 0;
+    if (n == 0) return (layer < 0 || layer >= p->cfg.n_layers) ? PIE_ERR_RANGE : PIE_OK;
+    out->moved.resize((size_t)n);
+    out->src.resize((size_t)n);
+    out->dst.resize((size_t)n);
+    out->elide.resize((size_t)n);
+    int st = p->table->swap(queue, layer, ids, n, &out->ticket, out->moved.data(), out->src.data(), out->dst.data(), &out->n_moved,
+                            out->waits, out->elide.data());
+    if (st != PIE_OK || out->n_moved == 0) return st;
+    p->last_swap_step = p->step;
+    for (int64_t i = 0; i < out->n_moved; ++i) out->n_elided += out->elide[(size_t)i];
+    // a unit that is pushed out belongs to the host-resident set from now on; bringing it in for a layer's
+    // turn does not take it out of the set (only a lower ratio does)
+    if (queue == PIE_Q_OUT)
+        for (int64_t i = 0; i < out->n_moved; ++i) {
+            pie::Unit &u = p->table->unit(layer, out->moved[(size_t)i]);
+            if (!u.home_host) {
+                u.home_host = 1;
+                p->home_count[(size_t)layer] += 1;
+                p->home_dirty[(size_t)layer] = 1;
+            }
+        }
+    return PIE_OK;
+}
+
+// Phase 1 is done: a failure from here on leaves the pool unusable (sticky) rather than inconsistent.
+#define PIE_STICKY(expr)                  \
+    do {                                  \
+        int st__ = (expr);                \
+        if (st__ != PIE_OK) {             \
+            p->sticky = st__;             \
+            return st__;                  \
+        }                                 \
+    } while (0)
+
+void swap_account(pie_pool *p, int queue, const SwapList &l) {
+    (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)(l.n_moved - l.n_elided) * (double)p->block_bytes;
+    p->stats.reserved[2] += (double)l.n_elided * (double)p->block_bytes;
+}
+
+// not_before: a compute ticket the copy must not start before (0 = none).  The decode loop uses it to start a
+// prefetch when the group of layers before it starts computing (Section 3.3), not as early as the host happens to run
+// ahead: that keeps a unit on the host for as long as possible and the GPU staging share at a few layers' worth.
+int swap_issue(pie_pool *p, int queue, SwapList &l, int32_t mode, int64_t not_before) {
+    if (l.n_moved == 0) return PIE_OK;
+    cudaStream_t stream = p->stream[queue];
+    PIE_STICKY(reserve_ticket_event(p, queue, l.ticket));
+    l.waits[PIE_Q_COMPUTE] = std::max(l.waits[PIE_Q_COMPUTE], not_before);
+    for (int q = 1; q <= 3; ++q) PIE_STICKY(wait_ticket(p, stream, q, l.waits[q]));
+    LayerEvents *le = timing_slot(p, l.layer);
+    if (le && cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream) != cudaSuccess) le = nullptr;
+    bool used_sm = false;
+    PIE_STICKY(do_copies(p, queue, l.src.data(), l.dst.data(), l.n_moved, l.moved.data(),
+                         p->slot_table_dev + (int64_t)l.layer * p->cfg.n_logical_blocks, mode, stream, l.ticket, l.elide.data(),
+                         queue == PIE_Q_IN ? p->arrive_dev + l.layer : nullptr, &used_sm));
+    if (queue == PIE_Q_IN) {
+        p->layer_in_last[(size_t)l.layer] = l.ticket;
+        if (used_sm) p->layer_in_sm[(size_t)l.layer] = l.ticket;
+    }
+    PIE_STICKY(record_ticket(p, queue, l.ticket));
+    if (le) {
+        (queue == PIE_Q_IN ? le->in1 : le->out1) = p->ticket_ev[queue][l.ticket % EV_RING];
+        (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
+        p->lev_last[p->step % TIMING_RING][queue] = p->ticket_ev[queue][l.ticket % EV_RING];
+    }
+    swap_account(p, queue, l);
+    return PIE_OK;
+}
+
+// The lists of a group of layers, issued together.  Where they can go by copy engine and every list moves one and the
+// same run of block ids, the group costs the copy stream three operations instead of three per layer: the blocks of all
+// lists in as few copies as their slots allow (slots handed out to consecutive requests are consecutive, so usually
+// one), the table entries of all layers in one strided copy, the arrival words in one.  Every list's ticket completes
+// when the group has.  Anything else goes list by list.
+int swap_issue_group(pie_pool *p, int queue, std::vector<SwapList> &lists, int32_t mode, int64_t not_before) {
+    std::vector<SwapList *> live;
+    for (SwapList &l : lists)
+        if (l.n_moved > 0) live.push_back(&l);
+    if (live.empty()) return PIE_OK;
+    const int32_t NB = p->cfg.n_logical_blocks;
+    const int64_t BB = p->block_bytes;
+    bool merge = live.size() > 1 && (mode == PIE_MODE_AUTO || mode == PIE_MODE_COPY_ENGINE);
+    const int64_t n0 = live[0]->n_moved;
+    for (size_t i = 0; merge && i < live.size(); ++i) {
+        const SwapList &l = *live[i];
+        merge = l.n_moved == n0 && l.layer == live[0]->layer + (int32_t)i && l.moved[0] == live[0]->moved[0];
+        for (int64_t j = 1; merge && j < l.n_moved; ++j) merge = l.moved[(size_t)j] == l.moved[(size_t)j - 1] + 1;
+    }
+    // the copies of the whole group, coalesced across the lists
+    struct Run {
+        int64_t src, dst, len;
+    };
+    std::vector<Run> runs;
+    if (merge) {
+        for (SwapList *l : live)
+            for (int64_t j = 0; j < l->n_moved; ++j) {
+                if (l->elide[(size_t)j]) continue;
+                const int64_t sj = l->src[(size_t)j], dj = l->dst[(size_t)j];
+                if (!runs.empty() && runs.back().src + runs.back().len == sj && runs.back().dst + runs.back().len == dj) runs.back().len += 1;
+                else runs.push_back({sj, dj, 1});
+            }
+        int64_t blocks = 0;
+        for (const Run &r : runs) blocks += r.len;
+        if (mode == PIE_MODE_AUTO && !runs.empty() &&
+            !((blocks * BB) / (int64_t)runs.size() >= AUTO_COPY_ENGINE_RUN_BYTES || (int64_t)runs.size() <= AUTO_COPY_ENGINE_MAX_RUNS * (int64_t)live.size()))
+            merge = false;   // scattered: the lists go through the gather/scatter kernel one by one
+    }
+    if (!merge) {
+        for (SwapList *l : live) {
+            int st = swap_issue(p, queue, *l, mode, not_before);
+            if (st != PIE_OK) return st;
+        }
+        return PIE_OK;
+    }
+    cudaStream_t stream = p->stream[queue];
+    int64_t waits[4] = {0, 0, 0, not_before};
+    for (SwapList *l : live) {
+        PIE_STICKY(reserve_ticket_event(p, queue, l->ticket));
+        for (int q = 1; q <= 3; ++q) waits[q] = std::max(waits[q], l->waits[q]);
+    }
+    for (int q = 1; q <= 3; ++q) PIE_STICKY(wait_ticket(p, stream, q, waits[q]));
+    // timing: the group's lists count as one, under its first layer
+    LayerEvents *le = timing_slot(p, live[0]->layer);
+    if (le && cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream) != cudaSuccess) le = nullptr;
+    const uint8_t *src_pool = queue == PIE_Q_IN ? p->host_base : p->gpu_base;
+    uint8_t *dst_pool = queue == PIE_Q_IN ? p->gpu_base : p->host_base;
+    const cudaMemcpyKind kind = queue == PIE_Q_IN ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+    for (const Run &r : runs)
+        if (cudaMemcpyAsync(dst_pool + r.dst * BB, src_pool + r.src * BB, (size_t)(r.len * BB), kind, stream) != cudaSuccess) {
+            p->sticky = PIE_ERR_CUDA;
+            return PIE_ERR_CUDA;
+        }
+    // table entries: one row of n0 entries per layer in the pinned ring, one strided copy into the layers' rows;
+    // arrival words (swap-in): the lists' tickets, one copy into the layers' consecutive words
+    const int64_t k = (int64_t)live.size();
+    const int64_t body = ((k * n0) + 3) & ~int64_t(3);
+    const int64_t words = body + (queue == PIE_Q_IN ? ((2 * k + 3) & ~int64_t(3)) : 0);
+    int64_t off = 0;
+    PIE_STICKY(list_alloc(p, words, &off));
+    int32_t *h = p->list_host + off;
+    for (int64_t i = 0; i < k; ++i)
+        for (int64_t j = 0; j < n0; ++j) h[i * n0 + j] = queue == PIE_Q_IN ? live[(size_t)i]->dst[(size_t)j] : -1;
+    cudaError_t e = cudaMemcpy2DAsync(p->slot_table_dev + (int64_t)live[0]->layer * NB + live[0]->moved[0], (size_t)NB * 4, h, (size_t)n0 * 4,
+                                      (size_t)n0 * 4, (size_t)k, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && queue == PIE_Q_IN) {
+        unsigned long long *t = reinterpret_cast<unsigned long long *>(h + body);
+        for (int64_t i = 0; i < k; ++i) t[i] = (unsigned long long)live[(size_t)i]->ticket;
+        e = cudaMemcpyAsync(p->arrive_dev + live[0]->layer, t, (size_t)k * 8, cudaMemcpyHostToDevice, stream);
+    }
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        p->sticky = PIE_ERR_CUDA;
+        return PIE_ERR_CUDA;
+    }
+    list_commit_ticket(p, off, words, queue, live.back()->ticket);
+    p->stats.calls_copy_engine += (double)k;
+    for (SwapList *l : live) {
+        if (queue == PIE_Q_IN) p->layer_in_last[(size_t)l->layer] = l->ticket;
+        PIE_STICKY(record_ticket(p, queue, l->ticket));
+        swap_account(p, queue, *l);
+    }
+    if (le) {
+        cudaEvent_t last = p->ticket_ev[queue][live.back()->ticket % EV_RING];
+        (queue == PIE_Q_IN ? le->in1 : le->out1) = last;
+        (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
+        p->lev_last[p->step % TIMING_RING][queue] = last;
+    }
+    return PIE_OK;
+}
+
 int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t n, int32_t mode, int64_t not_before = 0) {
     if (!p) return PIE_ERR_INVALID;
     if (p->sticky != PIE_OK) return p->sticky;
@@ -374,55 +665,28 @@ int pool_swap(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int64_t
     if (n < 0 || (n > 0 && !ids)) return PIE_ERR_INVALID;
     int st = poll(p);
     if (st != PIE_OK) return st;
-    if (n == 0) return (layer < 0 || layer >= p->cfg.n_layers) ? PIE_ERR_RANGE : PIE_OK;
-    if ((int64_t)p->v_moved.size() < n) {
-        p->v_moved.resize((size_t)n);
-        p->v_src.resize((size_t)n);
-        p->v_dst.resize((size_t)n);
-        p->v_elide.resize((size_t)n);
-    }
-    p->last_swap_step = p->step;
-    int64_t ticket = 0, n_moved = 0, waits[4];
-    st = p->table->swap(queue, layer, ids, n, &ticket, p->v_moved.data(), p->v_src.data(), p->v_dst.data(), &n_moved, waits,
-                        p->v_elide.data());
-    if (st != PIE_OK || n_moved == 0) return st;
-    int64_t n_elided = 0;
-    for (int64_t i = 0; i < n_moved; ++i) n_elided += p->v_elide[(size_t)i];
-    // a unit that is pushed out belongs to the host-resident set from now on; bringing it in for a layer's
-    // turn does not take it out of the set (only a lower ratio does)
-    if (queue == PIE_Q_OUT)
-        for (int64_t i = 0; i < n_moved; ++i) {
-            pie::Unit &u = p->table->unit(layer, p->v_moved[(size_t)i]);
-            if (!u.home_host) {
-                u.home_host = 1;
-                p->home_count[(size_t)layer] += 1;
-                p->home_dirty[(size_t)layer] = 1;
-            }
-        }
-    // from here on the table has been updated: a failure leaves the pool unusable (sticky) rather than inconsistent
-    cudaStream_t stream = p->stream[queue];
-    st = reserve_ticket_event(p, queue, ticket);
-    if (st != PIE_OK) { p->sticky = st; return st; }
-    waits[PIE_Q_COMPUTE] = std::max(waits[PIE_Q_COMPUTE], not_before);
-    for (int q = 1; q <= 3; ++q) {
-        st = wait_ticket(p, stream, q, waits[q]);
-        if (st != PIE_OK) { p->sticky = st; return st; }
-    }
-    LayerEvents *le = timing_slot(p, layer);
-    if (le && cudaEventRecord(queue == PIE_Q_IN ? le->in0 : le->out0, stream) != cudaSuccess) le = nullptr;
-    st = do_copies(p, queue, p->v_src.data(), p->v_dst.data(), n_moved, p->v_moved.data(),
-                   p->slot_table_dev + (int64_t)layer * p->cfg.n_logical_blocks, mode, stream, ticket, p->v_elide.data());
-    if (st != PIE_OK) { p->sticky = st; return st; }
-    st = record_ticket(p, queue, ticket);
-    if (st != PIE_OK) { p->sticky = st; return st; }
-    if (le) {
-        (queue == PIE_Q_IN ? le->in1 : le->out1) = p->ticket_ev[queue][ticket % EV_RING];
-        (queue == PIE_Q_IN ? le->has_in : le->has_out) = true;
-        p->lev_last[p->step % TIMING_RING][queue] = p->ticket_ev[queue][ticket % EV_RING];
-    }
-    (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)(n_moved - n_elided) * (double)p->block_bytes;
-    p->stats.reserved[2] += (double)n_elided * (double)p->block_bytes;
-    return PIE_OK;
+    SwapList &l = p->one_list;
+    st = swap_prepare(p, queue, layer, ids, n, &l);
+    if (st != PIE_OK) return st;
+    return swap_issue(p, queue, l, mode, not_before);
+}
+
+// does the device take 64-bit stream memory operations (stream waits by value)?
+bool can_wait_by_value(int dev) {
+    void *f_get = nullptr, *f_attr = nullptr;
+    cudaDriverEntryPointQueryResult q1, q2;
+    if (cudaGetDriverEntryPoint("cuDeviceGet", &f_get, cudaEnableDefault, &q1) != cudaSuccess || q1 != cudaDriverEntryPointSuccess || !f_get)
+        return false;
+    if (cudaGetDriverEntryPoint("cuDeviceGetAttribute", &f_attr, cudaEnableDefault, &q2) != cudaSuccess ||
+        q2 != cudaDriverEntryPointSuccess || !f_attr)
+        return false;
+    CUdevice cu_dev;
+    if (reinterpret_cast<CUresult (*)(CUdevice *, int)>(f_get)(&cu_dev, dev) != CUDA_SUCCESS) return false;
+    int can = 0;
+    if (reinterpret_cast<CUresult (*)(int *, CUdevice_attribute, CUdevice)>(f_attr)(&can, CU_DEVICE_ATTRIBUTE_CAN_USE_64_BIT_STREAM_MEM_OPS,
+                                                                                   cu_dev) != CUDA_SUCCESS)
+        return false;
+    return can != 0;
 }
 
 int sync_all(pie_pool *p, int64_t timeout_us) {
@@ -440,6 +704,10 @@ int sync_all(pie_pool *p, int64_t timeout_us) {
             if (timeout_us >= 0 && us > timeout_us) return PIE_ERR_TIMEOUT;
         }
     }
+    // the compute stream is idle: every compute ticket enqueued so far has completed, marked or not
+    p->compute_marks.clear();
+    p->compute_marked = p->recorded[PIE_Q_COMPUTE];
+    if (p->recorded[PIE_Q_COMPUTE] > p->table->done(PIE_Q_COMPUTE)) p->table->confirm(PIE_Q_COMPUTE, p->recorded[PIE_Q_COMPUTE]);
     return poll(p);
 }
 
@@ -465,6 +733,7 @@ int patch_units(pie_pool *p, const std::vector<int32_t> &entries) {
 
 void destroy_pool(pie_pool *p) {
     if (!p) return;
+    if (p->aux_stream) cudaStreamSynchronize(p->aux_stream);   // a stamp copy may still be writing the pinned buffer
     for (int q = 1; q <= 2; ++q)
         for (int i = 0; i < EV_RING; ++i)
             if (p->ticket_ev[q][i]) cudaEventDestroy(p->ticket_ev[q][i]);
@@ -478,8 +747,11 @@ void destroy_pool(pie_pool *p) {
         for (LayerEvents &e : p->lev[k])
             for (cudaEvent_t ev : {e.in0, e.out0})
                 if (ev) cudaEventDestroy(ev);
-    for (int k = 0; k < TIMING_RING; ++k)
+    for (int k = 0; k < TIMING_RING; ++k) {
         if (p->lev_anchor[k]) cudaEventDestroy(p->lev_anchor[k]);
+        if (p->lev_close_ev[k]) cudaEventDestroy(p->lev_close_ev[k]);
+    }
+    if (p->aux_stream) cudaStreamDestroy(p->aux_stream);
     for (cudaEvent_t ev : p->io_up)
         if (ev) cudaEventDestroy(ev);
     for (int i = 0; i < 2; ++i)
@@ -490,10 +762,13 @@ void destroy_pool(pie_pool *p) {
     if (p->own_gpu && p->gpu_base) cudaFree(p->gpu_base);
     if (p->own_host && p->host_base) cudaFreeHost(p->host_base);
     cudaFree(p->slot_table_dev);
+    cudaFree(p->arrive_dev);
+    cudaFree(p->done_dev);
     cudaFree(p->list_dev);
     if (p->list_host) cudaFreeHost(p->list_host);
     if (p->status_host) cudaFreeHost(p->status_host);
     if (p->stamps_host) cudaFreeHost(p->stamps_host);
+    cudaFree(p->stamps_dev);
     if (p->governor) pie_governor_destroy(p->governor);
     cudaFree(p->scratch.chunk_off);
     cudaFree(p->scratch.counters);
@@ -510,9 +785,11 @@ void destroy_pool(pie_pool *p) {
     delete p;
 }
 
+// dependent: the call follows the previous layer's attention call of the same decode step directly, with the same
+// lengths and tables: its kernel may be launched as a programmatic dependent of that call's last kernel.
 int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const int32_t *bt_dev, int32_t max_blocks,
                    const int32_t *ctx_dev, const int32_t *bt_host, const int32_t *ctx_host, int32_t n_seqs, float scale,
-                   const void *k_new, const void *v_new) {
+                   const void *k_new, const void *v_new, bool dependent = false) {
     if (!p) return PIE_ERR_INVALID;
     if (p->sticky != PIE_OK) return p->sticky;
     if (layer < 0 || layer >= p->cfg.n_layers) return PIE_ERR_RANGE;
@@ -562,7 +839,18 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     st = reserve_ticket_event(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) { p->sticky = st; return st; }
     LayerEvents *le = timing_slot(p, layer);
+    // Presence wait (Section 3.2).  Units that a list of this layer is still bringing in: the kernel itself waits for the
+    // layer's arrival word, so the compute stream carries no cross-stream wait (each costs the stream a few
+    // microseconds, layer after layer).  Anything else - a list an SM kernel moves, a slot inherited from a copy of
+    // another layer or direction - is waited for by the stream.
+    unsigned long long arrive_need = 0;
+    if (waits[PIE_Q_IN] > 0 && waits[PIE_Q_IN] <= p->layer_in_last[(size_t)layer] &&
+        p->layer_in_sm[(size_t)layer] <= p->table->done(PIE_Q_IN)) {
+        arrive_need = (unsigned long long)waits[PIE_Q_IN];
+        waits[PIE_Q_IN] = 0;
+    }
     for (int qd = 1; qd <= 2; ++qd) {
+        if (le && waits[qd] > p->table->done(qd)) le->stream_wait = true;
         st = wait_ticket(p, stream, qd, waits[qd]);
         if (st != PIE_OK) { p->sticky = st; return st; }
     }
@@ -587,6 +875,11 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.variant = p->cfg.reserved[0];
     a.status = p->status_dev;
     a.stamps = le ? stamp_dev(p, layer, STAMP_START) : nullptr;
+    a.arrive = p->arrive_dev + layer;
+    a.arrive_need = arrive_need;
+    a.done_word = p->done_dev;
+    a.done_value = (unsigned long long)ticket;
+    a.dependent_launch = dependent;
     if (le && p->cfg.timing >= 2 && !p->lev_anchored[p->step % TIMING_RING]) {
         const int k = (int)(p->step % TIMING_RING);
         if (cudaEventRecord(p->lev_anchor[k], stream) == cudaSuccess) p->lev_anchored[k] = true;
@@ -599,20 +892,53 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     }
     st = record_ticket(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) p->sticky = st;
+    p->last_attn_ticket = ticket;
     if (le && st == PIE_OK) {
         le->has_compute = true;
-        p->lev_last[p->step % TIMING_RING][PIE_Q_COMPUTE] = p->ticket_ev[PIE_Q_COMPUTE][ticket % EV_RING];
+        p->lev_closed[p->step % TIMING_RING] = false;   // the set's newest compute ticket has no mark yet (close_step_set)
     }
     return st;
 }
 
+// The timing set of the step in progress is complete once its newest compute ticket is: give that ticket its mark.
+int close_step_set(pie_pool *p) {
+    if (!p->cfg.timing || p->step <= 0) return PIE_OK;
+    const int k = (int)(p->step % TIMING_RING);
+    if (p->lev_step[k] != p->step || p->lev_closed[k]) return PIE_OK;
+    const size_t set_words = (size_t)p->cfg.n_layers * STAMP_WORDS;
+    if (p->wait_value64 && p->aux_stream && p->recorded[PIE_Q_COMPUTE] == p->last_attn_ticket) {
+        // a side stream waits for the step's last attention kernel by value, copies the stamps and records the event
+        // that closes the set: the compute stream carries nothing between two steps
+        if (p->wait_value64((CUstream)p->aux_stream, (CUdeviceptr)(uintptr_t)p->done_dev, (cuuint64_t)p->last_attn_ticket,
+                            CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS) {
+            g_last_cuda_error = (int)cudaErrorUnknown;
+            return PIE_ERR_CUDA;
+        }
+        PIE_CUDA(cudaMemcpyAsync(p->stamps_host + (size_t)k * set_words, p->stamps_dev + (size_t)k * set_words, set_words * 8,
+                                 cudaMemcpyDeviceToHost, p->aux_stream));
+        PIE_CUDA(cudaEventRecord(p->lev_close_ev[k], p->aux_stream));
+        p->lev_last[k][PIE_Q_COMPUTE] = p->lev_close_ev[k];
+        p->lev_closed[k] = true;
+        return PIE_OK;
+    }
+    PIE_CUDA(cudaMemcpyAsync(p->stamps_host + (size_t)k * set_words, p->stamps_dev + (size_t)k * set_words, set_words * 8,
+                             cudaMemcpyDeviceToHost, p->stream[PIE_Q_COMPUTE]));
+    cudaEvent_t ev = nullptr;
+    int st = push_mark(p, &ev);   // behind the copy
+    if (st != PIE_OK) return st;
+    p->lev_last[k][PIE_Q_COMPUTE] = ev;
+    p->lev_closed[k] = true;
+    return PIE_OK;
+}
+
 // the host-resident set of `layer` follows the ratio: mark / unmark units in id order
 // The GPU pool must hold every layer's resident share plus the host shares in transit (the layer computing and the
-// `lookahead` layers being prefetched): L (n - h) + (1 + lookahead) h <= n_gpu_slots bounds the host-resident count h
-// of a layer from below.
+// layers being prefetched): L (n - h) + transit * h <= n_gpu_slots bounds the host-resident count h of a layer
+// from below.
 int64_t min_home_count(const pie_pool *p) {
     const int64_t n_alloc = p->table->n_allocated(), L = p->cfg.n_layers;
-    const int64_t transit = 1 + std::min<int64_t>(p->lookahead, L - 1);  // this layer's share + the layers being prefetched
+    // the group that computes + the group being prefetched; a group is one layer unless the caller asked for more
+    const int64_t transit = std::min<int64_t>(2 * std::max(1, p->group_setting), L);
     if (L <= transit) return 0;
     const int64_t deficit = L * n_alloc - p->cfg.n_gpu_slots;
     return deficit > 0 ? std::min(n_alloc, (deficit + L - transit - 1) / (L - transit)) : 0;
@@ -706,6 +1032,58 @@ void plan_out(pie_pool *p, int32_t layer, std::vector<int32_t> &out_ids) {
 int plan_layer(pie_pool *p, int32_t layer, std::vector<int32_t> &in_ids, std::vector<int32_t> &out_ids) {
     plan_out(p, layer, out_ids);
     return plan_in(p, (layer + 1) % p->cfg.n_layers, in_ids);
+}
+
+// How many consecutive layers the decode loop treats as one group (their prefetches are issued together when the
+// group before them starts, their write-backs together when they have all computed: one mark on the compute stream
+// per group instead of one per layer).  A group in use, the next one arriving and the previous one leaving occupy GPU
+// slots at the same time, so the size follows what the pool can spare: three groups' host-resident shares.
+int32_t group_layers(pie_pool *p) {
+    const int32_t L = p->cfg.n_layers;
+    if (p->group_setting > 0) return std::max(1, std::min(p->group_setting, L / 2));
+    const int32_t cap = std::max(1, std::min(MAX_GROUP_LAYERS, L / 4));
+    const int64_t n_alloc = p->table->n_allocated();
+    int64_t h = p->ratio_mode != 0 ? std::max((int64_t)std::llround(p->ratio * (double)n_alloc), min_home_count(p)) : 0;
+    int64_t resident = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        h = std::max(h, p->home_count[(size_t)l]);
+        resident += n_alloc - p->home_count[(size_t)l];
+    }
+    if (h <= 0) return cap;
+    const int64_t spare = p->cfg.n_gpu_slots - std::max<int64_t>(resident, (int64_t)L * (n_alloc - h));
+    return (int32_t)std::max<int64_t>(1, std::min<int64_t>(cap, spare / (3 * h)));
+}
+
+// The layers of the group in progress that have computed push their host-resident shares out (Section 3.3: the layer
+// that has just finished is the coldest); the group is closed.
+int finish_group(pie_pool *p) {
+    if (p->group_done.empty()) {
+        p->group_len = 0;
+        return PIE_OK;
+    }
+    if (p->sticky != PIE_OK) return p->sticky;
+    struct PollHold {
+        pie_pool *p;
+        bool was;
+        ~PollHold() { p->poll_hold = was; }
+    } hold{p, p->poll_hold};
+    p->poll_hold = true;
+    std::vector<int32_t> layers;
+    layers.swap(p->group_done);
+    p->group_len = 0;
+    if (p->group_lists.size() < layers.size()) p->group_lists.resize(layers.size());
+    std::vector<SwapList> &lists = p->group_lists;
+    for (SwapList &l : lists) l.n_moved = 0;
+    int st = PIE_OK;
+    size_t n_lists = 0;
+    for (int32_t l : layers) {
+        plan_out(p, l, p->v_plan_out);
+        if (p->cfg.n_layers <= 1 || p->v_plan_out.empty()) continue;
+        st = swap_prepare(p, PIE_Q_OUT, l, p->v_plan_out.data(), (int64_t)p->v_plan_out.size(), &lists[n_lists++]);
+        if (st != PIE_OK) break;   // what was prepared before it still has to be issued
+    }
+    const int st2 = swap_issue_group(p, PIE_Q_OUT, lists, p->group_mode, 0);
+    return st != PIE_OK ? st : st2;
 }
 
 // streams and events of the host-buffer entry point's pipeline (created at its first use)
@@ -875,14 +1253,34 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
         }
         if (cfg->timing >= 2)
             for (int k = 0; k < TIMING_RING; ++k) PIE_TRY(cudaEventCreate(&p->lev_anchor[k]), PIE_ERR_CUDA);
+        PIE_TRY(cudaStreamCreateWithFlags(&p->aux_stream, cudaStreamNonBlocking), PIE_ERR_CUDA);
+        for (int k = 0; k < TIMING_RING; ++k) PIE_TRY(cudaEventCreateWithFlags(&p->lev_close_ev[k], cudaEventDisableTiming), PIE_ERR_CUDA);
+        // The kernels note their stamps in device memory and one copy per step brings a step's set to the host.  (Stamps
+        // in host-visible memory made every kernel end with a store across the host link; while swap lists were being
+        // copied out that store queued behind them, and the next kernel started 30 us late, layer after layer.)
         const size_t stamp_bytes = (size_t)TIMING_RING * (size_t)cfg->n_layers * STAMP_WORDS * 8;
-        PIE_TRY(cudaHostAlloc((void **)&p->stamps_host, stamp_bytes, cudaHostAllocMapped), PIE_ERR_NOMEM);
+        PIE_TRY(cudaHostAlloc((void **)&p->stamps_host, stamp_bytes, cudaHostAllocDefault), PIE_ERR_NOMEM);
         std::memset(p->stamps_host, 0, stamp_bytes);
-        PIE_TRY(cudaHostGetDevicePointer((void **)&p->stamps_dev, p->stamps_host, 0), PIE_ERR_CUDA);
+        PIE_TRY(cudaMalloc((void **)&p->stamps_dev, stamp_bytes), PIE_ERR_NOMEM);
+        PIE_TRY(cudaMemset(p->stamps_dev, 0, stamp_bytes), PIE_ERR_CUDA);
     }
     const size_t table_bytes = (size_t)cfg->n_layers * (size_t)cfg->n_logical_blocks * 4;
     PIE_TRY(cudaMalloc((void **)&p->slot_table_dev, table_bytes), PIE_ERR_NOMEM);
     PIE_TRY(cudaMemset(p->slot_table_dev, 0xff, table_bytes), PIE_ERR_CUDA);
+    PIE_TRY(cudaMalloc((void **)&p->done_dev, 64), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMemset(p->done_dev, 0, 64), PIE_ERR_CUDA);
+    {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuStreamWaitValue64", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess && fn != nullptr) {
+            if (can_wait_by_value(dev)) p->wait_value64 = reinterpret_cast<decltype(p->wait_value64)>(fn);
+        }
+    }
+    PIE_TRY(cudaMalloc((void **)&p->arrive_dev, (size_t)cfg->n_layers * 8), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMemset(p->arrive_dev, 0, (size_t)cfg->n_layers * 8), PIE_ERR_CUDA);
+    p->layer_in_sm.assign((size_t)cfg->n_layers, 0);
+    p->layer_in_last.assign((size_t)cfg->n_layers, 0);
     p->list_words = std::max<int64_t>(1 << 20, (int64_t)cfg->n_logical_blocks * 3 * 8);
     PIE_TRY(cudaHostAlloc((void **)&p->list_host, (size_t)p->list_words * 4, cudaHostAllocDefault), PIE_ERR_NOMEM);
     PIE_TRY(cudaMalloc((void **)&p->list_dev, (size_t)p->list_words * 4), PIE_ERR_NOMEM);
@@ -1089,6 +1487,15 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
 // wait = true blocks until the set's events have completed (used only when the ring is about to wrap).
 static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed) {
     std::vector<LayerEvents> &ev = pool->lev[k];
+    if (!pool->lev_closed[k]) {
+        // the set's newest compute ticket has no mark yet (a caller that went layer by layer and never ticked)
+        if (!wait) return 1;
+        const size_t set_words = (size_t)pool->cfg.n_layers * STAMP_WORDS;
+        PIE_CUDA(cudaMemcpyAsync(pool->stamps_host + (size_t)k * set_words, pool->stamps_dev + (size_t)k * set_words, set_words * 8,
+                                 cudaMemcpyDeviceToHost, pool->stream[PIE_Q_COMPUTE]));
+        PIE_CUDA(cudaStreamSynchronize(pool->stream[PIE_Q_COMPUTE]));
+        pool->lev_closed[k] = true;
+    }
     // every event of the set sits on one of three streams and a stream completes in order: the newest event of
     // each stream tells whether the whole set is complete
     for (int q = 1; q <= 3; ++q) {
@@ -1144,18 +1551,20 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     for (size_t l = 0; l < L; ++l) {
         const uint64_t S = stamps[l * STAMP_WORDS + STAMP_START], E = stamps[l * STAMP_WORDS + STAMP_END];
         if (!ev[l].has_compute || !S || !E || E < S) continue;
-        // units were brought in for this layer: by a list of this step, or - for the first layers - by the previous
-        // step's look-ahead across the token boundary
-        const bool fetched = ev[l].has_in || (chained && l < 8 && ((pool->prev_step_prefetched >> l) & 1u));
-        double layer_stall = 0.0;
-        if (fetched && prev_end && S > prev_end + usual_gap) layer_stall = (double)(S - prev_end - usual_gap) * 1e-6;
+        const bool fetched = ev[l].stream_wait;
+        // the presence wait: what the kernel itself waited for the layer's arrival word, plus - where the stream had to
+        // wait - what the gap before the kernel exceeds the usual gap by
+        const double kernel_wait = (double)stamps[l * STAMP_WORDS + STAMP_WAIT] * 1e-6;
+        double layer_stall = kernel_wait;
+        if (fetched && prev_end && S > prev_end + usual_gap) layer_stall += (double)(S - prev_end - usual_gap) * 1e-6;
         stall += layer_stall;
+
         if (!first) {
             // the step's first layer: its time starts with its own kernel (whatever the caller did between two steps
             // is not the layer's); a wait before it still counts as stall, and as part of the step
             first = S;
-            first_stall = layer_stall;
-            compute += (double)(E - S) * 1e-6;
+            first_stall = layer_stall - kernel_wait;   // the wait inside the kernel is part of E - S already
+            compute += std::max(0.0, (double)(E - S) * 1e-6 - (double)stamps[l * STAMP_WORDS + STAMP_WAIT] * 1e-6);
         } else {
             compute += std::max(0.0, (double)(E - prev_end) * 1e-6 - layer_stall);
         }
@@ -1164,9 +1573,6 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     if (last) {
         pool->prev_step_end = last;
         pool->prev_step_id = pool->lev_step[k];
-        pool->prev_step_prefetched = 0;   // lists this step issued for the first layers: they serve the next step
-        for (size_t l = 0; l < std::min<size_t>(8, L); ++l)
-            if (L > 1 && ev[l].has_in) pool->prev_step_prefetched |= 1u << l;
     }
     pool->lev_done[k] = true;
     if (first && pool->cfg.timing >= 2) {
@@ -1180,7 +1586,7 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
             float *row = pool->timeline.data() + l * 7;
             if (ev[l].has_compute && S && E) {
                 row[0] = rel(before);
-                row[1] = rel(S);
+                row[1] = rel(S + stamps[l * STAMP_WORDS + STAMP_WAIT]);   // past the presence wait inside the kernel
                 row[2] = rel(E);
                 before = E;
             }
@@ -1205,7 +1611,9 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     // Performance record (Section 3.4.2): attention time per context token on steps without swap traffic.  Copies
     // that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
     // wait, so the controller holds the ratio where wait + slow-down stays within its tolerance.
-    const double tokens = (double)((volatile int32_t *)pool->status_host)[3];
+    double tokens = 0.0;   // the step's own count (each kernel notes its batch's tokens beside its time stamps)
+    for (size_t l = 0; l < L && tokens == 0.0; ++l)
+        if (ev[l].has_compute) tokens = (double)stamps[l * STAMP_WORDS + STAMP_TOKENS];
     double slow = 0.0;
     if (tokens > 0 && compute > 0) {
         const double per_token = compute / tokens;
@@ -1231,7 +1639,8 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
 
 // evaluate, in step order, every completed set that has not been evaluated yet
 static int evaluate_completed(pie_pool *pool, int32_t *changed) {
-    for (int64_t st = std::max<int64_t>(1, pool->step - TIMING_RING + 1); st < pool->step; ++st) {
+    // (the step in progress counts once its set has been closed: pie_controller_tick after the last layer)
+    for (int64_t st = std::max<int64_t>(1, pool->step - TIMING_RING + 1); st <= pool->step; ++st) {
         const int k = (int)(st % TIMING_RING);
         if (pool->lev_step[k] != st || pool->lev_done[k]) continue;
         const int rc = evaluate_step_set(pool, k, false, changed);
@@ -1243,6 +1652,11 @@ static int evaluate_completed(pie_pool *pool, int32_t *changed) {
 
 int pie_step_begin(pie_pool *pool) {
     if (!pool) return PIE_ERR_INVALID;
+    {
+        int st = finish_group(pool);       // a caller that went layer by layer may have left a group open
+        if (st == PIE_OK) st = close_step_set(pool);
+        if (st != PIE_OK) return st;
+    }
     ++pool->step;
     if (pool->cfg.timing) {
         int st = evaluate_completed(pool, nullptr);
@@ -1255,7 +1669,8 @@ int pie_step_begin(pie_pool *pool) {
         }
         pool->lev_step[k] = pool->step;
         pool->lev_done[k] = false;
-        for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = false;
+        pool->lev_closed[k] = true;    // no compute ticket in the set yet
+        for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = e.stream_wait = false;
         for (int q = 0; q < 4; ++q) pool->lev_last[k][q] = nullptr;
         pool->lev_anchored[k] = false;
         // the set's kernels are launched after this point, and the previous user of the set has completed
@@ -1371,8 +1786,11 @@ int pie_set_kv_scales(pie_pool *pool, float k_scale, float v_scale) {
 }
 
 int pie_set_lookahead(pie_pool *pool, int32_t layers) {
-    if (!pool || layers < 1 || layers > 8) return PIE_ERR_INVALID;
-    pool->lookahead = layers;
+    if (!pool || layers < 0 || layers > MAX_GROUP_LAYERS) return PIE_ERR_INVALID;
+    int st = finish_group(pool);
+    if (st != PIE_OK) return st;
+    pool->group_setting = layers;
+    pool->lookahead = std::max(1, layers);
     return PIE_OK;
 }
 
@@ -1427,7 +1845,11 @@ int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in
 int pie_controller_tick(pie_pool *pool, int32_t *changed) {
     if (!pool) return PIE_ERR_INVALID;
     if (changed) *changed = 0;
+    int st = finish_group(pool);
+    if (st != PIE_OK) return st;
     if (!pool->cfg.timing) return PIE_OK;
+    st = close_step_set(pool);
+    if (st != PIE_OK) return st;
     return evaluate_completed(pool, changed);
 }
 
@@ -1463,7 +1885,9 @@ int pie_get_stats(pie_pool *pool, pie_stats *out) {
 int pie_sync(pie_pool *pool, int64_t timeout_us) {
     if (!pool) return PIE_ERR_INVALID;
     if (pool->sticky != PIE_OK) return pool->sticky;
-    int st = sync_all(pool, timeout_us);
+    int st = finish_group(pool);
+    if (st != PIE_OK) return st;
+    st = sync_all(pool, timeout_us);
     if (st != PIE_OK) return st;
     return check_status_word(pool);
 }
@@ -1484,7 +1908,9 @@ int pie_set_layer_policy(pie_pool *pool, int32_t gpu_regions, int32_t cpu_region
     }
     const int32_t L = pool->cfg.n_layers;
     if (gpu_regions <= 0 || cpu_regions < 0 || gpu_regions + cpu_regions < L) return PIE_ERR_INVALID;
-    int st = sync_all(pool, 30 * 1000 * 1000);  // layers must be settled, each wholly on one side
+    int st = finish_group(pool);
+    if (st != PIE_OK) return st;
+    st = sync_all(pool, 30 * 1000 * 1000);  // layers must be settled, each wholly on one side
     if (st != PIE_OK) return st;
     std::vector<uint8_t> on_cpu((size_t)L, 0);
     int32_t n_gpu = 0, n_cpu = 0;
@@ -1563,8 +1989,12 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
     for (int32_t k = 0; k < L; ++k) {
         // the control logic runs when layer k starts, i.e. when layer k-1 has finished: the host keeps step with
         // the device here (as the paper's per-layer control loop does), so completions are what they really are
-        const int64_t prev = pool->table->issued(PIE_Q_COMPUTE);
-        if (prev > pool->table->done(PIE_Q_COMPUTE)) PIE_CUDA(cudaEventSynchronize(pool->ticket_ev[PIE_Q_COMPUTE][prev % EV_RING]));
+        {
+            cudaEvent_t prev_ev = nullptr;
+            st = compute_mark(pool, pool->recorded[PIE_Q_COMPUTE], &prev_ev);
+            if (st != PIE_OK) return st;
+            if (prev_ev) PIE_CUDA(cudaEventSynchronize(prev_ev));
+        }
         st = fifo_apply_completions(pool);
         if (st != PIE_OK) return st;
         st = fifo_start_swaps(pool, k, mode, ids);
@@ -1595,10 +2025,11 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
 }
 
 // One layer of the control loop (Section 3.2; Section 4.2: what a model's forward pass calls per layer): fetch what the
-// layer still lacks, start the prefetch of the next layer, attend (and append), push this layer's host-resident share out.
+// layer still lacks, attend (and append); at the start of a group of layers start the prefetch of the next group, at
+// its end push the group's host-resident shares out.
 static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, const int32_t *block_table_dev,
                         int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new,
-                        const void *v_new, int32_t mode) {
+                        const void *v_new, int32_t mode, bool dependent = false) {
     const int32_t L = pool->cfg.n_layers;
     struct PollHold {
         pie_pool *p;
@@ -1612,40 +2043,57 @@ static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, con
         if (st != PIE_OK) return st;
     }
     pool->poll_hold = true;
-    // units of this layer that nobody prefetched (the very first layer of a run, a caller that skipped a layer):
-    // fetch them now; the attention call waits for the copy
+    int st = PIE_OK;
+    const bool continues = pool->group_len > 0 && l == pool->group_first + (int32_t)pool->group_done.size() &&
+                           l < pool->group_first + pool->group_len;
+    if (!continues) {
+        // a new group starts with this layer (Section 3.3: the swaps are decided when a layer starts computing)
+        st = finish_group(pool);
+        if (st != PIE_OK) return st;
+        const int32_t k = group_layers(pool);
+        pool->group_first = l;
+        pool->group_len = std::min(k, L - l);
+        pool->group_mode = mode;
+        // prefetch: the next group's layers (wrapping into the next token: the look-ahead of Section 3.4.2) that still
+        // have units on the host.  The copies start when this group starts, i.e. once the previous attention call has
+        // finished, and run back to back on the copy-in stream.  What the GPU pool cannot take now is fetched at
+        // that layer's turn.
+        const int32_t next_first = (l + pool->group_len) % L;
+        const int32_t next_len = std::min(k, L - next_first);
+        const int64_t start_with = pool->recorded[PIE_Q_COMPUTE];
+        std::vector<int32_t> &in_ids = pool->v_plan_in;
+        if (pool->group_lists.size() < (size_t)MAX_GROUP_LAYERS) pool->group_lists.resize(MAX_GROUP_LAYERS);
+        std::vector<SwapList> &lists = pool->group_lists;
+        for (SwapList &sl : lists) sl.n_moved = 0;
+        size_t n_lists = 0;
+        for (int32_t d = 0; d < next_len && L > 1 && st == PIE_OK; ++d) {
+            const int32_t target = next_first + d;
+            if (target >= l && target < l + pool->group_len) continue;   // fewer layers than two groups
+            plan_in(pool, target, in_ids);
+            if (in_ids.empty()) continue;
+            st = swap_prepare(pool, PIE_Q_IN, target, in_ids.data(), (int64_t)in_ids.size(), &lists[n_lists++]);
+        }
+        const int st2 = swap_issue_group(pool, PIE_Q_IN, lists, mode, start_with);   // what was prepared must be issued
+        if (st != PIE_OK) return st;
+        if (st2 != PIE_OK) return st2;
+    }
+    // units of this layer that nobody prefetched (the very first layers of a run, a caller that skipped a layer, a
+    // share the pool had no room for): fetch them now; the attention call waits for the copy
     {
         pool->v_in.clear();
         for (int32_t b : candidate_ids(pool, l))
             if (pool->table->unit(l, b).side == PIE_HOST) pool->v_in.push_back(b);
         if (!pool->v_in.empty()) {
             std::vector<int32_t> ids(pool->v_in);
-            int st = pool_swap(pool, PIE_Q_IN, l, ids.data(), (int64_t)ids.size(), mode);
-            if (st != PIE_OK) return st;
+            st = pool_swap(pool, PIE_Q_IN, l, ids.data(), (int64_t)ids.size(), mode);
+            if (st != PIE_OK) return st;   // nothing of this layer has been enqueued
         }
     }
-    std::vector<int32_t> &in_ids = pool->v_plan_in, &out_ids = pool->v_plan_out;
-    plan_out(pool, l, out_ids);
-    // prefetch: the layers up to `lookahead` ahead (wrapping into the next token) that still have units on the host;
-    // in a steady loop only the farthest one does.  The copies start when layer l starts, i.e. once the previous
-    // attention call has finished, and run back to back on the copy-in stream.
-    int st = PIE_OK;
-    const int64_t start_with = pool->table->issued(PIE_Q_COMPUTE);
-    for (int32_t d = 1; d <= std::min(pool->lookahead, L - 1); ++d) {
-        const int32_t target = (l + d) % L;
-        st = plan_in(pool, target, in_ids);
-        if (st != PIE_OK) return st;  // the GPU pool cannot take that layer's share: nothing was enqueued for it
-        if (in_ids.empty()) continue;
-        st = pool_swap(pool, PIE_Q_IN, target, in_ids.data(), (int64_t)in_ids.size(), mode, start_with);
-        if (st != PIE_OK) return st;
-    }
     st = attention_call(pool, l, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
-                        k_new, v_new);
+                        k_new, v_new, dependent);
     if (st != PIE_OK) return st;
-    if (L > 1 && !out_ids.empty()) {
-        st = pool_swap(pool, PIE_Q_OUT, l, out_ids.data(), (int64_t)out_ids.size(), mode);
-        if (st != PIE_OK) return st;
-    }
+    pool->group_done.push_back(l);
+    if ((int32_t)pool->group_done.size() >= pool->group_len) return finish_group(pool);
     return PIE_OK;
 }
 
@@ -1666,7 +2114,7 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
         st = decode_layer(pool, l, (const uint8_t *)q_all + l * q_stride, (uint8_t *)out_all + l * q_stride, block_table_dev,
                           max_blocks_per_seq, ctx_lens_dev, n_seqs, scale,
                           k_new_all ? (const uint8_t *)k_new_all + l * kv_stride : nullptr,
-                          v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr, mode);
+                          v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr, mode, l > 0);
         if (st != PIE_OK) return st;
     }
     return pie_controller_tick(pool, nullptr);
@@ -1756,13 +2204,13 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
         st = decode_layer(pool, l, (const uint8_t *)pool->stage_q + l * q_layer, (uint8_t *)pool->stage_out + l * q_layer,
                           pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
                           k_new_all_host ? (const uint8_t *)pool->stage_k + l * kv_layer : nullptr,
-                          k_new_all_host ? (const uint8_t *)pool->stage_v + l * kv_layer : nullptr, mode);
+                          k_new_all_host ? (const uint8_t *)pool->stage_v + l * kv_layer : nullptr, mode, l > 0);
         if (st != PIE_OK) break;
         if ((l + 1) % G == 0 || l + 1 == L) {
             // the group's results: behind the compute ticket of its last layer
             const int32_t l0 = (l / G) * G, nl = l + 1 - l0;
-            const int64_t t = pool->table->issued(PIE_Q_COMPUTE);
-            PIE_CUDA(cudaStreamWaitEvent(pool->io_stream[1], pool->ticket_ev[PIE_Q_COMPUTE][t % EV_RING], 0));
+            st = wait_ticket(pool, pool->io_stream[1], PIE_Q_COMPUTE, pool->recorded[PIE_Q_COMPUTE]);
+            if (st != PIE_OK) break;
             PIE_CUDA(cudaMemcpyAsync((uint8_t *)out_all_host + l0 * q_layer, (const uint8_t *)pool->stage_out + l0 * q_layer,
                                      (size_t)(nl * q_layer), cudaMemcpyDeviceToHost, pool->io_stream[1]));
         }
