@@ -654,9 +654,6 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     volatile int32_t *q_item = misc + 4;      // [4 .. 4 + QD)
     int32_t *co_smem = reinterpret_cast<int32_t *>(smem + SM::OFF_CO);
 
-    // The combine kernel that follows may become resident at once (its CTAs wait for this grid to complete before they
-    // read anything): its launch then costs nothing at the end of this kernel.
-    grid_launch_dependents();
     // Everything up to the dependency wait below touches only shared memory and the call's own inputs (lengths and
     // tables, which no kernel of the path writes): under a programmatic dependent launch it overlaps the tail of the
     // kernel before it in the stream.
@@ -786,7 +783,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             }
             item = __shfl_sync(0xffffffffu, item, 0);
             ++qn;
-            if (item < 0) break;
+            if (item < 0) {
+                // No work is left for this CTA.  Once every CTA has got here the combine kernel that follows may become
+                // resident (its CTAs wait for this grid to complete before they read anything): its launch then costs
+                // nothing at the end of this kernel.  (Signalled at the kernel's start, the waiting CTAs sat beside
+                // the attention warps for its whole duration and cost 8-head groups 9 %.)
+                grid_launch_dependents();
+                break;
+            }
             const ItemInfo it = decode_item(p, co, item);
             const int32_t *bt = p.block_table + (int64_t)it.s * p.max_blocks + (it.t0 >> 4);
             for (int32_t base = 0; base < it.ntiles; base += 32) {
@@ -1220,10 +1224,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 // =====================================================================================================
 // Combine: one CTA per (sequence, KV head, slice of head_dim) merges the sequence's chunk partials in chunk order with
 // the log-sum-exp rule, normalises and rounds to the 16-bit output type (nearest even).  Sequences with fewer than two
-// chunks were finished by the attention kernel.  The per-(head, chunk) weights are computed once in shared memory (sized
-// by the launch for the longest sequence the table allows, so that the whole grid is resident at once: the kernel sits
-// between two layers' attention kernels and every wave of it is dead time); the accumulation keeps eight 16-byte loads
-// in flight per thread.  The slice is the whole head_dim for batches of many (sequence, head) pairs and 32 for few.
+// chunks were finished by the attention kernel.  The chunks' (m, l) pairs go through shared memory (sized by the launch
+// for the longest sequence the table allows, so that the whole grid is resident at once: the kernel sits between two
+// layers' attention kernels and every wave of it is dead time); the accumulation keeps eight 16-byte loads in flight
+// per thread.
 // =====================================================================================================
 constexpr int COMB_THREADS = 64;
 constexpr int COMB_CAP = 256;  // chunks per sequence handled through shared memory; beyond that, plain loops
@@ -1255,22 +1259,15 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
             lbuf[g * cap + c] = part_ml[id * 2 + 1];
         }
         __syncthreads();
-        if (tid < group) {
-            float *w = wbuf + tid * cap, *l = lbuf + tid * cap;
-            float mm = -INFINITY;
-            for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, w[c]);
-            float ll = 0.f;
-            for (int32_t c = 0; c < nchunks; ++c) {
-                const float wt = w[c] == -INFINITY ? 0.f : fast_exp2(w[c] - mm);
-                ll += l[c] * wt;
-                w[c] = wt;
-            }
-            l[0] = ll > 0.f ? 1.f / ll : 0.f;
-        }
-        __syncthreads();
+        // every thread works the weights of its head out for itself (a few exponentials, in chunk order: the same
+        // sums whichever thread forms them), so there is no serial pass over the chunks between two barriers
         const int per_head = width / 4;   // float4 pieces per head in the slice
         for (int e4 = tid; e4 < group * per_head; e4 += COMB_THREADS) {
             const int g = e4 / per_head, d = d_lo + (e4 - g * per_head) * 4;
+            const float *w = wbuf + g * cap, *l = lbuf + g * cap;
+            float mm = -INFINITY;
+            for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, w[c]);
+            float ll = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int32_t c0 = 0; c0 < nchunks; c0 += 8) {
                 float4 v[8];
@@ -1283,14 +1280,15 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (c0 + j < nchunks) {
-                        const float wt = wbuf[g * cap + c0 + j];
+                        const float wt = w[c0 + j] == -INFINITY ? 0.f : fast_exp2(w[c0 + j] - mm);
+                        ll += l[c0 + j] * wt;
                         acc.x += v[j].x * wt;
                         acc.y += v[j].y * wt;
                         acc.z += v[j].z * wt;
                         acc.w += v[j].w * wt;
                     }
             }
-            const float inv = lbuf[g * cap];
+            const float inv = ll > 0.f ? 1.f / ll : 0.f;
             uint2 r;
             r.x = pack2<BF16>(acc.x * inv, acc.y * inv);
             r.y = pack2<BF16>(acc.z * inv, acc.w * inv);
@@ -1521,9 +1519,12 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     // chunks of the longest sequence the table allows (rounded up to a multiple of 8: the loads go in eights)
     const int64_t longest = ((int64_t)a.max_blocks * 16 + a.split_tokens - 1) / a.split_tokens;
     const int32_t cap = (int32_t)std::min<int64_t>(COMB_CAP, (longest + 7) / 8 * 8);
-    // whole head_dim per CTA where there are enough (sequence, head) pairs to fill the GPU; 32-wide slices otherwise
+    // slices of head_dim such that a thread merges one 16-byte piece of one head (the merge is a chain of dependent
+    // loads: what counts is how many rounds of them a thread makes), whole head_dim per CTA at most
     const int64_t pairs = (int64_t)a.n_seqs * sh.n_kv_heads;
-    cfg.gridDim = dim3((unsigned)pairs, (unsigned)(pairs >= 1024 ? 1 : sh.head_dim / 32));
+    int slices = 1;
+    while (slices < sh.head_dim / 32 && p.group * (sh.head_dim / 4) / slices > COMB_THREADS) slices *= 2;
+    cfg.gridDim = dim3((unsigned)pairs, (unsigned)slices);
     cfg.blockDim = dim3(COMB_THREADS);
     cfg.dynamicSmemBytes = (size_t)(2 * p.group * cap) * sizeof(float);
     cfg.stream = stream;
