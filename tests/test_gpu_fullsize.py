@@ -368,7 +368,7 @@ def test_bench_runs_at_reduced_scale_and_prints_the_contract_line():
     import sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--scale", "0.25", "--steps", "4", "--warmup", "3", "--ramp", "8",
-                        "--no-cpu-baseline"], capture_output=True, text=True, cwd=root, timeout=900)
+                        "--sweep-steps", "8", "--sweep-reps", "2", "--no-cpu-baseline"], capture_output=True, text=True, cwd=root, timeout=900)
     assert r.returncode == 0, r.stderr[-2000:]
     line = json.loads(r.stdout.strip().splitlines()[-1])
     for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline",
@@ -378,3 +378,12 @@ def test_bench_runs_at_reduced_scale_and_prints_the_contract_line():
     assert set(line["roofline"]) >= {"bound", "achieved", "peak", "unit", "frac", "traffic"} and 0.3 < line["roofline"]["frac"] < 1.2
     assert set(line["e2e"]) >= {"value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step"} and line["e2e"]["h2d_bytes_per_step"] > 0
     assert line["kv_fp8"]["resident"]["attn_gbs"] > 500
+    # the line says what it measured: the warm-up asked for, the ratio the timed region ran at, what it hid, and a roofline
+    # fraction that follows from the line's own bytes and time
+    assert line["warmup"] == 3 and line["steps"] == 4
+    assert line["config"]["extension_ratio"] == line["hidden_swap"]["ratio"] > 0 and line["hidden_swap_gbs"] > 0
+    rf = line["roofline"]
+    assert abs(rf["alg_bytes_per_launch"] / (rf["ms_per_launch"] * 1e-3) / 1e9 / rf["peak"] - rf["frac"]) < 1e-9
+    assert abs(line["value"] * line["ms_per_step"] * 1e-3 * 1e9 / (line["config"]["n_layers"] * 1) - rf["alg_bytes_per_launch"]) < 1e-3 * rf["alg_bytes_per_launch"]
+    for e in line["hidden_swap"]["fixed_ratio_sweep"]:
+        assert e["slowdown_min"] <= e["slowdown_mean"] <= e["slowdown_max"] and e["runs"] == 2
