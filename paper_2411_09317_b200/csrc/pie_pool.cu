@@ -165,6 +165,7 @@ struct pie_pool {
     cudaEvent_t lev_close_ev[TIMING_RING] = {}; // recorded there behind the copy
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
+    double free_contrast = -1.0;     // on swap-free steps: what the layers' times add up to above the fastest quarter's mean, / compute
     std::vector<float> timeline;     // last evaluated step: [L][7] ms from the step's first event (-1 = not recorded)
     pie_stats stats{};
     // scratch vectors
@@ -1534,6 +1535,7 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     uint64_t prev_end = chained ? pool->prev_step_end : 0, first = 0, last = 0;
     uint64_t usual_gap = 20000;
     double first_stall = 0.0;
+    std::vector<double> spans;   // per layer but the step's first: end of the previous layer's kernel to the end of its own, less the wait
     {
         uint64_t pe = 0, step_min = ~uint64_t(0);
         for (size_t l = 0; l < L; ++l) {
@@ -1566,7 +1568,9 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
             first_stall = layer_stall - kernel_wait;   // the wait inside the kernel is part of E - S already
             compute += std::max(0.0, (double)(E - S) * 1e-6 - (double)stamps[l * STAMP_WORDS + STAMP_WAIT] * 1e-6);
         } else {
-            compute += std::max(0.0, (double)(E - prev_end) * 1e-6 - layer_stall);
+            const double span = std::max(0.0, (double)(E - prev_end) * 1e-6 - layer_stall);
+            compute += span;
+            spans.push_back(span);
         }
         prev_end = last = E;
     }
@@ -1608,14 +1612,30 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     pool->stats.last_step_swap_out_ms = t_out;
     if (first && last) pool->stats.last_step_ms = (double)(last - first) * 1e-6 + first_stall;
     pool->stats.steps_measured += 1;
-    // Performance record (Section 3.4.2): attention time per context token on steps without swap traffic.  Copies
-    // that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
-    // wait, so the controller holds the ratio where wait + slow-down stays within its tolerance.
+    // Copies that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
+    // wait, so the controller holds the ratio where wait + slow-down stays within its tolerance.  Every layer of a step
+    // attends the same batch at the same lengths, and the swap lists of a group of layers are in flight during the first
+    // part of the group only: the step's undisturbed layers are its own yardstick.  The slow-down is what the layers'
+    // times add up to above the mean of the step's fastest quarter, less what that sum comes to on steps without swap
+    // traffic (a record, Section 3.4.2).  Nothing is compared across steps, so clocks drifting under the power cap and
+    // contexts growing do not look like a slow-down.  (Steps of fewer than nine layers fall back to a record of the
+    // time per context token taken on swap-free steps.)
     double tokens = 0.0;   // the step's own count (each kernel notes its batch's tokens beside its time stamps)
     for (size_t l = 0; l < L && tokens == 0.0; ++l)
         if (ev[l].has_compute) tokens = (double)stamps[l * STAMP_WORDS + STAMP_TOKENS];
     double slow = 0.0;
-    if (tokens > 0 && compute > 0) {
+    if (spans.size() >= 8 && compute > 0) {
+        std::vector<double> sorted(spans);
+        std::sort(sorted.begin(), sorted.end());
+        const size_t quarter = std::max<size_t>(2, sorted.size() / 4);
+        double ref = 0.0;
+        for (size_t i = 0; i < quarter; ++i) ref += sorted[i];
+        ref /= (double)quarter;
+        double above = 0.0;
+        for (double sp : spans) above += std::max(0.0, sp - ref);
+        if (!any_swap) pool->free_contrast = pool->free_contrast >= 0 ? 0.75 * pool->free_contrast + 0.25 * above / compute : above / compute;
+        else slow = std::max(0.0, above - std::max(0.0, pool->free_contrast) * compute);
+    } else if (tokens > 0 && compute > 0) {
         const double per_token = compute / tokens;
         if (!any_swap) pool->base_ms_per_token = pool->base_ms_per_token > 0 ? 0.75 * pool->base_ms_per_token + 0.25 * per_token : per_token;
         else if (pool->base_ms_per_token > 0) slow = std::max(0.0, compute - pool->base_ms_per_token * tokens);
