@@ -266,11 +266,11 @@ class Runner:
         return {"ms": ms, "ms_per_step": ms / n, "per_step": per_step, "after": after, "before": before,
                 "swap_in_gbs": (after["bytes_in"] - before["bytes_in"]) / sec / 1e9,
                 "swap_out_gbs": (after["bytes_out"] - before["bytes_out"]) / sec / 1e9,
-                "elided_gbs": (after["reserved"][2] - before["reserved"][2]) / sec / 1e9,
+                "elided_gbs": (after["bytes_out_elided"] - before["bytes_out_elided"]) / sec / 1e9,
                 "wait_share": after["last_step_stall_ms"] / max(after["last_step_ms"], 1e-9),
                 "kernel_ms_per_layer": float(np.mean([c["last_step_compute_ms"] for c in comp if c["steps_measured"] > 0] or [np.nan])) / dw.wl.n_layers,
                 "launches": 2 * dw.wl.n_layers * n + int(after["calls_kernel"] - before["calls_kernel"]) +
-                            int(after["reserved"][3] - before["reserved"][3])}
+                            int(after["patch_kernel_launches"] - before["patch_kernel_launches"])}
 
 
 def sweep(rn, pie, ratios, n, reps, warm, link_gbs):

@@ -53,7 +53,15 @@ typedef struct pie_table pie_table;
 typedef struct pie_fifo pie_fifo;
 typedef struct pie_governor pie_governor;
 
+/* 8-bit blocks: see pie_set_kv_scales */
+enum { PIE_KV_16BIT = 0, PIE_KV_E4M3 = 1 };
+
+/* Both structs start with their own size as the caller compiled it: the library reads (pie_pool_config) or writes
+ * (pie_stats) that many bytes at most, so a caller built against an older header keeps working when fields are added at
+ * the end; fields the caller's struct does not have read as 0.  A size smaller than the first release's struct is
+ * PIE_ERR_INVALID. */
 typedef struct pie_pool_config {
+    uint32_t struct_size;      /* sizeof(pie_pool_config) */
     int32_t n_layers;
     int32_t n_q_heads;
     int32_t n_kv_heads;        /* divides n_q_heads; n_q_heads / n_kv_heads <= 8 */
@@ -62,6 +70,7 @@ typedef struct pie_pool_config {
     int32_t dtype;             /* PIE_F16 or PIE_BF16 */
     int32_t n_logical_blocks;  /* logical block ids 0 .. n-1, shared by all layers */
     int32_t max_seqs;          /* largest batch pie_decode_attention will see (scratch sizing) */
+    int32_t own_streams;       /* 1: the library creates three non-blocking streams */
     int64_t n_gpu_slots;
     int64_t n_host_slots;
     void *gpu_base;            /* device memory of n_gpu_slots * block_bytes, 128-byte aligned, or NULL:
@@ -71,41 +80,51 @@ typedef struct pie_pool_config {
     void *compute_stream;      /* cudaStream_t values; used only when own_streams == 0 */
     void *copy_in_stream;
     void *copy_out_stream;
-    int32_t own_streams;       /* 1: the library creates three non-blocking streams */
     int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = default (512; 1024 where the pool is laid
                                 * out for long sequences: n_logical_blocks * 16 / max_seqs >= 6144) */
     int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
     int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
     int32_t timing;            /* 1: per-layer timing for pie_controller_tick / pie_get_stats (the attention kernel notes
-                                *    the GPU's timer in host-visible memory; timing events only on the copy streams);
+                                *    the GPU's timer in device memory, one copy per step brings the notes to the host;
+                                *    timing events only on the copy streams);
                                 * 2: also keep the per-layer timeline for pie_get_step_timeline */
-    int32_t reserved[7];       /* [0]: attention kernel variant for tuning (0 = default);
-                                * [1]: per-layer size visible to allocation at creation, in blocks (0 = n_logical_blocks;
-                                *      see pie_resize_begin);
-                                * [2]: 1 = the blocks hold K and V as FP8 E4M3 bytes (see pie_set_kv_scales): head_dim 128
-                                *      and variants 0 - 2 only (PIE_ERR_UNSUPPORTED otherwise), block_bytes halves; rest 0 */
+    int32_t attn_variant;      /* attention kernel variant, for tuning (0 = default) */
+    int32_t visible_blocks;    /* per-layer size visible to allocation at creation, in blocks (0 = n_logical_blocks;
+                                * see pie_resize_begin) */
+    int32_t kv_format;         /* PIE_KV_16BIT, or PIE_KV_E4M3: the blocks hold K and V as FP8 E4M3 bytes (see
+                                * pie_set_kv_scales): head_dim 128 and variants 0 - 2 only (PIE_ERR_UNSUPPORTED
+                                * otherwise), block_bytes halves */
+    int32_t reserved[5];       /* 0 */
 } pie_pool_config;
 
 typedef struct pie_stats {
+    uint32_t struct_size;                  /* sizeof(pie_stats): set it before pie_get_stats */
+    uint32_t governor_state;               /* the throughput governor's state (pie_governor_state numbering) */
     double bytes_in, bytes_out;            /* swapped so far, per direction */
     double calls_kernel, calls_copy_engine;
     double last_step_compute_ms;           /* sum over layers: end of the previous layer's attention kernel to the end
                                             * of this one's (append, combine and launch gap included), minus the stall */
-    double last_step_stall_ms;             /* sum over layers that had units brought in: what the gap before the layer's
-                                            * attention kernel exceeds the step's usual gap by (the presence wait) */
-    double last_step_swap_in_ms, last_step_swap_out_ms;
+    double last_step_stall_ms;             /* sum over layers: what the layer's attention kernel (or, for lists an SM
+                                            * kernel moved, the stream before it) waited for arriving units: the
+                                            * presence wait */
+    double last_step_swap_in_ms, last_step_swap_out_ms;   /* the copy streams' busy time: lists of a group count once */
     double last_step_ms;                   /* first layer's start to last layer's end */
     double ratio;                          /* current extension ratio */
     int64_t n_units_gpu, n_units_host, n_units_in_flight;
     int64_t steps_measured;
-    double reserved[8];                    /* [0]: last step's attention slow-down vs the no-swap record, ms;
-                                            * [2]: bytes of swap-out traffic elided so far (pie_set_retention);
-                                            * [3]: table-patch kernels launched after copy-engine lists (lists of few
-                                            *      id runs patch the table by copy and launch none);
-                                            * [1]: the smallest extension ratio the GPU pool's size allows with the
-                                            *      blocks allocated now (the controller never goes below it);
-                                            * [4]: the throughput governor's cap on the ratio (1 = none; 0 before the
-                                            *      first pie_report_throughput), [5]: its state */
+    double last_step_slowdown_ms;          /* what the step's layers took above its undisturbed ones (hidden copies share
+                                            * HBM with the attention kernel); the controller counts it as waiting */
+    double ratio_floor;                    /* the smallest extension ratio the GPU pool's size allows with the blocks
+                                            * allocated now (the controller never goes below it) */
+    double bytes_out_elided;               /* swap-out traffic elided so far (pie_set_retention) */
+    double patch_kernel_launches;          /* table-patch kernels launched after copy-engine lists (lists of few id runs
+                                            * patch the table by copy and launch none) */
+    double governor_cap;                   /* the governor's cap on the ratio (1 = none; 0 before the first
+                                            * pie_report_throughput) */
+    int64_t prefetch_lists;                /* swap-in lists the decode loop has started so far, and how many of them were for */
+    int64_t prefetch_violations;           /* layers of the NEXT token (Section 3.4.2's allowed rule violation) */
+    double last_step_violation_ratio;      /* the two, over the last evaluated step */
+    double reserved[4];                    /* 0 */
 } pie_stats;
 
 /* ---- pool (Section 3.1: the physical pools; Section 3.2: the mapping table) --------------------- */
@@ -218,6 +237,15 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
  * Every layer must be wholly on one side (PIE_ERR_INVALID otherwise); gpu_regions + cpu_regions >= n_layers;
  * the pools must hold that many layers' units.  gpu_regions <= 0 and cpu_regions <= 0: back to the block plan. */
 int pie_set_layer_policy(pie_pool *pool, int32_t gpu_regions, int32_t cpu_regions);
+/* Adaptive expansion in whole layers (Section 3.4.2 as the paper states it): with the whole-layer protocol set AND the
+ * ratio handed to the controller (pie_set_extension_ratio < 0), every pie_decode_step ends by deciding how many layers m
+ * live on the CPU from the next token on (pie_layer_controller_decide: one more when no swap-in was needed or the share
+ * of swap-ins that fetched a layer of the NEXT token reached the trigger; one fewer when the computation waited) and, if
+ * m changed, by moving whole layers until n - m GPU regions and m + 2 CPU regions hold them (the pools must be sized for
+ * the values m may take).  share: the trigger, in [0, 1]; 0 = the rule's default (0.3).  pie_stats counts the swap-in
+ * lists started and those for the next token in both modes (with equal shares of every layer on the host, the block
+ * plan's default, the share is one group of layers in n and says nothing: the trigger acts in whole-layer mode only). */
+int pie_set_violation_trigger(pie_pool *pool, double share);
 /* The decisions taken so far in whole-layer mode: int32 quadruples {step, layer starting, layer whose swap-out
  * started or -1, layer whose swap-in started or -1}.  log may be NULL to ask for the count only. */
 int pie_get_layer_log(pie_pool *pool, int32_t *log, int64_t capacity, int64_t *n_entries);
@@ -247,7 +275,7 @@ int pie_set_lookahead(pie_pool *pool, int32_t layers);
 
 /* ---- 8-bit blocks (a variant beyond the paper, whose blocks are 16-bit: a token costs half the bytes in HBM, in the
  * host pool and on the link, so the same link hides twice the tokens per layer - Section 3.1's condition in bytes) ----
- * A pool created with reserved[2] = 1 stores a block as [n_kv_heads][K|V][16 tokens][128] bytes of E4M3 (1-4-3 bits,
+ * A pool created with kv_format = PIE_KV_E4M3 stores a block as [n_kv_heads][K|V][16 tokens][128] bytes of E4M3 (1-4-3 bits,
  * bias 7, no infinities, largest value 448); a stored byte b stands for decode(b) * k_scale (keys) or * v_scale
  * (values), one pair of scales for the pool (default 1, 1).  q, out and the new token's k_new / v_new stay in the pool's
  * 16-bit type.  pie_decode_attention computes attention over the decoded values (scores and sums in fp32 as for 16-bit
@@ -284,13 +312,13 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
  * call gets them; otherwise the ids given to pie_declare_append_blocks (host, n ids; valid until replaced; the
  * caller vouches for them - a block that is written but not listed would leave a stale host copy); with
  * neither (n < 0 or never declared), every block of the layer counts as written and nothing is elided.
- * Switching off takes effect unit by unit at its next swap-in.  pie_stats.reserved[2] counts the bytes elided. */
+ * Switching off takes effect unit by unit at its next swap-in.  pie_stats.bytes_out_elided counts the bytes elided. */
 int pie_set_retention(pie_pool *pool, int32_t on);
 int pie_declare_append_blocks(pie_pool *pool, const int32_t *ids, int64_t n);
 
 /* ---- run-time resize of the per-layer cache size (Section 4.1) -----------------------------------
  * n_logical_blocks is the physical width of the per-layer tables; the size visible to allocation is
- * reserved[1] of the configuration at creation (0: the full width) and changes in two phases:
+ * visible_blocks of the configuration at creation (0: the full width) and changes in two phases:
  *   grow:   pie_resize_begin(new) starts it; ids in [old, new) become allocatable only after every layer has
  *           gone through a swap pass (pie_plan_layer / pie_decode_step on that layer, or a swap call on it) -
  *           the space is prepared first and made visible afterwards;
@@ -411,6 +439,19 @@ int pie_fifo_complete(pie_fifo *f, int32_t dir);
 int pie_fifo_layer_start(pie_fifo *f, int32_t k, int32_t *start_out, int32_t *start_in);
 /* 0 GPU, 1 CPU, 2 in transit to the CPU, 3 in transit to the GPU */
 int pie_fifo_location(pie_fifo *f, int32_t layer);
+/* Swap-ins started so far, and how many of them fetched a layer that only the NEXT token needs (a layer below the one
+ * starting): Section 3.4.2 allows that violation of "swap what the current token needs" to prevent waiting at the
+ * first layers, and takes its frequency as the sign that the expansion is too small.  Either pointer may be NULL. */
+int pie_fifo_counters(const pie_fifo *f, int64_t *in_starts, int64_t *violations);
+/* Section 3.4.2's rule for the number m of layers kept on the CPU, from one window's measurements (a token or several):
+ * the computation waited (stall > eps * compute) -> m - 1, and that m is left alone for a while (4 windows, twice as
+ * long after every failed return, at most 96); otherwise, if no swap-in was started at all or the share of swap-ins that
+ * were for the next token has reached v_trigger -> m + 1 (at most m_max); else m.  The link is busy the whole time under
+ * the whole-layer protocol, whatever m is, so link slack cannot be the signal here.  state: 4 doubles owned by the
+ * caller, zero-initialised.  Constants are this build's (the paper gives none): v_trigger <= 0 -> 0.3, eps <= 0 ->
+ * 0.02.  With m CPU layers the protocol runs with n - m GPU regions and m + 2 CPU regions (Section 3.3). */
+int32_t pie_layer_controller_decide(double *state, int32_t m, int32_t m_max, double stall, double compute, int64_t in_starts,
+                                    int64_t violations, double v_trigger, double eps);
 
 /* The controller's decision rule by itself.  state: 16 doubles owned by the caller, zero-initialised
  * (history in [0..4]; [5] = stall tolerance eps, [6] = link-busy ceiling u_hi, 0 = defaults 0.02 / 0.9; [7..11] the
@@ -437,8 +478,8 @@ double pie_governor_report(pie_governor *g, double ratio, double throughput);
 int pie_governor_state(const pie_governor *g, int32_t *state, int32_t *cap_steps);
 /* The same inside a pool in adaptive mode: report the window's throughput (e.g. tokens per second); the pool's ratio is
  * held at or below the governor's cap from the next controller tick on (and never below what the GPU pool's size
- * allows).  The governor's step is the controller's (pie_set_controller).  pie_stats.reserved[4] = the cap (1 = none),
- * reserved[5] = the governor's state.  PIE_ERR_INVALID for a throughput that is not finite or negative. */
+ * allows).  The governor's step is the controller's (pie_set_controller).  pie_stats.governor_cap = the cap (1 = none),
+ * governor_state = the governor's state.  PIE_ERR_INVALID for a throughput that is not finite or negative. */
 int pie_report_throughput(pie_pool *pool, double throughput);
 
 #ifdef __cplusplus

@@ -29,6 +29,8 @@ class ProtocolResult:
     max_off_gpu: int      # most layers simultaneously on the CPU or in transit
     swaps_per_token: float
     finish_time: float
+    in_starts: int = 0    # swap-ins started
+    violations: int = 0   # ... of which for a layer the NEXT token needs (Section 3.4.2's allowed rule violation)
 
 
 def simulate_protocol(n_layers, t_swap, gpu_regions, cpu_regions, cpu_layers, n_tokens, t_compute=1.0):
@@ -39,6 +41,7 @@ def simulate_protocol(n_layers, t_swap, gpu_regions, cpu_regions, cpu_layers, n_
     in_busy = None
     events, trips, open_trip = [], [], {}
     stall, now, max_off, n_swaps = 0.0, 0.0, 0, 0
+    counts = {"in": 0, "violations": 0}
 
     def dist(l, k):  # compute-steps until layer l is needed again, seen from the start of layer k
         return (l - k) % n_layers
@@ -76,6 +79,9 @@ def simulate_protocol(n_layers, t_swap, gpu_regions, cpu_regions, cpu_layers, n_
                 loc[hot] = IN
                 in_busy = (t + t_swap, hot)
                 events.append((t, "in", hot))
+                counts["in"] += 1
+                # the current token still needs layers k .. n; a lower one is fetched for the token after it
+                counts["violations"] += hot < k
 
     for _tok in range(n_tokens):
         for k in range(1, n_layers + 1):
@@ -89,7 +95,46 @@ def simulate_protocol(n_layers, t_swap, gpu_regions, cpu_regions, cpu_layers, n_
                 start_swaps(now, k)
             max_off = max(max_off, sum(v != GPU for v in loc.values()))
             now += t_compute
-    return ProtocolResult(events, stall, trips, max_off, n_swaps / n_tokens, now)
+    return ProtocolResult(events, stall, trips, max_off, n_swaps / n_tokens, now, counts["in"], counts["violations"])
+
+
+# ---------------------------------------------------------------------------------------------
+# Adaptive expansion in whole layers (Section 3.4.2 as the paper states it): m = layers kept on the CPU.
+#   - more swapping: whenever a swap could be started and no on-CPU layer is needed by the token being computed, the
+#     expansion is too small.  Rather than leave the link idle the protocol then fetches a layer of the NEXT token (the
+#     violation the paper allows "to prevent waiting"); the share of swap-ins that are such violations is high while m is
+#     small and falls as m grows.  When it reaches the preset ratio (or nothing is on the CPU at all), m grows by one.
+#     The link is as busy before as after (the protocol swaps all the time), so link slack cannot be the signal here.
+#   - less swapping: the computation had to wait (stall above eps of the compute time): m shrinks by one, and the
+#     value that stalled is left alone for `hold` windows, twice as long after every failed return (a performance
+#     record, as for the block-granular controller).
+# The paper gives no constants; these are the build's: v_trigger = 0.3, eps = 0.02, hold = 4 windows at first.
+# ---------------------------------------------------------------------------------------------
+@dataclasses.dataclass
+class LayerController:
+    m_max: int
+    v_trigger: float = 0.3
+    eps: float = 0.02
+    m: int = 0
+    bad: int = -1          # lowest m known to make the computation wait (-1: none)
+    hold: int = 0          # windows left before `bad` may be tried again
+    hold_len: int = 4
+
+    def update(self, stall, compute, in_starts, violations):
+        """One window's measurements -> the number of CPU layers for the next window."""
+        if stall > self.eps * compute:
+            self.bad = self.m if self.bad < 0 else min(self.bad, self.m)
+            self.m = max(0, self.m - 1)
+            self.hold, self.hold_len = self.hold_len, min(2 * self.hold_len, 96)
+            return self.m
+        too_small = in_starts == 0 or violations >= self.v_trigger * in_starts
+        if too_small and self.m < self.m_max:
+            if self.bad >= 0 and self.m + 1 >= self.bad:
+                if self.hold > 0:
+                    self.hold -= 1
+                    return self.m
+            self.m += 1
+        return self.m
 
 
 # ---------------------------------------------------------------------------------------------

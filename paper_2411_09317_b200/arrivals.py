@@ -248,8 +248,8 @@ def run(driver: Driver, requests, max_steps=100000, emit=None):
             pie.pie_report_throughput(driver.pool, tps)
             st = pie.pie_get_stats(driver.pool)
             row = {"t": now, "step": steps, "running": len(driver.running), "waiting": len(waiting), "done": done,
-                   "tokens_per_s": tps, "ratio": pie.pie_get_extension_ratio(driver.pool), "ratio_floor": st["reserved"][1],
-                   "cap": st["reserved"][4], "governor": int(st["reserved"][5]), "ms_per_step": 1e3 * win_t / driver.window,
+                   "tokens_per_s": tps, "ratio": pie.pie_get_extension_ratio(driver.pool), "ratio_floor": st["ratio_floor"],
+                   "cap": st["governor_cap"], "governor": int(st["governor_state"]), "ms_per_step": 1e3 * win_t / driver.window,
                    "swap_in_gb": st["bytes_in"] / 1e9, "swap_out_gb": st["bytes_out"] / 1e9}
             driver.log.append(row)
             if emit:

@@ -32,8 +32,8 @@ EXPORTS = [
     "pie_get_extension_ratio", "pie_set_controller", "pie_plan_layer", "pie_controller_tick", "pie_get_stats", "pie_get_step_timeline", "pie_sync", "pie_status_str",
     "pie_last_cuda_error", "pie_probe_link", "pie_probe_hbm", "pie_table_create", "pie_table_destroy", "pie_table_alloc",
     "pie_table_free", "pie_table_swap", "pie_table_attention", "pie_table_confirm", "pie_table_state", "pie_fifo_create",
-    "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_controller_decide",
-    "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_get_layer_log",
+    "pie_fifo_destroy", "pie_fifo_complete", "pie_fifo_layer_start", "pie_fifo_location", "pie_fifo_counters", "pie_layer_controller_decide", "pie_controller_decide",
+    "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_set_violation_trigger", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_kept_copies", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
     "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
@@ -43,32 +43,38 @@ EXPORTS = [
 
 class PoolConfig(ctypes.Structure):
     _fields_ = [
+        ("struct_size", ctypes.c_uint32),
         ("n_layers", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("block_tokens", ctypes.c_int32), ("dtype", ctypes.c_int32),
-        ("n_logical_blocks", ctypes.c_int32), ("max_seqs", ctypes.c_int32),
+        ("n_logical_blocks", ctypes.c_int32), ("max_seqs", ctypes.c_int32), ("own_streams", ctypes.c_int32),
         ("n_gpu_slots", ctypes.c_int64), ("n_host_slots", ctypes.c_int64),
         ("gpu_base", ctypes.c_void_p), ("host_base", ctypes.c_void_p),
         ("compute_stream", ctypes.c_void_p), ("copy_in_stream", ctypes.c_void_p), ("copy_out_stream", ctypes.c_void_p),
-        ("own_streams", ctypes.c_int32), ("split_tokens", ctypes.c_int32), ("swap_ctas", ctypes.c_int32),
-        ("attn_ctas_per_sm", ctypes.c_int32), ("timing", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7),
+        ("split_tokens", ctypes.c_int32), ("swap_ctas", ctypes.c_int32),
+        ("attn_ctas_per_sm", ctypes.c_int32), ("timing", ctypes.c_int32),
+        ("attn_variant", ctypes.c_int32), ("visible_blocks", ctypes.c_int32), ("kv_format", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 5),
     ]
 
 
 class Stats(ctypes.Structure):
     _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("governor_state", ctypes.c_uint32),
         ("bytes_in", ctypes.c_double), ("bytes_out", ctypes.c_double),
         ("calls_kernel", ctypes.c_double), ("calls_copy_engine", ctypes.c_double),
         ("last_step_compute_ms", ctypes.c_double), ("last_step_stall_ms", ctypes.c_double),
         ("last_step_swap_in_ms", ctypes.c_double), ("last_step_swap_out_ms", ctypes.c_double),
         ("last_step_ms", ctypes.c_double), ("ratio", ctypes.c_double),
         ("n_units_gpu", ctypes.c_int64), ("n_units_host", ctypes.c_int64), ("n_units_in_flight", ctypes.c_int64),
-        ("steps_measured", ctypes.c_int64), ("reserved", ctypes.c_double * 8),
+        ("steps_measured", ctypes.c_int64),
+        ("last_step_slowdown_ms", ctypes.c_double), ("ratio_floor", ctypes.c_double), ("bytes_out_elided", ctypes.c_double),
+        ("patch_kernel_launches", ctypes.c_double), ("governor_cap", ctypes.c_double),
+        ("prefetch_lists", ctypes.c_int64), ("prefetch_violations", ctypes.c_int64),
+        ("last_step_violation_ratio", ctypes.c_double), ("reserved", ctypes.c_double * 4),
     ]
 
     def as_dict(self):
-        d = {k: getattr(self, k) for k, _ in self._fields_ if k != "reserved"}
-        d["reserved"] = list(self.reserved)
-        return d
+        return {k: getattr(self, k) for k, _ in self._fields_ if k not in ("reserved", "struct_size")}
 
 
 lib = ctypes.CDLL(LIB_PATH)
@@ -141,6 +147,9 @@ _sig = {
     "pie_fifo_layer_start": (_i32, [_vp, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "pie_fifo_location": (_i32, [_vp, _i32]),
     "pie_controller_decide": (_f64, [_vp, _f64, _f64, _f64, _f64, _f64]),
+    "pie_set_violation_trigger": (_i32, [_vp, _f64]),
+    "pie_fifo_counters": (_i32, [_vp, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "pie_layer_controller_decide": (_i32, [_vp, _i32, _i32, _f64, _f64, _i64, _i64, _f64, _f64]),
     "pie_decode_attention_noalloc": (_i32, [_vp, _i64, _vp, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
                                             _i32, _f32, _vp, _vp]),
 }
@@ -182,9 +191,10 @@ def pie_pool_create(**kw) -> int:
     kw.setdefault("block_tokens", 16)
     kw.setdefault("own_streams", 1)
     kw.setdefault("max_seqs", 256)
-    cfg.reserved[0] = kw.pop("attn_variant", 0)
-    cfg.reserved[1] = kw.pop("visible_blocks", 0)
-    cfg.reserved[2] = int(kw.pop("kv_fp8", 0))
+    cfg.struct_size = ctypes.sizeof(PoolConfig)
+    cfg.attn_variant = kw.pop("attn_variant", 0)
+    cfg.visible_blocks = kw.pop("visible_blocks", 0)
+    cfg.kv_format = int(kw.pop("kv_fp8", 0))
     for k, v in kw.items():
         setattr(cfg, k, v)
     out = _vp()
@@ -199,6 +209,10 @@ def pie_pool_destroy(pool) -> None:
 def pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs) -> None:
     check(lib.pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq,
                            n_seqs), "pie_kv_write")
+
+
+def pie_set_violation_trigger(pool, share) -> None:
+    check(lib.pie_set_violation_trigger(pool, share), "pie_set_violation_trigger")
 
 
 def pie_set_lookahead(pool, layers) -> None:
@@ -389,6 +403,7 @@ def pie_controller_tick(pool) -> bool:
 
 def pie_get_stats(pool) -> dict:
     s = Stats()
+    s.struct_size = ctypes.sizeof(Stats)
     check(lib.pie_get_stats(pool, ctypes.byref(s)), "pie_get_stats")
     return s.as_dict()
 
@@ -533,10 +548,21 @@ class Fifo:
     def location(self, layer):
         return lib.pie_fifo_location(self.h, layer)
 
+    def counters(self):
+        """-> (swap-ins started, of which for a layer of the next token)"""
+        a, b = _i64(), _i64()
+        check(lib.pie_fifo_counters(self.h, ctypes.byref(a), ctypes.byref(b)), "pie_fifo_counters")
+        return a.value, b.value
+
 
 def pie_controller_decide(state: np.ndarray, ratio, step, stall, compute, swap_busy) -> float:
     assert state.dtype == np.float64 and state.size >= 8
     return lib.pie_controller_decide(_ptr(state), ratio, step, stall, compute, swap_busy)
+
+
+def pie_layer_controller_decide(state: np.ndarray, m, m_max, stall, compute, in_starts, violations, v_trigger=0.0, eps=0.0) -> int:
+    assert state.dtype == np.float64 and state.size >= 4
+    return lib.pie_layer_controller_decide(_ptr(state), m, m_max, stall, compute, in_starts, violations, v_trigger, eps)
 
 
 # ---- input generator kernels (separate library; inputs only) ---------------------------------------------------

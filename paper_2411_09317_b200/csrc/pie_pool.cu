@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <chrono>
 #include <cmath>
+#include <cstddef>
 #include <cstdio>
 #include <cstring>
 #include <deque>
@@ -72,7 +73,7 @@ struct SwapList {
 struct pie_pool {
     pie_pool_config cfg{};
     int64_t block_bytes = 0;
-    int kv_fp8 = 0;                       // blocks hold E4M3 bytes (cfg.reserved[2])
+    int kv_fp8 = 0;                       // blocks hold E4M3 bytes (cfg.kv_format)
     float k_scale = 1.f, v_scale = 1.f;   // a stored byte stands for decode(byte) * scale
     pie::Table *table = nullptr;
     uint8_t *gpu_base = nullptr, *host_base = nullptr;
@@ -149,6 +150,10 @@ struct pie_pool {
     std::vector<std::vector<int32_t>> home_list;  // per layer: ids the planner looks at (see candidate_ids)
     std::vector<uint8_t> home_dirty;              // per layer: home_list must be rebuilt
     // whole-layer protocol (Section 3.3): when set, pie_decode_step moves whole layers as the scheduler says
+    double layer_ctrl_state[4] = {};   // whole-layer adaptive rule (pie_layer_controller_decide)
+    double violation_trigger = 0.0;    // share of next-token prefetches that triggers an increase (0: the rule's default)
+    int64_t step_prefetch[TIMING_RING][2] = {};   // per step set: swap-in lists started, of which for the next token
+    int32_t fifo_cpu_layers = 0;       // whole-layer mode: m, the layers that live on the CPU (cpu_regions - 2)
     pie::Fifo *fifo = nullptr;
     int64_t fifo_ticket[3] = {0, 0, 0};        // ticket of the layer swap in flight, per queue (0 = none)
     std::vector<int32_t> fifo_log;             // {step, layer starting, swap-out started or -1, swap-in started or -1} x n
@@ -467,7 +472,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
             }
         } else if (slot_table_row) {
             PIE_CUDA(pie::launch_patch_from_list(slot_table_row, p->list_host + off, n, table_mode, stream));
-            p->stats.reserved[3] += 1;
+            p->stats.patch_kernel_launches += 1;
         }
         p->stats.calls_copy_engine += 1;
     }
@@ -526,7 +531,7 @@ int swap_prepare(pie_pool *p, int queue, int32_t layer, const int32_t *ids, int6
 
 void swap_account(pie_pool *p, int queue, const SwapList &l) {
     (queue == PIE_Q_IN ? p->stats.bytes_in : p->stats.bytes_out) += (double)(l.n_moved - l.n_elided) * (double)p->block_bytes;
-    p->stats.reserved[2] += (double)l.n_elided * (double)p->block_bytes;
+    p->stats.bytes_out_elided += (double)l.n_elided * (double)p->block_bytes;
 }
 
 // not_before: a compute ticket the copy must not start before (0 = none).  The decode loop uses it to start a
@@ -873,7 +878,7 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.gpu_pool = p->gpu_base;
     a.split_tokens = (int32_t)split;
     a.grid = p->attn_grid;
-    a.variant = p->cfg.reserved[0];
+    a.variant = p->cfg.attn_variant;
     a.status = p->status_dev;
     a.stamps = le ? stamp_dev(p, layer, STAMP_START) : nullptr;
     a.arrive = p->arrive_dev + layer;
@@ -1158,8 +1163,15 @@ int pie_last_cuda_error(void) { return g_last_cuda_error; }
 
 size_t pie_block_bytes(const pie_pool *pool) { return pool ? (size_t)pool->block_bytes : 0; }
 
-int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
-    if (!cfg || !out) return PIE_ERR_INVALID;
+int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
+    if (!cfg_in || !out) return PIE_ERR_INVALID;
+    // the caller's struct may be older (shorter) or newer (longer) than this build's: take what both know
+    if (cfg_in->struct_size < offsetof(pie_pool_config, timing) + sizeof(int32_t)) return PIE_ERR_INVALID;
+    pie_pool_config cfg_local;
+    std::memset(&cfg_local, 0, sizeof cfg_local);
+    std::memcpy(&cfg_local, cfg_in, std::min<size_t>(cfg_in->struct_size, sizeof cfg_local));
+    cfg_local.struct_size = (uint32_t)sizeof cfg_local;
+    const pie_pool_config *cfg = &cfg_local;
     if (cfg->n_layers <= 0 || cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->n_logical_blocks <= 0 ||
         cfg->n_gpu_slots <= 0 || cfg->n_host_slots < 0 || cfg->max_seqs <= 0)
         return PIE_ERR_INVALID;
@@ -1167,8 +1179,8 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     if (cfg->dtype != PIE_F16 && cfg->dtype != PIE_BF16) return PIE_ERR_INVALID;
     if (cfg->block_tokens != 16 || (cfg->head_dim != 64 && cfg->head_dim != 128)) return PIE_ERR_UNSUPPORTED;
     if (cfg->n_q_heads / cfg->n_kv_heads > 8) return PIE_ERR_UNSUPPORTED;
-    if (cfg->reserved[2] != 0 && cfg->reserved[2] != 1) return PIE_ERR_INVALID;
-    if (cfg->reserved[2] == 1 && (cfg->head_dim != 128 || cfg->reserved[0] < 0 || cfg->reserved[0] > 2)) return PIE_ERR_UNSUPPORTED;
+    if (cfg->kv_format != 0 && cfg->kv_format != 1) return PIE_ERR_INVALID;
+    if (cfg->kv_format == 1 && (cfg->head_dim != 128 || cfg->attn_variant < 0 || cfg->attn_variant > 2)) return PIE_ERR_UNSUPPORTED;
     if (cfg->split_tokens < 0 || cfg->split_tokens % 16 != 0) return PIE_ERR_INVALID;
     if (cfg->gpu_base && ((uintptr_t)cfg->gpu_base & 127)) return PIE_ERR_INVALID;
     if ((uint64_t)cfg->n_gpu_slots * (uint64_t)cfg->n_kv_heads * 32u > 0x7fffffffull) return PIE_ERR_UNSUPPORTED;
@@ -1193,12 +1205,12 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
     // (measured: +6.5 % on 17 sequences of 4k-32k tokens with 8-head groups, -1.5 % on the batched shapes).
     if (p->cfg.split_tokens == 0)
         p->cfg.split_tokens = (int64_t)cfg->n_logical_blocks * 16 / std::max(cfg->max_seqs, 1) >= 6144 ? 1024 : 512;
-    p->kv_fp8 = cfg->reserved[2];
+    p->kv_fp8 = cfg->kv_format;
     p->block_bytes = (int64_t)2 * 16 * cfg->n_kv_heads * cfg->head_dim * (p->kv_fp8 ? 1 : 2);
     p->n_sms = prop.multiProcessorCount;
     p->table = new (std::nothrow) pie::Table(cfg->n_layers, cfg->n_logical_blocks, cfg->n_gpu_slots, cfg->n_host_slots);
     if (!p->table) { destroy_pool(p); return PIE_ERR_NOMEM; }
-    if (cfg->reserved[1] != 0 && p->table->init_capacity(cfg->reserved[1]) != PIE_OK) { destroy_pool(p); return PIE_ERR_INVALID; }
+    if (cfg->visible_blocks != 0 && p->table->init_capacity(cfg->visible_blocks) != PIE_OK) { destroy_pool(p); return PIE_ERR_INVALID; }
     p->home_count.assign((size_t)cfg->n_layers, 0);
     p->home_list.assign((size_t)cfg->n_layers, std::vector<int32_t>());
     p->home_dirty.assign((size_t)cfg->n_layers, 1);
@@ -1313,7 +1325,7 @@ int pie_pool_create(const pie_pool_config *cfg, pie_pool **out) {
             if (env[0] == '1') p->use3d = 0;
     }
     int per_sm = 0;
-    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, cfg->reserved[0], &per_sm, p->kv_fp8), PIE_ERR_CUDA);
+    PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, cfg->attn_variant, &per_sm, p->kv_fp8), PIE_ERR_CUDA);
     if (per_sm <= 0) { destroy_pool(p); return PIE_ERR_UNSUPPORTED; }
     if (cfg->attn_ctas_per_sm > 0) per_sm = std::min(per_sm, cfg->attn_ctas_per_sm);
     p->attn_grid = per_sm * p->n_sms;
@@ -1612,6 +1624,8 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     pool->stats.last_step_swap_out_ms = t_out;
     if (first && last) pool->stats.last_step_ms = (double)(last - first) * 1e-6 + first_stall;
     pool->stats.steps_measured += 1;
+    pool->stats.last_step_violation_ratio =
+        pool->step_prefetch[k][0] > 0 ? (double)pool->step_prefetch[k][1] / (double)pool->step_prefetch[k][0] : 0.0;
     // Copies that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
     // wait, so the controller holds the ratio where wait + slow-down stays within its tolerance.  Every layer of a step
     // attends the same batch at the same lengths, and the swap lists of a group of layers are in flight during the first
@@ -1640,8 +1654,8 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         if (!any_swap) pool->base_ms_per_token = pool->base_ms_per_token > 0 ? 0.75 * pool->base_ms_per_token + 0.25 * per_token : per_token;
         else if (pool->base_ms_per_token > 0) slow = std::max(0.0, compute - pool->base_ms_per_token * tokens);
     }
-    pool->stats.reserved[0] = slow;
-    pool->stats.reserved[1] = ratio_floor(pool);
+    pool->stats.last_step_slowdown_ms = slow;
+    pool->stats.ratio_floor = ratio_floor(pool);
     if (pool->ratio_mode == 2 && compute > 0) {
         const double step = pool->ctrl_step > 0 ? pool->ctrl_step : 1.0 / (double)pool->cfg.n_layers;  // "one layer" (Section 3.4.2)
         // the rule never asks for less than the GPU pool's size allows: below that floor the number would drift
@@ -1693,6 +1707,7 @@ int pie_step_begin(pie_pool *pool) {
         for (LayerEvents &e : pool->lev[k]) e.has_in = e.has_out = e.has_compute = e.stream_wait = false;
         for (int q = 0; q < 4; ++q) pool->lev_last[k][q] = nullptr;
         pool->lev_anchored[k] = false;
+        pool->step_prefetch[k][0] = pool->step_prefetch[k][1] = 0;
         // the set's kernels are launched after this point, and the previous user of the set has completed
         std::memset(pool->stamps_host + (size_t)k * (size_t)pool->cfg.n_layers * STAMP_WORDS, 0,
                     (size_t)pool->cfg.n_layers * STAMP_WORDS * 8);
@@ -1792,8 +1807,8 @@ int pie_report_throughput(pie_pool *pool, double throughput) {
     pool->ratio_cap = pie_governor_report(pool->governor, pool->ratio, throughput);
     int32_t state = 0;
     pie_governor_state(pool->governor, &state, nullptr);
-    pool->stats.reserved[4] = pool->ratio_cap;
-    pool->stats.reserved[5] = state;
+    pool->stats.governor_cap = pool->ratio_cap;
+    pool->stats.governor_state = (uint32_t)state;
     return PIE_OK;
 }
 
@@ -1880,10 +1895,21 @@ int pie_get_step_timeline(pie_pool *pool, float *ms, int64_t capacity) {
     return PIE_OK;
 }
 
-int pie_get_stats(pie_pool *pool, pie_stats *out) {
-    if (!pool || !out) return PIE_ERR_INVALID;
+int pie_get_stats(pie_pool *pool, pie_stats *out_caller) {
+    if (!pool || !out_caller) return PIE_ERR_INVALID;
+    if (out_caller->struct_size < offsetof(pie_stats, steps_measured) + sizeof(int64_t)) return PIE_ERR_INVALID;
+    // filled in a struct of this build's layout, then as much of it copied out as the caller's struct holds
+    struct Copy {
+        pie_stats local;
+        pie_stats *dst;
+        ~Copy() {
+            const uint32_t n = std::min<uint32_t>(dst->struct_size, (uint32_t)sizeof local);
+            local.struct_size = dst->struct_size;
+            std::memcpy(dst, &local, n);
+        }
+    } copy{pool->stats, out_caller};
+    pie_stats *out = &copy.local;
     poll(pool);
-    *out = pool->stats;
     float r = 0;
     pie_get_extension_ratio(pool, &r);
     out->ratio = r;
@@ -1949,7 +1975,43 @@ int pie_set_layer_policy(pie_pool *pool, int32_t gpu_regions, int32_t cpu_region
     pool->fifo = new (std::nothrow) pie::Fifo(L, gpu_regions, cpu_regions, on_cpu.data());
     if (!pool->fifo) return PIE_ERR_NOMEM;
     pool->fifo_ticket[PIE_Q_IN] = pool->fifo_ticket[PIE_Q_OUT] = 0;
+    pool->fifo_cpu_layers = std::max(0, cpu_regions - 2);
     pool->fifo_log.clear();
+    return PIE_OK;
+}
+
+// Whole-layer mode with m layers on the CPU: n - m GPU regions and m + 2 CPU regions (Section 3.3).  Between two
+// tokens: everything settles, as many whole layers as the new region counts require move (the coldest GPU layers out -
+// the highest, seen from layer 0 - or the hottest CPU layers in), and the scheduler starts afresh from the placement.
+static int fifo_set_cpu_layers(pie_pool *pool, int32_t m, int32_t mode) {
+    const int32_t L = pool->cfg.n_layers;
+    m = std::max(0, std::min(m, L - 2));
+    std::vector<int32_t> ids;
+    all_block_ids(pool, ids);
+    for (int pass = 0; pass < 2 * L; ++pass) {
+        int st = sync_all(pool, 30 * 1000 * 1000);
+        if (st != PIE_OK) return st;
+        std::vector<int32_t> on_gpu, on_cpu;
+        for (int32_t l = 0; l < L; ++l) {
+            bool host = false;
+            for (int32_t b : ids) host = host || pool->table->unit(l, b).side == PIE_HOST;
+            (host ? on_cpu : on_gpu).push_back(l);
+        }
+        if ((int32_t)on_gpu.size() > L - m) st = pool_swap(pool, PIE_Q_OUT, on_gpu.back(), ids.data(), (int64_t)ids.size(), mode);
+        else if ((int32_t)on_cpu.size() > m + 2) st = pool_swap(pool, PIE_Q_IN, on_cpu.front(), ids.data(), (int64_t)ids.size(), mode);
+        else break;
+        if (st != PIE_OK) return st;
+    }
+    std::vector<int32_t> log;
+    log.swap(pool->fifo_log);            // the decisions so far stay readable across the change
+    const int st = pie_set_layer_policy(pool, L - m, m + 2);
+    pool->fifo_log.swap(log);
+    return st;
+}
+
+int pie_set_violation_trigger(pie_pool *pool, double share) {
+    if (!pool || share < 0 || share > 1 || share != share) return PIE_ERR_INVALID;
+    pool->violation_trigger = share;
     return PIE_OK;
 }
 
@@ -1962,6 +2024,16 @@ int pie_get_layer_log(pie_pool *pool, int32_t *log, int64_t capacity, int64_t *n
         std::copy(pool->fifo_log.begin(), pool->fifo_log.end(), log);
     }
     return PIE_OK;
+}
+
+// A swap-in list started by the decode loop; next_token: it serves a layer that only the next token needs (Section
+// 3.4.2's allowed rule violation: the prefetch that wraps around the last layer).
+static void count_prefetch(pie_pool *pool, bool next_token) {
+    pool->stats.prefetch_lists += 1;
+    pool->stats.prefetch_violations += next_token;
+    const int k = (int)(pool->step % TIMING_RING);
+    pool->step_prefetch[k][0] += 1;
+    pool->step_prefetch[k][1] += next_token;
 }
 
 // confirmed completions -> scheduler (a finished swap-out frees its GPU region, a finished swap-in its CPU region)
@@ -1982,6 +2054,7 @@ static int fifo_start_swaps(pie_pool *pool, int32_t k, int32_t mode, std::vector
     int st = pool->fifo->layer_start(k, &so, &si);
     if (st != PIE_OK) return st;
     pool->fifo_log.insert(pool->fifo_log.end(), {(int32_t)pool->step, k, so, si});
+    if (si >= 0) count_prefetch(pool, si < k);
     for (int which = 0; which < 2; ++which) {
         const int32_t layer = which == 0 ? so : si;
         const int q = which == 0 ? PIE_Q_OUT : PIE_Q_IN;
@@ -2006,6 +2079,8 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
     int st = pie_step_begin(pool);
     if (st != PIE_OK) return st;
     std::vector<int32_t> ids;
+    const auto t_step = std::chrono::steady_clock::now();
+    double waited_ms = 0.0;   // host clock: what the presence check below had to wait for layers still on the CPU
     for (int32_t k = 0; k < L; ++k) {
         // the control logic runs when layer k starts, i.e. when layer k-1 has finished: the host keeps step with
         // the device here (as the paper's per-layer control loop does), so completions are what they really are
@@ -2023,11 +2098,13 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
         for (int guard = 0; pool->fifo->location(k) == 1; ++guard) {
             if (guard > 4 * L) return PIE_ERR_TIMEOUT;
             bool waited = false;
+            const auto t_wait = std::chrono::steady_clock::now();
             for (int q : {PIE_Q_OUT, PIE_Q_IN})
                 if (pool->fifo_ticket[q] > 0) {
                     PIE_CUDA(cudaEventSynchronize(pool->ticket_ev[q][pool->fifo_ticket[q] % EV_RING]));
                     waited = true;
                 }
+            waited_ms += std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_wait).count();
             if (!waited) return PIE_ERR_NOMEM;  // nothing in flight and still no GPU region for layer k
             st = fifo_apply_completions(pool);
             if (st != PIE_OK) return st;
@@ -2041,7 +2118,17 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
                             v_new_all ? (const uint8_t *)v_new_all + k * kv_stride : nullptr);
         if (st != PIE_OK) return st;
     }
-    return pie_controller_tick(pool, nullptr);
+    st = pie_controller_tick(pool, nullptr);
+    if (st != PIE_OK || pool->ratio_mode != 2) return st;
+    // Adaptive expansion in whole layers (Section 3.4.2): this token's waiting and the share of its swap-ins that were
+    // for the next token decide how many layers live on the CPU from the next token on.
+    const double step_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_step).count();
+    const int k_set = (int)(pool->step % TIMING_RING);
+    const int32_t m = pool->fifo_cpu_layers;
+    const int32_t m_new = pie_layer_controller_decide(pool->layer_ctrl_state, m, std::max(0, L - 2), waited_ms,
+                                                      std::max(1e-9, step_ms - waited_ms), pool->step_prefetch[k_set][0],
+                                                      pool->step_prefetch[k_set][1], pool->violation_trigger, pool->ctrl_state[5]);
+    return m_new == m ? PIE_OK : fifo_set_cpu_layers(pool, m_new, mode);
 }
 
 // One layer of the control loop (Section 3.2; Section 4.2: what a model's forward pass calls per layer): fetch what the
@@ -2092,6 +2179,7 @@ static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, con
             plan_in(pool, target, in_ids);
             if (in_ids.empty()) continue;
             st = swap_prepare(pool, PIE_Q_IN, target, in_ids.data(), (int64_t)in_ids.size(), &lists[n_lists++]);
+            if (st == PIE_OK && lists[n_lists - 1].n_moved > 0) count_prefetch(pool, target < l);
         }
         const int st2 = swap_issue_group(pool, PIE_Q_IN, lists, mode, start_with);   // what was prepared must be issued
         if (st != PIE_OK) return st;

@@ -480,6 +480,10 @@ int Fifo::layer_start(int32_t k, int32_t *start_out, int32_t *start_in) {
             loc_[hot] = 3;
             in_layer_ = hot;
             *start_in = hot;
+            // the token being computed still needs layers k .. n-1: a lower one is fetched for the token after it
+            // (Section 3.4.2: the rule violation that is allowed "to prevent waiting")
+            ++in_starts_;
+            if (hot < k) ++violations_;
         }
     }
     return PIE_OK;
@@ -573,6 +577,36 @@ int pie_fifo_layer_start(pie_fifo *f, int32_t k, int32_t *start_out, int32_t *st
 }
 int pie_fifo_location(pie_fifo *f, int32_t layer) {
     return f ? reinterpret_cast<Fifo *>(f)->location(layer) : PIE_ERR_INVALID;
+}
+int pie_fifo_counters(const pie_fifo *f, int64_t *in_starts, int64_t *violations) {
+    if (!f) return PIE_ERR_INVALID;
+    if (in_starts) *in_starts = reinterpret_cast<const Fifo *>(f)->in_starts();
+    if (violations) *violations = reinterpret_cast<const Fifo *>(f)->violations();
+    return PIE_OK;
+}
+
+// state: [0] 1 + the lowest number of CPU layers known to make the computation wait (0: none), [1] windows left before
+// it may be tried again, [2] the length of the next such pause (0: the first, 4; doubles up to 96).
+int32_t pie_layer_controller_decide(double *state, int32_t m, int32_t m_max, double stall, double compute, int64_t in_starts,
+                                    int64_t violations, double v_trigger, double eps) {
+    if (v_trigger <= 0) v_trigger = 0.3;
+    if (eps <= 0) eps = 0.02;
+    if (state[2] <= 0) state[2] = 4;
+    if (stall > eps * compute) {
+        state[0] = state[0] > 0 ? std::min(state[0], 1.0 + m) : 1.0 + m;
+        state[1] = state[2];
+        state[2] = std::min(2.0 * state[2], 96.0);
+        return std::max(0, m - 1);
+    }
+    const bool too_small = in_starts == 0 || (double)violations >= v_trigger * (double)in_starts;
+    if (too_small && m < m_max) {
+        if (state[0] > 0 && m + 1 >= (int32_t)state[0] - 1 && state[1] > 0) {
+            state[1] -= 1;
+            return m;
+        }
+        return m + 1;
+    }
+    return m;
 }
 
 // state[0..3]: stalled flags of the last steps (newest last), state[4]: how many are valid,

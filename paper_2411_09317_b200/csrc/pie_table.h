@@ -145,8 +145,11 @@ class Fifo {
     int complete(int32_t dir);
     int layer_start(int32_t k, int32_t *start_out, int32_t *start_in);
     int location(int32_t layer) const;
+    int64_t in_starts() const { return in_starts_; }     // swap-ins started so far
+    int64_t violations() const { return violations_; }   // ... of which for a layer of the next token
 
   private:
+    int64_t in_starts_ = 0, violations_ = 0;
     int32_t n_, gpu_regions_, cpu_regions_;
     std::vector<uint8_t> loc_;  // 0 GPU, 1 CPU, 2 to CPU, 3 to GPU
     int32_t out_layer_ = -1, in_layer_ = -1;

@@ -152,7 +152,7 @@ def main(argv=None):
                   "wait_share": sa["last_step_stall_ms"] / max(sa["last_step_ms"], 1e-9),
                   "last_step": {k: sa[k] for k in ("last_step_ms", "last_step_compute_ms", "last_step_stall_ms",
                                                    "last_step_swap_in_ms", "last_step_swap_out_ms")},
-                  "elided_out_gbs": (sa["reserved"][2] - sb["reserved"][2]) / tot / 1e9,
+                  "elided_out_gbs": (sa["bytes_out_elided"] - sb["bytes_out_elided"]) / tot / 1e9,
                   "calls_kernel": sa["calls_kernel"] - sb["calls_kernel"],
                   "calls_copy_engine": sa["calls_copy_engine"] - sb["calls_copy_engine"],
                   "swap_frac_of_link": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9 / link["both_per_dir"]})
@@ -173,11 +173,11 @@ def main(argv=None):
         pie.pie_set_extension_ratio(dw.pool, -1.0)
         per, sb, sa, ctx0, per_stats = run_steps(dw, args.steps)
         for i, (ms, st) in enumerate(zip(per, per_stats)):
-            emit({"step": i, "ratio": st["ratio"], "ratio_floor": st["reserved"][1], "ms_per_step": ms,
+            emit({"step": i, "ratio": st["ratio"], "ratio_floor": st["ratio_floor"], "ms_per_step": ms,
                   "wait_share_of_last_measured_step": st["last_step_stall_ms"] / max(st["last_step_ms"], 1e-9),
-                  "slowdown_share_of_last_measured_step": st["reserved"][0] / max(st["last_step_compute_ms"], 1e-9)})
+                  "slowdown_share_of_last_measured_step": st["last_step_slowdown_ms"] / max(st["last_step_compute_ms"], 1e-9)})
         tot = sum(per) * 1e-3
-        emit({"summary": True, "final_ratio": sa["ratio"], "ratio_floor": sa["reserved"][1], "median_ms_per_step": float(np.median(per)),
+        emit({"summary": True, "final_ratio": sa["ratio"], "ratio_floor": sa["ratio_floor"], "median_ms_per_step": float(np.median(per)),
               "swap_in_gbs": (sa["bytes_in"] - sb["bytes_in"]) / tot / 1e9, "swap_out_gbs": (sa["bytes_out"] - sb["bytes_out"]) / tot / 1e9,
               "attn_gbs": attention_bytes(wl, ctx0 + args.steps // 2) / (float(np.median(per)) * 1e-3) / 1e9})
     dw.close()
@@ -307,7 +307,7 @@ def interference(args, wl, link, emit):
             dw.decode_step()
             st = pie.pie_get_stats(dw.pool)
             ratios.append(st["ratio"])
-            slow.append((st["last_step_stall_ms"] + st["reserved"][0]) / max(st["last_step_compute_ms"], 1e-9))
+            slow.append((st["last_step_stall_ms"] + st["last_step_slowdown_ms"]) / max(st["last_step_compute_ms"], 1e-9))
             with torch.cuda.stream(dw.s_compute):
                 marks[i + 1].record()
         dw.sync()

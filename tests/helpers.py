@@ -89,3 +89,17 @@ def dense_attention(q, K, V, scale):
         p /= p.sum()
         out[h] = p @ V[:, h // g, :]
     return out
+
+
+TOL = 2e-3   # max-abs bound on attention outputs (fp16 / bf16 inputs)
+
+
+def tolerance(want, dtype):
+    """Element-wise bound on |got - want|.  Flat 2e-3 wherever the exact output is small (|want| < 0.25: every element
+    of the N(0,1) workloads with contexts of a hundred tokens or more).  Where |want| >= 0.25 (very short contexts,
+    dominant keys, scaled inputs) rounding the output to 16 bits alone costs up to half an ulp - 2^-8 |want| in bf16
+    (8 significant bits), 2^-11 |want| in fp16 (11 bits) - and the bound is 2e-3 plus that."""
+    from paper_2411_09317_b200 import synth
+    want = np.asarray(want)
+    half_ulp = (2.0 ** -8 if dtype == synth.BF16 else 2.0 ** -11) * np.abs(want)
+    return TOL + np.where(np.abs(want) >= 0.25, half_ulp, 0.0)

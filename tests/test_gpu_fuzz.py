@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import Case
+from helpers import Case, tolerance
 from gpu_helpers import PoolCase, oracle_attention
 from oracle import fp8
 from paper_2411_09317_b200 import binding as pie
@@ -88,7 +88,7 @@ def test_random_case_matches_oracle(seed):
         want = oracle_attention(case, 0)
         pie.pie_sync(pc.pool)
     got = synth.bits16_to_f32(pc.out[0].cpu().numpy().view(np.uint16), case.dtype)
-    bound = TOL + (2.0 ** -8 if case.dtype == BF16 else 2.0 ** -11) * np.abs(want)
+    bound = tolerance(want, case.dtype)
     assert np.all(np.abs(got - want) <= bound), (c, float(np.abs(got - want).max()))
     pc.close()
 
@@ -150,7 +150,7 @@ def test_random_decode_steps_with_changing_ratio_match_oracle(seed):
                               case.block_table, cur, case.Hkv, case.D)
             want = oracle_attention(case, l)
             got = synth.bits16_to_f32(pc.out[l].cpu().numpy().view(np.uint16), dtype)
-            bound = TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
+            bound = tolerance(want, dtype)
             assert np.all(np.abs(got - want) <= bound), (seed, t, l, float(np.abs(got - want).max()))
     for l in range(L):
         for b in range(case.NB):
@@ -237,7 +237,7 @@ def test_random_pool_operations_keep_every_unit_and_attend_correctly(seed):
             slot_of[order] = np.arange(len(order))
             want = oracle.paged_attention(store, store, np.zeros(NB, np.int32), slot_of, q, bt, lens, hq, hkv, d, dtype, 1.0 / np.sqrt(d))
             got = synth.bits16_to_f32(out_dev.cpu().numpy().view(np.uint16), dtype)
-            bound = TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
+            bound = tolerance(want, dtype)
             assert np.all(np.abs(got - want) <= bound), (seed, step, float(np.abs(got - want).max()))
     pie.pie_sync(pool)
     for (l, b), bits in content.items():
@@ -293,7 +293,7 @@ def test_random_whole_layer_protocol_configurations_match_oracle(seed):
                           case.block_table, cur, case.Hkv, case.D)
             want = oracle_attention(case, l)
             got = synth.bits16_to_f32(out[l].cpu().numpy().view(np.uint16), dtype)
-            bound = TOL + (2.0 ** -8 if dtype == BF16 else 2.0 ** -11) * np.abs(want)
+            bound = tolerance(want, dtype)
             assert np.all(np.abs(got - want) <= bound), (seed, L, m, gpu_regions, cpu_regions, t, l)
     for l in range(L):
         for b in range(NB):

@@ -215,6 +215,7 @@ def drive_fifo(n, t_swap, gpu_regions, cpu_regions, cpu_layers, n_tokens):
                 complete(now)
                 start(now, k)
             now += 1.0
+    drive_fifo.counters = f.counters()
     return events, stall
 
 
@@ -238,6 +239,26 @@ def test_fifo_matches_oracle_protocol(n, t_swap, g, c, cpu):
     ref = policy.simulate_protocol(n, t_swap, g, c, cpu, 7)
     assert events == ref.events
     assert stall == pytest.approx(ref.stall)
+    assert drive_fifo.counters == (ref.in_starts, ref.violations)     # swap-ins started, of which for the next token
+
+
+@pytest.mark.parametrize("t_swap", [1.0, 1.5, 2.0, 3.0])
+def test_layer_controller_rule_matches_oracle_on_the_protocol_simulator(t_swap):
+    """Section 3.4.2's rule for the number of CPU layers: the library's against the oracle's, both fed by the protocol
+    simulator window after window (and by random measurements afterwards)."""
+    n = 9
+    c = policy.LayerController(m_max=n - 2)
+    state, m = np.zeros(4), 0
+    rng = random.Random(int(t_swap * 10))
+    for w in range(60):
+        if w < 40:
+            r = policy.simulate_protocol(n, t_swap, n - m, m + 2, set(range(n - m + 1, n + 1)), 5)
+            meas = (r.stall, 5.0 * n, r.in_starts, r.violations)
+        else:
+            meas = (rng.choice([0.0, 0.0, 3.0]), 45.0, rng.randint(0, 30), rng.randint(0, 12))
+        want = c.update(*meas)
+        m = pie.pie_layer_controller_decide(state, m, n - 2, *meas)
+        assert m == want, (w, meas)
 
 
 # ------------------------------------------------------------------------------------ controller rule

@@ -502,6 +502,42 @@ def test_protocol_reproduces_the_nine_layer_example():
     assert len(late) / 4 == pytest.approx(4.5)
 
 
+def test_next_token_prefetches_become_rare_as_more_layers_live_on_the_cpu():
+    """Section 3.4.2: fetching a layer that only the NEXT token needs is the rule violation the paper allows to prevent
+    waiting, says is rare, and takes - once its share reaches a preset ratio - as the sign that the expansion is too
+    small.  In the nine-layer example (swap = 2 compute): with one CPU layer nearly half of the swap-ins are such
+    prefetches, with two (the paper's choice) under a quarter, and the link is exactly as busy in both - link slack could
+    not tell them apart; with three the computation waits."""
+    n, res = 9, {}
+    for m in (1, 2, 3):
+        res[m] = policy.simulate_protocol(n, 2.0, n - m, m + 2, set(range(n - m + 1, n + 1)), 12)
+    share = {m: r.violations / r.in_starts for m, r in res.items()}
+    assert res[1].stall == res[2].stall == 0 and res[3].stall > 0
+    assert share[1] > 0.4 and 0.15 < share[2] < 0.3 and share[1] > share[2] > share[3]
+    assert res[1].swaps_per_token == res[2].swaps_per_token == 4.5
+    # by hand, token 2 of the paper's trace (two CPU layers): swap-ins of layers 1 (started while layer 8 computes: a
+    # violation), 3, 5, 7, 9 -> one in four and a half
+    ins = [(t, l) for t, kind, l in res[2].events if kind == "in" and 7 <= t < 16]
+    assert ins == [(7.0, 1), (9.0, 3), (11.0, 5), (13.0, 7), (15.0, 9)]
+
+
+@pytest.mark.parametrize("t_swap,want_m", [(2.0, 2), (1.5, 2), (1.0, 5), (3.0, 0)])
+def test_layer_controller_finds_the_papers_two_cpu_layers(t_swap, want_m):
+    """The whole-layer adaptive rule on the protocol simulator, window after window from everything on the GPU: it climbs
+    while the share of next-token prefetches is at or above its trigger, steps back when the computation waits, and comes
+    to rest at two CPU layers for the paper's nine-layer example (expansion 9 / 7 = 1.28, Section 3.3)."""
+    n = 9
+    c = policy.LayerController(m_max=n - 2)
+    traj = []
+    for _ in range(40):
+        m = c.m
+        r = policy.simulate_protocol(n, t_swap, n - m, m + 2, set(range(n - m + 1, n + 1)), 6)
+        c.update(r.stall, 6.0 * n, r.in_starts, r.violations)
+        traj.append(m)
+    assert traj[0] == 0 and traj[-1] == want_m and traj[-20:].count(want_m) >= 18, traj
+    assert max(traj) <= want_m + 1        # at most one probe beyond
+
+
 def test_protocol_sensitivity():
     # one GPU region fewer, or slower swaps: the computation has to wait (Section 3.4.1)
     assert policy.simulate_protocol(9, 2.0, 6, 4, {7, 8, 9}, 6).stall > 0

@@ -14,7 +14,7 @@ import torch
 from paper_2411_09317_b200 import binding as pie
 from paper_2411_09317_b200 import synth
 from tests.gpu_helpers import oracle_attention
-from tests.helpers import Case
+from tests.helpers import Case, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -64,7 +64,7 @@ def test_noalloc_matches_pool_entry_point_on_two_calls_in_a_row():
         assert np.array_equal(a, b)
         want = oracle_attention(case, 0)
         got = synth.bits16_to_f32(b, case.dtype)
-        bound = 2e-3 + (2.0 ** -8 if case.dtype == synth.BF16 else 2.0 ** -11) * np.abs(want)
+        bound = tolerance(want, case.dtype)
         assert np.all(np.abs(got - want) <= bound)
 
 
