@@ -302,6 +302,22 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
                  const int32_t *token_pos_dev, int64_t n_tokens, const int32_t *block_table_dev, int32_t max_blocks_per_seq,
                  int32_t n_seqs);
 
+/* ---- chunked-prefill attention (Section 2.1: the prefill stage computes all prompt tokens at once; Section 2.2: over the
+ * paged cache; the decode call above handles one query token per sequence, this one a chunk) ----------------------
+ * Sequence s contributes the query tokens q_offsets[s] .. q_offsets[s + 1] - 1 of the flat arrays q / out (device
+ * [n_tokens][n_q_heads][head_dim] in the pool's 16-bit type; q_offsets[0] = 0).  Its chunk of C tokens sits at the END of
+ * its context: ctx_lens[s] counts the chunk in, token i of the chunk is position ctx - C + i and attends to positions
+ * 0 .. ctx - C + i (causal inside the chunk, everything before it).  The chunk's own keys and values must be in the cache
+ * already: call pie_kv_write first.  Scores and sums in fp32, probabilities in the 16-bit type, out rounded to nearest.
+ * ctx_lens_host / q_offsets_host (host, required) size the launch and are checked before anything is enqueued: a chunk
+ * longer than its context or a context beyond the table is PIE_ERR_INVALID.  Enqueued on the compute stream behind every
+ * copy still bringing a unit of the layer in; every unit read must be GPU resident (a missing one raises the device
+ * status word: the next call returns PIE_ERR_NOT_RESIDENT).  The kernel runs on the tcgen05 tensor cores with its
+ * accumulators in tensor memory: 128 query rows (128 / group tokens) per CTA.  16-bit pools only (PIE_ERR_UNSUPPORTED). */
+int pie_prefill_attention(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
+                          int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, const int32_t *q_offsets_dev,
+                          const int32_t *ctx_lens_host, const int32_t *q_offsets_host, int32_t n_seqs, float scale);
+
 /* ---- kept host copies and write-back elision (a variant the paper does not have: Section 3.2 gives the
  * CPU region up once a unit has been swapped in) ---------------------------------------------------------
  * on != 0: a unit that is swapped in keeps its host slot; when it is swapped out again it returns to that slot, and

@@ -36,7 +36,7 @@ EXPORTS = [
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_set_violation_trigger", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_kept_copies", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
-    "pie_declare_append_blocks", "pie_kv_write", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
+    "pie_declare_append_blocks", "pie_kv_write", "pie_prefill_attention", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
     "pie_governor_create", "pie_governor_destroy", "pie_governor_report", "pie_governor_state", "pie_report_throughput",
 ]
 
@@ -148,6 +148,7 @@ _sig = {
     "pie_fifo_location": (_i32, [_vp, _i32]),
     "pie_controller_decide": (_f64, [_vp, _f64, _f64, _f64, _f64, _f64]),
     "pie_set_violation_trigger": (_i32, [_vp, _f64]),
+    "pie_prefill_attention": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _i32, _f32]),
     "pie_fifo_counters": (_i32, [_vp, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
     "pie_layer_controller_decide": (_i32, [_vp, _i32, _i32, _f64, _f64, _i64, _i64, _f64, _f64]),
     "pie_decode_attention_noalloc": (_i32, [_vp, _i64, _vp, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
@@ -209,6 +210,14 @@ def pie_pool_destroy(pool) -> None:
 def pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq, n_seqs) -> None:
     check(lib.pie_kv_write(pool, layer, k, v, token_seq_dev, token_pos_dev, n_tokens, block_table_dev, max_blocks_per_seq,
                            n_seqs), "pie_kv_write")
+
+
+def pie_prefill_attention(pool, layer, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, q_offsets_dev, ctx_lens_host,
+                          q_offsets_host, n_seqs, scale) -> None:
+    """q / out / *_dev: device pointers; ctx_lens_host [n_seqs], q_offsets_host [n_seqs + 1]: numpy int32."""
+    ch, qh = _np_i32(ctx_lens_host), _np_i32(q_offsets_host)
+    check(lib.pie_prefill_attention(pool, layer, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, q_offsets_dev, _ptr(ch),
+                                    _ptr(qh), n_seqs, scale), "pie_prefill_attention")
 
 
 def pie_set_violation_trigger(pool, share) -> None:

@@ -12,7 +12,7 @@ FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std
          "--use_fast_math"]
 
 LIBS = {
-    "libpie.so": ["pie_table.cpp", "pie_kernels.cu", "pie_pool.cu", "pie_noalloc.cu"],
+    "libpie.so": ["pie_table.cpp", "pie_kernels.cu", "pie_prefill.cu", "pie_pool.cu", "pie_noalloc.cu"],
     "libpie_synth.so": ["pie_synth.cu"],
 }
 

@@ -99,4 +99,24 @@ cudaError_t make_pool_tensor_map_fp8(void *gpu_pool, int64_t n_gpu_slots, int n_
 cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
                              int use3d, cudaStream_t stream);
 
+// ---- chunked-prefill attention (tcgen05 / TMEM) ----------------------------------------------------------------
+struct PrefillLaunch {
+    const void *q;               // [n_tokens][Hq][D], the chunks of all sequences one after the other
+    void *out;                   // same shape
+    const int32_t *block_table;  // device [n_seqs][max_blocks]
+    int32_t max_blocks;
+    const int32_t *ctx_lens;     // device [n_seqs]: context length including the chunk
+    const int32_t *q_offsets;    // device [n_seqs + 1]: first token of each sequence's chunk
+    const int32_t *tile_off;     // device [n_seqs + 1]: first 128-row tile of each sequence (a tile holds 128 / G tokens)
+    const int32_t *slot_table;   // this layer's row of the device slot table
+    int32_t n_seqs;
+    int32_t n_tiles;             // tile_off[n_seqs]
+    float scale;
+    int32_t *status;
+};
+// the pool's K and V rows as 16-row TMA tiles (box 64 elements x 16 rows, 128-byte swizzle)
+cudaError_t make_prefill_tensor_map(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, int head_dim, CUtensorMap *map);
+cudaError_t prefill_configure(int head_dim, int dtype);
+cudaError_t launch_prefill_attention(const AttnShape &sh, const PrefillLaunch &a, const CUtensorMap &map, cudaStream_t stream);
+
 }  // namespace pie

@@ -132,6 +132,8 @@ struct pie_pool {
     // attention
     pie::AttnScratch scratch{};
     CUtensorMap map3d{}, map2d{};
+    CUtensorMap map_prefill{};   // the pool's K and V rows as 16-row tiles (chunked-prefill attention; 16-bit pools)
+    bool prefill_ready = false;
     int use3d = 0, attn_grid = 0, n_sms = 0;
     // decode-step staging (device copies of host inputs)
     void *stage_q = nullptr, *stage_out = nullptr, *stage_k = nullptr, *stage_v = nullptr;
@@ -1323,6 +1325,7 @@ int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
                 PIE_ERR_CUDA);
         if (const char *env = std::getenv("PIE_TMA_2D"))
             if (env[0] == '1') p->use3d = 0;
+        PIE_TRY(pie::make_prefill_tensor_map(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, cfg->head_dim, &p->map_prefill), PIE_ERR_CUDA);
     }
     int per_sm = 0;
     PIE_TRY(pie::attn_configure(cfg->head_dim, cfg->dtype, cfg->attn_variant, &per_sm, p->kv_fp8), PIE_ERR_CUDA);
@@ -1793,6 +1796,82 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
         return PIE_ERR_CUDA;
     }
     st = record_ticket(pool, PIE_Q_COMPUTE, ticket);
+    if (st != PIE_OK) pool->sticky = st;
+    return st;
+}
+
+int pie_prefill_attention(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
+                          int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, const int32_t *q_offsets_dev,
+                          const int32_t *ctx_lens_host, const int32_t *q_offsets_host, int32_t n_seqs, float scale) {
+    if (!pool || !q || !out || !block_table_dev || !ctx_lens_dev || !q_offsets_dev || !ctx_lens_host || !q_offsets_host)
+        return PIE_ERR_INVALID;
+    if (n_seqs < 0 || max_blocks_per_seq <= 0) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;
+    if (pool->kv_fp8) return PIE_ERR_UNSUPPORTED;
+    if (layer < 0 || layer >= pool->cfg.n_layers) return PIE_ERR_RANGE;
+    int st = poll(pool);
+    if (st != PIE_OK) return st;
+    st = check_status_word(pool);
+    if (st != PIE_OK) return st;
+    if (n_seqs == 0) return PIE_OK;
+    // a chunk is at most its context, which is at most the table; 128 query rows per tile = 128 / G tokens
+    const int32_t G = pool->cfg.n_q_heads / pool->cfg.n_kv_heads, tile_tokens = 128 / G;
+    if (q_offsets_host[0] != 0) return PIE_ERR_INVALID;
+    int64_t n_tiles = 0;
+    for (int32_t s = 0; s < n_seqs; ++s) {
+        const int64_t c = (int64_t)q_offsets_host[s + 1] - q_offsets_host[s];
+        if (c < 0 || ctx_lens_host[s] < 0 || c > ctx_lens_host[s] || ctx_lens_host[s] > max_blocks_per_seq * 16) return PIE_ERR_INVALID;
+        n_tiles += (c + tile_tokens - 1) / tile_tokens;
+    }
+    if (n_tiles * pool->cfg.n_kv_heads > 0x7fffffffll) return PIE_ERR_INVALID;
+    if (n_tiles == 0) return PIE_OK;
+    if (!pool->prefill_ready) {
+        PIE_CUDA(pie::prefill_configure(pool->cfg.head_dim, pool->cfg.dtype));
+        pool->prefill_ready = true;
+    }
+    // like an attention call: a compute ticket, behind every copy that is still bringing a unit of the layer in
+    int64_t ticket = 0, waits[4];
+    st = pool->table->attention(layer, nullptr, 0, &ticket, waits);
+    if (st != PIE_OK) return st;
+    cudaStream_t stream = pool->stream[PIE_Q_COMPUTE];
+    for (int qd = 1; qd <= 2; ++qd) {
+        st = wait_ticket(pool, stream, qd, waits[qd]);
+        if (st != PIE_OK) { pool->sticky = st; return st; }
+    }
+    // the tiles' prefix sums go to the device through the list ring
+    int64_t off = 0;
+    st = list_alloc(pool, n_seqs + 1, &off);
+    if (st != PIE_OK) { pool->sticky = st; return st; }
+    int32_t *h = pool->list_host + off;
+    h[0] = 0;
+    for (int32_t s = 0; s < n_seqs; ++s)
+        h[s + 1] = h[s] + (q_offsets_host[s + 1] - q_offsets_host[s] + tile_tokens - 1) / tile_tokens;
+    cudaError_t e = cudaMemcpyAsync(pool->list_dev + off, h, (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) {
+        pie::AttnShape sh{pool->cfg.head_dim, pool->cfg.dtype, pool->cfg.n_q_heads, pool->cfg.n_kv_heads, pool->cfg.n_logical_blocks,
+                          pool->cfg.n_gpu_slots, 0};
+        pie::PrefillLaunch a{};
+        a.q = q;
+        a.out = out;
+        a.block_table = block_table_dev;
+        a.max_blocks = max_blocks_per_seq;
+        a.ctx_lens = ctx_lens_dev;
+        a.q_offsets = q_offsets_dev;
+        a.tile_off = pool->list_dev + off;
+        a.slot_table = pool->slot_table_dev + (int64_t)layer * pool->cfg.n_logical_blocks;
+        a.n_seqs = n_seqs;
+        a.n_tiles = (int32_t)n_tiles;
+        a.scale = scale;
+        a.status = pool->status_dev;
+        e = pie::launch_prefill_attention(sh, a, pool->map_prefill, stream);
+    }
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        pool->sticky = PIE_ERR_CUDA;
+        return PIE_ERR_CUDA;
+    }
+    st = list_commit(pool, off, n_seqs + 1, stream);
+    if (st == PIE_OK) st = record_ticket(pool, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) pool->sticky = st;
     return st;
 }

@@ -1,0 +1,501 @@
+// Chunked-prefill paged attention (Section 2.1: the prefill stage; Section 2.2: the paged KV cache) on the fifth-
+// generation tensor cores: tcgen05.mma issued by one thread per CTA, operands staged in shared memory by TMA,
+// accumulators in tensor memory (TMEM), read back with tcgen05.ld for the softmax.
+//
+// A chunk of C query tokens of a sequence whose context (chunk included) is ctx tokens long sits at positions
+// ctx - C .. ctx - 1; token i attends to every cached position up to its own.  The chunk's own K and V are in the cache
+// already (pie_kv_write comes first).
+//
+// Work item = (sequence, KV head, tile of 128 query rows).  A row is a (token, query head of the KV head's group) pair,
+// token-major, so a tile holds 128 / G tokens; the rows of a tile share every K and V tile they read, which is what makes
+// this a dense contraction: 128 rows per K and V tile against the decode kernel's G.  Per 64-token stage (four
+// 16-token blocks of the paged pool):
+//   - thread 0 issues the TMA copies of the blocks' K and V rows (two-dimensional tiles of 16 rows x 64 elements,
+//     128-byte swizzle, straight into the layout the tensor core's shared-memory descriptors expect: K as the K-major
+//     B operand of S = Q K^T, V as the MN-major B operand of O += P V), double buffered;
+//   - thread 0 issues D / 16 MMAs of shape 128 x 64 x 16 for S (fp32, 64 TMEM columns) and commits them to an mbarrier;
+//   - the four warps read their 32 rows of S from TMEM (a thread holds one whole row: the softmax needs no shuffles),
+//     apply the causal mask by selection, update the running maximum and sum, write P in the 16-bit type to shared
+//     memory as the next MMA's A operand, and rescale O in TMEM where a row's maximum moved;
+//   - thread 0 issues four MMAs of shape 128 x D x 16 for O += P V (fp32, D TMEM columns).
+// At the end every thread reads its row of O, divides by the row's sum and stores the 16-bit result.
+// Every wait is bounded; a wait that runs out raises the status word, and the CTA still frees its TMEM before it leaves.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <algorithm>
+
+#include "../../include/pie.h"
+#include "pie_kernels.h"
+
+namespace pie {
+
+namespace {
+
+constexpr int PF_M = 128;        // query rows per CTA (the MMA's M)
+constexpr int PF_KV = 64;        // KV tokens per stage
+constexpr int PF_THREADS = 128;  // four warps: warp w owns TMEM lanes 32 w .. 32 w + 31
+constexpr int PF_TMEM_COLS = 256;
+
+__device__ __forceinline__ uint32_t pf_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void pf_raise(int32_t *status, int32_t flag) {
+    *reinterpret_cast<volatile int32_t *>(status + (flag == STATUS_MISSING_UNIT ? 0 : flag == STATUS_CTX_TOO_LONG ? 1 : 2)) = 1;
+}
+__device__ __forceinline__ void pf_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void pf_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool pf_mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded: about a second of polling, then false
+__device__ __forceinline__ bool pf_mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (pf_mbar_try_wait(bar, parity)) return true;
+        if (i > 64) __nanosleep(200);
+    }
+    return false;
+}
+__device__ __forceinline__ void pf_tma_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+
+// ---- tensor memory ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (base lane + i), v[c] = column (base column + c)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+          "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+          "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+          "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+          "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]),
+          "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]),
+          "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// ---- MMA descriptors ---------------------------------------------------------------------------------------------------
+// Shared-memory operand descriptor, 128-byte swizzle: start address, leading-dimension and stride byte offsets in units
+// of 16 bytes, descriptor version 1, layout type 2.  For a K-major operand (rows of 128 bytes along the contraction) the
+// leading offset is not used (1) and the stride offset is the distance between groups of eight rows (1024 bytes); for an
+// MN-major operand the leading offset is the distance between 64-element chunks along MN.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(sbo_bytes >> 4) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, A and B both fp16 or both bf16, A K-major, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(bool bf16, int n, bool b_mn_major) {
+    return (1u << 4) | ((bf16 ? 1u : 0u) << 7) | ((bf16 ? 1u : 0u) << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(PF_M >> 4) << 24);
+}
+__device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ float pf_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+template <bool BF16>
+__device__ __forceinline__ uint32_t pf_pack2(float lo, float hi) {
+    if (BF16) {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&v);
+    } else {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&v);
+    }
+}
+
+struct PrefillParams {
+    const uint16_t *q;
+    uint16_t *out;
+    const int32_t *block_table, *ctx_lens, *q_offsets, *tile_off, *slot_table;
+    int32_t *status;
+    int64_t n_gpu_slots;
+    int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical;
+    float scale_log2e;
+};
+
+template <int D>
+struct PfSmem {
+    static constexpr int Q_BYTES = PF_M * D * 2;        // [D / 64][128 rows][128 B]
+    static constexpr int KV_BYTES = PF_KV * D * 2;      // [D / 64][64 tokens][128 B]
+    static constexpr int P_BYTES = PF_M * PF_KV * 2;    // [128 rows][128 B]
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + Q_BYTES;       // two stages (the next stage's K must be there when an iteration starts)
+    static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;  // one stage (V is needed only after the softmax: it has that long to arrive)
+    static constexpr int OFF_P = OFF_V + KV_BYTES;      // P, and for bf16 the rounding remainder of P as a second operand
+    static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES; // k_full[2], v_full, s_done, o_done
+    static constexpr int OFF_MISC = OFF_BAR + 64;       // [0] TMEM base, [1] abort
+    static constexpr int BYTES = OFF_MISC + 64;         // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
+};
+
+template <int D, bool BF16>
+__global__ void __launch_bounds__(PF_THREADS)
+prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParams p) {
+    using SM = PfSmem<D>;
+    constexpr int HALVES = D / 64;
+    extern __shared__ __align__(1024) uint8_t pf_smem[];
+    uint8_t *smem = pf_smem;
+    const uint32_t base = pf_smem_u32(pf_smem);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (base & 1023u) {   // the swizzled tiles need a 1024-byte boundary: never seen otherwise, but do not compute garbage
+        if (tid == 0) pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+        return;
+    }
+    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 24, bar_o = bar_k + 32;
+    volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + SM::OFF_MISC);
+
+    // ---- which tile
+    const int32_t item = blockIdx.x;
+    const int32_t tile_g = item / p.n_kv_heads, kvh = item - tile_g * p.n_kv_heads;
+    int32_t lo = 0, hi = p.n_seqs;  // largest s with tile_off[s] <= tile_g
+    while (hi - lo > 1) {
+        const int32_t mid = (lo + hi) >> 1;
+        if (__ldg(p.tile_off + mid) <= tile_g) lo = mid;
+        else hi = mid;
+    }
+    const int32_t s = lo;
+    const int32_t G = p.group, tile_tokens = PF_M / G;
+    const int32_t q0 = __ldg(p.q_offsets + s), C = __ldg(p.q_offsets + s + 1) - q0;
+    const int32_t ctx = min(__ldg(p.ctx_lens + s), p.max_blocks * 16);
+    const int32_t tok0 = (tile_g - __ldg(p.tile_off + s)) * tile_tokens;   // first chunk token of the tile
+    const int32_t ntok = min(tile_tokens, C - tok0);
+    const int32_t p0 = ctx - C;                                            // tokens cached before the chunk
+    const int32_t kv_len = p0 + tok0 + ntok;                               // what the tile's last token sees
+    const int32_t n_stages = (kv_len + PF_KV - 1) / PF_KV;
+    const bool bad = C > ctx || ntok <= 0;                                 // (flagged by the host where it has the lengths)
+
+    if (tid == 0) {
+        pf_mbar_init(bar_k, 1);
+        pf_mbar_init(bar_k + 8, 1);
+        pf_mbar_init(bar_v, 1);
+        pf_mbar_init(bar_s, 1);
+        pf_mbar_init(bar_o, 1);
+        misc[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(base + SM::OFF_MISC, PF_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc[0];
+    const uint32_t tmem_s = tmem, tmem_o = tmem + PF_KV;                   // S: columns 0 .. 63, O: 64 .. 64 + D - 1
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+
+    // ---- a stage's K (or V) tiles: one TMA copy per (block, 64-element half)
+    auto issue_tiles = [&](int32_t j, bool v_rows) {
+        const uint32_t bar = v_rows ? bar_v : bar_k + 8 * (uint32_t)(j & 1);
+        const uint32_t dst0 = v_rows ? base + SM::OFF_V : base + SM::OFF_K + (uint32_t)(j & 1) * SM::KV_BYTES;
+        const int32_t b0 = j * (PF_KV / 16);
+        const int32_t nb = min(PF_KV / 16, (kv_len + 15) / 16 - b0);
+        pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
+        for (int32_t i = 0; i < nb; ++i) {
+            const int32_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + b0 + i);
+            int32_t slot = (blk >= 0 && blk < p.n_logical) ? __ldcg(p.slot_table + blk) : -1;
+            if (slot < 0 || slot >= p.n_gpu_slots) {  // unit not on the GPU: flag it, stream slot 0 so the barrier completes
+                pf_raise(p.status, STATUS_MISSING_UNIT);
+                slot = 0;
+            }
+            const int32_t row0 = (slot * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
+#pragma unroll
+            for (int h = 0; h < HALVES; ++h) pf_tma_2d(dst0 + h * (PF_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
+        }
+    };
+    if (tid == 0 && !bad && n_stages > 0) {
+        issue_tiles(0, false);
+        issue_tiles(0, true);
+    }
+
+    // ---- Q: thread r brings row r (token tok0 + r / G, head kvh * G + r % G) into the K-major swizzled layout
+    const int r = tid;
+    const int32_t my_tok = r / G, my_g = r - my_tok * G;
+    const bool row_valid = !bad && my_tok < ntok;
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+            const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4 *>(smem + SM::OFF_Q + (c >> 3) * (PF_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int32_t my_pos = p0 + tok0 + my_tok;   // this row's position: it sees tokens 0 .. my_pos
+    float m_run = -INFINITY, l_run = 0.f;
+    constexpr uint32_t IDESC_S = instr_desc(BF16, PF_KV, false), IDESC_O = instr_desc(BF16, D, true);
+    bool ok = !bad;
+
+    for (int32_t j = 0; ok && j < n_stages; ++j) {
+        const uint32_t buf = (uint32_t)(j & 1);
+        // the next stage's K goes into the other buffer (stage j - 1's MMAs have been waited for); this stage's K has landed?
+        if (tid == 0 && j + 1 < n_stages) issue_tiles(j + 1, false);
+        if (!pf_mbar_wait(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1))) {
+            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+            misc[1] = 1;
+        }
+        tc_fence_before();
+        __syncthreads();
+        if (misc[1]) { ok = false; break; }
+        // ---- S = Q K^T
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const uint64_t a = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
+                const uint64_t b = smem_desc(base + SM::OFF_K + buf * SM::KV_BYTES + (ks >> 2) * (PF_KV * 128) + (ks & 3) * 32, 16, 1024);
+                mma_f16(tmem_s, a, b, IDESC_S, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(bar_s);
+        }
+        if (!pf_mbar_wait(bar_s, (uint32_t)(j & 1))) {
+            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+            misc[1] = 1;
+        }
+        tc_fence_after();
+        // ---- softmax of this thread's row over the stage's 64 tokens
+        uint32_t sv[2][32];
+        tmem_ld32(tmem_s + lane_addr, sv[0]);
+        tmem_ld32(tmem_s + lane_addr + 32, sv[1]);
+        tmem_wait_ld();
+        const int32_t t_base = j * PF_KV;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                float x = __uint_as_float(sv[h][c]) * p.scale_log2e;
+                x = (row_valid && t_base + h * 32 + c <= my_pos) ? x : -INFINITY;   // masked by selection (NaN scores too)
+                sv[h][c] = __float_as_uint(x);
+                mx = fmaxf(mx, x);
+            }
+        const float m_new = fmaxf(m_run, mx);
+        const float alpha = m_new == -INFINITY ? 1.f : pf_exp2(m_run - m_new);   // (m_run = -inf gives 0: nothing accumulated yet)
+        float sum = 0.f;
+        {
+            uint8_t *prow = smem + SM::OFF_P + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {   // eight tokens per 16-byte piece
+                uint32_t w[4];
+                [[maybe_unused]] uint32_t w2[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int c = cc * 8 + e * 2;
+                    const float x0 = __uint_as_float(sv[c >> 5][c & 31]), x1 = __uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]);
+                    const float e0 = m_new == -INFINITY ? 0.f : pf_exp2(x0 - m_new), e1 = m_new == -INFINITY ? 0.f : pf_exp2(x1 - m_new);
+                    w[e] = pf_pack2<BF16>(e0, e1);
+                    // the sum runs over what the tensor core will see: the rounded probabilities
+                    if (BF16) {
+                        // bf16 keeps 8 significant bits: the rounding remainder of P goes into a second bf16 operand, so
+                        // that the P V product sees about 16 bits (fp16's 11 bits need no correction)
+                        const float h0 = __uint_as_float(w[e] << 16), h1 = __uint_as_float(w[e] & 0xffff0000u);
+                        w2[e] = pf_pack2<true>(e0 - h0, e1 - h1);
+                        sum += (h0 + __uint_as_float(w2[e] << 16)) + (h1 + __uint_as_float(w2[e] & 0xffff0000u));
+                    } else {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[e]));
+                        sum += f.x + f.y;
+                    }
+                }
+                *reinterpret_cast<uint4 *>(prow + ((cc ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                if (BF16) *reinterpret_cast<uint4 *>(prow + SM::P_BYTES + ((cc ^ (r & 7)) << 4)) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+            }
+        }
+        l_run = l_run * alpha + sum;
+        m_run = m_new;
+        // this stage's V has landed?  Rows of V beyond what the tile may see hold whatever was there (a tail block's
+        // garbage, an earlier stage): masked tokens are excluded, not multiplied by zero, so clear them before they meet P = 0
+        if (!pf_mbar_wait(bar_v, (uint32_t)(j & 1))) {
+            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+            misc[1] = 1;
+        }
+        const int32_t n_seen = min(PF_KV, kv_len - j * PF_KV);
+        if (n_seen < PF_KV) {
+            for (int e = tid; e < (PF_KV - n_seen) * HALVES * 8; e += PF_THREADS) {
+                const int row = n_seen + e / (HALVES * 8), rem = e % (HALVES * 8);
+                *reinterpret_cast<uint4 *>(smem + SM::OFF_V + (rem >> 3) * (PF_KV * 128) + row * 128 + ((rem & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // ---- O *= alpha where a row's maximum moved (skipped by warps in which none did)
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t ov[32];
+                tmem_ld32(tmem_o + lane_addr + c0, ov);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+                tmem_st32(tmem_o + lane_addr + c0, ov);
+            }
+            tmem_wait_st();
+        }
+        tc_fence_before();
+        __syncthreads();
+        if (misc[1]) { ok = false; break; }
+        // ---- O += P V
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < PF_KV / 16; ++ks) {
+                const uint64_t a = smem_desc(base + SM::OFF_P + ks * 32, 16, 1024);
+                // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
+                const uint64_t b = smem_desc(base + SM::OFF_V + ks * 2048, PF_KV * 128, 1024);
+                mma_f16(tmem_o, a, b, IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
+                if (BF16) mma_f16(tmem_o, smem_desc(base + SM::OFF_P + SM::P_BYTES + ks * 32, 16, 1024), b, IDESC_O, 1u);
+            }
+            tc_commit(bar_o);
+        }
+        if (!pf_mbar_wait(bar_o, (uint32_t)(j & 1))) {
+            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+            misc[1] = 1;
+        }
+        tc_fence_after();
+        if (tid == 0 && j + 1 < n_stages && misc[1] == 0) issue_tiles(j + 1, true);   // V's buffer is free again
+    }
+
+    // ---- out = O / l, rounded to the 16-bit type (nearest even).  The TMEM loads are warp-wide: rows beyond the chunk
+    // take part in them and store nothing.
+    if (ok && n_stages > 0) {
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t ov[32];
+            tmem_ld32(tmem_o + lane_addr + c0, ov);
+            tmem_wait_ld();
+            if (row_valid) {
+#pragma unroll
+                for (int c = 0; c < 32; c += 8) {
+                    uint4 v;
+                    v.x = pf_pack2<BF16>(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                    v.y = pf_pack2<BF16>(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                    v.z = pf_pack2<BF16>(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                    v.w = pf_pack2<BF16>(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                    dst[(c0 + c) >> 3] = v;
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, PF_TMEM_COLS);
+}
+
+}  // namespace
+
+int prefill_smem_bytes(int head_dim) { return head_dim == 128 ? PfSmem<128>::BYTES : PfSmem<64>::BYTES; }
+
+// K and V rows of the pool as 16-row tiles: rows of head_dim elements, 32 per (slot, KV head): 16 of K, 16 of V.
+cudaError_t make_prefill_tensor_map(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, int head_dim, CUtensorMap *map) {
+    typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                      const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)n_gpu_slots * (cuuint64_t)n_kv_heads * 32u};
+    cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
+    cuuint32_t box[2] = {64, 16};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, gpu_pool, dims, strides, box, estr,
+                                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t prefill_configure(int head_dim, int dtype) {
+    const int smem = prefill_smem_bytes(head_dim);
+    const void *k = head_dim == 128 ? (dtype == PIE_BF16 ? (const void *)prefill_attn_kernel<128, true> : (const void *)prefill_attn_kernel<128, false>)
+                                    : (dtype == PIE_BF16 ? (const void *)prefill_attn_kernel<64, true> : (const void *)prefill_attn_kernel<64, false>);
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+}
+
+cudaError_t launch_prefill_attention(const AttnShape &sh, const PrefillLaunch &a, const CUtensorMap &map, cudaStream_t stream) {
+    if (a.n_tiles <= 0) return cudaSuccess;
+    PrefillParams p;
+    p.q = (const uint16_t *)a.q;
+    p.out = (uint16_t *)a.out;
+    p.block_table = a.block_table;
+    p.ctx_lens = a.ctx_lens;
+    p.q_offsets = a.q_offsets;
+    p.tile_off = a.tile_off;
+    p.slot_table = a.slot_table;
+    p.status = a.status;
+    p.n_gpu_slots = sh.n_gpu_slots;
+    p.max_blocks = a.max_blocks;
+    p.n_seqs = a.n_seqs;
+    p.n_q_heads = sh.n_q_heads;
+    p.n_kv_heads = sh.n_kv_heads;
+    p.group = sh.n_q_heads / sh.n_kv_heads;
+    p.n_logical = sh.n_logical;
+    p.scale_log2e = a.scale * 1.4426950408889634f;
+    const unsigned grid = (unsigned)((int64_t)a.n_tiles * sh.n_kv_heads);
+    const int smem = prefill_smem_bytes(sh.head_dim);
+    if (sh.head_dim == 128) {
+        if (sh.dtype == PIE_BF16) prefill_attn_kernel<128, true><<<grid, PF_THREADS, smem, stream>>>(map, p);
+        else prefill_attn_kernel<128, false><<<grid, PF_THREADS, smem, stream>>>(map, p);
+    } else {
+        if (sh.dtype == PIE_BF16) prefill_attn_kernel<64, true><<<grid, PF_THREADS, smem, stream>>>(map, p);
+        else prefill_attn_kernel<64, false><<<grid, PF_THREADS, smem, stream>>>(map, p);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace pie

@@ -1,0 +1,117 @@
+"""Chunked-prefill paged attention (tcgen05 / TMEM kernel) against the prefill oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import prefill
+from paper_2411_09317_b200 import binding as pie
+from paper_2411_09317_b200 import synth
+from tests.gpu_helpers import PoolCase
+from tests.helpers import Case, tolerance
+
+pytestmark = pytest.mark.gpu
+F16, BF16 = synth.F16, synth.BF16
+
+
+def run_prefill(case, pc, layer, chunk_lens, seed=9, ctx_lens=None):
+    """-> (got fp32 [n_tokens][Hq][D], want fp64) for chunks of the given lengths at the end of each context"""
+    ctx = np.asarray(case.ctx_lens if ctx_lens is None else ctx_lens, dtype=np.int32)
+    off = np.concatenate([[0], np.cumsum(chunk_lens)]).astype(np.int32)
+    n_tok = int(off[-1])
+    q = synth.tensor_bits(seed, synth.STREAM_Q, (n_tok, case.Hq, case.D), case.dtype)
+    dev = torch.device("cuda:0")
+    q_dev = torch.from_numpy(q.view(np.int16)).to(dev)
+    out_dev = torch.full_like(q_dev, 0x7e00 if case.dtype == F16 else 0x7fc0)     # NaN: every valid row must be written
+    off_dev = torch.from_numpy(off).to(dev)
+    ctx_dev = torch.from_numpy(ctx).to(dev)
+    pie.pie_prefill_attention(pc.pool, layer, q_dev.data_ptr(), out_dev.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                              ctx_dev.data_ptr(), off_dev.data_ptr(), ctx, off, len(ctx), case.scale)
+    pie.pie_sync(pc.pool)
+    got = synth.bits16_to_f32(out_dev.cpu().numpy().view(np.uint16), case.dtype)
+    want = prefill.prefill_attention(case.gpu_pool, case.host_pool, case.unit_side[layer], case.unit_slot[layer], q, off, case.block_table,
+                                     ctx, case.Hq, case.Hkv, case.D, case.dtype, case.scale)
+    return got, want
+
+
+def check(case, pc, layer, chunk_lens, **kw):
+    got, want = run_prefill(case, pc, layer, chunk_lens, **kw)
+    err = np.abs(got - want)
+    assert np.all(np.isfinite(got))
+    assert np.all(err <= tolerance(want, case.dtype)), float(err.max())
+    return float(err.max())
+
+
+def test_one_full_prompt_of_one_tile():
+    """The smallest case: one sequence, one KV head, 64 tokens fed as one chunk (one stage, one tile)."""
+    case = Case(1, 1, 1, 128, F16, [64], seed=61, host_frac=0.0, placement="identity")
+    pc = PoolCase(case, all_on_gpu=True)
+    check(case, pc, 0, [64])
+    pc.close()
+
+
+@pytest.mark.parametrize("hq,hkv,d,dtype", [(4, 4, 128, F16), (8, 2, 128, BF16), (8, 1, 128, F16), (4, 2, 64, BF16), (2, 2, 64, F16)])
+@pytest.mark.parametrize("chunk", [16, 64, 256])
+def test_chunks_after_ragged_prefixes(hq, hkv, d, dtype, chunk):
+    """Chunks of one length behind prefixes of every kind: none, shorter than a block, not a multiple of anything, several
+    stages long; group sizes 1, 2, 4 and 8, both types, both head sizes; scattered slots."""
+    prefixes = [0, 5, 100, 333, 16, 1000]
+    ctx = [p + chunk for p in prefixes]
+    case = Case(2, hq, hkv, d, dtype, ctx, seed=62, host_frac=0.0, placement="random")
+    pc = PoolCase(case, all_on_gpu=True)
+    check(case, pc, 1, [chunk] * len(prefixes))
+    pc.close()
+
+
+def test_ragged_chunk_lengths_in_one_call():
+    """Chunks of 1 to 1024 tokens in one batch (tiles with a single valid row, tiles that end mid-way, an empty chunk)."""
+    chunks = [1, 1024, 0, 37, 130, 64, 257]
+    prefixes = [50, 0, 200, 0, 7, 1, 700]
+    ctx = [p + c for p, c in zip(prefixes, chunks)]
+    case = Case(1, 8, 2, 128, BF16, ctx, seed=63, host_frac=0.0, placement="reversed")
+    pc = PoolCase(case, all_on_gpu=True)
+    check(case, pc, 0, chunks)
+    pc.close()
+
+
+def test_tail_garbage_and_future_tokens_do_not_leak():
+    """Causality and the tail rule on the device: NaN and Inf patterns in the cache beyond a chunk's last position (the
+    rest of its last block, and whole blocks of tokens that come later) change nothing."""
+    case = Case(1, 4, 2, 128, F16, [300, 90], seed=64, host_frac=0.0, placement="identity")
+    chunks = [100, 40]
+    clean = Case(1, 4, 2, 128, F16, [300, 90], seed=64, host_frac=0.0, placement="identity")
+    # the chunks end at positions 199 and 59: poison everything after them
+    for s, last in ((0, 199), (1, 59)):
+        for pos in range(last + 1, int(case.ctx_lens[s])):
+            tile = case.gpu_pool[case.unit_slot[0, case.block_table[s, pos // 16]]].reshape(2, 2, 16, 128)
+            tile[:, :, pos % 16, :] = np.array([0x7e00, 0x7c00, 0xfc00, 0x7bff], dtype=np.uint16)[pos % 4]
+    pc, pc_clean = PoolCase(case, all_on_gpu=True), PoolCase(clean, all_on_gpu=True)
+    ctx_now = np.array([200, 60], dtype=np.int32)
+    got, want = run_prefill(case, pc, 0, chunks, ctx_lens=ctx_now)
+    got_clean, _ = run_prefill(clean, pc_clean, 0, chunks, ctx_lens=ctx_now)
+    assert np.array_equal(got, got_clean)
+    assert np.all(np.abs(got - want) <= tolerance(want, F16))
+    pc.close()
+    pc_clean.close()
+
+
+def test_rejected_arguments_enqueue_nothing():
+    case = Case(1, 4, 2, 128, F16, [64, 64], seed=65, host_frac=0.0, placement="identity")
+    pc = PoolCase(case, all_on_gpu=True)
+    dev = torch.device("cuda:0")
+    q = torch.zeros((80, 4, 128), dtype=torch.int16, device=dev)
+    out = torch.zeros_like(q)
+    ctx = np.array([64, 64], np.int32)
+    ctx_dev = torch.from_numpy(ctx).to(dev)
+    for off in ([0, 70, 80], [1, 40, 80], [0, 40, 30]):               # chunk longer than its context; first offset; decreasing
+        off = np.array(off, np.int32)
+        with pytest.raises(pie.PieError) as e:
+            pie.pie_prefill_attention(pc.pool, 0, q.data_ptr(), out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                                      ctx_dev.data_ptr(), torch.from_numpy(off).to(dev).data_ptr(), ctx, off, 2, case.scale)
+        assert e.value.status == pie.PIE_ERR_INVALID
+    too_long = np.array([16 * case.block_table.shape[1] + 1, 64], np.int32)
+    with pytest.raises(pie.PieError):
+        pie.pie_prefill_attention(pc.pool, 0, q.data_ptr(), out.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                                  ctx_dev.data_ptr(), ctx_dev.data_ptr(), too_long, np.array([0, 40, 80], np.int32), 2, case.scale)
+    pie.pie_sync(pc.pool)
+    assert int(out.abs().sum()) == 0
+    pc.close()
