@@ -34,8 +34,14 @@ namespace {
 
 constexpr int PF_M = 128;        // query rows per CTA (the MMA's M)
 constexpr int PF_KV = 64;        // KV tokens per stage
-constexpr int PF_THREADS = 128;  // four warps: warp w owns TMEM lanes 32 w .. 32 w + 31
+constexpr int PF_ROWS_THREADS = 128;  // four softmax warps: warp w owns TMEM lanes 32 w .. 32 w + 31 (one thread per query row)
+constexpr int PF_THREADS = 160;       // + one warp that only issues: TMA copies, MMAs, block-table look-ups
 constexpr int PF_TMEM_COLS = 256;
+// The running maximum of a row is only raised - and the row's O and sum rescaled, a round trip through tensor memory for
+// the whole warp - when the stage's maximum exceeds it by more than this (in log2 units): until then the probabilities
+// are taken against the older maximum and may reach 2^8, which fp32 sums and both 16-bit types hold without loss.  With
+// an exact running maximum some row of a warp moves its maximum in most stages, even hundreds of stages in.
+constexpr float PF_LAZY = 8.f;
 
 __device__ __forceinline__ uint32_t pf_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -44,6 +50,9 @@ __device__ __forceinline__ void pf_raise(int32_t *status, int32_t flag) {
 }
 __device__ __forceinline__ void pf_mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void pf_mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void pf_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -141,6 +150,16 @@ __device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t a_desc, uint64
         : "memory");
 }
 
+// the same with the A operand in tensor memory (row r in lane r, two 16-bit elements of the contraction per 32-bit column)
+__device__ __forceinline__ void mma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 __device__ __forceinline__ float pf_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -171,14 +190,12 @@ template <int D>
 struct PfSmem {
     static constexpr int Q_BYTES = PF_M * D * 2;        // [D / 64][128 rows][128 B]
     static constexpr int KV_BYTES = PF_KV * D * 2;      // [D / 64][64 tokens][128 B]
-    static constexpr int P_BYTES = PF_M * PF_KV * 2;    // [128 rows][128 B]
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = OFF_Q + Q_BYTES;       // two stages (the next stage's K must be there when an iteration starts)
-    static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;  // one stage (V is needed only after the softmax: it has that long to arrive)
-    static constexpr int OFF_P = OFF_V + KV_BYTES;      // P, and for bf16 the rounding remainder of P as a second operand
-    static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES; // k_full[2], v_full, s_done, o_done
-    static constexpr int OFF_MISC = OFF_BAR + 64;       // [0] TMEM base, [1] abort
-    static constexpr int BYTES = OFF_MISC + 64;         // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
+    static constexpr int OFF_K = OFF_Q + Q_BYTES;       // two stages
+    static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;  // two stages
+    static constexpr int OFF_BAR = OFF_V + 2 * KV_BYTES; // k_full[2], v_full[2], s_done[2], o_done
+    static constexpr int OFF_MISC = OFF_BAR + 64;       // [0] TMEM base, [1] abort, [4 .. 19] slots of the stages in flight
+    static constexpr int BYTES = OFF_MISC + 128;        // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
 };
 
 template <int D, bool BF16>
@@ -189,12 +206,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
     extern __shared__ __align__(1024) uint8_t pf_smem[];
     uint8_t *smem = pf_smem;
     const uint32_t base = pf_smem_u32(pf_smem);
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (base & 1023u) {   // the swizzled tiles need a 1024-byte boundary: never seen otherwise, but do not compute garbage
         if (tid == 0) pf_raise(p.status, STATUS_WAIT_TIMEOUT);
         return;
     }
-    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 24, bar_o = bar_k + 32;
+    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 32, bar_o = bar_k + 48, bar_p = bar_k + 56;
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + SM::OFF_MISC);
 
     // ---- which tile
@@ -214,56 +231,47 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
     const int32_t ntok = min(tile_tokens, C - tok0);
     const int32_t p0 = ctx - C;                                            // tokens cached before the chunk
     const int32_t kv_len = p0 + tok0 + ntok;                               // what the tile's last token sees
-    const int32_t n_stages = (kv_len + PF_KV - 1) / PF_KV;
     const bool bad = C > ctx || ntok <= 0;                                 // (flagged by the host where it has the lengths)
+    const int32_t n_stages = bad ? 0 : (kv_len + PF_KV - 1) / PF_KV;
 
     if (tid == 0) {
-        pf_mbar_init(bar_k, 1);
-        pf_mbar_init(bar_k + 8, 1);
-        pf_mbar_init(bar_v, 1);
-        pf_mbar_init(bar_s, 1);
-        pf_mbar_init(bar_o, 1);
+        for (int i = 0; i < 7; ++i) pf_mbar_init(bar_k + 8 * i, 1);   // k_full[2], v_full[2], s_done[2], o_done
+        pf_mbar_init(bar_p, PF_ROWS_THREADS);                          // P of a stage is in place: every row's thread arrives
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 0) tmem_alloc(base + SM::OFF_MISC, PF_TMEM_COLS);
+    if (warp == 4) tmem_alloc(base + SM::OFF_MISC, PF_TMEM_COLS);
+    // ---- block table -> slot table -> slot, off the issuing thread's path: four of its warp's other lanes resolve the
+    // blocks of a stage three stages ahead into a small ring in shared memory (two dependent global loads each; done
+    // serially by the issuing thread they cost ten microseconds per stage)
+    volatile int32_t *slot_ring = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_MISC + 16);   // [4 stages][4 blocks]
+    auto resolve = [&](int32_t j, int32_t i) {
+        const int32_t b = j * (PF_KV / 16) + i;
+        int32_t slot = -1;
+        if (b < (kv_len + 15) / 16) {
+            const int32_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + b);
+            slot = (blk >= 0 && blk < p.n_logical) ? __ldcg(p.slot_table + blk) : -1;
+            if (slot < 0 || slot >= p.n_gpu_slots) {  // unit not on the GPU: flag it, stream slot 0 so the barriers complete
+                pf_raise(p.status, STATUS_MISSING_UNIT);
+                slot = 0;
+            }
+        }
+        slot_ring[(j & 3) * 4 + i] = slot;
+    };
+    if (warp == 4 && lane >= 4 && lane < 16 && ((lane - 4) >> 2) < n_stages) resolve((lane - 4) >> 2, (lane - 4) & 3);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = misc[0];
-    const uint32_t tmem_s = tmem, tmem_o = tmem + PF_KV;                   // S: columns 0 .. 63, O: 64 .. 64 + D - 1
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-
-    // ---- a stage's K (or V) tiles: one TMA copy per (block, 64-element half)
-    auto issue_tiles = [&](int32_t j, bool v_rows) {
-        const uint32_t bar = v_rows ? bar_v : bar_k + 8 * (uint32_t)(j & 1);
-        const uint32_t dst0 = v_rows ? base + SM::OFF_V : base + SM::OFF_K + (uint32_t)(j & 1) * SM::KV_BYTES;
-        const int32_t b0 = j * (PF_KV / 16);
-        const int32_t nb = min(PF_KV / 16, (kv_len + 15) / 16 - b0);
-        pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
-        for (int32_t i = 0; i < nb; ++i) {
-            const int32_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + b0 + i);
-            int32_t slot = (blk >= 0 && blk < p.n_logical) ? __ldcg(p.slot_table + blk) : -1;
-            if (slot < 0 || slot >= p.n_gpu_slots) {  // unit not on the GPU: flag it, stream slot 0 so the barrier completes
-                pf_raise(p.status, STATUS_MISSING_UNIT);
-                slot = 0;
-            }
-            const int32_t row0 = (slot * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
-#pragma unroll
-            for (int h = 0; h < HALVES; ++h) pf_tma_2d(dst0 + h * (PF_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
-        }
-    };
-    if (tid == 0 && !bad && n_stages > 0) {
-        issue_tiles(0, false);
-        issue_tiles(0, true);
-    }
+    const uint32_t tmem_o = tmem + 2 * PF_KV;   // S (and then P) of even stages: columns 0 .. 63, of odd stages: 64 .. 127; O: 128 .. 128 + D - 1
+    constexpr uint32_t IDESC_S = instr_desc(BF16, PF_KV, false), IDESC_O = instr_desc(BF16, D, true);
 
     // ---- Q: thread r brings row r (token tok0 + r / G, head kvh * G + r % G) into the K-major swizzled layout
     const int r = tid;
     const int32_t my_tok = r / G, my_g = r - my_tok * G;
-    const bool row_valid = !bad && my_tok < ntok;
-    {
+    const bool row_valid = !bad && tid < PF_ROWS_THREADS && my_tok < ntok;
+    if (tid < PF_ROWS_THREADS) {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
 #pragma unroll
         for (int c = 0; c < D / 8; ++c) {
@@ -272,166 +280,257 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    __syncthreads();
 
-    const int32_t my_pos = p0 + tok0 + my_tok;   // this row's position: it sees tokens 0 .. my_pos
-    float m_run = -INFINITY, l_run = 0.f;
-    constexpr uint32_t IDESC_S = instr_desc(BF16, PF_KV, false), IDESC_O = instr_desc(BF16, D, true);
-    bool ok = !bad;
-
-    for (int32_t j = 0; ok && j < n_stages; ++j) {
-        const uint32_t buf = (uint32_t)(j & 1);
-        // the next stage's K goes into the other buffer (stage j - 1's MMAs have been waited for); this stage's K has landed?
-        if (tid == 0 && j + 1 < n_stages) issue_tiles(j + 1, false);
-        if (!pf_mbar_wait(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1))) {
-            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-            misc[1] = 1;
-        }
-        tc_fence_before();
-        __syncthreads();
-        if (misc[1]) { ok = false; break; }
-        // ---- S = Q K^T
-        if (tid == 0) {
+    if (warp == 4) {
+        // =============================================================================== the issuing warp
+        // a stage's K (or V) tiles: one TMA copy per (block, 64-element half)
+        auto issue_tiles = [&](int32_t j, bool v_rows) {
+            const uint32_t buf = (uint32_t)(j & 1);
+            const uint32_t bar = (v_rows ? bar_v : bar_k) + 8 * buf;
+            const uint32_t dst0 = base + (v_rows ? SM::OFF_V : SM::OFF_K) + buf * SM::KV_BYTES;
+            const int32_t nb = min(PF_KV / 16, (kv_len + 15) / 16 - j * (PF_KV / 16));
+            pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
+            for (int32_t i = 0; i < nb; ++i) {
+                const int32_t row0 = (slot_ring[(j & 3) * 4 + i] * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
+#pragma unroll
+                for (int h = 0; h < HALVES; ++h) pf_tma_2d(dst0 + h * (PF_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
+            }
+        };
+        // S(j) = Q K(j)^T into the stage's half of the score columns (K(j) must have landed)
+        auto issue_qk = [&](int32_t j) {
+            const uint32_t buf = (uint32_t)(j & 1);
+            if (!pf_mbar_wait(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1))) {
+                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                misc[1] = 1;
+                return;
+            }
             tc_fence_after();
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 const uint64_t a = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
                 const uint64_t b = smem_desc(base + SM::OFF_K + buf * SM::KV_BYTES + (ks >> 2) * (PF_KV * 128) + (ks & 3) * 32, 16, 1024);
-                mma_f16(tmem_s, a, b, IDESC_S, ks > 0 ? 1u : 0u);
+                mma_f16(tmem + buf * PF_KV, a, b, IDESC_S, ks > 0 ? 1u : 0u);
             }
-            tc_commit(bar_s);
-        }
-        if (!pf_mbar_wait(bar_s, (uint32_t)(j & 1))) {
-            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-            misc[1] = 1;
-        }
-        tc_fence_after();
-        // ---- softmax of this thread's row over the stage's 64 tokens
-        uint32_t sv[2][32];
-        tmem_ld32(tmem_s + lane_addr, sv[0]);
-        tmem_ld32(tmem_s + lane_addr + 32, sv[1]);
-        tmem_wait_ld();
-        const int32_t t_base = j * PF_KV;
-        float mx = -INFINITY;
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                float x = __uint_as_float(sv[h][c]) * p.scale_log2e;
-                x = (row_valid && t_base + h * 32 + c <= my_pos) ? x : -INFINITY;   // masked by selection (NaN scores too)
-                sv[h][c] = __float_as_uint(x);
-                mx = fmaxf(mx, x);
+            tc_commit(bar_s + 8 * buf);
+        };
+        if (lane == 0)
+            for (int32_t j = 0; j < min(n_stages, 2); ++j) {
+                issue_tiles(j, false);
+                issue_tiles(j, true);
             }
-        const float m_new = fmaxf(m_run, mx);
-        const float alpha = m_new == -INFINITY ? 1.f : pf_exp2(m_run - m_new);   // (m_run = -inf gives 0: nothing accumulated yet)
-        float sum = 0.f;
-        {
-            uint8_t *prow = smem + SM::OFF_P + (r >> 3) * 1024 + (r & 7) * 128;
+        __syncthreads();   // Q is in shared memory
+        if (lane == 0 && n_stages > 0) issue_qk(0);
+        // Software pipeline: while the four softmax warps work on the scores of stage j, the tensor core computes those of
+        // stage j + 1 (into the other half of the score columns) and, before that, finishes O += P V of stage j - 1.
+        for (int32_t j = 0; j < n_stages; ++j) {
+            if (lane >= 4 && lane < 8 && j + 3 < n_stages) resolve(j + 3, lane - 4);   // read from the next iteration on
+            __syncwarp();
+            if (lane == 0 && misc[1] == 0) {
+                const uint32_t buf = (uint32_t)(j & 1);
+                // the other half of the score columns held P(j - 1), and stage j - 1's V buffer is the one stage j + 1
+                // needs: O += P V of stage j - 1 must have completed
+                if (j >= 1 && !pf_mbar_wait(bar_o, (uint32_t)((j - 1) & 1))) {
+                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                    misc[1] = 1;
+                }
+                if (misc[1] == 0 && j + 1 < n_stages) {
+                    if (j >= 1) issue_tiles(j + 1, true);
+                    issue_qk(j + 1);
+                }
+                // P(j) is in tensor memory (every row's thread has arrived): O += P V, then the K tiles of stage j + 2 into
+                // the buffer that S(j) no longer needs
+                if (misc[1] == 0 && !pf_mbar_wait(bar_p, (uint32_t)(j & 1))) {
+                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                    misc[1] = 1;
+                }
+                if (misc[1] == 0 && !pf_mbar_wait(bar_v + 8 * buf, (uint32_t)((j >> 1) & 1))) {   // V(j) has landed
+                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                    misc[1] = 1;
+                }
+                if (misc[1] == 0) {
+                    tc_fence_after();
+                    const uint32_t tmem_sj = tmem + buf * PF_KV;
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {   // eight tokens per 16-byte piece
-                uint32_t w[4];
-                [[maybe_unused]] uint32_t w2[4];
+                    for (int ks = 0; ks < PF_KV / 16; ++ks) {
+                        // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
+                        const uint64_t b = smem_desc(base + SM::OFF_V + buf * SM::KV_BYTES + ks * 2048, PF_KV * 128, 1024);
+                        mma_f16_ts(tmem_o, tmem_sj + ks * 8, b, IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
+                        if (BF16) mma_f16_ts(tmem_o, tmem_sj + 32 + ks * 8, b, IDESC_O, 1u);
+                    }
+                    tc_commit(bar_o);
+                    if (j + 2 < n_stages) issue_tiles(j + 2, false);
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // =============================================================================== the softmax warps
+        __syncthreads();   // Q is in shared memory
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const int32_t my_pos = p0 + tok0 + my_tok;   // this row's position: it sees tokens 0 .. my_pos
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int32_t j = 0; j < n_stages; ++j) {
+            const uint32_t buf = (uint32_t)(j & 1);
+            const uint32_t tmem_sj = tmem + buf * PF_KV;
+            // ---- the scores of stage j
+            if (!pf_mbar_wait(bar_s + 8 * buf, (uint32_t)((j >> 1) & 1))) {
+                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                misc[1] = 1;
+            }
+            if (__any_sync(0xffffffffu, misc[1] != 0)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t sv[2][32];
+            tmem_ld32(tmem_sj + lane_addr, sv[0]);
+            tmem_ld32(tmem_sj + lane_addr + 32, sv[1]);
+            tmem_wait_ld();
+            const int32_t t_base = j * PF_KV;
+            float m_new, alpha, sum;
+            uint32_t ph[32];
+            [[maybe_unused]] uint32_t pl[32];
+            // P in the 16-bit type, two tokens per 32-bit word: the A operand of O += P V, kept in tensor memory where the
+            // scores were.  bf16 keeps 8 significant bits: the rounding remainder of P goes into a second bf16 operand, so
+            // that the product sees about 16 bits (fp16's 11 bits need no correction).
+            if (t_base + PF_KV - 1 <= p0 + tok0 && p.scale_log2e > 0.f) {
+                // Every row of the tile sees every token of the stage (all stages but the last one or two of a tile): no
+                // mask, and the softmax is what bounds this kernel - 64 exponentials per row and stage on four warps - so it
+                // is written for the instruction count: the maximum over the raw scores (four chains), one fused
+                // multiply-add and one ex2 per element, sums in four chains over the unrounded probabilities (they differ from
+                // what the tensor core sees by the operand's rounding, 2^-12 or 2^-17 relative: nothing beside 2e-3).
+                float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = cc * 8 + e * 2;
-                    const float x0 = __uint_as_float(sv[c >> 5][c & 31]), x1 = __uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]);
-                    const float e0 = m_new == -INFINITY ? 0.f : pf_exp2(x0 - m_new), e1 = m_new == -INFINITY ? 0.f : pf_exp2(x1 - m_new);
-                    w[e] = pf_pack2<BF16>(e0, e1);
-                    // the sum runs over what the tensor core will see: the rounded probabilities
-                    if (BF16) {
-                        // bf16 keeps 8 significant bits: the rounding remainder of P goes into a second bf16 operand, so
-                        // that the P V product sees about 16 bits (fp16's 11 bits need no correction)
-                        const float h0 = __uint_as_float(w[e] << 16), h1 = __uint_as_float(w[e] & 0xffff0000u);
-                        w2[e] = pf_pack2<true>(e0 - h0, e1 - h1);
-                        sum += (h0 + __uint_as_float(w2[e] << 16)) + (h1 + __uint_as_float(w2[e] & 0xffff0000u));
+                for (int c = 0; c < 64; c += 4) {
+                    a0 = fmaxf(a0, __uint_as_float(sv[c >> 5][c & 31]));
+                    a1 = fmaxf(a1, __uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]));
+                    a2 = fmaxf(a2, __uint_as_float(sv[(c + 2) >> 5][(c + 2) & 31]));
+                    a3 = fmaxf(a3, __uint_as_float(sv[(c + 3) >> 5][(c + 3) & 31]));
+                }
+                const float m_cand = fmaxf(m_run, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * p.scale_log2e);
+                const bool grow = m_cand > m_run + PF_LAZY;   // (true at the first stage: m_run = -inf)
+                m_new = grow ? m_cand : m_run;
+                alpha = grow ? pf_exp2(m_run - m_cand) : 1.f;
+                const float neg_m = -m_new;
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int w = 0; w < 32; ++w) {
+                    const int c = 2 * w;
+                    const float e0 = pf_exp2(fmaf(__uint_as_float(sv[c >> 5][c & 31]), p.scale_log2e, neg_m));
+                    const float e1 = pf_exp2(fmaf(__uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]), p.scale_log2e, neg_m));
+                    ph[w] = pf_pack2<BF16>(e0, e1);
+                    if (BF16) pl[w] = pf_pack2<true>(e0 - __uint_as_float(ph[w] << 16), e1 - __uint_as_float(ph[w] & 0xffff0000u));
+                    if (w & 1) {
+                        s2 += e0;
+                        s3 += e1;
                     } else {
-                        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[e]));
-                        sum += f.x + f.y;
+                        s0 += e0;
+                        s1 += e1;
                     }
                 }
-                *reinterpret_cast<uint4 *>(prow + ((cc ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                if (BF16) *reinterpret_cast<uint4 *>(prow + SM::P_BYTES + ((cc ^ (r & 7)) << 4)) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+                sum = (s0 + s1) + (s2 + s3);
+            } else {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        float x = __uint_as_float(sv[h][c]) * p.scale_log2e;
+                        x = (row_valid && t_base + h * 32 + c <= my_pos) ? x : -INFINITY;   // masked by selection (NaN scores too)
+                        sv[h][c] = __float_as_uint(x);
+                        mx = fmaxf(mx, x);
+                    }
+                const float m_cand = fmaxf(m_run, mx);
+                const bool grow = m_cand > m_run + PF_LAZY;   // (m_run = -inf: true unless the row has seen nothing yet)
+                m_new = grow ? m_cand : m_run;
+                alpha = grow ? pf_exp2(m_run - m_cand) : 1.f;   // (m_run = -inf gives 0: nothing accumulated yet)
+                sum = 0.f;
+#pragma unroll
+                for (int w = 0; w < 32; ++w) {
+                    const int c = 2 * w;
+                    const float x0 = __uint_as_float(sv[c >> 5][c & 31]), x1 = __uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]);
+                    const float e0 = m_new == -INFINITY ? 0.f : pf_exp2(x0 - m_new), e1 = m_new == -INFINITY ? 0.f : pf_exp2(x1 - m_new);
+                    ph[w] = pf_pack2<BF16>(e0, e1);
+                    if (BF16) pl[w] = pf_pack2<true>(e0 - __uint_as_float(ph[w] << 16), e1 - __uint_as_float(ph[w] & 0xffff0000u));
+                    sum += e0 + e1;
+                }
             }
-        }
-        l_run = l_run * alpha + sum;
-        m_run = m_new;
-        // this stage's V has landed?  Rows of V beyond what the tile may see hold whatever was there (a tail block's
-        // garbage, an earlier stage): masked tokens are excluded, not multiplied by zero, so clear them before they meet P = 0
-        if (!pf_mbar_wait(bar_v, (uint32_t)(j & 1))) {
-            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-            misc[1] = 1;
-        }
-        const int32_t n_seen = min(PF_KV, kv_len - j * PF_KV);
-        if (n_seen < PF_KV) {
-            for (int e = tid; e < (PF_KV - n_seen) * HALVES * 8; e += PF_THREADS) {
-                const int row = n_seen + e / (HALVES * 8), rem = e % (HALVES * 8);
-                *reinterpret_cast<uint4 *>(smem + SM::OFF_V + (rem >> 3) * (PF_KV * 128) + row * 128 + ((rem & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+            l_run = l_run * alpha + sum;
+            m_run = m_new;
+            tmem_st32(tmem_sj + lane_addr, ph);            // a thread overwrites only its own row's scores, which it has read
+            if (BF16) tmem_st32(tmem_sj + lane_addr + 32, pl);
+            // ---- O *= alpha where a row's maximum moved (skipped by warps in which none did); O += P V of stage j - 1 first
+            if (j >= 1) {
+                if (!pf_mbar_wait(bar_o, (uint32_t)((j - 1) & 1))) {
+                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                    misc[1] = 1;
+                }
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t ov[32];
+                        tmem_ld32(tmem_o + lane_addr + c0, ov);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+                        tmem_st32(tmem_o + lane_addr + c0, ov);
+                    }
+                }
             }
+            tmem_wait_st();
+            // ---- this stage's V has landed?  Rows of V beyond what the tile may see hold whatever was there (a tail
+            // block's garbage, an earlier stage): masked tokens are excluded, not multiplied by zero, so clear them before
+            // they meet P = 0
+            const int32_t n_seen = min(PF_KV, kv_len - j * PF_KV);
+            if (n_seen < PF_KV) {
+                if (!pf_mbar_wait(bar_v + 8 * buf, (uint32_t)((j >> 1) & 1))) {
+                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                    misc[1] = 1;
+                }
+                for (int e = tid; e < (PF_KV - n_seen) * HALVES * 8; e += PF_ROWS_THREADS) {
+                    const int row = n_seen + e / (HALVES * 8), rem = e % (HALVES * 8);
+                    *reinterpret_cast<uint4 *>(smem + SM::OFF_V + buf * SM::KV_BYTES + (rem >> 3) * (PF_KV * 128) + row * 128 + ((rem & 7) << 4)) =
+                        make_uint4(0u, 0u, 0u, 0u);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+            tc_fence_before();
+            pf_mbar_arrive(bar_p);
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        // ---- O *= alpha where a row's maximum moved (skipped by warps in which none did)
-        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        if (ok && n_stages > 0) {
+            if (!pf_mbar_wait(bar_o, (uint32_t)((n_stages - 1) & 1))) {
+                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                misc[1] = 1;
+            }
+            tc_fence_after();
+            ok = !__any_sync(0xffffffffu, misc[1] != 0);
+        }
+        // ---- out = O / l, rounded to the 16-bit type (nearest even).  The TMEM loads are warp-wide: rows beyond the chunk
+        // take part in them and store nothing.
+        if (ok && n_stages > 0) {
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
 #pragma unroll
             for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t ov[32];
                 tmem_ld32(tmem_o + lane_addr + c0, ov);
                 tmem_wait_ld();
+                if (row_valid) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-                tmem_st32(tmem_o + lane_addr + c0, ov);
-            }
-            tmem_wait_st();
-        }
-        tc_fence_before();
-        __syncthreads();
-        if (misc[1]) { ok = false; break; }
-        // ---- O += P V
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < PF_KV / 16; ++ks) {
-                const uint64_t a = smem_desc(base + SM::OFF_P + ks * 32, 16, 1024);
-                // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
-                const uint64_t b = smem_desc(base + SM::OFF_V + ks * 2048, PF_KV * 128, 1024);
-                mma_f16(tmem_o, a, b, IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
-                if (BF16) mma_f16(tmem_o, smem_desc(base + SM::OFF_P + SM::P_BYTES + ks * 32, 16, 1024), b, IDESC_O, 1u);
-            }
-            tc_commit(bar_o);
-        }
-        if (!pf_mbar_wait(bar_o, (uint32_t)(j & 1))) {
-            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-            misc[1] = 1;
-        }
-        tc_fence_after();
-        if (tid == 0 && j + 1 < n_stages && misc[1] == 0) issue_tiles(j + 1, true);   // V's buffer is free again
-    }
-
-    // ---- out = O / l, rounded to the 16-bit type (nearest even).  The TMEM loads are warp-wide: rows beyond the chunk
-    // take part in them and store nothing.
-    if (ok && n_stages > 0) {
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-        uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t ov[32];
-            tmem_ld32(tmem_o + lane_addr + c0, ov);
-            tmem_wait_ld();
-            if (row_valid) {
-#pragma unroll
-                for (int c = 0; c < 32; c += 8) {
-                    uint4 v;
-                    v.x = pf_pack2<BF16>(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
-                    v.y = pf_pack2<BF16>(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
-                    v.z = pf_pack2<BF16>(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
-                    v.w = pf_pack2<BF16>(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
-                    dst[(c0 + c) >> 3] = v;
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 v;
+                        v.x = pf_pack2<BF16>(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                        v.y = pf_pack2<BF16>(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                        v.z = pf_pack2<BF16>(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                        v.w = pf_pack2<BF16>(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                        dst[(c0 + c) >> 3] = v;
+                    }
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, PF_TMEM_COLS);
+    if (warp == 4) tmem_dealloc(tmem, PF_TMEM_COLS);
 }
 
 }  // namespace

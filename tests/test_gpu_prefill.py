@@ -3,6 +3,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from oracle import prefill
 from paper_2411_09317_b200 import binding as pie
 from paper_2411_09317_b200 import synth
@@ -114,4 +115,46 @@ def test_rejected_arguments_enqueue_nothing():
                                   ctx_dev.data_ptr(), ctx_dev.data_ptr(), too_long, np.array([0, 40, 80], np.int32), 2, case.scale)
     pie.pie_sync(pc.pool)
     assert int(out.abs().sum()) == 0
+    pc.close()
+
+
+def test_prompt_in_chunks_through_write_swap_and_attend():
+    """The serving order of a chunked prefill: the prompt's K and V enter the cache chunk by chunk (pie_kv_write), blocks of
+    earlier chunks are swapped out to the host and brought back before the layer is used again, and each chunk attends to
+    everything cached so far.  Outputs of every chunk match the oracle fed the same K and V."""
+    hq, hkv, d, dtype = 8, 2, 128, BF16
+    lens = [700, 333]
+    case = Case(1, hq, hkv, d, dtype, lens, seed=66, host_frac=0.0, placement="identity")
+    pc = PoolCase(case, all_on_gpu=True, n_host_slots=case.NB + 4)
+    dev = torch.device("cuda:0")
+    # the prompt's K and V rows, written by the library instead of by the test's set-up: clear the pool first
+    k_all = synth.tensor_bits(66, synth.STREAM_KNEW, (sum(lens), hkv, d), dtype)
+    v_all = synth.tensor_bits(66, synth.STREAM_VNEW, (sum(lens), hkv, d), dtype)
+    case.gpu_pool[:] = 0
+    for b in range(case.NB):
+        pie.pie_block_write(pc.pool, 0, b, case.gpu_pool[case.unit_slot[0, b]])
+    starts = np.concatenate([[0], np.cumsum(lens)])
+    done = np.zeros(2, np.int32)
+    chunk = 256
+    while np.any(done < lens):
+        c = np.minimum(chunk, np.array(lens) - done).astype(np.int32)
+        seq = np.concatenate([np.full(c[s], s, np.int32) for s in range(2)])
+        pos = np.concatenate([done[s] + np.arange(c[s], dtype=np.int32) for s in range(2)])
+        rows = np.concatenate([starts[s] + done[s] + np.arange(c[s]) for s in range(2)])
+        k_dev = torch.from_numpy(k_all[rows].view(np.int16)).to(dev)
+        v_dev = torch.from_numpy(v_all[rows].view(np.int16)).to(dev)
+        seq_dev, pos_dev = torch.from_numpy(seq).to(dev), torch.from_numpy(pos).to(dev)   # (kept alive until the sync below)
+        pie.pie_kv_write(pc.pool, 0, k_dev.data_ptr(), v_dev.data_ptr(), seq_dev.data_ptr(), pos_dev.data_ptr(), len(seq),
+                         pc.bt.data_ptr(), case.block_table.shape[1], 2)
+        assert oracle.kv_write(case.gpu_pool, case.host_pool, case.unit_side[0], case.unit_slot[0], k_all[rows], v_all[rows], seq, pos,
+                               case.block_table, hkv, d) == 0
+        ctx = (done + c).astype(np.int32)
+        got, want = run_prefill(case, pc, 0, c.tolist(), seed=100 + int(done[0]), ctx_lens=ctx)
+        assert np.all(np.abs(got - want) <= tolerance(want, dtype)), (done, float(np.abs(got - want).max()))
+        done = done + c
+        # the blocks written so far leave for the host and come back into other slots before the next chunk
+        used = np.unique(np.concatenate([case.block_table[s, :(done[s] + 15) // 16] for s in range(2)]))
+        pie.pie_swap_out(pc.pool, 0, used)
+        pie.pie_swap_in(pc.pool, 0, used[::-1].copy())
+    pie.pie_sync(pc.pool)
     pc.close()
