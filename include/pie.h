@@ -204,18 +204,25 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
                          const int32_t *ctx_lens_host, int32_t n_seqs, float scale, const void *k_new,
                          const void *v_new);
 
-/* One decode step: for every layer l, prefetch layer l+1's host-resident units (wrapping to layer 0 of
- * the next token, Section 3.4.2), run layer l's attention, push layer l's share back out (Section 3.3:
- * the layer that just finished is the coldest).  With timing enabled the host runs at most 4 steps ahead.  PIE_ERR_NOMEM if the GPU pool cannot take a layer's
- * host-resident share (the layers before it have been enqueued).  q_all/out_all: device [n_layers][n_seqs][Hq][D];
- * k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D] or NULL.  Runs pie_controller_tick at the end. */
+/* One decode step: for every layer, run its attention; by groups of layers (pie_set_lookahead) prefetch the next group's
+ * host-resident units when a group starts (wrapping to the first layers of the next token, Section 3.4.2) and push the
+ * group's share back out when it has computed (Section 3.3: the layer that just finished is the coldest).  Nothing but
+ * the layers' kernels is enqueued on the compute stream: a layer's kernel waits for its arriving units itself (a device
+ * word the copy-in stream sets behind each list), the copy streams wait for the kernels by value, and from the second
+ * layer on each attention kernel is launched as a programmatic dependent of the one before it (the layers' q / k_new /
+ * v_new must therefore all be ready when the call is made - they are: the arrays hold every layer).  With timing enabled
+ * the host runs at most 4 steps ahead.  A share the GPU pool has no room for when its group is prefetched is fetched at its
+ * layer's turn; if there is no room even then the call returns PIE_ERR_NOMEM with the layers before it enqueued and nothing
+ * of that layer.  q_all/out_all: device [n_layers][n_seqs][Hq][D]; k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D]
+ * or NULL.  Runs pie_controller_tick at the end. */
 int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int32_t *block_table_dev,
                     int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale,
                     const void *k_new_all, const void *v_new_all, int32_t mode);
 /* One layer of pie_decode_step by itself, for callers that run other work between the layers (Section 4.2: supporting
  * a model means adding this control loop to its forward pass): fetches whatever the layer still lacks, starts the
  * prefetch of layer (layer+1) mod n_layers, runs the attention (and the append, if k_new / v_new are given) and
- * pushes this layer's host-resident share out behind it.  q / out / k_new / v_new are this layer's device arrays
+ * pushes this layer's host-resident share out behind it (by groups of layers, as pie_decode_step does: a group left open
+ * is closed by pie_controller_tick, pie_step_begin or pie_sync).  q / out / k_new / v_new are this layer's device arrays
  * ([n_seqs][n_q_heads][head_dim], [n_seqs][n_kv_heads][head_dim]).  Call pie_step_begin before layer 0 and
  * pie_controller_tick after the last layer when timing is on.  PIE_ERR_UNSUPPORTED under pie_set_layer_policy. */
 int pie_decode_layer(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
@@ -262,15 +269,19 @@ int pie_get_extension_ratio(pie_pool *pool, float *r);
 /* Controller constants (the paper gives none): step = ratio change per adjustment (default 1 / n_layers,
  * "one layer"), eps = stall / compute above which a step counts as stalled (0.02), u_hi = link-busy /
  * compute below which the ratio may grow (0.9).  A value <= 0 keeps the current setting.
- * What counts as "stall" is the compute stream's wait for arriving units plus the attention time in excess of
- * the time-per-token record taken on steps without swap traffic (copies that are hidden can still slow the
- * attention down through shared HBM bandwidth). */
+ * What counts as "stall" is the wait for arriving units plus the attention's slow-down: what the step's layers took above
+ * its own undisturbed ones (copies that are hidden can still slow the attention down through shared HBM bandwidth; every
+ * layer of a step attends the same batch, and the lists of a group of layers are in flight during the first part of the
+ * group only, so the step is its own yardstick and clock drift between steps does not read as a slow-down). */
 int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
-/* Look-ahead depth of the decode loop (pie_decode_step / pie_decode_layer): while layer l computes, the host-resident
- * shares of layers l+1 .. l+layers are on their way (wrapping into the next token).  1 is the paper's look-ahead
- * (Section 3.4.2).  A deeper one gives each copy several layers' time to arrive - the copy stream then only has to
- * keep up on average, not layer by layer - at the price of as many more layers' shares of GPU staging slots.
- * 1 <= layers <= 8 (PIE_ERR_INVALID otherwise). */
+/* Group size of the decode loop (pie_decode_step / pie_decode_layer): the loop issues swap lists for `layers`
+ * consecutive layers at a time - while a group computes, the next group's host-resident shares are on their way (wrapping
+ * into the next token) and the previous group's are going back.  1 is the paper's per-layer look-ahead (Section 3.4.2).
+ * A larger group gives each copy several layers' time to arrive, lets the copies of the group go as one (its blocks in as
+ * few copies as their slots allow, its table entries in one strided copy) and costs the compute stream nothing per layer;
+ * the price is GPU staging: three groups' shares are on the GPU at a time.  0 (the default): chosen per group from the
+ * slots the GPU pool can spare, at most 8 and at most a quarter of the layers.  0 <= layers <= 8 (PIE_ERR_INVALID
+ * otherwise); an explicit value is capped at half the layers. */
 int pie_set_lookahead(pie_pool *pool, int32_t layers);
 
 /* ---- 8-bit blocks (a variant beyond the paper, whose blocks are 16-bit: a token costs half the bytes in HBM, in the
@@ -359,11 +370,12 @@ int pie_controller_tick(pie_pool *pool, int32_t *changed);
 int pie_get_stats(pie_pool *pool, pie_stats *out);
 /* Per-layer timeline of the most recently evaluated step (timing = 2 in the configuration; timing = 1 keeps the
  * statistics and the controller but not this table): ms[l][7] = {end of the previous layer's attention kernel,
- * start of this layer's, its end, swap-in list start, end, swap-out list start, end} in ms from the start of the
- * step's first attention kernel; -1 where nothing was recorded.  The compute columns are the kernels' own GPU-timer
- * stamps; the copy columns are copy-stream events tied to them through one event recorded just before the step's
- * first kernel (a few us of slack).  capacity = floats available (>= 7 * n_layers).  PIE_ERR_INVALID if no step has
- * been evaluated yet.  Shows what overlapped with what. */
+ * start of this layer's - past its presence wait -, its end, swap-in list start, end, swap-out list start, end} in ms from
+ * the start of the step's first attention kernel; -1 where nothing was recorded.  The lists of a group of layers that went
+ * as one appear under the group's first layer.  The compute columns are the kernels' own GPU-timer stamps; the copy columns
+ * are copy-stream events tied to them through one event recorded just before the step's first kernel (a few us of slack).
+ * capacity = floats available (>= 7 * n_layers).  PIE_ERR_INVALID if no step has been evaluated yet.  Shows what
+ * overlapped with what. */
 int pie_get_step_timeline(pie_pool *pool, float *ms, int64_t capacity);
 /* Wait until everything enqueued so far has completed, at most timeout_us (PIE_ERR_TIMEOUT); applies
  * phase-2 updates and reports a pending device status word (PIE_ERR_NOT_RESIDENT ...). */
@@ -390,13 +402,19 @@ int pie_probe_hbm(int64_t bytes, int32_t reps, double *gbps);
  *   slot_table  device int32 [n_logical_blocks]: GPU slot of each logical block of this layer, -1 if absent
  *   q, out, block_table_dev, ctx_lens_dev, scale   as for pie_decode_attention (no append)
  *   ctx_lens_host  host copy of the lengths (required: sizes are checked before anything is enqueued)
- *   status_dev  optional device int32[4]; word 0 is set to 1 if a referenced block had no slot, word 3
- *               receives the batch's context-token count
+ *   status_dev  device int32[4], cleared by the caller, or NULL.  The kernels raise (set to 1) word 0 if a referenced
+ *               block had no slot (slot_table entry negative or >= n_slots: that tile then reads slot 0 and the output of
+ *               its sequence is wrong), word 1 if ctx_lens_dev holds a length beyond the table or more chunks than
+ *               ctx_lens_host sized the scratch for (clamped: nothing is computed in the second case), word 2 if a
+ *               bounded wait ran out; word 3 receives the batch's context-token count (batches of at most 1024
+ *               sequences only).  Nothing clears the words.  With NULL these device-side conditions CANNOT be detected:
+ *               the call still returns PIE_OK - pass the words unless the tables are known good
  *   stream      a cudaStream_t
  * The split-K scratch (chunk offsets, fp32 partials) is a static device array of PIE_NOALLOC_SCRATCH_BYTES
  * that every GPU loading the library holds until the process exits.  A call whose partials would not fit
  * (sum over sequences of ceil(ctx / split_tokens), times n_q_heads * (head_dim + 2) * 4 bytes, plus 17 KiB)
- * or with more than PIE_NOALLOC_MAX_SEQS sequences returns PIE_ERR_NOMEM and enqueues nothing.
+ * or with more than PIE_NOALLOC_MAX_SEQS sequences returns PIE_ERR_NOMEM and enqueues nothing; so does every other
+ * argument error.  (A CUDA error from the memset or a launch - PIE_ERR_CUDA - may leave the memset enqueued.)
  * All calls on a device share that array and it keeps the previous call's contents: each call clears the
  * counters it needs at zero (a memset on `stream`) and writes every other word before reading it; two calls
  * that overlap on the GPU (different streams, no dependency) race - order them.  The first call on each device looks up the array's device

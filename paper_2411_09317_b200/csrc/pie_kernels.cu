@@ -466,6 +466,9 @@ struct AttnParams {
     unsigned long long done_value;
     const unsigned long long *arrive;  // device word of this layer, or NULL
     unsigned long long arrive_need;    // 0: nothing to wait for
+    // the same for the call's own inputs (q, k_new, v_new), where a copy stream brings them (host-buffer entry point)
+    const unsigned long long *inputs_arrive;
+    unsigned long long inputs_need;
     int64_t n_gpu_slots;
     int32_t max_blocks, n_seqs, n_q_heads, n_kv_heads, group, n_logical, split_tokens, use3d, max_chunks;
     float scale_log2e;      // softmax scale * log2(e) (* the key scale of an 8-bit pool)
@@ -715,7 +718,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     grid_dependency_wait();
     if (tid == 0 && p.stamps != nullptr && blockIdx.x == 0) {
         *reinterpret_cast<volatile uint64_t *>(p.stamps) = globaltimer_ns();
-        if (p.arrive_need == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = 0;   // every launch writes all its stamps
+        if (p.arrive_need == 0 && p.inputs_need == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = 0;   // every launch writes all its stamps
     }
     const int32_t *co = co_in_smem ? co_smem : p.chunk_off_global;
     int32_t n_chunks_total = co[p.n_seqs];
@@ -731,12 +734,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         // ------------------------------------------------------------------ producer warp
         // presence wait (Section 3.2): no slot-table entry of this layer is read before the list that brings the
         // layer's units has landed.  Bounded (about half a second of polling): then the CTA flags it and leaves.
-        if (p.arrive_need != 0) {
+        if (p.arrive_need != 0 || p.inputs_need != 0) {
             if (lane == 0) {
                 const uint64_t t_begin = globaltimer_ns();
                 bool there = false;
                 for (uint32_t i = 0; i < (1u << 21); ++i) {
-                    if (ld_acquire_u64(p.arrive) >= p.arrive_need) {
+                    if ((p.arrive_need == 0 || ld_acquire_u64(p.arrive) >= p.arrive_need) &&
+                        (p.inputs_need == 0 || ld_acquire_u64(p.inputs_arrive) >= p.inputs_need)) {
                         there = true;
                         break;
                     }
@@ -747,7 +751,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     *abort_flag = 1;
                 }
                 if (p.stamps != nullptr && blockIdx.x == 0)
-                    *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = globaltimer_ns() - t_begin;
+                    *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = p.arrive_need != 0 ? globaltimer_ns() - t_begin : 0;
             }
             __syncwarp();
         }
@@ -1477,6 +1481,8 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.done_value = a.done_value;
     p.arrive = a.arrive;
     p.arrive_need = a.arrive != nullptr ? a.arrive_need : 0ull;
+    p.inputs_arrive = a.inputs_arrive;
+    p.inputs_need = a.inputs_arrive != nullptr ? a.inputs_need : 0ull;
     p.n_gpu_slots = sh.n_gpu_slots;
     p.max_blocks = a.max_blocks;
     p.n_seqs = a.n_seqs;

@@ -82,6 +82,8 @@ struct AttnLaunch {
     int32_t *tokens_out = nullptr;  // optional, device-visible: receives the batch's context-token count
     const unsigned long long *arrive = nullptr;  // presence wait inside the kernel: wait until *arrive >= arrive_need
     unsigned long long arrive_need = 0;          // (the copy-in stream stores a list's ticket there behind its copies)
+    const unsigned long long *inputs_arrive = nullptr;  // the same for the call's q / k_new / v_new where a copy stream brings
+    unsigned long long inputs_need = 0;                 // them: no input is read before *inputs_arrive >= inputs_need
     bool dependent_launch = false;  // launch with programmatic stream serialization: only where the kernel before it in
                                     // the stream writes none of this call's lengths and tables
     float k_scale = 1.f, v_scale = 1.f;  // 8-bit pools: a stored byte stands for decode(byte) * scale

@@ -109,6 +109,8 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
     sc.counters = reinterpret_cast<int32_t *>(setup->scratch + OFF_PART);
     sc.part_ml = reinterpret_cast<float *>(setup->scratch + OFF_PART + cnt_bytes);
     sc.part_o = reinterpret_cast<float *>(setup->scratch + OFF_PART + cnt_bytes + ml_bytes);
+    const int32_t grid = setup->ctas_per_sm[head_dim == 128][dtype] * setup->n_sms;
+    if (grid <= 0) return PIE_ERR_UNSUPPORTED;   // nothing has been enqueued yet
     // the array keeps the last call's contents: the work and completion counters must start at zero
     if (cudaMemsetAsync(sc.counters, 0, (size_t)cnt_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PIE_ERR_CUDA;
     sc.max_items = items;
@@ -127,10 +129,10 @@ extern "C" int pie_decode_attention_noalloc(const void *kv_pool, int64_t n_slots
     a.gpu_pool = const_cast<void *>(kv_pool);
     a.split_tokens = split_tokens;
     a.variant = 0;
-    a.grid = setup->ctas_per_sm[head_dim == 128][dtype] * setup->n_sms;
+    a.grid = grid;
+    // without status words of the caller's the kernels' flags land in the shared scratch, where nobody reads them
     a.status = status_dev ? status_dev : reinterpret_cast<int32_t *>(setup->scratch + OFF_STATUS);
     a.tokens_out = a.status + 3;
-    if (a.grid <= 0) return PIE_ERR_UNSUPPORTED;
     if (pie::launch_attention(sh, sc, a, use3d ? map3d : map2d, use3d, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return PIE_ERR_CUDA;
     return PIE_OK;

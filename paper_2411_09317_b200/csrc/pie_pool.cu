@@ -181,7 +181,9 @@ struct pie_pool {
     std::vector<SwapList> group_lists;  // the lists of a group of layers (decode loop)
     std::vector<uint8_t> v_elide;
     cudaStream_t io_stream[2] = {nullptr, nullptr};  // pie_decode_step_host: inputs up / results down
-    std::vector<cudaEvent_t> io_up;                   // one per group of layers: its inputs have arrived
+    unsigned long long *io_arrive_dev = nullptr;     // counts the groups of layers whose inputs have arrived (set by io_stream[0])
+    unsigned long long io_groups_up = 0;             // ... as issued by the host
+    unsigned long long inputs_need = 0;              // what the next attention call's kernel has to wait for (0: nothing)
     std::vector<int32_t> v_plan_in, v_plan_out;  // one layer's plan inside the decode loop
     std::vector<int32_t> append_ids;  // blocks the coming appends write (pie_declare_append_blocks)
     bool append_declared = false;
@@ -760,8 +762,6 @@ void destroy_pool(pie_pool *p) {
         if (p->lev_close_ev[k]) cudaEventDestroy(p->lev_close_ev[k]);
     }
     if (p->aux_stream) cudaStreamDestroy(p->aux_stream);
-    for (cudaEvent_t ev : p->io_up)
-        if (ev) cudaEventDestroy(ev);
     for (int i = 0; i < 2; ++i)
         if (p->io_stream[i]) cudaStreamDestroy(p->io_stream[i]);
     if (p->own_streams)
@@ -771,6 +771,7 @@ void destroy_pool(pie_pool *p) {
     if (p->own_host && p->host_base) cudaFreeHost(p->host_base);
     cudaFree(p->slot_table_dev);
     cudaFree(p->arrive_dev);
+    cudaFree(p->io_arrive_dev);
     cudaFree(p->done_dev);
     cudaFree(p->list_dev);
     if (p->list_host) cudaFreeHost(p->list_host);
@@ -885,6 +886,8 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.stamps = le ? stamp_dev(p, layer, STAMP_START) : nullptr;
     a.arrive = p->arrive_dev + layer;
     a.arrive_need = arrive_need;
+    a.inputs_arrive = p->io_arrive_dev;
+    a.inputs_need = p->inputs_need;
     a.done_word = p->done_dev;
     a.done_value = (unsigned long long)ticket;
     a.dependent_launch = dependent;
@@ -1094,14 +1097,13 @@ int finish_group(pie_pool *p) {
     return st != PIE_OK ? st : st2;
 }
 
-// streams and events of the host-buffer entry point's pipeline (created at its first use)
+// streams and the arrival word of the host-buffer entry point's pipeline (created at its first use)
 int ensure_io(pie_pool *p) {
     if (p->io_stream[0]) return PIE_OK;
     PIE_CUDA(cudaStreamCreateWithFlags(&p->io_stream[0], cudaStreamNonBlocking));
     PIE_CUDA(cudaStreamCreateWithFlags(&p->io_stream[1], cudaStreamNonBlocking));
-    const int n_groups = (p->cfg.n_layers + IO_GROUP_LAYERS - 1) / IO_GROUP_LAYERS;
-    p->io_up.assign((size_t)n_groups, nullptr);
-    for (cudaEvent_t &ev : p->io_up) PIE_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    PIE_CUDA(cudaMalloc((void **)&p->io_arrive_dev, 64));
+    PIE_CUDA(cudaMemset(p->io_arrive_dev, 0, 64));
     return PIE_OK;
 }
 
@@ -2382,26 +2384,55 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
             PIE_CUDA(cudaMemcpyAsync((uint8_t *)pool->stage_v + l0 * kv_layer, (const uint8_t *)v_new_all_host + l0 * kv_layer,
                                      (size_t)(nl * kv_layer), cudaMemcpyHostToDevice, pool->io_stream[0]));
         }
-        PIE_CUDA(cudaEventRecord(pool->io_up[(size_t)g], pool->io_stream[0]));
+        // the group's arrival: the count of groups brought up so far, stored behind the group's copies; the group's first
+        // attention kernel waits for it itself (a stream-level wait would cost the compute stream its chain of dependent launches)
+        int64_t woff = 0;
+        st = list_alloc(pool, 4, &woff);
+        if (st != PIE_OK) return st;
+        unsigned long long *w = reinterpret_cast<unsigned long long *>(pool->list_host + woff);
+        *w = ++pool->io_groups_up;
+        PIE_CUDA(cudaMemcpyAsync(pool->io_arrive_dev, w, 8, cudaMemcpyHostToDevice, pool->io_stream[0]));
+        st = list_commit(pool, woff, 4, pool->io_stream[0]);
+        if (st != PIE_OK) return st;
     }
+    const unsigned long long groups_before = pool->io_groups_up - (unsigned long long)n_groups;
     st = pie_step_begin(pool);
     if (st != PIE_OK) return st;
+    int32_t pending_group = -1;   // a group whose layers are enqueued and whose results wait for the next layer's kernel
+    auto download = [&](int32_t g, bool by_value) -> int {
+        const int32_t l0 = g * G, nl = std::min(G, L - l0);
+        int rc = PIE_OK;
+        if (by_value && pool->wait_value64 && pool->recorded[PIE_Q_COMPUTE] == pool->last_attn_ticket) {
+            // the kernel of the layer after the group has completed -> so has the group's last combine kernel before it
+            if (pool->wait_value64((CUstream)pool->io_stream[1], (CUdeviceptr)(uintptr_t)pool->done_dev, (cuuint64_t)pool->last_attn_ticket,
+                                   CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
+                rc = PIE_ERR_CUDA;
+        } else {
+            cudaEvent_t ev = nullptr;
+            rc = push_mark(pool, &ev);
+            if (rc == PIE_OK && cudaStreamWaitEvent(pool->io_stream[1], ev, 0) != cudaSuccess) rc = PIE_ERR_CUDA;
+        }
+        if (rc != PIE_OK) return rc;
+        PIE_CUDA(cudaMemcpyAsync((uint8_t *)out_all_host + l0 * q_layer, (const uint8_t *)pool->stage_out + l0 * q_layer,
+                                 (size_t)(nl * q_layer), cudaMemcpyDeviceToHost, pool->io_stream[1]));
+        return PIE_OK;
+    };
     for (int32_t l = 0; l < L; ++l) {
-        if (l % G == 0) PIE_CUDA(cudaStreamWaitEvent(s, pool->io_up[(size_t)(l / G)], 0));
+        pool->inputs_need = l % G == 0 ? groups_before + (unsigned long long)(l / G) + 1 : 0;
         st = decode_layer(pool, l, (const uint8_t *)pool->stage_q + l * q_layer, (uint8_t *)pool->stage_out + l * q_layer,
                           pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
                           k_new_all_host ? (const uint8_t *)pool->stage_k + l * kv_layer : nullptr,
                           k_new_all_host ? (const uint8_t *)pool->stage_v + l * kv_layer : nullptr, mode, l > 0);
+        pool->inputs_need = 0;
         if (st != PIE_OK) break;
-        if ((l + 1) % G == 0 || l + 1 == L) {
-            // the group's results: behind the compute ticket of its last layer
-            const int32_t l0 = (l / G) * G, nl = l + 1 - l0;
-            st = wait_ticket(pool, pool->io_stream[1], PIE_Q_COMPUTE, pool->recorded[PIE_Q_COMPUTE]);
+        if (pending_group >= 0) {   // the group before this layer: its results come down once this layer's kernel has run
+            st = download(pending_group, true);
+            pending_group = -1;
             if (st != PIE_OK) break;
-            PIE_CUDA(cudaMemcpyAsync((uint8_t *)out_all_host + l0 * q_layer, (const uint8_t *)pool->stage_out + l0 * q_layer,
-                                     (size_t)(nl * q_layer), cudaMemcpyDeviceToHost, pool->io_stream[1]));
         }
+        if ((l + 1) % G == 0 || l + 1 == L) pending_group = l / G;
     }
+    if (st == PIE_OK && pending_group >= 0) st = download(pending_group, false);   // the last group: behind a mark
     // whatever happened, nothing of this call may still be in flight when it returns (the caller owns the host buffers)
     cudaError_t e1 = cudaStreamSynchronize(pool->io_stream[0]);
     cudaError_t e2 = cudaStreamSynchronize(s);
