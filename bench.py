@@ -192,8 +192,8 @@ def run_reference(args):
 
 # -------------------------------------------------------------------------------------------------------
 SWEEP_RATIOS = {"llama2_7b": [0.003, 0.004, 0.005, 0.0055, 0.006, 0.007],
-                "llama3_8b": [0.003, 0.004, 0.005, 0.006, 0.007],
-                "llama3_70b": [0.002, 0.003, 0.004, 0.005]}
+                "llama3_8b": [0.003, 0.004, 0.005, 0.0055, 0.006, 0.007],
+                "llama3_70b": [0.003, 0.004, 0.005, 0.0055, 0.006]}
 KEPT_RATIOS = {"llama2_7b": [0.006, 0.007, 0.008, 0.009], "llama3_8b": [0.006, 0.007, 0.008], "llama3_70b": [0.004, 0.005, 0.006]}
 DTYPE_NAME = {synth.F16: "f16", synth.BF16: "bf16"}
 

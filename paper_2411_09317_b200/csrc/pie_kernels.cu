@@ -673,6 +673,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // Presence, first look (the thread that would poll below): the arrival words are stored by copies, not by the kernel
+    // before this one, so they may be read ahead of the dependency wait.  A list that has landed by now - the usual case,
+    // the lists run a group of layers ahead - costs the kernel nothing: the load's latency hides behind the plan.
+    bool there_early = false;
+    if (tid == ATT_NW * 32 && (p.arrive_need != 0 || p.inputs_need != 0))
+        there_early = (p.arrive_need == 0 || ld_acquire_u64(p.arrive) >= p.arrive_need) &&
+                      (p.inputs_need == 0 || ld_acquire_u64(p.inputs_arrive) >= p.inputs_need);
     // ---- plan: chunk offsets of the batch (exclusive scan of the per-sequence chunk counts)
     const bool co_in_smem = p.n_seqs <= ATT_SMEM_SEQS;
     if (co_in_smem) {
@@ -735,7 +742,9 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         // presence wait (Section 3.2): no slot-table entry of this layer is read before the list that brings the
         // layer's units has landed.  Bounded (about half a second of polling): then the CTA flags it and leaves.
         if (p.arrive_need != 0 || p.inputs_need != 0) {
-            if (lane == 0) {
+            if (lane == 0 && there_early) {
+                if (p.stamps != nullptr && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = 0;
+            } else if (lane == 0) {
                 const uint64_t t_begin = globaltimer_ns();
                 bool there = false;
                 for (uint32_t i = 0; i < (1u << 21); ++i) {
