@@ -452,7 +452,13 @@ struct AttnParams {
     uint4 *pool;
     float *part_o;
     float *part_ml;
-    int32_t *counters;  // [0] next item, [1] CTAs that have left
+    // Deferred combine: the partials the call BEFORE this one left (same batch, same lengths, the other pair of partial
+    // buffers) are merged into prev_out by this kernel's consumer warps once their CTA has run out of attention work -
+    // in the tail of the launch, where SMs would idle - instead of by a kernel of its own between the two layers.
+    const float *prev_part_o;
+    const float *prev_part_ml;
+    uint16_t *prev_out;  // NULL: nothing to merge
+    int32_t *counters;  // [0] next item, [1] CTAs that have left, [2] next piece of the deferred combine
     uint64_t *stamps;   // optional, host visible: [0] when CTA 0 started its main work, [1] when the last CTA left
                         // (globaltimer ns), [2] how long CTA 0 waited for the layer's arriving units (ns), [3] the
                         // batch's context tokens
@@ -626,6 +632,44 @@ cudaError_t launch_kv_write8(const void *k, const void *v, const int32_t *token_
                                                                    per_cta, block_table, max_blocks, n_seqs, slot_table, n_logical,
                                                                    n_gpu_slots, (uint8_t *)gpu_pool, n_kv_heads, k_scale, v_scale, status);
     return cudaGetLastError();
+}
+
+// One 16-byte piece (four consecutive d of head g) of a sequence's output from its chunk partials: log-sum-exp merge in
+// chunk order, normalised, rounded to the 16-bit type.  get_ml(c) -> {m, l} of chunk c for this head.  Used by the combine
+// kernel and by the deferred combine in the attention kernel's tail: the same arithmetic in the same order, so the same
+// bits whoever merges.
+template <int D, bool BF16, typename GetML>
+__device__ __forceinline__ uint2 merge_piece(const float *__restrict__ part_o, int32_t chunk0, int32_t nchunks, int32_t n_kv_heads,
+                                             int32_t kvh, int32_t group, int g, int d, GetML get_ml) {
+    float mm = -INFINITY;
+    for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, get_ml(c).x);
+    float ll = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int32_t c0 = 0; c0 < nchunks; c0 += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (c0 + j < nchunks) {
+                const int64_t id = ((int64_t)(chunk0 + c0 + j) * n_kv_heads + kvh) * group + g;
+                v[j] = *reinterpret_cast<const float4 *>(part_o + id * D + d);
+            }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (c0 + j < nchunks) {
+                const float2 w = get_ml(c0 + j);
+                const float wt = w.x == -INFINITY ? 0.f : fast_exp2(w.x - mm);
+                ll += w.y * wt;
+                acc.x += v[j].x * wt;
+                acc.y += v[j].y * wt;
+                acc.z += v[j].z * wt;
+                acc.w += v[j].w * wt;
+            }
+    }
+    const float inv = ll > 0.f ? 1.f / ll : 0.f;
+    uint2 r;
+    r.x = pack2<BF16>(acc.x * inv, acc.y * inv);
+    r.y = pack2<BF16>(acc.z * inv, acc.w * inv);
+    return r;
 }
 
 // The second launch bound: for 16-bit pools it only tells the assembler that it need not hold registers back for more
@@ -1215,9 +1259,36 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (lane == 0) mbar_arrive(bar_qempty + 8 * qs);
         ++qn;
     }
+    // ---- deferred combine of the call before this one (its partials are complete: that grid has finished).  Pieces of
+    // 32 float4 each, handed out warp by warp from a counter of their own; sequences of a single chunk were finished by
+    // their own kernel.
+    if (p.prev_out != nullptr && n_items > 0 && *abort_flag == 0) {
+        constexpr int PIECES = D / 4;
+        const int per_pair = p.group * PIECES;
+        const int slices = (per_pair + 31) / 32;
+        const int32_t total = p.n_seqs * p.n_kv_heads * slices;
+        for (;;) {
+            int32_t ci = 0;
+            if (lane == 0) ci = atomicAdd(p.counters + 2, 1);
+            ci = __shfl_sync(0xffffffffu, ci, 0);
+            if (ci >= total) break;
+            const int32_t pair = ci / slices, e4 = (ci - pair * slices) * 32 + lane;
+            const int32_t s = pair / p.n_kv_heads, kvh = pair - s * p.n_kv_heads;
+            const int32_t chunk0 = co[s], nchunks = co[s + 1] - chunk0;
+            if (nchunks >= 2 && e4 < per_pair) {
+                const int g = e4 / PIECES, d = (e4 - g * PIECES) * 4;
+                const float *pml = p.prev_part_ml;
+                const int32_t hkv = p.n_kv_heads, grp = p.group;
+                const uint2 r = merge_piece<D, BF16>(p.prev_part_o, chunk0, nchunks, hkv, kvh, grp, g, d, [&](int32_t c) {
+                    return *reinterpret_cast<const float2 *>(pml + ((((int64_t)(chunk0 + c) * hkv + kvh) * grp + g) << 1));
+                });
+                *reinterpret_cast<uint2 *>(p.prev_out + ((int64_t)s * p.n_q_heads + (int64_t)kvh * grp + g) * D + d) = r;
+            }
+        }
+    }
     // the last CTA to leave resets the work counter for the next launch (every CTA has drawn its end marker by then)
-    if (p.done_word != nullptr) {
-        consumer_sync<NCONS>();   // the CTA's consumer warps have issued all their writes
+    if (p.done_word != nullptr || p.prev_out != nullptr) {
+        consumer_sync<NCONS>();   // the CTA's consumer warps have issued all their writes (and drawn their last piece)
     }
     if (tid == 0) {
         if (p.done_word != nullptr) __threadfence();   // ... and they are visible before this CTA counts as gone
@@ -1225,6 +1296,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (old == (int32_t)gridDim.x - 1) {
             p.counters[0] = 0;
             p.counters[1] = 0;
+            p.counters[2] = 0;
             if (p.stamps != nullptr) *reinterpret_cast<volatile uint64_t *>(p.stamps + 1) = globaltimer_ns();
             if (p.done_word != nullptr) {
                 __threadfence();
@@ -1278,33 +1350,8 @@ combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_
         for (int e4 = tid; e4 < group * per_head; e4 += COMB_THREADS) {
             const int g = e4 / per_head, d = d_lo + (e4 - g * per_head) * 4;
             const float *w = wbuf + g * cap, *l = lbuf + g * cap;
-            float mm = -INFINITY;
-            for (int32_t c = 0; c < nchunks; ++c) mm = fmaxf(mm, w[c]);
-            float ll = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int32_t c0 = 0; c0 < nchunks; c0 += 8) {
-                float4 v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (c0 + j < nchunks) {
-                        const int64_t id = ((int64_t)(chunk0 + c0 + j) * n_kv_heads + kvh) * group + g;
-                        v[j] = *reinterpret_cast<const float4 *>(part_o + id * D + d);
-                    }
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (c0 + j < nchunks) {
-                        const float wt = w[c0 + j] == -INFINITY ? 0.f : fast_exp2(w[c0 + j] - mm);
-                        ll += l[c0 + j] * wt;
-                        acc.x += v[j].x * wt;
-                        acc.y += v[j].y * wt;
-                        acc.z += v[j].z * wt;
-                        acc.w += v[j].w * wt;
-                    }
-            }
-            const float inv = ll > 0.f ? 1.f / ll : 0.f;
-            uint2 r;
-            r.x = pack2<BF16>(acc.x * inv, acc.y * inv);
-            r.y = pack2<BF16>(acc.z * inv, acc.w * inv);
+            const uint2 r = merge_piece<D, BF16>(part_o, chunk0, nchunks, n_kv_heads, kvh, group, g, d,
+                                                 [&](int32_t c) { return make_float2(w[c], l[c]); });
             *reinterpret_cast<uint2 *>(out + row0 + g * D + d) = r;
         }
         return;
@@ -1480,8 +1527,14 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.k_new = (const uint4 *)a.k_new;
     p.v_new = (const uint4 *)a.v_new;
     p.pool = (uint4 *)a.gpu_pool;
-    p.part_o = sc.part_o;
-    p.part_ml = sc.part_ml;
+    // two pairs of partial buffers where the pool has them: a call whose merge is deferred leaves its partials in the pair
+    // of its parity, and the next call (the other parity) merges them while it fills its own
+    const bool alt = a.parity != 0 && sc.part_o_alt != nullptr;
+    p.part_o = alt ? sc.part_o_alt : sc.part_o;
+    p.part_ml = alt ? sc.part_ml_alt : sc.part_ml;
+    p.prev_part_o = alt ? sc.part_o : sc.part_o_alt;
+    p.prev_part_ml = alt ? sc.part_ml : sc.part_ml_alt;
+    p.prev_out = sc.part_o_alt != nullptr ? (uint16_t *)a.prev_out : nullptr;
     p.counters = sc.counters;
     p.stamps = a.stamps;
     p.status = a.status;
@@ -1529,29 +1582,37 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
         return cudaLaunchKernelEx(&lc, kernel, map, p);
     });
     if (e != cudaSuccess) return e;
-    // merge the partials of sequences that span several chunks (CTAs of single-chunk sequences return at once)
+    if (a.defer_combine && sc.part_o_alt != nullptr) return cudaSuccess;   // the next call's kernel merges them
+    return launch_combine(sh, sc, a.out, a.n_seqs, a.max_blocks, a.split_tokens, alt ? 1 : 0, stream);
+}
+
+// merge the partials of sequences that span several chunks (CTAs of single-chunk sequences return at once)
+cudaError_t launch_combine(const AttnShape &sh, const AttnScratch &sc, void *out_ptr, int32_t n_seqs, int32_t max_blocks,
+                           int32_t split_tokens, int parity, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
+    const int32_t group = sh.n_q_heads / sh.n_kv_heads;
     // chunks of the longest sequence the table allows (rounded up to a multiple of 8: the loads go in eights)
-    const int64_t longest = ((int64_t)a.max_blocks * 16 + a.split_tokens - 1) / a.split_tokens;
+    const int64_t longest = ((int64_t)max_blocks * 16 + split_tokens - 1) / split_tokens;
     const int32_t cap = (int32_t)std::min<int64_t>(COMB_CAP, (longest + 7) / 8 * 8);
     // slices of head_dim such that a thread merges one 16-byte piece of one head (the merge is a chain of dependent
     // loads: what counts is how many rounds of them a thread makes), whole head_dim per CTA at most
-    const int64_t pairs = (int64_t)a.n_seqs * sh.n_kv_heads;
+    const int64_t pairs = (int64_t)n_seqs * sh.n_kv_heads;
     int slices = 1;
-    while (slices < sh.head_dim / 32 && p.group * (sh.head_dim / 4) / slices > COMB_THREADS) slices *= 2;
+    while (slices < sh.head_dim / 32 && group * (sh.head_dim / 4) / slices > COMB_THREADS) slices *= 2;
     cfg.gridDim = dim3((unsigned)pairs, (unsigned)slices);
     cfg.blockDim = dim3(COMB_THREADS);
-    cfg.dynamicSmemBytes = (size_t)(2 * p.group * cap) * sizeof(float);
+    cfg.dynamicSmemBytes = (size_t)(2 * group * cap) * sizeof(float);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    uint16_t *out = (uint16_t *)a.out;
-    const float *po = sc.part_o, *pml = sc.part_ml;
+    uint16_t *out = (uint16_t *)out_ptr;
+    const bool alt = parity != 0 && sc.part_o_alt != nullptr;
+    const float *po = alt ? sc.part_o_alt : sc.part_o, *pml = alt ? sc.part_ml_alt : sc.part_ml;
     const int32_t *co = sc.chunk_off;
-    const int32_t hq = sh.n_q_heads, hkv = sh.n_kv_heads, group = p.group;
+    const int32_t hq = sh.n_q_heads, hkv = sh.n_kv_heads;
     if (sh.head_dim == 128)
         return sh.dtype == PIE_BF16 ? cudaLaunchKernelEx(&cfg, combine_kernel<128, true>, po, pml, co, out, hq, hkv, group, cap)
                                     : cudaLaunchKernelEx(&cfg, combine_kernel<128, false>, po, pml, co, out, hq, hkv, group, cap);

@@ -56,6 +56,8 @@ struct AttnScratch {
     int32_t *counters;   // attn_counter_words(max_seqs, n_kv_heads) int32, zero before the first launch
     float *part_o;       // [max_items][G][D]
     float *part_ml;      // [max_items][G][2]
+    float *part_o_alt = nullptr;   // optional second pair of partial buffers (deferred combine: AttnLaunch::defer_combine)
+    float *part_ml_alt = nullptr;
     int64_t max_items;   // capacity in items (chunk, kv head)
     int32_t max_seqs;
 };
@@ -87,6 +89,14 @@ struct AttnLaunch {
     bool dependent_launch = false;  // launch with programmatic stream serialization: only where the kernel before it in
                                     // the stream writes none of this call's lengths and tables
     float k_scale = 1.f, v_scale = 1.f;  // 8-bit pools: a stored byte stands for decode(byte) * scale
+    // Deferred combine (needs the scratch's second pair of partial buffers; ignored without it).  defer_combine: no
+    // combine kernel follows this call - the NEXT call must name this call's out as its prev_out, have the other parity,
+    // and attend the same batch with the same lengths and split; its kernel merges this call's partials in the tail of
+    // its launch, so this call's out is complete when the next call's kernel is.  Whoever defers must see to it that the
+    // next call happens (or launch_combine with this call's parity).
+    bool defer_combine = false;
+    void *prev_out = nullptr;
+    int parity = 0;
 };
 
 // Build the TMA descriptors of the HBM pool: map3d covers a whole K+V tile in one copy
@@ -100,6 +110,9 @@ cudaError_t attn_configure(int head_dim, int dtype, int variant, int *ctas_per_s
 cudaError_t make_pool_tensor_map_fp8(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, CUtensorMap *map2d);
 cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const AttnLaunch &a, const CUtensorMap &map,
                              int use3d, cudaStream_t stream);
+// the combine kernel by itself (what launch_attention launches behind a call that does not defer its merge)
+cudaError_t launch_combine(const AttnShape &sh, const AttnScratch &sc, void *out, int32_t n_seqs, int32_t max_blocks,
+                           int32_t split_tokens, int parity, cudaStream_t stream);
 
 // ---- chunked-prefill attention (tcgen05 / TMEM) ----------------------------------------------------------------
 struct PrefillLaunch {

@@ -178,6 +178,14 @@ struct pie_pool {
     // scratch vectors
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
     SwapList one_list;                  // the list of a single swap call
+    // split-K merge left to the next attention call of the decode step (its kernel merges in the tail of its launch)
+    struct Deferred {
+        bool on = false;
+        void *out = nullptr;
+        const int32_t *ctx = nullptr;
+        int parity = 0;
+        int32_t n_seqs = 0, max_blocks = 0, split = 0;
+    } deferred;
     std::vector<SwapList> group_lists;  // the lists of a group of layers (decode loop)
     std::vector<uint8_t> v_elide;
     cudaStream_t io_stream[2] = {nullptr, nullptr};  // pie_decode_step_host: inputs up / results down
@@ -783,6 +791,8 @@ void destroy_pool(pie_pool *p) {
     cudaFree(p->scratch.counters);
     cudaFree(p->scratch.part_o);
     cudaFree(p->scratch.part_ml);
+    cudaFree(p->scratch.part_o_alt);
+    cudaFree(p->scratch.part_ml_alt);
     cudaFree(p->stage_q);
     cudaFree(p->stage_out);
     cudaFree(p->stage_k);
@@ -794,11 +804,29 @@ void destroy_pool(pie_pool *p) {
     delete p;
 }
 
+// A merge that was left to a next call that does not come (an error, a different batch): launch the combine kernel now.
+int flush_deferred_combine(pie_pool *p) {
+    if (!p->deferred.on) return PIE_OK;
+    p->deferred.on = false;
+    pie::AttnShape sh{p->cfg.head_dim, p->cfg.dtype, p->cfg.n_q_heads, p->cfg.n_kv_heads, p->cfg.n_logical_blocks,
+                      p->cfg.n_gpu_slots, p->kv_fp8};
+    cudaError_t e = pie::launch_combine(sh, p->scratch, p->deferred.out, p->deferred.n_seqs, p->deferred.max_blocks,
+                                        p->deferred.split, p->deferred.parity, p->stream[PIE_Q_COMPUTE]);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        p->sticky = PIE_ERR_CUDA;
+        return PIE_ERR_CUDA;
+    }
+    return PIE_OK;
+}
+
 // dependent: the call follows the previous layer's attention call of the same decode step directly, with the same
 // lengths and tables: its kernel may be launched as a programmatic dependent of that call's last kernel.
+// defer: the merge of this call's split-K partials is left to the next call's kernel (the caller promises that call, or
+// flush_deferred_combine); a merge that an earlier call left (p->deferred) is taken on by this call's kernel.
 int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const int32_t *bt_dev, int32_t max_blocks,
                    const int32_t *ctx_dev, const int32_t *bt_host, const int32_t *ctx_host, int32_t n_seqs, float scale,
-                   const void *k_new, const void *v_new, bool dependent = false) {
+                   const void *k_new, const void *v_new, bool dependent = false, bool defer = false) {
     if (!p) return PIE_ERR_INVALID;
     if (p->sticky != PIE_OK) return p->sticky;
     if (layer < 0 || layer >= p->cfg.n_layers) return PIE_ERR_RANGE;
@@ -891,6 +919,16 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.done_word = p->done_dev;
     a.done_value = (unsigned long long)ticket;
     a.dependent_launch = dependent;
+    // a merge the call before this one left: this kernel takes it on if it attends the same batch (else it is merged now)
+    if (p->deferred.on && !(dependent && p->deferred.n_seqs == n_seqs && p->deferred.max_blocks == max_blocks && p->deferred.ctx == ctx_dev)) {
+        st = flush_deferred_combine(p);
+        if (st != PIE_OK) return st;
+    }
+    if (p->deferred.on) {
+        a.prev_out = p->deferred.out;
+        a.parity = p->deferred.parity ^ 1;
+    }
+    a.defer_combine = defer;
     if (le && p->cfg.timing >= 2 && !p->lev_anchored[p->step % TIMING_RING]) {
         const int k = (int)(p->step % TIMING_RING);
         if (cudaEventRecord(p->lev_anchor[k], stream) == cudaSuccess) p->lev_anchored[k] = true;
@@ -901,6 +939,13 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         p->sticky = PIE_ERR_CUDA;
         return PIE_ERR_CUDA;
     }
+    p->deferred.on = defer && n_seqs > 0;
+    p->deferred.out = out;
+    p->deferred.parity = a.parity;
+    p->deferred.n_seqs = n_seqs;
+    p->deferred.max_blocks = max_blocks;
+    p->deferred.ctx = ctx_dev;
+    p->deferred.split = (int32_t)split;
     st = record_ticket(p, PIE_Q_COMPUTE, ticket);
     if (st != PIE_OK) p->sticky = st;
     p->last_attn_ticket = ticket;
@@ -1318,6 +1363,9 @@ int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
     }
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_o, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
+    // second pair: the decode step defers every layer's merge into the tail of the next layer's kernel
+    PIE_TRY(cudaMalloc((void **)&p->scratch.part_o_alt, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
+    PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml_alt, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
     if (p->kv_fp8) {
         PIE_TRY(pie::make_pool_tensor_map_fp8(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, &p->map2d), PIE_ERR_CUDA);
         p->use3d = 0;
@@ -2217,7 +2265,7 @@ static int decode_step_layers(pie_pool *pool, const void *q_all, void *out_all, 
 // its end push the group's host-resident shares out.
 static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, const int32_t *block_table_dev,
                         int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, int32_t n_seqs, float scale, const void *k_new,
-                        const void *v_new, int32_t mode, bool dependent = false) {
+                        const void *v_new, int32_t mode, bool dependent = false, bool defer = false) {
     const int32_t L = pool->cfg.n_layers;
     struct PollHold {
         pie_pool *p;
@@ -2279,7 +2327,7 @@ static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, con
         }
     }
     st = attention_call(pool, l, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
-                        k_new, v_new, dependent);
+                        k_new, v_new, dependent, defer);
     if (st != PIE_OK) return st;
     pool->group_done.push_back(l);
     if ((int32_t)pool->group_done.size() >= pool->group_len) return finish_group(pool);
@@ -2303,8 +2351,11 @@ int pie_decode_step(pie_pool *pool, const void *q_all, void *out_all, const int3
         st = decode_layer(pool, l, (const uint8_t *)q_all + l * q_stride, (uint8_t *)out_all + l * q_stride, block_table_dev,
                           max_blocks_per_seq, ctx_lens_dev, n_seqs, scale,
                           k_new_all ? (const uint8_t *)k_new_all + l * kv_stride : nullptr,
-                          v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr, mode, l > 0);
-        if (st != PIE_OK) return st;
+                          v_new_all ? (const uint8_t *)v_new_all + l * kv_stride : nullptr, mode, l > 0, l + 1 < L);
+        if (st != PIE_OK) {
+            flush_deferred_combine(pool);   // the layers already enqueued keep their results
+            return st;
+        }
     }
     return pie_controller_tick(pool, nullptr);
 }
@@ -2422,9 +2473,12 @@ int pie_decode_step_host(pie_pool *pool, const void *q_all_host, void *out_all_h
         st = decode_layer(pool, l, (const uint8_t *)pool->stage_q + l * q_layer, (uint8_t *)pool->stage_out + l * q_layer,
                           pool->stage_bt, max_blocks_per_seq, pool->stage_ctx, n_seqs, scale,
                           k_new_all_host ? (const uint8_t *)pool->stage_k + l * kv_layer : nullptr,
-                          k_new_all_host ? (const uint8_t *)pool->stage_v + l * kv_layer : nullptr, mode, l > 0);
+                          k_new_all_host ? (const uint8_t *)pool->stage_v + l * kv_layer : nullptr, mode, l > 0, l + 1 < L);
         pool->inputs_need = 0;
-        if (st != PIE_OK) break;
+        if (st != PIE_OK) {
+            flush_deferred_combine(pool);
+            break;
+        }
         if (pending_group >= 0) {   // the group before this layer: its results come down once this layer's kernel has run
             st = download(pending_group, true);
             pending_group = -1;

@@ -82,7 +82,7 @@ def main(argv=None):
                          "step then runs layer by layer through pie_decode_layer")
     ap.add_argument("--swap-mode", default="auto", choices=["auto", "kernel", "copy_engine", "bulk_kernel"],
                     help="how swap lists are moved (PIE_MODE_*)")
-    ap.add_argument("--lookahead", type=int, default=1, help="layers prefetched ahead (pie_set_lookahead)")
+    ap.add_argument("--lookahead", type=int, default=0, help="layers per prefetch group (pie_set_lookahead; 0: the library chooses)")
     ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
     ap.add_argument("--attn-variant", type=int, default=0, help="attention kernel variant (tuning)")
     ap.add_argument("--kv-fp8", action="store_true", help="blocks of E4M3 bytes (half the bytes per token; head_dim 128)")
