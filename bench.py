@@ -269,7 +269,9 @@ class Runner:
                 "elided_gbs": (after["bytes_out_elided"] - before["bytes_out_elided"]) / sec / 1e9,
                 "wait_share": after["last_step_stall_ms"] / max(after["last_step_ms"], 1e-9),
                 "kernel_ms_per_layer": float(np.mean([c["last_step_compute_ms"] for c in comp if c["steps_measured"] > 0] or [np.nan])) / dw.wl.n_layers,
-                "launches": 2 * dw.wl.n_layers * n + int(after["calls_kernel"] - before["calls_kernel"]) +
+                # per step one attention kernel per layer (each merges the layer before it in its tail) and one combine
+                # kernel behind the last layer, plus whatever swap and table kernels the lists needed
+                "launches": (dw.wl.n_layers + 1) * n + int(after["calls_kernel"] - before["calls_kernel"]) +
                             int(after["patch_kernel_launches"] - before["patch_kernel_launches"])}
 
 
@@ -488,7 +490,7 @@ def main():
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": int(TRAFFIC_PER_ALG_BYTE * alg_bytes_per_launch),
                 "traffic_note": "ncu dram bytes of a quarter-scale launch scaled by the KV bytes read", "peak_kind": peak_kind,
-                "kernel": "paged_decode_attn_kernel (plan and append fused) + combine_kernel, one pair per layer: timed region / (layers x steps), "
+                "kernel": "paged_decode_attn_kernel (plan, append and the previous layer's split-K merge fused), one per layer, + one combine_kernel per step: timed region / (layers x steps), "
                           "the gaps between launches included",
                 "alg_bytes_per_launch": alg_bytes_per_launch, "ms_per_launch": ms_per_launch,
                 "kernel_only_ms_per_launch": head["kernel_ms_per_layer"],

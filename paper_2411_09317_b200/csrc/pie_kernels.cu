@@ -429,9 +429,12 @@ cudaError_t launch_swap_bulk(const void *src_pool, void *dst_pool, const int32_t
 //     tile holding position ctx-1 patches the new token's K and V rows into the staged tile and into the pool;
 //   - the combine of single-chunk sequences: normalised and rounded to 16 bits (nearest even) right here.  A
 //     sequence with several chunks gets one fp32 partial (m, l, unnormalised acc) per item, merged in chunk order
-//     by combine_kernel right after.  (A fused "last CTA to finish the pair merges it" variant was measured: its
-//     per-item release/acquire atomics and the serial merges cost more than the extra launch, badly so for 8-head
-//     groups and long contexts.)
+//     by combine_kernel right after - or, inside a decode step, by the NEXT layer's launch of this kernel: a CTA that
+//     has run out of attention work merges pieces of the previous layer's partials (the other pair of partial buffers)
+//     while the launch's last CTAs finish, so that between two layers there is one kernel boundary and the merge costs
+//     no time of its own.  (A fused "last CTA to finish the pair merges it" variant was measured: its per-item
+//     release/acquire atomics and the serial merges cost more than the extra launch, badly so for 8-head groups and
+//     long contexts.)
 // Every reduction order depends only on the logical token order and on ctx_len (tile -> warp by index, warps
 // merged in warp order, chunks merged in chunk order), never on slot ids, on which CTA ran an item or on
 // timing, so a run with swapped blocks reproduces a resident run bit for bit.
@@ -1567,8 +1570,9 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
             kernel<<<a.grid, (nw + 1) * 32, smem, stream>>>(map, p);
             return cudaGetLastError();
         }
-        // behind the previous layer's combine kernel: the CTAs may become resident, set their barriers up and scan the
-        // batch's lengths while that kernel drains; they wait for it before anything else
+        // behind the previous layer's last kernel (its attention kernel, where the merge is deferred): the CTAs may
+        // become resident, set their barriers up and scan the batch's lengths while that kernel drains; they wait for
+        // it before anything else
         cudaLaunchConfig_t lc = {};
         lc.gridDim = dim3((unsigned)a.grid);
         lc.blockDim = dim3((unsigned)((nw + 1) * 32));
