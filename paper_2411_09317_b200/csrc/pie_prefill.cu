@@ -194,7 +194,7 @@ struct PfSmem {
     static constexpr int OFF_K = OFF_Q + Q_BYTES;       // two stages
     static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;  // two stages
     static constexpr int OFF_BAR = OFF_V + 2 * KV_BYTES; // k_full[2], v_full[2], s_done[2], o_done
-    static constexpr int OFF_MISC = OFF_BAR + 64;       // [0] TMEM base, [1] abort, [4 .. 19] slots of the stages in flight
+    static constexpr int OFF_MISC = OFF_BAR + 64;       // [0] TMEM base, [1] abort, [4 .. 19] slots of the stages in flight, [24 .. 25] p_done[1]
     static constexpr int BYTES = OFF_MISC + 128;        // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
 };
 
@@ -211,7 +211,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
         if (tid == 0) pf_raise(p.status, STATUS_WAIT_TIMEOUT);
         return;
     }
-    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 32, bar_o = bar_k + 48, bar_p = bar_k + 56;
+    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 32, bar_o = bar_k + 48;
+    // "P of stage j is in place" has a barrier per stage parity: a softmax warp may be a stage ahead of another (the scores
+    // of stage j + 1 do not wait for P(j)), and two arrivals of one thread must never count towards one phase
+    const uint32_t bar_p2[2] = {bar_k + 56, base + SM::OFF_MISC + 96};
+    const uint32_t bar_done = base + SM::OFF_MISC + 104;   // O is final: used once (a barrier that is waited for in passing,
+                                                           // as bar_o is by warps that rescale, cannot also be waited for late)
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + SM::OFF_MISC);
 
     // ---- which tile
@@ -236,7 +241,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
 
     if (tid == 0) {
         for (int i = 0; i < 7; ++i) pf_mbar_init(bar_k + 8 * i, 1);   // k_full[2], v_full[2], s_done[2], o_done
-        pf_mbar_init(bar_p, PF_ROWS_THREADS);                          // P of a stage is in place: every row's thread arrives
+        pf_mbar_init(bar_p2[0], PF_ROWS_THREADS);                      // P of a stage is in place: every row's thread arrives
+        pf_mbar_init(bar_p2[1], PF_ROWS_THREADS);
+        pf_mbar_init(bar_done, 1);
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -283,84 +290,97 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
 
     if (warp == 4) {
         // =============================================================================== the issuing warp
-        // a stage's K (or V) tiles: one TMA copy per (block, 64-element half)
+        // The whole warp walks through the stages together: every lane waits on the barriers, lane 0 issues the MMAs, and a
+        // stage's K (or V) tiles - one TMA copy per (block, 64-element half), up to eight - are issued by as many lanes
+        // at once (issued one after the other by a single thread they cost it ~200 cycles each: half of a stage's time).
+        auto dead = [&]() { return __shfl_sync(0xffffffffu, misc[1] != 0 ? 1 : 0, 0) != 0; };
+        auto wait_all = [&](uint32_t bar, uint32_t parity) {
+            if (!pf_mbar_wait(bar, parity)) {
+                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                misc[1] = 1;
+            }
+            __syncwarp();
+        };
         auto issue_tiles = [&](int32_t j, bool v_rows) {
             const uint32_t buf = (uint32_t)(j & 1);
             const uint32_t bar = (v_rows ? bar_v : bar_k) + 8 * buf;
             const uint32_t dst0 = base + (v_rows ? SM::OFF_V : SM::OFF_K) + buf * SM::KV_BYTES;
             const int32_t nb = min(PF_KV / 16, (kv_len + 15) / 16 - j * (PF_KV / 16));
-            pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
-            for (int32_t i = 0; i < nb; ++i) {
+            if (lane == 0) pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
+            __syncwarp();
+            const int32_t i = lane / HALVES, h = lane - i * HALVES;
+            if (i < nb) {
                 const int32_t row0 = (slot_ring[(j & 3) * 4 + i] * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
-#pragma unroll
-                for (int h = 0; h < HALVES; ++h) pf_tma_2d(dst0 + h * (PF_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
+                pf_tma_2d(dst0 + h * (PF_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
             }
+            __syncwarp();
         };
         // S(j) = Q K(j)^T into the stage's half of the score columns (K(j) must have landed)
         auto issue_qk = [&](int32_t j) {
             const uint32_t buf = (uint32_t)(j & 1);
-            if (!pf_mbar_wait(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1))) {
-                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-                misc[1] = 1;
-                return;
-            }
-            tc_fence_after();
+            wait_all(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1));
+            if (dead()) return;
+            if (lane == 0) {
+                tc_fence_after();
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint64_t a = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
-                const uint64_t b = smem_desc(base + SM::OFF_K + buf * SM::KV_BYTES + (ks >> 2) * (PF_KV * 128) + (ks & 3) * 32, 16, 1024);
-                mma_f16(tmem + buf * PF_KV, a, b, IDESC_S, ks > 0 ? 1u : 0u);
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint64_t a = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
+                    const uint64_t b = smem_desc(base + SM::OFF_K + buf * SM::KV_BYTES + (ks >> 2) * (PF_KV * 128) + (ks & 3) * 32, 16, 1024);
+                    mma_f16(tmem + buf * PF_KV, a, b, IDESC_S, ks > 0 ? 1u : 0u);
+                }
+                tc_commit(bar_s + 8 * buf);
             }
-            tc_commit(bar_s + 8 * buf);
+            __syncwarp();
         };
-        if (lane == 0)
-            for (int32_t j = 0; j < min(n_stages, 2); ++j) {
-                issue_tiles(j, false);
-                issue_tiles(j, true);
-            }
+        for (int32_t j = 0; j < min(n_stages, 2); ++j) {
+            issue_tiles(j, false);
+            issue_tiles(j, true);
+        }
         __syncthreads();   // Q is in shared memory
-        if (lane == 0 && n_stages > 0) issue_qk(0);
+        if (n_stages > 0) issue_qk(0);
         // Software pipeline: while the four softmax warps work on the scores of stage j, the tensor core computes those of
         // stage j + 1 (into the other half of the score columns) and, before that, finishes O += P V of stage j - 1.
         for (int32_t j = 0; j < n_stages; ++j) {
             if (lane >= 4 && lane < 8 && j + 3 < n_stages) resolve(j + 3, lane - 4);   // read from the next iteration on
             __syncwarp();
-            if (lane == 0 && misc[1] == 0) {
-                const uint32_t buf = (uint32_t)(j & 1);
-                // the other half of the score columns held P(j - 1), and stage j - 1's V buffer is the one stage j + 1
-                // needs: O += P V of stage j - 1 must have completed
-                if (j >= 1 && !pf_mbar_wait(bar_o, (uint32_t)((j - 1) & 1))) {
-                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-                    misc[1] = 1;
-                }
-                if (misc[1] == 0 && j + 1 < n_stages) {
-                    if (j >= 1) issue_tiles(j + 1, true);
-                    issue_qk(j + 1);
-                }
-                // P(j) is in tensor memory (every row's thread has arrived): O += P V, then the K tiles of stage j + 2 into
-                // the buffer that S(j) no longer needs
-                if (misc[1] == 0 && !pf_mbar_wait(bar_p, (uint32_t)(j & 1))) {
-                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-                    misc[1] = 1;
-                }
-                if (misc[1] == 0 && !pf_mbar_wait(bar_v + 8 * buf, (uint32_t)((j >> 1) & 1))) {   // V(j) has landed
-                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-                    misc[1] = 1;
-                }
-                if (misc[1] == 0) {
-                    tc_fence_after();
-                    const uint32_t tmem_sj = tmem + buf * PF_KV;
-#pragma unroll
-                    for (int ks = 0; ks < PF_KV / 16; ++ks) {
-                        // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
-                        const uint64_t b = smem_desc(base + SM::OFF_V + buf * SM::KV_BYTES + ks * 2048, PF_KV * 128, 1024);
-                        mma_f16_ts(tmem_o, tmem_sj + ks * 8, b, IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
-                        if (BF16) mma_f16_ts(tmem_o, tmem_sj + 32 + ks * 8, b, IDESC_O, 1u);
-                    }
-                    tc_commit(bar_o);
-                    if (j + 2 < n_stages) issue_tiles(j + 2, false);
-                }
+            if (dead()) break;
+            const uint32_t buf = (uint32_t)(j & 1);
+            // S(j) is complete (the softmax warps wait for the same barrier): its K buffer is free, and the K tiles of
+            // stage j + 2 go there now, two stages ahead of their use
+            if (j + 2 < n_stages) {
+                wait_all(bar_s + 8 * buf, (uint32_t)((j >> 1) & 1));
+                if (dead()) break;
+                issue_tiles(j + 2, false);
             }
+            // the other half of the score columns held P(j - 1), and stage j - 1's V buffer is the one stage j + 1
+            // needs: O += P V of stage j - 1 must have completed
+            if (j >= 1) {
+                wait_all(bar_o, (uint32_t)((j - 1) & 1));
+                if (dead()) break;
+            }
+            if (j + 1 < n_stages) {
+                if (j >= 1) issue_tiles(j + 1, true);
+                issue_qk(j + 1);
+                if (dead()) break;
+            }
+            // P(j) is in tensor memory (every row's thread has arrived) and V(j) has landed: O += P V
+            wait_all(bar_p2[buf], (uint32_t)((j >> 1) & 1));
+            wait_all(bar_v + 8 * buf, (uint32_t)((j >> 1) & 1));
+            if (dead()) break;
+            if (lane == 0) {
+                tc_fence_after();
+                const uint32_t tmem_sj = tmem + buf * PF_KV;
+#pragma unroll
+                for (int ks = 0; ks < PF_KV / 16; ++ks) {
+                    // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
+                    const uint64_t b = smem_desc(base + SM::OFF_V + buf * SM::KV_BYTES + ks * 2048, PF_KV * 128, 1024);
+                    mma_f16_ts(tmem_o, tmem_sj + ks * 8, b, IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
+                    if (BF16) mma_f16_ts(tmem_o, tmem_sj + 32 + ks * 8, b, IDESC_O, 1u);
+                }
+                tc_commit(bar_o);
+                if (j + 1 == n_stages) tc_commit(bar_done);   // O is final
+            }
+            __syncwarp();
         }
         __syncwarp();
     } else {
@@ -458,13 +478,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
             tmem_st32(tmem_sj + lane_addr, ph);            // a thread overwrites only its own row's scores, which it has read
             if (BF16) tmem_st32(tmem_sj + lane_addr + 32, pl);
             // ---- O *= alpha where a row's maximum moved (skipped by warps in which none did); O += P V of stage j - 1 first
-            if (j >= 1) {
+            if (j >= 1 && __any_sync(0xffffffffu, alpha != 1.f)) {
                 if (!pf_mbar_wait(bar_o, (uint32_t)((j - 1) & 1))) {
                     pf_raise(p.status, STATUS_WAIT_TIMEOUT);
                     misc[1] = 1;
                 }
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                {
 #pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 32) {
                         uint32_t ov[32];
@@ -494,10 +514,10 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             tc_fence_before();
-            pf_mbar_arrive(bar_p);
+            pf_mbar_arrive(bar_p2[buf]);
         }
         if (ok && n_stages > 0) {
-            if (!pf_mbar_wait(bar_o, (uint32_t)((n_stages - 1) & 1))) {
+            if (!pf_mbar_wait(bar_done, 0u)) {
                 pf_raise(p.status, STATUS_WAIT_TIMEOUT);
                 misc[1] = 1;
             }
