@@ -35,7 +35,7 @@ namespace {
 constexpr int PF_M = 128;        // query rows per CTA (the MMA's M)
 constexpr int PF_KV = 64;        // KV tokens per stage
 constexpr int PF_ROWS_THREADS = 128;  // four softmax warps: warp w owns TMEM lanes 32 w .. 32 w + 31 (one thread per query row)
-constexpr int PF_THREADS = 160;       // + one warp that only issues: TMA copies, MMAs, block-table look-ups
+constexpr int PF_THREADS = 192;       // + a warp that issues the MMAs (warp 4) and one that loads: block-table look-ups, TMA copies (warp 5)
 constexpr int PF_TMEM_COLS = 256;
 // The running maximum of a row is only raised - and the row's O and sum rescaled, a round trip through tensor memory for
 // the whole warp - when the stage's maximum exceeds it by more than this (in log2 units): until then the probabilities
@@ -193,9 +193,9 @@ struct PfSmem {
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;       // two stages
     static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;  // two stages
-    static constexpr int OFF_BAR = OFF_V + 2 * KV_BYTES; // k_full[2], v_full[2], s_done[2], o_done
-    static constexpr int OFF_MISC = OFF_BAR + 64;       // [0] TMEM base, [1] abort, [4 .. 19] slots of the stages in flight, [24 .. 25] p_done[1]
-    static constexpr int BYTES = OFF_MISC + 128;        // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
+    static constexpr int OFF_BAR = OFF_V + 2 * KV_BYTES; // k_full[2], v_full[2], s_done[2], o_done[2], p_done[2], done
+    static constexpr int OFF_MISC = OFF_BAR + 128;      // [0] TMEM base, [1] abort, [4 .. 35] slots of eight stages' blocks
+    static constexpr int BYTES = OFF_MISC + 256;        // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
 };
 
 template <int D, bool BF16>
@@ -211,12 +211,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
         if (tid == 0) pf_raise(p.status, STATUS_WAIT_TIMEOUT);
         return;
     }
-    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 32, bar_o = bar_k + 48;
-    // "P of stage j is in place" has a barrier per stage parity: a softmax warp may be a stage ahead of another (the scores
-    // of stage j + 1 do not wait for P(j)), and two arrivals of one thread must never count towards one phase
-    const uint32_t bar_p2[2] = {bar_k + 56, base + SM::OFF_MISC + 96};
-    const uint32_t bar_done = base + SM::OFF_MISC + 104;   // O is final: used once (a barrier that is waited for in passing,
-                                                           // as bar_o is by warps that rescale, cannot also be waited for late)
+    // Every barrier exists once per stage parity.  A parity wait may be at most one phase behind, and the warps of this
+    // kernel run at their own pace (a softmax warp may be a stage ahead of another, the loading warp behind the issuing
+    // one): with a barrier per parity, the next phase of the barrier a warp waits on cannot complete before that warp
+    // has passed its wait (it needs what the warp does afterwards), whoever is slow.
+    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 16, bar_s = bar_k + 32, bar_o2 = bar_k + 48, bar_p = bar_k + 64;
+    const uint32_t bar_p2[2] = {bar_p, bar_p + 8};
+    const uint32_t bar_done = bar_k + 80;   // O is final (used once)
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + SM::OFF_MISC);
 
     // ---- which tile
@@ -240,7 +241,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
     const int32_t n_stages = bad ? 0 : (kv_len + PF_KV - 1) / PF_KV;
 
     if (tid == 0) {
-        for (int i = 0; i < 7; ++i) pf_mbar_init(bar_k + 8 * i, 1);   // k_full[2], v_full[2], s_done[2], o_done
+        for (int i = 0; i < 8; ++i) pf_mbar_init(bar_k + 8 * i, 1);   // k_full[2], v_full[2], s_done[2], o_done[2]
         pf_mbar_init(bar_p2[0], PF_ROWS_THREADS);                      // P of a stage is in place: every row's thread arrives
         pf_mbar_init(bar_p2[1], PF_ROWS_THREADS);
         pf_mbar_init(bar_done, 1);
@@ -249,24 +250,30 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 4) tmem_alloc(base + SM::OFF_MISC, PF_TMEM_COLS);
-    // ---- block table -> slot table -> slot, off the issuing thread's path: four of its warp's other lanes resolve the
-    // blocks of a stage three stages ahead into a small ring in shared memory (two dependent global loads each; done
-    // serially by the issuing thread they cost ten microseconds per stage)
-    volatile int32_t *slot_ring = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_MISC + 16);   // [4 stages][4 blocks]
-    auto resolve = [&](int32_t j, int32_t i) {
+    // ---- block table -> slot table -> slot: lanes of the loading warp resolve the blocks of a stage well ahead of the
+    // stage's copies into a ring in shared memory (two dependent global loads each; done serially by the thread that
+    // issues the copies they cost ten microseconds per stage)
+    volatile int32_t *slot_ring = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_MISC + 16);   // [8 stages][4 blocks]
+    const int32_t n_blocks = (kv_len + 15) / 16;
+    auto load_blk = [&](int32_t j, int32_t i) -> int32_t {   // the block's logical id, -1: the stage has no such block
         const int32_t b = j * (PF_KV / 16) + i;
-        int32_t slot = -1;
-        if (b < (kv_len + 15) / 16) {
-            const int32_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + b);
-            slot = (blk >= 0 && blk < p.n_logical) ? __ldcg(p.slot_table + blk) : -1;
-            if (slot < 0 || slot >= p.n_gpu_slots) {  // unit not on the GPU: flag it, stream slot 0 so the barriers complete
-                pf_raise(p.status, STATUS_MISSING_UNIT);
-                slot = 0;
-            }
-        }
-        slot_ring[(j & 3) * 4 + i] = slot;
+        if (j >= n_stages || b >= n_blocks) return -1;
+        const int32_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + b);
+        return blk < 0 ? p.n_logical : blk;   // an id that names nothing is a missing unit, not a missing block
     };
-    if (warp == 4 && lane >= 4 && lane < 16 && ((lane - 4) >> 2) < n_stages) resolve((lane - 4) >> 2, (lane - 4) & 3);
+    auto load_slot = [&](int32_t blk) -> int32_t {           // its slot, -2: no such unit on the GPU
+        if (blk < 0) return -1;
+        const int32_t v = blk < p.n_logical ? __ldcg(p.slot_table + blk) : -2;
+        return v < 0 ? -2 : v;
+    };
+    auto store_slot = [&](int32_t j, int32_t i, int32_t slot) {
+        if (slot < -1 || slot >= p.n_gpu_slots) {  // unit not on the GPU: flag it, stream slot 0 so the barriers complete
+            pf_raise(p.status, STATUS_MISSING_UNIT);
+            slot = 0;
+        }
+        slot_ring[(j & 7) * 4 + i] = slot;
+    };
+    if (warp == 5 && lane < 16) store_slot(lane >> 2, lane & 3, load_slot(load_blk(lane >> 2, lane & 3)));   // stages 0 .. 3
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -288,78 +295,113 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
 
-    if (warp == 4) {
-        // =============================================================================== the issuing warp
-        // The whole warp walks through the stages together: every lane waits on the barriers, lane 0 issues the MMAs, and a
-        // stage's K (or V) tiles - one TMA copy per (block, 64-element half), up to eight - are issued by as many lanes
-        // at once (issued one after the other by a single thread they cost it ~200 cycles each: half of a stage's time).
-        auto dead = [&]() { return __shfl_sync(0xffffffffu, misc[1] != 0 ? 1 : 0, 0) != 0; };
-        auto wait_all = [&](uint32_t bar, uint32_t parity) {
-            if (!pf_mbar_wait(bar, parity)) {
-                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
-                misc[1] = 1;
-            }
-            __syncwarp();
-        };
+    auto dead = [&]() { return __shfl_sync(0xffffffffu, misc[1] != 0 ? 1 : 0, 0) != 0; };
+    auto wait_all = [&](uint32_t bar, uint32_t parity) {   // by every lane of a warp
+        if (!pf_mbar_wait(bar, parity)) {
+            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+            misc[1] = 1;
+        }
+        __syncwarp();
+    };
+    if (warp == 5) {
+        // =============================================================================== the loading warp
+        // A stage's K (or V) tiles - one TMA copy per (block, 64-element half), up to eight - are issued by as many lanes at
+        // once.  K(j + 2) goes out as soon as the scores of stage j are complete (its buffer is free then), V(j + 1) as soon
+        // as O += P V of stage j - 1 is.  The TMA unit takes a stage's 32 KiB at its own pace (the issue blocks meanwhile),
+        // which is why this is a warp of its own: the MMAs must not queue behind it.
+        int32_t last_k[2] = {-1, -1}, last_v[2] = {-1, -1};   // newest stage issued into each buffer
         auto issue_tiles = [&](int32_t j, bool v_rows) {
             const uint32_t buf = (uint32_t)(j & 1);
             const uint32_t bar = (v_rows ? bar_v : bar_k) + 8 * buf;
             const uint32_t dst0 = base + (v_rows ? SM::OFF_V : SM::OFF_K) + buf * SM::KV_BYTES;
-            const int32_t nb = min(PF_KV / 16, (kv_len + 15) / 16 - j * (PF_KV / 16));
+            const int32_t nb = min(PF_KV / 16, n_blocks - j * (PF_KV / 16));
             if (lane == 0) pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
             __syncwarp();
             const int32_t i = lane / HALVES, h = lane - i * HALVES;
             if (i < nb) {
-                const int32_t row0 = (slot_ring[(j & 3) * 4 + i] * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
+                const int32_t row0 = (slot_ring[(j & 7) * 4 + i] * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
                 pf_tma_2d(dst0 + h * (PF_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
             }
             __syncwarp();
-        };
-        // S(j) = Q K(j)^T into the stage's half of the score columns (K(j) must have landed)
-        auto issue_qk = [&](int32_t j) {
-            const uint32_t buf = (uint32_t)(j & 1);
-            wait_all(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1));
-            if (dead()) return;
-            if (lane == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint64_t a = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
-                    const uint64_t b = smem_desc(base + SM::OFF_K + buf * SM::KV_BYTES + (ks >> 2) * (PF_KV * 128) + (ks & 3) * 32, 16, 1024);
-                    mma_f16(tmem + buf * PF_KV, a, b, IDESC_S, ks > 0 ? 1u : 0u);
-                }
-                tc_commit(bar_s + 8 * buf);
-            }
-            __syncwarp();
+            (v_rows ? last_v : last_k)[buf] = j;
         };
         for (int32_t j = 0; j < min(n_stages, 2); ++j) {
             issue_tiles(j, false);
             issue_tiles(j, true);
         }
+        __syncthreads();   // (Q is in shared memory: nothing of this warp's depends on it)
+        // look-ups in flight across iterations: lanes 0 .. 3 hold the slot of a block of stage j + 4 and the id of one of
+        // stage j + 5; their loads are issued in one iteration and used in the next
+        int32_t slot_pend = -1, blk_pend = -1;
+        if (lane < 4) {
+            slot_pend = load_slot(load_blk(4, lane));
+            blk_pend = load_blk(5, lane);
+        }
+        for (int32_t j = 0; j < n_stages; ++j) {
+            if (lane < 4) {
+                store_slot(j + 4, lane, slot_pend);
+                slot_pend = load_slot(blk_pend);
+                blk_pend = load_blk(j + 6, lane);
+            }
+            __syncwarp();
+            if (dead()) break;
+            if (j + 2 < n_stages) {
+                wait_all(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1));
+                if (dead()) break;
+                issue_tiles(j + 2, false);
+            }
+            if (j >= 1 && j + 1 < n_stages) {
+                wait_all(bar_o2 + 8 * ((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1));
+                if (dead()) break;
+                issue_tiles(j + 1, true);
+            }
+        }
+        if (dead()) {
+            // giving up: the copies already issued still write into this CTA's shared memory - wait (bounded) for them
+            for (int b2 = 0; b2 < 2; ++b2) {
+                if (last_k[b2] >= 0) pf_mbar_wait(bar_k + 8 * b2, (uint32_t)((last_k[b2] >> 1) & 1));
+                if (last_v[b2] >= 0) pf_mbar_wait(bar_v + 8 * b2, (uint32_t)((last_v[b2] >> 1) & 1));
+            }
+        }
+        __syncwarp();
+    } else if (warp == 4) {
+        // =============================================================================== the issuing warp
+        // (operand descriptors are formed by the whole warp, outside the branch of the lane that issues: values every lane
+        // holds alike can live in the uniform registers the MMA instruction takes its operands from)
+        uint64_t q_desc[D / 16];
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) q_desc[ks] = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
+        // S(j) = Q K(j)^T into the stage's half of the score columns (K(j) must have landed)
+        auto issue_qk = [&](int32_t j) {
+            const uint32_t buf = (uint32_t)(j & 1);
+            wait_all(bar_k + 8 * buf, (uint32_t)((j >> 1) & 1));
+            if (dead()) return;
+            uint64_t k_desc[D / 16];
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+                k_desc[ks] = smem_desc(base + SM::OFF_K + buf * SM::KV_BYTES + (ks >> 2) * (PF_KV * 128) + (ks & 3) * 32, 16, 1024);
+            const uint32_t d_addr = tmem + buf * PF_KV;
+            if (lane == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) mma_f16(d_addr, q_desc[ks], k_desc[ks], IDESC_S, ks > 0 ? 1u : 0u);
+                tc_commit(bar_s + 8 * buf);
+            }
+            __syncwarp();
+        };
         __syncthreads();   // Q is in shared memory
         if (n_stages > 0) issue_qk(0);
         // Software pipeline: while the four softmax warps work on the scores of stage j, the tensor core computes those of
         // stage j + 1 (into the other half of the score columns) and, before that, finishes O += P V of stage j - 1.
         for (int32_t j = 0; j < n_stages; ++j) {
-            if (lane >= 4 && lane < 8 && j + 3 < n_stages) resolve(j + 3, lane - 4);   // read from the next iteration on
-            __syncwarp();
             if (dead()) break;
             const uint32_t buf = (uint32_t)(j & 1);
-            // S(j) is complete (the softmax warps wait for the same barrier): its K buffer is free, and the K tiles of
-            // stage j + 2 go there now, two stages ahead of their use
-            if (j + 2 < n_stages) {
-                wait_all(bar_s + 8 * buf, (uint32_t)((j >> 1) & 1));
-                if (dead()) break;
-                issue_tiles(j + 2, false);
-            }
-            // the other half of the score columns held P(j - 1), and stage j - 1's V buffer is the one stage j + 1
-            // needs: O += P V of stage j - 1 must have completed
+            // the other half of the score columns held P(j - 1): O += P V of stage j - 1 must have completed
             if (j >= 1) {
-                wait_all(bar_o, (uint32_t)((j - 1) & 1));
+                wait_all(bar_o2 + 8 * ((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1));
                 if (dead()) break;
             }
             if (j + 1 < n_stages) {
-                if (j >= 1) issue_tiles(j + 1, true);
                 issue_qk(j + 1);
                 if (dead()) break;
             }
@@ -367,17 +409,20 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
             wait_all(bar_p2[buf], (uint32_t)((j >> 1) & 1));
             wait_all(bar_v + 8 * buf, (uint32_t)((j >> 1) & 1));
             if (dead()) break;
+            // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
+            uint64_t v_desc[PF_KV / 16];
+#pragma unroll
+            for (int ks = 0; ks < PF_KV / 16; ++ks) v_desc[ks] = smem_desc(base + SM::OFF_V + buf * SM::KV_BYTES + ks * 2048, PF_KV * 128, 1024);
+            const uint32_t tmem_sj = tmem + buf * PF_KV;
+            const uint32_t acc0 = j > 0 ? 1u : 0u;
             if (lane == 0) {
                 tc_fence_after();
-                const uint32_t tmem_sj = tmem + buf * PF_KV;
 #pragma unroll
                 for (int ks = 0; ks < PF_KV / 16; ++ks) {
-                    // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PF_KV * 128 bytes apart
-                    const uint64_t b = smem_desc(base + SM::OFF_V + buf * SM::KV_BYTES + ks * 2048, PF_KV * 128, 1024);
-                    mma_f16_ts(tmem_o, tmem_sj + ks * 8, b, IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
-                    if (BF16) mma_f16_ts(tmem_o, tmem_sj + 32 + ks * 8, b, IDESC_O, 1u);
+                    mma_f16_ts(tmem_o, tmem_sj + ks * 8, v_desc[ks], IDESC_O, ks > 0 ? 1u : acc0);
+                    if (BF16) mma_f16_ts(tmem_o, tmem_sj + 32 + ks * 8, v_desc[ks], IDESC_O, 1u);
                 }
-                tc_commit(bar_o);
+                tc_commit(bar_o2 + 8 * buf);
                 if (j + 1 == n_stages) tc_commit(bar_done);   // O is final
             }
             __syncwarp();
@@ -479,7 +524,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
             if (BF16) tmem_st32(tmem_sj + lane_addr + 32, pl);
             // ---- O *= alpha where a row's maximum moved (skipped by warps in which none did); O += P V of stage j - 1 first
             if (j >= 1 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                if (!pf_mbar_wait(bar_o, (uint32_t)((j - 1) & 1))) {
+                if (!pf_mbar_wait(bar_o2 + 8 * ((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1))) {
                     pf_raise(p.status, STATUS_WAIT_TIMEOUT);
                     misc[1] = 1;
                 }
