@@ -36,7 +36,7 @@ from paper_2411_09317_b200 import synth  # noqa: E402
 WORKLOAD = "llama2_7b"
 # dram__bytes_read + dram__bytes_write per algorithmic byte of the attention kernel, from the ncu capture summarised in
 # profiles/paged_decode_attn_llama2_7b_quarter.md (quarter-scale case; traffic grows in proportion to the KV bytes)
-TRAFFIC_PER_ALG_BYTE = 1.021
+TRAFFIC_PER_ALG_BYTE = 1.023
 METRIC = "paged decode-attn GB/s over whole decode steps with the swap path running at the largest ratio found inside 2% slow-down"
 
 
