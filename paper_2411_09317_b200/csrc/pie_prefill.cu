@@ -10,16 +10,22 @@
 // token-major, so a tile holds 128 / G tokens; the rows of a tile share every K and V tile they read, which is what makes
 // this a dense contraction: 128 rows per K and V tile against the decode kernel's G.  Per 64-token stage (four
 // 16-token blocks of the paged pool):
-//   - thread 0 issues the TMA copies of the blocks' K and V rows (two-dimensional tiles of 16 rows x 64 elements,
-//     128-byte swizzle, straight into the layout the tensor core's shared-memory descriptors expect: K as the K-major
-//     B operand of S = Q K^T, V as the MN-major B operand of O += P V), double buffered;
-//   - thread 0 issues D / 16 MMAs of shape 128 x 64 x 16 for S (fp32, 64 TMEM columns) and commits them to an mbarrier;
-//   - the four warps read their 32 rows of S from TMEM (a thread holds one whole row: the softmax needs no shuffles),
-//     apply the causal mask by selection, update the running maximum and sum, write P in the 16-bit type to shared
-//     memory as the next MMA's A operand, and rescale O in TMEM where a row's maximum moved;
-//   - thread 0 issues four MMAs of shape 128 x D x 16 for O += P V (fp32, D TMEM columns).
+//   - the loading warp (warp 5) resolves the blocks' slots several stages ahead and issues the TMA copies of their K and V
+//     rows, eight lanes at once (two-dimensional tiles of 16 rows x 64 elements, 128-byte swizzle, straight into the layout
+//     the tensor core's shared-memory descriptors expect: K as the K-major B operand of S = Q K^T, V as the MN-major B
+//     operand of O += P V), double buffered: K(j + 2) once S(j) is complete, V(j + 1) once O += P V of stage j - 1 is;
+//   - one thread of the issuing warp (warp 4) issues D / 16 MMAs of shape 128 x 64 x 16 for S (fp32, 64 TMEM columns, two
+//     buffers: the scores of stage j + 1 are computed while the softmax of stage j runs) and commits them to an mbarrier;
+//   - the four softmax warps read their 32 rows of S from TMEM (a thread holds one whole row: the softmax needs no
+//     shuffles), apply the causal mask by selection, update the running maximum (lazily) and the sum, write P in the 16-bit
+//     type back over the scores in TMEM as the next MMA's A operand, and rescale O in TMEM where a row's maximum moved;
+//   - the issuing thread issues four MMAs (bf16: eight, the second operand carrying P's rounding remainder) of shape
+//     128 x D x 16 for O += P V (fp32, D TMEM columns), A operand from TMEM.
 // At the end every thread reads its row of O, divides by the row's sum and stores the 16-bit result.
-// Every wait is bounded; a wait that runs out raises the status word, and the CTA still frees its TMEM before it leaves.
+// Every mbarrier exists once per stage parity and the end of the last product has a barrier of its own (a parity wait may
+// be at most one phase behind, and the warps run at their own pace).  Every wait is bounded; a wait that runs out raises
+// the status word, the loading warp waits (bounded) for its copies in flight, and the CTA still frees its TMEM before it
+// leaves.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
