@@ -40,7 +40,7 @@ def main(argv=None):
     ap.add_argument("--seqs", type=int, default=128)
     ap.add_argument("--ctx", type=int, default=4096)
     ap.add_argument("--swap-ctas", type=int, default=0)
-    ap.add_argument("--part", default="12")
+    ap.add_argument("--part", default="12", help="1 swap alone, 2 behind attention, 3 prefill-side write, 4 pairings of movers for the two directions")
     ap.add_argument("--q-heads", type=int, default=32)
     ap.add_argument("--kv-heads", type=int, default=8)
     ap.add_argument("--fp16", action="store_true", help="fp16 instead of bf16")
@@ -190,6 +190,35 @@ def main(argv=None):
         # K and V rows read once (16-bit) and written once (16-bit, or one byte per value into an 8-bit pool)
         nbytes = 2 * T * wl.n_kv_heads * wl.head_dim * (2 + (1 if wl.kv_fp8 else 2))
         emit({"part": "kv_write", "tokens": T, "ms": ms, "gbs_read_plus_write": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes})
+    # ---------------------------------------------------------------- part 4: both directions at once, every pairing of who moves
+    # which direction (does host traffic issued by SMs slow the other direction down, whoever moves that one?)
+    if "4" in args.part:
+        n = 4096 if not args.quick else 1024
+        modes = {"bulk_kernel": pie.PIE_MODE_KERNEL_BULK, "kernel": pie.PIE_MODE_KERNEL, "copy_engine": pie.PIE_MODE_COPY_ENGINE}
+        for pattern in ("contiguous", "scattered"):
+            src, dst = swap_lists(n, pattern, n_swap_slots, 100 + n)
+            for m_in in (None, "bulk_kernel", "kernel", "copy_engine"):
+                for m_out in (None, "bulk_kernel", "kernel", "copy_engine"):
+                    if m_in is None and m_out is None:
+                        continue
+                    best = None
+                    for r in range(4):
+                        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                        torch.cuda.synchronize()
+                        e0.record(s_in)
+                        s_out.wait_event(e0)
+                        if m_in:
+                            pie.pie_swap_raw(dw.pool, pie.PIE_H2D, src + host_lo, dst + gpu_lo, modes[m_in], s_in.cuda_stream)
+                        e1.record(s_in)
+                        if m_out:
+                            pie.pie_swap_raw(dw.pool, pie.PIE_D2H, src + gpu_lo, dst + host_lo, modes[m_out], s_out.cuda_stream)
+                        e2.record(s_out)
+                        torch.cuda.synchronize()
+                        ms = max(e0.elapsed_time(e1), e0.elapsed_time(e2))
+                        if r > 0:
+                            best = ms if best is None else min(best, ms)
+                    emit({"part": "swap_pairings", "pattern": pattern, "blocks": n, "in": m_in, "out": m_out, "swap_ctas": args.swap_ctas,
+                          "gbs_per_dir": n * BB / (best * 1e-3) / 1e9})
     dw.close()
 
 
