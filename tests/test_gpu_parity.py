@@ -428,6 +428,34 @@ def test_layer_by_layer_loop_with_other_work_in_between_equals_the_whole_step():
     assert np.array_equal(a[2], b[2]) and a[3] == b[3] > 0 and a[4] == b[4] > 0
 
 
+@pytest.mark.parametrize("hq,hkv,d,dtype,layers", [(8, 1, 128, BF16, 5), (4, 4, 64, F16, 2), (8, 2, 128, F16, 3)])
+def test_split_k_merge_in_the_next_layers_kernel_equals_the_combine_kernel(hq, hkv, d, dtype, layers):
+    """Inside pie_decode_step a layer's split-K partials are merged by the NEXT layer's attention kernel (in the tail of its
+    launch); pie_decode_layer and the last layer of a step use the combine kernel.  Sequences of one to a dozen chunks (and
+    an empty one), group sizes 1, 4 and 8, odd and even layer counts: the same bits either way, and the oracle's values."""
+    from paper_2411_09317_b200.harness import DeviceWorkload
+    lens = np.array([700, 33, 0, 64, 65, 511, 129, 1], dtype=np.int32)
+    wl = synth.Workload("merge", 72, layers, hq, hkv, d, dtype, lens, 3, 0.3)
+    runs = []
+    for manual in (False, True):
+        dw = DeviceWorkload(wl, timing=True, split_tokens=64)
+        scratch = torch.zeros(1 << 16, dtype=torch.float32, device=dw.dev)
+        outs = []
+        for step in range(3):
+            dw.advance_context()
+            dw.decode_step(between_layers=(lambda l: scratch.add_(1.0)) if manual else None)
+            dw.sync()
+            outs.append(dw.out_bits().copy())
+        runs.append(outs)
+        if not manual:
+            from tests.test_gpu_fullsize import check_samples
+            # a layer whose merge was deferred and the last one, the longest sequence and two short ones, after three steps
+            check_samples(dw, [(0, 0), (layers - 1, 0), (0, 5), (layers - 1, 6), (0, 7)], 3)
+        dw.close()
+    for x, y in zip(*runs):
+        assert np.array_equal(x, y)
+
+
 def test_kept_host_slots_are_given_back_when_units_leave_the_host_resident_set():
     """Kept host copies hold host slots while their units are on the GPU.  When the ratio drops, the units that leave the
     host-resident set must give those slots up: afterwards the whole host pool can be allocated again."""
