@@ -95,6 +95,44 @@ def test_tail_garbage_and_future_tokens_do_not_leak():
     pc_clean.close()
 
 
+def test_several_waves_of_tiles_sampled_against_the_decode_oracle():
+    """More CTAs than the GPU holds at once (fourteen sequences x sixteen tiles x two KV heads), chunks of 512 tokens behind
+    1536 cached ones, 32 stages per tile: the warps of a CTA run at their own pace here (softmax warps a stage apart, the
+    loading warp behind or ahead of the issuing one).  Sampled rows - first, last and seeded tokens of the chunks - against
+    single-token calls of the decode oracle at the token's own context length; every row finite."""
+    n_seqs, prefix, chunk = 14, 1536, 512
+    ctx = [prefix + chunk] * (n_seqs - 2) + [prefix + chunk - 7, 40 + chunk]
+    case = Case(1, 8, 2, 128, BF16, ctx, seed=68, host_frac=0.0, placement="random")
+    pc = PoolCase(case, all_on_gpu=True)
+    chunks = [chunk] * n_seqs
+    off = np.concatenate([[0], np.cumsum(chunks)]).astype(np.int32)
+    n_tok = int(off[-1])
+    q = synth.tensor_bits(19, synth.STREAM_Q, (n_tok, case.Hq, case.D), case.dtype)
+    dev = torch.device("cuda:0")
+    q_dev = torch.from_numpy(q.view(np.int16)).to(dev)
+    out_dev = torch.full_like(q_dev, 0x7fc0)
+    off_dev = torch.from_numpy(off).to(dev)
+    ctx_np = np.asarray(ctx, dtype=np.int32)
+    ctx_dev = torch.from_numpy(ctx_np).to(dev)
+    for _ in range(3):      # (repeated: the failure this guards against depended on timing)
+        pie.pie_prefill_attention(pc.pool, 0, q_dev.data_ptr(), out_dev.data_ptr(), pc.bt.data_ptr(), case.block_table.shape[1],
+                                  ctx_dev.data_ptr(), off_dev.data_ptr(), ctx_np, off, n_seqs, case.scale)
+    pie.pie_sync(pc.pool)
+    got = synth.bits16_to_f32(out_dev.cpu().numpy().view(np.uint16), case.dtype)
+    assert np.all(np.isfinite(got))
+    rng = np.random.default_rng(5)
+    samples = [(0, 0), (0, chunk - 1), (n_seqs - 1, 0), (n_seqs - 1, chunk - 1), (n_seqs - 2, 255), (5, 31), (5, 32), (7, 480)]
+    samples += [(int(rng.integers(0, n_seqs)), int(rng.integers(0, chunk))) for _ in range(8)]
+    for s, i in samples:
+        pos = ctx[s] - chunk + i
+        want = oracle.paged_attention(case.gpu_pool, case.host_pool, case.unit_side[0], case.unit_slot[0], q[off[s] + i][None],
+                                      case.block_table[s:s + 1], np.array([pos + 1], np.int32), case.Hq, case.Hkv, case.D,
+                                      case.dtype, case.scale, "f64")[0]
+        err = np.abs(got[off[s] + i] - want)
+        assert np.all(err <= tolerance(want, case.dtype)), (s, i, float(err.max()))
+    pc.close()
+
+
 def test_rejected_arguments_enqueue_nothing():
     case = Case(1, 4, 2, 128, F16, [64, 64], seed=65, host_frac=0.0, placement="identity")
     pc = PoolCase(case, all_on_gpu=True)
