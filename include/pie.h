@@ -324,7 +324,8 @@ int pie_kv_write(pie_pool *pool, int32_t layer, const void *k, const void *v, co
  * longer than its context or a context beyond the table is PIE_ERR_INVALID.  Enqueued on the compute stream behind every
  * copy still bringing a unit of the layer in; every unit read must be GPU resident (a missing one raises the device
  * status word: the next call returns PIE_ERR_NOT_RESIDENT).  The kernel runs on the tcgen05 tensor cores with its
- * accumulators in tensor memory: 128 query rows (128 / group tokens) per CTA.  16-bit pools only (PIE_ERR_UNSUPPORTED). */
+ * accumulators in tensor memory: 128 query rows (128 / group tokens) per CTA, streamed against the context in stages of 64
+ * (bf16 pools) or 128 (fp16 pools) tokens.  16-bit pools only (PIE_ERR_UNSUPPORTED). */
 int pie_prefill_attention(pie_pool *pool, int32_t layer, const void *q, void *out, const int32_t *block_table_dev,
                           int32_t max_blocks_per_seq, const int32_t *ctx_lens_dev, const int32_t *q_offsets_dev,
                           const int32_t *ctx_lens_host, const int32_t *q_offsets_host, int32_t n_seqs, float scale);

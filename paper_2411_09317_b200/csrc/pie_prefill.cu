@@ -604,9 +604,420 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParam
     if (warp == 4) tmem_dealloc(tmem, PF_TMEM_COLS);
 }
 
+// ---------------------------------------------------------------------------------------------------------------------
+// The same tile with stages of 128 KV tokens and ONE score buffer of 128 columns (fp16 pools).  A stage's scores are then
+// eight MMAs of 128 x 128 x 16: the Q tile is re-read from shared memory half as often per token as with 64-token stages,
+// which is what held the tensor pipe.  A CTA's stages run strictly one after the other - S(j), softmax(j), O += P V (j),
+// then S(j + 1) over the columns P(j) lay in - and the overlap comes from the SM's other CTA: while one CTA's warps do
+// the softmax, the other's MMAs run.  K and V need one buffer each (K(j + 1) is loaded during the softmax and O += P V
+// of stage j, V(j + 1) during the scores and the softmax of stage j + 1).  The softmax takes a row's 128 scores in two
+// halves of 64 and in two passes (the maximum, then the probabilities: a thread cannot hold the whole row).  bf16 pools
+// keep the 64-token kernel above: with their second P operand O += P V is sixteen MMAs per stage, and strictly serial
+// stages lose more there than the wider score tile gains (602 against 642 TFLOP/s; fp16: 816 against 698).
+constexpr int PFW_KV = 128;
+constexpr int PFW_TMEM_COLS = 256;
+
+template <int D>
+struct PfSmemWide {
+    static constexpr int Q_BYTES = PF_M * D * 2;        // [D / 64][128 rows][128 B]
+    static constexpr int KV_BYTES = PFW_KV * D * 2;      // [D / 64][128 tokens][128 B]
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + Q_BYTES;       // one stage
+    static constexpr int OFF_V = OFF_K + KV_BYTES;      // one stage
+    static constexpr int OFF_BAR = OFF_V + KV_BYTES;    // k_full, v_full, s_done, o_done, p_done, done
+    static constexpr int OFF_MISC = OFF_BAR + 128;      // [0] TMEM base, [1] abort, [4 .. 35] slots of eight stages' blocks
+    static constexpr int BYTES = OFF_MISC + 256;        // two CTAs per SM (with TMEM for two: 2 x 256 of 512 columns)
+};
+
+template <int D, bool BF16>
+__global__ void __launch_bounds__(PF_THREADS)
+prefill_attn_wide_kernel(const __grid_constant__ CUtensorMap tmap, const PrefillParams p) {
+    using SM = PfSmemWide<D>;
+    constexpr int HALVES = D / 64;
+    extern __shared__ __align__(1024) uint8_t pf_smem[];
+    uint8_t *smem = pf_smem;
+    const uint32_t base = pf_smem_u32(pf_smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (base & 1023u) {   // the swizzled tiles need a 1024-byte boundary: never seen otherwise, but do not compute garbage
+        if (tid == 0) pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+        return;
+    }
+    // One barrier of each kind, phase = stage parity.  A CTA's stages run one after the other - S(j), softmax(j), O += P V
+    // (j), then S(j + 1) over the same columns - so no waiter can fall two phases behind the barrier it waits on: the next
+    // phase of each needs what the waiter does after its wait.  (The overlap comes from the SM's other CTA: while one
+    // CTA's warps do the softmax, the other's MMAs run.)
+    const uint32_t bar_k = base + SM::OFF_BAR, bar_v = bar_k + 8, bar_s = bar_k + 16, bar_o = bar_k + 24, bar_p = bar_k + 32;
+    const uint32_t bar_done = bar_k + 40;   // O is final (used once: the softmax warps do not follow bar_o)
+    volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + SM::OFF_MISC);
+
+    // ---- which tile
+    const int32_t item = blockIdx.x;
+    const int32_t tile_g = item / p.n_kv_heads, kvh = item - tile_g * p.n_kv_heads;
+    int32_t lo = 0, hi = p.n_seqs;  // largest s with tile_off[s] <= tile_g
+    while (hi - lo > 1) {
+        const int32_t mid = (lo + hi) >> 1;
+        if (__ldg(p.tile_off + mid) <= tile_g) lo = mid;
+        else hi = mid;
+    }
+    const int32_t s = lo;
+    const int32_t G = p.group, tile_tokens = PF_M / G;
+    const int32_t q0 = __ldg(p.q_offsets + s), C = __ldg(p.q_offsets + s + 1) - q0;
+    const int32_t ctx = min(__ldg(p.ctx_lens + s), p.max_blocks * 16);
+    const int32_t tok0 = (tile_g - __ldg(p.tile_off + s)) * tile_tokens;   // first chunk token of the tile
+    const int32_t ntok = min(tile_tokens, C - tok0);
+    const int32_t p0 = ctx - C;                                            // tokens cached before the chunk
+    const int32_t kv_len = p0 + tok0 + ntok;                               // what the tile's last token sees
+    const bool bad = C > ctx || ntok <= 0;                                 // (flagged by the host where it has the lengths)
+    const int32_t n_stages = bad ? 0 : (kv_len + PFW_KV - 1) / PFW_KV;
+
+    if (tid == 0) {
+        for (int i = 0; i < 4; ++i) pf_mbar_init(bar_k + 8 * i, 1);   // k_full, v_full, s_done, o_done
+        pf_mbar_init(bar_p, PF_ROWS_THREADS);                          // P of a stage is in place: every row's thread arrives
+        pf_mbar_init(bar_done, 1);
+        misc[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(base + SM::OFF_MISC, PFW_TMEM_COLS);
+    // ---- block table -> slot table -> slot: lanes of the loading warp resolve the blocks of a stage well ahead of the
+    // stage's copies into a ring in shared memory (two dependent global loads each; done serially by the thread that
+    // issues the copies they cost ten microseconds per stage)
+    volatile int32_t *slot_ring = reinterpret_cast<volatile int32_t *>(smem + SM::OFF_MISC + 16);   // [4 stages][8 blocks]
+    const int32_t n_blocks = (kv_len + 15) / 16;
+    auto load_blk = [&](int32_t j, int32_t i) -> int32_t {   // the block's logical id, -1: the stage has no such block
+        const int32_t b = j * (PFW_KV / 16) + i;
+        if (j >= n_stages || b >= n_blocks) return -1;
+        const int32_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + b);
+        return blk < 0 ? p.n_logical : blk;   // an id that names nothing is a missing unit, not a missing block
+    };
+    auto load_slot = [&](int32_t blk) -> int32_t {           // its slot, -2: no such unit on the GPU
+        if (blk < 0) return -1;
+        const int32_t v = blk < p.n_logical ? __ldcg(p.slot_table + blk) : -2;
+        return v < 0 ? -2 : v;
+    };
+    auto store_slot = [&](int32_t j, int32_t i, int32_t slot) {
+        if (slot < -1 || slot >= p.n_gpu_slots) {  // unit not on the GPU: flag it, stream slot 0 so the barriers complete
+            pf_raise(p.status, STATUS_MISSING_UNIT);
+            slot = 0;
+        }
+        slot_ring[(j & 3) * 8 + i] = slot;
+    };
+    if (warp == 5 && lane < 16) store_slot(lane >> 3, lane & 7, load_slot(load_blk(lane >> 3, lane & 7)));   // stages 0 and 1
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc[0];
+    const uint32_t tmem_o = tmem + PFW_KV;   // S (and then P): columns 0 .. 127; O: 128 .. 128 + D - 1
+    constexpr uint32_t IDESC_S = instr_desc(BF16, PFW_KV, false), IDESC_O = instr_desc(BF16, D, true);
+
+    // ---- Q: thread r brings row r (token tok0 + r / G, head kvh * G + r % G) into the K-major swizzled layout
+    const int r = tid;
+    const int32_t my_tok = r / G, my_g = r - my_tok * G;
+    const bool row_valid = !bad && tid < PF_ROWS_THREADS && my_tok < ntok;
+    if (tid < PF_ROWS_THREADS) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+            const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4 *>(smem + SM::OFF_Q + (c >> 3) * (PF_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+
+    auto dead = [&]() { return __shfl_sync(0xffffffffu, misc[1] != 0 ? 1 : 0, 0) != 0; };
+    auto wait_all = [&](uint32_t bar, uint32_t parity) {   // by every lane of a warp
+        if (!pf_mbar_wait(bar, parity)) {
+            pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+            misc[1] = 1;
+        }
+        __syncwarp();
+    };
+    if (warp == 5) {
+        // =============================================================================== the loading warp
+        // A stage's K (or V) tiles - one TMA copy per (block, 64-element half), up to sixteen - are issued by as many lanes
+        // at once.  K(j + 1) goes out as soon as the scores of stage j are complete (the buffer is free then: the softmax and
+        // O += P V of stage j give it time to land), V(j + 1) as soon as O += P V of stage j is.  The TMA unit takes a stage's
+        // 32 KiB at its own pace (the issue blocks meanwhile), which is why this is a warp of its own.
+        int32_t last_k = -1, last_v = -1;   // newest stage issued into each buffer
+        auto issue_tiles = [&](int32_t j, bool v_rows) {
+            const uint32_t bar = v_rows ? bar_v : bar_k;
+            const uint32_t dst0 = base + (v_rows ? SM::OFF_V : SM::OFF_K);
+            const int32_t nb = min(PFW_KV / 16, n_blocks - j * (PFW_KV / 16));
+            if (lane == 0) pf_mbar_expect_tx(bar, (uint32_t)nb * 16u * D * 2u);
+            __syncwarp();
+            const int32_t i = lane / HALVES, h = lane - i * HALVES;
+            if (i < nb) {
+                const int32_t row0 = (slot_ring[(j & 3) * 8 + i] * p.n_kv_heads + kvh) * 32 + (v_rows ? 16 : 0);
+                pf_tma_2d(dst0 + h * (PFW_KV * 128) + i * 2048, &tmap, h * 64, row0, bar);
+            }
+            __syncwarp();
+            (v_rows ? last_v : last_k) = j;
+        };
+        if (n_stages > 0) {
+            issue_tiles(0, false);
+            issue_tiles(0, true);
+        }
+        __syncthreads();   // (Q is in shared memory: nothing of this warp's depends on it)
+        // look-ups in flight across iterations: lanes 0 .. 7 hold the slot of a block of stage j + 2 and the id of one of
+        // stage j + 3; their loads are issued in one iteration and used in the next
+        int32_t slot_pend = -1, blk_pend = -1;
+        if (lane < 8) {
+            slot_pend = load_slot(load_blk(2, lane));
+            blk_pend = load_blk(3, lane);
+        }
+        for (int32_t j = 0; j < n_stages; ++j) {
+            if (lane < 8) {
+                store_slot(j + 2, lane, slot_pend);
+                slot_pend = load_slot(blk_pend);
+                blk_pend = load_blk(j + 4, lane);
+            }
+            __syncwarp();
+            if (dead() || j + 1 >= n_stages) break;
+            wait_all(bar_s, (uint32_t)(j & 1));
+            if (dead()) break;
+            issue_tiles(j + 1, false);
+            wait_all(bar_o, (uint32_t)(j & 1));
+            if (dead()) break;
+            issue_tiles(j + 1, true);
+        }
+        if (dead()) {
+            // giving up: the copies already issued still write into this CTA's shared memory - wait (bounded) for them
+            if (last_k >= 0) pf_mbar_wait(bar_k, (uint32_t)(last_k & 1));
+            if (last_v >= 0) pf_mbar_wait(bar_v, (uint32_t)(last_v & 1));
+        }
+        __syncwarp();
+    } else if (warp == 4) {
+        // =============================================================================== the issuing warp
+        // (operand descriptors are formed by the whole warp, outside the branch of the lane that issues: values every lane
+        // holds alike can live in the uniform registers the MMA instruction takes its operands from)
+        uint64_t q_desc[D / 16];
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) q_desc[ks] = smem_desc(base + SM::OFF_Q + (ks >> 2) * (PF_M * 128) + (ks & 3) * 32, 16, 1024);
+        // S(j) = Q K(j)^T (K(j) must have landed)
+        auto issue_qk = [&](int32_t j) {
+            wait_all(bar_k, (uint32_t)(j & 1));
+            if (dead()) return;
+            uint64_t k_desc[D / 16];
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) k_desc[ks] = smem_desc(base + SM::OFF_K + (ks >> 2) * (PFW_KV * 128) + (ks & 3) * 32, 16, 1024);
+            if (lane == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) mma_f16(tmem, q_desc[ks], k_desc[ks], IDESC_S, ks > 0 ? 1u : 0u);
+                tc_commit(bar_s);
+            }
+            __syncwarp();
+        };
+        __syncthreads();   // Q is in shared memory
+        if (n_stages > 0) issue_qk(0);
+        // V: 16 tokens (two groups of eight rows) further per step; 64-element chunks of D are PFW_KV * 128 bytes apart
+        uint64_t v_desc[PFW_KV / 16];
+#pragma unroll
+        for (int ks = 0; ks < PFW_KV / 16; ++ks) v_desc[ks] = smem_desc(base + SM::OFF_V + ks * 2048, PFW_KV * 128, 1024);
+        for (int32_t j = 0; j < n_stages; ++j) {
+            if (dead()) break;
+            // P(j) is in tensor memory (every row's thread has arrived) and V(j) has landed: O += P V.  P of the stage's
+            // half h lies where the half's scores were: 32 columns of 16-bit pairs (bf16: 32 more with the remainders)
+            wait_all(bar_p, (uint32_t)(j & 1));
+            wait_all(bar_v, (uint32_t)(j & 1));
+            if (dead()) break;
+            const uint32_t acc0 = j > 0 ? 1u : 0u;
+            if (lane == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < PFW_KV / 16; ++ks) {
+                    const uint32_t a_addr = tmem + (ks >> 2) * 64 + (ks & 3) * 8;
+                    mma_f16_ts(tmem_o, a_addr, v_desc[ks], IDESC_O, ks > 0 ? 1u : acc0);
+                    if (BF16) mma_f16_ts(tmem_o, a_addr + 32, v_desc[ks], IDESC_O, 1u);
+                }
+                tc_commit(bar_o);
+                if (j + 1 == n_stages) tc_commit(bar_done);   // O is final
+            }
+            __syncwarp();
+            if (j + 1 < n_stages) {
+                // the scores of the next stage go where P(j) lies: O += P V of stage j must have completed
+                wait_all(bar_o, (uint32_t)(j & 1));
+                if (dead()) break;
+                issue_qk(j + 1);
+            }
+        }
+        __syncwarp();
+    } else {
+        // =============================================================================== the softmax warps
+        __syncthreads();   // Q is in shared memory
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const int32_t my_pos = p0 + tok0 + my_tok;   // this row's position: it sees tokens 0 .. my_pos
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int32_t j = 0; j < n_stages; ++j) {
+            // ---- the scores of stage j: 128 columns, taken in two halves of 64 (a thread holds one half of its row at a time)
+            if (!pf_mbar_wait(bar_s, (uint32_t)(j & 1))) {
+                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                misc[1] = 1;
+            }
+            if (__any_sync(0xffffffffu, misc[1] != 0)) { ok = false; break; }
+            tc_fence_after();
+            const int32_t t_base = j * PFW_KV;
+            // Every row of the tile sees every token of the stage (all stages but the last one or two of a tile): no mask, and
+            // the softmax is written for the instruction count - the maximum over the raw scores (four chains), one fused
+            // multiply-add and one ex2 per element, sums in four chains over the unrounded probabilities (they differ from
+            // what the tensor core sees by the operand's rounding, 2^-12 or 2^-17 relative: nothing beside 2e-3).
+            const bool plain = t_base + PFW_KV - 1 <= p0 + tok0 && p.scale_log2e > 0.f;
+            // ---- first pass: the row's maximum over the stage
+            float mx = -INFINITY;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t sv[2][32];
+                tmem_ld32(tmem + lane_addr + 64 * h, sv[0]);
+                tmem_ld32(tmem + lane_addr + 64 * h + 32, sv[1]);
+                tmem_wait_ld();
+                if (plain) {
+                    float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 64; c += 4) {
+                        a0 = fmaxf(a0, __uint_as_float(sv[c >> 5][c & 31]));
+                        a1 = fmaxf(a1, __uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]));
+                        a2 = fmaxf(a2, __uint_as_float(sv[(c + 2) >> 5][(c + 2) & 31]));
+                        a3 = fmaxf(a3, __uint_as_float(sv[(c + 3) >> 5][(c + 3) & 31]));
+                    }
+                    mx = fmaxf(mx, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * p.scale_log2e);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) {
+                        const float x = __uint_as_float(sv[c >> 5][c & 31]) * p.scale_log2e;
+                        // masked by selection (NaN scores too)
+                        mx = fmaxf(mx, (row_valid && t_base + 64 * h + c <= my_pos) ? x : -INFINITY);
+                    }
+                }
+            }
+            const float m_cand = fmaxf(m_run, mx);
+            const bool grow = m_cand > m_run + PF_LAZY;   // (m_run = -inf: true unless the row has seen nothing yet)
+            const float m_new = grow ? m_cand : m_run;
+            const float alpha = grow ? pf_exp2(m_run - m_cand) : 1.f;   // (m_run = -inf gives 0: nothing accumulated yet)
+            // ---- second pass: P in the 16-bit type, two tokens per 32-bit word: the A operand of O += P V, kept in tensor
+            // memory where the half's scores were.  bf16 keeps 8 significant bits: the rounding remainder of P goes into a
+            // second bf16 operand, so that the product sees about 16 bits (fp16's 11 bits need no correction).
+            float sum = 0.f;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t sv[2][32];
+                tmem_ld32(tmem + lane_addr + 64 * h, sv[0]);
+                tmem_ld32(tmem + lane_addr + 64 * h + 32, sv[1]);
+                tmem_wait_ld();
+                uint32_t ph[32];
+                [[maybe_unused]] uint32_t pl[32];
+                if (plain) {
+                    const float neg_m = -m_new;
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 32; ++w) {
+                        const int c = 2 * w;
+                        const float e0 = pf_exp2(fmaf(__uint_as_float(sv[c >> 5][c & 31]), p.scale_log2e, neg_m));
+                        const float e1 = pf_exp2(fmaf(__uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]), p.scale_log2e, neg_m));
+                        ph[w] = pf_pack2<BF16>(e0, e1);
+                        if (BF16) pl[w] = pf_pack2<true>(e0 - __uint_as_float(ph[w] << 16), e1 - __uint_as_float(ph[w] & 0xffff0000u));
+                        if (w & 1) {
+                            s2 += e0;
+                            s3 += e1;
+                        } else {
+                            s0 += e0;
+                            s1 += e1;
+                        }
+                    }
+                    sum += (s0 + s1) + (s2 + s3);
+                } else {
+#pragma unroll
+                    for (int w = 0; w < 32; ++w) {
+                        const int c = 2 * w;
+                        const bool see0 = row_valid && t_base + 64 * h + c <= my_pos, see1 = row_valid && t_base + 64 * h + c + 1 <= my_pos;
+                        const float x0 = __uint_as_float(sv[c >> 5][c & 31]) * p.scale_log2e;
+                        const float x1 = __uint_as_float(sv[(c + 1) >> 5][(c + 1) & 31]) * p.scale_log2e;
+                        const float e0 = (see0 && m_new != -INFINITY) ? pf_exp2(x0 - m_new) : 0.f;
+                        const float e1 = (see1 && m_new != -INFINITY) ? pf_exp2(x1 - m_new) : 0.f;
+                        ph[w] = pf_pack2<BF16>(e0, e1);
+                        if (BF16) pl[w] = pf_pack2<true>(e0 - __uint_as_float(ph[w] << 16), e1 - __uint_as_float(ph[w] & 0xffff0000u));
+                        sum += e0 + e1;
+                    }
+                }
+                tmem_st32(tmem + lane_addr + 64 * h, ph);   // a thread overwrites only its own row's scores, which it has read
+                if (BF16) tmem_st32(tmem + lane_addr + 64 * h + 32, pl);
+            }
+            l_run = l_run * alpha + sum;
+            m_run = m_new;
+            // ---- O *= alpha where a row's maximum moved (skipped by warps in which none did).  O += P V of stage j - 1 is
+            // complete: this stage's scores were issued behind it.
+            if (j >= 1 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t ov[32];
+                    tmem_ld32(tmem_o + lane_addr + c0, ov);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+                    tmem_st32(tmem_o + lane_addr + c0, ov);
+                }
+            }
+            tmem_wait_st();
+            // ---- this stage's V has landed?  Rows of V beyond what the tile may see hold whatever was there (a tail
+            // block's garbage, an earlier stage): masked tokens are excluded, not multiplied by zero, so clear them before
+            // they meet P = 0
+            const int32_t n_seen = min(PFW_KV, kv_len - j * PFW_KV);
+            if (n_seen < PFW_KV) {
+                if (!pf_mbar_wait(bar_v, (uint32_t)(j & 1))) {
+                    pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                    misc[1] = 1;
+                }
+                for (int e = tid; e < (PFW_KV - n_seen) * HALVES * 8; e += PF_ROWS_THREADS) {
+                    const int row = n_seen + e / (HALVES * 8), rem = e % (HALVES * 8);
+                    *reinterpret_cast<uint4 *>(smem + SM::OFF_V + (rem >> 3) * (PFW_KV * 128) + row * 128 + ((rem & 7) << 4)) =
+                        make_uint4(0u, 0u, 0u, 0u);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+            tc_fence_before();
+            pf_mbar_arrive(bar_p);
+        }
+        if (ok && n_stages > 0) {
+            if (!pf_mbar_wait(bar_done, 0u)) {
+                pf_raise(p.status, STATUS_WAIT_TIMEOUT);
+                misc[1] = 1;
+            }
+            tc_fence_after();
+            ok = !__any_sync(0xffffffffu, misc[1] != 0);
+        }
+        // ---- out = O / l, rounded to the 16-bit type (nearest even).  The TMEM loads are warp-wide: rows beyond the chunk
+        // take part in them and store nothing.
+        if (ok && n_stages > 0) {
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((int64_t)(q0 + tok0 + my_tok) * p.n_q_heads + kvh * G + my_g) * D);
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t ov[32];
+                tmem_ld32(tmem_o + lane_addr + c0, ov);
+                tmem_wait_ld();
+                if (row_valid) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 v;
+                        v.x = pf_pack2<BF16>(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                        v.y = pf_pack2<BF16>(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                        v.z = pf_pack2<BF16>(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                        v.w = pf_pack2<BF16>(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                        dst[(c0 + c) >> 3] = v;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, PFW_TMEM_COLS);
+}
+
 }  // namespace
 
 int prefill_smem_bytes(int head_dim) { return head_dim == 128 ? PfSmem<128>::BYTES : PfSmem<64>::BYTES; }
+static int prefill_wide_smem_bytes(int head_dim) { return head_dim == 128 ? PfSmemWide<128>::BYTES : PfSmemWide<64>::BYTES; }
 
 // K and V rows of the pool as 16-row tiles: rows of head_dim elements, 32 per (slot, KV head): 16 of K, 16 of V.
 cudaError_t make_prefill_tensor_map(void *gpu_pool, int64_t n_gpu_slots, int n_kv_heads, int head_dim, CUtensorMap *map) {
@@ -629,9 +1040,11 @@ cudaError_t make_prefill_tensor_map(void *gpu_pool, int64_t n_gpu_slots, int n_k
 }
 
 cudaError_t prefill_configure(int head_dim, int dtype) {
-    const int smem = prefill_smem_bytes(head_dim);
-    const void *k = head_dim == 128 ? (dtype == PIE_BF16 ? (const void *)prefill_attn_kernel<128, true> : (const void *)prefill_attn_kernel<128, false>)
-                                    : (dtype == PIE_BF16 ? (const void *)prefill_attn_kernel<64, true> : (const void *)prefill_attn_kernel<64, false>);
+    // bf16 pools: stages of 64 tokens, two score buffers; fp16 pools: stages of 128 tokens, one score buffer
+    const bool wide = dtype != PIE_BF16;
+    const int smem = wide ? prefill_wide_smem_bytes(head_dim) : prefill_smem_bytes(head_dim);
+    const void *k = wide ? (head_dim == 128 ? (const void *)prefill_attn_wide_kernel<128, false> : (const void *)prefill_attn_wide_kernel<64, false>)
+                         : (head_dim == 128 ? (const void *)prefill_attn_kernel<128, true> : (const void *)prefill_attn_kernel<64, true>);
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -657,13 +1070,14 @@ cudaError_t launch_prefill_attention(const AttnShape &sh, const PrefillLaunch &a
     p.n_logical = sh.n_logical;
     p.scale_log2e = a.scale * 1.4426950408889634f;
     const unsigned grid = (unsigned)((int64_t)a.n_tiles * sh.n_kv_heads);
-    const int smem = prefill_smem_bytes(sh.head_dim);
-    if (sh.head_dim == 128) {
-        if (sh.dtype == PIE_BF16) prefill_attn_kernel<128, true><<<grid, PF_THREADS, smem, stream>>>(map, p);
-        else prefill_attn_kernel<128, false><<<grid, PF_THREADS, smem, stream>>>(map, p);
+    if (sh.dtype == PIE_BF16) {
+        const int smem = prefill_smem_bytes(sh.head_dim);
+        if (sh.head_dim == 128) prefill_attn_kernel<128, true><<<grid, PF_THREADS, smem, stream>>>(map, p);
+        else prefill_attn_kernel<64, true><<<grid, PF_THREADS, smem, stream>>>(map, p);
     } else {
-        if (sh.dtype == PIE_BF16) prefill_attn_kernel<64, true><<<grid, PF_THREADS, smem, stream>>>(map, p);
-        else prefill_attn_kernel<64, false><<<grid, PF_THREADS, smem, stream>>>(map, p);
+        const int smem = prefill_wide_smem_bytes(sh.head_dim);
+        if (sh.head_dim == 128) prefill_attn_wide_kernel<128, false><<<grid, PF_THREADS, smem, stream>>>(map, p);
+        else prefill_attn_wide_kernel<64, false><<<grid, PF_THREADS, smem, stream>>>(map, p);
     }
     return cudaGetLastError();
 }
