@@ -302,6 +302,30 @@ def test_large_batch_uses_the_separate_plan_kernel():
     pc.close()
 
 
+def test_large_batch_through_whole_decode_steps():
+    """The same beyond 1024 sequences through pie_decode_step: plan_kernel before every layer's attention kernel, the
+    split-K merge of a layer in the next layer's kernel, swaps in flight; against pie_decode_layer (combine kernel) bit for
+    bit and against the oracle on sampled sequences."""
+    from paper_2411_09317_b200.harness import DeviceWorkload
+    from tests.test_gpu_fullsize import check_samples
+    lens = synth.uniform_lengths(43, 1100, 0, 60)
+    lens[7], lens[500], lens[1099] = 200, 333, 64
+    wl = synth.Workload("many", 43, 3, 4, 2, 64, F16, lens, 2, 0.3)
+    runs = []
+    for manual in (False, True):
+        dw = DeviceWorkload(wl, timing=True, split_tokens=32)
+        scratch = torch.zeros(16, dtype=torch.float32, device=dw.dev)
+        for step in range(2):
+            dw.advance_context()
+            dw.decode_step(between_layers=(lambda l: scratch.add_(1.0)) if manual else None)
+            dw.sync()
+        runs.append(dw.out_bits().copy())
+        if not manual:
+            check_samples(dw, [(0, 7), (1, 500), (2, 1099), (0, 0), (2, 3), (1, 777)], 2)
+        dw.close()
+    assert np.array_equal(runs[0], runs[1])
+
+
 @pytest.mark.parametrize("retention,lookahead", [("off", 1), ("declared", 1), ("undeclared", 1), ("host_tables", 1), ("off", 2),
                                                  ("declared", 3)])
 def test_multi_step_decode_with_append_matches_oracle_every_step(retention, lookahead):
