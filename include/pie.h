@@ -372,7 +372,9 @@ int pie_get_stats(pie_pool *pool, pie_stats *out);
 /* Per-layer timeline of the most recently evaluated step (timing = 2 in the configuration; timing = 1 keeps the
  * statistics and the controller but not this table): ms[l][7] = {end of the previous layer's attention kernel,
  * start of this layer's - past its presence wait -, its end, swap-in list start, end, swap-out list start, end} in ms from
- * the start of the step's first attention kernel; -1 where nothing was recorded.  The lists of a group of layers that went
+ * the start of the step's first attention kernel; -1 where nothing was recorded.  Inside pie_decode_step a layer's kernel
+ * starts beside the tail of the layer before it (its first CTAs take the SMs the other's CTAs leave), so its start may lie
+ * some microseconds before the previous layer's end.  The lists of a group of layers that went
  * as one appear under the group's first layer.  The compute columns are the kernels' own GPU-timer stamps; the copy columns
  * are copy-stream events tied to them through one event recorded just before the step's first kernel (a few us of slack).
  * capacity = floats available (>= 7 * n_layers).  PIE_ERR_INVALID if no step has been evaluated yet.  Shows what

@@ -461,7 +461,9 @@ struct AttnParams {
     const float *prev_part_o;
     const float *prev_part_ml;
     uint16_t *prev_out;  // NULL: nothing to merge
-    int32_t *counters;  // [0] next item, [1] CTAs that have left, [2] next piece of the deferred combine
+    int32_t early_trigger;  // the kernel after this one in the stream is the next layer's launch of this kernel: let it start
+                            // beside this launch's tail (see below)
+    int32_t *counters;  // this call's set: [0] next item, [1] CTAs that have left, [2] next piece of the deferred combine
     uint64_t *stamps;   // optional, host visible: [0] when CTA 0 started its main work, [1] when the last CTA left
                         // (globaltimer ns), [2] how long CTA 0 waited for the layer's arriving units (ns), [3] the
                         // batch's context tokens
@@ -769,7 +771,15 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
     }
     __syncthreads();
-    grid_dependency_wait();
+    // Programmatic dependent launch, layer after layer.  Nothing in a layer's attention depends on the layer before it: its
+    // own keys and values, query rows, slot-table row, partial buffers and counters (three sets, taken in turn) - so
+    // the dependency wait comes AFTER the launch's attention work, in front of the two things that do depend on the
+    // launch before (merging that layer's partials, and the completion word, which must not overtake that layer's), and
+    // the trigger comes first: the next layer's CTAs take the place of this launch's CTAs as these leave and go straight
+    // to work, so the tail of one launch and the head of the next overlap.  A launch never gets two launches ahead: its
+    // dependents start only when all its CTAs are resident, that is when the launch before it has left the SMs.
+    if (p.early_trigger) grid_launch_dependents();
+    if (!co_in_smem) grid_dependency_wait();   // (the chunk offsets come from plan_kernel, the launch before this one)
     if (tid == 0 && p.stamps != nullptr && blockIdx.x == 0) {
         *reinterpret_cast<volatile uint64_t *>(p.stamps) = globaltimer_ns();
         if (p.arrive_need == 0 && p.inputs_need == 0) *reinterpret_cast<volatile uint64_t *>(p.stamps + 2) = 0;   // every launch writes all its stamps
@@ -844,11 +854,11 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             item = __shfl_sync(0xffffffffu, item, 0);
             ++qn;
             if (item < 0) {
-                // No work is left for this CTA.  Once every CTA has got here the combine kernel that follows may become
-                // resident (its CTAs wait for this grid to complete before they read anything): its launch then costs
-                // nothing at the end of this kernel.  (Signalled at the kernel's start, the waiting CTAs sat beside
-                // the attention warps for its whole duration and cost 8-head groups 9 %.)
-                grid_launch_dependents();
+                // No work is left for this CTA.  Where the combine kernel follows, it may become resident once every CTA
+                // has got here (its CTAs wait for this grid to complete before they read anything): its launch then costs
+                // nothing at the end of this kernel.  (Signalled at the kernel's start, its small CTAs sat beside the
+                // attention warps for the kernel's whole duration and cost 8-head groups 9 %.)
+                if (!p.early_trigger) grid_launch_dependents();
                 break;
             }
             const ItemInfo it = decode_item(p, co, item);
@@ -1262,6 +1272,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (lane == 0) mbar_arrive(bar_qempty + 8 * qs);
         ++qn;
     }
+    // ---- from here on the launch before this one must have completed
+    grid_dependency_wait();
     // ---- deferred combine of the call before this one (its partials are complete: that grid has finished).  Pieces of
     // 32 float4 each, handed out warp by warp from a counter of their own; sequences of a single chunk were finished by
     // their own kernel.
@@ -1532,13 +1544,17 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
     p.pool = (uint4 *)a.gpu_pool;
     // two pairs of partial buffers where the pool has them: a call whose merge is deferred leaves its partials in the pair
     // of its parity, and the next call (the other parity) merges them while it fills its own
-    const bool alt = a.parity != 0 && sc.part_o_alt != nullptr;
-    p.part_o = alt ? sc.part_o_alt : sc.part_o;
-    p.part_ml = alt ? sc.part_ml_alt : sc.part_ml;
-    p.prev_part_o = alt ? sc.part_o : sc.part_o_alt;
-    p.prev_part_ml = alt ? sc.part_ml : sc.part_ml_alt;
-    p.prev_out = sc.part_o_alt != nullptr ? (uint16_t *)a.prev_out : nullptr;
-    p.counters = sc.counters;
+    const int turn = sc.part_o_more[0] != nullptr ? a.parity % 3 : 0, before = (turn + 2) % 3;
+    auto buf_o = [&](int t) { return t == 0 ? sc.part_o : sc.part_o_more[t - 1]; };
+    auto buf_ml = [&](int t) { return t == 0 ? sc.part_ml : sc.part_ml_more[t - 1]; };
+    p.part_o = buf_o(turn);
+    p.part_ml = buf_ml(turn);
+    p.prev_part_o = buf_o(before);
+    p.prev_part_ml = buf_ml(before);
+    const bool can_defer = sc.part_o_more[0] != nullptr;
+    p.prev_out = can_defer ? (uint16_t *)a.prev_out : nullptr;
+    p.early_trigger = can_defer && a.defer_combine ? 1 : 0;
+    p.counters = sc.counters + 4 * turn;
     p.stamps = a.stamps;
     p.status = a.status;
     p.tokens_out = a.tokens_out;
@@ -1586,8 +1602,8 @@ cudaError_t launch_attention(const AttnShape &sh, const AttnScratch &sc, const A
         return cudaLaunchKernelEx(&lc, kernel, map, p);
     });
     if (e != cudaSuccess) return e;
-    if (a.defer_combine && sc.part_o_alt != nullptr) return cudaSuccess;   // the next call's kernel merges them
-    return launch_combine(sh, sc, a.out, a.n_seqs, a.max_blocks, a.split_tokens, alt ? 1 : 0, stream);
+    if (a.defer_combine && can_defer) return cudaSuccess;   // the next call's kernel merges them
+    return launch_combine(sh, sc, a.out, a.n_seqs, a.max_blocks, a.split_tokens, turn, stream);
 }
 
 // merge the partials of sequences that span several chunks (CTAs of single-chunk sequences return at once)
@@ -1613,8 +1629,8 @@ cudaError_t launch_combine(const AttnShape &sh, const AttnScratch &sc, void *out
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     uint16_t *out = (uint16_t *)out_ptr;
-    const bool alt = parity != 0 && sc.part_o_alt != nullptr;
-    const float *po = alt ? sc.part_o_alt : sc.part_o, *pml = alt ? sc.part_ml_alt : sc.part_ml;
+    const int turn = sc.part_o_more[0] != nullptr ? parity % 3 : 0;
+    const float *po = turn == 0 ? sc.part_o : sc.part_o_more[turn - 1], *pml = turn == 0 ? sc.part_ml : sc.part_ml_more[turn - 1];
     const int32_t *co = sc.chunk_off;
     const int32_t hq = sh.n_q_heads, hkv = sh.n_kv_heads;
     if (sh.head_dim == 128)

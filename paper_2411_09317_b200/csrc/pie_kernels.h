@@ -56,8 +56,8 @@ struct AttnScratch {
     int32_t *counters;   // attn_counter_words(max_seqs, n_kv_heads) int32, zero before the first launch
     float *part_o;       // [max_items][G][D]
     float *part_ml;      // [max_items][G][2]
-    float *part_o_alt = nullptr;   // optional second pair of partial buffers (deferred combine: AttnLaunch::defer_combine)
-    float *part_ml_alt = nullptr;
+    float *part_o_more[2] = {nullptr, nullptr};   // optional second and third pair of partial buffers (deferred combine:
+    float *part_ml_more[2] = {nullptr, nullptr};  // AttnLaunch::defer_combine; the counters then hold three sets of four words)
     int64_t max_items;   // capacity in items (chunk, kv head)
     int32_t max_seqs;
 };
@@ -89,11 +89,12 @@ struct AttnLaunch {
     bool dependent_launch = false;  // launch with programmatic stream serialization: only where the kernel before it in
                                     // the stream writes none of this call's lengths and tables
     float k_scale = 1.f, v_scale = 1.f;  // 8-bit pools: a stored byte stands for decode(byte) * scale
-    // Deferred combine (needs the scratch's second pair of partial buffers; ignored without it).  defer_combine: no
-    // combine kernel follows this call - the NEXT call must name this call's out as its prev_out, have the other parity,
-    // and attend the same batch with the same lengths and split; its kernel merges this call's partials in the tail of
-    // its launch, so this call's out is complete when the next call's kernel is.  Whoever defers must see to it that the
-    // next call happens (or launch_combine with this call's parity).
+    // Deferred combine (needs the scratch's further pairs of partial buffers; ignored without them).  defer_combine: no
+    // combine kernel follows this call - the NEXT call must name this call's out as its prev_out, have parity + 1 (the
+    // buffers and counter sets are taken in turns of three), follow this call directly in the stream as a dependent
+    // launch, and attend the same batch with the same lengths and split; its kernel starts beside this call's tail and
+    // merges this call's partials at the end of its own launch, so this call's out is complete when the next call's
+    // kernel is.  Whoever defers must see to it that the next call happens (or launch_combine with this call's parity).
     bool defer_combine = false;
     void *prev_out = nullptr;
     int parity = 0;

