@@ -179,6 +179,7 @@ struct pie_pool {
     std::vector<int32_t> v_moved, v_src, v_dst, v_in, v_out;
     SwapList one_list;                  // the list of a single swap call
     // split-K merge left to the next attention call of the decode step (its kernel merges in the tail of its launch)
+    bool auto_split = false;            // the configuration left the split-K chunk to the library
     struct Deferred {
         bool on = false;
         void *out = nullptr;
@@ -828,7 +829,7 @@ int flush_deferred_combine(pie_pool *p) {
 // flush_deferred_combine); a merge that an earlier call left (p->deferred) is taken on by this call's kernel.
 int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const int32_t *bt_dev, int32_t max_blocks,
                    const int32_t *ctx_dev, const int32_t *bt_host, const int32_t *ctx_host, int32_t n_seqs, float scale,
-                   const void *k_new, const void *v_new, bool dependent = false, bool defer = false) {
+                   const void *k_new, const void *v_new, bool dependent = false, bool defer = false, bool in_loop = false) {
     if (!p) return PIE_ERR_INVALID;
     if (p->sticky != PIE_OK) return p->sticky;
     if (layer < 0 || layer >= p->cfg.n_layers) return PIE_ERR_RANGE;
@@ -841,7 +842,20 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     st = check_status_word(p);  // a flag raised by an earlier call's kernels
     if (st != PIE_OK) return st;
     if (n_seqs == 0) return PIE_OK;
-    const int64_t split = p->cfg.split_tokens;
+    // Split-K chunk.  In the decode loop consecutive layers' launches overlap at their ends, so a launch's slowest CTA no
+    // longer holds the SMs up and long work items win (fewer partials, less work per token around the items): where the
+    // caller left the choice to the library, the largest of 2048 / 1024 tokens that still gives every CTA an item (counted
+    // from the blocks allocated) - measured on the three shapes: 6.27 -> 6.86, 6.60 -> 7.05 and 6.89 -> 7.22 TB/s against 512
+    // / 1024 / 512 tokens.  Single calls keep the pool's chunk: nothing hides their tail.
+    int64_t split = p->cfg.split_tokens;
+    if (in_loop && p->auto_split) {
+        const int64_t tokens = (int64_t)p->table->n_allocated() * 16;
+        for (int64_t s = 2048; s > split; s /= 2)
+            if (tokens / s * p->cfg.n_kv_heads >= p->attn_grid) {
+                split = s;
+                break;
+            }
+    }
     // host-side checks when the caller supplied host copies of the tables
     int64_t ticket = 0, waits[4];
     if (bt_host) {
@@ -922,7 +936,8 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     a.done_value = (unsigned long long)ticket;
     a.dependent_launch = dependent;
     // a merge the call before this one left: this kernel takes it on if it attends the same batch (else it is merged now)
-    if (p->deferred.on && !(dependent && p->deferred.n_seqs == n_seqs && p->deferred.max_blocks == max_blocks && p->deferred.ctx == ctx_dev)) {
+    if (p->deferred.on && !(dependent && p->deferred.n_seqs == n_seqs && p->deferred.max_blocks == max_blocks && p->deferred.ctx == ctx_dev &&
+                            p->deferred.split == (int32_t)split)) {
         st = flush_deferred_combine(p);
         if (st != PIE_OK) return st;
     }
@@ -1254,6 +1269,7 @@ int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
     // Split-K chunk: 512 tokens balances the persistent grid best on batches of many short sequences; where the pool
     // is laid out for few long ones (>= 6144 tokens per sequence on average) 1024 halves the partials and the merge
     // (measured: +6.5 % on 17 sequences of 4k-32k tokens with 8-head groups, -1.5 % on the batched shapes).
+    p->auto_split = p->cfg.split_tokens == 0;
     if (p->cfg.split_tokens == 0)
         p->cfg.split_tokens = (int64_t)cfg->n_logical_blocks * 16 / std::max(cfg->max_seqs, 1) >= 6144 ? 1024 : 512;
     p->kv_fp8 = cfg->kv_format;
@@ -2332,7 +2348,7 @@ static int decode_layer(pie_pool *pool, int32_t l, const void *q, void *out, con
         }
     }
     st = attention_call(pool, l, q, out, block_table_dev, max_blocks_per_seq, ctx_lens_dev, nullptr, nullptr, n_seqs, scale,
-                        k_new, v_new, dependent, defer);
+                        k_new, v_new, dependent, defer, true);
     if (st != PIE_OK) return st;
     pool->group_done.push_back(l);
     if ((int32_t)pool->group_done.size() >= pool->group_len) return finish_group(pool);
