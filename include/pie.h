@@ -126,7 +126,8 @@ typedef struct pie_stats {
     int64_t prefetch_lists;                /* swap-in lists the decode loop has started so far, and how many of them were for */
     int64_t prefetch_violations;           /* layers of the NEXT token (Section 3.4.2's allowed rule violation) */
     double last_step_violation_ratio;      /* the two, over the last evaluated step */
-    double reserved[4];                    /* 0 */
+    double copy_engine_copies;             /* data copies given to the copy engines so far (one per run of consecutive slots) */
+    double reserved[3];                    /* 0 */
 } pie_stats;
 
 /* ---- pool (Section 3.1: the physical pools; Section 3.2: the mapping table) --------------------- */
@@ -258,7 +259,11 @@ int pie_set_violation_trigger(pie_pool *pool, double share);
 /* The decisions taken so far in whole-layer mode: int32 quadruples {step, layer starting, layer whose swap-out
  * started or -1, layer whose swap-in started or -1}.  log may be NULL to ask for the count only. */
 int pie_get_layer_log(pie_pool *pool, int32_t *log, int64_t capacity, int64_t *n_entries);
-/* Marks a step boundary for the per-step timing sets (pie_decode_step calls it itself). */
+/* Marks a step boundary (pie_decode_step calls it itself): the per-step timing sets turn over, and the host thread waits
+ * here until the GPU has finished the step before the previous one - the host enqueues one step while the one before it
+ * runs, and no further.  (Slots freed by a step's swap lists are only known free once their copies have completed; a host
+ * several steps ahead would be handed slots still in flight, in the order they were released, and its lists would break
+ * into many short copies.) */
 int pie_step_begin(pie_pool *pool);
 
 /* ---- policy and controller (Section 3.3, Section 3.4.2) ------------------------------------------ */
@@ -367,8 +372,8 @@ int pie_resize_status(pie_pool *pool, int32_t *visible, int32_t *alloc_limit, in
  * computed.  Arrays are host, capacity n_logical_blocks each. */
 int pie_plan_layer(pie_pool *pool, int32_t layer, int32_t *in_ids, int64_t *n_in, int32_t *out_ids, int64_t *n_out);
 /* Evaluate, in step order, the event sets of earlier steps that have completed (no blocking), update the
- * stats, and in adaptive mode adjust the ratio.  The library keeps 4 steps of events: pie_step_begin waits
- * for the oldest step when the host gets that far ahead of the GPU. */
+ * stats, and in adaptive mode adjust the ratio.  The library keeps 4 steps of events (callers that go layer by layer
+ * without pie_step_begin: the oldest step is waited for when the host gets that far ahead of the GPU). */
 int pie_controller_tick(pie_pool *pool, int32_t *changed);
 int pie_get_stats(pie_pool *pool, pie_stats *out);
 /* Per-layer timeline of the most recently evaluated step (timing = 2 in the configuration; timing = 1 keeps the

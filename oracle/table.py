@@ -18,16 +18,19 @@ handed out again at once, but whoever receives it must wait for that ticket.  So
 overwritten before the copy reading it has finished, and a unit's bytes are never read at the
 destination before the copy writing them has finished.
 
-Slot hand-out order (shared rule, so that two implementations can be compared slot by slot):
+Slot hand-out order (shared rule, so that two implementations can be compared slot by slot; the paper
+leaves open which free region a block receives, Section 3.2 only asks that the table name it):
 ``ready`` holds the slots that are free for certain; ``pending`` is a queue of released slots still
 waiting for their ticket.  At the start of every call pending slots whose ticket is confirmed move to
-``ready``.  A request for n slots takes the first n of the lowest run of consecutive ready slots that
-has at least n; failing that, whole runs, longest first (lowest first among equals), until it is
-served; what ``ready`` cannot give comes from the front of ``pending``, and the tickets to wait for
-are reported.  (Lists of swapped blocks thus land in consecutive slots whenever the pool has room for
-that, however the set of free slots came about; a first-in-first-out hand-out keeps whatever order
-the slots were released in, and that order degrades once the host-resident sets change one block at
-a time.)
+``ready``.  A request for n >= 2 slots goes through the runs of consecutive ready slots in ascending
+order and takes the first n of the first run that has n slots at or after the cursor; failing that -
+and for a request for a single slot, which does not move the cursor - the first n of the lowest run
+that has at least n; failing that, whole runs, longest first (lowest first among equals), until it is
+served.  The cursor then stands behind the slots taken last.  What ``ready`` cannot give comes from the
+front of ``pending``, and the tickets to wait for are reported.  (Swap lists release their slots in
+about the order they took them, so the hand-out walks round the spare part of a pool like a ring and
+lists land in consecutive slots whatever sizes the lists before them had; single slots - allocations -
+fill the lowest holes.)
 """
 from __future__ import annotations
 
@@ -49,6 +52,7 @@ Q_NONE, Q_IN, Q_OUT, Q_COMPUTE = 0, 1, 2, 3
 class _SlotPool:
     def __init__(self, n):
         self.ready = list(range(n))   # kept in ascending order
+        self.cursor = 0               # behind the slots the last request for two or more took from ready
         self.pending = []  # (slot, queue, ticket)
 
     def _add_ready(self, slot):
@@ -79,19 +83,30 @@ class _SlotPool:
     def take(self, n):
         """-> (slots, {queue: max ticket to wait for}, per-slot (queue, ticket) tags)"""
         slots, waits, tags = [], {}, []
+        rove = n >= 2
         while len(slots) < n and self.ready:
             want = n - len(slots)
             runs = self._runs()
-            fit = [r for r in runs if r[1] >= want]
-            if fit:
-                start, length = fit[0]                       # the lowest run that serves the rest of the request
-            else:
-                start, length = max(runs, key=lambda r: (r[1], -r[0]))   # else whole runs, longest first, lowest among equals
-            got = list(range(start, start + min(want, length)))
+            first = None
+            if rove:                                         # the first run with `want` slots at or after the cursor
+                for start, length in runs:
+                    a = max(start, self.cursor)
+                    if start + length - a >= want:
+                        first, count = a, want
+                        break
+            if first is None:
+                fit = [r for r in runs if r[1] >= want]
+                if fit:
+                    first, count = fit[0][0], want           # the lowest run that serves the rest of the request
+                else:                                        # else whole runs, longest first, lowest among equals
+                    first, count = max(runs, key=lambda r: (r[1], -r[0]))
+            got = list(range(first, first + count))
             for s in got:
                 self.ready.remove(s)
             slots += got
             tags += [(Q_NONE, 0)] * len(got)
+            if rove:
+                self.cursor = first + count
         while len(slots) < n:
             slot, qu, tk = self.pending.pop(0)
             slots.append(slot)

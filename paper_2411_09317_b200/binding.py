@@ -70,7 +70,8 @@ class Stats(ctypes.Structure):
         ("last_step_slowdown_ms", ctypes.c_double), ("ratio_floor", ctypes.c_double), ("bytes_out_elided", ctypes.c_double),
         ("patch_kernel_launches", ctypes.c_double), ("governor_cap", ctypes.c_double),
         ("prefetch_lists", ctypes.c_int64), ("prefetch_violations", ctypes.c_int64),
-        ("last_step_violation_ratio", ctypes.c_double), ("reserved", ctypes.c_double * 4),
+        ("last_step_violation_ratio", ctypes.c_double), ("copy_engine_copies", ctypes.c_double),
+        ("reserved", ctypes.c_double * 3),
     ]
 
     def as_dict(self):

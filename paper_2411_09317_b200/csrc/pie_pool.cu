@@ -170,9 +170,12 @@ struct pie_pool {
     cudaEvent_t lev_last[TIMING_RING][4] = {};  // the set's newest event on each queue's stream (its streams complete in order)
     cudaStream_t aux_stream = nullptr;          // brings a step's stamps to the host without touching the compute stream
     cudaEvent_t lev_close_ev[TIMING_RING] = {}; // recorded there behind the copy
+    cudaEvent_t step_end_ev[TIMING_RING] = {};  // recorded there once a step's last attention kernel has completed
+    int64_t step_end_of[TIMING_RING] = {};      // ... the step each of them stands for (0 = none)
+    int64_t step_end_ticket = 0;                // the compute ticket the newest of them waits for
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
-    double free_contrast = -1.0;     // on swap-free steps: what the layers' times add up to above the fastest quarter's mean, / compute
+    double free_contrast = -1.0;     // on swap-free steps: the contrast of the layers' four-layer mean times (see evaluate_step_set)
     std::vector<float> timeline;     // last evaluated step: [L][7] ms from the step's first event (-1 = not recorded)
     pie_stats stats{};
     // scratch vectors
@@ -473,6 +476,7 @@ int do_copies(pie_pool *p, int dir_queue, const int32_t *src, const int32_t *dst
             while (j < n && !(elide && elide[j]) && src[j] == src[j - 1] + 1 && dst[j] == dst[j - 1] + 1) ++j;
             PIE_CUDA(cudaMemcpyAsync(dst_pool + (int64_t)dst[i] * BB, src_pool + (int64_t)src[i] * BB, (size_t)((j - i) * BB),
                                      kind, stream));
+            p->stats.copy_engine_copies += 1;
             i = j;
         }
         if (dma_patch) {
@@ -663,6 +667,7 @@ int swap_issue_group(pie_pool *p, int queue, std::vector<SwapList> &lists, int32
     }
     list_commit_ticket(p, off, words, queue, live.back()->ticket);
     p->stats.calls_copy_engine += (double)k;
+    p->stats.copy_engine_copies += (double)runs.size();
     for (SwapList *l : live) {
         if (queue == PIE_Q_IN) p->layer_in_last[(size_t)l->layer] = l->ticket;
         PIE_STICKY(record_ticket(p, queue, l->ticket));
@@ -769,6 +774,7 @@ void destroy_pool(pie_pool *p) {
     for (int k = 0; k < TIMING_RING; ++k) {
         if (p->lev_anchor[k]) cudaEventDestroy(p->lev_anchor[k]);
         if (p->lev_close_ev[k]) cudaEventDestroy(p->lev_close_ev[k]);
+        if (p->step_end_ev[k]) cudaEventDestroy(p->step_end_ev[k]);
     }
     if (p->aux_stream) cudaStreamDestroy(p->aux_stream);
     for (int i = 0; i < 2; ++i)
@@ -971,6 +977,27 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
         p->lev_closed[p->step % TIMING_RING] = false;   // the set's newest compute ticket has no mark yet (close_step_set)
     }
     return st;
+}
+
+// The host enqueues one decode step while the step before it runs, and no further (pie_step_begin waits for the step
+// before that).  Slots released by a step's swap lists can only be handed out as free for certain once their copies are
+// known complete; a host that is several steps ahead finds nothing but slots still in flight, takes them in the order
+// they were released, mixed with what has just come back, and the lists break into several runs (measured on 17 long
+// sequences and 80 layers: 3 runs per list of 20 blocks, and the copy engines at 22 GB/s instead of 40).  The event is
+// recorded on the side stream behind a wait by value for the step's last attention kernel: nothing on the compute stream.
+int mark_step_end(pie_pool *p) {
+    if (p->step <= 0 || !p->wait_value64 || !p->aux_stream || p->last_attn_ticket <= p->step_end_ticket) return PIE_OK;
+    if (p->recorded[PIE_Q_COMPUTE] != p->last_attn_ticket) return PIE_OK;
+    const int k = (int)(p->step % TIMING_RING);
+    if (p->wait_value64((CUstream)p->aux_stream, (CUdeviceptr)(uintptr_t)p->done_dev, (cuuint64_t)p->last_attn_ticket,
+                        CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS) {
+        g_last_cuda_error = (int)cudaErrorUnknown;
+        return PIE_ERR_CUDA;
+    }
+    PIE_CUDA(cudaEventRecord(p->step_end_ev[k], p->aux_stream));
+    p->step_end_of[k] = p->step;
+    p->step_end_ticket = p->last_attn_ticket;
+    return PIE_OK;
 }
 
 // The timing set of the step in progress is complete once its newest compute ticket is: give that ticket its mark.
@@ -1324,6 +1351,8 @@ int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
         p->ticket_ev[PIE_Q_COMPUTE][i] = p->compute_ev_plain[i];
     }
     for (int i = 0; i < LIST_EVENTS; ++i) PIE_TRY(cudaEventCreateWithFlags(&p->list_events[i], cudaEventDisableTiming), PIE_ERR_CUDA);
+    PIE_TRY(cudaStreamCreateWithFlags(&p->aux_stream, cudaStreamNonBlocking), PIE_ERR_CUDA);
+    for (int k = 0; k < TIMING_RING; ++k) PIE_TRY(cudaEventCreateWithFlags(&p->step_end_ev[k], cudaEventDisableTiming), PIE_ERR_CUDA);
     if (cfg->timing) {
         for (int k = 0; k < TIMING_RING; ++k) {
             p->lev[k].resize((size_t)cfg->n_layers);
@@ -1333,7 +1362,6 @@ int pie_pool_create(const pie_pool_config *cfg_in, pie_pool **out) {
         }
         if (cfg->timing >= 2)
             for (int k = 0; k < TIMING_RING; ++k) PIE_TRY(cudaEventCreate(&p->lev_anchor[k]), PIE_ERR_CUDA);
-        PIE_TRY(cudaStreamCreateWithFlags(&p->aux_stream, cudaStreamNonBlocking), PIE_ERR_CUDA);
         for (int k = 0; k < TIMING_RING; ++k) PIE_TRY(cudaEventCreateWithFlags(&p->lev_close_ev[k], cudaEventDisableTiming), PIE_ERR_CUDA);
         // The kernels note their stamps in device memory and one copy per step brings a step's set to the host.  (Stamps
         // in host-visible memory made every kernel end with a store across the host link; while swap lists were being
@@ -1703,9 +1731,13 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
     // Copies that are hidden behind compute can still slow the compute down (they share HBM); that excess counts as a
     // wait, so the controller holds the ratio where wait + slow-down stays within its tolerance.  Every layer of a step
     // attends the same batch at the same lengths, and the swap lists of a group of layers are in flight during the first
-    // part of the group only: the step's undisturbed layers are its own yardstick.  The slow-down is what the layers'
-    // times add up to above the mean of the step's fastest quarter, less what that sum comes to on steps without swap
-    // traffic (a record, Section 3.4.2).  Nothing is compared across steps, so clocks drifting under the power cap and
+    // part of the group only: the step's undisturbed layers are its own yardstick.  The contrast of a series of layer
+    // times = what they add up to above the mean of the series' fastest quarter, over their sum.  Consecutive launches
+    // overlap at their ends, so the end stamp of a layer moves by a few per cent of a layer from one to the next (what one
+    // layer's time gains the next one's loses) while copies slow several layers in a row: the slow-down is the contrast
+    // of the four-layer means, less the larger of what that comes to on steps without swap traffic (a record,
+    // Section 3.4.2) and 0.3 of the contrast of the single layers (measured: alternating end stamps pass a four-layer
+    // mean at a quarter of their size).  Nothing is compared across steps, so clocks drifting under the power cap and
     // contexts growing do not look like a slow-down.  (Steps of fewer than nine layers fall back to a record of the
     // time per context token taken on swap-free steps.)
     double tokens = 0.0;   // the step's own count (each kernel notes its batch's tokens beside its time stamps)
@@ -1713,16 +1745,24 @@ static int evaluate_step_set(pie_pool *pool, int k, bool wait, int32_t *changed)
         if (ev[l].has_compute) tokens = (double)stamps[l * STAMP_WORDS + STAMP_TOKENS];
     double slow = 0.0;
     if (spans.size() >= 8 && compute > 0) {
-        std::vector<double> sorted(spans);
-        std::sort(sorted.begin(), sorted.end());
-        const size_t quarter = std::max<size_t>(2, sorted.size() / 4);
-        double ref = 0.0;
-        for (size_t i = 0; i < quarter; ++i) ref += sorted[i];
-        ref /= (double)quarter;
-        double above = 0.0;
-        for (double sp : spans) above += std::max(0.0, sp - ref);
-        if (!any_swap) pool->free_contrast = pool->free_contrast >= 0 ? 0.75 * pool->free_contrast + 0.25 * above / compute : above / compute;
-        else slow = std::max(0.0, above - std::max(0.0, pool->free_contrast) * compute);
+        auto contrast = [](const std::vector<double> &v) {
+            std::vector<double> sorted(v);
+            std::sort(sorted.begin(), sorted.end());
+            const size_t quarter = std::max<size_t>(2, sorted.size() / 4);
+            double ref = 0.0, sum = 0.0, above = 0.0;
+            for (size_t i = 0; i < quarter; ++i) ref += sorted[i];
+            ref /= (double)quarter;
+            for (double x : v) {
+                sum += x;
+                above += std::max(0.0, x - ref);
+            }
+            return sum > 0 ? above / sum : 0.0;
+        };
+        std::vector<double> means(spans.size() - 3);
+        for (size_t i = 0; i + 3 < spans.size(); ++i) means[i] = 0.25 * (spans[i] + spans[i + 1] + spans[i + 2] + spans[i + 3]);
+        const double smooth = contrast(means);
+        if (!any_swap) pool->free_contrast = pool->free_contrast >= 0 ? 0.75 * pool->free_contrast + 0.25 * smooth : smooth;
+        else slow = std::max(0.0, smooth - std::max(std::max(0.0, pool->free_contrast), 0.3 * contrast(spans))) * compute;
     } else if (tokens > 0 && compute > 0) {
         const double per_token = compute / tokens;
         if (!any_swap) pool->base_ms_per_token = pool->base_ms_per_token > 0 ? 0.75 * pool->base_ms_per_token + 0.25 * per_token : per_token;
@@ -1763,9 +1803,15 @@ int pie_step_begin(pie_pool *pool) {
     {
         int st = finish_group(pool);       // a caller that went layer by layer may have left a group open
         if (st == PIE_OK) st = close_step_set(pool);
+        if (st == PIE_OK) st = mark_step_end(pool);
         if (st != PIE_OK) return st;
     }
     ++pool->step;
+    if (pool->step >= 3) {   // one step ahead of the GPU at most (mark_step_end)
+        const int64_t old = pool->step - 2;
+        const int k = (int)(old % TIMING_RING);
+        if (pool->step_end_of[k] == old) PIE_CUDA(cudaEventSynchronize(pool->step_end_ev[k]));
+    }
     if (pool->cfg.timing) {
         int st = evaluate_completed(pool, nullptr);
         if (st != PIE_OK) return st;

@@ -55,28 +55,45 @@ void SlotPool::settle(const int64_t *done) {
 
 void SlotPool::take_n(int64_t n, int32_t *slots, SlotTag *tags) {
     int64_t k = 0;
+    const bool rove = n >= 2;
     while (k < n && !runs_.empty()) {
         const int64_t want = n - k;
-        auto pick = runs_.end(), longest = runs_.begin();
-        for (auto it = runs_.begin(); it != runs_.end(); ++it) {
-            if (it->second >= want) {
-                pick = it;  // the lowest run that serves the rest of the request
-                break;
+        auto pick = runs_.end();
+        int32_t from = 0;
+        if (rove)  // the first run that has `want` slots at or after the cursor
+            for (auto it = runs_.begin(); it != runs_.end(); ++it) {
+                const int32_t a = std::max(it->first, cursor_);
+                if ((int64_t)it->first + it->second - a >= want) {
+                    pick = it;
+                    from = a;
+                    break;
+                }
             }
-            if (it->second > longest->second) longest = it;
+        if (pick == runs_.end()) {
+            auto longest = runs_.begin();
+            for (auto it = runs_.begin(); it != runs_.end(); ++it) {
+                if (it->second >= want) {
+                    pick = it;  // the lowest run that serves the rest of the request
+                    break;
+                }
+                if (it->second > longest->second) longest = it;
+            }
+            if (pick == runs_.end()) pick = longest;
+            from = pick->first;
         }
-        if (pick == runs_.end()) pick = longest;
         const int32_t start = pick->first, len = pick->second;
-        const int32_t m = (int32_t)std::min<int64_t>(want, len);
+        const int32_t m = (int32_t)std::min<int64_t>(want, (int64_t)start + len - from);
         for (int32_t i = 0; i < m; ++i) {
-            slots[k] = start + i;
+            slots[k] = from + i;
             tags[k].queue = PIE_Q_NONE;
             tags[k].ticket = 0;
             ++k;
         }
         runs_.erase(pick);
-        if (m < len) runs_[start + m] = len - m;
+        if (from > start) runs_[start] = from - start;
+        if (from + m < start + len) runs_[from + m] = start + len - (from + m);
         n_ready_ -= m;
+        if (rove) cursor_ = from + m;
     }
     while (k < n) {
         Pending p = pending_.front();

@@ -19,10 +19,16 @@ struct SlotTag {
 // Free slots of one pool.  `ready` holds slots that are free for certain, as runs of consecutive numbers; `pending`
 // is a queue of slots released by a copy that may not have finished: they can be handed out, but the receiver must
 // wait for the tag's ticket.  Hand-out rule (shared with the oracle, so that the two can be compared slot by slot):
-// a request for n slots takes the first n of the lowest ready run that has at least n; failing that, whole runs,
-// longest first (lowest first among equals), until it is served; what ready cannot give comes from the front of
-// pending.  Lists of swapped blocks thus land in consecutive slots whenever the pool has room for that, however the
-// set of free slots came about - which is what lets a few large copies move them.
+// a request for n >= 2 slots looks, in ascending order, for the first ready run that has n slots at or after the
+// cursor and takes the first n of those; failing that (and for a single slot, which leaves the cursor alone), the first
+// n of the lowest ready run that has at least n; failing that, whole runs, longest first (lowest first among equals),
+// until it is served; the cursor then stands behind the slots taken last.  What ready cannot give comes from the front
+// of pending.  The slots of swap lists are released in about the order they were taken, so the hand-out walks round the
+// pool's spare part like a ring: lists land in consecutive slots, and consecutive lists beside each other, whatever
+// their sizes were before - which is what lets a few large copies move them.  (Taking the lowest run that fits, the
+// rule before this one, serves a steady ratio as well but splinters the spare part once the lists grow and shrink by a
+// few blocks at a time: after a ramp of the adaptive controller a list of 20 blocks came in three runs.)  Single slots -
+// allocations, which live long - fill the lowest holes and stay out of the ring's way.
 class SlotPool {
   public:
     explicit SlotPool(int64_t n);
@@ -46,6 +52,7 @@ class SlotPool {
     void add_ready(int32_t slot);
     std::map<int32_t, int32_t> runs_;  // start -> length of a run of ready slots
     int64_t n_ready_ = 0;
+    int32_t cursor_ = 0;  // behind the slots that the last request of two or more took from ready
     std::deque<Pending> pending_;
 };
 

@@ -255,8 +255,8 @@ def test_kept_host_copy_is_reused_and_written_blocks_are_copied():
 
 
 def test_slot_hand_out_prefers_runs_of_consecutive_slots():
-    """The shared hand-out rule by hand: the lowest run that serves the request; else whole runs, longest first; pending
-    slots (with their tickets) only when nothing else is left."""
+    """The shared hand-out rule by hand: the first run with n slots at or after the cursor; else the lowest run that serves
+    the request; else whole runs, longest first; pending slots (with their tickets) only when nothing else is left."""
     p = table._SlotPool(10)
     assert p.take(3)[0] == [0, 1, 2]
     assert p.take(1)[0] == [3]
@@ -275,6 +275,36 @@ def test_slot_hand_out_prefers_runs_of_consecutive_slots():
     for s in (5, 40, 41, 42, 43, 9, 44, 45, 13, 46, 47):
         q.release(s, table.Q_NONE, 0)
     assert q.take(6)[0] == [40, 41, 42, 43, 44, 45]
+
+
+def test_slot_hand_out_walks_round_the_pool():
+    """The cursor by hand: lists that grow and shrink while their slots come back in the order they went keep landing in
+    consecutive slots, one list beside the other; a single slot fills the lowest hole and leaves the cursor alone."""
+    p = table._SlotPool(24)
+    assert p.take(4)[0] == [0, 1, 2, 3]                # a long-lived allocation; the cursor stands at 4
+    a = p.take(3)[0]
+    b = p.take(3)[0]
+    assert (a, b) == ([4, 5, 6], [7, 8, 9])
+    for s in a:
+        p.release(s, table.Q_NONE, 0)                  # ready: {4..6}, {10..23}
+    assert p.take(4)[0] == [10, 11, 12, 13]            # the freed run of three lies behind the cursor, and is too short anyway
+    assert p.take(2)[0] == [14, 15]                    # ... and a list that WOULD fit there still goes on from the cursor
+    assert p.take(1)[0] == [4]                         # one slot: the lowest hole
+    assert p.take(3)[0] == [16, 17, 18]                # ... which did not move the cursor
+    for s in b + [10, 11, 12, 13]:
+        p.release(s, table.Q_NONE, 0)                  # ready: {5..13}, {19..23}
+    assert p.take(5)[0] == [19, 20, 21, 22, 23]        # up to the end of the pool
+    assert p.take(5)[0] == [5, 6, 7, 8, 9]             # nothing at or after the cursor: round again, from the lowest run that fits
+    assert p.take(3)[0] == [10, 11, 12]                # on from the cursor, inside that run
+    p.release(14, table.Q_NONE, 0); p.release(15, table.Q_NONE, 0)   # ready: {13..15}
+    assert p.take(2)[0] == [13, 14]
+    # the cursor inside a run: slots that came back just below it are passed over while the part above serves the request
+    q = table._SlotPool(16)
+    assert q.take(6)[0] == [0, 1, 2, 3, 4, 5]
+    for s in (3, 4, 5):
+        q.release(s, table.Q_NONE, 0)                  # ready: {3..15} as one run, cursor at 6
+    assert q.take(4)[0] == [6, 7, 8, 9]
+    assert q.take(7)[0] == [10, 11, 12, 13, 14, 15, 3]   # no run of seven: the longest whole, the rest from the lowest
 
 
 def test_table_error_codes_and_two_phase_states():
