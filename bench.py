@@ -194,7 +194,7 @@ def run_reference(args):
 SWEEP_RATIOS = {"llama2_7b": [0.003, 0.004, 0.005, 0.0055, 0.006, 0.007],
                 "llama3_8b": [0.003, 0.004, 0.005, 0.0055, 0.006, 0.007],
                 "llama3_70b": [0.003, 0.004, 0.005, 0.0055, 0.006]}
-KEPT_RATIOS = {"llama2_7b": [0.006, 0.007, 0.008, 0.009], "llama3_8b": [0.006, 0.007, 0.008], "llama3_70b": [0.004, 0.005, 0.006]}
+KEPT_RATIOS = {"llama2_7b": [0.005, 0.006, 0.007, 0.008], "llama3_8b": [0.006, 0.007, 0.008], "llama3_70b": [0.005, 0.006, 0.007]}
 DTYPE_NAME = {synth.F16: "f16", synth.BF16: "bf16"}
 
 
@@ -354,12 +354,15 @@ def main():
     longest_run = max(n_sweep + warm_sweep, args.steps + args.warmup, args.ramp + args.steps) + 2
     n_blocks = int(((wl.ctx_lens.astype(np.int64) + longest_run + 15) // 16).sum())
     r_cap = 1.25 * max(sweep_ratios + kept_ratios) + 0.001
-    # the GPU pool holds the fully resident batch plus, for ratios up to r_cap, three groups of up to eight layers'
-    # host-resident shares (arriving, in use, leaving); the host pool the host-resident shares of all layers
+    # the GPU pool holds the fully resident batch plus, for ratios up to r_cap, two steps' worth of host-resident shares:
+    # three groups of up to eight layers are in transit at any time (arriving, in use, leaving), and the host enqueues up
+    # to a step ahead, so with this much to spare a swap list's slots come from the part of the pool that is free for
+    # certain, in one run; the host pool holds the host-resident shares of all layers and as much again in transit
     share = int(r_cap * n_blocks) + 1
+    spare_lists = max(26, 2 * L + 8)
     dw = DeviceWorkload(wl, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
-                        attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=26 * share + 64,
-                        extra_host_slots=(L + 26) * share + 64, extra_tokens=longest_run)
+                        attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=spare_lists * share + 64,
+                        extra_host_slots=(L + spare_lists) * share + 64, extra_tokens=longest_run)
     rn = Runner(dw, torch, pie)
     bytes_layer0 = dw.attention_bytes_per_layer()
 
@@ -464,8 +467,8 @@ def main():
         wl8 = dataclasses.replace(wl, kv_fp8=True)
         n8, r8 = 32, 0.0075
         dw8 = DeviceWorkload(wl8, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
-                             attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=26 * share + 64,
-                             extra_host_slots=(L + 26) * share + 64, extra_tokens=n8 + 8)
+                             attn_ctas_per_sm=args.ctas_per_sm, extra_gpu_slots=spare_lists * share + 64,
+                             extra_host_slots=(L + spare_lists) * share + 64, extra_tokens=n8 + 8)
         r8n = Runner(dw8, torch, pie)
         pie.pie_set_extension_ratio(dw8.pool, 0.0)
         a8 = r8n.run(n8, 4)
