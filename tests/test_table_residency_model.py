@@ -193,6 +193,67 @@ def test_every_short_call_sequence_keeps_the_rules_with_kept_host_copies(impl):
     assert n > 3500 and elided > 300
 
 
+def _decode_loop_with_changing_shares(view, L, shares, lag):
+    """The decode loop's calls on the bare table: per step and layer, bring in the layer's units that are on the host or
+    on their way there, attend, and push the first m units (ascending ids) out again; copies are confirmed `lag` tickets
+    late, in order.  -> per list (step, direction, (id, source slot, destination slot) triples)."""
+    lists, open_tickets = [], []
+    for step, m in enumerate(shares):
+        for l in range(L):
+            away = [b for b in range(view.NB) if view.state(l, b)[0] in (otable.HOST, otable.TO_HOST)]
+            if away:
+                st, tk, pairs, _ = view.swap(otable.Q_IN, l, away)
+                assert st == 0
+                lists.append((step, "in", pairs))
+                open_tickets.append((otable.Q_IN, tk))
+            st, ctk, _ = view.attention(l, list(range(view.NB)))
+            assert st == 0
+            open_tickets.append((otable.Q_COMPUTE, ctk))
+            if m:
+                st, tk, pairs, _ = view.swap(otable.Q_OUT, l, list(range(m)))
+                assert st == 0
+                lists.append((step, "out", pairs))
+                open_tickets.append((otable.Q_OUT, tk))
+            while len(open_tickets) > lag:
+                q, tk = open_tickets.pop(0)
+                assert view.confirm(q, tk) == 0
+    return lists
+
+
+def _runs(pairs):
+    return 1 + sum(1 for a, b in zip(pairs, pairs[1:]) if b[1] != a[1] + 1 or b[2] != a[2] + 1)
+
+
+@pytest.mark.parametrize("impl", ["oracle", "library"])
+def test_lists_stay_whole_while_the_host_resident_share_grows_and_shrinks(impl):
+    """The hand-out rule's purpose, on both implementations: with the spare part of the pools a few lists larger than what
+    is in flight, a layer's swap list lands in ONE run of consecutive slots on both sides however the share changed before -
+    except in the step of a change itself, where the units that join come from the scattered slots they lived in.  (Sizes
+    chosen so that "the lowest run that fits", without the cursor, leaves two of these lists in two runs.)"""
+    L, NB = 4, 40
+    shares = [3, 3, 4, 4, 6, 6, 9, 9, 7, 7, 4, 4, 5, 5, 8, 8, 8, 8]
+    view = VIEWS[impl](L, NB, L * NB + 30, 80)
+    for b in range(NB):
+        assert view.alloc(b) == 0
+    lists = _decode_loop_with_changing_shares(view, L, shares, lag=10)
+    steady = [pairs for step, _, pairs in lists if step > 0 and shares[step] == shares[step - 1]]
+    assert len(steady) == 10 * 2 * L
+    assert all(len(pairs) == shares[step] for step, _, pairs in lists if step > 0 and shares[step] == shares[step - 1])
+    assert [_runs(pairs) for pairs in steady] == [1] * len(steady)
+
+
+def test_both_implementations_hand_out_the_same_slots_through_a_ramp():
+    L, NB = 3, 32
+    shares = [2, 2, 5, 5, 3, 3, 3, 7, 7, 1, 1, 6]
+    out = []
+    for impl in ("oracle", "library"):
+        view = VIEWS[impl](L, NB, L * NB + 24, 40)      # tight: requests also reach the pending queue
+        for b in range(NB):
+            assert view.alloc(b) == 0
+        out.append(_decode_loop_with_changing_shares(view, L, shares, lag=9))
+    assert out[0] == out[1] and len(out[0]) > 60
+
+
 @pytest.mark.parametrize("impl", ["oracle", "library"])
 @pytest.mark.parametrize("retain", [False, True])
 def test_long_random_runs_keep_the_rules(impl, retain):
