@@ -82,8 +82,9 @@ typedef struct pie_pool_config {
     void *copy_out_stream;
     int32_t split_tokens;      /* split-K chunk in tokens, multiple of 16; 0 = the library chooses: 512 (1024 where the pool
                                 * is laid out for long sequences: n_logical_blocks * 16 / max_seqs >= 6144) for single
-                                * calls, and inside the decode loop (pie_decode_step, pie_decode_layer), whose launches
-                                * overlap at their ends, up to 2048 while every CTA still gets a work item */
+                                * calls and for pie_decode_layer (whose caller puts its own kernels between the layers),
+                                * and inside pie_decode_step / pie_decode_step_host, whose launches overlap at their
+                                * ends, up to 2048 while every CTA still gets a work item */
     int32_t swap_ctas;         /* CTAs of the swap kernel; 0 = default (16) */
     int32_t attn_ctas_per_sm;  /* 0 = as many as fit */
     int32_t timing;            /* 1: per-layer timing for pie_controller_tick / pie_get_stats (the attention kernel notes

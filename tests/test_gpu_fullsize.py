@@ -240,6 +240,27 @@ def test_llama3_70b_shape_longest_sequences_in_512_token_chunks():
     free(dw)
 
 
+def test_the_host_stays_one_decode_step_ahead_of_the_gpu():
+    """pie_decode_step returns once the step is enqueued, but it does not start enqueueing step s before step s - 2 has
+    finished on the GPU: with a workload the GPU paces, every step but the newest two has been evaluated by the time the
+    call returns (the library's ring of timing sets alone would let the host get four steps ahead)."""
+    lens = np.full(32, 8192, dtype=np.int32)
+    wl = synth.Workload("pace", 7, 8, 8, 8, 128, synth.F16, lens, 24, 0.0)
+    nb = int(((lens.astype(np.int64) + 24 + 15) // 16).sum())
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=1, extra_gpu_slots=3 * nb, extra_host_slots=5 * nb)
+    pie.pie_set_extension_ratio(dw.pool, 0.0)
+    behind = []
+    for s in range(1, 17):
+        dw.advance_context()
+        dw.decode_step()
+        pie.pie_controller_tick(dw.pool)
+        behind.append(s - pie.pie_get_stats(dw.pool)["steps_measured"])
+    dw.sync()
+    assert max(behind[2:]) <= 2, behind
+    assert max(behind) >= 1, behind            # ... and it does run ahead: the call does not wait for its own step
+    dw.close()
+
+
 def test_step_timing_from_gpu_timer_stamps_and_timeline():
     """The per-step statistics come from time stamps the attention kernel writes itself (no timing events on the
     compute stream): they must agree with CUDA events around the same step, report no stall while nothing is swapped
