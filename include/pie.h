@@ -291,6 +291,11 @@ int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
  * slots the GPU pool can spare, at most 8 and at most a quarter of the layers.  0 <= layers <= 8 (PIE_ERR_INVALID
  * otherwise); an explicit value is capped at half the layers. */
 int pie_set_lookahead(pie_pool *pool, int32_t layers);
+/* How many decode steps the host may be ahead of the GPU when pie_step_begin returns: 1 (the default) to 3.  With 1
+ * the host enqueues a step while the one before it runs; a larger value lets a caller with a slow or bursty control
+ * thread queue more work, at the price described at pie_step_begin (swap lists break into short copies once the slots
+ * they are given are still in flight).  PIE_ERR_INVALID outside 1..3. */
+int pie_set_run_ahead(pie_pool *pool, int32_t steps);
 
 /* ---- 8-bit blocks (a variant beyond the paper, whose blocks are 16-bit: a token costs half the bytes in HBM, in the
  * host pool and on the link, so the same link hides twice the tokens per layer - Section 3.1's condition in bytes) ----

@@ -36,7 +36,7 @@ EXPORTS = [
     "pie_decode_attention_noalloc", "pie_set_layer_policy", "pie_set_violation_trigger", "pie_get_layer_log",
     "pie_resize_begin", "pie_resize_status", "pie_table_init_capacity", "pie_table_resize_begin", "pie_table_layer_pass",
     "pie_table_capacity", "pie_table_swap_ex", "pie_table_set_retention", "pie_table_kept_copies", "pie_table_mark_dirty", "pie_table_drop_host_copy", "pie_set_retention",
-    "pie_declare_append_blocks", "pie_kv_write", "pie_prefill_attention", "pie_decode_layer", "pie_set_lookahead", "pie_set_kv_scales",
+    "pie_declare_append_blocks", "pie_kv_write", "pie_prefill_attention", "pie_decode_layer", "pie_set_lookahead", "pie_set_run_ahead", "pie_set_kv_scales",
     "pie_governor_create", "pie_governor_destroy", "pie_governor_report", "pie_governor_state", "pie_report_throughput",
 ]
 
@@ -127,6 +127,7 @@ _sig = {
     "pie_table_drop_host_copy": (_i32, [_vp, _i32, _i32]),
     "pie_set_retention": (_i32, [_vp, _i32]),
     "pie_set_lookahead": (_i32, [_vp, _i32]),
+    "pie_set_run_ahead": (_i32, [_vp, _i32]),
     "pie_set_kv_scales": (_i32, [_vp, ctypes.c_float, ctypes.c_float]),
     "pie_governor_create": (_vp, [_f64, _f64, _i32, _i32]),
     "pie_governor_destroy": (None, [_vp]),
@@ -227,6 +228,10 @@ def pie_set_violation_trigger(pool, share) -> None:
 
 def pie_set_lookahead(pool, layers) -> None:
     check(lib.pie_set_lookahead(pool, layers), "pie_set_lookahead")
+
+
+def pie_set_run_ahead(pool, steps) -> None:
+    check(lib.pie_set_run_ahead(pool, steps), "pie_set_run_ahead")
 
 
 def pie_set_kv_scales(pool, k_scale, v_scale) -> None:

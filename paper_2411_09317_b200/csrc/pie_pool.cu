@@ -173,6 +173,7 @@ struct pie_pool {
     cudaEvent_t step_end_ev[TIMING_RING] = {};  // recorded there once a step's last attention kernel has completed
     int64_t step_end_of[TIMING_RING] = {};      // ... the step each of them stands for (0 = none)
     int64_t step_end_ticket = 0;                // the compute ticket the newest of them waits for
+    int32_t run_ahead = 1;                      // steps the host may be ahead of the GPU (pie_set_run_ahead)
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
     double free_contrast = -1.0;     // on swap-free steps: the contrast of the layers' four-layer mean times (see evaluate_step_set)
@@ -1807,8 +1808,8 @@ int pie_step_begin(pie_pool *pool) {
         if (st != PIE_OK) return st;
     }
     ++pool->step;
-    if (pool->step >= 3) {   // one step ahead of the GPU at most (mark_step_end)
-        const int64_t old = pool->step - 2;
+    if (pool->step >= 2 + pool->run_ahead) {   // run_ahead steps (one, by default) ahead of the GPU at most (mark_step_end)
+        const int64_t old = pool->step - 1 - pool->run_ahead;
         const int k = (int)(old % TIMING_RING);
         if (pool->step_end_of[k] == old) PIE_CUDA(cudaEventSynchronize(pool->step_end_ev[k]));
     }
@@ -2022,6 +2023,12 @@ int pie_set_lookahead(pie_pool *pool, int32_t layers) {
     if (st != PIE_OK) return st;
     pool->group_setting = layers;
     pool->lookahead = std::max(1, layers);
+    return PIE_OK;
+}
+
+int pie_set_run_ahead(pie_pool *pool, int32_t steps) {
+    if (!pool || steps < 1 || steps > TIMING_RING - 1) return PIE_ERR_INVALID;
+    pool->run_ahead = steps;
     return PIE_OK;
 }
 

@@ -83,6 +83,7 @@ def main(argv=None):
     ap.add_argument("--swap-mode", default="auto", choices=["auto", "kernel", "copy_engine", "bulk_kernel"],
                     help="how swap lists are moved (PIE_MODE_*)")
     ap.add_argument("--lookahead", type=int, default=0, help="layers per prefetch group (pie_set_lookahead; 0: the library chooses)")
+    ap.add_argument("--run-ahead", type=int, default=1, help="decode steps the host may be ahead of the GPU (pie_set_run_ahead)")
     ap.add_argument("--split", type=int, default=0, help="split-K chunk in tokens (0: the library's default)")
     ap.add_argument("--attn-variant", type=int, default=0, help="attention kernel variant (tuning)")
     ap.add_argument("--kv-fp8", action="store_true", help="blocks of E4M3 bytes (half the bytes per token; head_dim 128)")
@@ -131,6 +132,7 @@ def main(argv=None):
                             split_tokens=args.split, attn_variant=args.attn_variant)
         dw.set_retention(args.kept_copies)
         pie.pie_set_lookahead(dw.pool, args.lookahead)
+        pie.pie_set_run_ahead(dw.pool, args.run_ahead)
         emit({"workload": args.workload, "layers": L, "seqs": wl.n_seqs, "blocks_per_layer": nb, "block_bytes": wl.block_bytes,
               "kv_gb": L * nb * wl.block_bytes / 1e9, "kept_copies": args.kept_copies, "other_mb_per_layer": args.other_mb,
               "lookahead": args.lookahead,
@@ -246,6 +248,7 @@ def expansion_throughput(args, wl, link, emit):
                             initial_host_blocks=h if r > 0 else 0)
         dw.set_retention(args.kept_copies)
         pie.pie_set_lookahead(dw.pool, args.lookahead)
+        pie.pie_set_run_ahead(dw.pool, args.run_ahead)
         pie.pie_set_extension_ratio(dw.pool, r)
         run_steps(dw, 2)
         per, sb, sa, ctx0, _ = run_steps(dw, args.steps)
