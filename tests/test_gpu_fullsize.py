@@ -127,10 +127,12 @@ def test_llama2_7b_full_size_kept_host_copies_layer_by_layer_matches_resident_ru
     assert stats["bytes_out"] <= (wl.n_layers * n_host + (steps - 1) * wl.n_layers * wl.n_seqs) * wl.block_bytes
     swapped = dw.out_all.cpu().numpy().copy()
     free(dw)
+    # (through the same entry point: the order in which a sequence's chunks are merged is the split-K chunk's, and the
+    # per-layer entry point keeps the pool's chunk where pie_decode_step takes longer work items)
     dw2 = DeviceWorkload(wl, host_frac=0.0, timing=False)
     for _ in range(steps):
         dw2.advance_context()
-        dw2.decode_step()
+        dw2.decode_step(between_layers=lambda l: None)
     dw2.sync()
     assert np.array_equal(swapped, dw2.out_all.cpu().numpy())
     free(dw2)
@@ -245,8 +247,8 @@ def test_the_host_stays_one_decode_step_ahead_of_the_gpu():
     finished on the GPU: with a workload the GPU paces, every step but the newest two has been evaluated by the time the
     call returns (the library's ring of timing sets alone would let the host get four steps ahead)."""
     lens = np.full(32, 8192, dtype=np.int32)
-    wl = synth.Workload("pace", 7, 8, 8, 8, 128, synth.F16, lens, 24, 0.0)
-    nb = int(((lens.astype(np.int64) + 24 + 15) // 16).sum())
+    wl = synth.Workload("pace", 7, 8, 8, 8, 128, synth.F16, lens, 40, 0.0)
+    nb = int(((lens.astype(np.int64) + 40 + 15) // 16).sum())
     dw = DeviceWorkload(wl, host_frac=0.0, timing=1, extra_gpu_slots=3 * nb, extra_host_slots=5 * nb)
     pie.pie_set_extension_ratio(dw.pool, 0.0)
     behind = []
@@ -258,6 +260,21 @@ def test_the_host_stays_one_decode_step_ahead_of_the_gpu():
     dw.sync()
     assert max(behind[2:]) <= 2, behind
     assert max(behind) >= 1, behind            # ... and it does run ahead: the call does not wait for its own step
+    # the limit is a setting (1 to 3 steps)
+    for bad in (0, 4, -1):
+        with pytest.raises(pie.PieError):
+            pie.pie_set_run_ahead(dw.pool, bad)
+    pie.pie_set_run_ahead(dw.pool, 3)
+    pie.pie_controller_tick(dw.pool)
+    base = pie.pie_get_stats(dw.pool)["steps_measured"]
+    behind = []
+    for s in range(1, 17):
+        dw.advance_context()
+        dw.decode_step()
+        pie.pie_controller_tick(dw.pool)
+        behind.append(s - (pie.pie_get_stats(dw.pool)["steps_measured"] - base))
+    dw.sync()
+    assert 3 <= max(behind) <= 4, behind
     dw.close()
 
 
