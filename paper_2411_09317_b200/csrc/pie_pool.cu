@@ -1801,6 +1801,7 @@ static int evaluate_completed(pie_pool *pool, int32_t *changed) {
 
 int pie_step_begin(pie_pool *pool) {
     if (!pool) return PIE_ERR_INVALID;
+    if (pool->sticky != PIE_OK) return pool->sticky;   // (a launch that failed stores no ticket: nothing may wait for one)
     {
         int st = finish_group(pool);       // a caller that went layer by layer may have left a group open
         if (st == PIE_OK) st = close_step_set(pool);
