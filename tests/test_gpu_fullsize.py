@@ -242,6 +242,44 @@ def test_llama3_70b_shape_longest_sequences_in_512_token_chunks():
     free(dw)
 
 
+def test_adaptive_controller_settles_on_the_benchmark_shape_and_its_lists_stay_whole():
+    """The controller on the benchmark workload, from everything on the GPU: it climbs to a ratio near the link's share of a
+    layer and stays there (consecutive launches overlap, so single layers' end stamps alternate by a few per cent: the
+    slow-down estimate must not read that as interference and walk back to zero), and after the ramp - lists that grew by
+    a few blocks every four steps - a step's lists still go in a handful of copies."""
+    wl = synth.workload("llama2_7b")
+    steps = 150
+    wl = dataclasses.replace(wl, decode_steps=steps + 8)
+    _, _, nb = wl.tables()
+    share = int(0.0125 * nb) + 1
+    L = wl.n_layers
+    dw = DeviceWorkload(wl, host_frac=0.0, timing=True, extra_gpu_slots=(2 * L + 8) * share + 64,
+                        extra_host_slots=(3 * L + 8) * share + 64)
+    pie.pie_set_extension_ratio(dw.pool, 0.0)
+    for _ in range(6):
+        dw.advance_context()
+        dw.decode_step()
+    pie.pie_set_controller(dw.pool, 1.0 / 4096.0, 0.0, 0.0)
+    pie.pie_set_extension_ratio(dw.pool, -1.0)
+    ratios, copies = [], []
+    before = pie.pie_get_stats(dw.pool)["copy_engine_copies"]
+    for _ in range(steps - 6):
+        dw.advance_context()
+        dw.decode_step()
+        st = pie.pie_get_stats(dw.pool)
+        ratios.append(st["ratio"])
+        copies.append(st["copy_engine_copies"] - before)
+        before = st["copy_engine_copies"]
+    dw.sync()
+    tail = ratios[-40:]
+    assert min(tail) >= 0.002, (max(ratios), tail)                 # it holds what it reached
+    assert max(tail) - min(tail) <= 4.0 / 4096.0 + 1e-9, tail       # ... within a few steps of the rule
+    # 2 L lists per step; in steady steps a group's eight lists go in one copy per direction
+    assert np.median(copies[-40:]) <= L, copies[-40:]
+    check_samples(dw, spread_samples(wl, L, 4, seed=5), steps)
+    free(dw)
+
+
 def test_the_host_stays_one_decode_step_ahead_of_the_gpu():
     """pie_decode_step returns once the step is enqueued, but it does not start enqueueing step s before step s - 2 has
     finished on the GPU: with a workload the GPU paces, every step but the newest two has been evaluated by the time the
