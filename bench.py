@@ -268,6 +268,7 @@ class Runner:
                 "swap_out_gbs": (after["bytes_out"] - before["bytes_out"]) / sec / 1e9,
                 "elided_gbs": (after["bytes_out_elided"] - before["bytes_out_elided"]) / sec / 1e9,
                 "wait_share": after["last_step_stall_ms"] / max(after["last_step_ms"], 1e-9),
+                "copies_per_step": (after["copy_engine_copies"] - before["copy_engine_copies"]) / n,
                 "kernel_ms_per_layer": float(np.mean([c["last_step_compute_ms"] for c in comp if c["steps_measured"] > 0] or [np.nan])) / dw.wl.n_layers,
                 # per step one attention kernel per layer (each merges the layer before it in its tail) and one combine
                 # kernel behind the last layer, plus whatever swap and table kernels the lists needed
@@ -297,7 +298,7 @@ def sweep(rn, pie, ratios, n, reps, warm, link_gbs):
         e = {"ratio": r, "slowdown_mean": float(np.mean(sl)), "slowdown_min": float(min(sl)), "slowdown_max": float(max(sl)),
              "swap_in_gbs": float(np.mean([x["swap_in_gbs"] for x in runs])), "swap_out_gbs": float(np.mean([x["swap_out_gbs"] for x in runs])),
              "ms_per_step": float(np.mean([x["ms_per_step"] for x in runs])), "wait_share": float(np.mean([x["wait_share"] for x in runs])),
-             "steps_per_run": n, "runs": reps}
+             "copies_per_step": float(np.mean([x["copies_per_step"] for x in runs])), "steps_per_run": n, "runs": reps}
         e["frac_of_link"] = e["swap_in_gbs"] / max(link_gbs, 1e-9)
         if e["slowdown_max"] <= 0.02 and (best is None or e["swap_in_gbs"] > best["swap_in_gbs"]):
             best = e
@@ -430,7 +431,7 @@ def main():
         res_c = rn.run(args.steps, args.ramp)
         controller = {"ratio": c["after"]["ratio"], "swap_in_gbs": c["swap_in_gbs"], "swap_out_gbs": c["swap_out_gbs"],
                       "frac_of_link": c["swap_in_gbs"] / max(link["both"], 1e-9), "slowdown": c["ms"] / res_c["ms"] - 1.0,
-                      "wait_share": c["wait_share"], "ramp_steps": 2 * args.ramp + 2,
+                      "wait_share": c["wait_share"], "copies_per_step": c["copies_per_step"], "ramp_steps": 2 * args.ramp + 2,
                       "note": "adaptive mode (pie_set_extension_ratio < 0), step 1/4096; slow-down against a resident run at the same contexts"}
 
     def release(d):
