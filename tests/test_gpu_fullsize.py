@@ -272,8 +272,8 @@ def test_adaptive_controller_settles_on_the_benchmark_shape_and_its_lists_stay_w
         before = st["copy_engine_copies"]
     dw.sync()
     tail = ratios[-40:]
-    assert min(tail) >= 0.002, (max(ratios), tail)                 # it holds what it reached
-    assert max(tail) - min(tail) <= 4.0 / 4096.0 + 1e-9, tail       # ... within a few steps of the rule
+    assert min(tail) >= 0.0015, (max(ratios), tail)                # it holds what it reached (0.004-0.005 on a quiet link)
+    assert max(tail) - min(tail) <= 8.0 / 4096.0 + 1e-9, tail       # ... within a few steps of the rule
     # 2 L lists per step; in steady steps a group's eight lists go in one copy per direction
     assert np.median(copies[-40:]) <= L, copies[-40:]
     check_samples(dw, spread_samples(wl, L, 4, seed=5), steps)
