@@ -214,8 +214,9 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
  * the layers' kernels is enqueued on the compute stream: a layer's kernel waits for its arriving units itself (a device
  * word the copy-in stream sets behind each list), the copy streams wait for the kernels by value, and from the second
  * layer on each attention kernel is launched as a programmatic dependent of the one before it (the layers' q / k_new /
- * v_new must therefore all be ready when the call is made - they are: the arrays hold every layer).  With timing enabled
- * the host runs at most 4 steps ahead.  A share the GPU pool has no room for when its group is prefetched is fetched at its
+ * v_new must therefore all be ready when the call is made - they are: the arrays hold every layer).  The call returns once
+ * the step is enqueued; it does not start before the GPU has finished the step before the previous one (pie_step_begin,
+ * pie_set_run_ahead).  A share the GPU pool has no room for when its group is prefetched is fetched at its
  * layer's turn; if there is no room even then the call returns PIE_ERR_NOMEM with the layers before it enqueued and nothing
  * of that layer.  q_all/out_all: device [n_layers][n_seqs][Hq][D]; k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D]
  * or NULL.  Runs pie_controller_tick at the end. */
