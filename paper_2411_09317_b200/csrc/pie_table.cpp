@@ -16,40 +16,48 @@ SlotPool::SlotPool(int64_t n) {
     n_ready_ = n;
 }
 
-void SlotPool::add_ready(int32_t slot) {
-    auto next = runs_.lower_bound(slot);
-    bool joined = false;
+void SlotPool::add_ready_run(int32_t start, int32_t len) {
+    // one map operation per run of consecutive slots: joined to the run before it and / or the run after it
+    auto next = runs_.lower_bound(start);
+    int32_t s = start, l = len;
     if (next != runs_.begin()) {
         auto prev = std::prev(next);
-        if (prev->first + prev->second == slot) {  // extends the run before it
-            prev->second += 1;
-            joined = true;
-            if (next != runs_.end() && next->first == slot + 1) {  // ... and closes the gap to the run after it
-                prev->second += next->second;
-                runs_.erase(next);
-            }
+        if (prev->first + prev->second == start) {  // extends the run before it
+            s = prev->first;
+            l += prev->second;
+            runs_.erase(prev);
         }
     }
-    if (!joined) {
-        if (next != runs_.end() && next->first == slot + 1) {  // extends the run after it downwards
-            const int32_t len = next->second + 1;
-            runs_.erase(next);
-            runs_[slot] = len;
-        } else {
-            runs_[slot] = 1;
-        }
+    if (next != runs_.end() && next->first == start + len) {  // closes the gap to the run after it
+        l += next->second;
+        runs_.erase(next);
     }
-    ++n_ready_;
+    runs_[s] = l;
+    n_ready_ += len;
 }
+
+void SlotPool::add_ready(int32_t slot) { add_ready_run(slot, 1); }
 
 void SlotPool::settle(const int64_t *done) {
     if (pending_.empty()) return;
+    // swap lists release their slots in runs: confirmed neighbours in the queue that are neighbours in the pool go in as one
     size_t keep = 0;
+    int32_t run_start = 0, run_len = 0;
     for (size_t i = 0; i < pending_.size(); ++i) {
         const Pending p = pending_[i];
-        if (p.ticket <= done[p.queue]) add_ready(p.slot);
-        else pending_[keep++] = p;
+        if (p.ticket <= done[p.queue]) {
+            if (run_len > 0 && p.slot == run_start + run_len) {
+                ++run_len;
+            } else {
+                if (run_len > 0) add_ready_run(run_start, run_len);
+                run_start = p.slot;
+                run_len = 1;
+            }
+        } else {
+            pending_[keep++] = p;
+        }
     }
+    if (run_len > 0) add_ready_run(run_start, run_len);
     pending_.resize(keep);
 }
 

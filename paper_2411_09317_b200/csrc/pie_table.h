@@ -50,6 +50,7 @@ class SlotPool {
         int64_t ticket;
     };
     void add_ready(int32_t slot);
+    void add_ready_run(int32_t start, int32_t len);
     std::map<int32_t, int32_t> runs_;  // start -> length of a run of ready slots
     int64_t n_ready_ = 0;
     int32_t cursor_ = 0;  // behind the slots that the last request of two or more took from ready
