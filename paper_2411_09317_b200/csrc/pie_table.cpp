@@ -61,9 +61,9 @@ void SlotPool::settle(const int64_t *done) {
     pending_.resize(keep);
 }
 
-void SlotPool::take_n(int64_t n, int32_t *slots, SlotTag *tags) {
+void SlotPool::take_n(int64_t n, int32_t *slots, SlotTag *tags, bool lists) {
     int64_t k = 0;
-    const bool rove = n >= 2;
+    const bool rove = lists && n >= 2;
     while (k < n && !runs_.empty()) {
         const int64_t want = n - k;
         auto pick = runs_.end();
@@ -217,8 +217,9 @@ int Table::alloc_bulk(const int32_t *blocks, int64_t n, const uint8_t *on_host) 
         take_tags_.resize((size_t)want_gpu);
         host_slots.resize((size_t)(n - want_gpu));
         host_tags.resize((size_t)(n - want_gpu));
-        if (want_gpu > 0) gpu_.take_n(want_gpu, take_slots_.data(), take_tags_.data());
-        if (n - want_gpu > 0) host_.take_n(n - want_gpu, host_slots.data(), host_tags.data());
+        // (allocations live long: they fill the lowest runs that fit and leave the swap lists' cursor alone)
+        if (want_gpu > 0) gpu_.take_n(want_gpu, take_slots_.data(), take_tags_.data(), false);
+        if (n - want_gpu > 0) host_.take_n(n - want_gpu, host_slots.data(), host_tags.data(), false);
         int64_t ig = 0, ih = 0;
         for (int64_t i = 0; i < n; ++i) {
             Unit &u = unit(l, blocks[i]);

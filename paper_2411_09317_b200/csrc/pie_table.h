@@ -27,15 +27,17 @@ struct SlotTag {
 // pool's spare part like a ring: lists land in consecutive slots, and consecutive lists beside each other, whatever
 // their sizes were before - which is what lets a few large copies move them.  (Taking the lowest run that fits, the
 // rule before this one, serves a steady ratio as well but splinters the spare part once the lists grow and shrink by a
-// few blocks at a time: after a ramp of the adaptive controller a list of 20 blocks came in three runs.)  Single slots -
-// allocations, which live long - fill the lowest holes and stay out of the ring's way.
+// few blocks at a time: after a ramp of the adaptive controller a list of 20 blocks came in three runs.)  Allocations,
+// which live long - single slots, and the pool's layer-by-layer requests for several blocks at once - fill the lowest
+// runs that fit and stay out of the ring's way.
 class SlotPool {
   public:
     explicit SlotPool(int64_t n);
     void settle(const int64_t *done);
     int64_t available() const { return n_ready_ + (int64_t)pending_.size(); }
     // n slots into slots[0..n), their tags into tags[0..n); the caller has checked available() >= n
-    void take_n(int64_t n, int32_t *slots, SlotTag *tags);
+    // lists = false: an allocation (long-lived): the cursor is neither used nor moved
+    void take_n(int64_t n, int32_t *slots, SlotTag *tags, bool lists = true);
     int32_t take(SlotTag *tag) {
         int32_t s;
         take_n(1, &s, tag);
