@@ -69,6 +69,9 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
+    def count(self):
+        return len(self.lines) if self.proc is not None else 1 << 30
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -309,7 +312,7 @@ def sweep(rn, pie, ratios, n, reps, warm, link_gbs):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="llama2_7b", choices=sorted(SWEEP_RATIOS))
@@ -357,8 +360,8 @@ def main():
     r_cap = 1.25 * max(sweep_ratios + kept_ratios) + 0.001
     # the GPU pool holds the fully resident batch plus, for ratios up to r_cap, two steps' worth of host-resident shares:
     # three groups of up to eight layers are in transit at any time (arriving, in use, leaving), and the host enqueues up
-    # to a step ahead, so with this much to spare a swap list's slots come from the part of the pool that is free for
-    # certain, in one run; the host pool holds the host-resident shares of all layers and as much again in transit
+    # to two steps ahead, so with this much to spare at the ratios that matter (r_cap is twice those) a swap list's slots
+    # come from the part of the pool that is free for certain, in one run; the host pool holds the host-resident shares of all layers and as much again in transit
     share = int(r_cap * n_blocks) + 1
     spare_lists = max(26, 2 * L + 8)
     dw = DeviceWorkload(wl, host_frac=0.0, timing=True, split_tokens=args.split, swap_ctas=args.swap_ctas,
@@ -378,20 +381,30 @@ def main():
 
     # ---- phase 2: the headline region at the ratio found, between two resident regions (A/B/A) -----------------------
     head_ratio = best["ratio"] if best else min(sweep_ratios)
+    # Clocks are sampled under this load, and the three regions (resident, headline, resident) all run with the sampler
+    # going: the same steps run untimed while nvidia-smi comes up (its start holds the driver for tens of milliseconds:
+    # inside a timed region of 20 short steps that once read as a 35 % slow-down), and again behind the last region until
+    # three more samples have been taken.
     pie.pie_set_extension_ratio(dw.pool, 0.0)
+    sampler = ClockSampler(local)
+    sampler.start()
+    t_wait = time.perf_counter()
+    while sampler.count() < 1 and time.perf_counter() - t_wait < 3.0:
+        rn.run(4, 0)
+    n_before = sampler.count()
     res_a = rn.run(args.steps, args.warmup)
     pie.pie_set_extension_ratio(dw.pool, head_ratio)
     rn.run(8, 4)                                   # the host-resident sets settle at the new ratio
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.4)                                # nvidia-smi takes a moment to come up
     barrier()
     head = rn.run(args.steps, args.warmup)
     barrier()
-    clocks = sampler.stop()
     ms_run = max_over_ranks(head["ms"])
     pie.pie_set_extension_ratio(dw.pool, 0.0)
     res_b = rn.run(args.steps, args.warmup)
+    t_wait = time.perf_counter()
+    while sampler.count() < n_before + 3 and time.perf_counter() - t_wait < 2.0:
+        rn.run(4, 0)
+    clocks = sampler.stop()
     step_bytes = rn.bytes_of_steps(args.steps, args.warmup)
     value_1gpu = step_bytes / (ms_run * 1e-3) / 1e9
     resident_gbs = step_bytes / (0.5 * (res_a["ms"] + res_b["ms"]) * 1e-3) / 1e9

@@ -215,8 +215,7 @@ int pie_decode_attention(pie_pool *pool, int32_t layer, const void *q, void *out
  * word the copy-in stream sets behind each list), the copy streams wait for the kernels by value, and from the second
  * layer on each attention kernel is launched as a programmatic dependent of the one before it (the layers' q / k_new /
  * v_new must therefore all be ready when the call is made - they are: the arrays hold every layer).  The call returns once
- * the step is enqueued; it does not start before the GPU has finished the step before the previous one (pie_step_begin,
- * pie_set_run_ahead).  A share the GPU pool has no room for when its group is prefetched is fetched at its
+ * the step is enqueued; it does not start while the GPU is more than two steps behind (pie_step_begin, pie_set_run_ahead).  A share the GPU pool has no room for when its group is prefetched is fetched at its
  * layer's turn; if there is no room even then the call returns PIE_ERR_NOMEM with the layers before it enqueued and nothing
  * of that layer.  q_all/out_all: device [n_layers][n_seqs][Hq][D]; k_new_all/v_new_all: device [n_layers][n_seqs][Hkv][D]
  * or NULL.  Runs pie_controller_tick at the end. */
@@ -262,10 +261,10 @@ int pie_set_violation_trigger(pie_pool *pool, double share);
  * started or -1, layer whose swap-in started or -1}.  log may be NULL to ask for the count only. */
 int pie_get_layer_log(pie_pool *pool, int32_t *log, int64_t capacity, int64_t *n_entries);
 /* Marks a step boundary (pie_decode_step calls it itself): the per-step timing sets turn over, and the host thread waits
- * here until the GPU has finished the step before the previous one - the host enqueues one step while the one before it
- * runs, and no further.  (Slots freed by a step's swap lists are only known free once their copies have completed; a host
- * several steps ahead would be handed slots still in flight, in the order they were released, and its lists would break
- * into many short copies.) */
+ * here until the GPU has finished the step three before the one that begins - the host enqueues up to two steps beyond
+ * the one the GPU is working on, and no further (pie_set_run_ahead).  (Slots freed by a step's swap lists are only known
+ * free once their copies have completed; a host many steps ahead would be handed slots still in flight, in the order they
+ * were released, and its lists would break into many short copies.) */
 int pie_step_begin(pie_pool *pool);
 
 /* ---- policy and controller (Section 3.3, Section 3.4.2) ------------------------------------------ */
@@ -292,10 +291,12 @@ int pie_set_controller(pie_pool *pool, double step, double eps, double u_hi);
  * slots the GPU pool can spare, at most 8 and at most a quarter of the layers.  0 <= layers <= 8 (PIE_ERR_INVALID
  * otherwise); an explicit value is capped at half the layers. */
 int pie_set_lookahead(pie_pool *pool, int32_t layers);
-/* How many decode steps the host may be ahead of the GPU when pie_step_begin returns: 1 (the default) to 3.  With 1
- * the host enqueues a step while the one before it runs; a larger value lets a caller with a slow or bursty control
- * thread queue more work, at the price described at pie_step_begin (swap lists break into short copies once the slots
- * they are given are still in flight).  PIE_ERR_INVALID outside 1..3. */
+/* How many decode steps the host may be ahead of the GPU when pie_step_begin returns: 1 to 3, 2 by default.  With 1
+ * the host enqueues a step while the one before it runs and the GPU pool needs the least spare room for whole swap lists
+ * (about two steps' host-resident shares), but any delay of the host thread longer than the rest of the running step
+ * leaves the GPU idle; each further step absorbs that much more delay and asks for one more step's shares of spare
+ * slots (without them swap lists break into short copies: the slots they are given are still in flight).
+ * PIE_ERR_INVALID outside 1..3. */
 int pie_set_run_ahead(pie_pool *pool, int32_t steps);
 
 /* ---- 8-bit blocks (a variant beyond the paper, whose blocks are 16-bit: a token costs half the bytes in HBM, in the

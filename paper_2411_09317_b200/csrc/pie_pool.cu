@@ -173,7 +173,7 @@ struct pie_pool {
     cudaEvent_t step_end_ev[TIMING_RING] = {};  // recorded there once a step's last attention kernel has completed
     int64_t step_end_of[TIMING_RING] = {};      // ... the step each of them stands for (0 = none)
     int64_t step_end_ticket = 0;                // the compute ticket the newest of them waits for
-    int32_t run_ahead = 1;                      // steps the host may be ahead of the GPU (pie_set_run_ahead)
+    int32_t run_ahead = 2;                      // steps the host may be ahead of the GPU (pie_set_run_ahead)
     int64_t step = 0;
     double base_ms_per_token = 0.0;  // attention time per context token measured on steps without swap traffic
     double free_contrast = -1.0;     // on swap-free steps: the contrast of the layers' four-layer mean times (see evaluate_step_set)
@@ -980,8 +980,8 @@ int attention_call(pie_pool *p, int32_t layer, const void *q, void *out, const i
     return st;
 }
 
-// The host enqueues one decode step while the step before it runs, and no further (pie_step_begin waits for the step
-// before that).  Slots released by a step's swap lists can only be handed out as free for certain once their copies are
+// The host enqueues at most two decode steps beyond the one the GPU is working on (pie_step_begin waits; one step of
+// slack beyond the minimum, so that a few milliseconds' delay of the host thread does not leave the GPU idle).  Slots released by a step's swap lists can only be handed out as free for certain once their copies are
 // known complete; a host that is several steps ahead finds nothing but slots still in flight, takes them in the order
 // they were released, mixed with what has just come back, and the lists break into several runs (measured on 17 long
 // sequences and 80 layers: 3 runs per list of 20 blocks, and the copy engines at 22 GB/s instead of 40).  The event is
@@ -1809,7 +1809,7 @@ int pie_step_begin(pie_pool *pool) {
         if (st != PIE_OK) return st;
     }
     ++pool->step;
-    if (pool->step >= 2 + pool->run_ahead) {   // run_ahead steps (one, by default) ahead of the GPU at most (mark_step_end)
+    if (pool->step >= 2 + pool->run_ahead) {   // run_ahead steps (two, by default) ahead of the GPU at most (mark_step_end)
         const int64_t old = pool->step - 1 - pool->run_ahead;
         const int k = (int)(old % TIMING_RING);
         if (pool->step_end_of[k] == old) PIE_CUDA(cudaEventSynchronize(pool->step_end_ev[k]));
